@@ -1,0 +1,213 @@
+/*
+ * libspecstream - streamed-KV verification attention for speculative decoding (C ABI).
+ *
+ * One verification round of one layer: the T_q candidate queries of every request
+ * (pending committed token + drafts), times the GQA group, attend to the request's
+ * committed KV history as it arrives chunk by chunk, plus the on-GPU candidate KV
+ * under a chain or tree mask.  Each chunk is read from HBM once and serves every
+ * query of the round; it yields per-row partial states (m, l, a) that are merged by
+ * online softmax, so the result equals full attention over [history ; candidates].
+ * A bit-exact commit-gather appends the accepted candidates' KV to the committed
+ * buffer.  (Paper Section 4.2: Eq. 12 defines the result, Eq. 13 the per-chunk
+ * state, Eq. 14 the merge, Eq. 17 the equivalence; Section 4.1 the commit rule.)
+ *
+ * Conventions
+ *  - All tensor pointers are DEVICE pointers unless a comment says HOST.  Element type
+ *    of Q/K/V/O is bf16 (16-bit words); LSE is fp32.
+ *  - ss_tensor strides are in ELEMENTS; the innermost (head-dim) axis is contiguous,
+ *    base pointers and all strides are multiples of 8 elements (16 bytes).
+ *  - Ownership: the caller owns every tensor and the workspace.  The library allocates
+ *    no device memory on these calls and keeps no caller pointer after finalize,
+ *    except Q between begin and finalize.
+ *  - Asynchrony: every call validates its arguments on the host, enqueues work on the
+ *    given CUDA stream and returns; results are valid once the stream reaches that
+ *    point.  All calls of one round must use the same stream.
+ *  - Call order per round: begin -> {chunk | local}* -> finalize.  Chunks may come in
+ *    any order and any number (including zero); local at most once.  Anything else
+ *    returns SS_ERR_STATE.
+ *  - Errors: host-detectable problems return a code and enqueue nothing.  Problems only
+ *    the device can see (valid_len outside [0, L_c], accept index outside [0, T_loc),
+ *    destination overflow, a bounded wait that expired) set a status word in the
+ *    workspace, skip the offending item, never trap; read it with ss_poll_status.
+ *  - Determinism: same inputs, same call sequence, same config -> bitwise-same output.
+ *  - A query row with no visible key yields O = 0 and LSE = -inf.
+ */
+#ifndef SPECSTREAM_H_
+#define SPECSTREAM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ss_ctx ss_ctx; /* opaque */
+
+typedef enum {
+  SS_OK = 0,
+  SS_ERR_ARG = 1,         /* null pointer, non-positive size */
+  SS_ERR_SHAPE = 2,       /* exceeds the limits given at ss_create, H_q % H_kv, d not in {64,128} */
+  SS_ERR_ALIGN = 3,       /* base or stride not a multiple of 16 bytes */
+  SS_ERR_STATE = 4,       /* call order violated */
+  SS_ERR_CAPACITY = 5,    /* workspace too small */
+  SS_ERR_UNSUPPORTED = 6, /* device is not sm_100 */
+  SS_ERR_CUDA = 7,        /* a CUDA runtime/driver call failed; see ss_last_cuda_error */
+  SS_ERR_DEVICE_FLAG = 8, /* the device status word is non-zero (see SS_DEV_*) */
+  SS_ERR_TIMEOUT = 9      /* a host wait ran past its deadline */
+} ss_status;
+
+/* bits of the device status word */
+#define SS_DEV_BAD_VALID_LEN 1u /* valid_len[b] outside [0, L_c]: clamped             */
+#define SS_DEV_BAD_ACCEPT 2u    /* accept_cnt/accept_idx out of range: row skipped     */
+#define SS_DEV_DST_OVERFLOW 4u  /* dst_off + k outside [0, cap): row skipped           */
+#define SS_DEV_WAIT_EXPIRED 8u  /* a bounded in-kernel wait gave up: round is invalid  */
+
+typedef struct {
+  int32_t max_B;      /* requests per call                                          */
+  int32_t H_q, H_kv;  /* query heads, kv heads (H_q % H_kv == 0)                     */
+  int32_t d;          /* head dim, 64 or 128                                         */
+  int32_t max_Tq;     /* candidate queries per request                               */
+  int32_t max_Tloc;   /* local candidate KV tokens per request (<= 1024)             */
+  int32_t max_Lc;     /* tokens per history chunk call                               */
+  int32_t max_chunks; /* chunk calls held as separate partial sets before the library
+                         folds them (any number of calls stays legal); 0 = default 64 */
+  int32_t device;     /* CUDA device ordinal                                         */
+  uint32_t flags;     /* SS_FLAG_*                                                   */
+} ss_config;
+
+/* Force the CUDA-core chunk kernel even where the tensor-core kernel applies. */
+#define SS_FLAG_FORCE_SIMT 1u
+/* Let successive chunk kernels of a round overlap on the GPU (programmatic dependent
+ * launch).  The caller promises that Q and the K/V of a chunk call are complete in
+ * memory before the PREVIOUS ss_ call of the round was enqueued on the stream, or were
+ * produced by a copy / an event the stream waited on - not by a kernel enqueued on the
+ * same stream between two ss_ calls. */
+#define SS_FLAG_OVERLAP_CHUNKS 2u
+
+typedef struct {
+  const void* ptr;                      /* device pointer, bf16                      */
+  int64_t stride_b, stride_h, stride_t; /* elements; innermost dim contiguous        */
+} ss_tensor;
+
+typedef enum { SS_MASK_CHAIN = 0, SS_MASK_TREE_BITS = 1 } ss_mask_kind;
+
+/* Bytes of device workspace a context with this config needs (0 on invalid config). */
+size_t ss_workspace_bytes(const ss_config* cfg);
+
+/* Create a context over a caller-allocated device workspace (256-byte aligned, at least
+ * ss_workspace_bytes).  Synchronous; clears the device status word on `stream` 0. */
+ss_status ss_create(ss_ctx** out, const ss_config* cfg, void* workspace, size_t workspace_bytes);
+ss_status ss_destroy(ss_ctx* ctx);
+
+/* a1. Start a round: bind Q [B, H_q, T_q, d] and reset every row's state to the
+ * identity (m, l, a) = (-inf, 0, 0) (Section 4.2, accumulator initialisation).
+ * `scale` multiplies the scores (1/sqrt(d) in the paper) and is applied in fp32. */
+ss_status ss_verify_begin(ss_ctx* ctx, ss_tensor Q, int32_t B, int32_t T_q, float scale,
+                          void* stream);
+
+/* a2+a3. One history chunk for the whole batch: K, V [B, H_kv, L_c, d]; valid_len
+ * (device, [B], may be NULL = all L_c) gives the number of leading valid tokens of each
+ * request's chunk; tokens past it are invisible and may hold anything, NaN included.
+ * Computes the chunk-local state of Eq. 13 for every query row (all T_q*H_q/H_kv rows of
+ * a kv-head share one pass over its K/V) and records it for the Eq. 14 merge.  History
+ * is visible to every query of the round.  An on-GPU Active Tail is passed the same way. */
+ss_status ss_verify_chunk(ss_ctx* ctx, ss_tensor K, ss_tensor V, int32_t L_c,
+                          const int32_t* valid_len, void* stream);
+
+/* a4. The on-GPU candidate segment: K_loc, V_loc [B, H_kv, T_loc, d].  Query i of request
+ * b sees local token j iff
+ *   SS_MASK_CHAIN:     j <= i + (T_loc - T_q)   (causal, inclusive; mask_bits ignored)
+ *   SS_MASK_TREE_BITS: bit j of mask_bits[b][i][j/64] is set (device uint64
+ *                      [B, T_q, ceil(T_loc/64)]; row i = ancestors of node i and i itself). */
+ss_status ss_verify_local(ss_ctx* ctx, ss_tensor K_loc, ss_tensor V_loc, int32_t T_loc,
+                          ss_mask_kind kind, const uint64_t* mask_bits, void* stream);
+
+/* a5. Merge all partial states (Eq. 14), O = a / l as bf16 (round to nearest even) into
+ * O [B, H_q, T_q, d] (contiguous), LSE = m + ln l (natural log, of the scaled masked
+ * scores) into LSE [B, H_q, T_q] fp32 (may be NULL).  Ends the round. */
+ss_status ss_verify_finalize(ss_ctx* ctx, void* O, float* LSE, void* stream);
+
+/* a6. Commit-gather (Section 4.1: accepted candidates join the committed prefix).  For each
+ * request b and k < accept_cnt[b]: row accept_idx[b][k] of K_loc/V_loc (all kv heads) is
+ * copied, bit for bit, to row dst_off[b] + k of K_dst/V_dst [B, H_kv, cap, d].  Nothing else
+ * is written.  accept_idx is [B, T_loc] int32, accept_cnt and dst_off are [B] int32, all on
+ * the device.  Independent of the round state; may be called at any time. */
+ss_status ss_commit_gather(ss_ctx* ctx, ss_tensor K_loc, ss_tensor V_loc, int32_t B,
+                           int32_t T_loc, const int32_t* accept_idx, const int32_t* accept_cnt,
+                           ss_tensor K_dst, ss_tensor V_dst, int32_t cap, const int32_t* dst_off,
+                           void* stream);
+
+/* Read (and clear) the device status word after synchronising `stream`, waiting at most
+ * timeout_ms (<= 0: wait without limit).  SS_OK, SS_ERR_DEVICE_FLAG (bits in *dev_bits if
+ * non-NULL) or SS_ERR_TIMEOUT. */
+ss_status ss_poll_status(ss_ctx* ctx, void* stream, int32_t timeout_ms, uint32_t* dev_bits);
+
+/* a7. Streamed round (Section 4.2, pipelined KV transfers): the committed history lives in
+ * pinned HOST memory and crosses the host link once per round through two device staging
+ * buffers; copies run on a copy stream while the attention stream works on the other buffer.
+ *
+ * Host layout of request b: for chunk j = 0..ceil(hist_len[b]/L_c)-1 a block of
+ * [2 (K,V)][H_kv][L_c][d] bf16 at hist[b] + j * 2*H_kv*L_c*d elements (last block partial:
+ * only the first valid tokens of each head row are read).
+ * Device staging: stage_k[s], stage_v[s], s = 0,1, each [B, H_kv, batch_chunks*L_c, d]
+ * contiguous; one fill carries batch_chunks adjacent chunks (a transfer batch) and is
+ * consumed by one chunk-attention call.  Requests sorted by decreasing length keep the
+ * active requests of late fills a prefix of the batch, but any order is correct.
+ * After the attention the accepted rows are gathered into commit_k/commit_v
+ * [B, H_kv, T_q, d] (device) at row 0 and the buffers copied to host_commit_k/v (pinned
+ * HOST, same shape).  O_host / LSE_host (pinned HOST, may be NULL) receive the outputs.
+ * Synchronous: returns when the round is complete. */
+typedef struct {
+  int32_t B, T_q, L_c;
+  float scale;
+  const void* const* hist;   /* HOST array [B] of pinned HOST pointers                    */
+  const int32_t* hist_len;   /* HOST [B]                                                  */
+  int32_t batch_chunks;      /* adjacent chunk indices per staging-buffer fill (>= 1)     */
+  void* stage_k[2];          /* device, each [B, H_kv, batch_chunks * L_c, d]             */
+  void* stage_v[2];
+  int32_t scratch_fills;     /* capacity of the two scratch arrays, in fills              */
+  int32_t* valid_len_host;   /* pinned HOST scratch [scratch_fills * B]                   */
+  int32_t* valid_len_dev;    /* device scratch      [scratch_fills * B]                   */
+  ss_tensor Q, K_loc, V_loc; /* device; T_loc = T_q                                       */
+  ss_mask_kind mask_kind;
+  const uint64_t* mask_bits; /* device                                                    */
+  void* O;                   /* device [B,H_q,T_q,d] bf16                                 */
+  float* LSE;                /* device [B,H_q,T_q]                                        */
+  const int32_t* accept_idx; /* device [B,T_q]; NULL skips the commit step                */
+  const int32_t* accept_cnt; /* device [B]                                                */
+  const int32_t* zero_off;   /* device [B] of zeros (destination offsets)                 */
+  void* commit_k;            /* device [B,H_kv,T_q,d]                                     */
+  void* commit_v;
+  void* host_commit_k;       /* pinned HOST, same shape; receives the whole buffer        */
+  void* host_commit_v;
+  void* O_host;              /* pinned HOST or NULL                                       */
+  float* LSE_host;           /* pinned HOST or NULL                                       */
+  int32_t copy_only;         /* 1: issue the same copies but no attention (control run)   */
+} ss_stream_desc;
+
+typedef struct {
+  double ms_total;      /* host wall time of the round                                    */
+  float ms_device;      /* first copy enqueued -> last D2H done, CUDA events              */
+  int64_t h2d_bytes;    /* valid K/V bytes moved host -> device                           */
+  int64_t d2h_bytes;
+  int32_t chunk_calls;
+  int32_t copies;
+} ss_stream_stats;
+
+ss_status ss_stream_round(ss_ctx* ctx, const ss_stream_desc* desc, ss_stream_stats* stats);
+
+const char* ss_strerror(ss_status s);
+/* sizeof(ss_stream_desc) as compiled, for bindings that mirror the struct. */
+size_t ss_sizeof_stream_desc(void);
+/* Last CUDA error code seen by this context (cudaError_t as int), 0 if none. */
+int32_t ss_last_cuda_error(ss_ctx* ctx);
+/* Number of kernels this context has launched since creation. */
+int64_t ss_launch_count(ss_ctx* ctx);
+/* "simt" or "tcgen05": the chunk kernel the last ss_verify_chunk used. */
+const char* ss_last_chunk_kernel(ss_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECSTREAM_H_ */

@@ -1,0 +1,244 @@
+"""ctypes binding of libspecstream: the same entry points as include/specstream.h.
+
+Argument marshalling only - every step of the path runs in the library's CUDA
+kernels.  PyTorch supplies device memory and streams.  There is no fallback: if
+the shared library is missing or the device is not sm_100, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libspecstream.so")
+
+SS_OK = 0
+STATUS_NAMES = ["SS_OK", "SS_ERR_ARG", "SS_ERR_SHAPE", "SS_ERR_ALIGN", "SS_ERR_STATE",
+                "SS_ERR_CAPACITY", "SS_ERR_UNSUPPORTED", "SS_ERR_CUDA", "SS_ERR_DEVICE_FLAG",
+                "SS_ERR_TIMEOUT"]
+(SS_ERR_ARG, SS_ERR_SHAPE, SS_ERR_ALIGN, SS_ERR_STATE, SS_ERR_CAPACITY, SS_ERR_UNSUPPORTED,
+ SS_ERR_CUDA, SS_ERR_DEVICE_FLAG, SS_ERR_TIMEOUT) = range(1, 10)
+SS_DEV_BAD_VALID_LEN, SS_DEV_BAD_ACCEPT, SS_DEV_DST_OVERFLOW, SS_DEV_WAIT_EXPIRED = 1, 2, 4, 8
+SS_FLAG_FORCE_SIMT, SS_FLAG_OVERLAP_CHUNKS = 1, 2
+SS_MASK_CHAIN, SS_MASK_TREE_BITS = 0, 1
+
+EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "ss_verify_chunk",
+           "ss_verify_local", "ss_verify_finalize", "ss_commit_gather", "ss_poll_status",
+           "ss_stream_round", "ss_strerror", "ss_sizeof_stream_desc", "ss_last_cuda_error", "ss_launch_count",
+           "ss_last_chunk_kernel"]
+
+
+class ss_config(C.Structure):
+    _fields_ = [("max_B", C.c_int32), ("H_q", C.c_int32), ("H_kv", C.c_int32), ("d", C.c_int32),
+                ("max_Tq", C.c_int32), ("max_Tloc", C.c_int32), ("max_Lc", C.c_int32),
+                ("max_chunks", C.c_int32), ("device", C.c_int32), ("flags", C.c_uint32)]
+
+
+class ss_tensor(C.Structure):
+    _fields_ = [("ptr", C.c_void_p), ("stride_b", C.c_int64), ("stride_h", C.c_int64),
+                ("stride_t", C.c_int64)]
+
+
+class ss_stream_desc(C.Structure):
+    _fields_ = [("B", C.c_int32), ("T_q", C.c_int32), ("L_c", C.c_int32), ("scale", C.c_float),
+                ("hist", C.POINTER(C.c_void_p)), ("hist_len", C.POINTER(C.c_int32)),
+                ("batch_chunks", C.c_int32),
+                ("stage_k", C.c_void_p * 2), ("stage_v", C.c_void_p * 2),
+                ("scratch_fills", C.c_int32),
+                ("valid_len_host", C.c_void_p), ("valid_len_dev", C.c_void_p),
+                ("Q", ss_tensor), ("K_loc", ss_tensor), ("V_loc", ss_tensor),
+                ("mask_kind", C.c_int), ("mask_bits", C.c_void_p),
+                ("O", C.c_void_p), ("LSE", C.c_void_p),
+                ("accept_idx", C.c_void_p), ("accept_cnt", C.c_void_p), ("zero_off", C.c_void_p),
+                ("commit_k", C.c_void_p), ("commit_v", C.c_void_p),
+                ("host_commit_k", C.c_void_p), ("host_commit_v", C.c_void_p),
+                ("O_host", C.c_void_p), ("LSE_host", C.c_void_p),
+                ("copy_only", C.c_int32)]
+
+
+class ss_stream_stats(C.Structure):
+    _fields_ = [("ms_total", C.c_double), ("ms_device", C.c_float), ("h2d_bytes", C.c_int64),
+                ("d2h_bytes", C.c_int64), ("chunk_calls", C.c_int32), ("copies", C.c_int32)]
+
+
+_lib = None
+
+
+def load() -> C.CDLL:
+    """Load the shared library (raises if it has not been built)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} not found: build it with "
+                           "`python -m paper_2609_33184_b200.build` (there is no fallback path)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, u32p = C.c_void_p, C.c_int32, C.POINTER(C.c_uint32)
+    lib.ss_workspace_bytes.restype = C.c_size_t
+    lib.ss_workspace_bytes.argtypes = [C.POINTER(ss_config)]
+    lib.ss_create.restype = C.c_int
+    lib.ss_create.argtypes = [C.POINTER(vp), C.POINTER(ss_config), vp, C.c_size_t]
+    lib.ss_destroy.restype = C.c_int
+    lib.ss_destroy.argtypes = [vp]
+    lib.ss_verify_begin.restype = C.c_int
+    lib.ss_verify_begin.argtypes = [vp, ss_tensor, i32, i32, C.c_float, vp]
+    lib.ss_verify_chunk.restype = C.c_int
+    lib.ss_verify_chunk.argtypes = [vp, ss_tensor, ss_tensor, i32, vp, vp]
+    lib.ss_verify_local.restype = C.c_int
+    lib.ss_verify_local.argtypes = [vp, ss_tensor, ss_tensor, i32, C.c_int, vp, vp]
+    lib.ss_verify_finalize.restype = C.c_int
+    lib.ss_verify_finalize.argtypes = [vp, vp, vp, vp]
+    lib.ss_commit_gather.restype = C.c_int
+    lib.ss_commit_gather.argtypes = [vp, ss_tensor, ss_tensor, i32, i32, vp, vp, ss_tensor,
+                                     ss_tensor, i32, vp, vp]
+    lib.ss_poll_status.restype = C.c_int
+    lib.ss_poll_status.argtypes = [vp, vp, i32, u32p]
+    lib.ss_stream_round.restype = C.c_int
+    lib.ss_stream_round.argtypes = [vp, C.POINTER(ss_stream_desc), C.POINTER(ss_stream_stats)]
+    lib.ss_strerror.restype = C.c_char_p
+    lib.ss_strerror.argtypes = [C.c_int]
+    lib.ss_sizeof_stream_desc.restype = C.c_size_t
+    lib.ss_sizeof_stream_desc.argtypes = []
+    lib.ss_last_cuda_error.restype = i32
+    lib.ss_last_cuda_error.argtypes = [vp]
+    lib.ss_launch_count.restype = C.c_int64
+    lib.ss_launch_count.argtypes = [vp]
+    lib.ss_last_chunk_kernel.restype = C.c_char_p
+    lib.ss_last_chunk_kernel.argtypes = [vp]
+    _lib = lib
+    return lib
+
+
+class SpecStreamError(RuntimeError):
+    def __init__(self, status: int, where: str, cuda: int = 0):
+        self.status = status
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        msg = f"{where}: {name} ({load().ss_strerror(status).decode()})"
+        if cuda:
+            msg += f" [cudaError {cuda}]"
+        super().__init__(msg)
+
+
+def as_ss_tensor(t: torch.Tensor) -> ss_tensor:
+    """[B, H, T, d] bf16 torch tensor -> ss_tensor (strides in elements)."""
+    assert t.dim() == 4 and t.dtype == torch.bfloat16 and t.stride(3) == 1, (t.shape, t.dtype, t.stride())
+    return ss_tensor(t.data_ptr(), t.stride(0), t.stride(1), t.stride(2))
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+class Context:
+    """Owns an ss_ctx and its torch-allocated workspace.  Methods mirror the C entry points."""
+
+    def __init__(self, max_B: int, H_q: int, H_kv: int, d: int, max_Tq: int, max_Tloc: int,
+                 max_Lc: int, max_chunks: int = 0, device: int = 0, flags: int = 0):
+        self.lib = load()
+        self.cfg = ss_config(max_B, H_q, H_kv, d, max_Tq, max_Tloc, max_Lc, max_chunks, device, flags)
+        n = self.lib.ss_workspace_bytes(C.byref(self.cfg))
+        if n == 0:
+            raise SpecStreamError(SS_ERR_SHAPE, "ss_workspace_bytes")
+        self.workspace = torch.empty(n, dtype=torch.uint8, device=f"cuda:{device}")
+        self.handle = C.c_void_p()
+        st = self.lib.ss_create(C.byref(self.handle), C.byref(self.cfg), self.workspace.data_ptr(), n)
+        if st != SS_OK:
+            raise SpecStreamError(st, "ss_create")
+        self.H_q, self.H_kv, self.d = H_q, H_kv, d
+
+    def _check(self, st: int, where: str):
+        if st != SS_OK:
+            raise SpecStreamError(st, where, self.lib.ss_last_cuda_error(self.handle))
+
+    def close(self):
+        if self.handle:
+            self.lib.ss_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # --- the five calls of the path -------------------------------------------------------
+    def ss_verify_begin(self, Q: torch.Tensor, scale: float, stream=None):
+        B, H_q, T_q, d = Q.shape
+        assert H_q == self.H_q and d == self.d
+        self._check(self.lib.ss_verify_begin(self.handle, as_ss_tensor(Q), B, T_q, scale,
+                                             _stream_ptr(stream)), "ss_verify_begin")
+
+    def ss_verify_chunk(self, K: torch.Tensor, V: torch.Tensor, valid_len: Optional[torch.Tensor] = None,
+                        stream=None):
+        L_c = K.shape[2]
+        if valid_len is not None:
+            assert valid_len.dtype == torch.int32 and valid_len.is_cuda
+        self._check(self.lib.ss_verify_chunk(self.handle, as_ss_tensor(K), as_ss_tensor(V), L_c,
+                                             _ptr(valid_len), _stream_ptr(stream)), "ss_verify_chunk")
+
+    def ss_verify_local(self, K_loc: torch.Tensor, V_loc: torch.Tensor, mask_kind: int = SS_MASK_CHAIN,
+                        mask_bits: Optional[torch.Tensor] = None, stream=None):
+        T_loc = K_loc.shape[2]
+        if mask_bits is not None:
+            assert mask_bits.dtype == torch.int64 and mask_bits.is_contiguous()
+        self._check(self.lib.ss_verify_local(self.handle, as_ss_tensor(K_loc), as_ss_tensor(V_loc),
+                                             T_loc, mask_kind, _ptr(mask_bits), _stream_ptr(stream)),
+                    "ss_verify_local")
+
+    def ss_verify_finalize(self, O: torch.Tensor, LSE: Optional[torch.Tensor], stream=None):
+        assert O.dtype == torch.bfloat16 and O.is_contiguous()
+        if LSE is not None:
+            assert LSE.dtype == torch.float32 and LSE.is_contiguous()
+        self._check(self.lib.ss_verify_finalize(self.handle, O.data_ptr(), _ptr(LSE),
+                                                _stream_ptr(stream)), "ss_verify_finalize")
+
+    def ss_commit_gather(self, K_loc, V_loc, accept_idx, accept_cnt, K_dst, V_dst, dst_off, stream=None):
+        B, _, T_loc, _ = K_loc.shape
+        cap = K_dst.shape[2]
+        for t in (accept_idx, accept_cnt, dst_off):
+            assert t.dtype == torch.int32 and t.is_contiguous() and t.is_cuda
+        self._check(self.lib.ss_commit_gather(self.handle, as_ss_tensor(K_loc), as_ss_tensor(V_loc), B,
+                                              T_loc, accept_idx.data_ptr(), accept_cnt.data_ptr(),
+                                              as_ss_tensor(K_dst), as_ss_tensor(V_dst), cap,
+                                              dst_off.data_ptr(), _stream_ptr(stream)), "ss_commit_gather")
+
+    def ss_poll_status(self, stream=None, timeout_ms: int = 0):
+        """Returns (status, device_bits)."""
+        bits = C.c_uint32(0)
+        st = self.lib.ss_poll_status(self.handle, _stream_ptr(stream), timeout_ms, C.byref(bits))
+        return st, bits.value
+
+    def ss_stream_round(self, desc: ss_stream_desc) -> ss_stream_stats:
+        stats = ss_stream_stats()
+        self._check(self.lib.ss_stream_round(self.handle, C.byref(desc), C.byref(stats)), "ss_stream_round")
+        return stats
+
+    def launch_count(self) -> int:
+        return int(self.lib.ss_launch_count(self.handle))
+
+    def last_chunk_kernel(self) -> str:
+        return self.lib.ss_last_chunk_kernel(self.handle).decode()
+
+
+def verify_round(ctx: Context, Q, chunks: Sequence, K_loc, V_loc, scale: float, mask_kind=SS_MASK_CHAIN,
+                 mask_bits=None, O=None, LSE=None, stream=None):
+    """One full round through the five-call boundary.  ``chunks`` = [(K, V, valid_len|None), ...]."""
+    B, H_q, T_q, d = Q.shape
+    if O is None:
+        O = torch.empty(B, H_q, T_q, d, dtype=torch.bfloat16, device=Q.device)
+    if LSE is None:
+        LSE = torch.empty(B, H_q, T_q, dtype=torch.float32, device=Q.device)
+    ctx.ss_verify_begin(Q, scale, stream)
+    for K, V, vl in chunks:
+        ctx.ss_verify_chunk(K, V, vl, stream)
+    if K_loc is not None:
+        ctx.ss_verify_local(K_loc, V_loc, mask_kind, mask_bits, stream)
+    ctx.ss_verify_finalize(O, LSE, stream)
+    return O, LSE

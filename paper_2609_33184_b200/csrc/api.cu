@@ -1,0 +1,585 @@
+// Host side of libspecstream: argument validation, round state machine, workspace layout,
+// tensor-map cache and kernel launches.  Allocates no device memory.
+#include <chrono>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "ss_internal.h"
+
+struct ss_ctx {
+  ss_config cfg;
+  int G, R_max, R_stride;
+  int slots_per_set;       // (split, b, kvh) slots of one partial set
+  int n_set_cap;           // chunk sets (the local set is one more)
+  uint8_t* ws;
+  size_t ws_bytes;
+  uint32_t* status;        // device status word
+  float2* part_ml;
+  float* part_a;
+  int64_t set_stride_ml, set_stride_a;
+  bool tc_ok;              // device can run the tensor-core kernel
+  // round state
+  enum { IDLE, OPEN } state;
+  ss_tensor Q;
+  int B, T_q;
+  float scale;
+  int n_sets;
+  uint8_t splits[ss::kMaxSets];
+  bool has_local;
+  bool first_launch;       // next kernel is the first of the round (or follows a fold)
+  cudaStream_t stream;
+  int32_t last_cuda;
+  int64_t launches;
+  const char* last_kernel;
+  int force_splits;        // SS_SPLITS env override (0 = automatic)
+  int target_ctas;
+  // tensor-map cache
+  struct TmEntry {
+    const void* ptr;
+    int64_t sb, sh, st;
+    int B, L_c;
+    CUtensorMap map;
+    uint64_t age;
+  } tm[64];
+  int tm_n;
+  uint64_t tm_clock;
+  // pipeline resources (created lazily by ss_stream_round)
+  cudaStream_t copy_stream, attn_stream;
+  cudaEvent_t ev_ready[2], ev_free[2], ev_t0, ev_t1;
+  bool pipe_ready;
+  bool no_overlap;          // set while ss_stream_round drives the context
+};
+
+namespace {
+
+using ss::kMaxSets;
+using ss::kMaxSplits;
+using ss::kTileKeys;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool cfg_valid(const ss_config* c) {
+  if (!c) return false;
+  if (c->max_B <= 0 || c->H_q <= 0 || c->H_kv <= 0 || c->max_Tq <= 0 || c->max_Tloc < 0 ||
+      c->max_Lc <= 0)
+    return false;
+  if (c->H_q % c->H_kv) return false;
+  if (c->d != 64 && c->d != 128) return false;
+  if (c->max_Tloc > 1024) return false;
+  if (c->max_chunks < 0 || c->max_chunks > kMaxSets) return false;
+  if ((int64_t)c->max_Tq * (c->H_q / c->H_kv) > 4096) return false;
+  return true;
+}
+
+int set_cap(const ss_config* c) { return c->max_chunks ? c->max_chunks : 64; }
+
+int target_ctas_default() {
+  const char* e = getenv("SS_TARGET_CTAS");
+  int v = e ? atoi(e) : 0;
+  return v > 0 ? v : 2 * ss::kNumSM;
+}
+
+// (split, b, kvh) slots one chunk call may use: enough for ~2 CTAs per SM at the largest batch.
+int slots_for(const ss_config* c) {
+  const int pairs = c->max_B * c->H_kv;
+  int s = (target_ctas_default() + pairs - 1) / pairs;
+  if (s < 1) s = 1;
+  if (s > kMaxSplits) s = kMaxSplits;
+  return pairs * s;
+}
+
+struct Layout {
+  size_t off_ml, off_a, total;
+  int64_t set_stride_ml, set_stride_a;
+  int R_stride;
+};
+
+Layout layout_for(const ss_config* c) {
+  Layout L;
+  const int G = c->H_q / c->H_kv;
+  L.R_stride = c->max_Tq * G;
+  const int64_t rows = (int64_t)slots_for(c) * L.R_stride;
+  L.set_stride_ml = rows;                 // float2 elements
+  L.set_stride_a = rows * c->d;           // float elements
+  const int sets = set_cap(c) + 1;
+  L.off_ml = 256;
+  L.off_a = align_up(L.off_ml + (size_t)sets * rows * sizeof(float2), 256);
+  L.total = align_up(L.off_a + (size_t)sets * rows * c->d * sizeof(float), 256);
+  return L;
+}
+
+bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+bool tensor_ok(const ss_tensor& t) {
+  return aligned16(t.ptr) && (t.stride_b % 8 == 0) && (t.stride_h % 8 == 0) && (t.stride_t % 8 == 0);
+}
+
+ss_status cuda_fail(ss_ctx* c, cudaError_t e) {
+  c->last_cuda = (int32_t)e;
+  return SS_ERR_CUDA;
+}
+
+// Tensor map over K or V [B, H_kv, L_c, d] with a [64 tokens][64 d] box and 128-byte swizzle.
+bool get_tensor_map(ss_ctx* c, const ss_tensor& t, int B, int L_c, CUtensorMap* out) {
+  for (int i = 0; i < c->tm_n; ++i) {
+    ss_ctx::TmEntry& e = c->tm[i];
+    if (e.ptr == t.ptr && e.sb == t.stride_b && e.sh == t.stride_h && e.st == t.stride_t &&
+        e.B == B && e.L_c == L_c) {
+      e.age = ++c->tm_clock;
+      *out = e.map;
+      return true;
+    }
+  }
+  if (!g_encode) return false;
+  const int H_kv = c->cfg.H_kv, d = c->cfg.d;
+  cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)L_c, (cuuint64_t)H_kv, (cuuint64_t)B};
+  // unused outer strides still have to be positive multiples of 16 bytes
+  const int64_t st = t.stride_t, sh = (H_kv > 1 || t.stride_h > 0) ? t.stride_h : (int64_t)L_c * st;
+  const int64_t sb = (B > 1 || t.stride_b > 0) ? t.stride_b : (int64_t)H_kv * sh;
+  if (st <= 0 || sh <= 0 || sb <= 0) return false;
+  cuuint64_t strides[3] = {(cuuint64_t)st * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
+  cuuint32_t box[4] = {64, (cuuint32_t)kTileKeys, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUtensorMap m;
+  CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(t.ptr), dims,
+                        strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  int slot = c->tm_n;
+  if (c->tm_n < 64) {
+    ++c->tm_n;
+  } else {
+    slot = 0;
+    for (int i = 1; i < 64; ++i)
+      if (c->tm[i].age < c->tm[slot].age) slot = i;
+  }
+  c->tm[slot] = {t.ptr, t.stride_b, t.stride_h, t.stride_t, B, L_c, m, ++c->tm_clock};
+  *out = m;
+  return true;
+}
+
+bool use_pdl(ss_ctx* c) {
+  return (c->cfg.flags & SS_FLAG_OVERLAP_CHUNKS) && !c->first_launch && !c->no_overlap;
+}
+
+void fill_merge(ss_ctx* c, ss::MergeParams* m) {
+  memset(m, 0, sizeof(*m));
+  m->part_ml = c->part_ml;
+  m->part_a = c->part_a;
+  m->set_stride_ml = c->set_stride_ml;
+  m->set_stride_a = c->set_stride_a;
+  m->n_sets = c->n_sets;
+  m->has_local = c->has_local ? 1 : 0;
+  m->local_set = c->n_set_cap;
+  m->B = c->B;
+  m->H_q = c->cfg.H_q;
+  m->H_kv = c->cfg.H_kv;
+  m->G = c->G;
+  m->T_q = c->T_q;
+  m->d = c->cfg.d;
+  m->R_stride = c->R_stride;
+  memcpy(m->splits, c->splits, sizeof(m->splits));
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t ss_workspace_bytes(const ss_config* cfg) {
+  if (!cfg_valid(cfg)) return 0;
+  return layout_for(cfg).total;
+}
+
+ss_status ss_create(ss_ctx** out, const ss_config* cfg, void* workspace, size_t workspace_bytes) {
+  if (!out || !cfg || !workspace) return SS_ERR_ARG;
+  if (!cfg_valid(cfg)) return SS_ERR_SHAPE;
+  if ((uintptr_t)workspace & 255) return SS_ERR_ALIGN;
+  const Layout L = layout_for(cfg);
+  if (workspace_bytes < L.total) return SS_ERR_CAPACITY;
+  cudaDeviceProp prop;
+  cudaError_t e = cudaGetDeviceProperties(&prop, cfg->device);
+  if (e != cudaSuccess) return SS_ERR_CUDA;
+  if (prop.major != 10) return SS_ERR_UNSUPPORTED;
+  e = cudaSetDevice(cfg->device);
+  if (e != cudaSuccess) return SS_ERR_CUDA;
+
+  ss_ctx* c = new (std::nothrow) ss_ctx();
+  if (!c) return SS_ERR_ARG;
+  memset(c, 0, sizeof(*c));
+  c->cfg = *cfg;
+  c->G = cfg->H_q / cfg->H_kv;
+  c->R_max = cfg->max_Tq * c->G;
+  c->R_stride = L.R_stride;
+  c->slots_per_set = slots_for(cfg);
+  c->n_set_cap = set_cap(cfg);
+  c->ws = (uint8_t*)workspace;
+  c->ws_bytes = workspace_bytes;
+  c->status = (uint32_t*)c->ws;
+  c->part_ml = (float2*)(c->ws + L.off_ml);
+  c->part_a = (float*)(c->ws + L.off_a);
+  c->set_stride_ml = L.set_stride_ml;
+  c->set_stride_a = L.set_stride_a;
+  c->state = ss_ctx::IDLE;
+  c->last_kernel = "none";
+  c->target_ctas = target_ctas_default();
+  const char* fs = getenv("SS_SPLITS");
+  c->force_splits = fs ? atoi(fs) : 0;
+
+  if (!g_encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) ==
+            cudaSuccess &&
+        qr == cudaDriverEntryPointSuccess)
+      g_encode = (EncodeTiledFn)fn;
+  }
+  c->tc_ok = (g_encode != nullptr) && (cfg->d == 128) && !(cfg->flags & SS_FLAG_FORCE_SIMT);
+  if (c->tc_ok) {
+    e = ss::chunk_tc_prepare();
+    if (e != cudaSuccess) {
+      delete c;
+      return SS_ERR_CUDA;
+    }
+  }
+  e = cudaMemset(c->status, 0, 256);
+  if (e != cudaSuccess) {
+    delete c;
+    return SS_ERR_CUDA;
+  }
+  *out = c;
+  return SS_OK;
+}
+
+ss_status ss_destroy(ss_ctx* c) {
+  if (!c) return SS_ERR_ARG;
+  if (c->pipe_ready) {
+    cudaStreamDestroy(c->copy_stream);
+    cudaStreamDestroy(c->attn_stream);
+    for (int i = 0; i < 2; ++i) {
+      cudaEventDestroy(c->ev_ready[i]);
+      cudaEventDestroy(c->ev_free[i]);
+    }
+    cudaEventDestroy(c->ev_t0);
+    cudaEventDestroy(c->ev_t1);
+  }
+  delete c;
+  return SS_OK;
+}
+
+ss_status ss_verify_begin(ss_ctx* c, ss_tensor Q, int32_t B, int32_t T_q, float scale,
+                          void* stream) {
+  if (!c || !Q.ptr) return SS_ERR_ARG;
+  if (B <= 0 || T_q <= 0) return SS_ERR_ARG;
+  if (B > c->cfg.max_B || T_q > c->cfg.max_Tq) return SS_ERR_SHAPE;
+  if (!tensor_ok(Q)) return SS_ERR_ALIGN;
+  if (c->state != ss_ctx::IDLE) return SS_ERR_STATE;
+  // The identity state (m, l, a) = (-inf, 0, 0) of every row is represented by an empty
+  // list of partial sets: finalize starts its merge from the identity.
+  c->Q = Q;
+  c->B = B;
+  c->T_q = T_q;
+  c->scale = scale;
+  c->n_sets = 0;
+  c->has_local = false;
+  c->first_launch = true;
+  c->stream = (cudaStream_t)stream;
+  c->state = ss_ctx::OPEN;
+  return SS_OK;
+}
+
+ss_status ss_verify_chunk(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c,
+                          const int32_t* valid_len, void* stream) {
+  if (!c || !K.ptr || !V.ptr) return SS_ERR_ARG;
+  if (L_c <= 0) return SS_ERR_ARG;
+  if (L_c > c->cfg.max_Lc) return SS_ERR_SHAPE;
+  if (!tensor_ok(K) || !tensor_ok(V)) return SS_ERR_ALIGN;
+  if (valid_len && ((uintptr_t)valid_len & 3)) return SS_ERR_ALIGN;
+  if (c->state != ss_ctx::OPEN || (cudaStream_t)stream != c->stream) return SS_ERR_STATE;
+  cudaStream_t s = c->stream;
+
+  if (c->n_sets == c->n_set_cap) {
+    // all partial sets in use: fold them into set 0 (Eq. 14 is associative)
+    ss::MergeParams m;
+    fill_merge(c, &m);
+    m.has_local = 0;
+    m.fold_ml = c->part_ml;
+    m.fold_a = c->part_a;
+    cudaError_t e = ss::launch_fold(m, s);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    ++c->launches;
+    c->n_sets = 1;
+    c->splits[0] = 1;
+    c->first_launch = true;  // the next kernel must not overlap the fold
+  }
+
+  const int R = c->T_q * c->G;
+  const int pairs = c->B * c->cfg.H_kv;
+  const int n_tiles = (L_c + kTileKeys - 1) / kTileKeys;
+  CUtensorMap tmK, tmV;
+  bool tc = c->tc_ok;
+  if (tc) tc = get_tensor_map(c, K, c->B, L_c, &tmK) && get_tensor_map(c, V, c->B, L_c, &tmV);
+
+  ss::ChunkParams p;
+  memset(&p, 0, sizeof(p));
+  if (tc) {
+    p.row_tiles = (R + 127) / 128;
+    p.rows_per_tile = (R + p.row_tiles - 1) / p.row_tiles;
+    p.groups = p.rows_per_tile <= 32 ? 4 : (p.rows_per_tile <= 64 ? 2 : 1);
+  } else {
+    p.rows_per_tile = 32;
+    p.row_tiles = (R + 31) / 32;
+    p.groups = 1;
+  }
+  int splits = c->force_splits > 0 ? c->force_splits
+                                   : (c->target_ctas + pairs * p.row_tiles - 1) / (pairs * p.row_tiles);
+  const int max_by_slots = c->slots_per_set / pairs;
+  if (splits > max_by_slots) splits = max_by_slots;
+  if (splits > kMaxSplits) splits = kMaxSplits;
+  if (splits > (n_tiles + 1) / 2) splits = (n_tiles + 1) / 2;  // at least two tiles per split
+  if (splits < 1) splits = 1;
+  p.tiles_per_split = (n_tiles + splits - 1) / splits;
+  splits = (n_tiles + p.tiles_per_split - 1) / p.tiles_per_split;
+  p.splits = splits;
+
+  p.Q = (const __nv_bfloat16*)c->Q.ptr;
+  p.q_sb = c->Q.stride_b;
+  p.q_sh = c->Q.stride_h;
+  p.q_st = c->Q.stride_t;
+  p.K = (const __nv_bfloat16*)K.ptr;
+  p.V = (const __nv_bfloat16*)V.ptr;
+  p.k_sb = K.stride_b;
+  p.k_sh = K.stride_h;
+  p.k_st = K.stride_t;
+  p.v_sb = V.stride_b;
+  p.v_sh = V.stride_h;
+  p.v_st = V.stride_t;
+  p.valid_len = valid_len;
+  p.B = c->B;
+  p.H_kv = c->cfg.H_kv;
+  p.G = c->G;
+  p.T_q = c->T_q;
+  p.R = R;
+  p.d = c->cfg.d;
+  p.L_c = L_c;
+  p.scale_log2 = c->scale * 1.4426950408889634f;
+  p.part_ml = c->part_ml + (int64_t)c->n_sets * c->set_stride_ml;
+  p.part_a = c->part_a + (int64_t)c->n_sets * c->set_stride_a;
+  p.R_stride = c->R_stride;
+  p.status = c->status;
+  p.wait_first = 0;
+
+  const bool pdl = use_pdl(c);
+  cudaError_t e = tc ? ss::launch_chunk_tc(p, tmK, tmV, s, pdl) : ss::launch_chunk_simt(p, s, pdl);
+  if (e != cudaSuccess) return cuda_fail(c, e);
+  c->last_kernel = tc ? "tcgen05" : "simt";
+  ++c->launches;
+  c->splits[c->n_sets] = (uint8_t)splits;
+  ++c->n_sets;
+  c->first_launch = false;
+  return SS_OK;
+}
+
+ss_status ss_verify_local(ss_ctx* c, ss_tensor K_loc, ss_tensor V_loc, int32_t T_loc,
+                          ss_mask_kind kind, const uint64_t* mask_bits, void* stream) {
+  if (!c || !K_loc.ptr || !V_loc.ptr) return SS_ERR_ARG;
+  if (T_loc <= 0) return SS_ERR_ARG;
+  if (T_loc > c->cfg.max_Tloc) return SS_ERR_SHAPE;
+  if (kind != SS_MASK_CHAIN && kind != SS_MASK_TREE_BITS) return SS_ERR_ARG;
+  if (kind == SS_MASK_TREE_BITS && !mask_bits) return SS_ERR_ARG;
+  if (!tensor_ok(K_loc) || !tensor_ok(V_loc)) return SS_ERR_ALIGN;
+  if (mask_bits && ((uintptr_t)mask_bits & 7)) return SS_ERR_ALIGN;
+  if (c->state != ss_ctx::OPEN || (cudaStream_t)stream != c->stream || c->has_local)
+    return SS_ERR_STATE;
+  ss::LocalParams p;
+  memset(&p, 0, sizeof(p));
+  p.Q = (const __nv_bfloat16*)c->Q.ptr;
+  p.q_sb = c->Q.stride_b;
+  p.q_sh = c->Q.stride_h;
+  p.q_st = c->Q.stride_t;
+  p.K = (const __nv_bfloat16*)K_loc.ptr;
+  p.V = (const __nv_bfloat16*)V_loc.ptr;
+  p.k_sb = K_loc.stride_b;
+  p.k_sh = K_loc.stride_h;
+  p.k_st = K_loc.stride_t;
+  p.v_sb = V_loc.stride_b;
+  p.v_sh = V_loc.stride_h;
+  p.v_st = V_loc.stride_t;
+  p.mask_bits = (kind == SS_MASK_TREE_BITS) ? mask_bits : nullptr;
+  p.B = c->B;
+  p.H_q = c->cfg.H_q;
+  p.H_kv = c->cfg.H_kv;
+  p.G = c->G;
+  p.T_q = c->T_q;
+  p.T_loc = T_loc;
+  p.d = c->cfg.d;
+  p.mask_words = (T_loc + 63) / 64;
+  p.scale_log2 = c->scale * 1.4426950408889634f;
+  p.part_ml = c->part_ml + (int64_t)c->n_set_cap * c->set_stride_ml;
+  p.part_a = c->part_a + (int64_t)c->n_set_cap * c->set_stride_a;
+  p.R_stride = c->R_stride;
+  cudaError_t e = ss::launch_local(p, c->stream, use_pdl(c));
+  if (e != cudaSuccess) return cuda_fail(c, e);
+  ++c->launches;
+  c->has_local = true;
+  c->first_launch = false;
+  return SS_OK;
+}
+
+ss_status ss_verify_finalize(ss_ctx* c, void* O, float* LSE, void* stream) {
+  if (!c || !O) return SS_ERR_ARG;
+  if (!aligned16(O) || (LSE && ((uintptr_t)LSE & 3))) return SS_ERR_ALIGN;
+  if (c->state != ss_ctx::OPEN || (cudaStream_t)stream != c->stream) return SS_ERR_STATE;
+  ss::MergeParams m;
+  fill_merge(c, &m);
+  m.O = (__nv_bfloat16*)O;
+  m.LSE = LSE;
+  cudaError_t e = ss::launch_finalize(m, c->stream, use_pdl(c));
+  if (e != cudaSuccess) return cuda_fail(c, e);
+  ++c->launches;
+  c->state = ss_ctx::IDLE;
+  c->Q.ptr = nullptr;
+  return SS_OK;
+}
+
+ss_status ss_commit_gather(ss_ctx* c, ss_tensor K_loc, ss_tensor V_loc, int32_t B, int32_t T_loc,
+                           const int32_t* accept_idx, const int32_t* accept_cnt, ss_tensor K_dst,
+                           ss_tensor V_dst, int32_t cap, const int32_t* dst_off, void* stream) {
+  if (!c || !K_loc.ptr || !V_loc.ptr || !K_dst.ptr || !V_dst.ptr || !accept_idx || !accept_cnt ||
+      !dst_off)
+    return SS_ERR_ARG;
+  if (B <= 0 || T_loc <= 0 || cap <= 0) return SS_ERR_ARG;
+  if (B > c->cfg.max_B || T_loc > c->cfg.max_Tloc) return SS_ERR_SHAPE;
+  if (!tensor_ok(K_loc) || !tensor_ok(V_loc) || !tensor_ok(K_dst) || !tensor_ok(V_dst))
+    return SS_ERR_ALIGN;
+  ss::GatherParams p;
+  memset(&p, 0, sizeof(p));
+  p.K_loc = (const uint16_t*)K_loc.ptr;
+  p.V_loc = (const uint16_t*)V_loc.ptr;
+  p.ks_b = K_loc.stride_b;
+  p.ks_h = K_loc.stride_h;
+  p.ks_t = K_loc.stride_t;
+  p.vs_b = V_loc.stride_b;
+  p.vs_h = V_loc.stride_h;
+  p.vs_t = V_loc.stride_t;
+  p.K_dst = (uint16_t*)K_dst.ptr;
+  p.V_dst = (uint16_t*)V_dst.ptr;
+  p.kd_b = K_dst.stride_b;
+  p.kd_h = K_dst.stride_h;
+  p.kd_t = K_dst.stride_t;
+  p.vd_b = V_dst.stride_b;
+  p.vd_h = V_dst.stride_h;
+  p.vd_t = V_dst.stride_t;
+  p.accept_idx = accept_idx;
+  p.accept_cnt = accept_cnt;
+  p.dst_off = dst_off;
+  p.B = B;
+  p.H_kv = c->cfg.H_kv;
+  p.T_loc = T_loc;
+  p.d = c->cfg.d;
+  p.cap = cap;
+  p.status = c->status;
+  cudaError_t e = ss::launch_gather(p, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(c, e);
+  ++c->launches;
+  return SS_OK;
+}
+
+ss_status ss_poll_status(ss_ctx* c, void* stream, int32_t timeout_ms, uint32_t* dev_bits) {
+  if (!c) return SS_ERR_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (timeout_ms > 0) {
+    const auto t0 = std::chrono::steady_clock::now();
+    for (;;) {
+      cudaError_t q = cudaStreamQuery(s);
+      if (q == cudaSuccess) break;
+      if (q != cudaErrorNotReady) return cuda_fail(c, q);
+      const auto ms = std::chrono::duration_cast<std::chrono::milliseconds>(
+                          std::chrono::steady_clock::now() - t0)
+                          .count();
+      if (ms > timeout_ms) return SS_ERR_TIMEOUT;
+    }
+  } else {
+    cudaError_t e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+  }
+  uint32_t bits = 0;
+  cudaError_t e = cudaMemcpy(&bits, c->status, 4, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(c, e);
+  if (dev_bits) *dev_bits = bits;
+  if (bits) {
+    e = cudaMemset(c->status, 0, 4);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    return SS_ERR_DEVICE_FLAG;
+  }
+  return SS_OK;
+}
+
+const char* ss_strerror(ss_status s) {
+  switch (s) {
+    case SS_OK: return "ok";
+    case SS_ERR_ARG: return "invalid argument";
+    case SS_ERR_SHAPE: return "shape outside the configured limits";
+    case SS_ERR_ALIGN: return "pointer or stride not 16-byte aligned";
+    case SS_ERR_STATE: return "call order violated";
+    case SS_ERR_CAPACITY: return "workspace too small";
+    case SS_ERR_UNSUPPORTED: return "device is not sm_100";
+    case SS_ERR_CUDA: return "CUDA call failed";
+    case SS_ERR_DEVICE_FLAG: return "device status word set";
+    case SS_ERR_TIMEOUT: return "timed out";
+  }
+  return "unknown";
+}
+
+size_t ss_sizeof_stream_desc(void) { return sizeof(ss_stream_desc); }
+int32_t ss_last_cuda_error(ss_ctx* c) { return c ? c->last_cuda : 0; }
+int64_t ss_launch_count(ss_ctx* c) { return c ? c->launches : 0; }
+const char* ss_last_chunk_kernel(ss_ctx* c) { return c ? c->last_kernel : "none"; }
+
+}  // extern "C"
+
+// accessors for the pipeline translation unit
+namespace ss {
+struct PipeRes {
+  cudaStream_t copy_stream, attn_stream;
+  cudaEvent_t *ev_ready, *ev_free, ev_t0, ev_t1;
+};
+cudaError_t ctx_pipeline(ss_ctx* c, PipeRes* out) {
+  if (!c->pipe_ready) {
+    cudaError_t e;
+    if ((e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking)) != cudaSuccess) return e;
+    if ((e = cudaStreamCreateWithFlags(&c->attn_stream, cudaStreamNonBlocking)) != cudaSuccess) return e;
+    for (int i = 0; i < 2; ++i) {
+      if ((e = cudaEventCreateWithFlags(&c->ev_ready[i], cudaEventDisableTiming)) != cudaSuccess) return e;
+      if ((e = cudaEventCreateWithFlags(&c->ev_free[i], cudaEventDisableTiming)) != cudaSuccess) return e;
+    }
+    if ((e = cudaEventCreate(&c->ev_t0)) != cudaSuccess) return e;
+    if ((e = cudaEventCreate(&c->ev_t1)) != cudaSuccess) return e;
+    c->pipe_ready = true;
+  }
+  out->copy_stream = c->copy_stream;
+  out->attn_stream = c->attn_stream;
+  out->ev_ready = c->ev_ready;
+  out->ev_free = c->ev_free;
+  out->ev_t0 = c->ev_t0;
+  out->ev_t1 = c->ev_t1;
+  return cudaSuccess;
+}
+int ctx_dims(ss_ctx* c, int* H_q, int* H_kv, int* d) {
+  *H_q = c->cfg.H_q;
+  *H_kv = c->cfg.H_kv;
+  *d = c->cfg.d;
+  return c->cfg.max_B;
+}
+void ctx_set_cuda_error(ss_ctx* c, cudaError_t e) { c->last_cuda = (int32_t)e; }
+void ctx_pipeline_mode(ss_ctx* c, bool on) {
+  c->no_overlap = on;
+  if (!on) c->state = ss_ctx::IDLE;  // a round the pipeline left open (error path) is dropped
+}
+}  // namespace ss

@@ -1,0 +1,549 @@
+// Tensor-core chunk attention for sm_100a: TMA-staged K/V tiles, tcgen05 MMAs with the
+// score tile S, the probabilities P and the unnormalised output O held in tensor memory.
+//
+// One CTA owns one (request, kv-head, token split, tile of <= 128 query rows).  All rows of
+// the kv-head (T_q candidate queries x G query heads) ride in the M dimension of the MMAs,
+// so every K/V byte is fetched from HBM once and serves the whole query group.
+//
+//   warp 4 (one lane)  TMA producer: K tile and V tile of 64 tokens per stage, 2 stages,
+//                      128-byte swizzle, evict-first L2 policy (the history is streamed).
+//   warp 5 (one lane)  MMA issuer:   S = Q K^T   (M=128, N=64,  K=d=128: 8 x k16, smem x smem)
+//                                    O += P V    (M=128, N=128, K=64:    4 x k16, tmem x smem)
+//   warps 0-3          softmax: each thread owns one TMEM lane (= one MMA row): reads its
+//                      scores, keeps (m, l) in registers, writes P as packed bf16 to TMEM.
+//
+// When the row tile has <= 32 (<= 64) rows the Q rows are replicated 4x (2x) along M and
+// each replica takes a quarter (half) of the tile's keys: lane L holds row L % R_pad and
+// key group L / R_pad.  All four softmax warps then work on every tile, and the four
+// replicas are four independent online-softmax states that are merged when the CTA ends.
+//
+// Running maximum: a row's reference maximum m only moves when the tile maximum exceeds it
+// by more than 8 (base-2 domain), which keeps exp2(s - m) <= 256 and makes the rescale of O
+// in tensor memory rare.  Two CTAs fit per SM (about 100 KB shared memory, 256 TMEM
+// columns each), so one CTA's ramp-up and tail overlap the other's steady state.
+//
+// Every wait on an mbarrier is bounded; on expiry the CTA raises SS_DEV_WAIT_EXPIRED, lets
+// its own copies land (bounded), frees its tensor memory and returns.
+#include "ss_internal.h"
+
+namespace ss {
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kStages = 2;
+constexpr int kD = 128;
+constexpr int kQBytes = 128 * kD * 2;               // 32 KB: two 64-column halves of 128 rows
+constexpr int kHalfTile = kTileKeys * 64 * 2;       // 8 KB: [64 keys][64 d] bf16
+constexpr int kTileBytes = 2 * kHalfTile;           // 16 KB: one K tile or one V tile
+constexpr int kStageBytes = 2 * kTileBytes;         // K then V
+constexpr int kSmemData = kQBytes + kStages * kStageBytes;  // 96 KB
+constexpr int kSmemCtl = 2048;
+constexpr int kSmemTotal = kSmemData + kSmemCtl + 1024;     // + alignment slack
+constexpr uint32_t kTmemCols = 256;
+constexpr uint32_t kColS = 0, kColP = 64, kColO = 128;
+constexpr float kRescaleThreshold = 8.f;
+constexpr unsigned long long kWaitNs = 2000000000ull;       // 2 s
+
+struct Ctl {
+  uint64_t kfull[kStages], vfull[kStages], empty[kStages];
+  uint64_t sfull, pready, pvdone;
+  uint32_t tmem_base;
+  volatile uint32_t abort;
+  float2 ml[128];
+};
+static_assert(sizeof(Ctl) <= kSmemCtl, "control block");
+
+// ---- small PTX wrappers ------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ unsigned long long gtime_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
+               "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the deadline passed or another role aborted.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Ctl* ctl,
+                                          uint32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = gtime_ns();
+  uint32_t spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 255u) == 0) {
+      if (ctl->abort) return false;
+      if (gtime_ns() - t0 > kWaitNs) {
+        ctl->abort = 1;
+        atomicOr(status, SS_DEV_WAIT_EXPIRED);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ void fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                   smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_wait_st() {
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void named_bar_sync(int id, int n) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
+}
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+// TMA tiled load of one [64 tokens][64 d] box into shared memory, completion on an mbarrier.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, int c0, int c1,
+                                            int c2, int c3, uint64_t* bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3, %4, %5}], [%6], %7;" ::"r"(dst),
+      "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar)), "l"(policy)
+      : "memory");
+}
+// tcgen05.mma, A and B from shared memory descriptors.
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                       uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// tcgen05.mma, A from tensor memory, B from a shared memory descriptor.
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
+                                       uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+        "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+      "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+      : "memory");
+}
+
+// Shared-memory matrix descriptors (sm_100 format: version 1 at bit 46, 128-byte swizzle).
+// K-major operand (rows of 128 bytes, 8-row atoms 1024 bytes apart).
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr) {
+  return (uint64_t)((saddr >> 4) & 0x3FFF) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// MN-major operand: 64 MN-elements (128 bytes) contiguous per k row, 8-k-row atoms 1024
+// bytes apart, the next 64 MN-elements `lbo_bytes` away.
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr, uint32_t lbo_bytes) {
+  return (uint64_t)((saddr >> 4) & 0x3FFF) | ((uint64_t)(lbo_bytes >> 4) << 16) |
+         ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, A K-major.
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) |
+         ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// ---- softmax of one tile for one TMEM lane --------------------------------------------------
+// NC = number of key columns this lane owns in a 64-key tile.
+template <int NC>
+__device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_p, uint32_t t_o, int c0,
+                                             int n_valid, bool have_o, float scale_log2, float& m,
+                                             float& l) {
+  uint32_t raw[NC / 16][16];
+#pragma unroll
+  for (int q = 0; q < NC / 16; ++q) tmem_ld16(t_s + c0 + q * 16, raw[q]);
+  tc_wait_ld();
+  float s[NC];
+  float mx = -INFINITY;
+#pragma unroll
+  for (int c = 0; c < NC; ++c) {
+    float v = __uint_as_float(raw[c / 16][c % 16]) * scale_log2;
+    if (c0 + c >= n_valid) v = -INFINITY;
+    s[c] = v;
+    mx = fmaxf(mx, v);
+  }
+  float f = 1.f;
+  if (mx > m + kRescaleThreshold) {  // also the first finite maximum (m = -inf)
+    f = (m == -INFINITY) ? 0.f : exp2f(m - mx);
+    l *= f;
+    m = mx;
+  }
+  const bool need = have_o && (f != 1.f);
+  if (__any_sync(0xffffffffu, need)) {
+    // rare: move this lane's O row to the new reference maximum
+#pragma unroll 1
+    for (int q = 0; q < kD / 16; ++q) {
+      uint32_t o[16];
+      tmem_ld16(t_o + q * 16, o);
+      tc_wait_ld();
+#pragma unroll
+      for (int c = 0; c < 16; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * f);
+      tmem_st16(t_o + q * 16, o);
+    }
+  }
+  const float m_use = (m == -INFINITY) ? 0.f : m;
+  uint32_t pk[NC / 2];
+  float sum = 0.f;
+#pragma unroll
+  for (int c = 0; c < NC; c += 2) {
+    const float p0 = exp2f(s[c] - m_use), p1 = exp2f(s[c + 1] - m_use);
+    sum += p0 + p1;
+    __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);  // low half = even key
+    pk[c / 2] = *reinterpret_cast<uint32_t*>(&h);
+  }
+  l += sum;
+#pragma unroll
+  for (int q = 0; q < NC / 16; ++q) tmem_st8(t_p + c0 / 2 + q * 8, &pk[q * 8]);
+  tc_wait_st();
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
+chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
+                const __grid_constant__ CUtensorMap tmV) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* q_s = smem;
+  uint8_t* st_s = smem + kQBytes;
+  Ctl* ctl = reinterpret_cast<Ctl*>(smem + kSmemData);
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int rt = blockIdx.x % p.row_tiles;
+  const int split = blockIdx.x / p.row_tiles;
+  const int kvh = blockIdx.y, b = blockIdx.z;
+  const int row0 = rt * p.rows_per_tile;
+  const int nrows = min(p.rows_per_tile, p.R - row0);
+  const int r_pad = 128 / p.groups;
+
+  if (p.wait_first) pdl_wait_prior();
+  pdl_launch_dependents();
+
+  int valid = p.L_c;
+  if (p.valid_len) {
+    valid = p.valid_len[b];
+    if (valid < 0 || valid > p.L_c) {
+      if (tid == 0) atomicOr(p.status, SS_DEV_BAD_VALID_LEN);
+      valid = max(0, min(valid, p.L_c));
+    }
+  }
+  const int tok0 = split * p.tiles_per_split * kTileKeys;
+  const int tok1 = min(valid, tok0 + p.tiles_per_split * kTileKeys);
+  const int n_tiles = (tok1 > tok0) ? (tok1 - tok0 + kTileKeys - 1) / kTileKeys : 0;
+
+  const size_t slot = ((size_t)split * p.B + b) * p.H_kv + kvh;
+  float2* out_ml = p.part_ml + slot * p.R_stride + row0;
+  float* out_a = p.part_a + (slot * p.R_stride + row0) * kD;
+
+  if (n_tiles == 0) {  // nothing visible here: identity state, no tensor memory taken
+    if (tid < nrows) out_ml[tid] = make_float2(-INFINITY, 0.f);
+    if (!p.wait_first) pdl_wait_prior();
+    return;
+  }
+
+  // ---- set-up: barriers, tensor memory, Q rows -> swizzled shared memory ------------------
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&ctl->kfull[s], 1);
+      mbar_init(&ctl->vfull[s], 1);
+      mbar_init(&ctl->empty[s], 1);
+    }
+    mbar_init(&ctl->sfull, 1);
+    mbar_init(&ctl->pready, 128);
+    mbar_init(&ctl->pvdone, 1);
+    ctl->abort = 0;
+    fence_barrier_init();
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(&ctl->tmem_base)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // Q: lane L of the MMA's M dimension holds row (L % r_pad) of this row tile (zero if padding).
+  for (int i = tid; i < 128 * (kD / 8); i += kThreads) {
+    const int L = i / (kD / 8), c8 = i % (kD / 8);
+    const int r = L % r_pad;
+    uint4 raw = make_uint4(0, 0, 0, 0);
+    if (r < nrows) {
+      const int rg = row0 + r, g = rg / p.T_q, t = rg % p.T_q;
+      raw = *reinterpret_cast<const uint4*>(p.Q + b * p.q_sb +
+                                            (int64_t)(kvh * p.G + g) * p.q_sh + t * p.q_st + c8 * 8);
+    }
+    const int half = c8 >> 3, j = c8 & 7;
+    *reinterpret_cast<uint4*>(q_s + half * (128 * 128) + L * 128 + ((j ^ (L & 7)) << 4)) = raw;
+  }
+  fence_proxy_async();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = ctl->tmem_base;
+
+  if (warp == 4) {
+    // ===== TMA producer =====
+    if (lane == 0) {
+      const uint64_t pol = l2_evict_first_policy();
+      int issued = 0;
+      for (int it = 0; it < n_tiles; ++it) {
+        const int s = it % kStages;
+        const uint32_t ph = (it / kStages) & 1;
+        if (!mbar_wait(&ctl->empty[s], ph ^ 1, ctl, p.status)) break;
+        const int tok = tok0 + it * kTileKeys;
+        const uint32_t kdst = smem_u32(st_s + s * kStageBytes);
+        const uint32_t vdst = kdst + kTileBytes;
+        mbar_expect_tx(&ctl->kfull[s], kTileBytes);
+        tma_load_4d(kdst, &tmK, 0, tok, kvh, b, &ctl->kfull[s], pol);
+        tma_load_4d(kdst + kHalfTile, &tmK, 64, tok, kvh, b, &ctl->kfull[s], pol);
+        mbar_expect_tx(&ctl->vfull[s], kTileBytes);
+        tma_load_4d(vdst, &tmV, 0, tok, kvh, b, &ctl->vfull[s], pol);
+        tma_load_4d(vdst + kHalfTile, &tmV, 64, tok, kvh, b, &ctl->vfull[s], pol);
+        issued = it + 1;
+      }
+      if (ctl->abort) {
+        // let the copies this thread started land before the CTA leaves (bounded)
+        for (int it = max(0, issued - kStages); it < issued; ++it) {
+          const int s = it % kStages;
+          const uint32_t ph = (it / kStages) & 1;
+          const unsigned long long t0 = gtime_ns();
+          while (!(mbar_try_wait(&ctl->kfull[s], ph) && mbar_try_wait(&ctl->vfull[s], ph)) &&
+                 gtime_ns() - t0 < kWaitNs) {
+          }
+        }
+      }
+    }
+  } else if (warp == 5) {
+    // ===== MMA issuer =====
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = make_idesc(128, kTileKeys, false);
+      constexpr uint32_t idesc_pv = make_idesc(128, kD, true);
+      const uint32_t q_addr = smem_u32(q_s);
+      bool ok = mbar_wait(&ctl->kfull[0], 0, ctl, p.status);
+      if (ok) {
+        tc_fence_after();
+        const uint32_t k_addr = smem_u32(st_s);
+#pragma unroll
+        for (int kk = 0; kk < kD / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * (128 * 128) + (kk & 3) * 32;
+          const uint32_t koff = (kk >> 2) * kHalfTile + (kk & 3) * 32;
+          mma_ss(tmem + kColS, desc_kmajor(q_addr + off), desc_kmajor(k_addr + koff), idesc_qk,
+                 kk > 0);
+        }
+        tc_commit(&ctl->sfull);
+      }
+      for (int it = 0; ok && it < n_tiles; ++it) {
+        const int s = it % kStages;
+        const uint32_t ph = (it / kStages) & 1;
+        ok = mbar_wait(&ctl->pready, it & 1, ctl, p.status) &&
+             mbar_wait(&ctl->vfull[s], ph, ctl, p.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t v_addr = smem_u32(st_s + s * kStageBytes + kTileBytes);
+#pragma unroll
+        for (int kk = 0; kk < kTileKeys / 16; ++kk) {
+          mma_ts(tmem + kColO, tmem + kColP + kk * 8, desc_mnmajor(v_addr + kk * 2048, kHalfTile),
+                 idesc_pv, (it > 0 || kk > 0));
+        }
+        tc_commit(&ctl->empty[s]);
+        if (it + 1 < n_tiles) {
+          const int s2 = (it + 1) % kStages;
+          const uint32_t ph2 = ((it + 1) / kStages) & 1;
+          ok = mbar_wait(&ctl->kfull[s2], ph2, ctl, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t k_addr = smem_u32(st_s + s2 * kStageBytes);
+#pragma unroll
+          for (int kk = 0; kk < kD / 16; ++kk) {
+            const uint32_t off = (kk >> 2) * (128 * 128) + (kk & 3) * 32;
+            const uint32_t koff = (kk >> 2) * kHalfTile + (kk & 3) * 32;
+            mma_ss(tmem + kColS, desc_kmajor(q_addr + off), desc_kmajor(k_addr + koff), idesc_qk,
+                   kk > 0);
+          }
+          tc_commit(&ctl->sfull);
+        } else {
+          tc_commit(&ctl->pvdone);
+        }
+      }
+    }
+  } else {
+    // ===== softmax warps: thread = TMEM lane =====
+    const int L = tid;  // 0..127
+    const int grp = L / r_pad;
+    const int nc = kTileKeys / p.groups;
+    const int c0 = grp * nc;
+    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    const uint32_t t_s = tmem + lane_off + kColS;
+    const uint32_t t_p = tmem + lane_off + kColP;
+    const uint32_t t_o = tmem + lane_off + kColO;
+    float m = -INFINITY, l = 0.f;
+    {  // P columns outside this lane's key group stay zero for the whole kernel
+      uint32_t z[16];
+#pragma unroll
+      for (int c = 0; c < 16; ++c) z[c] = 0;
+      tmem_st16(t_p, z);
+      tmem_st16(t_p + 16, z);
+      tc_wait_st();
+    }
+    bool ok = true;
+    for (int it = 0; it < n_tiles; ++it) {
+      const int s = it % kStages;
+      const uint32_t ph = (it / kStages) & 1;
+      ok = mbar_wait(&ctl->sfull, it & 1, ctl, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      const int n_valid = min(kTileKeys, tok1 - (tok0 + it * kTileKeys));
+      if (n_valid < kTileKeys) {
+        // ragged tail: rows past the valid length may hold anything; P is 0 there, so V must
+        // be finite: clear those rows of the staged V tile (whole 128-byte rows, both halves)
+        ok = mbar_wait(&ctl->vfull[s], ph, ctl, p.status);
+        if (!ok) break;
+        uint8_t* v_s = st_s + s * kStageBytes + kTileBytes;
+        const int n_vec = (kTileKeys - n_valid) * 16;
+        for (int i = L; i < n_vec; i += 128) {
+          const int row = n_valid + (i >> 4), half = (i >> 3) & 1, ch = i & 7;
+          *reinterpret_cast<uint4*>(v_s + half * kHalfTile + row * 128 + ch * 16) =
+              make_uint4(0, 0, 0, 0);
+        }
+        fence_proxy_async();
+      }
+      if (nc == 16)
+        softmax_tile<16>(t_s, t_p, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+      else if (nc == 32)
+        softmax_tile<32>(t_s, t_p, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+      else
+        softmax_tile<64>(t_s, t_p, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+      tc_fence_before();
+      mbar_arrive(&ctl->pready);
+    }
+    ok = ok && mbar_wait(&ctl->pvdone, 0, ctl, p.status);
+    if (ok) {
+      tc_fence_after();
+      // ---- merge the key groups of each row and write the partial state ----
+      float* o_s = reinterpret_cast<float*>(st_s);  // [128][128] fp32 over the free stage buffers
+      ctl->ml[L] = make_float2(m, l);
+      named_bar_sync(1, 128);
+      const int r = L % r_pad;
+      float M = -INFINITY;
+      for (int g = 0; g < p.groups; ++g) M = fmaxf(M, ctl->ml[g * r_pad + r].x);
+      const float f = (m == -INFINITY) ? 0.f : exp2f(m - M);
+#pragma unroll 1
+      for (int q = 0; q < kD / 16; ++q) {
+        uint32_t o[16];
+        tmem_ld16(t_o + q * 16, o);
+        tc_wait_ld();
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) {
+          float4 v;
+          v.x = __uint_as_float(o[c4 * 4 + 0]) * f;
+          v.y = __uint_as_float(o[c4 * 4 + 1]) * f;
+          v.z = __uint_as_float(o[c4 * 4 + 2]) * f;
+          v.w = __uint_as_float(o[c4 * 4 + 3]) * f;
+          *reinterpret_cast<float4*>(&o_s[L * kD + (((q * 4 + c4) ^ (L & 31)) << 2)]) = v;
+        }
+      }
+      if (L < nrows) {
+        float lt = 0.f;
+        for (int g = 0; g < p.groups; ++g) {
+          const float2 st = ctl->ml[g * r_pad + r];
+          if (st.x > -INFINITY) lt += exp2f(st.x - M) * st.y;
+        }
+        out_ml[L] = make_float2(lt > 0.f ? M : -INFINITY, lt);
+      }
+      named_bar_sync(1, 128);
+      for (int rr = warp; rr < nrows; rr += 4) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int g = 0; g < p.groups; ++g) {
+          const int LL = g * r_pad + rr;
+          const float4 v = *reinterpret_cast<const float4*>(&o_s[LL * kD + ((lane ^ (LL & 31)) << 2)]);
+          acc.x += v.x;
+          acc.y += v.y;
+          acc.z += v.z;
+          acc.w += v.w;
+        }
+        *reinterpret_cast<float4*>(out_a + (size_t)rr * kD + lane * 4) = acc;
+      }
+    }
+  }
+
+  // ---- teardown ----
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols)
+                 : "memory");
+  }
+  if (!p.wait_first) pdl_wait_prior();  // keep completion order along the stream
+}
+
+}  // namespace
+
+cudaError_t chunk_tc_prepare() {
+  return cudaFuncSetAttribute(chunk_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              kSmemTotal);
+}
+
+cudaError_t launch_chunk_tc(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                            cudaStream_t s, bool pdl) {
+  dim3 grid(p.splits * p.row_tiles, p.H_kv, p.B), block(kThreads);
+  return launch_kernel(chunk_tc_kernel, grid, block, kSmemTotal, s, pdl, p, tmK, tmV);
+}
+
+}  // namespace ss

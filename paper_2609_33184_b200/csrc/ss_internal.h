@@ -1,0 +1,129 @@
+// Internal declarations shared by the host API and the kernels of libspecstream.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "specstream.h"
+
+namespace ss {
+
+constexpr int kMaxSets = 128;      // chunk-call partial sets a finalize launch can take
+constexpr int kMaxSplits = 16;     // token splits of one chunk call
+constexpr int kTileKeys = 64;      // keys per shared-memory tile of the tensor-core kernel
+constexpr int kNumSM = 148;
+
+// Partial state of one (set, split, request, kv-head): for each of its R rows the pair
+// (m, l) and the unnormalised output a[d].  m is the row maximum of
+// score * scale * log2(e) (base-2 domain), l = sum exp2(s2 - m), a = sum exp2(s2 - m) v.
+// An untouched or empty row is the identity (m = -inf, l = 0); its a[] is never read.
+struct PartialView {
+  float2* ml;        // [slots][R_stride]
+  float* a;          // [slots][R_stride][d]
+};
+
+struct ChunkParams {
+  const __nv_bfloat16* Q;
+  int64_t q_sb, q_sh, q_st;
+  const __nv_bfloat16* K;
+  const __nv_bfloat16* V;
+  int64_t k_sb, k_sh, k_st, v_sb, v_sh, v_st;
+  const int32_t* valid_len;  // device [B] or null
+  int B, H_kv, G, T_q, R, d, L_c;
+  int splits;           // token splits (grid.x / row_tiles)
+  int tiles_per_split;  // kTileKeys-token tiles per split
+  int row_tiles;        // tiles of query rows per (b, kvh)
+  int rows_per_tile;    // rows in each row tile but possibly the last
+  int groups;           // key groups sharing the 128 TMEM lanes (tensor-core kernel)
+  float scale_log2;     // scale * log2(e)
+  float2* part_ml;      // partial set of this call
+  float* part_a;
+  int R_stride;
+  uint32_t* status;
+  int wait_first;       // 1: wait for the preceding kernel before reading inputs
+};
+
+struct LocalParams {
+  const __nv_bfloat16* Q;
+  int64_t q_sb, q_sh, q_st;
+  const __nv_bfloat16* K;
+  const __nv_bfloat16* V;
+  int64_t k_sb, k_sh, k_st, v_sb, v_sh, v_st;
+  const uint64_t* mask_bits;  // null for chain
+  int B, H_q, H_kv, G, T_q, T_loc, d, mask_words;
+  float scale_log2;
+  float2* part_ml;  // local set: slot = b * H_kv + kvh
+  float* part_a;
+  int R_stride;
+};
+
+struct MergeParams {
+  const float2* part_ml;  // set 0
+  const float* part_a;
+  int64_t set_stride_ml;  // elements between sets
+  int64_t set_stride_a;
+  int n_sets;
+  int has_local;
+  int local_set;          // index of the local set
+  int B, H_q, H_kv, G, T_q, d, R_stride;
+  uint8_t splits[kMaxSets];
+  // finalize outputs
+  __nv_bfloat16* O;
+  float* LSE;
+  // fold output (set 0, split 0)
+  float2* fold_ml;
+  float* fold_a;
+};
+
+struct GatherParams {
+  const uint16_t* K_loc;
+  const uint16_t* V_loc;
+  int64_t ks_b, ks_h, ks_t, vs_b, vs_h, vs_t;
+  uint16_t* K_dst;
+  uint16_t* V_dst;
+  int64_t kd_b, kd_h, kd_t, vd_b, vd_h, vd_t;
+  const int32_t* accept_idx;
+  const int32_t* accept_cnt;
+  const int32_t* dst_off;
+  int B, H_kv, T_loc, d, cap;
+  uint32_t* status;
+};
+
+// launchers (each returns the cudaError_t of the launch)
+cudaError_t launch_chunk_simt(const ChunkParams& p, cudaStream_t s, bool pdl);
+cudaError_t launch_chunk_tc(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                            cudaStream_t s, bool pdl);
+cudaError_t chunk_tc_prepare();  // one-time function attributes
+cudaError_t launch_local(const LocalParams& p, cudaStream_t s, bool pdl);
+cudaError_t launch_finalize(const MergeParams& p, cudaStream_t s, bool pdl);
+cudaError_t launch_fold(const MergeParams& p, cudaStream_t s);
+cudaError_t launch_gather(const GatherParams& p, cudaStream_t s);
+
+// Launch helper: optional programmatic stream serialization attribute.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                 cudaStream_t s, bool pdl, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// Device-side programmatic-dependent-launch controls (no-ops when the kernel was
+// launched without the attribute).
+__device__ __forceinline__ void pdl_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait_prior() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+}  // namespace ss

@@ -1,0 +1,177 @@
+// Streamed round: pinned-host history -> two device staging buffers on a copy stream,
+// chunk attention on an attention stream, hand-off by events (Section 4.2, pipelined KV
+// transfers).  While the attention stream works on buffer A, buffer B receives the next
+// fill; a fill carries `batch_chunks` adjacent chunks (a transfer batch).
+#include <chrono>
+#include <cstring>
+
+#include "ss_internal.h"
+
+namespace ss {
+struct PipeRes {
+  cudaStream_t copy_stream, attn_stream;
+  cudaEvent_t *ev_ready, *ev_free, ev_t0, ev_t1;
+};
+cudaError_t ctx_pipeline(ss_ctx* c, PipeRes* out);
+int ctx_dims(ss_ctx* c, int* H_q, int* H_kv, int* d);
+void ctx_set_cuda_error(ss_ctx* c, cudaError_t e);
+void ctx_pipeline_mode(ss_ctx* c, bool on);
+}  // namespace ss
+
+#define SS_CK(expr)                          \
+  do {                                       \
+    cudaError_t e_ = (expr);                 \
+    if (e_ != cudaSuccess) {                 \
+      ss::ctx_set_cuda_error(ctx, e_);       \
+      return SS_ERR_CUDA;                    \
+    }                                        \
+  } while (0)
+#define SS_ST(expr)                  \
+  do {                               \
+    ss_status s_ = (expr);           \
+    if (s_ != SS_OK) return s_;      \
+  } while (0)
+
+static ss_status stream_round_impl(ss_ctx* ctx, const ss_stream_desc* d, ss_stream_stats* stats) {
+  if (!ctx || !d || !d->hist || !d->hist_len) return SS_ERR_ARG;
+  if (d->B <= 0 || d->T_q <= 0 || d->L_c <= 0 || d->batch_chunks <= 0) return SS_ERR_ARG;
+  if (!d->stage_k[0] || !d->stage_k[1] || !d->stage_v[0] || !d->stage_v[1]) return SS_ERR_ARG;
+  if (!d->valid_len_host || !d->valid_len_dev) return SS_ERR_ARG;
+  if (!d->copy_only && (!d->Q.ptr || !d->K_loc.ptr || !d->V_loc.ptr || !d->O)) return SS_ERR_ARG;
+  int H_q, H_kv, hd;
+  const int max_B = ss::ctx_dims(ctx, &H_q, &H_kv, &hd);
+  if (d->B > max_B) return SS_ERR_SHAPE;
+  const int B = d->B, L_c = d->L_c, bc = d->batch_chunks;
+  const int64_t Ls = (int64_t)bc * L_c;  // tokens per staging buffer row
+  int max_len = 0;
+  for (int b = 0; b < B; ++b) {
+    if (d->hist_len[b] < 0 || (d->hist_len[b] > 0 && !d->hist[b])) return SS_ERR_ARG;
+    if (d->hist_len[b] > max_len) max_len = d->hist_len[b];
+  }
+  const int n_chunks = (max_len + L_c - 1) / L_c;
+  const int n_fills = (n_chunks + bc - 1) / bc;
+  if (n_fills > d->scratch_fills) return SS_ERR_CAPACITY;
+
+  ss::PipeRes r;
+  SS_CK(ss::ctx_pipeline(ctx, &r));
+  const auto wall0 = std::chrono::steady_clock::now();
+
+  for (int f = 0; f < n_fills; ++f)
+    for (int b = 0; b < B; ++b) {
+      int64_t v = (int64_t)d->hist_len[b] - (int64_t)f * Ls;
+      v = v < 0 ? 0 : (v > Ls ? Ls : v);
+      d->valid_len_host[f * B + b] = (int32_t)v;
+    }
+  SS_CK(cudaEventRecord(r.ev_t0, r.copy_stream));
+  if (n_fills)
+    SS_CK(cudaMemcpyAsync(d->valid_len_dev, d->valid_len_host, sizeof(int32_t) * n_fills * B,
+                          cudaMemcpyHostToDevice, r.copy_stream));
+  if (!d->copy_only) SS_ST(ss_verify_begin(ctx, d->Q, B, d->T_q, d->scale, r.attn_stream));
+
+  int64_t h2d = 0;
+  int copies = 0, calls = 0;
+  const size_t esz = 2;
+  const int64_t head_elems = (int64_t)L_c * hd;          // one head row of a host block
+  const int64_t block_elems = 2 * (int64_t)H_kv * head_elems;
+  for (int f = 0; f < n_fills; ++f) {
+    const int buf = f & 1;
+    if (f >= 2) SS_CK(cudaStreamWaitEvent(r.copy_stream, r.ev_free[buf], 0));
+    for (int jj = 0; jj < bc; ++jj) {
+      const int j = f * bc + jj;
+      for (int b = 0; b < B; ++b) {
+        int64_t v = (int64_t)d->hist_len[b] - (int64_t)j * L_c;
+        if (v <= 0) continue;
+        if (v > L_c) v = L_c;
+        const uint16_t* src = (const uint16_t*)d->hist[b] + (int64_t)j * block_elems;
+        for (int kv = 0; kv < 2; ++kv) {
+          uint16_t* dst = (uint16_t*)(kv ? d->stage_v[buf] : d->stage_k[buf]) +
+                          ((int64_t)b * H_kv * Ls + (int64_t)jj * L_c) * hd;
+          const uint16_t* s = src + (int64_t)kv * H_kv * head_elems;
+          if (v == L_c && bc == 1) {
+            SS_CK(cudaMemcpyAsync(dst, s, (size_t)H_kv * head_elems * esz, cudaMemcpyHostToDevice,
+                                  r.copy_stream));
+          } else {
+            SS_CK(cudaMemcpy2DAsync(dst, (size_t)Ls * hd * esz, s, (size_t)head_elems * esz,
+                                    (size_t)v * hd * esz, H_kv, cudaMemcpyHostToDevice,
+                                    r.copy_stream));
+          }
+          h2d += (int64_t)H_kv * v * hd * esz;
+          ++copies;
+        }
+      }
+    }
+    SS_CK(cudaEventRecord(r.ev_ready[buf], r.copy_stream));
+    SS_CK(cudaStreamWaitEvent(r.attn_stream, r.ev_ready[buf], 0));
+    if (!d->copy_only) {
+      ss_tensor K = {d->stage_k[buf], (int64_t)H_kv * Ls * hd, Ls * hd, hd};
+      ss_tensor V = {d->stage_v[buf], (int64_t)H_kv * Ls * hd, Ls * hd, hd};
+      SS_ST(ss_verify_chunk(ctx, K, V, (int32_t)Ls, d->valid_len_dev + (int64_t)f * B,
+                            r.attn_stream));
+      ++calls;
+    }
+    SS_CK(cudaEventRecord(r.ev_free[buf], r.attn_stream));
+  }
+  if (n_fills == 0) {
+    // nothing to stream: the attention stream still has to follow the copy stream's start
+    SS_CK(cudaEventRecord(r.ev_ready[0], r.copy_stream));
+    SS_CK(cudaStreamWaitEvent(r.attn_stream, r.ev_ready[0], 0));
+  }
+  int64_t d2h = 0;
+  if (!d->copy_only) {
+    SS_ST(ss_verify_local(ctx, d->K_loc, d->V_loc, d->T_q, d->mask_kind, d->mask_bits,
+                          r.attn_stream));
+    SS_ST(ss_verify_finalize(ctx, d->O, d->LSE, r.attn_stream));
+    if (d->accept_idx) {
+      if (!d->accept_cnt || !d->zero_off || !d->commit_k || !d->commit_v) return SS_ERR_ARG;
+      const int64_t row = hd, tl = d->T_q;
+      ss_tensor Kd = {d->commit_k, (int64_t)H_kv * tl * row, tl * row, row};
+      ss_tensor Vd = {d->commit_v, (int64_t)H_kv * tl * row, tl * row, row};
+      SS_ST(ss_commit_gather(ctx, d->K_loc, d->V_loc, B, d->T_q, d->accept_idx, d->accept_cnt, Kd,
+                             Vd, d->T_q, d->zero_off, r.attn_stream));
+      const size_t bytes = (size_t)B * H_kv * tl * row * esz;
+      if (d->host_commit_k) {
+        SS_CK(cudaMemcpyAsync(d->host_commit_k, d->commit_k, bytes, cudaMemcpyDeviceToHost,
+                              r.attn_stream));
+        d2h += bytes;
+      }
+      if (d->host_commit_v) {
+        SS_CK(cudaMemcpyAsync(d->host_commit_v, d->commit_v, bytes, cudaMemcpyDeviceToHost,
+                              r.attn_stream));
+        d2h += bytes;
+      }
+    }
+    if (d->O_host) {
+      const size_t bytes = (size_t)B * H_q * d->T_q * hd * esz;
+      SS_CK(cudaMemcpyAsync(d->O_host, d->O, bytes, cudaMemcpyDeviceToHost, r.attn_stream));
+      d2h += bytes;
+    }
+    if (d->LSE_host && d->LSE) {
+      const size_t bytes = (size_t)B * H_q * d->T_q * sizeof(float);
+      SS_CK(cudaMemcpyAsync(d->LSE_host, d->LSE, bytes, cudaMemcpyDeviceToHost, r.attn_stream));
+      d2h += bytes;
+    }
+  }
+  SS_CK(cudaEventRecord(r.ev_t1, r.attn_stream));
+  SS_CK(cudaEventSynchronize(r.ev_t1));
+  SS_CK(cudaStreamSynchronize(r.copy_stream));
+  if (stats) {
+    float ms = 0.f;
+    SS_CK(cudaEventElapsedTime(&ms, r.ev_t0, r.ev_t1));
+    stats->ms_device = ms;
+    stats->ms_total = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - wall0)
+                          .count();
+    stats->h2d_bytes = h2d;
+    stats->d2h_bytes = d2h;
+    stats->chunk_calls = calls;
+    stats->copies = copies;
+  }
+  return SS_OK;
+}
+
+extern "C" ss_status ss_stream_round(ss_ctx* ctx, const ss_stream_desc* d, ss_stream_stats* stats) {
+  if (!ctx) return SS_ERR_ARG;
+  ss::ctx_pipeline_mode(ctx, true);
+  const ss_status st = stream_round_impl(ctx, d, stats);
+  ss::ctx_pipeline_mode(ctx, false);
+  return st;
+}

@@ -1,0 +1,206 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU oracle,
+element by element on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_33184_b200 import inputs
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def _ssb():
+    from paper_2609_33184_b200 import binding
+    return binding
+
+
+def _run(cfg, lens=None, flags=0, fill=None, order=None, local_at=None, strict=True, kernel=None,
+         max_chunks=0):
+    lens = inputs.history_lengths(cfg) if lens is None else lens
+    case = util.gen_case(cfg, lens, DEV, fill)
+    ctx = util.make_ctx(cfg, flags=flags, max_chunks=max_chunks)
+    O, LSE = util.gpu_case(ctx, cfg, *case, order=order, local_at=local_at)
+    st, bits = ctx.ss_poll_status()
+    assert st == 0 and bits == 0, (st, bits)
+    if kernel and case[1]:
+        assert ctx.last_chunk_kernel() == kernel
+    ref = util.oracle_case(cfg, lens, *case)
+    worst = util.compare(cfg, O, LSE, ref, strict=strict)
+    ctx.close()
+    return O, LSE, worst
+
+
+def test_c1_tiny_chain_exact_config():
+    cfg = inputs.CONFIGS["c1_tiny_chain"]
+    _run(cfg, kernel="simt")
+
+
+def _small(name, **kw):
+    return inputs.scaled(inputs.CONFIGS[name], **kw)
+
+
+def test_c2_shape_scaled_tensor_core_path():
+    cfg = _small("c2_qwen3_8b", B=2, H_q=8, H_kv=2, L_c=256, len_lo=1000, len_hi=1000)
+    _run(cfg, kernel="tcgen05")
+
+
+def test_c3_shape_scaled_ragged_nan_padding():
+    cfg = _small("c3_internlm25_7b_ragged", B=3, H_q=8, H_kv=2, L_c=256, len_lo=65, len_hi=700)
+    _run(cfg, kernel="tcgen05")  # padding past valid_len is NaN by default
+
+
+def test_c4_shape_scaled_tree():
+    cfg = _small("c4_tree", B=2, H_q=10, H_kv=2, L_c=256, len_lo=600, len_hi=600)
+    _run(cfg, kernel="tcgen05")
+
+
+@pytest.mark.parametrize("flags", [0, 1])
+@pytest.mark.parametrize("n", [0, 1, 15, 16, 17, 63, 64, 65, 127, 129, 255, 256, 257])
+def test_short_histories(flags, n):
+    # short histories give the masks and the local segment real weight
+    cfg = _small("c2_qwen3_8b", B=2, H_q=8, H_kv=2, L_c=128, len_lo=n, len_hi=n, k_mult=1.0)
+    _run(cfg, flags=flags)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("G", [1, 4, 5, 8])
+@pytest.mark.parametrize("mask", ["chain", "tree"])
+def test_group_sizes_and_head_dims(d, G, mask):
+    cfg = inputs.VerifyConfig("v", 0x77 + G + d, 2, 2 * G, 2, d, 96, 7, 40, 300, mask=mask, k_mult=2.0)
+    _run(cfg)
+
+
+@pytest.mark.parametrize("T_q", [1, 2, 3, 5, 9, 16, 33])
+def test_query_counts_odd_rows(T_q):
+    cfg = inputs.VerifyConfig("v", 0x99 + T_q, 2, 8, 2, 128, 128, T_q, 100, 400, k_mult=2.0)
+    _run(cfg, kernel="tcgen05")
+
+
+@pytest.mark.parametrize("k_mult", [4.0, 8.0])
+@pytest.mark.parametrize("flags", [0, 1])
+def test_peaked_softmax(k_mult, flags):
+    cfg = inputs.VerifyConfig("v", 0x1234, 2, 8, 2, 128, 192, 8, 50, 700, k_mult=k_mult)
+    _run(cfg, flags=flags)
+
+
+def test_needle_keys_and_rescale_path():
+    # one key per request with a score ~ +20 above the rest, placed late in the history, so the
+    # running maximum jumps by more than the rescale threshold after many tiles
+    cfg = inputs.VerifyConfig("v", 0x4321, 2, 8, 2, 128, 256, 8, 900, 900)
+    lens = [900, 900]
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    for b, (j, t) in enumerate([(3, 100), (2, 255)]):
+        K = chunks[j][0]
+        for h in range(cfg.H_kv):
+            q = Q[b, h * cfg.G].float().mean(0)
+            K[b, h, t] = (q / q.norm() * 30.0).to(torch.bfloat16)
+    # and one needle in the local segment
+    K_loc[0, 0, 2] = (Q[0, 0, 5].float() / Q[0, 0, 5].float().norm() * 25.0).to(torch.bfloat16)
+    for flags in (0, 1):
+        ctx = util.make_ctx(cfg, flags=flags)
+        O, LSE = util.gpu_case(ctx, cfg, Q, chunks, K_loc, V_loc, bits)
+        ref = util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits)
+        util.compare(cfg, O, LSE, ref)
+        ctx.close()
+
+
+def test_empty_chunks_reverse_order_local_first():
+    cfg = inputs.VerifyConfig("v", 0x55, 3, 8, 2, 128, 128, 6, 0, 600)
+    lens = [600, 0, 130]
+    n = inputs.num_chunks(cfg, lens)
+    O1, L1, _ = _run(cfg, lens=lens)
+    O2, L2, _ = _run(cfg, lens=lens, order=list(range(n))[::-1], local_at=0)
+    assert (O1.float() - O2.float()).abs().max() < 2e-2
+    assert (L1 - L2).abs().max() < 1e-4
+
+
+def test_more_chunk_calls_than_partial_sets_folds():
+    cfg = inputs.VerifyConfig("v", 0x56, 2, 8, 2, 128, 64, 5, 500, 700)
+    _run(cfg, max_chunks=3)
+
+
+@pytest.mark.parametrize("flags", [0, 1])
+def test_deterministic_bitwise(flags):
+    cfg = inputs.VerifyConfig("v", 0x57, 2, 8, 2, 128, 256, 8, 300, 900)
+    lens = inputs.history_lengths(cfg)
+    case = util.gen_case(cfg, lens, DEV)
+    ctx = util.make_ctx(cfg, flags=flags)
+    O1, L1 = util.gpu_case(ctx, cfg, *case)
+    O1, L1 = O1.clone(), L1.clone()
+    O2, L2 = util.gpu_case(ctx, cfg, *case)
+    assert torch.equal(O1.view(torch.int16), O2.view(torch.int16)) and torch.equal(L1, L2)
+    ctx.close()
+
+
+def test_simt_and_tensor_core_kernels_agree():
+    cfg = inputs.VerifyConfig("v", 0x58, 2, 16, 4, 128, 320, 8, 100, 1200, k_mult=2.0)
+    lens = inputs.history_lengths(cfg)
+    case = util.gen_case(cfg, lens, DEV)
+    outs = []
+    for flags in (0, 1):
+        ctx = util.make_ctx(cfg, flags=flags)
+        O, L = util.gpu_case(ctx, cfg, *case)
+        assert ctx.last_chunk_kernel() == ("simt" if flags else "tcgen05")
+        outs.append((O.float(), L))
+        ctx.close()
+    assert (outs[0][0] - outs[1][0]).abs().max() < 2e-2
+    assert (outs[0][1] - outs[1][1]).abs().max() < 1e-4
+
+
+def test_overlap_flag_same_result():
+    ssb = _ssb()
+    cfg = inputs.VerifyConfig("v", 0x59, 4, 16, 4, 128, 512, 8, 1500, 2500)
+    lens = inputs.history_lengths(cfg)
+    case = util.gen_case(cfg, lens, DEV)
+    torch.cuda.synchronize()
+    res = []
+    for flags in (0, ssb.SS_FLAG_OVERLAP_CHUNKS):
+        ctx = util.make_ctx(cfg, flags=flags)
+        for _ in range(3):
+            O, L = util.gpu_case(ctx, cfg, *case)
+        res.append((O.clone(), L.clone()))
+        st, bits = ctx.ss_poll_status()
+        assert st == 0
+        ctx.close()
+    assert torch.equal(res[0][0].view(torch.int16), res[1][0].view(torch.int16))
+    assert torch.equal(res[0][1], res[1][1])
+    ref = util.oracle_case(cfg, lens, *case, groups=[(0, 0), (3, 3)])
+    util.compare(cfg, res[1][0], res[1][1], ref)
+
+
+def test_strided_inputs():
+    # K/V chunks that are views into a larger buffer (token stride > d, head stride padded)
+    cfg = inputs.VerifyConfig("v", 0x5A, 2, 8, 2, 128, 128, 4, 128, 128)
+    lens = [128, 128]
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    K, V, vl = chunks[0]
+    big_k = torch.full((2, 2, 160, 256), float("nan"), dtype=torch.bfloat16, device=DEV)
+    big_v = torch.full_like(big_k, float("nan"))
+    big_k[:, :, 16:144, 128:] = K
+    big_v[:, :, 16:144, :128] = V
+    Kv, Vv = big_k[:, :, 16:144, 128:], big_v[:, :, 16:144, :128]
+    for flags in (0, 1):
+        ctx = util.make_ctx(cfg, flags=flags)
+        O, L = util.gpu_case(ctx, cfg, Q, [(Kv, Vv, vl)], K_loc, V_loc, bits)
+        ref = util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits)
+        util.compare(cfg, O, L, ref)
+        ctx.close()
+
+
+def test_bad_valid_len_sets_status_and_is_clamped():
+    ssb = _ssb()
+    cfg = inputs.VerifyConfig("v", 0x5B, 2, 8, 2, 128, 128, 4, 128, 128)
+    lens = [128, 128]
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    K, V, vl = chunks[0]
+    bad = torch.tensor([500, -3], dtype=torch.int32, device=DEV)
+    ctx = util.make_ctx(cfg)
+    util.gpu_case(ctx, cfg, Q, [(K, V, bad)], K_loc, V_loc, bits)
+    st, b = ctx.ss_poll_status()
+    assert st == ssb.SS_ERR_DEVICE_FLAG and b & ssb.SS_DEV_BAD_VALID_LEN
+    st, b = ctx.ss_poll_status()
+    assert st == 0 and b == 0  # cleared
+    ctx.close()
