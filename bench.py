@@ -1,0 +1,436 @@
+"""Benchmark of the streamed-KV verification-attention hot path on B200.
+
+A step is one verification round of one layer over one batch: begin -> one chunk call per
+history chunk -> local candidate segment -> finalize.  The headline `value` is verify-attention
+KV GB/s (committed-history K/V bytes read per round / round time) with the history resident in
+HBM; `e2e` is the same metric through ss_stream_round with the history in pinned HOST memory
+(host->device copies and the device->host read of the result inside the timed region).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2_qwen3_8b] [--impl reference]
+
+Prints ONE JSON line on stdout.  With --gpus N > 1 (under torchrun) every rank runs the same
+per-GPU workload on its own requests (the path shards by request, no data-path collective).
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes as C
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2609_33184_b200 import inputs  # noqa: E402
+
+METRIC = "verify_attention_kv_GBps"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# DRAM bytes (read + write) per chunk-kernel launch from an ncu capture of the same kernel;
+# filled from the summaries under profiles/ (None until a capture exists for the workload).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons while the GPU is under load."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.samples = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, t0: float, t1: float):
+        sm, mx, reasons = [], [], set()
+        for t, line in self.samples:
+            if not (t0 <= t <= t1):
+                continue
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                "sw_power_cap"), f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def kv_bytes(cfg, lens):
+    return sum(lens) * cfg.H_kv * cfg.d * 2 * 2
+
+
+def build_resident(cfg, lens, dev):
+    """History as distinct per-chunk device buffers + the round's other tensors."""
+    Q = inputs.make_q(cfg, dev)
+    K_loc, V_loc = inputs.make_local(cfg, dev)
+    bits = inputs.make_mask_bits(cfg, dev)
+    chunks = [inputs.make_history_chunk(cfg, j, lens, dev, fill=0.0)
+              for j in range(inputs.num_chunks(cfg, lens))]
+    return Q, chunks, K_loc, V_loc, bits
+
+
+def run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, ev_pair=None):
+    kind = ssb.SS_MASK_TREE_BITS if cfg.mask == "tree" else ssb.SS_MASK_CHAIN
+    ctx.ss_verify_begin(Q, cfg.scale)
+    if ev_pair:
+        ev_pair[0].record()
+    for K, V, vl in chunks:
+        ctx.ss_verify_chunk(K, V, vl)
+    if ev_pair:
+        ev_pair[1].record()
+    ctx.ss_verify_local(K_loc, V_loc, kind, bits if cfg.mask == "tree" else None)
+    ctx.ss_verify_finalize(O, LSE)
+
+
+def cpu_baseline(cfg, lens, Q, chunks, K_loc, V_loc, bits, budget_s=15.0, max_groups=64):
+    """The oracle, as it stands, timed on this machine's host cores on a bounded sample of the
+    same workload: whole (request, kv-head) groups until about `budget_s` seconds are spent."""
+    from tests import util
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    groups = [(b, h) for b in range(cfg.B) for h in range(cfg.H_kv)]
+    done, t0, nbytes = 0, time.perf_counter(), 0
+    for g in groups[:max_groups]:
+        util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits, groups=[g])
+        done += 1
+        nbytes += lens[g[0]] * cfg.d * 2 * 2
+        if time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    return {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{done} of {len(groups)} (request, kv-head) groups of {cfg.name}, all "
+                      f"{cfg.G * cfg.T_q} query rows each, {dt:.1f} s",
+            "rounds_per_s": nbytes / dt / kv_bytes(cfg, lens)}
+
+
+def pinned_history(cfg, lens, chunks):
+    """Host layout of ss_stream_round: per request, per chunk, [2][H_kv][L_c][d] bf16, pinned."""
+    J = len(chunks)
+    host = torch.empty(cfg.B, J, 2, cfg.H_kv, cfg.L_c, cfg.d, dtype=torch.bfloat16).pin_memory()
+    for j, (K, V, _) in enumerate(chunks):
+        host[:, j, 0].copy_(K)
+        host[:, j, 1].copy_(V)
+    torch.cuda.synchronize()
+    return host
+
+
+def make_stream_desc(ssb, cfg, lens, host, dev, Q, K_loc, V_loc, bits, O, LSE, bufs, batch_chunks=1,
+                     accept=None, copy_only=0):
+    d = ssb.ss_stream_desc()
+    d.B, d.T_q, d.L_c, d.scale = cfg.B, cfg.T_q, cfg.L_c, cfg.scale
+    ptrs = (C.c_void_p * cfg.B)(*[host[b].data_ptr() for b in range(cfg.B)])
+    hl = (C.c_int32 * cfg.B)(*lens)
+    d.hist = C.cast(ptrs, C.POINTER(C.c_void_p))
+    d.hist_len = C.cast(hl, C.POINTER(C.c_int32))
+    d.batch_chunks = batch_chunks
+    for s in range(2):
+        d.stage_k[s] = bufs["stage_k"][s].data_ptr()
+        d.stage_v[s] = bufs["stage_v"][s].data_ptr()
+    d.scratch_fills = bufs["fills"]
+    d.valid_len_host = bufs["vl_host"].data_ptr()
+    d.valid_len_dev = bufs["vl_dev"].data_ptr()
+    d.Q, d.K_loc, d.V_loc = ssb.as_ss_tensor(Q), ssb.as_ss_tensor(K_loc), ssb.as_ss_tensor(V_loc)
+    d.mask_kind = ssb.SS_MASK_TREE_BITS if cfg.mask == "tree" else ssb.SS_MASK_CHAIN
+    d.mask_bits = bits.data_ptr() if cfg.mask == "tree" else None
+    d.O, d.LSE = O.data_ptr(), LSE.data_ptr()
+    if accept is not None:
+        d.accept_idx, d.accept_cnt = accept["idx"].data_ptr(), accept["cnt"].data_ptr()
+        d.zero_off = accept["zero"].data_ptr()
+        d.commit_k, d.commit_v = accept["ck"].data_ptr(), accept["cv"].data_ptr()
+        d.host_commit_k, d.host_commit_v = accept["hk"].data_ptr(), accept["hv"].data_ptr()
+    d.O_host, d.LSE_host = bufs["O_host"].data_ptr(), bufs["LSE_host"].data_ptr()
+    d.copy_only = copy_only
+    d._keep = (ptrs, hl)  # keep the ctypes arrays alive
+    return d
+
+
+def stream_buffers(cfg, dev, n_chunks, batch_chunks=1):
+    Ls = cfg.L_c * batch_chunks
+    fills = (n_chunks + batch_chunks - 1) // batch_chunks + 1
+    return {
+        "stage_k": [torch.zeros(cfg.B, cfg.H_kv, Ls, cfg.d, dtype=torch.bfloat16, device=dev) for _ in range(2)],
+        "stage_v": [torch.zeros(cfg.B, cfg.H_kv, Ls, cfg.d, dtype=torch.bfloat16, device=dev) for _ in range(2)],
+        "fills": fills,
+        "vl_host": torch.zeros(fills * cfg.B, dtype=torch.int32).pin_memory(),
+        "vl_dev": torch.zeros(fills * cfg.B, dtype=torch.int32, device=dev),
+        "O_host": torch.zeros(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16).pin_memory(),
+        "LSE_host": torch.zeros(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32).pin_memory(),
+    }
+
+
+def run_reference(args, cfg, rank):
+    """--impl reference: the CPU oracle, as it stands, on a bounded sample per step."""
+    if rank != 0:
+        return
+    lens = inputs.history_lengths(cfg)
+    # a sample of 2 (request, kv-head) groups per step keeps the whole run within minutes
+    small = inputs.scaled(cfg, B=1, H_kv=2, H_q=2 * cfg.G)
+    lens1 = lens[:1]
+    Q, chunks, K_loc, V_loc, bits = build_resident(small, lens1, "cpu")
+    from tests import util
+    times = []
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        util.oracle_case(small, lens1, Q, chunks, K_loc, V_loc, bits)
+        if i >= args.warmup:
+            times.append(time.perf_counter() - t0)
+    dt = sum(times) / len(times)
+    val = kv_bytes(small, lens1) / dt / 1e9
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    sample = f"per step: 2 (request, kv-head) groups of {cfg.name} ({lens1[0]} tokens, {cfg.G * cfg.T_q} rows each)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2_qwen3_8b", choices=sorted(inputs.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true", help="plain launches (no programmatic dependent launch)")
+    ap.add_argument("--simt", action="store_true", help="force the CUDA-core chunk kernel")
+    ap.add_argument("--history-tokens", type=int, default=0,
+                    help="shrink every request's history to this many tokens (small cases for profiler captures)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    cfg = inputs.CONFIGS[args.workload]
+    if args.history_tokens:
+        cfg = inputs.scaled(cfg, len_lo=args.history_tokens, len_hi=args.history_tokens)
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, cfg, rank)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    from paper_2609_33184_b200 import binding as ssb
+    from paper_2609_33184_b200 import build as ssbuild
+    ssbuild.build()
+
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    # per-rank requests: same shapes, rank-specific seed (weak scaling, sharded by request)
+    if rank:
+        cfg = inputs.scaled(cfg, seed=cfg.seed + 0x100 * rank)
+    lens = inputs.history_lengths(cfg)
+    Q, chunks, K_loc, V_loc, bits = build_resident(cfg, lens, dev)
+    flags = 0 if args.no_overlap else ssb.SS_FLAG_OVERLAP_CHUNKS
+    if args.simt:
+        flags |= ssb.SS_FLAG_FORCE_SIMT
+    ctx = ssb.Context(cfg.B, cfg.H_q, cfg.H_kv, cfg.d, cfg.T_q, cfg.T_q, cfg.L_c, max_chunks=len(chunks) or 1,
+                      device=local_rank, flags=flags)
+    O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=dev)
+    LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=dev)
+    nbytes = kv_bytes(cfg, lens)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+
+    for _ in range(args.warmup):
+        run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE)
+    barrier()
+    # ---- timed region: exactly K rounds, history resident in HBM -----------------------------
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = ctx.launch_count()
+    t_wall0 = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE)
+    e1.record()
+    barrier()
+    t_wall1 = time.time()
+    launches = ctx.launch_count() - launches0
+    ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * nbytes / (ms_per_step * 1e-3) / 1e9
+    st, dev_bits = ctx.ss_poll_status()
+    if st != 0:
+        raise SystemExit(f"device status word set: {dev_bits}")
+
+    # clocks: sampled during the timed region; if it was too short for 3 samples, identical
+    # untimed rounds are run for about a second to collect them
+    clocks = None
+    if rank == 0:
+        clocks = sampler.summary(t_wall0, t_wall1)
+        clocks["sampled"] = "timed region"
+        if clocks["samples"] < 3:
+            t0 = time.time()
+            while time.time() - t0 < 1.2:
+                for _ in range(20):
+                    run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE)
+                torch.cuda.synchronize()
+            clocks = sampler.summary(t0, time.time())
+            clocks["sampled"] = "identical rounds run right after the timed region (it was too short)"
+
+    # ---- dominant kernel: chunk attention, per-launch time over the same rounds --------------
+    n_chunk_calls = len(chunks)
+    chunk_ms = None
+    if n_chunk_calls:
+        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                 for _ in range(min(args.steps, 50))]
+        for p in pairs:
+            run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, ev_pair=p)
+        torch.cuda.synchronize()
+        chunk_ms = statistics.mean(a.elapsed_time(b) for a, b in pairs) / n_chunk_calls
+    peak, peak_kind = peaks()
+    alg_bytes_per_launch = nbytes / max(n_chunk_calls, 1)
+    achieved = alg_bytes_per_launch / (chunk_ms * 1e-3) / 1e9 if chunk_ms else None
+    roofline = {"bound": "hbm", "kernel": f"chunk attention ({ctx.last_chunk_kernel()})",
+                "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                "frac": (achieved / peak) if achieved else None,
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(cfg.name),
+                "algorithmic_bytes_per_launch": alg_bytes_per_launch,
+                "us_per_launch": chunk_ms * 1e3 if chunk_ms else None}
+
+    # ---- end to end: history in pinned host memory, streamed through ss_stream_round ---------
+    e2e = None
+    if not args.no_e2e and n_chunk_calls:
+        host = pinned_history(cfg, lens, chunks)
+        bufs = stream_buffers(cfg, dev, n_chunk_calls)
+        Qh, Klh, Vlh = Q.cpu().pin_memory(), K_loc.cpu().pin_memory(), V_loc.cpu().pin_memory()
+        Qd, Kld, Vld = torch.empty_like(Q), torch.empty_like(K_loc), torch.empty_like(V_loc)
+        desc = make_stream_desc(ssb, cfg, lens, host, dev, Qd, Kld, Vld, bits, O, LSE, bufs)
+        n_e2e = max(3, min(args.steps, 10))
+        times = []
+        for i in range(2 + n_e2e):
+            barrier()
+            t0 = time.perf_counter()
+            Qd.copy_(Qh, non_blocking=True)
+            Kld.copy_(Klh, non_blocking=True)
+            Vld.copy_(Vlh, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+            stats = ctx.ss_stream_round(desc)  # returns after the D2H of O and LSE
+            dt = time.perf_counter() - t0
+            if i >= 2:
+                times.append(dt)
+        if dist is not None:
+            t = torch.tensor([statistics.mean(times)], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        else:
+            dt = statistics.mean(times)
+        small_in = (Qh.numel() + Klh.numel() + Vlh.numel()) * 2
+        e2e = {"value": world * nbytes / dt / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": int(stats.h2d_bytes + small_in),
+               "d2h_bytes_per_step": int(stats.d2h_bytes), "ms_per_step": dt * 1e3,
+               "api": "ss_stream_round (pinned host history, 2 staging buffers)"}
+        del host
+
+    cpu = None
+    if rank == 0:
+        sampler.stop()
+        if not args.no_cpu_baseline:
+            cpu = cpu_baseline(cfg, lens, Q, chunks, K_loc, V_loc, bits)
+
+    if rank == 0:
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg.name, "B": cfg.B, "H_q": cfg.H_q, "H_kv": cfg.H_kv, "d": cfg.d,
+                       "T_q": cfg.T_q, "L_c": cfg.L_c, "history_tokens": lens if len(set(lens)) > 1 else lens[0],
+                       "chunk_calls_per_round": n_chunk_calls, "mask": cfg.mask,
+                       "kv_bytes_per_round": nbytes,
+                       "l2": "inputs larger than L2 (each round streams all history chunks, "
+                             f"{nbytes / 2**20:.0f} MiB, through distinct buffers)",
+                       "overlap_chunks": not args.no_overlap},
+            "rounds_per_s": world * 1e3 / ms_per_step,
+            "pct_hbm_nominal_8TBps": 100.0 * value / world / 8000.0,
+            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            "roofline": roofline, "cpu_baseline": cpu,
+        }
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

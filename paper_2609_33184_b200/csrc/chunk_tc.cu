@@ -5,12 +5,19 @@
 // the kv-head (T_q candidate queries x G query heads) ride in the M dimension of the MMAs,
 // so every K/V byte is fetched from HBM once and serves the whole query group.
 //
-//   warp 4 (one lane)  TMA producer: K tile and V tile of 64 tokens per stage, 2 stages,
+//   warp 4 (one lane)  TMA producer: K tile and V tile of 64 tokens per stage, 3 stages,
 //                      128-byte swizzle, evict-first L2 policy (the history is streamed).
-//   warp 5 (one lane)  MMA issuer:   S = Q K^T   (M=128, N=64,  K=d=128: 8 x k16, smem x smem)
+//                      A K tile is released as soon as its score MMAs retire, a V tile
+//                      after its output MMAs.
+//   warp 5 (one lane)  MMA issuer:   S = Q K^T   (M=128, N=64,  K=d=128: 8 x k16, tmem x smem)
 //                                    O += P V    (M=128, N=128, K=64:    4 x k16, tmem x smem)
-//   warps 0-3          softmax: each thread owns one TMEM lane (= one MMA row): reads its
-//                      scores, keeps (m, l) in registers, writes P as packed bf16 to TMEM.
+//   warps 0-3          softmax: each thread owns one TMEM lane (= one MMA row): loads its
+//                      Q row into tensor memory once, then per tile reads its scores, keeps
+//                      (m, l) in registers and writes P as packed bf16 over the score columns.
+//
+// Tensor memory (256 columns): [0,64) S (fp32) with P (bf16 pairs) over [0,32); [64,128) Q
+// (bf16 pairs); [128,256) O (fp32).  Shared memory holds nothing but K/V tiles, so three
+// stages (96 KB) fit twice per SM and about 128 KB per SM are in flight from HBM.
 //
 // When the row tile has <= 32 (<= 64) rows the Q rows are replicated 4x (2x) along M and
 // each replica takes a quarter (half) of the tile's keys: lane L holds row L % R_pad and
@@ -19,8 +26,8 @@
 //
 // Running maximum: a row's reference maximum m only moves when the tile maximum exceeds it
 // by more than 8 (base-2 domain), which keeps exp2(s - m) <= 256 and makes the rescale of O
-// in tensor memory rare.  Two CTAs fit per SM (about 100 KB shared memory, 256 TMEM
-// columns each), so one CTA's ramp-up and tail overlap the other's steady state.
+// in tensor memory rare.  Two CTAs fit per SM, so one CTA's ramp-up and tail overlap the
+// other's steady state.
 //
 // Every wait on an mbarrier is bounded; on expiry the CTA raises SS_DEV_WAIT_EXPIRED, lets
 // its own copies land (bounded), frees its tensor memory and returns.
@@ -30,22 +37,21 @@ namespace ss {
 namespace {
 
 constexpr int kThreads = 192;
-constexpr int kStages = 2;
+constexpr int kStages = 3;
 constexpr int kD = 128;
-constexpr int kQBytes = 128 * kD * 2;               // 32 KB: two 64-column halves of 128 rows
 constexpr int kHalfTile = kTileKeys * 64 * 2;       // 8 KB: [64 keys][64 d] bf16
 constexpr int kTileBytes = 2 * kHalfTile;           // 16 KB: one K tile or one V tile
 constexpr int kStageBytes = 2 * kTileBytes;         // K then V
-constexpr int kSmemData = kQBytes + kStages * kStageBytes;  // 96 KB
+constexpr int kSmemData = kStages * kStageBytes;            // 96 KB
 constexpr int kSmemCtl = 2048;
 constexpr int kSmemTotal = kSmemData + kSmemCtl + 1024;     // + alignment slack
 constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColS = 0, kColP = 64, kColO = 128;
+constexpr uint32_t kColS = 0, kColP = 0, kColQ = 64, kColO = 128;
 constexpr float kRescaleThreshold = 8.f;
 constexpr unsigned long long kWaitNs = 2000000000ull;       // 2 s
 
 struct Ctl {
-  uint64_t kfull[kStages], vfull[kStages], empty[kStages];
+  uint64_t kfull[kStages], vfull[kStages], kempty[kStages], vempty[kStages];
   uint64_t sfull, pready, pvdone;
   uint32_t tmem_base;
   volatile uint32_t abort;
@@ -178,7 +184,7 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
       "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
-__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr),
       "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
@@ -203,12 +209,26 @@ __host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool b_mn_major)
          ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+// P (bf16 pairs) over the 32 leading score columns in 4 blocks of 8: blocks
+// [FIRST, FIRST + NC/16) hold this lane's keys, the others are zero.
+template <int NC, int FIRST>
+__device__ __forceinline__ void store_p(uint32_t t_s, const uint32_t (&pk)[NC / 16][8]) {
+  const uint32_t zero[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    if (q >= FIRST && q < FIRST + NC / 16)
+      tmem_st8(t_s + q * 8, pk[(q >= FIRST && q < FIRST + NC / 16) ? q - FIRST : 0]);
+    else
+      tmem_st8(t_s + q * 8, zero);
+  }
+}
+
 // ---- softmax of one tile for one TMEM lane --------------------------------------------------
-// NC = number of key columns this lane owns in a 64-key tile.
+// NC = number of key columns this lane owns in a 64-key tile.  P (bf16 pairs) is written
+// over the first 32 score columns: this lane's keys at [c0/2, c0/2 + NC/2), zeros elsewhere.
 template <int NC>
-__device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_p, uint32_t t_o, int c0,
-                                             int n_valid, bool have_o, float scale_log2, float& m,
-                                             float& l) {
+__device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_o, int c0, int n_valid,
+                                             bool have_o, float scale_log2, float& m, float& l) {
   uint32_t raw[NC / 16][16];
 #pragma unroll
   for (int q = 0; q < NC / 16; ++q) tmem_ld16(t_s + c0 + q * 16, raw[q]);
@@ -242,18 +262,30 @@ __device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_p, uint32_
     }
   }
   const float m_use = (m == -INFINITY) ? 0.f : m;
-  uint32_t pk[NC / 2];
+  uint32_t pk[NC / 16][8];
   float sum = 0.f;
 #pragma unroll
   for (int c = 0; c < NC; c += 2) {
     const float p0 = exp2f(s[c] - m_use), p1 = exp2f(s[c + 1] - m_use);
     sum += p0 + p1;
     __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);  // low half = even key
-    pk[c / 2] = *reinterpret_cast<uint32_t*>(&h);
+    pk[c / 16][(c / 2) % 8] = *reinterpret_cast<uint32_t*>(&h);
   }
   l += sum;
-#pragma unroll
-  for (int q = 0; q < NC / 16; ++q) tmem_st8(t_p + c0 / 2 + q * 8, &pk[q * 8]);
+  // c0 is uniform across a warp; dispatching on it keeps pk[] in registers
+  if (NC == 64) {
+    store_p<NC, 0>(t_s, pk);
+  } else if (NC == 32) {
+    if (c0 == 0) store_p<NC, 0>(t_s, pk);
+    else store_p<NC, 2>(t_s, pk);
+  } else {
+    switch (c0 / 16) {
+      case 0: store_p<NC, 0>(t_s, pk); break;
+      case 1: store_p<NC, 1>(t_s, pk); break;
+      case 2: store_p<NC, 2>(t_s, pk); break;
+      default: store_p<NC, 3>(t_s, pk); break;
+    }
+  }
   tc_wait_st();
 }
 
@@ -262,8 +294,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* q_s = smem;
-  uint8_t* st_s = smem + kQBytes;
+  uint8_t* st_s = smem;
   Ctl* ctl = reinterpret_cast<Ctl*>(smem + kSmemData);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -299,12 +330,13 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     return;
   }
 
-  // ---- set-up: barriers, tensor memory, Q rows -> swizzled shared memory ------------------
+  // ---- set-up: barriers, tensor memory -------------------------------------------------------
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&ctl->kfull[s], 1);
       mbar_init(&ctl->vfull[s], 1);
-      mbar_init(&ctl->empty[s], 1);
+      mbar_init(&ctl->kempty[s], 1);
+      mbar_init(&ctl->vempty[s], 1);
     }
     mbar_init(&ctl->sfull, 1);
     mbar_init(&ctl->pready, 128);
@@ -319,20 +351,6 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  // Q: lane L of the MMA's M dimension holds row (L % r_pad) of this row tile (zero if padding).
-  for (int i = tid; i < 128 * (kD / 8); i += kThreads) {
-    const int L = i / (kD / 8), c8 = i % (kD / 8);
-    const int r = L % r_pad;
-    uint4 raw = make_uint4(0, 0, 0, 0);
-    if (r < nrows) {
-      const int rg = row0 + r, g = rg / p.T_q, t = rg % p.T_q;
-      raw = *reinterpret_cast<const uint4*>(p.Q + b * p.q_sb +
-                                            (int64_t)(kvh * p.G + g) * p.q_sh + t * p.q_st + c8 * 8);
-    }
-    const int half = c8 >> 3, j = c8 & 7;
-    *reinterpret_cast<uint4*>(q_s + half * (128 * 128) + L * 128 + ((j ^ (L & 7)) << 4)) = raw;
-  }
-  fence_proxy_async();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -342,31 +360,35 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     // ===== TMA producer =====
     if (lane == 0) {
       const uint64_t pol = l2_evict_first_policy();
-      int issued = 0;
+      int issued_k = 0, issued_v = 0;
       for (int it = 0; it < n_tiles; ++it) {
         const int s = it % kStages;
         const uint32_t ph = (it / kStages) & 1;
-        if (!mbar_wait(&ctl->empty[s], ph ^ 1, ctl, p.status)) break;
         const int tok = tok0 + it * kTileKeys;
         const uint32_t kdst = smem_u32(st_s + s * kStageBytes);
         const uint32_t vdst = kdst + kTileBytes;
+        if (!mbar_wait(&ctl->kempty[s], ph ^ 1, ctl, p.status)) break;
         mbar_expect_tx(&ctl->kfull[s], kTileBytes);
         tma_load_4d(kdst, &tmK, 0, tok, kvh, b, &ctl->kfull[s], pol);
         tma_load_4d(kdst + kHalfTile, &tmK, 64, tok, kvh, b, &ctl->kfull[s], pol);
+        issued_k = it + 1;
+        if (!mbar_wait(&ctl->vempty[s], ph ^ 1, ctl, p.status)) break;
         mbar_expect_tx(&ctl->vfull[s], kTileBytes);
         tma_load_4d(vdst, &tmV, 0, tok, kvh, b, &ctl->vfull[s], pol);
         tma_load_4d(vdst + kHalfTile, &tmV, 64, tok, kvh, b, &ctl->vfull[s], pol);
-        issued = it + 1;
+        issued_v = it + 1;
       }
       if (ctl->abort) {
         // let the copies this thread started land before the CTA leaves (bounded)
-        for (int it = max(0, issued - kStages); it < issued; ++it) {
+        const unsigned long long t0 = gtime_ns();
+        for (int it = max(0, issued_k - kStages); it < issued_k; ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1;
-          const unsigned long long t0 = gtime_ns();
-          while (!(mbar_try_wait(&ctl->kfull[s], ph) && mbar_try_wait(&ctl->vfull[s], ph)) &&
-                 gtime_ns() - t0 < kWaitNs) {
+          while (!mbar_try_wait(&ctl->kfull[s], ph) && gtime_ns() - t0 < kWaitNs) {
           }
+          if (it < issued_v)
+            while (!mbar_try_wait(&ctl->vfull[s], ph) && gtime_ns() - t0 < kWaitNs) {
+            }
         }
       }
     }
@@ -375,24 +397,24 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     if (lane == 0) {
       constexpr uint32_t idesc_qk = make_idesc(128, kTileKeys, false);
       constexpr uint32_t idesc_pv = make_idesc(128, kD, true);
-      const uint32_t q_addr = smem_u32(q_s);
-      bool ok = mbar_wait(&ctl->kfull[0], 0, ctl, p.status);
+      // Q is in tensor memory once the softmax warps have arrived on pready (phase 0)
+      bool ok = mbar_wait(&ctl->pready, 0, ctl, p.status) &&
+                mbar_wait(&ctl->kfull[0], 0, ctl, p.status);
       if (ok) {
         tc_fence_after();
         const uint32_t k_addr = smem_u32(st_s);
 #pragma unroll
         for (int kk = 0; kk < kD / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * (128 * 128) + (kk & 3) * 32;
           const uint32_t koff = (kk >> 2) * kHalfTile + (kk & 3) * 32;
-          mma_ss(tmem + kColS, desc_kmajor(q_addr + off), desc_kmajor(k_addr + koff), idesc_qk,
-                 kk > 0);
+          mma_ts(tmem + kColS, tmem + kColQ + kk * 8, desc_kmajor(k_addr + koff), idesc_qk, kk > 0);
         }
+        tc_commit(&ctl->kempty[0]);
         tc_commit(&ctl->sfull);
       }
       for (int it = 0; ok && it < n_tiles; ++it) {
         const int s = it % kStages;
         const uint32_t ph = (it / kStages) & 1;
-        ok = mbar_wait(&ctl->pready, it & 1, ctl, p.status) &&
+        ok = mbar_wait(&ctl->pready, (it + 1) & 1, ctl, p.status) &&
              mbar_wait(&ctl->vfull[s], ph, ctl, p.status);
         if (!ok) break;
         tc_fence_after();
@@ -402,7 +424,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
           mma_ts(tmem + kColO, tmem + kColP + kk * 8, desc_mnmajor(v_addr + kk * 2048, kHalfTile),
                  idesc_pv, (it > 0 || kk > 0));
         }
-        tc_commit(&ctl->empty[s]);
+        tc_commit(&ctl->vempty[s]);
         if (it + 1 < n_tiles) {
           const int s2 = (it + 1) % kStages;
           const uint32_t ph2 = ((it + 1) / kStages) & 1;
@@ -410,13 +432,15 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
           if (!ok) break;
           tc_fence_after();
           const uint32_t k_addr = smem_u32(st_s + s2 * kStageBytes);
+          // overwrites the S/P columns: the tensor pipe runs this thread's MMAs in issue
+          // order, so the P V products above have consumed P before these write S
 #pragma unroll
           for (int kk = 0; kk < kD / 16; ++kk) {
-            const uint32_t off = (kk >> 2) * (128 * 128) + (kk & 3) * 32;
             const uint32_t koff = (kk >> 2) * kHalfTile + (kk & 3) * 32;
-            mma_ss(tmem + kColS, desc_kmajor(q_addr + off), desc_kmajor(k_addr + koff), idesc_qk,
+            mma_ts(tmem + kColS, tmem + kColQ + kk * 8, desc_kmajor(k_addr + koff), idesc_qk,
                    kk > 0);
           }
+          tc_commit(&ctl->kempty[s2]);
           tc_commit(&ctl->sfull);
         } else {
           tc_commit(&ctl->pvdone);
@@ -426,21 +450,37 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   } else {
     // ===== softmax warps: thread = TMEM lane =====
     const int L = tid;  // 0..127
+    const int r = L % r_pad;
     const int grp = L / r_pad;
     const int nc = kTileKeys / p.groups;
     const int c0 = grp * nc;
     const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
     const uint32_t t_s = tmem + lane_off + kColS;
-    const uint32_t t_p = tmem + lane_off + kColP;
     const uint32_t t_o = tmem + lane_off + kColO;
     float m = -INFINITY, l = 0.f;
-    {  // P columns outside this lane's key group stay zero for the whole kernel
-      uint32_t z[16];
+    {  // this lane's Q row -> tensor memory as bf16 pairs (zero for padding rows)
+      const uint4* src = nullptr;
+      if (r < nrows) {
+        const int rg = row0 + r, g = rg / p.T_q, t = rg % p.T_q;
+        src = reinterpret_cast<const uint4*>(p.Q + b * p.q_sb +
+                                             (int64_t)(kvh * p.G + g) * p.q_sh + t * p.q_st);
+      }
 #pragma unroll
-      for (int c = 0; c < 16; ++c) z[c] = 0;
-      tmem_st16(t_p, z);
-      tmem_st16(t_p + 16, z);
+      for (int q = 0; q < 4; ++q) {
+        uint32_t w[16];
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          const uint4 x = src ? src[q * 4 + v] : make_uint4(0, 0, 0, 0);
+          w[v * 4 + 0] = x.x;
+          w[v * 4 + 1] = x.y;
+          w[v * 4 + 2] = x.z;
+          w[v * 4 + 3] = x.w;
+        }
+        tmem_st16(tmem + lane_off + kColQ + q * 16, w);
+      }
       tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(&ctl->pready);  // phase 0: Q is in place
     }
     bool ok = true;
     for (int it = 0; it < n_tiles; ++it) {
@@ -465,11 +505,11 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         fence_proxy_async();
       }
       if (nc == 16)
-        softmax_tile<16>(t_s, t_p, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+        softmax_tile<16>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
       else if (nc == 32)
-        softmax_tile<32>(t_s, t_p, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+        softmax_tile<32>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
       else
-        softmax_tile<64>(t_s, t_p, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+        softmax_tile<64>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
       tc_fence_before();
       mbar_arrive(&ctl->pready);
     }
@@ -480,7 +520,6 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       float* o_s = reinterpret_cast<float*>(st_s);  // [128][128] fp32 over the free stage buffers
       ctl->ml[L] = make_float2(m, l);
       named_bar_sync(1, 128);
-      const int r = L % r_pad;
       float M = -INFINITY;
       for (int g = 0; g < p.groups; ++g) M = fmaxf(M, ctl->ml[g * r_pad + r].x);
       const float f = (m == -INFINITY) ? 0.f : exp2f(m - M);

@@ -95,10 +95,15 @@ def compare(cfg, O, LSE, ref, strict=True):
         assert np.array_equal(np.isfinite(lg), fin), f"LSE finiteness differs in {(b, kvh)}"
         if fin.any():
             worst["lse"] = max(worst["lse"], np.abs(lg[fin] - Lr[fin]).max())
-        assert err.max() <= TOL_MAX_O and err.mean() <= TOL_MEAN_O, (b, kvh, err.max(), err.mean())
+        # contract tolerances hold for |O| <= 1 (the workloads); a bf16 output in [2^k, 2^(k+1)) has a
+        # half-ulp of 2^(k-8), so for larger magnitudes the bound scales with max|O_ref|
+        mag = max(1.0, float(np.abs(Or).max()))
+        assert err.max() <= TOL_MAX_O * mag and err.mean() <= TOL_MEAN_O * mag, (b, kvh, err.max(), err.mean())
         if strict:
-            rms = max(float(np.sqrt((Or ** 2).mean())), 1e-3)
-            assert err.max() <= 2.0 ** -6 * max(rms, np.abs(Or).max() / 4), (b, kvh, err.max(), rms)
+            # tighter than the contract: bf16 rounding of O (2^-9 relative) and of P leave a 4x margin
+            rms = float(np.sqrt((Or ** 2).mean()))
+            bound = 2.0 ** -7 * (np.abs(Or) + rms) + 1e-5
+            assert (err <= bound).all(), (b, kvh, err.max(), rms, float((err / bound).max()))
             for g in range(G):
                 a, r = og[g].ravel(), Or[g].ravel()
                 if np.linalg.norm(r) > 0:
