@@ -202,6 +202,16 @@ const char* ss_strerror(ss_status s);
 size_t ss_sizeof_stream_desc(void);
 /* Last CUDA error code seen by this context (cudaError_t as int), 0 if none. */
 int32_t ss_last_cuda_error(ss_ctx* ctx);
+/* Tracing.  While enabled, CTA (0,0,0) of every tensor-core chunk kernel stamps the SM clock
+ * at fixed points of its tile loop into a region of the workspace: words
+ * [role][tile < 32][event < 8], role 0 = TMA producer (0 loop top, 1 K slot free, 2 V slot
+ * free), 1 = MMA issuer (0 loop top, 1 P ready, 2 V landed, 3 output MMAs issued, 4 next K
+ * landed, 5 next score MMAs issued), 2 = softmax lane 0 (0 loop top, 1 scores ready, 2 P
+ * written).  Enabling clears the region (synchronous).  ss_trace_read synchronises nothing:
+ * call it after the stream is idle; it copies up to max_words 64-bit words to HOST memory
+ * and returns the count. */
+ss_status ss_trace_enable(ss_ctx* ctx, int32_t on);
+int32_t ss_trace_read(ss_ctx* ctx, uint64_t* out, int32_t max_words);
 /* Number of kernels this context has launched since creation. */
 int64_t ss_launch_count(ss_ctx* ctx);
 /* "simt" or "tcgen05": the chunk kernel the last ss_verify_chunk used. */

@@ -28,7 +28,7 @@ SS_MASK_CHAIN, SS_MASK_TREE_BITS = 0, 1
 EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "ss_verify_chunk",
            "ss_verify_local", "ss_verify_finalize", "ss_commit_gather", "ss_poll_status",
            "ss_stream_round", "ss_strerror", "ss_sizeof_stream_desc", "ss_last_cuda_error", "ss_launch_count",
-           "ss_last_chunk_kernel"]
+           "ss_last_chunk_kernel", "ss_trace_enable", "ss_trace_read"]
 
 
 class ss_config(C.Structure):
@@ -104,6 +104,10 @@ def load() -> C.CDLL:
     lib.ss_sizeof_stream_desc.argtypes = []
     lib.ss_last_cuda_error.restype = i32
     lib.ss_last_cuda_error.argtypes = [vp]
+    lib.ss_trace_enable.restype = C.c_int
+    lib.ss_trace_enable.argtypes = [vp, i32]
+    lib.ss_trace_read.restype = i32
+    lib.ss_trace_read.argtypes = [vp, C.POINTER(C.c_uint64), i32]
     lib.ss_launch_count.restype = C.c_int64
     lib.ss_launch_count.argtypes = [vp]
     lib.ss_last_chunk_kernel.restype = C.c_char_p
@@ -219,6 +223,16 @@ class Context:
         stats = ss_stream_stats()
         self._check(self.lib.ss_stream_round(self.handle, C.byref(desc), C.byref(stats)), "ss_stream_round")
         return stats
+
+    def ss_trace_enable(self, on: bool):
+        self._check(self.lib.ss_trace_enable(self.handle, 1 if on else 0), "ss_trace_enable")
+
+    def ss_trace_read(self):
+        """[3 roles][32 tiles][8 events] clock stamps of CTA (0,0,0) of the last traced chunk kernel."""
+        n = 3 * 32 * 8
+        buf = (C.c_uint64 * n)()
+        got = self.lib.ss_trace_read(self.handle, buf, n)
+        return [[[buf[(r * 32 + t) * 8 + e] for e in range(8)] for t in range(32)] for r in range(3)][:3] if got else None
 
     def launch_count(self) -> int:
         return int(self.lib.ss_launch_count(self.handle))

@@ -49,6 +49,8 @@ struct ss_ctx {
   cudaEvent_t ev_ready[2], ev_free[2], ev_t0, ev_t1;
   bool pipe_ready;
   bool no_overlap;          // set while ss_stream_round drives the context
+  unsigned long long* trace;  // device trace region (in the workspace)
+  bool trace_on;
 };
 
 namespace {
@@ -83,13 +85,14 @@ int set_cap(const ss_config* c) { return c->max_chunks ? c->max_chunks : 64; }
 int target_ctas_default() {
   const char* e = getenv("SS_TARGET_CTAS");
   int v = e ? atoi(e) : 0;
-  return v > 0 ? v : 2 * ss::kNumSM;
+  return v > 0 ? v : ss::kNumSM;
 }
 
-// (split, b, kvh) slots one chunk call may use: enough for ~2 CTAs per SM at the largest batch.
+// (split, b, kvh) slots one chunk call may use: about one CTA per SM at the largest batch
+// (successive chunk kernels overlap, so a second CTA per SM comes from the next launch).
 int slots_for(const ss_config* c) {
   const int pairs = c->max_B * c->H_kv;
-  int s = (target_ctas_default() + pairs - 1) / pairs;
+  int s = target_ctas_default() / pairs;
   if (s < 1) s = 1;
   if (s > kMaxSplits) s = kMaxSplits;
   return pairs * s;
@@ -109,7 +112,7 @@ Layout layout_for(const ss_config* c) {
   L.set_stride_ml = rows;                 // float2 elements
   L.set_stride_a = rows * c->d;           // float elements
   const int sets = set_cap(c) + 1;
-  L.off_ml = 256;
+  L.off_ml = 256 + align_up(ss::kTraceWords * sizeof(unsigned long long), 256);
   L.off_a = align_up(L.off_ml + (size_t)sets * rows * sizeof(float2), 256);
   L.total = align_up(L.off_a + (size_t)sets * rows * c->d * sizeof(float), 256);
   return L;
@@ -222,6 +225,7 @@ ss_status ss_create(ss_ctx** out, const ss_config* cfg, void* workspace, size_t 
   c->ws = (uint8_t*)workspace;
   c->ws_bytes = workspace_bytes;
   c->status = (uint32_t*)c->ws;
+  c->trace = (unsigned long long*)(c->ws + 256);
   c->part_ml = (float2*)(c->ws + L.off_ml);
   c->part_a = (float*)(c->ws + L.off_a);
   c->set_stride_ml = L.set_stride_ml;
@@ -338,7 +342,7 @@ ss_status ss_verify_chunk(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c,
     p.groups = 1;
   }
   int splits = c->force_splits > 0 ? c->force_splits
-                                   : (c->target_ctas + pairs * p.row_tiles - 1) / (pairs * p.row_tiles);
+                                   : c->target_ctas / (pairs * p.row_tiles);
   const int max_by_slots = c->slots_per_set / pairs;
   if (splits > max_by_slots) splits = max_by_slots;
   if (splits > kMaxSplits) splits = kMaxSplits;
@@ -374,6 +378,7 @@ ss_status ss_verify_chunk(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c,
   p.R_stride = c->R_stride;
   p.status = c->status;
   p.wait_first = 0;
+  p.trace = c->trace_on ? c->trace : nullptr;
 
   const bool pdl = use_pdl(c);
   cudaError_t e = tc ? ss::launch_chunk_tc(p, tmK, tmV, s, pdl) : ss::launch_chunk_simt(p, s, pdl);
@@ -539,6 +544,24 @@ const char* ss_strerror(ss_status s) {
 
 size_t ss_sizeof_stream_desc(void) { return sizeof(ss_stream_desc); }
 int32_t ss_last_cuda_error(ss_ctx* c) { return c ? c->last_cuda : 0; }
+ss_status ss_trace_enable(ss_ctx* c, int32_t on) {
+  if (!c) return SS_ERR_ARG;
+  c->trace_on = on != 0;
+  if (on) {
+    cudaError_t e = cudaMemset(c->trace, 0, ss::kTraceWords * sizeof(unsigned long long));
+    if (e != cudaSuccess) return cuda_fail(c, e);
+  }
+  return SS_OK;
+}
+
+int32_t ss_trace_read(ss_ctx* c, uint64_t* out, int32_t max_words) {
+  if (!c || !out || max_words <= 0) return 0;
+  const int n = max_words < ss::kTraceWords ? max_words : ss::kTraceWords;
+  if (cudaMemcpy(out, c->trace, (size_t)n * sizeof(uint64_t), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return 0;
+  return n;
+}
+
 int64_t ss_launch_count(ss_ctx* c) { return c ? c->launches : 0; }
 const char* ss_last_chunk_kernel(ss_ctx* c) { return c ? c->last_kernel : "none"; }
 

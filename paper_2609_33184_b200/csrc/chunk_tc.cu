@@ -59,6 +59,12 @@ struct Ctl {
 };
 static_assert(sizeof(Ctl) <= kSmemCtl, "control block");
 
+// Optional trace: CTA (0,0,0) stamps clock64 at fixed points of each role's tile loop.
+// role 0 = TMA producer, 1 = MMA issuer, 2 = softmax thread 0.
+__device__ __forceinline__ void trace(unsigned long long* tr, int role, int it, int ev) {
+  if (tr && it < kTraceTiles) tr[(role * kTraceTiles + it) * 8 + ev] = clock64();
+}
+
 // ---- small PTX wrappers ------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -107,6 +113,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Ctl* c
     }
   }
   return true;
+}
+// One lane of a converged warp gets true.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
 }
 __device__ __forceinline__ void fence_proxy_async() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -304,6 +320,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   const int row0 = rt * p.rows_per_tile;
   const int nrows = min(p.rows_per_tile, p.R - row0);
   const int r_pad = 128 / p.groups;
+  unsigned long long* tr = (blockIdx.x | blockIdx.y | blockIdx.z) ? nullptr : p.trace;
 
   if (p.wait_first) pdl_wait_prior();
   pdl_launch_dependents();
@@ -330,110 +347,164 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     return;
   }
 
-  // ---- set-up: barriers, tensor memory -------------------------------------------------------
-  if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(&ctl->kfull[s], 1);
-      mbar_init(&ctl->vfull[s], 1);
-      mbar_init(&ctl->kempty[s], 1);
-      mbar_init(&ctl->vempty[s], 1);
-    }
-    mbar_init(&ctl->sfull, 1);
-    mbar_init(&ctl->pready, 128);
-    mbar_init(&ctl->pvdone, 1);
-    ctl->abort = 0;
-    fence_barrier_init();
-  }
+  // ---- set-up: barriers, first loads, tensor memory ------------------------------------------
+  auto issue_tile = [&](int it, uint64_t pol) {
+    const int s = it % kStages;
+    const int tok = tok0 + it * kTileKeys;
+    const uint32_t kdst = smem_u32(st_s + s * kStageBytes);
+    const uint32_t vdst = kdst + kTileBytes;
+    mbar_expect_tx(&ctl->kfull[s], kTileBytes);
+    tma_load_4d(kdst, &tmK, 0, tok, kvh, b, &ctl->kfull[s], pol);
+    tma_load_4d(kdst + kHalfTile, &tmK, 64, tok, kvh, b, &ctl->kfull[s], pol);
+    mbar_expect_tx(&ctl->vfull[s], kTileBytes);
+    tma_load_4d(vdst, &tmV, 0, tok, kvh, b, &ctl->vfull[s], pol);
+    tma_load_4d(vdst + kHalfTile, &tmV, 64, tok, kvh, b, &ctl->vfull[s], pol);
+  };
+  const int n_pre = min(n_tiles, kStages);
+  uint32_t qreg[64];  // softmax threads: this lane's Q row (bf16 pairs)
   if (warp == 4) {
+    if (lane == 0) {
+      for (int s = 0; s < kStages; ++s) {
+        mbar_init(&ctl->kfull[s], 1);
+        mbar_init(&ctl->vfull[s], 1);
+        mbar_init(&ctl->kempty[s], 1);
+        mbar_init(&ctl->vempty[s], 1);
+      }
+      mbar_init(&ctl->sfull, 1);
+      mbar_init(&ctl->pready, 128);
+      mbar_init(&ctl->pvdone, 1);
+      ctl->abort = 0;
+      fence_barrier_init();
+      // the first tiles go out before the rest of the CTA is set up
+      const uint64_t pol = l2_evict_first_policy();
+      for (int it = 0; it < n_pre; ++it) issue_tile(it, pol);
+    }
+    __syncwarp();
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                      smem_u32(&ctl->tmem_base)),
                  "r"(kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  } else if (warp < 4) {
+    const int r = tid % r_pad;
+    const uint4* src = nullptr;
+    if (r < nrows) {
+      const int rg = row0 + r, g = rg / p.T_q, t = rg % p.T_q;
+      src = reinterpret_cast<const uint4*>(p.Q + b * p.q_sb + (int64_t)(kvh * p.G + g) * p.q_sh +
+                                           t * p.q_st);
+    }
+#pragma unroll
+    for (int v = 0; v < 16; ++v) {
+      const uint4 x = src ? src[v] : make_uint4(0, 0, 0, 0);
+      qreg[v * 4 + 0] = x.x;
+      qreg[v * 4 + 1] = x.y;
+      qreg[v * 4 + 2] = x.z;
+      qreg[v * 4 + 3] = x.w;
+    }
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = ctl->tmem_base;
+  unsigned long long* trl = lane == 0 ? tr : nullptr;
 
   if (warp == 4) {
     // ===== TMA producer =====
     if (lane == 0) {
       const uint64_t pol = l2_evict_first_policy();
-      int issued_k = 0, issued_v = 0;
-      for (int it = 0; it < n_tiles; ++it) {
+      int issued = n_pre;
+      for (int it = n_pre; it < n_tiles; ++it) {
         const int s = it % kStages;
         const uint32_t ph = (it / kStages) & 1;
         const int tok = tok0 + it * kTileKeys;
         const uint32_t kdst = smem_u32(st_s + s * kStageBytes);
         const uint32_t vdst = kdst + kTileBytes;
+        trace(tr, 0, it, 0);
         if (!mbar_wait(&ctl->kempty[s], ph ^ 1, ctl, p.status)) break;
+        trace(tr, 0, it, 1);
         mbar_expect_tx(&ctl->kfull[s], kTileBytes);
         tma_load_4d(kdst, &tmK, 0, tok, kvh, b, &ctl->kfull[s], pol);
         tma_load_4d(kdst + kHalfTile, &tmK, 64, tok, kvh, b, &ctl->kfull[s], pol);
-        issued_k = it + 1;
-        if (!mbar_wait(&ctl->vempty[s], ph ^ 1, ctl, p.status)) break;
+        // the V slot frees after the K slot; its load is accounted with the K load: on a
+        // failed wait the K copy above is still waited for below through `issued`
+        if (!mbar_wait(&ctl->vempty[s], ph ^ 1, ctl, p.status)) {
+          mbar_expect_tx(&ctl->vfull[s], 0);  // nothing will arrive for V
+          issued = it + 1;
+          break;
+        }
+        trace(tr, 0, it, 2);
         mbar_expect_tx(&ctl->vfull[s], kTileBytes);
         tma_load_4d(vdst, &tmV, 0, tok, kvh, b, &ctl->vfull[s], pol);
         tma_load_4d(vdst + kHalfTile, &tmV, 64, tok, kvh, b, &ctl->vfull[s], pol);
-        issued_v = it + 1;
+        issued = it + 1;
       }
       if (ctl->abort) {
         // let the copies this thread started land before the CTA leaves (bounded)
         const unsigned long long t0 = gtime_ns();
-        for (int it = max(0, issued_k - kStages); it < issued_k; ++it) {
+        for (int it = max(0, issued - kStages); it < issued; ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1;
           while (!mbar_try_wait(&ctl->kfull[s], ph) && gtime_ns() - t0 < kWaitNs) {
           }
-          if (it < issued_v)
-            while (!mbar_try_wait(&ctl->vfull[s], ph) && gtime_ns() - t0 < kWaitNs) {
-            }
+          while (!mbar_try_wait(&ctl->vfull[s], ph) && gtime_ns() - t0 < kWaitNs) {
+          }
         }
       }
     }
   } else if (warp == 5) {
-    // ===== MMA issuer =====
-    if (lane == 0) {
-      constexpr uint32_t idesc_qk = make_idesc(128, kTileKeys, false);
-      constexpr uint32_t idesc_pv = make_idesc(128, kD, true);
-      // Q is in tensor memory once the softmax warps have arrived on pready (phase 0)
-      bool ok = mbar_wait(&ctl->pready, 0, ctl, p.status) &&
-                mbar_wait(&ctl->kfull[0], 0, ctl, p.status);
-      if (ok) {
-        tc_fence_after();
-        const uint32_t k_addr = smem_u32(st_s);
+    // ===== MMA issuer: the whole warp walks the loop (uniform descriptors), one elected
+    // lane issues =====
+    constexpr uint32_t idesc_qk = make_idesc(128, kTileKeys, false);
+    constexpr uint32_t idesc_pv = make_idesc(128, kD, true);
+    const bool leader = elect_one();
+    const uint32_t st_addr = smem_u32(st_s);
+    // Q is in tensor memory once the softmax warps have arrived on pready (phase 0)
+    bool ok = mbar_wait(&ctl->pready, 0, ctl, p.status) && mbar_wait(&ctl->kfull[0], 0, ctl, p.status);
+    if (ok) {
+      tc_fence_after();
+      if (leader) {
 #pragma unroll
         for (int kk = 0; kk < kD / 16; ++kk) {
           const uint32_t koff = (kk >> 2) * kHalfTile + (kk & 3) * 32;
-          mma_ts(tmem + kColS, tmem + kColQ + kk * 8, desc_kmajor(k_addr + koff), idesc_qk, kk > 0);
+          mma_ts(tmem + kColS, tmem + kColQ + kk * 8, desc_kmajor(st_addr + koff), idesc_qk, kk > 0);
         }
         tc_commit(&ctl->kempty[0]);
         tc_commit(&ctl->sfull);
       }
-      for (int it = 0; ok && it < n_tiles; ++it) {
-        const int s = it % kStages;
-        const uint32_t ph = (it / kStages) & 1;
-        ok = mbar_wait(&ctl->pready, (it + 1) & 1, ctl, p.status) &&
-             mbar_wait(&ctl->vfull[s], ph, ctl, p.status);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t v_addr = smem_u32(st_s + s * kStageBytes + kTileBytes);
+      __syncwarp();
+    }
+    for (int it = 0; ok && it < n_tiles; ++it) {
+      const int s = it % kStages;
+      const uint32_t ph = (it / kStages) & 1;
+      trace(trl, 1, it, 0);
+      ok = mbar_wait(&ctl->pready, (it + 1) & 1, ctl, p.status);
+      trace(trl, 1, it, 1);
+      ok = ok && mbar_wait(&ctl->vfull[s], ph, ctl, p.status);
+      if (!ok) break;
+      trace(trl, 1, it, 2);
+      tc_fence_after();
+      const uint32_t v_addr = st_addr + s * kStageBytes + kTileBytes;
+      if (leader) {
 #pragma unroll
         for (int kk = 0; kk < kTileKeys / 16; ++kk) {
           mma_ts(tmem + kColO, tmem + kColP + kk * 8, desc_mnmajor(v_addr + kk * 2048, kHalfTile),
                  idesc_pv, (it > 0 || kk > 0));
         }
         tc_commit(&ctl->vempty[s]);
-        if (it + 1 < n_tiles) {
-          const int s2 = (it + 1) % kStages;
-          const uint32_t ph2 = ((it + 1) / kStages) & 1;
-          ok = mbar_wait(&ctl->kfull[s2], ph2, ctl, p.status);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t k_addr = smem_u32(st_s + s2 * kStageBytes);
-          // overwrites the S/P columns: the tensor pipe runs this thread's MMAs in issue
-          // order, so the P V products above have consumed P before these write S
+      }
+      __syncwarp();
+      trace(trl, 1, it, 3);
+      if (it + 1 < n_tiles) {
+        const int s2 = (it + 1) % kStages;
+        const uint32_t ph2 = ((it + 1) / kStages) & 1;
+        ok = mbar_wait(&ctl->kfull[s2], ph2, ctl, p.status);
+        if (!ok) break;
+        trace(trl, 1, it, 4);
+        tc_fence_after();
+        const uint32_t k_addr = st_addr + s2 * kStageBytes;
+        // overwrites the S/P columns: the tensor pipe runs this thread's MMAs in issue
+        // order, so the P V products above have consumed P before these write S
+        if (leader) {
 #pragma unroll
           for (int kk = 0; kk < kD / 16; ++kk) {
             const uint32_t koff = (kk >> 2) * kHalfTile + (kk & 3) * 32;
@@ -442,9 +513,12 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
           }
           tc_commit(&ctl->kempty[s2]);
           tc_commit(&ctl->sfull);
-        } else {
-          tc_commit(&ctl->pvdone);
         }
+        __syncwarp();
+        trace(trl, 1, it, 5);
+      } else {
+        if (leader) tc_commit(&ctl->pvdone);
+        __syncwarp();
       }
     }
   } else {
@@ -459,23 +533,11 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     const uint32_t t_o = tmem + lane_off + kColO;
     float m = -INFINITY, l = 0.f;
     {  // this lane's Q row -> tensor memory as bf16 pairs (zero for padding rows)
-      const uint4* src = nullptr;
-      if (r < nrows) {
-        const int rg = row0 + r, g = rg / p.T_q, t = rg % p.T_q;
-        src = reinterpret_cast<const uint4*>(p.Q + b * p.q_sb +
-                                             (int64_t)(kvh * p.G + g) * p.q_sh + t * p.q_st);
-      }
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         uint32_t w[16];
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          const uint4 x = src ? src[q * 4 + v] : make_uint4(0, 0, 0, 0);
-          w[v * 4 + 0] = x.x;
-          w[v * 4 + 1] = x.y;
-          w[v * 4 + 2] = x.z;
-          w[v * 4 + 3] = x.w;
-        }
+        for (int v = 0; v < 16; ++v) w[v] = qreg[q * 16 + v];
         tmem_st16(tmem + lane_off + kColQ + q * 16, w);
       }
       tc_wait_st();
@@ -486,9 +548,11 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     for (int it = 0; it < n_tiles; ++it) {
       const int s = it % kStages;
       const uint32_t ph = (it / kStages) & 1;
+      if (L == 0) trace(tr, 2, it, 0);
       ok = mbar_wait(&ctl->sfull, it & 1, ctl, p.status);
       if (!ok) break;
       tc_fence_after();
+      if (L == 0) trace(tr, 2, it, 1);
       const int n_valid = min(kTileKeys, tok1 - (tok0 + it * kTileKeys));
       if (n_valid < kTileKeys) {
         // ragged tail: rows past the valid length may hold anything; P is 0 there, so V must
@@ -512,6 +576,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         softmax_tile<64>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
       tc_fence_before();
       mbar_arrive(&ctl->pready);
+      if (L == 0) trace(tr, 2, it, 2);
     }
     ok = ok && mbar_wait(&ctl->pvdone, 0, ctl, p.status);
     if (ok) {

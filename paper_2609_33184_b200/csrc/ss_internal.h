@@ -13,6 +13,8 @@ constexpr int kMaxSets = 128;      // chunk-call partial sets a finalize launch 
 constexpr int kMaxSplits = 16;     // token splits of one chunk call
 constexpr int kTileKeys = 64;      // keys per shared-memory tile of the tensor-core kernel
 constexpr int kNumSM = 148;
+constexpr int kTraceTiles = 32;    // tiles of CTA (0,0,0) a trace records
+constexpr int kTraceWords = 3 * kTraceTiles * 8;  // [role][tile][event] clock64 stamps
 
 // Partial state of one (set, split, request, kv-head): for each of its R rows the pair
 // (m, l) and the unnormalised output a[d].  m is the row maximum of
@@ -42,6 +44,7 @@ struct ChunkParams {
   int R_stride;
   uint32_t* status;
   int wait_first;       // 1: wait for the preceding kernel before reading inputs
+  unsigned long long* trace;  // optional: per-tile clock stamps of CTA (0,0,0), see ss_trace_read
 };
 
 struct LocalParams {

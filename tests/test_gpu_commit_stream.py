@@ -1,0 +1,203 @@
+"""GPU tests of commit-gather (bit exact), the streamed round, the call-order state machine
+and the trace facility, all through the C ABI."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+import bench
+from paper_2609_33184_b200 import inputs
+from tests import util
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _ssb():
+    from paper_2609_33184_b200 import binding
+    return binding
+
+
+def _u16(t):
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_commit_gather_bit_exact(d):
+    import oracle
+    ssb = _ssb()
+    B, H_kv, T, cap = 5, 3, 9, 20
+    ctx = ssb.Context(B, 2 * H_kv, H_kv, d, T, T, 64)
+    g = torch.Generator().manual_seed(d)
+    rnd = lambda *s: torch.randint(-32768, 32767, s, generator=g, dtype=torch.int16)
+    K_loc, V_loc = rnd(B, H_kv, T, d).to(DEV).view(torch.bfloat16), rnd(B, H_kv, T, d).to(DEV).view(torch.bfloat16)
+    # destination: a strided view into a larger canary-filled buffer
+    Kbig, Vbig = rnd(B, H_kv, cap + 4, d + 8).to(DEV), rnd(B, H_kv, cap + 4, d + 8).to(DEV)
+    K0, V0 = Kbig.clone(), Vbig.clone()
+    K_dst = Kbig.view(torch.bfloat16)[:, :, 2:2 + cap, 8:]
+    V_dst = Vbig.view(torch.bfloat16)[:, :, 2:2 + cap, :d]
+    idx = torch.tensor([[0, 1, 2, 3, 4, 5, 6, 7, 8], [8, 6, 4, 2, 0, 1, 3, 5, 7], [3, 3, 3, 3, 3, 3, 3, 3, 3],
+                        [0, 4, 8, 0, 0, 0, 0, 0, 0], [1, 2, 0, 0, 0, 0, 0, 0, 0]], dtype=torch.int32)
+    cnt = torch.tensor([9, 5, 9, 3, 0], dtype=torch.int32)
+    off = torch.tensor([0, 15, 11, 7, 19], dtype=torch.int32)
+    ctx.ss_commit_gather(K_loc, V_loc, idx.to(DEV), cnt.to(DEV), K_dst, V_dst, off.to(DEV))
+    st, bits = ctx.ss_poll_status()
+    assert st == 0, bits
+    ko, vo = oracle.commit_gather(_u16(K_loc), _u16(V_loc), idx.numpy(), cnt.numpy(),
+                                  _u16(K0.view(torch.bfloat16)[:, :, 2:2 + cap, 8:]),
+                                  _u16(V0.view(torch.bfloat16)[:, :, 2:2 + cap, :d]), off.numpy())
+    assert np.array_equal(_u16(K_dst), ko) and np.array_equal(_u16(V_dst), vo)
+    # nothing outside the destination view changed
+    Kchk, Vchk = Kbig.clone(), Vbig.clone()
+    Kchk.view(torch.bfloat16)[:, :, 2:2 + cap, 8:] = K0.view(torch.bfloat16)[:, :, 2:2 + cap, 8:]
+    Vchk.view(torch.bfloat16)[:, :, 2:2 + cap, :d] = V0.view(torch.bfloat16)[:, :, 2:2 + cap, :d]
+    assert torch.equal(Kchk, K0) and torch.equal(Vchk, V0)
+    ctx.close()
+
+
+def test_commit_gather_device_detected_errors():
+    import oracle
+    ssb = _ssb()
+    B, H_kv, T, d, cap = 3, 2, 4, 128, 6
+    ctx = ssb.Context(B, 2 * H_kv, H_kv, d, T, T, 64)
+    K_loc = inputs.normal_bf16(1, 1, (B, H_kv, T, d), device=DEV)
+    V_loc = inputs.normal_bf16(1, 2, (B, H_kv, T, d), device=DEV)
+    K_dst = torch.zeros(B, H_kv, cap, d, dtype=torch.bfloat16, device=DEV)
+    V_dst = torch.zeros_like(K_dst)
+    idx = torch.tensor([[0, 7, 2, 3], [0, 1, 2, 3], [0, -1, 2, 3]], dtype=torch.int32)
+    cnt = torch.tensor([3, 4, 9], dtype=torch.int32)     # request 2: count out of range
+    off = torch.tensor([0, 4, 0], dtype=torch.int32)     # request 1: rows 2,3 overflow cap
+    ctx.ss_commit_gather(K_loc, V_loc, idx.to(DEV), cnt.to(DEV), K_dst, V_dst, off.to(DEV))
+    st, bits = ctx.ss_poll_status()
+    assert st == ssb.SS_ERR_DEVICE_FLAG
+    assert bits & ssb.SS_DEV_BAD_ACCEPT and bits & ssb.SS_DEV_DST_OVERFLOW
+    ko, vo = oracle.commit_gather(_u16(K_loc), _u16(V_loc), idx.numpy(), cnt.numpy(),
+                                  np.zeros((B, H_kv, cap, d), np.uint16), np.zeros((B, H_kv, cap, d), np.uint16),
+                                  off.numpy())
+    assert np.array_equal(_u16(K_dst), ko) and np.array_equal(_u16(V_dst), vo)   # offending rows skipped
+    ctx.close()
+
+
+def test_call_order_and_argument_errors():
+    ssb = _ssb()
+    cfg = inputs.VerifyConfig("v", 0x61, 2, 8, 2, 128, 128, 4, 128, 128)
+    lens = [128, 128]
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    K, V, vl = chunks[0]
+    O = torch.empty(2, 8, 4, 128, dtype=torch.bfloat16, device=DEV)
+    ctx = util.make_ctx(cfg)
+
+    def status(fn, *a):
+        with pytest.raises(ssb.SpecStreamError) as e:
+            fn(*a)
+        return e.value.status
+
+    assert status(ctx.ss_verify_chunk, K, V, vl) == ssb.SS_ERR_STATE          # before begin
+    assert status(ctx.ss_verify_finalize, O, None) == ssb.SS_ERR_STATE
+    ctx.ss_verify_begin(Q, cfg.scale)
+    assert status(ctx.ss_verify_begin, Q, cfg.scale) == ssb.SS_ERR_STATE       # begin twice
+    ctx.ss_verify_local(K_loc, V_loc)
+    assert status(ctx.ss_verify_local, K_loc, V_loc) == ssb.SS_ERR_STATE       # local twice
+    other = torch.cuda.Stream()
+    assert status(ctx.ss_verify_chunk, K, V, vl, other) == ssb.SS_ERR_STATE    # another stream
+    big = torch.zeros(2, 2, 256, 128, dtype=torch.bfloat16, device=DEV)
+    assert status(ctx.ss_verify_chunk, big, big, None) == ssb.SS_ERR_SHAPE     # L_c > max_Lc
+    mis = torch.zeros(2 * 2 * 128 * 128 + 8, dtype=torch.bfloat16, device=DEV)[4:-4].view(2, 2, 128, 128)
+    assert status(ctx.ss_verify_chunk, mis, V, vl) == ssb.SS_ERR_ALIGN         # base not 16-byte aligned
+    assert status(ctx.ss_verify_local, K_loc, V_loc, ssb.SS_MASK_TREE_BITS, None) in (ssb.SS_ERR_ARG, ssb.SS_ERR_STATE)
+    ctx.ss_verify_finalize(O, None)                                            # LSE may be NULL
+    torch.cuda.synchronize()
+    # no chunk at all and no local: every row is empty -> O = 0
+    ctx.ss_verify_begin(Q, cfg.scale)
+    L = torch.empty(2, 8, 4, dtype=torch.float32, device=DEV)
+    ctx.ss_verify_finalize(O, L)
+    torch.cuda.synchronize()
+    assert (O == 0).all() and torch.isinf(L).all() and (L < 0).all()
+    too_many = torch.zeros(3, 8, 4, 128, dtype=torch.bfloat16, device=DEV)
+    assert status(ctx.ss_verify_begin, too_many, cfg.scale) == ssb.SS_ERR_SHAPE
+    ctx.close()
+    with pytest.raises(ssb.SpecStreamError):
+        ssb.Context(2, 9, 2, 128, 4, 4, 128)       # H_q % H_kv != 0
+
+
+def _stream_case(cfg, lens, batch_chunks=1, copy_only=0, accept=True):
+    ssb = _ssb()
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV, fill=0.0)
+    host = bench.pinned_history(cfg, lens, chunks)
+    # poison the padding of partial host blocks: those tokens must never be read into results
+    for b in range(cfg.B):
+        j, r = divmod(lens[b], cfg.L_c)
+        if r and j < host.shape[1]:
+            host[b, j, :, :, r:] = float("nan")
+    bufs = bench.stream_buffers(cfg, DEV, len(chunks), batch_chunks)
+    for s in range(2):
+        bufs["stage_k"][s].fill_(float("nan"))
+        bufs["stage_v"][s].fill_(float("nan"))
+    O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
+    LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
+    acc = None
+    if accept:
+        idx, cnt = inputs.make_accept(cfg)
+        shape = (cfg.B, cfg.H_kv, cfg.T_q, cfg.d)
+        acc = {"idx": idx.to(DEV), "cnt": cnt.to(DEV), "zero": torch.zeros(cfg.B, dtype=torch.int32, device=DEV),
+               "ck": torch.zeros(shape, dtype=torch.bfloat16, device=DEV),
+               "cv": torch.zeros(shape, dtype=torch.bfloat16, device=DEV),
+               "hk": torch.zeros(shape, dtype=torch.bfloat16).pin_memory(),
+               "hv": torch.zeros(shape, dtype=torch.bfloat16).pin_memory(), "cnt_host": cnt, "idx_host": idx}
+    ctx = ssb.Context(cfg.B, cfg.H_q, cfg.H_kv, cfg.d, cfg.T_q, cfg.T_q, cfg.L_c * batch_chunks)
+    desc = bench.make_stream_desc(ssb, cfg, lens, host, DEV, Q, K_loc, V_loc, bits, O, LSE, bufs,
+                                  batch_chunks=batch_chunks, accept=acc, copy_only=copy_only)
+    stats = ctx.ss_stream_round(desc)
+    st, dev_bits = ctx.ss_poll_status()
+    assert st == 0, dev_bits
+    return ctx, (Q, chunks, K_loc, V_loc, bits), O, LSE, bufs, acc, stats, desc
+
+
+@pytest.mark.parametrize("batch_chunks", [1, 2, 3])
+def test_stream_round_matches_oracle_ragged(batch_chunks):
+    import oracle
+    cfg = inputs.VerifyConfig("v", 0x62, 5, 8, 2, 128, 128, 8, 0, 900, accept=True)
+    lens = [900, 0, 128, 257, 513]
+    ctx, case, O, LSE, bufs, acc, stats, _ = _stream_case(cfg, lens, batch_chunks)
+    ref = util.oracle_case(cfg, lens, *case)
+    util.compare(cfg, O, LSE, ref)
+    assert torch.equal(bufs["O_host"], O.cpu()) and torch.equal(bufs["LSE_host"], LSE.cpu())
+    assert stats.h2d_bytes == sum(lens) * cfg.H_kv * cfg.d * 4
+    n_fills = (max(lens) + cfg.L_c * batch_chunks - 1) // (cfg.L_c * batch_chunks)
+    assert stats.chunk_calls == n_fills
+    # committed rows arrived on the host, bit exact
+    zero = np.zeros((cfg.B, cfg.H_kv, cfg.T_q, cfg.d), np.uint16)
+    ko, vo = oracle.commit_gather(_u16(case[2]), _u16(case[3]), acc["idx_host"].numpy(), acc["cnt_host"].numpy(),
+                                  zero, zero, np.zeros(cfg.B, np.int32))
+    assert np.array_equal(_u16(acc["hk"]), ko) and np.array_equal(_u16(acc["hv"]), vo)
+    ctx.close()
+
+
+def test_stream_round_copy_only_and_reuse():
+    cfg = inputs.VerifyConfig("v", 0x63, 3, 8, 2, 128, 256, 6, 300, 1500)
+    lens = inputs.history_lengths(cfg)
+    ctx, case, O, LSE, bufs, acc, stats, desc = _stream_case(cfg, lens, accept=False)
+    O1 = O.clone()
+    desc.copy_only = 1
+    s2 = ctx.ss_stream_round(desc)
+    assert s2.chunk_calls == 0 and s2.h2d_bytes == stats.h2d_bytes and s2.copies == stats.copies
+    desc.copy_only = 0
+    ctx.ss_stream_round(desc)        # the context is reusable and deterministic
+    assert torch.equal(O.view(torch.int16), O1.view(torch.int16))
+    ctx.close()
+
+
+def test_trace_records_tile_loop():
+    ssb = _ssb()
+    cfg = inputs.VerifyConfig("v", 0x64, 2, 8, 2, 128, 512, 8, 512, 512)
+    lens = [512, 512]
+    case = util.gen_case(cfg, lens, DEV)
+    ctx = util.make_ctx(cfg)
+    ctx.ss_trace_enable(True)
+    util.gpu_case(ctx, cfg, *case)
+    tr = ctx.ss_trace_read()
+    ctx.ss_trace_enable(False)
+    mma = [t[1] for t in tr[1] if t[1]]
+    assert len(mma) >= 2 and all(b > a for a, b in zip(mma, mma[1:]))
+    ctx.close()
