@@ -47,7 +47,10 @@ def peaks():
 
 # DRAM bytes (read + write) per chunk-kernel launch from an ncu capture of the same kernel;
 # filled from the summaries under profiles/ (None until a capture exists for the workload).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {
+    # profiles/chunk_tc_kernel_c2_qwen3_8b.md: 135.33 MB read + 4.1 MB written per launch
+    "c2_qwen3_8b": 139.4e6,
+}
 
 
 class ClockSampler:
