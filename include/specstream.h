@@ -197,6 +197,40 @@ typedef struct {
 
 ss_status ss_stream_round(ss_ctx* ctx, const ss_stream_desc* desc, ss_stream_stats* stats);
 
+/* A whole round (one history chunk + local segment -> O, LSE) that allocates nothing and
+ * needs no context or workspace.  The paper has no counterpart: this exists for callers that
+ * cannot call cudaMalloc where they need attention (code in a region that must not
+ * synchronise the device, plug-ins that do not own the process's memory pool, start-up paths
+ * that run before the host framework's allocator exists).  The per-row partial states live in
+ * a fixed SS_STATIC_SCRATCH_BYTES array inside the library's device image; each GPU that
+ * loads the library holds it until the process exits.
+ *  - Same tensors, layouts, masks and results as begin/chunk/local/finalize with one chunk
+ *    call (K/V [B,H_kv,L_c,d], L_c may be 0 to skip the history; T_loc may be 0 to skip the
+ *    local segment, not both).  The CUDA-core chunk kernel is used.
+ *  - Returns SS_ERR_CAPACITY, enqueuing nothing, when the round's partial states
+ *    (2 * splits * B * H_kv * T_q * G rows of (d + 2) floats, splits <= 16) do not fit.
+ *  - The first call on a device looks up the array's device address (with that device
+ *    current); make that first call before any stream capture.  No call allocates or frees.
+ *  - All calls share the array: it keeps the last call's contents (the call clears what must
+ *    start at zero), and calls whose kernels may overlap on the GPU race - serialise them.
+ *  - `status` (optional DEVICE word, OR-ed with SS_DEV_* bits) receives device-detected
+ *    problems; with NULL they are only clamped. */
+#define SS_STATIC_SCRATCH_BYTES (4u << 20)
+typedef struct {
+  int32_t B, H_q, H_kv, d, T_q, T_loc, L_c;
+  float scale;
+  ss_tensor Q;              /* [B, H_q, T_q, d]                                          */
+  ss_tensor K, V;           /* [B, H_kv, L_c, d]; ignored when L_c == 0                  */
+  const int32_t* valid_len; /* device [B] or NULL                                        */
+  ss_tensor K_loc, V_loc;   /* [B, H_kv, T_loc, d]; ignored when T_loc == 0              */
+  ss_mask_kind mask_kind;
+  const uint64_t* mask_bits;
+  void* O;                  /* device [B, H_q, T_q, d] bf16                              */
+  float* LSE;               /* device [B, H_q, T_q] or NULL                              */
+  uint32_t* status;         /* device word or NULL                                       */
+} ss_static_round;
+ss_status ss_verify_round_static(const ss_static_round* round, void* stream);
+
 const char* ss_strerror(ss_status s);
 /* sizeof(ss_stream_desc) as compiled, for bindings that mirror the struct. */
 size_t ss_sizeof_stream_desc(void);

@@ -28,7 +28,7 @@ SS_MASK_CHAIN, SS_MASK_TREE_BITS = 0, 1
 EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "ss_verify_chunk",
            "ss_verify_local", "ss_verify_finalize", "ss_commit_gather", "ss_poll_status",
            "ss_stream_round", "ss_strerror", "ss_sizeof_stream_desc", "ss_last_cuda_error", "ss_launch_count",
-           "ss_last_chunk_kernel", "ss_trace_enable", "ss_trace_read"]
+           "ss_last_chunk_kernel", "ss_trace_enable", "ss_trace_read", "ss_verify_round_static"]
 
 
 class ss_config(C.Structure):
@@ -57,6 +57,18 @@ class ss_stream_desc(C.Structure):
                 ("host_commit_k", C.c_void_p), ("host_commit_v", C.c_void_p),
                 ("O_host", C.c_void_p), ("LSE_host", C.c_void_p),
                 ("copy_only", C.c_int32)]
+
+
+class ss_static_round(C.Structure):
+    _fields_ = [("B", C.c_int32), ("H_q", C.c_int32), ("H_kv", C.c_int32), ("d", C.c_int32),
+                ("T_q", C.c_int32), ("T_loc", C.c_int32), ("L_c", C.c_int32), ("scale", C.c_float),
+                ("Q", ss_tensor), ("K", ss_tensor), ("V", ss_tensor), ("valid_len", C.c_void_p),
+                ("K_loc", ss_tensor), ("V_loc", ss_tensor), ("mask_kind", C.c_int),
+                ("mask_bits", C.c_void_p), ("O", C.c_void_p), ("LSE", C.c_void_p),
+                ("status", C.c_void_p)]
+
+
+SS_STATIC_SCRATCH_BYTES = 4 << 20
 
 
 class ss_stream_stats(C.Structure):
@@ -108,6 +120,8 @@ def load() -> C.CDLL:
     lib.ss_trace_enable.argtypes = [vp, i32]
     lib.ss_trace_read.restype = i32
     lib.ss_trace_read.argtypes = [vp, C.POINTER(C.c_uint64), i32]
+    lib.ss_verify_round_static.restype = C.c_int
+    lib.ss_verify_round_static.argtypes = [C.POINTER(ss_static_round), vp]
     lib.ss_launch_count.restype = C.c_int64
     lib.ss_launch_count.argtypes = [vp]
     lib.ss_last_chunk_kernel.restype = C.c_char_p
