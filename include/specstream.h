@@ -84,6 +84,9 @@ typedef struct {
  * produced by a copy / an event the stream waited on - not by a kernel enqueued on the
  * same stream between two ss_ calls. */
 #define SS_FLAG_OVERLAP_CHUNKS 2u
+/* Use the rows-on-M tensor-core chunk kernel even when the kv-head has <= 32 query rows
+ * (where the keys-on-M kernel is the default).  For cross-checks. */
+#define SS_FLAG_ROWS_ON_M 4u
 
 typedef struct {
   const void* ptr;                      /* device pointer, bf16                      */
@@ -238,12 +241,11 @@ size_t ss_sizeof_stream_desc(void);
 int32_t ss_last_cuda_error(ss_ctx* ctx);
 /* Tracing.  While enabled, CTA (0,0,0) of every tensor-core chunk kernel stamps the SM clock
  * at fixed points of its tile loop into a region of the workspace: words
- * [role][tile < 32][event < 8], role 0 = TMA producer (0 loop top, 1 K slot free, 2 V slot
- * free), 1 = MMA issuer (0 loop top, 1 P ready, 2 V landed, 3 output MMAs issued, 4 next K
- * landed, 5 next score MMAs issued), 2 = softmax lane 0 (0 loop top, 1 scores ready, 2 P
- * written).  Enabling clears the region (synchronous).  ss_trace_read synchronises nothing:
- * call it after the stream is idle; it copies up to max_words 64-bit words to HOST memory
- * and returns the count. */
+ * [role][tile < 32][event < 8], role 0 = TMA producer, 1 = MMA issuer, 2 = softmax lane 0;
+ * event 0 is the top of the role's loop for that tile, the other events are the kernel's own
+ * wait / issue points (see the kernel sources).  Enabling clears the region (synchronous).
+ * ss_trace_read synchronises nothing: call it after the stream is idle; it copies up to
+ * max_words 64-bit words to HOST memory and returns the count. */
 ss_status ss_trace_enable(ss_ctx* ctx, int32_t on);
 int32_t ss_trace_read(ss_ctx* ctx, uint64_t* out, int32_t max_words);
 /* Number of kernels this context has launched since creation. */

@@ -33,12 +33,13 @@ struct ss_ctx {
   int64_t launches;
   const char* last_kernel;
   int force_splits;        // SS_SPLITS env override (0 = automatic)
+  bool force_rows_kernel;  // SS_CHUNK_KERNEL=rows: rows-on-M tensor-core kernel even for few rows
   int target_ctas;
   // tensor-map cache
   struct TmEntry {
     const void* ptr;
     int64_t sb, sh, st;
-    int B, L_c;
+    int B, L_c, box_tokens;
     CUtensorMap map;
     uint64_t age;
   } tm[64];
@@ -128,12 +129,12 @@ ss_status cuda_fail(ss_ctx* c, cudaError_t e) {
   return SS_ERR_CUDA;
 }
 
-// Tensor map over K or V [B, H_kv, L_c, d] with a [64 tokens][64 d] box and 128-byte swizzle.
-bool get_tensor_map(ss_ctx* c, const ss_tensor& t, int B, int L_c, CUtensorMap* out) {
+// Tensor map over K or V [B, H_kv, L_c, d] with a [box_tokens][64 d] box and 128-byte swizzle.
+bool get_tensor_map(ss_ctx* c, const ss_tensor& t, int B, int L_c, int box_tokens, CUtensorMap* out) {
   for (int i = 0; i < c->tm_n; ++i) {
     ss_ctx::TmEntry& e = c->tm[i];
     if (e.ptr == t.ptr && e.sb == t.stride_b && e.sh == t.stride_h && e.st == t.stride_t &&
-        e.B == B && e.L_c == L_c) {
+        e.B == B && e.L_c == L_c && e.box_tokens == box_tokens) {
       e.age = ++c->tm_clock;
       *out = e.map;
       return true;
@@ -147,7 +148,7 @@ bool get_tensor_map(ss_ctx* c, const ss_tensor& t, int B, int L_c, CUtensorMap* 
   const int64_t sb = (B > 1 || t.stride_b > 0) ? t.stride_b : (int64_t)H_kv * sh;
   if (st <= 0 || sh <= 0 || sb <= 0) return false;
   cuuint64_t strides[3] = {(cuuint64_t)st * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
-  cuuint32_t box[4] = {64, (cuuint32_t)kTileKeys, 1, 1};
+  cuuint32_t box[4] = {64, (cuuint32_t)box_tokens, 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUtensorMap m;
   CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(t.ptr), dims,
@@ -163,7 +164,7 @@ bool get_tensor_map(ss_ctx* c, const ss_tensor& t, int B, int L_c, CUtensorMap* 
     for (int i = 1; i < 64; ++i)
       if (c->tm[i].age < c->tm[slot].age) slot = i;
   }
-  c->tm[slot] = {t.ptr, t.stride_b, t.stride_h, t.stride_t, B, L_c, m, ++c->tm_clock};
+  c->tm[slot] = {t.ptr, t.stride_b, t.stride_h, t.stride_t, B, L_c, box_tokens, m, ++c->tm_clock};
   *out = m;
   return true;
 }
@@ -235,6 +236,8 @@ ss_status ss_create(ss_ctx** out, const ss_config* cfg, void* workspace, size_t 
   c->target_ctas = target_ctas_default();
   const char* fs = getenv("SS_SPLITS");
   c->force_splits = fs ? atoi(fs) : 0;
+  const char* ck = getenv("SS_CHUNK_KERNEL");
+  c->force_rows_kernel = (ck && strcmp(ck, "rows") == 0) || (cfg->flags & SS_FLAG_ROWS_ON_M);
 
   if (!g_encode) {
     void* fn = nullptr;
@@ -247,6 +250,7 @@ ss_status ss_create(ss_ctx** out, const ss_config* cfg, void* workspace, size_t 
   c->tc_ok = (g_encode != nullptr) && (cfg->d == 128) && !(cfg->flags & SS_FLAG_FORCE_SIMT);
   if (c->tc_ok) {
     e = ss::chunk_tc_prepare();
+    if (e == cudaSuccess) e = ss::chunk_tc_keys_prepare();
     if (e != cudaSuccess) {
       delete c;
       return SS_ERR_CUDA;
@@ -328,11 +332,18 @@ ss_status ss_verify_chunk(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c,
   const int n_tiles = (L_c + kTileKeys - 1) / kTileKeys;
   CUtensorMap tmK, tmV;
   bool tc = c->tc_ok;
-  if (tc) tc = get_tensor_map(c, K, c->B, L_c, &tmK) && get_tensor_map(c, V, c->B, L_c, &tmV);
+  // few rows per kv-head: keys ride the MMA's M axis (tiles of 128 tokens); otherwise rows do
+  const bool keys_on_m = tc && R <= 32 && !c->force_rows_kernel;
+  const int box = keys_on_m ? 128 : kTileKeys;
+  if (tc) tc = get_tensor_map(c, K, c->B, L_c, box, &tmK) && get_tensor_map(c, V, c->B, L_c, box, &tmV);
 
   ss::ChunkParams p;
   memset(&p, 0, sizeof(p));
-  if (tc) {
+  if (tc && keys_on_m) {
+    p.row_tiles = 1;
+    p.rows_per_tile = R;
+    p.groups = 1;
+  } else if (tc) {
     p.row_tiles = (R + 127) / 128;
     p.rows_per_tile = (R + p.row_tiles - 1) / p.row_tiles;
     p.groups = p.rows_per_tile <= 32 ? 4 : (p.rows_per_tile <= 64 ? 2 : 1);
@@ -349,6 +360,7 @@ ss_status ss_verify_chunk(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c,
   if (splits > (n_tiles + 1) / 2) splits = (n_tiles + 1) / 2;  // at least two tiles per split
   if (splits < 1) splits = 1;
   p.tiles_per_split = (n_tiles + splits - 1) / splits;
+  if (tc && keys_on_m) p.tiles_per_split += p.tiles_per_split & 1;  // whole 128-token tiles
   splits = (n_tiles + p.tiles_per_split - 1) / p.tiles_per_split;
   p.splits = splits;
 
@@ -381,9 +393,11 @@ ss_status ss_verify_chunk(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c,
   p.trace = c->trace_on ? c->trace : nullptr;
 
   const bool pdl = use_pdl(c);
-  cudaError_t e = tc ? ss::launch_chunk_tc(p, tmK, tmV, s, pdl) : ss::launch_chunk_simt(p, s, pdl);
+  cudaError_t e = !tc ? ss::launch_chunk_simt(p, s, pdl)
+                  : keys_on_m ? ss::launch_chunk_tc_keys(p, tmK, tmV, s, pdl)
+                              : ss::launch_chunk_tc(p, tmK, tmV, s, pdl);
   if (e != cudaSuccess) return cuda_fail(c, e);
-  c->last_kernel = tc ? "tcgen05" : "simt";
+  c->last_kernel = !tc ? "simt" : keys_on_m ? "tcgen05-keys" : "tcgen05";
   ++c->launches;
   c->splits[c->n_sets] = (uint8_t)splits;
   ++c->n_sets;

@@ -98,6 +98,9 @@ cudaError_t launch_chunk_simt(const ChunkParams& p, cudaStream_t s, bool pdl);
 cudaError_t launch_chunk_tc(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
                             cudaStream_t s, bool pdl);
 cudaError_t chunk_tc_prepare();  // one-time function attributes
+cudaError_t launch_chunk_tc_keys(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                                 cudaStream_t s, bool pdl);
+cudaError_t chunk_tc_keys_prepare();
 cudaError_t launch_local(const LocalParams& p, cudaStream_t s, bool pdl);
 cudaError_t launch_finalize(const MergeParams& p, cudaStream_t s, bool pdl);
 cudaError_t launch_fold(const MergeParams& p, cudaStream_t s);

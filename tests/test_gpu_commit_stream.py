@@ -190,14 +190,15 @@ def test_stream_round_copy_only_and_reuse():
 
 def test_trace_records_tile_loop():
     ssb = _ssb()
-    cfg = inputs.VerifyConfig("v", 0x64, 2, 8, 2, 128, 512, 8, 512, 512)
-    lens = [512, 512]
+    cfg = inputs.VerifyConfig("v", 0x64, 1, 4, 1, 128, 8192, 8, 8192, 8192)
+    lens = [8192]
     case = util.gen_case(cfg, lens, DEV)
     ctx = util.make_ctx(cfg)
     ctx.ss_trace_enable(True)
     util.gpu_case(ctx, cfg, *case)
     tr = ctx.ss_trace_read()
     ctx.ss_trace_enable(False)
-    mma = [t[1] for t in tr[1] if t[1]]
-    assert len(mma) >= 2 and all(b > a for a, b in zip(mma, mma[1:]))
+    for role in (1, 2):      # MMA issuer and softmax lane 0 stamp event 0 at the top of every tile
+        tops = [t[0] for t in tr[role] if t[0]]
+        assert len(tops) >= 2 and all(b > a for a, b in zip(tops, tops[1:]))
     ctx.close()
