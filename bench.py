@@ -48,7 +48,7 @@ def peaks():
 # DRAM bytes (read + write) per chunk-kernel launch from an ncu capture of the same kernel;
 # filled from the summaries under profiles/ (None until a capture exists for the workload).
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    # profiles/chunk_tc_kernel_c2_qwen3_8b.md: 135.33 MB read + 4.1 MB written per launch
+    # profiles/chunk_tc_keys_kernel_c2_qwen3_8b.md: 135.34 MB read + 4.06 MB written per launch
     "c2_qwen3_8b": 139.4e6,
 }
 
@@ -393,7 +393,7 @@ def main():
         probe_h = torch.empty(256 << 20, dtype=torch.uint8).pin_memory()
         probe_d = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
         best = 0.0
-        for _ in range(5):
+        for _ in range(10):
             a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
             probe_d.copy_(probe_h, non_blocking=True)
