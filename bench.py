@@ -126,13 +126,22 @@ def build_resident(cfg, lens, dev):
     return Q, chunks, K_loc, V_loc, bits
 
 
-def run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, ev_pair=None):
+def host_valid(cfg, lens, n_chunks):
+    """Host copies of every chunk call's valid lengths (scheduling hint), as ctypes arrays."""
+    return [(C.c_int32 * cfg.B)(*[max(0, min(cfg.L_c, l - j * cfg.L_c)) for l in lens])
+            for j in range(n_chunks)]
+
+
+def run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, ev_pair=None, hints=None):
     kind = ssb.SS_MASK_TREE_BITS if cfg.mask == "tree" else ssb.SS_MASK_CHAIN
     ctx.ss_verify_begin(Q, cfg.scale)
     if ev_pair:
         ev_pair[0].record()
-    for K, V, vl in chunks:
-        ctx.ss_verify_chunk(K, V, vl)
+    for j, (K, V, vl) in enumerate(chunks):
+        if hints is not None:
+            ctx.ss_verify_chunk_hinted(K, V, vl, hints[j])
+        else:
+            ctx.ss_verify_chunk(K, V, vl)
     if ev_pair:
         ev_pair[1].record()
     ctx.ss_verify_local(K_loc, V_loc, kind, bits if cfg.mask == "tree" else None)
@@ -301,6 +310,9 @@ def main():
     O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=dev)
     LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=dev)
     nbytes = kv_bytes(cfg, lens)
+    hints = host_valid(cfg, lens, len(chunks)) if len(set(lens)) > 1 else None
+    import functools
+    run = functools.partial(run_round, hints=hints)
 
     def barrier():
         ssdist.barrier(cuda=True)
@@ -310,7 +322,7 @@ def main():
         sampler.start()
 
     for _ in range(args.warmup):
-        run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE)
+        run(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE)
     barrier()
     # ---- timed region: exactly K rounds, history resident in HBM -----------------------------
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -318,7 +330,7 @@ def main():
     t_wall0 = time.time()
     e0.record()
     for _ in range(args.steps):
-        run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE)
+        run(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE)
     e1.record()
     barrier()
     t_wall1 = time.time()
@@ -341,7 +353,7 @@ def main():
             t0 = time.time()
             while time.time() - t0 < 1.2:
                 for _ in range(20):
-                    run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE)
+                    run(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE)
                 torch.cuda.synchronize()
             clocks = sampler.summary(t0, time.time())
             clocks["sampled"] = "identical rounds run right after the timed region (it was too short)"
@@ -353,7 +365,7 @@ def main():
         pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
                  for _ in range(min(args.steps, 50))]
         for p in pairs:
-            run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, ev_pair=p)
+            run(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, ev_pair=p)
         torch.cuda.synchronize()
         chunk_ms = statistics.mean(a.elapsed_time(b) for a, b in pairs) / n_chunk_calls
     peak, peak_kind = peaks()
@@ -434,7 +446,7 @@ def main():
                        "kv_bytes_per_round": nbytes,
                        "l2": "inputs larger than L2 (each round streams all history chunks, "
                              f"{nbytes / 2**20:.0f} MiB, through distinct buffers)",
-                       "overlap_chunks": not args.no_overlap},
+                       "overlap_chunks": not args.no_overlap, "host_length_hints": hints is not None},
             "rounds_per_s": world * 1e3 / ms_per_step,
             "pct_hbm_nominal_8TBps": 100.0 * value / world / 8000.0,
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,

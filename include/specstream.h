@@ -118,6 +118,15 @@ ss_status ss_verify_begin(ss_ctx* ctx, ss_tensor Q, int32_t B, int32_t T_q, floa
 ss_status ss_verify_chunk(ss_ctx* ctx, ss_tensor K, ss_tensor V, int32_t L_c,
                           const int32_t* valid_len, void* stream);
 
+/* Same as ss_verify_chunk, with a HOST copy of valid_len ([B], may be NULL) as a scheduling
+ * hint: the token splits are sized for the requests that are still active, which keeps the GPU
+ * full when most of a ragged batch has run out of history.  The device array stays
+ * authoritative for the result; a wrong hint can cost speed or, if it understates a length,
+ * drop the tokens past the hinted maximum of the batch - pass the same values. */
+ss_status ss_verify_chunk_hinted(ss_ctx* ctx, ss_tensor K, ss_tensor V, int32_t L_c,
+                                 const int32_t* valid_len, const int32_t* valid_len_host,
+                                 void* stream);
+
 /* a4. The on-GPU candidate segment: K_loc, V_loc [B, H_kv, T_loc, d].  Query i of request
  * b sees local token j iff
  *   SS_MASK_CHAIN:     j <= i + (T_loc - T_q)   (causal, inclusive; mask_bits ignored)

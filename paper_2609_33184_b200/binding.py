@@ -28,7 +28,7 @@ SS_MASK_CHAIN, SS_MASK_TREE_BITS = 0, 1
 EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "ss_verify_chunk",
            "ss_verify_local", "ss_verify_finalize", "ss_commit_gather", "ss_poll_status",
            "ss_stream_round", "ss_strerror", "ss_sizeof_stream_desc", "ss_last_cuda_error", "ss_launch_count",
-           "ss_last_chunk_kernel", "ss_trace_enable", "ss_trace_read", "ss_verify_round_static"]
+           "ss_last_chunk_kernel", "ss_trace_enable", "ss_trace_read", "ss_verify_round_static", "ss_verify_chunk_hinted"]
 
 
 class ss_config(C.Structure):
@@ -99,6 +99,8 @@ def load() -> C.CDLL:
     lib.ss_verify_begin.argtypes = [vp, ss_tensor, i32, i32, C.c_float, vp]
     lib.ss_verify_chunk.restype = C.c_int
     lib.ss_verify_chunk.argtypes = [vp, ss_tensor, ss_tensor, i32, vp, vp]
+    lib.ss_verify_chunk_hinted.restype = C.c_int
+    lib.ss_verify_chunk_hinted.argtypes = [vp, ss_tensor, ss_tensor, i32, vp, C.POINTER(C.c_int32), vp]
     lib.ss_verify_local.restype = C.c_int
     lib.ss_verify_local.argtypes = [vp, ss_tensor, ss_tensor, i32, C.c_int, vp, vp]
     lib.ss_verify_finalize.restype = C.c_int
@@ -200,6 +202,16 @@ class Context:
             assert valid_len.dtype == torch.int32 and valid_len.is_cuda
         self._check(self.lib.ss_verify_chunk(self.handle, as_ss_tensor(K), as_ss_tensor(V), L_c,
                                              _ptr(valid_len), _stream_ptr(stream)), "ss_verify_chunk")
+
+    def ss_verify_chunk_hinted(self, K: torch.Tensor, V: torch.Tensor, valid_len: torch.Tensor,
+                               valid_len_host, stream=None):
+        """valid_len_host: a ctypes int32 array (or a list of ints) with the same values as valid_len."""
+        L_c = K.shape[2]
+        if not isinstance(valid_len_host, C.Array):
+            valid_len_host = (C.c_int32 * len(valid_len_host))(*valid_len_host)
+        self._check(self.lib.ss_verify_chunk_hinted(self.handle, as_ss_tensor(K), as_ss_tensor(V), L_c,
+                                                    _ptr(valid_len), valid_len_host, _stream_ptr(stream)),
+                    "ss_verify_chunk_hinted")
 
     def ss_verify_local(self, K_loc: torch.Tensor, V_loc: torch.Tensor, mask_kind: int = SS_MASK_CHAIN,
                         mask_bits: Optional[torch.Tensor] = None, stream=None):

@@ -302,8 +302,22 @@ ss_status ss_verify_begin(ss_ctx* c, ss_tensor Q, int32_t B, int32_t T_q, float 
   return SS_OK;
 }
 
+static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, const int32_t* valid_len,
+                            const int32_t* valid_len_host, void* stream);
+
 ss_status ss_verify_chunk(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c,
                           const int32_t* valid_len, void* stream) {
+  return chunk_impl(c, K, V, L_c, valid_len, nullptr, stream);
+}
+
+ss_status ss_verify_chunk_hinted(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c,
+                                 const int32_t* valid_len, const int32_t* valid_len_host,
+                                 void* stream) {
+  return chunk_impl(c, K, V, L_c, valid_len, valid_len_host, stream);
+}
+
+static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, const int32_t* valid_len,
+                            const int32_t* valid_len_host, void* stream) {
   if (!c || !K.ptr || !V.ptr) return SS_ERR_ARG;
   if (L_c <= 0) return SS_ERR_ARG;
   if (L_c > c->cfg.max_Lc) return SS_ERR_SHAPE;
@@ -330,6 +344,19 @@ ss_status ss_verify_chunk(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c,
   const int R = c->T_q * c->G;
   const int pairs = c->B * c->cfg.H_kv;
   const int n_tiles = (L_c + kTileKeys - 1) / kTileKeys;
+  // host copy of the valid lengths (a hint): size the splits for the requests that are active
+  int active_pairs = pairs, used_tiles = n_tiles;
+  if (valid_len && valid_len_host) {
+    int active = 0, longest = 0;
+    for (int b = 0; b < c->B; ++b) {
+      int v = valid_len_host[b];
+      v = v < 0 ? 0 : (v > L_c ? L_c : v);
+      if (v > 0) ++active;
+      if (v > longest) longest = v;
+    }
+    active_pairs = (active > 0 ? active : 1) * c->cfg.H_kv;
+    used_tiles = longest > 0 ? (longest + kTileKeys - 1) / kTileKeys : 1;
+  }
   CUtensorMap tmK, tmV;
   bool tc = c->tc_ok;
   // few rows per kv-head: keys ride the MMA's M axis (tiles of 128 tokens); otherwise rows do
@@ -353,15 +380,17 @@ ss_status ss_verify_chunk(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c,
     p.groups = 1;
   }
   int splits = c->force_splits > 0 ? c->force_splits
-                                   : c->target_ctas / (pairs * p.row_tiles);
+                                   : c->target_ctas / (active_pairs * p.row_tiles);
   const int max_by_slots = c->slots_per_set / pairs;
   if (splits > max_by_slots) splits = max_by_slots;
   if (splits > kMaxSplits) splits = kMaxSplits;
-  if (splits > (n_tiles + 1) / 2) splits = (n_tiles + 1) / 2;  // at least two tiles per split
+  // tensor-core CTAs amortise their set-up over at least 256 tokens; CUDA-core CTAs take one tile
+  const int min_tiles = tc ? 4 : 1;
+  if (splits > (used_tiles + min_tiles - 1) / min_tiles) splits = (used_tiles + min_tiles - 1) / min_tiles;
   if (splits < 1) splits = 1;
-  p.tiles_per_split = (n_tiles + splits - 1) / splits;
+  p.tiles_per_split = (used_tiles + splits - 1) / splits;
   if (tc && keys_on_m) p.tiles_per_split += p.tiles_per_split & 1;  // whole 128-token tiles
-  splits = (n_tiles + p.tiles_per_split - 1) / p.tiles_per_split;
+  splits = (used_tiles + p.tiles_per_split - 1) / p.tiles_per_split;
   p.splits = splits;
 
   p.Q = (const __nv_bfloat16*)c->Q.ptr;

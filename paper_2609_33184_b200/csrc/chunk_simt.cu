@@ -32,6 +32,7 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const ChunkParams 
   const int row0 = rt * kRows;
   const int nrows = min(kRows, p.R - row0);
 
+  const bool chain_cta = (blockIdx.x | blockIdx.y | blockIdx.z) == 0;
   if (p.wait_first) pdl_wait_prior();
   pdl_launch_dependents();
 
@@ -52,7 +53,7 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const ChunkParams 
 
   if (tok0 >= tok1) {  // nothing visible here: identity state
     if (tid < nrows) out_ml[tid] = make_float2(-INFINITY, 0.f);
-    if (!p.wait_first) pdl_wait_prior();
+    if (!p.wait_first && chain_cta) pdl_wait_prior();
     return;
   }
 
@@ -203,7 +204,9 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const ChunkParams 
         *reinterpret_cast<const float4*>(&red[r * D + c4 * 4]);
   }
   if (tid < nrows) out_ml[tid] = make_float2(m_s[tid], l_s[tid]);
-  if (!p.wait_first) pdl_wait_prior();  // keep completion order along the stream
+  // Completion order along the stream: one CTA of this grid waits for the previous grid, so
+  // this grid cannot complete before it (the other CTAs leave at once and free their SM slot).
+  if (!p.wait_first && chain_cta) pdl_wait_prior();
 }
 
 }  // namespace

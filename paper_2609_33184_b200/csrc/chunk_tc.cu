@@ -167,6 +167,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   const int r_pad = 128 / p.groups;
   unsigned long long* tr = (blockIdx.x | blockIdx.y | blockIdx.z) ? nullptr : p.trace;
 
+  const bool chain_cta = (blockIdx.x | blockIdx.y | blockIdx.z) == 0;
   if (p.wait_first) pdl_wait_prior();
   pdl_launch_dependents();
 
@@ -188,7 +189,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
 
   if (n_tiles == 0) {  // nothing visible here: identity state, no tensor memory taken
     if (tid < nrows) out_ml[tid] = make_float2(-INFINITY, 0.f);
-    if (!p.wait_first) pdl_wait_prior();
+    if (!p.wait_first && chain_cta) pdl_wait_prior();
     return;
   }
 
@@ -480,7 +481,9 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols)
                  : "memory");
   }
-  if (!p.wait_first) pdl_wait_prior();  // keep completion order along the stream
+  // Completion order along the stream: one CTA of this grid waits for the previous grid, so
+  // this grid cannot complete before it (the other CTAs leave at once and free their SM slot).
+  if (!p.wait_first && chain_cta) pdl_wait_prior();
 }
 
 }  // namespace

@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) local_kernel(const LocalPar
     else
       *reinterpret_cast<float2*>(out) = make_float2(acc[0], acc[1]);
   }
-  pdl_wait_prior();
+  if (blockIdx.x == 0) pdl_wait_prior();  // one CTA keeps the completion order along the stream
 }
 
 // ---------------------------------------------------------------------------------------

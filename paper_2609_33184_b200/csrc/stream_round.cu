@@ -105,8 +105,8 @@ static ss_status stream_round_impl(ss_ctx* ctx, const ss_stream_desc* d, ss_stre
     if (!d->copy_only) {
       ss_tensor K = {d->stage_k[buf], (int64_t)H_kv * Ls * hd, Ls * hd, hd};
       ss_tensor V = {d->stage_v[buf], (int64_t)H_kv * Ls * hd, Ls * hd, hd};
-      SS_ST(ss_verify_chunk(ctx, K, V, (int32_t)Ls, d->valid_len_dev + (int64_t)f * B,
-                            r.attn_stream));
+      SS_ST(ss_verify_chunk_hinted(ctx, K, V, (int32_t)Ls, d->valid_len_dev + (int64_t)f * B,
+                                   d->valid_len_host + (int64_t)f * B, r.attn_stream));
       ++calls;
     }
     SS_CK(cudaEventRecord(r.ev_free[buf], r.attn_stream));

@@ -35,8 +35,9 @@ def _resident(name, n_samples):
                       flags=ssb.SS_FLAG_OVERLAP_CHUNKS)
     O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
     LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
+    hints = bench.host_valid(cfg, lens, len(chunks)) if len(set(lens)) > 1 else None   # as bench.py does
     for _ in range(2):
-        bench.run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE)
+        bench.run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, hints=hints)
     torch.cuda.synchronize()
     st, dev_bits = ctx.ss_poll_status()
     assert st == 0, dev_bits

@@ -205,3 +205,24 @@ def test_bad_valid_len_sets_status_and_is_clamped():
     st, b = ctx.ss_poll_status()
     assert st == 0 and b == 0  # cleared
     ctx.close()
+
+
+def test_hinted_chunk_calls_match_unhinted():
+    # host copies of valid_len only change the split sizes, never the result's correctness
+    cfg = inputs.VerifyConfig("v", 0x5C, 6, 8, 2, 128, 512, 8, 10, 1500)
+    lens = [1500, 10, 700, 513, 0, 1024]
+    case = util.gen_case(cfg, lens, DEV)
+    Q, chunks, K_loc, V_loc, bits = case
+    ref = util.oracle_case(cfg, lens, *case)
+    import bench
+    hints = bench.host_valid(cfg, lens, len(chunks))
+    ssb = _ssb()
+    ctx = util.make_ctx(cfg)
+    O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
+    LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
+    bench.run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, hints=hints)
+    torch.cuda.synchronize()
+    st, dev_bits = ctx.ss_poll_status()
+    assert st == 0, dev_bits
+    util.compare(cfg, O, LSE, ref)
+    ctx.close()
