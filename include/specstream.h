@@ -84,8 +84,8 @@ typedef struct {
  * produced by a copy / an event the stream waited on - not by a kernel enqueued on the
  * same stream between two ss_ calls. */
 #define SS_FLAG_OVERLAP_CHUNKS 2u
-/* Use the rows-on-M tensor-core chunk kernel even when the kv-head has <= 32 query rows
- * (where the keys-on-M kernel is the default).  For cross-checks. */
+/* Use the tensor-core chunk kernel that puts the query rows on the MMA's M axis instead of
+ * the default one that puts the keys there.  For cross-checks. */
 #define SS_FLAG_ROWS_ON_M 4u
 
 typedef struct {

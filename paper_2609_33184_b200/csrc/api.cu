@@ -359,16 +359,19 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   }
   CUtensorMap tmK, tmV;
   bool tc = c->tc_ok;
-  // few rows per kv-head: keys ride the MMA's M axis (tiles of 128 tokens); otherwise rows do
-  const bool keys_on_m = tc && R <= 32 && !c->force_rows_kernel;
+  // up to 64 rows per kv-head the keys ride the MMA's M axis (tiles of 128 tokens); with more
+  // rows the kernel with the rows on M is faster (measured); SS_FLAG_ROWS_ON_M forces it
+  const char* ck = getenv("SS_CHUNK_KERNEL");
+  const bool force_keys = ck && strcmp(ck, "keys") == 0;
+  const bool keys_on_m = tc && !c->force_rows_kernel && (R <= 64 || force_keys);
   const int box = keys_on_m ? 128 : kTileKeys;
   if (tc) tc = get_tensor_map(c, K, c->B, L_c, box, &tmK) && get_tensor_map(c, V, c->B, L_c, box, &tmV);
 
   ss::ChunkParams p;
   memset(&p, 0, sizeof(p));
   if (tc && keys_on_m) {
-    p.row_tiles = 1;
-    p.rows_per_tile = R;
+    p.row_tiles = (R + 127) / 128;
+    p.rows_per_tile = R < 128 ? R : 128;
     p.groups = 1;
   } else if (tc) {
     p.row_tiles = (R + 127) / 128;
@@ -379,14 +382,35 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
     p.row_tiles = (R + 31) / 32;
     p.groups = 1;
   }
-  int splits = c->force_splits > 0 ? c->force_splits
-                                   : c->target_ctas / (active_pairs * p.row_tiles);
-  const int max_by_slots = c->slots_per_set / pairs;
-  if (splits > max_by_slots) splits = max_by_slots;
-  if (splits > kMaxSplits) splits = kMaxSplits;
   // tensor-core CTAs amortise their set-up over at least 256 tokens; CUDA-core CTAs take one tile
   const int min_tiles = tc ? 4 : 1;
-  if (splits > (used_tiles + min_tiles - 1) / min_tiles) splits = (used_tiles + min_tiles - 1) / min_tiles;
+  int max_splits = c->slots_per_set / pairs;
+  if (max_splits > kMaxSplits) max_splits = kMaxSplits;
+  if (max_splits > (used_tiles + min_tiles - 1) / min_tiles) max_splits = (used_tiles + min_tiles - 1) / min_tiles;
+  if (max_splits < 1) max_splits = 1;
+  const int ctas1 = active_pairs * p.row_tiles;  // CTAs with work when splits = 1
+  int splits;
+  if (c->force_splits > 0) {
+    splits = c->force_splits;
+  } else if (tc && keys_on_m && R > 32) {
+    // one CTA per SM and no co-residency with the next launch: pick the split count whose CTA
+    // count fills whole waves of SMs best (smallest such count: fewer partial states)
+    double best = 0.0;
+    splits = 1;
+    for (int sp = 1; sp <= max_splits; ++sp) {
+      const int ctas = ctas1 * sp;
+      const int waves = (ctas + ss::kNumSM - 1) / ss::kNumSM;
+      const double eff = (double)ctas / ((double)waves * ss::kNumSM);
+      if (eff > best + 0.05) {
+        best = eff;
+        splits = sp;
+      }
+    }
+  } else {
+    // about one CTA per SM: a second CTA per SM comes from the next (overlapping) launch
+    splits = c->target_ctas / ctas1;
+  }
+  if (splits > max_splits) splits = max_splits;
   if (splits < 1) splits = 1;
   p.tiles_per_split = (used_tiles + splits - 1) / splits;
   if (tc && keys_on_m) p.tiles_per_split += p.tiles_per_split & 1;  // whole 128-token tiles

@@ -95,14 +95,15 @@ __device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_o, int c0,
   for (int q = 0; q < NC / 16; ++q) tmem_ld16(t_s + c0 + q * 16, raw[q]);
   tc_wait_ld();
   float s[NC];
-  float mx = -INFINITY;
+  float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // independent chains
 #pragma unroll
   for (int c = 0; c < NC; ++c) {
     float v = __uint_as_float(raw[c / 16][c % 16]) * scale_log2;
     if (c0 + c >= n_valid) v = -INFINITY;
     s[c] = v;
-    mx = fmaxf(mx, v);
+    mx4[c & 3] = fmaxf(mx4[c & 3], v);
   }
+  const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
   float f = 1.f;
   if (mx > m + kRescaleThreshold) {  // also the first finite maximum (m = -inf)
     f = (m == -INFINITY) ? 0.f : exp2f(m - mx);
@@ -124,15 +125,15 @@ __device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_o, int c0,
   }
   const float m_use = (m == -INFINITY) ? 0.f : m;
   uint32_t pk[NC / 16][8];
-  float sum = 0.f;
+  float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
   for (int c = 0; c < NC; c += 2) {
-    const float p0 = exp2f(s[c] - m_use), p1 = exp2f(s[c + 1] - m_use);
-    sum += p0 + p1;
+    const float p0 = ex2_ftz(s[c] - m_use), p1 = ex2_ftz(s[c + 1] - m_use);
+    sum4[(c >> 1) & 3] += p0 + p1;
     __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);  // low half = even key
     pk[c / 16][(c / 2) % 8] = *reinterpret_cast<uint32_t*>(&h);
   }
-  l += sum;
+  l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
   // c0 is uniform across a warp; dispatching on it keeps pk[] in registers
   if (NC == 64) {
     store_p<NC, 0>(t_s, pk);
@@ -222,7 +223,8 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       ctl->abort = 0;
       fence_barrier_init();
       // the first tiles go out before the rest of the CTA is set up
-      const uint64_t pol = l2_evict_first_policy();
+      // streamed once: evict first; shared by the row groups of a kv-head through L2: keep
+      const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
       for (int it = 0; it < n_pre; ++it) issue_tile(it, pol);
     }
     __syncwarp();
@@ -257,7 +259,8 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   if (warp == 4) {
     // ===== TMA producer =====
     if (lane == 0) {
-      const uint64_t pol = l2_evict_first_policy();
+      // streamed once: evict first; shared by the row groups of a kv-head through L2: keep
+      const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
       int issued = n_pre;
       for (int it = n_pre; it < n_tiles; ++it) {
         const int s = it % kStages;

@@ -1,36 +1,40 @@
-// Tensor-core chunk attention for few rows per kv-head (R <= 32): keys on the MMA's M axis.
+// Tensor-core chunk attention with the keys on the MMA's M axis.
 //
-// With R = T_q * G <= 32 query rows per kv-head, putting the rows on the 128-wide M axis wastes
-// three quarters of every MMA.  Here the contraction is transposed instead:
+// The rows of a kv-head (T_q candidate queries x G query heads) are few compared with the
+// 128-wide M axis of tcgen05.mma, so the contraction is transposed:
 //
-//   S^T = K Q^T   M = 128 keys of the tile, N = 32 rows, K = d = 128   (8 x k16, smem x smem)
-//   O^T = V^T P^T M = 128 head dims,        N = 32 rows, K = 128 keys  (8 x k16, smem x smem)
+//   S^T = K Q^T   M = 128 keys of the tile, N = rows (16..128), K = d = 128   (8 x k16)
+//   O^T = V^T P^T M = 128 head dims,        N = rows,           K = 128 keys  (8 x k16)
 //
-// so the tensor work is proportional to the rows that exist.  One CTA = one (request, kv-head,
-// token split); 192 threads: warps 0-3 softmax, warp 4 TMA producer, warp 5 MMA issuer.
+// and the tensor work is proportional to the rows that exist (no padding of M).  One CTA =
+// one (request, kv-head, token split, group of <= 128 rows); kv-heads with more rows use
+// several row groups (their CTAs are adjacent in the grid and share K/V through L2).
 //
-//  * K and V tiles of 128 tokens (two [128][64] bf16 boxes each, 128-byte swizzle) go through
-//    a ring of three 32 KB units in the order K0 V0 K1 V1 ...; a K unit is released when its
-//    score MMAs retire, a V unit after its output MMAs.  V^T is fed as an MN-major A operand
-//    straight from the [token][d] tile.
-//  * S^T sits in tensor memory, double buffered (2 x 32 columns): thread L of the softmax
-//    warps owns TMEM lane L = key L of the tile and sees that key's scores against all rows.
-//    Ragged tails are a per-thread select (key >= valid -> weight 0).
+//  * Warps: 4*WG softmax warps, one TMA producer warp, one MMA issuer warp.
+//  * K and V tiles of 128 tokens (two [128][64] bf16 boxes each, 128-byte swizzle, evict-first)
+//    go through a ring of 32 KB units in the order K0 V0 K1 V1 ...; a K unit is released when
+//    its score MMAs retire, a V unit after its output MMAs.  V^T is fed as an MN-major A
+//    operand straight from the [token][d] tile.
+//  * S^T sits in tensor memory, double buffered: a softmax thread owns TMEM lane L = key L of
+//    the tile and a block of the score columns (= rows); with WG = 2 two threads share a lane
+//    and split the columns.  Ragged tails are a per-thread select (key >= valid -> weight 0).
 //  * The row reference m[r] is shared by all keys, so it cannot follow each tile's maximum
-//    without a cross-lane reduction.  It is kept lazily: weights are exp2(x - m[r]) with the
-//    current m[r]; only if some x - m[r] exceeds 16 (always on the first tile, where
-//    m = -inf) do the 128 threads agree (one named barrier per tile) to take the exact tile
-//    maxima (warp shuffles + shared memory), raise m, and rescale O^T and the row sums.
-//    Any common reference gives the same a / l (Eq. 17), so this is exact.
-//  * Row sums l[r] accumulate per thread (per key lane) in registers and are reduced across
-//    the 128 lanes once, when the CTA ends.
-//  * P^T goes to shared memory as the MN-major B operand (unswizzled 8x8 core matrices: each
-//    thread writes four 16-byte pieces, a warp's pieces are contiguous).
-//  * O^T accumulates in tensor memory (32 columns); at the end thread L holds head dim L of
-//    every row and writes a[r][L], coalesced over L.
+//    without a cross-lane reduction.  It is kept lazily: weights are exp2(s - m[r]) with the
+//    current m[r]; only if some s - m[r] exceeds 16 (always on the first tile, m = -inf) do
+//    the softmax threads agree (one named barrier per tile) to take the exact tile maxima
+//    (warp shuffles + shared memory), raise m, and rescale O^T and the row sums.  Any common
+//    reference gives the same a / l (Eq. 17), so this is exact.
+//  * Row sums l[r] accumulate per thread in registers and are reduced across the 128 key
+//    lanes once, when the CTA ends.
+//  * P^T goes to shared memory as the MN-major B operand (unswizzled 8x8 core matrices: a
+//    thread writes 16-byte pieces, a warp's pieces are contiguous).
+//  * O^T accumulates in tensor memory; at the end a thread holds head dim L of its rows and
+//    writes a[r][L], coalesced over L.
 //
-// 112 KB of shared memory and 128 TMEM columns per CTA: two CTAs per SM, so one CTA's ramp-up
-// and tail overlap the other's steady state (also across consecutive chunk kernels).
+// Rows <= 32: 3 ring units, 113 KB shared memory, 128 TMEM columns -> two CTAs per SM, so one
+// CTA's ramp-up and tail overlap the other's steady state (also across consecutive kernels).
+// Rows up to 64 / 128: 5 ring units, one CTA per SM, 8 / 16 softmax warps (the latency of
+// tensor-memory loads is hidden by warps, not by holding more columns per thread).
 // Every mbarrier wait is bounded; on expiry the CTA raises SS_DEV_WAIT_EXPIRED, lets its own
 // copies land (bounded), frees its tensor memory and returns.
 #include <cstddef>
@@ -43,56 +47,65 @@ namespace {
 
 using namespace ss::tc;
 
-constexpr int kThreads = 192;
 constexpr int kD = 128;
-constexpr int kKeys = 128;                     // keys per tile = MMA M
-constexpr int kN = 32;                         // padded query rows = MMA N
-constexpr int kUnits = 3;                      // ring of K / V tiles
-constexpr int kHalf = kKeys * 64 * 2;          // 16 KB: [128 keys][64 d] bf16
-constexpr int kUnitBytes = 2 * kHalf;          // 32 KB: one K tile or one V tile
-constexpr int kQHalf = kN * 64 * 2;            // 4 KB: [32 rows][64 d]
-constexpr int kQBytes = 2 * kQHalf;            // 8 KB
-constexpr int kPBytes = kKeys * kN * 2;        // 8 KB: P^T
-constexpr int kOffQ = kUnits * kUnitBytes;     // 96 KB
-constexpr int kOffP = kOffQ + kQBytes;
-constexpr int kOffCtl = kOffP + kPBytes;       // 112 KB
-constexpr int kCtlBytes = 1024;
-constexpr int kSmemTotal = kOffCtl + kCtlBytes;
-constexpr uint32_t kTmemCols = 128;
-constexpr uint32_t kColS = 0, kColO = 2 * kN;  // S^T buffers at 0 and 32, O^T at 64
+constexpr int kKeys = 128;                  // keys per tile = MMA M
+constexpr int kHalf = kKeys * 64 * 2;       // 16 KB: [128 keys][64 d] bf16
+constexpr int kUnitBytes = 2 * kHalf;       // 32 KB: one K tile or one V tile
 constexpr float kLazyThreshold = 16.f;
 
-struct Ctl {
-  uint64_t ufull[kUnits], uempty[kUnits];
+template <int N>
+struct alignas(16) Ctl {
+  uint64_t ufull[8], uempty[8];
   uint64_t sfull[2], pready, pfree;
   uint32_t tmem_base;
   volatile uint32_t abort;
   volatile uint32_t flag[3];
-  alignas(16) float m_ref[kN];  // read as float4
-  alignas(16) float smax[4][kN];
+  alignas(16) float m_ref[N];     // read as float4
+  alignas(16) float smax[4][N];   // per lane quadrant
 };
-static_assert(offsetof(Ctl, m_ref) % 16 == 0, "m_ref is read with 16-byte loads");
-static_assert(sizeof(Ctl) <= kCtlBytes, "control block");
 
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Ctl* ctl, uint32_t* status) {
-  return mbar_wait_abortable(bar, parity, &ctl->abort, status);
-}
+// NC = score columns per softmax thread, WG = softmax warpgroups (threads sharing a TMEM lane),
+// UNITS = ring units.  N = NC * WG is the widest row group the instantiation takes.
+template <int NC, int WG, int UNITS>
+struct Cfg {
+  static constexpr int N = NC * WG;
+  static constexpr int kSoft = 128 * WG;              // softmax threads
+  static constexpr int kThreads = kSoft + 64;
+  static constexpr int kQHalf = N * 64 * 2;           // [N rows][64 d]
+  static constexpr int kOffQ = UNITS * kUnitBytes;
+  static constexpr int kOffP = kOffQ + 2 * kQHalf;
+  static constexpr int kOffCtl = kOffP + kKeys * N * 2;
+  static constexpr int kCtlBytes = (sizeof(Ctl<N>) + 1023) / 1024 * 1024;
+  static constexpr int kSmem = kOffCtl + kCtlBytes;
+  static constexpr uint32_t kTmemCols = (3 * N <= 128) ? 128 : (3 * N <= 256 ? 256 : 512);
+  static constexpr uint32_t kColO = 2 * N;            // S^T buffers at 0 and N, O^T at 2N
+  static constexpr int kMinBlocks = (kSmem <= 113 * 1024 && kTmemCols <= 256) ? 2 : 1;
+  static_assert(kSmem <= 227 * 1024, "shared memory");
+  static_assert(NC % 16 == 0 && UNITS <= 8, "shape");
+};
+
 __device__ __forceinline__ void trace(unsigned long long* tr, int role, int it, int ev) {
   if (tr && it < kTraceTiles) tr[(role * kTraceTiles + it) * 8 + ev] = clock64();
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+template <int NC, int WG, int UNITS>
+__global__ void __launch_bounds__(Cfg<NC, WG, UNITS>::kThreads, Cfg<NC, WG, UNITS>::kMinBlocks)
 chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
                      const __grid_constant__ CUtensorMap tmV) {
+  using C = Cfg<NC, WG, UNITS>;
+  constexpr int N = C::N;
   extern __shared__ __align__(1024) uint8_t smem[];
-  Ctl* ctl = reinterpret_cast<Ctl*>(smem + kOffCtl);
-  uint8_t* q_s = smem + kOffQ;
-  uint8_t* p_s = smem + kOffP;
+  Ctl<N>* ctl = reinterpret_cast<Ctl<N>*>(smem + C::kOffCtl);
+  uint8_t* q_s = smem + C::kOffQ;
+  uint8_t* p_s = smem + C::kOffP;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int split = blockIdx.x;
+  const int rt = blockIdx.x % p.row_tiles;
+  const int split = blockIdx.x / p.row_tiles;
   const int kvh = blockIdx.y, b = blockIdx.z;
-  const int nrows = p.R;  // <= kN
+  const int row0 = rt * p.rows_per_tile;
+  const int nrows = min(p.rows_per_tile, p.R - row0);  // <= N
+  const int n_mma = (nrows + 15) & ~15;                 // MMA N of this CTA
   unsigned long long* tr = (blockIdx.x | blockIdx.y | blockIdx.z) ? nullptr : p.trace;
 
   const bool chain_cta = (blockIdx.x | blockIdx.y | blockIdx.z) == 0;
@@ -113,8 +126,8 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
   const int n_tiles = (tok1 > tok0) ? (tok1 - tok0 + kKeys - 1) / kKeys : 0;
 
   const size_t slot = ((size_t)split * p.B + b) * p.H_kv + kvh;
-  float2* out_ml = p.part_ml + slot * p.R_stride;
-  float* out_a = p.part_a + slot * p.R_stride * kD;
+  float2* out_ml = p.part_ml + slot * p.R_stride + row0;
+  float* out_a = p.part_a + (slot * p.R_stride + row0) * kD;
 
   if (n_tiles == 0 || (smem_u32(smem) & 1023u)) {
     // nothing visible here (identity state, no tensor memory taken); a misaligned shared
@@ -124,56 +137,65 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
     if (!p.wait_first && chain_cta) pdl_wait_prior();
     return;
   }
+  auto mwait = [&](uint64_t* bar, uint32_t parity) {
+    return mbar_wait_abortable(bar, parity, &ctl->abort, p.status);
+  };
 
   // ---- set-up ------------------------------------------------------------------------------
-  // use j of the ring: K of tile t is j = 2t, V of tile t is j = 2t + 1; unit j % 3
+  // use j of the ring: K of tile t is j = 2t, V of tile t is j = 2t + 1; unit j % UNITS
   auto issue_use = [&](int j, uint64_t pol) {
-    const int u = j % kUnits;
+    const int u = j % UNITS;
     const int tok = tok0 + (j >> 1) * kKeys;
     const uint32_t dst = smem_u32(smem + u * kUnitBytes);
-    const CUtensorMap* tm = (j & 1) ? &tmV : &tmK;
     mbar_expect_tx(&ctl->ufull[u], kUnitBytes);
-    tma_load_4d(dst, tm, 0, tok, kvh, b, &ctl->ufull[u], pol);
-    tma_load_4d(dst + kHalf, tm, 64, tok, kvh, b, &ctl->ufull[u], pol);
+    if (j & 1) {  // (no runtime-selected pointer: the tensor maps stay in the parameter space)
+      tma_load_4d(dst, &tmV, 0, tok, kvh, b, &ctl->ufull[u], pol);
+      tma_load_4d(dst + kHalf, &tmV, 64, tok, kvh, b, &ctl->ufull[u], pol);
+    } else {
+      tma_load_4d(dst, &tmK, 0, tok, kvh, b, &ctl->ufull[u], pol);
+      tma_load_4d(dst + kHalf, &tmK, 64, tok, kvh, b, &ctl->ufull[u], pol);
+    }
   };
   const int n_uses = 2 * n_tiles;
-  const int n_pre = min(n_uses, kUnits);
-  if (warp == 4) {
+  const int n_pre = min(n_uses, UNITS);
+  constexpr int kProducerWarp = 4 * WG, kMmaWarp = 4 * WG + 1;
+  if (warp == kProducerWarp) {
     if (lane == 0) {
-      for (int u = 0; u < kUnits; ++u) {
+      for (int u = 0; u < UNITS; ++u) {
         mbar_init(&ctl->ufull[u], 1);
         mbar_init(&ctl->uempty[u], 1);
       }
       mbar_init(&ctl->sfull[0], 1);
       mbar_init(&ctl->sfull[1], 1);
-      mbar_init(&ctl->pready, 128);
+      mbar_init(&ctl->pready, C::kSoft);
       mbar_init(&ctl->pfree, 1);
       ctl->abort = 0;
       ctl->flag[0] = ctl->flag[1] = ctl->flag[2] = 0;
       fence_barrier_init();
-      const uint64_t pol = l2_evict_first_policy();
+      // streamed once: evict first; shared by the row groups of a kv-head through L2: keep
+      const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
       for (int j = 0; j < n_pre; ++j) issue_use(j, pol);  // first loads before the rest is set up
     }
     __syncwarp();
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                      smem_u32(&ctl->tmem_base)),
-                 "r"(kTmemCols)
+                 "r"(C::kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  } else if (warp < 4) {
+  } else if (warp < 4 * WG) {
     // Q rows -> shared memory as the K-major B operand (128-byte swizzle), zero padding rows
-    for (int i = tid; i < kN * (kD / 8); i += 128) {
+    for (int i = tid; i < n_mma * (kD / 8); i += C::kSoft) {
       const int n = i / (kD / 8), c8 = i % (kD / 8);
       uint4 raw = make_uint4(0, 0, 0, 0);
       if (n < nrows) {
-        const int g = n / p.T_q, t = n % p.T_q;
+        const int rg = row0 + n, g = rg / p.T_q, t = rg % p.T_q;
         raw = *reinterpret_cast<const uint4*>(p.Q + b * p.q_sb + (int64_t)(kvh * p.G + g) * p.q_sh +
                                               t * p.q_st + c8 * 8);
       }
       const int half = c8 >> 3, j = c8 & 7;
-      *reinterpret_cast<uint4*>(q_s + half * kQHalf + n * 128 + ((j ^ (n & 7)) << 4)) = raw;
+      *reinterpret_cast<uint4*>(q_s + half * C::kQHalf + n * 128 + ((j ^ (n & 7)) << 4)) = raw;
     }
-    if (tid < kN) ctl->m_ref[tid] = -INFINITY;
+    if (tid < N) ctl->m_ref[tid] = -INFINITY;
     fence_proxy_async();
   }
   tc_fence_before();
@@ -182,16 +204,17 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
   const uint32_t tmem = ctl->tmem_base;
   unsigned long long* trl = lane == 0 ? tr : nullptr;
 
-  if (warp == 4) {
+  if (warp == kProducerWarp) {
     // ===== TMA producer =====
     if (lane == 0) {
-      const uint64_t pol = l2_evict_first_policy();
+      // streamed once: evict first; shared by the row groups of a kv-head through L2: keep
+      const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
       int issued = n_pre;
       for (int j = n_pre; j < n_uses; ++j) {
-        const int u = j % kUnits;
-        const uint32_t ph = (j / kUnits) & 1;
+        const int u = j % UNITS;
+        const uint32_t ph = (j / UNITS) & 1;
         trace(tr, 0, j >> 1, (j & 1) * 2);
-        if (!mbar_wait(&ctl->uempty[u], ph ^ 1, ctl, p.status)) break;
+        if (!mwait(&ctl->uempty[u], ph ^ 1)) break;
         trace(tr, 0, j >> 1, (j & 1) * 2 + 1);
         issue_use(j, pol);
         issued = j + 1;
@@ -199,34 +222,33 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
       if (ctl->abort) {
         // let the copies this thread started land before the CTA leaves (bounded)
         const unsigned long long t0 = gtime_ns();
-        for (int j = max(0, issued - kUnits); j < issued; ++j)
-          while (!mbar_try_wait(&ctl->ufull[j % kUnits], (j / kUnits) & 1) &&
-                 gtime_ns() - t0 < kWaitNs) {
+        for (int j = max(0, issued - UNITS); j < issued; ++j)
+          while (!mbar_try_wait(&ctl->ufull[j % UNITS], (j / UNITS) & 1) && gtime_ns() - t0 < kWaitNs) {
           }
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == kMmaWarp) {
     // ===== MMA issuer: the whole warp walks the loop, one elected lane issues =====
-    constexpr uint32_t idesc_qk = make_idesc_major(128, kN, false, false);
-    constexpr uint32_t idesc_pv = make_idesc_major(128, kN, true, true);
+    const uint32_t idesc_qk = make_idesc_major(128, n_mma, false, false);
+    const uint32_t idesc_pv = make_idesc_major(128, n_mma, true, true);
     const bool leader = elect_one();
     const uint32_t base = smem_u32(smem);
     const uint32_t q_addr = smem_u32(q_s), p_addr = smem_u32(p_s);
     auto issue_qk = [&](int t) {  // S^T[t & 1] = K(t) Q^T
-      const uint32_t k_addr = base + ((2 * t) % kUnits) * kUnitBytes;
+      const uint32_t k_addr = base + ((2 * t) % UNITS) * kUnitBytes;
       if (leader) {
 #pragma unroll
         for (int kk = 0; kk < kD / 16; ++kk) {
           const uint32_t off = (kk & 3) * 32;
-          mma_ss(tmem + kColS + (t & 1) * kN, desc_kmajor(k_addr + (kk >> 2) * kHalf + off),
-                 desc_kmajor(q_addr + (kk >> 2) * kQHalf + off), idesc_qk, kk > 0);
+          mma_ss(tmem + (t & 1) * N, desc_kmajor(k_addr + (kk >> 2) * kHalf + off),
+                 desc_kmajor(q_addr + (kk >> 2) * C::kQHalf + off), idesc_qk, kk > 0);
         }
-        tc_commit(&ctl->uempty[(2 * t) % kUnits]);
+        tc_commit(&ctl->uempty[(2 * t) % UNITS]);
         tc_commit(&ctl->sfull[t & 1]);
       }
       __syncwarp();
     };
-    bool ok = mbar_wait(&ctl->ufull[0], 0, ctl, p.status);
+    bool ok = mwait(&ctl->ufull[0], 0);
     if (ok) {
       tc_fence_after();
       issue_qk(0);
@@ -237,7 +259,7 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
         // scores of the next tile go out first: its softmax overlaps this tile's output MMAs.
         // S^T[(t+1) & 1] was last read for tile t-1, whose pready was awaited in iteration t-1.
         const int j = 2 * (t + 1);
-        ok = mbar_wait(&ctl->ufull[j % kUnits], (j / kUnits) & 1, ctl, p.status);
+        ok = mwait(&ctl->ufull[j % UNITS], (j / UNITS) & 1);
         if (!ok) break;
         trace(trl, 1, t, 1);
         tc_fence_after();
@@ -245,192 +267,251 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
         trace(trl, 1, t, 2);
       }
       const int jv = 2 * t + 1;
-      ok = mbar_wait(&ctl->pready, t & 1, ctl, p.status);
+      ok = mwait(&ctl->pready, t & 1);
       trace(trl, 1, t, 3);
-      ok = ok && mbar_wait(&ctl->ufull[jv % kUnits], (jv / kUnits) & 1, ctl, p.status);
+      ok = ok && mwait(&ctl->ufull[jv % UNITS], (jv / UNITS) & 1);
       if (!ok) break;
       trace(trl, 1, t, 4);
       tc_fence_after();
-      const uint32_t v_addr = base + (jv % kUnits) * kUnitBytes;
+      const uint32_t v_addr = base + (jv % UNITS) * kUnitBytes;
       if (leader) {
 #pragma unroll
         for (int kk = 0; kk < kKeys / 16; ++kk) {
           // A = V^T: MN-major, 64 head dims (128 bytes) per token row, 8-token atoms 1024 bytes
           // apart, the other 64 head dims one half-tile away.  B = P^T: plain 8x8 core matrices.
-          mma_ss(tmem + kColO, desc_mnmajor(v_addr + kk * 2048, kHalf),
-                 desc_mnmajor_plain(p_addr + kk * 256, 128, kKeys * 16), idesc_pv,
-                 (t > 0 || kk > 0));
+          mma_ss(tmem + C::kColO, desc_mnmajor(v_addr + kk * 2048, kHalf),
+                 desc_mnmajor_plain(p_addr + kk * 256, 128, kKeys * 16), idesc_pv, (t > 0 || kk > 0));
         }
-        tc_commit(&ctl->uempty[jv % kUnits]);
+        tc_commit(&ctl->uempty[jv % UNITS]);
         tc_commit(&ctl->pfree);
       }
       __syncwarp();
       trace(trl, 1, t, 5);
     }
   } else {
-    // ===== softmax warps: thread L = TMEM lane L = key L of the tile =====
+    // ===== softmax warps: TMEM lane L = key L of the tile; columns [c0, c0 + cn) = rows =====
     // A wait that gives up makes the whole warp `dead`: it keeps walking the loop and the
     // named barriers (so nobody is left waiting) but touches nothing else.
-    const int L = tid;
-    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    // tensor-memory loads in flight per wait: with 16 softmax warps the load latency is hidden
+    // by the other warps and registers are scarce; with fewer warps two loads go out together
+    constexpr int kBatch = (WG >= 4) ? 1 : 2;
+    const int L = (warp & 3) * 32 + lane;
+    const int cg = (WG == 1) ? 0 : (warp >> 2);                // column group (0..WG-1)
+    const int cpg = ((n_mma / WG) + 15) & ~15;                 // columns per group
+    const int c0 = cg * cpg;
+    const int cn = max(0, min(cpg, n_mma - c0));               // multiple of 16, <= NC
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     bool dead = false;
     auto wait = [&](uint64_t* bar, uint32_t parity) {
-      if (!dead && !mbar_wait(bar, parity, ctl, p.status)) dead = true;
+      if (!dead && !mwait(bar, parity)) dead = true;
       dead = __any_sync(0xffffffffu, dead);
     };
-    float lsum[kN];
+    float lsum[NC];
 #pragma unroll
-    for (int r = 0; r < kN; ++r) lsum[r] = 0.f;
+    for (int r = 0; r < NC; ++r) lsum[r] = 0.f;
     for (int t = 0; t < n_tiles; ++t) {
-      if (L == 0) trace(tr, 2, t, 0);
+      if (tid == 0) trace(tr, 2, t, 0);
       wait(&ctl->sfull[t & 1], (t >> 1) & 1);
       tc_fence_after();
-      if (L == 0) trace(tr, 2, t, 1);
+      if (tid == 0) trace(tr, 2, t, 1);
       const int n_valid = min(kKeys, tok1 - (tok0 + t * kKeys));
       const bool key_ok = L < n_valid;
       if (n_valid < kKeys) {
         // ragged tail: tokens past the valid length may hold anything; their weights are 0, so
         // V must be finite there: clear those rows of the staged V tile (both halves)
         const int jv = 2 * t + 1;
-        wait(&ctl->ufull[jv % kUnits], (jv / kUnits) & 1);
+        wait(&ctl->ufull[jv % UNITS], (jv / UNITS) & 1);
         if (!dead) {
-          uint8_t* v_s = smem + (jv % kUnits) * kUnitBytes;
+          uint8_t* v_s = smem + (jv % UNITS) * kUnitBytes;
           const int n_vec = (kKeys - n_valid) * 16;
-          for (int i = L; i < n_vec; i += 128) {
+          for (int i = tid; i < n_vec; i += C::kSoft) {
             const int row = n_valid + (i >> 4), half = (i >> 3) & 1, ch = i & 7;
             *reinterpret_cast<uint4*>(v_s + half * kHalf + row * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
           }
         }
         // made visible to the tensor core by the proxy fence before pready below
       }
-      uint32_t raw[2][16];
-      float x[kN];
+      // The scores are read from tensor memory twice (first for the overflow test, then for the
+      // weights) instead of being held in registers across the barrier below.
+      const uint32_t t_s = tmem + lane_off + (t & 1) * N + c0;
       bool over = false;
       if (!dead) {
-        tmem_ld16(tmem + lane_off + kColS + (t & 1) * kN, raw[0]);
-        tmem_ld16(tmem + lane_off + kColS + (t & 1) * kN + 16, raw[1]);
-        tc_wait_ld();
-        float mx = -INFINITY;
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // independent chains
 #pragma unroll
-        for (int r4 = 0; r4 < kN / 4; ++r4) {
-          const float4 mr = *reinterpret_cast<const float4*>(&ctl->m_ref[r4 * 4]);
-          const float mm[4] = {mr.x, mr.y, mr.z, mr.w};
+        for (int q0 = 0; q0 < NC / 16; q0 += kBatch) {  // kBatch loads, one wait
+          uint32_t raw[kBatch][16];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int r = r4 * 4 + e;
-            const float s2 = __uint_as_float(raw[r / 16][r % 16]) * p.scale_log2;
-            x[r] = s2 - mm[e];  // +inf while m_ref is -inf
-            mx = fmaxf(mx, x[r]);
+          for (int h = 0; h < kBatch; ++h)
+            if ((q0 + h) * 16 < cn) tmem_ld16(t_s + (q0 + h) * 16, raw[h]);
+          tc_wait_ld();
+#pragma unroll
+          for (int h = 0; h < kBatch; ++h) {
+            const int q = q0 + h;
+            if (q * 16 < cn) {
+#pragma unroll
+              for (int c4 = 0; c4 < 4; ++c4) {
+                const float4 mr = *reinterpret_cast<const float4*>(&ctl->m_ref[c0 + q * 16 + c4 * 4]);
+                const float mm[4] = {mr.x, mr.y, mr.z, mr.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)  // +inf while m_ref is -inf
+                  mx4[e] = fmaxf(mx4[e], fmaf(__uint_as_float(raw[h][c4 * 4 + e]), p.scale_log2, -mm[e]));
+              }
+            }
           }
         }
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
         over = key_ok && (mx > kLazyThreshold);
       }
-      if (L == 0) ctl->flag[(t + 1) % 3] = 0;
+      if (tid == 0) trace(tr, 2, t, 3);
+      if (tid == 0) ctl->flag[(t + 1) % 3] = 0;
       if (__any_sync(0xffffffffu, over) && lane == 0) ctl->flag[t % 3] = 1;
-      named_bar_sync(1, 128);
+      named_bar_sync(1, C::kSoft);
+      if (tid == 0) trace(tr, 2, t, 4);
       if (ctl->flag[t % 3]) {
         // ---- raise the row references to the exact tile maxima (rare after the first tile) ----
         if (!dead) {
 #pragma unroll
-          for (int r = 0; r < kN; ++r) {
-            float v = key_ok ? __uint_as_float(raw[r / 16][r % 16]) * p.scale_log2 : -INFINITY;
-            v = warp_max_f(v);
-            if (lane == 0) ctl->smax[warp][r] = v;
+          for (int q = 0; q < NC / 16; ++q) {
+            if (q * 16 < cn) {
+              uint32_t raw[16];
+              tmem_ld16(t_s + q * 16, raw);
+              tc_wait_ld();
+#pragma unroll
+              for (int c = 0; c < 16; ++c) {
+                float v = key_ok ? __uint_as_float(raw[c]) * p.scale_log2 : -INFINITY;
+                v = warp_max_f(v);
+                if (lane == 0) ctl->smax[warp & 3][c0 + q * 16 + c] = v;
+              }
+            }
           }
         }
-        named_bar_sync(1, 128);
+        named_bar_sync(1, C::kSoft);
         if (t > 0) {  // O^T must be at rest: the output MMAs of tile t-1 have retired
           wait(&ctl->pfree, (t - 1) & 1);
           tc_fence_after();
         }
         if (!dead) {
-          float f[kN];
 #pragma unroll
-          for (int r = 0; r < kN; ++r) {
-            const float m_old = ctl->m_ref[r];
-            const float m_new = fmaxf(fmaxf(m_old, ctl->smax[0][r]),
-                                      fmaxf(fmaxf(ctl->smax[1][r], ctl->smax[2][r]), ctl->smax[3][r]));
-            f[r] = (m_old == -INFINITY) ? 0.f : exp2f(m_old - m_new);
-            lsum[r] *= f[r];
-            x[r] = __uint_as_float(raw[r / 16][r % 16]) * p.scale_log2 - m_new;
-          }
-          if (t > 0) {
+          for (int q = 0; q < NC / 16; ++q) {
+            if (q * 16 < cn) {
+              float f[16];
 #pragma unroll
-            for (int q = 0; q < kN / 16; ++q) {
-              uint32_t o[16];
-              tmem_ld16(tmem + lane_off + kColO + q * 16, o);
-              tc_wait_ld();
+              for (int c = 0; c < 16; ++c) {
+                const int r = c0 + q * 16 + c;
+                const float m_old = ctl->m_ref[r];
+                const float m_new = fmaxf(fmaxf(m_old, ctl->smax[0][r]),
+                                          fmaxf(fmaxf(ctl->smax[1][r], ctl->smax[2][r]), ctl->smax[3][r]));
+                f[c] = (m_old == -INFINITY) ? 0.f : exp2f(m_old - m_new);
+                lsum[q * 16 + c] *= f[c];
+              }
+              if (t > 0) {
+                uint32_t o[16];
+                tmem_ld16(tmem + lane_off + C::kColO + c0 + q * 16, o);
+                tc_wait_ld();
 #pragma unroll
-              for (int c = 0; c < 16; ++c)
-                o[c] = __float_as_uint(__uint_as_float(o[c]) * f[q * 16 + c]);
-              tmem_st16(tmem + lane_off + kColO + q * 16, o);
+                for (int c = 0; c < 16; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * f[c]);
+                tmem_st16(tmem + lane_off + C::kColO + c0 + q * 16, o);
+              }
             }
-            tc_wait_st();
           }
+          tc_wait_st();
         }
-        named_bar_sync(1, 128);  // every thread has read the old references
-        if (L < kN && !dead) {
-          const float m_old = ctl->m_ref[L];
-          ctl->m_ref[L] = fmaxf(fmaxf(m_old, ctl->smax[0][L]),
-                                fmaxf(fmaxf(ctl->smax[1][L], ctl->smax[2][L]), ctl->smax[3][L]));
+        named_bar_sync(1, C::kSoft);  // every thread has read the old references
+        if (tid < n_mma && !dead) {
+          const float m_old = ctl->m_ref[tid];
+          ctl->m_ref[tid] = fmaxf(fmaxf(m_old, ctl->smax[0][tid]),
+                                  fmaxf(fmaxf(ctl->smax[1][tid], ctl->smax[2][tid]), ctl->smax[3][tid]));
         }
-        named_bar_sync(1, 128);
-      }
-      // weights, row sums, P^T as bf16
-      uint32_t pk[kN / 2];
-      if (!dead) {
-#pragma unroll
-        for (int r = 0; r < kN; r += 2) {
-          const float p0 = key_ok ? exp2f(x[r]) : 0.f;
-          const float p1 = key_ok ? exp2f(x[r + 1]) : 0.f;
-          lsum[r] += p0;
-          lsum[r + 1] += p1;
-          __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);  // low half = even row
-          pk[r / 2] = *reinterpret_cast<uint32_t*>(&h);
-        }
+        named_bar_sync(1, C::kSoft);
       }
       if (t > 0) wait(&ctl->pfree, (t - 1) & 1);  // the output MMAs of tile t-1 consumed P^T
+      if (tid == 0) trace(tr, 2, t, 5);
       if (!dead) {
+        // weights, row sums, P^T as bf16: rows c0+8c .. c0+8c+7 of key L form one 16-byte piece
 #pragma unroll
-        for (int c = 0; c < kN / 8; ++c)  // rows 8c..8c+7 of key L: one 16-byte piece
-          *reinterpret_cast<uint4*>(p_s + c * (kKeys * 16) + L * 16) =
-              make_uint4(pk[c * 4], pk[c * 4 + 1], pk[c * 4 + 2], pk[c * 4 + 3]);
+        for (int q0 = 0; q0 < NC / 16; q0 += kBatch) {  // kBatch loads, one wait
+          uint32_t raw2[kBatch][16];
+#pragma unroll
+          for (int h = 0; h < kBatch; ++h)
+            if ((q0 + h) * 16 < cn) tmem_ld16(t_s + (q0 + h) * 16, raw2[h]);
+          tc_wait_ld();
+#pragma unroll
+          for (int h = 0; h < kBatch; ++h) {
+          const int q = q0 + h;
+          const uint32_t (&raw)[16] = raw2[h];
+          if (q * 16 < cn) {
+            // staged so that the 16 exponentials of a chunk are independent instructions
+            float pv[16];
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {
+              const float4 mr = *reinterpret_cast<const float4*>(&ctl->m_ref[c0 + q * 16 + c4 * 4]);
+              pv[c4 * 4 + 0] = fmaf(__uint_as_float(raw[c4 * 4 + 0]), p.scale_log2, -mr.x);
+              pv[c4 * 4 + 1] = fmaf(__uint_as_float(raw[c4 * 4 + 1]), p.scale_log2, -mr.y);
+              pv[c4 * 4 + 2] = fmaf(__uint_as_float(raw[c4 * 4 + 2]), p.scale_log2, -mr.z);
+              pv[c4 * 4 + 3] = fmaf(__uint_as_float(raw[c4 * 4 + 3]), p.scale_log2, -mr.w);
+            }
+#pragma unroll
+            for (int c = 0; c < 16; ++c) pv[c] = ex2_ftz(pv[c]);
+#pragma unroll
+            for (int c = 0; c < 16; ++c) pv[c] = key_ok ? pv[c] : 0.f;
+#pragma unroll
+            for (int c = 0; c < 16; ++c) lsum[q * 16 + c] += pv[c];
+            uint32_t pk[8];
+#pragma unroll
+            for (int c = 0; c < 16; c += 2) {
+              __nv_bfloat162 hh = __floats2bfloat162_rn(pv[c], pv[c + 1]);  // low half = even row
+              pk[c / 2] = *reinterpret_cast<uint32_t*>(&hh);
+            }
+#pragma unroll
+            for (int h8 = 0; h8 < 2; ++h8)
+              *reinterpret_cast<uint4*>(p_s + ((c0 >> 3) + q * 2 + h8) * (kKeys * 16) + L * 16) =
+                  make_uint4(pk[h8 * 4], pk[h8 * 4 + 1], pk[h8 * 4 + 2], pk[h8 * 4 + 3]);
+          }
+          }
+        }
         fence_proxy_async();
         tc_fence_before();
       }
       mbar_arrive(&ctl->pready);
-      if (L == 0) trace(tr, 2, t, 2);
+      if (tid == 0) trace(tr, 2, t, 2);
     }
     wait(&ctl->pfree, (n_tiles - 1) & 1);
-    named_bar_sync(1, 128);
-    if (ctl->abort == 0) {  // uniform over the 128 threads after the barrier
+    named_bar_sync(1, C::kSoft);
+    if (ctl->abort == 0) {  // uniform over the softmax threads after the barrier
       tc_fence_after();
       // ---- row sums across the 128 key lanes, then the partial state ----
-      float* red = reinterpret_cast<float*>(smem);  // [128][33] over the free ring
+      float* red = reinterpret_cast<float*>(smem);  // [128][N + 1] over the free ring
 #pragma unroll
-      for (int r = 0; r < kN; ++r) red[L * (kN + 1) + r] = lsum[r];
-      named_bar_sync(1, 128);
-      if (L < nrows) {
+      for (int r = 0; r < NC; ++r)
+        if (r < cn) red[L * (N + 1) + c0 + r] = lsum[r];
+      named_bar_sync(1, C::kSoft);
+      if (tid < nrows) {
         float lt = 0.f;
-        for (int k = 0; k < kKeys; ++k) lt += red[k * (kN + 1) + L];
-        out_ml[L] = make_float2(lt > 0.f ? ctl->m_ref[L] : -INFINITY, lt);
+        for (int k = 0; k < kKeys; ++k) lt += red[k * (N + 1) + tid];
+        out_ml[tid] = make_float2(lt > 0.f ? ctl->m_ref[tid] : -INFINITY, lt);
       }
-      // thread L holds head dim L of every row
-      uint32_t o[2][16];
-      tmem_ld16(tmem + lane_off + kColO, o[0]);
-      tmem_ld16(tmem + lane_off + kColO + 16, o[1]);
-      tc_wait_ld();
+      // thread (L, cg) holds head dim L of its rows
 #pragma unroll
-      for (int r = 0; r < kN; ++r)
-        if (r < nrows) out_a[(size_t)r * kD + L] = __uint_as_float(o[r / 16][r % 16]);
+      for (int q = 0; q < NC / 16; ++q) {
+        if (q * 16 < cn) {
+          uint32_t o[16];
+          tmem_ld16(tmem + lane_off + C::kColO + c0 + q * 16, o);
+          tc_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            const int r = c0 + q * 16 + c;
+            if (r < nrows) out_a[(size_t)r * kD + L] = __uint_as_float(o[c]);
+          }
+        }
+      }
     }
   }
 
   // ---- teardown ----
   tc_fence_before();
   __syncthreads();
-  if (warp == 4) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols)
+  if (warp == kProducerWarp) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::kTmemCols)
                  : "memory");
   }
   // Completion order along the stream: one CTA of this grid waits for the previous grid, so
@@ -438,17 +519,36 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
   if (!p.wait_first && chain_cta) pdl_wait_prior();
 }
 
+template <int NC, int WG, int UNITS>
+cudaError_t launch_cfg(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                       cudaStream_t s, bool pdl) {
+  using C = Cfg<NC, WG, UNITS>;
+  dim3 grid(p.splits * p.row_tiles, p.H_kv, p.B), block(C::kThreads);
+  return launch_kernel(chunk_tc_keys_kernel<NC, WG, UNITS>, grid, block, C::kSmem, s, pdl, p, tmK, tmV);
+}
+
+template <int NC, int WG, int UNITS>
+cudaError_t prepare_cfg() {
+  return cudaFuncSetAttribute(chunk_tc_keys_kernel<NC, WG, UNITS>,
+                              cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<NC, WG, UNITS>::kSmem);
+}
+
 }  // namespace
 
 cudaError_t chunk_tc_keys_prepare() {
-  return cudaFuncSetAttribute(chunk_tc_keys_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              kSmemTotal);
+  cudaError_t e = prepare_cfg<32, 1, 3>();
+  if (e == cudaSuccess) e = prepare_cfg<32, 2, 5>();
+  if (e == cudaSuccess) e = prepare_cfg<32, 4, 5>();
+  return e;
 }
 
+// Rows per CTA (p.rows_per_tile): <= 32 -> two CTAs per SM with 4 softmax warps; <= 64 and
+// <= 128 -> one CTA per SM with 8 and 16 softmax warps (32 score columns per thread each).
 cudaError_t launch_chunk_tc_keys(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
                                  cudaStream_t s, bool pdl) {
-  dim3 grid(p.splits, p.H_kv, p.B), block(kThreads);
-  return launch_kernel(chunk_tc_keys_kernel, grid, block, kSmemTotal, s, pdl, p, tmK, tmV);
+  if (p.rows_per_tile <= 32) return launch_cfg<32, 1, 3>(p, tmK, tmV, s, pdl);
+  if (p.rows_per_tile <= 64) return launch_cfg<32, 2, 5>(p, tmK, tmV, s, pdl);
+  return launch_cfg<32, 4, 5>(p, tmK, tmV, s, pdl);
 }
 
 }  // namespace ss
