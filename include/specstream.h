@@ -87,6 +87,8 @@ typedef struct {
 /* Use the tensor-core chunk kernel that puts the query rows on the MMA's M axis instead of
  * the default one that puts the keys there.  For cross-checks. */
 #define SS_FLAG_ROWS_ON_M 4u
+/* Use the keys-on-M kernel for any number of rows per kv-head (default: up to 32). */
+#define SS_FLAG_KEYS_ON_M 8u
 
 typedef struct {
   const void* ptr;                      /* device pointer, bf16                      */
@@ -105,7 +107,8 @@ ss_status ss_destroy(ss_ctx* ctx);
 
 /* a1. Start a round: bind Q [B, H_q, T_q, d] and reset every row's state to the
  * identity (m, l, a) = (-inf, 0, 0) (Section 4.2, accumulator initialisation).
- * `scale` multiplies the scores (1/sqrt(d) in the paper) and is applied in fp32. */
+ * `scale` multiplies the scores (1/sqrt(d) in the paper), is applied in fp32 and must be
+ * positive and finite (SS_ERR_ARG otherwise). */
 ss_status ss_verify_begin(ss_ctx* ctx, ss_tensor Q, int32_t B, int32_t T_q, float scale,
                           void* stream);
 

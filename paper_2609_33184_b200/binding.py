@@ -22,7 +22,7 @@ STATUS_NAMES = ["SS_OK", "SS_ERR_ARG", "SS_ERR_SHAPE", "SS_ERR_ALIGN", "SS_ERR_S
 (SS_ERR_ARG, SS_ERR_SHAPE, SS_ERR_ALIGN, SS_ERR_STATE, SS_ERR_CAPACITY, SS_ERR_UNSUPPORTED,
  SS_ERR_CUDA, SS_ERR_DEVICE_FLAG, SS_ERR_TIMEOUT) = range(1, 10)
 SS_DEV_BAD_VALID_LEN, SS_DEV_BAD_ACCEPT, SS_DEV_DST_OVERFLOW, SS_DEV_WAIT_EXPIRED = 1, 2, 4, 8
-SS_FLAG_FORCE_SIMT, SS_FLAG_OVERLAP_CHUNKS, SS_FLAG_ROWS_ON_M = 1, 2, 4
+SS_FLAG_FORCE_SIMT, SS_FLAG_OVERLAP_CHUNKS, SS_FLAG_ROWS_ON_M, SS_FLAG_KEYS_ON_M = 1, 2, 4, 8
 SS_MASK_CHAIN, SS_MASK_TREE_BITS = 0, 1
 
 EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "ss_verify_chunk",

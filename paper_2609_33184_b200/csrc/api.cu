@@ -34,6 +34,7 @@ struct ss_ctx {
   const char* last_kernel;
   int force_splits;        // SS_SPLITS env override (0 = automatic)
   bool force_rows_kernel;  // SS_CHUNK_KERNEL=rows: rows-on-M tensor-core kernel even for few rows
+  bool force_keys_kernel;  // SS_CHUNK_KERNEL=keys: keys-on-M tensor-core kernel for any row count
   int target_ctas;
   // tensor-map cache
   struct TmEntry {
@@ -238,6 +239,7 @@ ss_status ss_create(ss_ctx** out, const ss_config* cfg, void* workspace, size_t 
   c->force_splits = fs ? atoi(fs) : 0;
   const char* ck = getenv("SS_CHUNK_KERNEL");
   c->force_rows_kernel = (ck && strcmp(ck, "rows") == 0) || (cfg->flags & SS_FLAG_ROWS_ON_M);
+  c->force_keys_kernel = (ck && strcmp(ck, "keys") == 0) || (cfg->flags & SS_FLAG_KEYS_ON_M);
 
   if (!g_encode) {
     void* fn = nullptr;
@@ -285,6 +287,7 @@ ss_status ss_verify_begin(ss_ctx* c, ss_tensor Q, int32_t B, int32_t T_q, float 
                           void* stream) {
   if (!c || !Q.ptr) return SS_ERR_ARG;
   if (B <= 0 || T_q <= 0) return SS_ERR_ARG;
+  if (!(scale > 0.f) || !(scale < 3.0e38f)) return SS_ERR_ARG;  // positive and finite
   if (B > c->cfg.max_B || T_q > c->cfg.max_Tq) return SS_ERR_SHAPE;
   if (!tensor_ok(Q)) return SS_ERR_ALIGN;
   if (c->state != ss_ctx::IDLE) return SS_ERR_STATE;
@@ -359,11 +362,10 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   }
   CUtensorMap tmK, tmV;
   bool tc = c->tc_ok;
-  // up to 64 rows per kv-head the keys ride the MMA's M axis (tiles of 128 tokens); with more
-  // rows the kernel with the rows on M is faster (measured); SS_FLAG_ROWS_ON_M forces it
-  const char* ck = getenv("SS_CHUNK_KERNEL");
-  const bool force_keys = ck && strcmp(ck, "keys") == 0;
-  const bool keys_on_m = tc && !c->force_rows_kernel && (R <= 64 || force_keys);
+  // up to 32 rows per kv-head the keys ride the MMA's M axis (tiles of 128 tokens); with more
+  // rows the kernel with the rows on M is faster (measured).  SS_FLAG_ROWS_ON_M /
+  // SS_FLAG_KEYS_ON_M (or SS_CHUNK_KERNEL=rows|keys) force one of them.
+  const bool keys_on_m = tc && !c->force_rows_kernel && (R <= 32 || c->force_keys_kernel);
   const int box = keys_on_m ? 128 : kTileKeys;
   if (tc) tc = get_tensor_map(c, K, c->B, L_c, box, &tmK) && get_tensor_map(c, V, c->B, L_c, box, &tmV);
 

@@ -87,23 +87,25 @@ __device__ __forceinline__ void store_p(uint32_t t_s, const uint32_t (&pk)[NC / 
 // ---- softmax of one tile for one TMEM lane --------------------------------------------------
 // NC = number of key columns this lane owns in a 64-key tile.  P (bf16 pairs) is written
 // over the first 32 score columns: this lane's keys at [c0/2, c0/2 + NC/2), zeros elsewhere.
-template <int NC>
+// MASK = the tile straddles the valid length (columns >= n_valid are invisible).  The scale is
+// positive (checked at ss_verify_begin), so the maximum is taken on the raw scores and the
+// scaling rides in the FMA that subtracts the reference.
+template <int NC, bool MASK>
 __device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_o, int c0, int n_valid,
                                              bool have_o, float scale_log2, float& m, float& l) {
   uint32_t raw[NC / 16][16];
 #pragma unroll
   for (int q = 0; q < NC / 16; ++q) tmem_ld16(t_s + c0 + q * 16, raw[q]);
   tc_wait_ld();
-  float s[NC];
   float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // independent chains
 #pragma unroll
   for (int c = 0; c < NC; ++c) {
-    float v = __uint_as_float(raw[c / 16][c % 16]) * scale_log2;
-    if (c0 + c >= n_valid) v = -INFINITY;
-    s[c] = v;
+    float v = __uint_as_float(raw[c / 16][c % 16]);
+    if (MASK && c0 + c >= n_valid) v = -INFINITY;
+    if (MASK) raw[c / 16][c % 16] = __float_as_uint(v);
     mx4[c & 3] = fmaxf(mx4[c & 3], v);
   }
-  const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+  const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
   float f = 1.f;
   if (mx > m + kRescaleThreshold) {  // also the first finite maximum (m = -inf)
     f = (m == -INFINITY) ? 0.f : exp2f(m - mx);
@@ -123,12 +125,13 @@ __device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_o, int c0,
       tmem_st16(t_o + q * 16, o);
     }
   }
-  const float m_use = (m == -INFINITY) ? 0.f : m;
+  const float neg_m = (m == -INFINITY) ? 0.f : -m;
   uint32_t pk[NC / 16][8];
   float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
   for (int c = 0; c < NC; c += 2) {
-    const float p0 = ex2_ftz(s[c] - m_use), p1 = ex2_ftz(s[c + 1] - m_use);
+    const float p0 = ex2_ftz(fmaf(__uint_as_float(raw[c / 16][c % 16]), scale_log2, neg_m));
+    const float p1 = ex2_ftz(fmaf(__uint_as_float(raw[(c + 1) / 16][(c + 1) % 16]), scale_log2, neg_m));
     sum4[(c >> 1) & 3] += p0 + p1;
     __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);  // low half = even key
     pk[c / 16][(c / 2) % 8] = *reinterpret_cast<uint32_t*>(&h);
@@ -417,12 +420,21 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         }
         fence_proxy_async();
       }
-      if (nc == 16)
-        softmax_tile<16>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
-      else if (nc == 32)
-        softmax_tile<32>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
-      else
-        softmax_tile<64>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+      if (n_valid < kTileKeys) {
+        if (nc == 16)
+          softmax_tile<16, true>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+        else if (nc == 32)
+          softmax_tile<32, true>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+        else
+          softmax_tile<64, true>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+      } else {
+        if (nc == 16)
+          softmax_tile<16, false>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+        else if (nc == 32)
+          softmax_tile<32, false>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+        else
+          softmax_tile<64, false>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+      }
       tc_fence_before();
       mbar_arrive(&ctl->pready);
       if (L == 0) trace(tr, 2, it, 2);

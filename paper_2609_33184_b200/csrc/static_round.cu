@@ -64,6 +64,7 @@ extern "C" ss_status ss_verify_round_static(const ss_static_round* r, void* stre
     return SS_ERR_ARG;
   if (r->H_q % r->H_kv || (r->d != 64 && r->d != 128) || r->T_loc > 1024) return SS_ERR_SHAPE;
   if (r->L_c == 0 && r->T_loc == 0) return SS_ERR_ARG;
+  if (!(r->scale > 0.f) || !(r->scale < 3.0e38f)) return SS_ERR_ARG;
   if (!tensor_ok(r->Q) || !aligned16(r->O)) return SS_ERR_ALIGN;
   if (r->L_c > 0 && (!tensor_ok(r->K) || !tensor_ok(r->V))) return SS_ERR_ALIGN;
   if (r->T_loc > 0 && (!tensor_ok(r->K_loc) || !tensor_ok(r->V_loc))) return SS_ERR_ALIGN;

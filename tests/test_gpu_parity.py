@@ -52,9 +52,10 @@ def test_c3_shape_scaled_ragged_nan_padding():
     _run(cfg, kernel="tcgen05")  # padding past valid_len is NaN by default
 
 
-def test_c4_shape_scaled_tree():
+@pytest.mark.parametrize("flags", [0, 8])
+def test_c4_shape_scaled_tree(flags):
     cfg = _small("c4_tree", B=2, H_q=10, H_kv=2, L_c=256, len_lo=600, len_hi=600)
-    _run(cfg, kernel="tcgen05")
+    _run(cfg, flags=flags, kernel="tcgen05-keys" if flags else "tcgen05")
 
 
 @pytest.mark.parametrize("flags", [0, 1, 4])   # keys-on-M, CUDA cores, rows-on-M
@@ -71,12 +72,16 @@ def test_short_histories(flags, n):
 def test_group_sizes_and_head_dims(d, G, mask):
     cfg = inputs.VerifyConfig("v", 0x77 + G + d, 2, 2 * G, 2, d, 96, 7, 40, 300, mask=mask, k_mult=2.0)
     _run(cfg)
+    if d == 128:
+        _run(cfg, flags=8)   # keys-on-M kernel for every row count
 
 
-@pytest.mark.parametrize("T_q", [1, 2, 3, 5, 9, 16, 33])
-def test_query_counts_odd_rows(T_q):
+@pytest.mark.parametrize("flags", [0, 8])
+@pytest.mark.parametrize("T_q", [1, 2, 3, 5, 9, 16, 25, 33])
+def test_query_counts_odd_rows(T_q, flags):
+    # R = 4 T_q rows per kv-head: 4 .. 132 (one and two row groups, 4 / 8 / 16 softmax warps)
     cfg = inputs.VerifyConfig("v", 0x99 + T_q, 2, 8, 2, 128, 128, T_q, 100, 400, k_mult=2.0)
-    _run(cfg, kernel="tcgen05")
+    _run(cfg, flags=flags, kernel="tcgen05-keys" if flags else "tcgen05")
 
 
 @pytest.mark.parametrize("k_mult", [4.0, 8.0])
