@@ -376,9 +376,11 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
     p.rows_per_tile = R < 128 ? R : 128;
     p.groups = 1;
   } else if (tc) {
+    // row tiles of 128 rows and a remainder tile; a tile with <= 64 (<= 32) rows replicates its
+    // rows 2x (4x) along M, so no lane computes padding
     p.row_tiles = (R + 127) / 128;
-    p.rows_per_tile = (R + p.row_tiles - 1) / p.row_tiles;
-    p.groups = p.rows_per_tile <= 32 ? 4 : (p.rows_per_tile <= 64 ? 2 : 1);
+    p.rows_per_tile = R < 128 ? R : 128;
+    p.groups = 0;  // decided per CTA from its row count
   } else {
     p.rows_per_tile = 32;
     p.row_tiles = (R + 31) / 32;

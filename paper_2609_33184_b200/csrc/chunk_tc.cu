@@ -168,7 +168,9 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   const int kvh = blockIdx.y, b = blockIdx.z;
   const int row0 = rt * p.rows_per_tile;
   const int nrows = min(p.rows_per_tile, p.R - row0);
-  const int r_pad = 128 / p.groups;
+  // key groups sharing the 128 lanes: the Q rows are replicated when the tile has few rows
+  const int groups = nrows <= 32 ? 4 : (nrows <= 64 ? 2 : 1);
+  const int r_pad = 128 / groups;
   unsigned long long* tr = (blockIdx.x | blockIdx.y | blockIdx.z) ? nullptr : p.trace;
 
   const bool chain_cta = (blockIdx.x | blockIdx.y | blockIdx.z) == 0;
@@ -378,7 +380,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     const int L = tid;  // 0..127
     const int r = L % r_pad;
     const int grp = L / r_pad;
-    const int nc = kTileKeys / p.groups;
+    const int nc = kTileKeys / groups;
     const int c0 = grp * nc;
     const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
     const uint32_t t_s = tmem + lane_off + kColS;
@@ -448,7 +450,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       ctl->ml[L] = make_float2(m, l);
       named_bar_sync(1, 128);
       float M = -INFINITY;
-      for (int g = 0; g < p.groups; ++g) M = fmaxf(M, ctl->ml[g * r_pad + r].x);
+      for (int g = 0; g < groups; ++g) M = fmaxf(M, ctl->ml[g * r_pad + r].x);
       const float f = (m == -INFINITY) ? 0.f : exp2f(m - M);
 #pragma unroll 1
       for (int q = 0; q < kD / 16; ++q) {
@@ -467,7 +469,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       }
       if (L < nrows) {
         float lt = 0.f;
-        for (int g = 0; g < p.groups; ++g) {
+        for (int g = 0; g < groups; ++g) {
           const float2 st = ctl->ml[g * r_pad + r];
           if (st.x > -INFINITY) lt += exp2f(st.x - M) * st.y;
         }
@@ -476,7 +478,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       named_bar_sync(1, 128);
       for (int rr = warp; rr < nrows; rr += 4) {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int g = 0; g < p.groups; ++g) {
+        for (int g = 0; g < groups; ++g) {
           const int LL = g * r_pad + rr;
           const float4 v = *reinterpret_cast<const float4*>(&o_s[LL * kD + ((lane ^ (LL & 31)) << 2)]);
           acc.x += v.x;

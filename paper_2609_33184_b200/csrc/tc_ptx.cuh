@@ -6,6 +6,9 @@ namespace ss {
 namespace tc {
 
 constexpr unsigned long long kWaitNs = 2000000000ull;  // bound of every in-kernel wait: 2 s
+// A waiting thread may stay suspended this long inside one try_wait (it still resumes as soon
+// as the phase completes), so waiting warps spend few issue slots.
+constexpr uint32_t kSuspendHintNs = 20000;
 
 // ---- small PTX wrappers ------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -31,10 +34,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendHintNs)
       : "memory");
   return ok != 0;
 }
