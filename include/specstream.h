@@ -138,6 +138,15 @@ ss_status ss_verify_chunk_hinted(ss_ctx* ctx, ss_tensor K, ss_tensor V, int32_t 
 ss_status ss_verify_local(ss_ctx* ctx, ss_tensor K_loc, ss_tensor V_loc, int32_t T_loc,
                           ss_mask_kind kind, const uint64_t* mask_bits, void* stream);
 
+/* Checkpoint of a round (between begin and finalize).  export writes, for every query row in
+ * [B, H_q, T_q] order, the merged state of everything seen so far: ml[row] = (m, l) with m in
+ * the base-2 domain (maximum reference of score*scale*log2(e); -inf and l = 0 for an empty
+ * row) and a[row][d] = sum exp2(s2 - m) v, both fp32 device buffers.  The round stays open.
+ * import adds such a state to the open round as one more partial (Eq. 14 is associative and
+ * order-free), e.g. the states other GPUs reduced over their share of the history chunks. */
+ss_status ss_verify_export_state(ss_ctx* ctx, float* ml, float* a, void* stream);
+ss_status ss_verify_import_state(ss_ctx* ctx, const float* ml, const float* a, void* stream);
+
 /* a5. Merge all partial states (Eq. 14), O = a / l as bf16 (round to nearest even) into
  * O [B, H_q, T_q, d] (contiguous), LSE = m + ln l (natural log, of the scaled masked
  * scores) into LSE [B, H_q, T_q] fp32 (may be NULL).  Ends the round. */

@@ -28,7 +28,8 @@ SS_MASK_CHAIN, SS_MASK_TREE_BITS = 0, 1
 EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "ss_verify_chunk",
            "ss_verify_local", "ss_verify_finalize", "ss_commit_gather", "ss_poll_status",
            "ss_stream_round", "ss_strerror", "ss_sizeof_stream_desc", "ss_last_cuda_error", "ss_launch_count",
-           "ss_last_chunk_kernel", "ss_trace_enable", "ss_trace_read", "ss_verify_round_static", "ss_verify_chunk_hinted"]
+           "ss_last_chunk_kernel", "ss_trace_enable", "ss_trace_read", "ss_verify_round_static", "ss_verify_chunk_hinted", "ss_verify_export_state",
+           "ss_verify_import_state"]
 
 
 class ss_config(C.Structure):
@@ -103,6 +104,10 @@ def load() -> C.CDLL:
     lib.ss_verify_chunk_hinted.argtypes = [vp, ss_tensor, ss_tensor, i32, vp, C.POINTER(C.c_int32), vp]
     lib.ss_verify_local.restype = C.c_int
     lib.ss_verify_local.argtypes = [vp, ss_tensor, ss_tensor, i32, C.c_int, vp, vp]
+    lib.ss_verify_export_state.restype = C.c_int
+    lib.ss_verify_export_state.argtypes = [vp, vp, vp, vp]
+    lib.ss_verify_import_state.restype = C.c_int
+    lib.ss_verify_import_state.argtypes = [vp, vp, vp, vp]
     lib.ss_verify_finalize.restype = C.c_int
     lib.ss_verify_finalize.argtypes = [vp, vp, vp, vp]
     lib.ss_commit_gather.restype = C.c_int
@@ -221,6 +226,16 @@ class Context:
         self._check(self.lib.ss_verify_local(self.handle, as_ss_tensor(K_loc), as_ss_tensor(V_loc),
                                              T_loc, mask_kind, _ptr(mask_bits), _stream_ptr(stream)),
                     "ss_verify_local")
+
+    def ss_verify_export_state(self, ml: torch.Tensor, a: torch.Tensor, stream=None):
+        assert ml.dtype == torch.float32 and a.dtype == torch.float32 and ml.is_contiguous() and a.is_contiguous()
+        self._check(self.lib.ss_verify_export_state(self.handle, ml.data_ptr(), a.data_ptr(),
+                                                    _stream_ptr(stream)), "ss_verify_export_state")
+
+    def ss_verify_import_state(self, ml: torch.Tensor, a: torch.Tensor, stream=None):
+        assert ml.dtype == torch.float32 and a.dtype == torch.float32 and ml.is_contiguous() and a.is_contiguous()
+        self._check(self.lib.ss_verify_import_state(self.handle, ml.data_ptr(), a.data_ptr(),
+                                                    _stream_ptr(stream)), "ss_verify_import_state")
 
     def ss_verify_finalize(self, O: torch.Tensor, LSE: Optional[torch.Tensor], stream=None):
         assert O.dtype == torch.bfloat16 and O.is_contiguous()

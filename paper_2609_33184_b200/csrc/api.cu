@@ -193,6 +193,22 @@ void fill_merge(ss_ctx* c, ss::MergeParams* m) {
   memcpy(m->splits, c->splits, sizeof(m->splits));
 }
 
+// All partial sets in use: fold them into set 0 (Eq. 14 is associative).
+cudaError_t fold_sets(ss_ctx* c, cudaStream_t s) {
+  ss::MergeParams m;
+  fill_merge(c, &m);
+  m.has_local = 0;
+  m.fold_ml = c->part_ml;
+  m.fold_a = c->part_a;
+  cudaError_t e = ss::launch_fold(m, s);
+  if (e != cudaSuccess) return e;
+  ++c->launches;
+  c->n_sets = 1;
+  c->splits[0] = 1;
+  c->first_launch = true;  // the next kernel must not overlap the fold
+  return cudaSuccess;
+}
+
 }  // namespace
 
 extern "C" {
@@ -330,18 +346,8 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   cudaStream_t s = c->stream;
 
   if (c->n_sets == c->n_set_cap) {
-    // all partial sets in use: fold them into set 0 (Eq. 14 is associative)
-    ss::MergeParams m;
-    fill_merge(c, &m);
-    m.has_local = 0;
-    m.fold_ml = c->part_ml;
-    m.fold_a = c->part_a;
-    cudaError_t e = ss::launch_fold(m, s);
+    cudaError_t e = fold_sets(c, s);
     if (e != cudaSuccess) return cuda_fail(c, e);
-    ++c->launches;
-    c->n_sets = 1;
-    c->splits[0] = 1;
-    c->first_launch = true;  // the next kernel must not overlap the fold
   }
 
   const int R = c->T_q * c->G;
@@ -505,6 +511,44 @@ ss_status ss_verify_local(ss_ctx* c, ss_tensor K_loc, ss_tensor V_loc, int32_t T
   ++c->launches;
   c->has_local = true;
   c->first_launch = false;
+  return SS_OK;
+}
+
+ss_status ss_verify_export_state(ss_ctx* c, float* ml, float* a, void* stream) {
+  if (!c || !ml || !a) return SS_ERR_ARG;
+  if (((uintptr_t)ml & 7) || !aligned16(a)) return SS_ERR_ALIGN;
+  if (c->state != ss_ctx::OPEN || (cudaStream_t)stream != c->stream) return SS_ERR_STATE;
+  ss::MergeParams m;
+  fill_merge(c, &m);
+  m.fold_ml = (float2*)ml;
+  m.fold_a = a;
+  cudaError_t e = ss::launch_export(m, c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e);
+  ++c->launches;
+  c->first_launch = true;  // reads every partial: the next kernel must not overlap it
+  return SS_OK;
+}
+
+ss_status ss_verify_import_state(ss_ctx* c, const float* ml, const float* a, void* stream) {
+  if (!c || !ml || !a) return SS_ERR_ARG;
+  if (((uintptr_t)ml & 7) || !aligned16(a)) return SS_ERR_ALIGN;
+  if (c->state != ss_ctx::OPEN || (cudaStream_t)stream != c->stream) return SS_ERR_STATE;
+  if (c->n_sets == c->n_set_cap) {
+    cudaError_t e = fold_sets(c, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+  }
+  ss::MergeParams m;
+  fill_merge(c, &m);
+  m.part_ml = (const float2*)ml;
+  m.part_a = a;
+  m.fold_ml = c->part_ml + (int64_t)c->n_sets * c->set_stride_ml;
+  m.fold_a = c->part_a + (int64_t)c->n_sets * c->set_stride_a;
+  cudaError_t e = ss::launch_import(m, c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e);
+  ++c->launches;
+  c->splits[c->n_sets] = 1;
+  ++c->n_sets;
+  c->first_launch = true;
   return SS_OK;
 }
 

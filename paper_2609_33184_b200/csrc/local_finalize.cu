@@ -113,13 +113,15 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) local_kernel(const LocalPar
 // the same value as the serial recurrence up to rounding order), then either O = a / l
 // and LSE (finalize) or the merged state itself (fold).  One warp per row.
 // ---------------------------------------------------------------------------------------
-template <int D, bool FOLD>
+// MODE 0: finalize (O, LSE); 1: fold into set 0; 2: export the merged state in row order.
+template <int D, int MODE>
 __global__ void __launch_bounds__(kWarpsPerCta * 32) merge_kernel(const MergeParams p) {
+  constexpr bool FOLD = MODE == 1;
   constexpr int CPL = D / 32;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t row_id = (int64_t)blockIdx.x * kWarpsPerCta + warp;
   const int64_t n_rows = (int64_t)p.B * p.H_q * p.T_q;
-  if (!FOLD) pdl_wait_prior();  // every partial of the round must be complete
+  if (MODE == 0) pdl_wait_prior();  // every partial of the round must be complete
   if (row_id >= n_rows) return;
   const int i = (int)(row_id % p.T_q);
   const int h = (int)((row_id / p.T_q) % p.H_q);
@@ -172,7 +174,14 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) merge_kernel(const MergePar
       }
     }
   }
-  if (FOLD) {
+  if (MODE == 2) {
+    if (lane == 0) p.fold_ml[row_id] = make_float2(L > 0.f ? M : -INFINITY, L);
+    float* out = p.fold_a + row_id * D + lane * CPL;
+    if (CPL == 4)
+      *reinterpret_cast<float4*>(out) = make_float4(acc[0], acc[1], acc[CPL - 2], acc[CPL - 1]);
+    else
+      *reinterpret_cast<float2*>(out) = make_float2(acc[0], acc[1]);
+  } else if (FOLD) {
     const size_t idx = slot0 * p.R_stride + r;
     if (lane == 0) p.fold_ml[idx] = make_float2(L > 0.f ? M : -INFINITY, L);
     float* out = p.fold_a + idx * D + lane * CPL;
@@ -196,6 +205,26 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) merge_kernel(const MergePar
     if (p.LSE && lane == 0)
       p.LSE[row_id] = (L > 0.f) ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
   }
+}
+
+// ---------------------------------------------------------------------------------------
+// Import: a merged state in row order [B, H_q, T_q] -> one partial set (split 0).
+// ---------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(kWarpsPerCta * 32) import_kernel(const MergeParams p) {
+  constexpr int CPL = D / 32;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t row_id = (int64_t)blockIdx.x * kWarpsPerCta + warp;
+  if (row_id >= (int64_t)p.B * p.H_q * p.T_q) return;
+  const int i = (int)(row_id % p.T_q);
+  const int h = (int)((row_id / p.T_q) % p.H_q);
+  const int b = (int)(row_id / ((int64_t)p.T_q * p.H_q));
+  const size_t idx = ((size_t)b * p.H_kv + h / p.G) * p.R_stride + (h % p.G) * p.T_q + i;
+  if (lane == 0) p.fold_ml[idx] = reinterpret_cast<const float2*>(p.part_ml)[row_id];
+  const float* src = p.part_a + row_id * D + lane * CPL;
+  float* dst = p.fold_a + idx * D + lane * CPL;
+#pragma unroll
+  for (int c = 0; c < CPL; ++c) dst[c] = src[c];
 }
 
 // ---------------------------------------------------------------------------------------
@@ -256,15 +285,29 @@ cudaError_t launch_local(const LocalParams& p, cudaStream_t s, bool pdl) {
 cudaError_t launch_finalize(const MergeParams& p, cudaStream_t s, bool pdl) {
   const int64_t rows = (int64_t)p.B * p.H_q * p.T_q;
   dim3 grid((unsigned)((rows + kWarpsPerCta - 1) / kWarpsPerCta)), block(kWarpsPerCta * 32);
-  if (p.d == 128) return launch_kernel(merge_kernel<128, false>, grid, block, 0, s, pdl, p);
-  return launch_kernel(merge_kernel<64, false>, grid, block, 0, s, pdl, p);
+  if (p.d == 128) return launch_kernel(merge_kernel<128, 0>, grid, block, 0, s, pdl, p);
+  return launch_kernel(merge_kernel<64, 0>, grid, block, 0, s, pdl, p);
 }
 
 cudaError_t launch_fold(const MergeParams& p, cudaStream_t s) {
   const int64_t rows = (int64_t)p.B * p.H_q * p.T_q;
   dim3 grid((unsigned)((rows + kWarpsPerCta - 1) / kWarpsPerCta)), block(kWarpsPerCta * 32);
-  if (p.d == 128) return launch_kernel(merge_kernel<128, true>, grid, block, 0, s, false, p);
-  return launch_kernel(merge_kernel<64, true>, grid, block, 0, s, false, p);
+  if (p.d == 128) return launch_kernel(merge_kernel<128, 1>, grid, block, 0, s, false, p);
+  return launch_kernel(merge_kernel<64, 1>, grid, block, 0, s, false, p);
+}
+
+cudaError_t launch_export(const MergeParams& p, cudaStream_t s) {
+  const int64_t rows = (int64_t)p.B * p.H_q * p.T_q;
+  dim3 grid((unsigned)((rows + kWarpsPerCta - 1) / kWarpsPerCta)), block(kWarpsPerCta * 32);
+  if (p.d == 128) return launch_kernel(merge_kernel<128, 2>, grid, block, 0, s, false, p);
+  return launch_kernel(merge_kernel<64, 2>, grid, block, 0, s, false, p);
+}
+
+cudaError_t launch_import(const MergeParams& p, cudaStream_t s) {
+  const int64_t rows = (int64_t)p.B * p.H_q * p.T_q;
+  dim3 grid((unsigned)((rows + kWarpsPerCta - 1) / kWarpsPerCta)), block(kWarpsPerCta * 32);
+  if (p.d == 128) return launch_kernel(import_kernel<128>, grid, block, 0, s, false, p);
+  return launch_kernel(import_kernel<64>, grid, block, 0, s, false, p);
 }
 
 cudaError_t launch_gather(const GatherParams& p, cudaStream_t s) {

@@ -104,6 +104,8 @@ cudaError_t chunk_tc_keys_prepare();
 cudaError_t launch_local(const LocalParams& p, cudaStream_t s, bool pdl);
 cudaError_t launch_finalize(const MergeParams& p, cudaStream_t s, bool pdl);
 cudaError_t launch_fold(const MergeParams& p, cudaStream_t s);
+cudaError_t launch_export(const MergeParams& p, cudaStream_t s);  // fold_ml/fold_a = caller buffers
+cudaError_t launch_import(const MergeParams& p, cudaStream_t s);  // part_ml/part_a = caller buffers
 cudaError_t launch_gather(const GatherParams& p, cudaStream_t s);
 
 // Launch helper: optional programmatic stream serialization attribute.

@@ -202,3 +202,55 @@ def test_trace_records_tile_loop():
         tops = [t[0] for t in tr[role] if t[0]]
         assert len(tops) >= 2 and all(b > a for a, b in zip(tops, tops[1:]))
     ctx.close()
+
+
+def test_export_import_state_shards_the_history_by_chunks():
+    """Two contexts each reduce half of the history chunks (what two GPUs would do), export
+    their merged states, a third imports both, adds the local segment and finalizes: the result
+    equals full attention (Eq. 17: the merge is order-free)."""
+    from oracle import streaming
+    cfg = inputs.VerifyConfig("v", 0x65, 2, 8, 2, 128, 256, 6, 700, 1500, k_mult=2.0)
+    lens = inputs.history_lengths(cfg)
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    rows = cfg.B * cfg.H_q * cfg.T_q
+    states = []
+    for part in (chunks[0::2], chunks[1::2]):
+        ctx = util.make_ctx(cfg)
+        ml = torch.empty(rows, 2, dtype=torch.float32, device=DEV)
+        a = torch.empty(rows, cfg.d, dtype=torch.float32, device=DEV)
+        ctx.ss_verify_begin(Q, cfg.scale)
+        for K, V, vl in part:
+            ctx.ss_verify_chunk(K, V, vl)
+        ctx.ss_verify_export_state(ml, a)
+        O_part = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
+        ctx.ss_verify_finalize(O_part, None)      # the round stays usable after an export
+        torch.cuda.synchronize()
+        states.append((ml, a))
+        ctx.close()
+    # an exported state is (m, l, a) of Eq. 13/14 up to the common reference: check a/l and
+    # m + log2 l of one shard against the literal chunk-state routine of the oracle
+    ml0, a0 = states[0]
+    b, h, i = 1, 5, 3
+    row = (b * cfg.H_q + h) * cfg.T_q + i
+    kvh = h // cfg.G
+    st = streaming.IDENTITY(1, cfg.d)
+    for K, V, vl in chunks[0::2]:
+        n = int(vl[b])
+        st = streaming.merge(st, streaming.chunk_partial(util.f64(Q[b, h, i:i + 1]), util.f64(K[b, kvh, :n]),
+                                                         util.f64(V[b, kvh, :n]), cfg.scale))
+    o_ref, lse_ref = streaming.finalize(st)
+    m, l = ml0[row].tolist()
+    assert abs((m + np.log2(l)) * np.log(2.0) - lse_ref[0]) < 1e-3
+    assert np.abs(a0[row].cpu().double().numpy() / l - o_ref[0]).max() < 2e-2 * max(1.0, np.abs(o_ref).max())
+    # combine the shards
+    ctx = util.make_ctx(cfg)
+    O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
+    LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
+    ctx.ss_verify_begin(Q, cfg.scale)
+    for ml, a in states:
+        ctx.ss_verify_import_state(ml, a)
+    ctx.ss_verify_local(K_loc, V_loc)
+    ctx.ss_verify_finalize(O, LSE)
+    torch.cuda.synchronize()
+    util.compare(cfg, O, LSE, util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits))
+    ctx.close()
