@@ -272,6 +272,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="plain launches (no programmatic dependent launch)")
     ap.add_argument("--simt", action="store_true", help="force the CUDA-core chunk kernel")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="also time N streamed layers back to back in the three pipeline modes "
+                         "(cross-layer prefetch / layer by layer / restore-then-verify)")
     ap.add_argument("--history-tokens", type=int, default=0,
                     help="shrink every request's history to this many tokens (small cases for profiler captures)")
     args = ap.parse_args()
@@ -428,6 +431,23 @@ def main():
                "h2d_GBps": h2d_gbps, "link_peak_GBps": best, "pct_of_link": 100.0 * h2d_gbps / best,
                "copies_per_round": int(stats.copies)}
         del probe_h, probe_d
+        if args.layers > 1 and rank == 0:
+            # N layers sharing this layer's host history (same lengths); one descriptor each
+            descs = [make_stream_desc(ssb, cfg, lens, host, dev, Qd, Kld, Vld, bits, O, LSE, bufs)
+                     for _ in range(args.layers)]
+            rk = torch.empty(cfg.B, cfg.H_kv, n_chunk_calls * cfg.L_c, cfg.d, dtype=torch.bfloat16, device=dev)
+            rv = torch.empty_like(rk)
+            abl = {}
+            for name, mode in (("stream_prefetch", ssb.SS_LAYERS_PREFETCH), ("stream_layerwise", ssb.SS_LAYERS_STREAM),
+                               ("restore_then_verify", ssb.SS_LAYERS_RESTORE)):
+                restore = (rk, rv) if mode == ssb.SS_LAYERS_RESTORE else (None, None)
+                ms_l = [ctx.ss_stream_layers(descs, mode, *restore).ms_device for _ in range(3)]
+                abl[name + "_ms"] = min(ms_l)
+            abl["layers"] = args.layers
+            abl["prefetch_vs_layerwise"] = abl["stream_layerwise_ms"] / abl["stream_prefetch_ms"]
+            abl["stream_vs_restore"] = abl["restore_then_verify_ms"] / abl["stream_layerwise_ms"]
+            e2e["layers_ablation"] = abl
+            del rk, rv
         del host
 
     cpu = None

@@ -221,6 +221,30 @@ typedef struct {
 
 ss_status ss_stream_round(ss_ctx* ctx, const ss_stream_desc* desc, ss_stream_stats* stats);
 
+/* Several layers back to back through the same two staging buffers (Section 4.2, pipelined KV
+ * transfers and prefetching; the modes mirror the paper's ablation of streaming designs):
+ *   SS_LAYERS_PREFETCH  stream-and-reduce with cross-layer prefetch: the copy stream starts the
+ *                       next layer's first fills as soon as a staging buffer frees, while the
+ *                       current layer's last attention, finalize and commit still run;
+ *   SS_LAYERS_STREAM    stream-and-reduce, layer by layer: a layer's copies start only when the
+ *                       previous layer's work is done;
+ *   SS_LAYERS_RESTORE   restore-then-verify baseline: the whole history of a layer is copied into
+ *                       restore_k / restore_v (device, [B, H_kv, restore_tokens, d]) and only then
+ *                       attended to; layers run strictly one after the other.
+ * Every layer has its own descriptor (history, Q, local KV, outputs); all layers use the same
+ * B, T_q, L_c, batch_chunks and staging buffers.  Layers may share the valid_len scratch arrays
+ * only if their history lengths are identical.  Synchronous; `total` covers all layers. */
+typedef enum { SS_LAYERS_PREFETCH = 0, SS_LAYERS_STREAM = 1, SS_LAYERS_RESTORE = 2 } ss_layers_mode;
+typedef struct {
+  int32_t n_layers;            /* <= 256                                                   */
+  const ss_stream_desc* layers; /* HOST array [n_layers]                                   */
+  int32_t mode;                /* ss_layers_mode                                           */
+  void* restore_k;             /* device; SS_LAYERS_RESTORE only                           */
+  void* restore_v;
+  int64_t restore_tokens;      /* token capacity of a restore buffer row                   */
+} ss_layers_desc;
+ss_status ss_stream_layers(ss_ctx* ctx, const ss_layers_desc* layers, ss_stream_stats* total);
+
 /* A whole round (one history chunk + local segment -> O, LSE) that allocates nothing and
  * needs no context or workspace.  The paper has no counterpart: this exists for callers that
  * cannot call cudaMalloc where they need attention (code in a region that must not

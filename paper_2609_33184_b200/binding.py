@@ -29,7 +29,7 @@ EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "
            "ss_verify_local", "ss_verify_finalize", "ss_commit_gather", "ss_poll_status",
            "ss_stream_round", "ss_strerror", "ss_sizeof_stream_desc", "ss_last_cuda_error", "ss_launch_count",
            "ss_last_chunk_kernel", "ss_trace_enable", "ss_trace_read", "ss_verify_round_static", "ss_verify_chunk_hinted", "ss_verify_export_state",
-           "ss_verify_import_state"]
+           "ss_verify_import_state", "ss_stream_layers"]
 
 
 class ss_config(C.Structure):
@@ -58,6 +58,14 @@ class ss_stream_desc(C.Structure):
                 ("host_commit_k", C.c_void_p), ("host_commit_v", C.c_void_p),
                 ("O_host", C.c_void_p), ("LSE_host", C.c_void_p),
                 ("copy_only", C.c_int32)]
+
+
+class ss_layers_desc(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("layers", C.POINTER(ss_stream_desc)), ("mode", C.c_int32),
+                ("restore_k", C.c_void_p), ("restore_v", C.c_void_p), ("restore_tokens", C.c_int64)]
+
+
+SS_LAYERS_PREFETCH, SS_LAYERS_STREAM, SS_LAYERS_RESTORE = 0, 1, 2
 
 
 class ss_static_round(C.Structure):
@@ -117,6 +125,8 @@ def load() -> C.CDLL:
     lib.ss_poll_status.argtypes = [vp, vp, i32, u32p]
     lib.ss_stream_round.restype = C.c_int
     lib.ss_stream_round.argtypes = [vp, C.POINTER(ss_stream_desc), C.POINTER(ss_stream_stats)]
+    lib.ss_stream_layers.restype = C.c_int
+    lib.ss_stream_layers.argtypes = [vp, C.POINTER(ss_layers_desc), C.POINTER(ss_stream_stats)]
     lib.ss_strerror.restype = C.c_char_p
     lib.ss_strerror.argtypes = [C.c_int]
     lib.ss_sizeof_stream_desc.restype = C.c_size_t
@@ -274,6 +284,15 @@ class Context:
         buf = (C.c_uint64 * n)()
         got = self.lib.ss_trace_read(self.handle, buf, n)
         return [[[buf[(r * 32 + t) * 8 + e] for e in range(8)] for t in range(32)] for r in range(3)][:3] if got else None
+
+    def ss_stream_layers(self, descs, mode: int = SS_LAYERS_PREFETCH, restore_k=None, restore_v=None) -> ss_stream_stats:
+        """descs: list of ss_stream_desc, one per layer."""
+        arr = (ss_stream_desc * len(descs))(*descs)
+        ld = ss_layers_desc(len(descs), arr, mode, _ptr(restore_k), _ptr(restore_v),
+                            restore_k.shape[2] if restore_k is not None else 0)
+        stats = ss_stream_stats()
+        self._check(self.lib.ss_stream_layers(self.handle, C.byref(ld), C.byref(stats)), "ss_stream_layers")
+        return stats
 
     def launch_count(self) -> int:
         return int(self.lib.ss_launch_count(self.handle))

@@ -1,7 +1,10 @@
-// Streamed round: pinned-host history -> two device staging buffers on a copy stream,
-// chunk attention on an attention stream, hand-off by events (Section 4.2, pipelined KV
-// transfers).  While the attention stream works on buffer A, buffer B receives the next
-// fill; a fill carries `batch_chunks` adjacent chunks (a transfer batch).
+// Streamed rounds: pinned-host history -> two device staging buffers on a copy stream, chunk
+// attention on an attention stream, hand-off by events (Section 4.2, pipelined KV transfers and
+// prefetching).  While the attention stream works on buffer A, buffer B receives the next fill;
+// a fill carries `batch_chunks` adjacent chunks (a transfer batch).  ss_stream_layers runs
+// several layers back to back: with cross-layer prefetch the copy stream starts the next
+// layer's first fills as soon as a staging buffer frees, without waiting for the current
+// layer's remaining attention, finalize and commit.
 #include <chrono>
 #include <cstring>
 
@@ -32,50 +35,64 @@ void ctx_pipeline_mode(ss_ctx* c, bool on);
     if (s_ != SS_OK) return s_;      \
   } while (0)
 
-static ss_status stream_round_impl(ss_ctx* ctx, const ss_stream_desc* d, ss_stream_stats* stats) {
-  if (!ctx || !d || !d->hist || !d->hist_len) return SS_ERR_ARG;
+namespace {
+
+struct LayerCounts {
+  int64_t h2d = 0, d2h = 0;
+  int copies = 0, calls = 0, fills = 0;
+};
+
+ss_status validate_desc(ss_ctx* ctx, const ss_stream_desc* d, int* n_fills_out) {
+  if (!d || !d->hist || !d->hist_len) return SS_ERR_ARG;
   if (d->B <= 0 || d->T_q <= 0 || d->L_c <= 0 || d->batch_chunks <= 0) return SS_ERR_ARG;
   if (!d->stage_k[0] || !d->stage_k[1] || !d->stage_v[0] || !d->stage_v[1]) return SS_ERR_ARG;
   if (!d->valid_len_host || !d->valid_len_dev) return SS_ERR_ARG;
   if (!d->copy_only && (!d->Q.ptr || !d->K_loc.ptr || !d->V_loc.ptr || !d->O)) return SS_ERR_ARG;
   int H_q, H_kv, hd;
-  const int max_B = ss::ctx_dims(ctx, &H_q, &H_kv, &hd);
-  if (d->B > max_B) return SS_ERR_SHAPE;
-  const int B = d->B, L_c = d->L_c, bc = d->batch_chunks;
-  const int64_t Ls = (int64_t)bc * L_c;  // tokens per staging buffer row
+  if (d->B > ss::ctx_dims(ctx, &H_q, &H_kv, &hd)) return SS_ERR_SHAPE;
   int max_len = 0;
-  for (int b = 0; b < B; ++b) {
+  for (int b = 0; b < d->B; ++b) {
     if (d->hist_len[b] < 0 || (d->hist_len[b] > 0 && !d->hist[b])) return SS_ERR_ARG;
     if (d->hist_len[b] > max_len) max_len = d->hist_len[b];
   }
-  const int n_chunks = (max_len + L_c - 1) / L_c;
-  const int n_fills = (n_chunks + bc - 1) / bc;
+  const int n_chunks = (max_len + d->L_c - 1) / d->L_c;
+  const int n_fills = (n_chunks + d->batch_chunks - 1) / d->batch_chunks;
   if (n_fills > d->scratch_fills) return SS_ERR_CAPACITY;
+  *n_fills_out = n_fills;
+  return SS_OK;
+}
 
-  ss::PipeRes r;
-  SS_CK(ss::ctx_pipeline(ctx, &r));
-  const auto wall0 = std::chrono::steady_clock::now();
+// Enqueue one layer's round on the two streams; synchronises nothing.  `fill_base` numbers the
+// fills across layers so that consecutive layers keep alternating the two staging buffers.
+// restore_k != null: the restore-then-verify baseline - the whole history of the layer is
+// copied into restore_k / restore_v first and only then attended to.
+ss_status enqueue_layer(ss_ctx* ctx, const ss_stream_desc* d, const ss::PipeRes& r, int n_fills,
+                        int fill_base, void* restore_k, void* restore_v, int64_t restore_tokens,
+                        LayerCounts* cnt) {
+  int H_q, H_kv, hd;
+  ss::ctx_dims(ctx, &H_q, &H_kv, &hd);
+  const int B = d->B, L_c = d->L_c, bc = d->batch_chunks;
+  const bool restore = restore_k != nullptr;
+  const int64_t Ls = restore ? restore_tokens : (int64_t)bc * L_c;  // tokens per device buffer row
+  if (restore && (int64_t)n_fills * bc * L_c > restore_tokens) return SS_ERR_CAPACITY;
 
   for (int f = 0; f < n_fills; ++f)
     for (int b = 0; b < B; ++b) {
-      int64_t v = (int64_t)d->hist_len[b] - (int64_t)f * Ls;
-      v = v < 0 ? 0 : (v > Ls ? Ls : v);
+      int64_t v = (int64_t)d->hist_len[b] - (int64_t)f * bc * L_c;
+      v = v < 0 ? 0 : (v > (int64_t)bc * L_c ? (int64_t)bc * L_c : v);
       d->valid_len_host[f * B + b] = (int32_t)v;
     }
-  SS_CK(cudaEventRecord(r.ev_t0, r.copy_stream));
   if (n_fills)
     SS_CK(cudaMemcpyAsync(d->valid_len_dev, d->valid_len_host, sizeof(int32_t) * n_fills * B,
                           cudaMemcpyHostToDevice, r.copy_stream));
   if (!d->copy_only) SS_ST(ss_verify_begin(ctx, d->Q, B, d->T_q, d->scale, r.attn_stream));
 
-  int64_t h2d = 0;
-  int copies = 0, calls = 0;
   const size_t esz = 2;
   const int64_t head_elems = (int64_t)L_c * hd;          // one head row of a host block
   const int64_t block_elems = 2 * (int64_t)H_kv * head_elems;
   for (int f = 0; f < n_fills; ++f) {
-    const int buf = f & 1;
-    if (f >= 2) SS_CK(cudaStreamWaitEvent(r.copy_stream, r.ev_free[buf], 0));
+    const int buf = (fill_base + f) & 1;
+    if (!restore && fill_base + f >= 2) SS_CK(cudaStreamWaitEvent(r.copy_stream, r.ev_free[buf], 0));
     for (int jj = 0; jj < bc; ++jj) {
       const int j = f * bc + jj;
       for (int b = 0; b < B; ++b) {
@@ -84,10 +101,12 @@ static ss_status stream_round_impl(ss_ctx* ctx, const ss_stream_desc* d, ss_stre
         if (v > L_c) v = L_c;
         const uint16_t* src = (const uint16_t*)d->hist[b] + (int64_t)j * block_elems;
         for (int kv = 0; kv < 2; ++kv) {
-          uint16_t* dst = (uint16_t*)(kv ? d->stage_v[buf] : d->stage_k[buf]) +
-                          ((int64_t)b * H_kv * Ls + (int64_t)jj * L_c) * hd;
+          uint16_t* base = restore ? (uint16_t*)(kv ? restore_v : restore_k)
+                                   : (uint16_t*)(kv ? d->stage_v[buf] : d->stage_k[buf]);
+          const int64_t tok = restore ? (int64_t)j * L_c : (int64_t)jj * L_c;
+          uint16_t* dst = base + ((int64_t)b * H_kv * Ls + tok) * hd;
           const uint16_t* s = src + (int64_t)kv * H_kv * head_elems;
-          if (v == L_c && bc == 1) {
+          if (v == L_c && Ls == L_c) {
             SS_CK(cudaMemcpyAsync(dst, s, (size_t)H_kv * head_elems * esz, cudaMemcpyHostToDevice,
                                   r.copy_stream));
           } else {
@@ -95,11 +114,12 @@ static ss_status stream_round_impl(ss_ctx* ctx, const ss_stream_desc* d, ss_stre
                                     (size_t)v * hd * esz, H_kv, cudaMemcpyHostToDevice,
                                     r.copy_stream));
           }
-          h2d += (int64_t)H_kv * v * hd * esz;
-          ++copies;
+          cnt->h2d += (int64_t)H_kv * v * hd * esz;
+          ++cnt->copies;
         }
       }
     }
+    if (restore) continue;  // attention starts after the last copy of the layer
     SS_CK(cudaEventRecord(r.ev_ready[buf], r.copy_stream));
     SS_CK(cudaStreamWaitEvent(r.attn_stream, r.ev_ready[buf], 0));
     if (!d->copy_only) {
@@ -107,71 +127,140 @@ static ss_status stream_round_impl(ss_ctx* ctx, const ss_stream_desc* d, ss_stre
       ss_tensor V = {d->stage_v[buf], (int64_t)H_kv * Ls * hd, Ls * hd, hd};
       SS_ST(ss_verify_chunk_hinted(ctx, K, V, (int32_t)Ls, d->valid_len_dev + (int64_t)f * B,
                                    d->valid_len_host + (int64_t)f * B, r.attn_stream));
-      ++calls;
+      ++cnt->calls;
     }
     SS_CK(cudaEventRecord(r.ev_free[buf], r.attn_stream));
   }
-  if (n_fills == 0) {
-    // nothing to stream: the attention stream still has to follow the copy stream's start
+  if (restore || n_fills == 0) {
+    // the attention stream follows the copy stream (whole history restored / nothing to stream)
     SS_CK(cudaEventRecord(r.ev_ready[0], r.copy_stream));
     SS_CK(cudaStreamWaitEvent(r.attn_stream, r.ev_ready[0], 0));
   }
-  int64_t d2h = 0;
+  if (restore && !d->copy_only) {
+    for (int f = 0; f < n_fills; ++f) {  // the streamed path's chunk calls, on the restored copy
+      const int64_t tok = (int64_t)f * bc * L_c;
+      ss_tensor K = {(uint16_t*)restore_k + tok * hd, (int64_t)H_kv * Ls * hd, Ls * hd, hd};
+      ss_tensor V = {(uint16_t*)restore_v + tok * hd, (int64_t)H_kv * Ls * hd, Ls * hd, hd};
+      SS_ST(ss_verify_chunk_hinted(ctx, K, V, bc * L_c, d->valid_len_dev + (int64_t)f * B,
+                                   d->valid_len_host + (int64_t)f * B, r.attn_stream));
+      ++cnt->calls;
+    }
+  }
+  cnt->fills += n_fills;
   if (!d->copy_only) {
-    SS_ST(ss_verify_local(ctx, d->K_loc, d->V_loc, d->T_q, d->mask_kind, d->mask_bits,
-                          r.attn_stream));
+    SS_ST(ss_verify_local(ctx, d->K_loc, d->V_loc, d->T_q, d->mask_kind, d->mask_bits, r.attn_stream));
     SS_ST(ss_verify_finalize(ctx, d->O, d->LSE, r.attn_stream));
     if (d->accept_idx) {
       if (!d->accept_cnt || !d->zero_off || !d->commit_k || !d->commit_v) return SS_ERR_ARG;
       const int64_t row = hd, tl = d->T_q;
       ss_tensor Kd = {d->commit_k, (int64_t)H_kv * tl * row, tl * row, row};
       ss_tensor Vd = {d->commit_v, (int64_t)H_kv * tl * row, tl * row, row};
-      SS_ST(ss_commit_gather(ctx, d->K_loc, d->V_loc, B, d->T_q, d->accept_idx, d->accept_cnt, Kd,
-                             Vd, d->T_q, d->zero_off, r.attn_stream));
+      SS_ST(ss_commit_gather(ctx, d->K_loc, d->V_loc, B, d->T_q, d->accept_idx, d->accept_cnt, Kd, Vd,
+                             d->T_q, d->zero_off, r.attn_stream));
       const size_t bytes = (size_t)B * H_kv * tl * row * esz;
       if (d->host_commit_k) {
-        SS_CK(cudaMemcpyAsync(d->host_commit_k, d->commit_k, bytes, cudaMemcpyDeviceToHost,
-                              r.attn_stream));
-        d2h += bytes;
+        SS_CK(cudaMemcpyAsync(d->host_commit_k, d->commit_k, bytes, cudaMemcpyDeviceToHost, r.attn_stream));
+        cnt->d2h += bytes;
       }
       if (d->host_commit_v) {
-        SS_CK(cudaMemcpyAsync(d->host_commit_v, d->commit_v, bytes, cudaMemcpyDeviceToHost,
-                              r.attn_stream));
-        d2h += bytes;
+        SS_CK(cudaMemcpyAsync(d->host_commit_v, d->commit_v, bytes, cudaMemcpyDeviceToHost, r.attn_stream));
+        cnt->d2h += bytes;
       }
     }
     if (d->O_host) {
       const size_t bytes = (size_t)B * H_q * d->T_q * hd * esz;
       SS_CK(cudaMemcpyAsync(d->O_host, d->O, bytes, cudaMemcpyDeviceToHost, r.attn_stream));
-      d2h += bytes;
+      cnt->d2h += bytes;
     }
     if (d->LSE_host && d->LSE) {
       const size_t bytes = (size_t)B * H_q * d->T_q * sizeof(float);
       SS_CK(cudaMemcpyAsync(d->LSE_host, d->LSE, bytes, cudaMemcpyDeviceToHost, r.attn_stream));
-      d2h += bytes;
+      cnt->d2h += bytes;
     }
+  }
+  return SS_OK;
+}
+
+void fill_stats(ss_stream_stats* st, const LayerCounts& c, float ms_device, double ms_total) {
+  if (!st) return;
+  st->ms_device = ms_device;
+  st->ms_total = ms_total;
+  st->h2d_bytes = c.h2d;
+  st->d2h_bytes = c.d2h;
+  st->chunk_calls = c.calls;
+  st->copies = c.copies;
+}
+
+ss_status stream_round_impl(ss_ctx* ctx, const ss_stream_desc* d, ss_stream_stats* stats) {
+  int n_fills = 0;
+  SS_ST(validate_desc(ctx, d, &n_fills));
+  ss::PipeRes r;
+  SS_CK(ss::ctx_pipeline(ctx, &r));
+  const auto wall0 = std::chrono::steady_clock::now();
+  SS_CK(cudaEventRecord(r.ev_t0, r.copy_stream));
+  LayerCounts cnt;
+  SS_ST(enqueue_layer(ctx, d, r, n_fills, 0, nullptr, nullptr, 0, &cnt));
+  SS_CK(cudaEventRecord(r.ev_t1, r.attn_stream));
+  SS_CK(cudaEventSynchronize(r.ev_t1));
+  SS_CK(cudaStreamSynchronize(r.copy_stream));
+  float ms = 0.f;
+  SS_CK(cudaEventElapsedTime(&ms, r.ev_t0, r.ev_t1));
+  fill_stats(stats, cnt, ms,
+             std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - wall0).count());
+  return SS_OK;
+}
+
+ss_status stream_layers_impl(ss_ctx* ctx, const ss_layers_desc* ld, ss_stream_stats* total) {
+  if (!ld || !ld->layers || ld->n_layers <= 0) return SS_ERR_ARG;
+  if (ld->mode < SS_LAYERS_PREFETCH || ld->mode > SS_LAYERS_RESTORE) return SS_ERR_ARG;
+  if (ld->mode == SS_LAYERS_RESTORE && (!ld->restore_k || !ld->restore_v || ld->restore_tokens <= 0))
+    return SS_ERR_ARG;
+  if (ld->n_layers > 256) return SS_ERR_SHAPE;
+  ss::PipeRes r;
+  SS_CK(ss::ctx_pipeline(ctx, &r));
+  int n_fills[256];
+  for (int l = 0; l < ld->n_layers; ++l) SS_ST(validate_desc(ctx, &ld->layers[l], &n_fills[l]));
+
+  const auto wall0 = std::chrono::steady_clock::now();
+  SS_CK(cudaEventRecord(r.ev_t0, r.copy_stream));
+  LayerCounts cnt;
+  int fill_base = 0;
+  const bool restore = ld->mode == SS_LAYERS_RESTORE;
+  for (int l = 0; l < ld->n_layers; ++l) {
+    if (l > 0 && ld->mode != SS_LAYERS_PREFETCH) {
+      // no prefetch: the next layer's copies start only when this layer's work is done
+      SS_CK(cudaEventRecord(r.ev_t1, r.attn_stream));
+      SS_CK(cudaStreamWaitEvent(r.copy_stream, r.ev_t1, 0));
+    }
+    SS_ST(enqueue_layer(ctx, &ld->layers[l], r, n_fills[l], restore ? 0 : fill_base,
+                        restore ? ld->restore_k : nullptr, restore ? ld->restore_v : nullptr,
+                        ld->restore_tokens, &cnt));
+    if (!restore) fill_base += n_fills[l];
   }
   SS_CK(cudaEventRecord(r.ev_t1, r.attn_stream));
   SS_CK(cudaEventSynchronize(r.ev_t1));
   SS_CK(cudaStreamSynchronize(r.copy_stream));
-  if (stats) {
-    float ms = 0.f;
-    SS_CK(cudaEventElapsedTime(&ms, r.ev_t0, r.ev_t1));
-    stats->ms_device = ms;
-    stats->ms_total = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - wall0)
-                          .count();
-    stats->h2d_bytes = h2d;
-    stats->d2h_bytes = d2h;
-    stats->chunk_calls = calls;
-    stats->copies = copies;
-  }
+  float ms = 0.f;
+  SS_CK(cudaEventElapsedTime(&ms, r.ev_t0, r.ev_t1));
+  fill_stats(total, cnt, ms,
+             std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - wall0).count());
   return SS_OK;
 }
+
+}  // namespace
 
 extern "C" ss_status ss_stream_round(ss_ctx* ctx, const ss_stream_desc* d, ss_stream_stats* stats) {
   if (!ctx) return SS_ERR_ARG;
   ss::ctx_pipeline_mode(ctx, true);
   const ss_status st = stream_round_impl(ctx, d, stats);
+  ss::ctx_pipeline_mode(ctx, false);
+  return st;
+}
+
+extern "C" ss_status ss_stream_layers(ss_ctx* ctx, const ss_layers_desc* layers, ss_stream_stats* total) {
+  if (!ctx) return SS_ERR_ARG;
+  ss::ctx_pipeline_mode(ctx, true);
+  const ss_status st = stream_layers_impl(ctx, layers, total);
   ss::ctx_pipeline_mode(ctx, false);
   return st;
 }

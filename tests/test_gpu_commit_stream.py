@@ -254,3 +254,54 @@ def test_export_import_state_shards_the_history_by_chunks():
     torch.cuda.synchronize()
     util.compare(cfg, O, LSE, util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits))
     ctx.close()
+
+
+def _layer_descs(ssb, cfg, lens, n_layers, bufs):
+    """One stream descriptor per layer: own history / Q / local KV / outputs, shared staging."""
+    import dataclasses
+    layers = []
+    for l in range(n_layers):
+        cfg_l = dataclasses.replace(cfg, seed=cfg.seed + 17 * l)
+        Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg_l, lens, DEV, fill=0.0)
+        host = bench.pinned_history(cfg_l, lens, chunks)
+        O = torch.zeros(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
+        LSE = torch.zeros(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
+        lb = dict(bufs)
+        lb["O_host"] = torch.zeros(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16).pin_memory()
+        lb["LSE_host"] = torch.zeros(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32).pin_memory()
+        desc = bench.make_stream_desc(ssb, cfg_l, lens, host, DEV, Q, K_loc, V_loc, bits, O, LSE, lb)
+        layers.append(dict(cfg=cfg_l, case=(Q, chunks, K_loc, V_loc, bits), host=host, O=O, LSE=LSE, desc=desc,
+                           bufs=lb))
+    return layers
+
+
+def test_stream_layers_modes_match_oracle_and_each_other():
+    ssb = _ssb()
+    cfg = inputs.VerifyConfig("v", 0x66, 3, 8, 2, 128, 256, 8, 200, 1300)
+    lens = [1300, 200, 777]
+    n_chunks = inputs.num_chunks(cfg, lens)
+    bufs = bench.stream_buffers(cfg, DEV, n_chunks)
+    layers = _layer_descs(ssb, cfg, lens, 3, bufs)
+    ctx = ssb.Context(cfg.B, cfg.H_q, cfg.H_kv, cfg.d, cfg.T_q, cfg.T_q, cfg.L_c)
+    rk = torch.full((cfg.B, cfg.H_kv, n_chunks * cfg.L_c, cfg.d), float("nan"), dtype=torch.bfloat16, device=DEV)
+    rv = torch.full_like(rk, float("nan"))
+    outs = {}
+    for mode in (ssb.SS_LAYERS_PREFETCH, ssb.SS_LAYERS_STREAM, ssb.SS_LAYERS_RESTORE):
+        for L in layers:
+            L["O"].zero_()
+            L["LSE"].zero_()
+        restore = (rk, rv) if mode == ssb.SS_LAYERS_RESTORE else (None, None)
+        stats = ctx.ss_stream_layers([L["desc"] for L in layers], mode, *restore)
+        st, dev_bits = ctx.ss_poll_status()
+        assert st == 0, dev_bits
+        assert stats.h2d_bytes == 3 * sum(lens) * cfg.H_kv * cfg.d * 4
+        assert stats.chunk_calls == 3 * n_chunks
+        outs[mode] = [(L["O"].clone(), L["LSE"].clone()) for L in layers]
+        for L in layers:
+            assert torch.equal(L["bufs"]["O_host"], L["O"].cpu())
+    for L, (O, LSE) in zip(layers, outs[ssb.SS_LAYERS_PREFETCH]):
+        util.compare(L["cfg"], O, LSE, util.oracle_case(L["cfg"], lens, *L["case"]))
+    for mode in (ssb.SS_LAYERS_STREAM, ssb.SS_LAYERS_RESTORE):
+        for (O0, L0), (O1, L1) in zip(outs[ssb.SS_LAYERS_PREFETCH], outs[mode]):
+            assert torch.equal(O0.view(torch.int16), O1.view(torch.int16)) and torch.equal(L0, L1)
+    ctx.close()
