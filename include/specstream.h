@@ -208,6 +208,13 @@ typedef struct {
   void* O_host;              /* pinned HOST or NULL                                       */
   float* LSE_host;           /* pinned HOST or NULL                                       */
   int32_t copy_only;         /* 1: issue the same copies but no attention (control run)   */
+  /* optional on-GPU Active Tail (committed KV not yet offloaded): attended to as one more chunk */
+  ss_tensor tail_K, tail_V;  /* device [B, H_kv, tail_Lc, d]; tail_K.ptr NULL = none           */
+  int32_t tail_Lc;
+  const int32_t* tail_len;   /* device [B] valid tokens of the tail                           */
+  int32_t commit_cap;        /* token capacity of commit_k / commit_v rows (0 = T_q); with a
+                                tail, commit_k/v may be the tail buffers and zero_off their
+                                lengths, so accepted rows are appended to the tail in place   */
 } ss_stream_desc;
 
 typedef struct {
@@ -234,6 +241,39 @@ ss_status ss_stream_round(ss_ctx* ctx, const ss_stream_desc* desc, ss_stream_sta
  * Every layer has its own descriptor (history, Q, local KV, outputs); all layers use the same
  * B, T_q, L_c, batch_chunks and staging buffers.  Layers may share the valid_len scratch arrays
  * only if their history lengths are identical.  Synchronous; `total` covers all layers. */
+/* Commit-aware KV tiering (Section 4.1).  Per request: Sealed History [0, H) in pinned host
+ * memory (chunk-block layout of ss_stream_round), Active Tail [H, C) in a device buffer
+ * [B, H_kv, tail_capacity, d] (token t at index t - H).  ss_tier_commit advances C by the rows a
+ * commit-gather appended; ss_tier_migrate computes the Eq. 9 end point
+ * E = max{H, g * floor(max(0, C - T) / g)} per request and starts the asynchronous copy of
+ * [H, E) to the host; ss_tier_poll advances H to E only once that copy is confirmed and then
+ * moves the surviving tails to the front of the other tail buffer (all requests swap together).
+ * Rejected candidates live past C and never reach the host, so there is no host-side rollback.
+ * Host logic only; every copy is enqueued on the given stream.  len_dev (device [B]) always holds
+ * C - H: the valid length of the tail chunk and the offset the next commit-gather appends at.
+ * len_host is pinned HOST scratch of 4 * B int32. */
+typedef struct ss_tier ss_tier;
+typedef struct {
+  int32_t B, H_kv, d, L_c;
+  int32_t tail_target;   /* T: committed tokens kept on the GPU                                */
+  int32_t granularity;   /* g: offload batch, H stays a multiple of it                         */
+  int32_t tail_capacity; /* tokens per tail buffer row, >= T + g (+ a round of accepted rows)  */
+} ss_tier_config;
+ss_status ss_tier_create(ss_tier** out, const ss_tier_config* cfg, void* const* host_hist,
+                         const int64_t* host_capacity_tokens, void* tail_k0, void* tail_v0,
+                         void* tail_k1, void* tail_v1, int32_t* len_dev, int32_t* len_host);
+ss_status ss_tier_destroy(ss_tier* tier);
+/* Set the boundaries (HOST [B] each; H multiple of g, tail data already at index t - H of buffer 0). */
+ss_status ss_tier_reset(ss_tier* tier, const int32_t* H, const int32_t* C, void* stream);
+/* Read the boundaries (any pointer may be NULL); pending_E = end point of the copy in flight. */
+ss_status ss_tier_get(ss_tier* tier, int32_t* H, int32_t* C, int32_t* pending_E, int32_t* cur_buffer);
+/* Current tail view and the device array of tail lengths. */
+ss_status ss_tier_tail(ss_tier* tier, ss_tensor* K, ss_tensor* V, const int32_t** tail_len_dev);
+ss_status ss_tier_commit(ss_tier* tier, const int32_t* cnt_host, void* stream);
+ss_status ss_tier_migrate(ss_tier* tier, void* stream, int32_t* n_requests);
+ss_status ss_tier_poll(ss_tier* tier, int32_t wait, void* stream, int32_t* advanced);
+int64_t ss_tier_d2h_bytes(ss_tier* tier);
+
 typedef enum { SS_LAYERS_PREFETCH = 0, SS_LAYERS_STREAM = 1, SS_LAYERS_RESTORE = 2 } ss_layers_mode;
 typedef struct {
   int32_t n_layers;            /* <= 256                                                   */

@@ -29,7 +29,9 @@ EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "
            "ss_verify_local", "ss_verify_finalize", "ss_commit_gather", "ss_poll_status",
            "ss_stream_round", "ss_strerror", "ss_sizeof_stream_desc", "ss_last_cuda_error", "ss_launch_count",
            "ss_last_chunk_kernel", "ss_trace_enable", "ss_trace_read", "ss_verify_round_static", "ss_verify_chunk_hinted", "ss_verify_export_state",
-           "ss_verify_import_state", "ss_stream_layers"]
+           "ss_verify_import_state", "ss_stream_layers", "ss_tier_create", "ss_tier_destroy",
+           "ss_tier_reset", "ss_tier_get", "ss_tier_tail", "ss_tier_commit", "ss_tier_migrate", "ss_tier_poll",
+           "ss_tier_d2h_bytes"]
 
 
 class ss_config(C.Structure):
@@ -57,7 +59,14 @@ class ss_stream_desc(C.Structure):
                 ("commit_k", C.c_void_p), ("commit_v", C.c_void_p),
                 ("host_commit_k", C.c_void_p), ("host_commit_v", C.c_void_p),
                 ("O_host", C.c_void_p), ("LSE_host", C.c_void_p),
-                ("copy_only", C.c_int32)]
+                ("copy_only", C.c_int32),
+                ("tail_K", ss_tensor), ("tail_V", ss_tensor), ("tail_Lc", C.c_int32),
+                ("tail_len", C.c_void_p), ("commit_cap", C.c_int32)]
+
+
+class ss_tier_config(C.Structure):
+    _fields_ = [("B", C.c_int32), ("H_kv", C.c_int32), ("d", C.c_int32), ("L_c", C.c_int32),
+                ("tail_target", C.c_int32), ("granularity", C.c_int32), ("tail_capacity", C.c_int32)]
 
 
 class ss_layers_desc(C.Structure):
@@ -127,6 +136,26 @@ def load() -> C.CDLL:
     lib.ss_stream_round.argtypes = [vp, C.POINTER(ss_stream_desc), C.POINTER(ss_stream_stats)]
     lib.ss_stream_layers.restype = C.c_int
     lib.ss_stream_layers.argtypes = [vp, C.POINTER(ss_layers_desc), C.POINTER(ss_stream_stats)]
+    i32p, i64p = C.POINTER(C.c_int32), C.POINTER(C.c_int64)
+    lib.ss_tier_create.restype = C.c_int
+    lib.ss_tier_create.argtypes = [C.POINTER(vp), C.POINTER(ss_tier_config), C.POINTER(vp), i64p, vp, vp, vp, vp,
+                                   vp, vp]
+    lib.ss_tier_destroy.restype = C.c_int
+    lib.ss_tier_destroy.argtypes = [vp]
+    lib.ss_tier_reset.restype = C.c_int
+    lib.ss_tier_reset.argtypes = [vp, i32p, i32p, vp]
+    lib.ss_tier_get.restype = C.c_int
+    lib.ss_tier_get.argtypes = [vp, i32p, i32p, i32p, i32p]
+    lib.ss_tier_tail.restype = C.c_int
+    lib.ss_tier_tail.argtypes = [vp, C.POINTER(ss_tensor), C.POINTER(ss_tensor), C.POINTER(vp)]
+    lib.ss_tier_commit.restype = C.c_int
+    lib.ss_tier_commit.argtypes = [vp, i32p, vp]
+    lib.ss_tier_migrate.restype = C.c_int
+    lib.ss_tier_migrate.argtypes = [vp, vp, i32p]
+    lib.ss_tier_poll.restype = C.c_int
+    lib.ss_tier_poll.argtypes = [vp, i32, vp, i32p]
+    lib.ss_tier_d2h_bytes.restype = C.c_int64
+    lib.ss_tier_d2h_bytes.argtypes = [vp]
     lib.ss_strerror.restype = C.c_char_p
     lib.ss_strerror.argtypes = [C.c_int]
     lib.ss_sizeof_stream_desc.restype = C.c_size_t
@@ -316,3 +345,69 @@ def verify_round(ctx: Context, Q, chunks: Sequence, K_loc, V_loc, scale: float, 
         ctx.ss_verify_local(K_loc, V_loc, mask_kind, mask_bits, stream)
     ctx.ss_verify_finalize(O, LSE, stream)
     return O, LSE
+
+
+class Tier:
+    """Owns an ss_tier: boundaries H <= C per request, tail buffers, offload of [H, E) (Eq. 9)."""
+
+    def __init__(self, B, H_kv, d, L_c, tail_target, granularity, tail_capacity, host_hist, device="cuda:0"):
+        self.lib = load()
+        self.cfg = ss_tier_config(B, H_kv, d, L_c, tail_target, granularity, tail_capacity)
+        self.host_hist = host_hist  # list of pinned tensors, chunk-block layout
+        self.tail_k = [torch.zeros(B, H_kv, tail_capacity, d, dtype=torch.bfloat16, device=device) for _ in range(2)]
+        self.tail_v = [torch.zeros(B, H_kv, tail_capacity, d, dtype=torch.bfloat16, device=device) for _ in range(2)]
+        self.len_dev = torch.zeros(B, dtype=torch.int32, device=device)
+        self.len_host = torch.zeros(4 * B, dtype=torch.int32).pin_memory()
+        ptrs = (C.c_void_p * B)(*[h.data_ptr() for h in host_hist])
+        caps = (C.c_int64 * B)(*[h.numel() // (2 * H_kv * d) for h in host_hist])
+        self.handle = C.c_void_p()
+        st = self.lib.ss_tier_create(C.byref(self.handle), C.byref(self.cfg), ptrs, caps,
+                                     self.tail_k[0].data_ptr(), self.tail_v[0].data_ptr(),
+                                     self.tail_k[1].data_ptr(), self.tail_v[1].data_ptr(),
+                                     self.len_dev.data_ptr(), self.len_host.data_ptr())
+        if st != SS_OK:
+            raise SpecStreamError(st, "ss_tier_create")
+        self.B = B
+
+    def _arr(self, xs):
+        return (C.c_int32 * self.B)(*[int(x) for x in xs])
+
+    def _check(self, st, where):
+        if st != SS_OK:
+            raise SpecStreamError(st, where)
+
+    def reset(self, H, Cc, stream=None):
+        self._check(self.lib.ss_tier_reset(self.handle, self._arr(H), self._arr(Cc), _stream_ptr(stream)), "ss_tier_reset")
+
+    def get(self):
+        H, Cc, E = self._arr([0] * self.B), self._arr([0] * self.B), self._arr([0] * self.B)
+        cur = C.c_int32(0)
+        self._check(self.lib.ss_tier_get(self.handle, H, Cc, E, C.byref(cur)), "ss_tier_get")
+        return list(H), list(Cc), list(E), cur.value
+
+    def tail(self):
+        K, V, p = ss_tensor(), ss_tensor(), C.c_void_p()
+        self._check(self.lib.ss_tier_tail(self.handle, C.byref(K), C.byref(V), C.byref(p)), "ss_tier_tail")
+        cur = self.get()[3]
+        return self.tail_k[cur], self.tail_v[cur], K, V
+
+    def commit(self, cnt, stream=None):
+        self._check(self.lib.ss_tier_commit(self.handle, self._arr(cnt), _stream_ptr(stream)), "ss_tier_commit")
+
+    def migrate(self, stream=None) -> int:
+        n = C.c_int32(0)
+        self._check(self.lib.ss_tier_migrate(self.handle, _stream_ptr(stream), C.byref(n)), "ss_tier_migrate")
+        return n.value
+
+    def poll(self, wait: bool, stream=None) -> bool:
+        adv = C.c_int32(0)
+        self._check(self.lib.ss_tier_poll(self.handle, 1 if wait else 0, _stream_ptr(stream), C.byref(adv)), "ss_tier_poll")
+        return bool(adv.value)
+
+    def d2h_bytes(self) -> int:
+        return int(self.lib.ss_tier_d2h_bytes(self.handle))
+
+    def close(self):
+        if self.handle:
+            self.lib.ss_tier_destroy(self.handle)
+            self.handle = C.c_void_p()

@@ -85,7 +85,14 @@ ss_status enqueue_layer(ss_ctx* ctx, const ss_stream_desc* d, const ss::PipeRes&
   if (n_fills)
     SS_CK(cudaMemcpyAsync(d->valid_len_dev, d->valid_len_host, sizeof(int32_t) * n_fills * B,
                           cudaMemcpyHostToDevice, r.copy_stream));
-  if (!d->copy_only) SS_ST(ss_verify_begin(ctx, d->Q, B, d->T_q, d->scale, r.attn_stream));
+  if (!d->copy_only) {
+    SS_ST(ss_verify_begin(ctx, d->Q, B, d->T_q, d->scale, r.attn_stream));
+    if (d->tail_K.ptr) {  // on-GPU Active Tail: no copy, runs while the first fills arrive
+      if (!d->tail_V.ptr || d->tail_Lc <= 0) return SS_ERR_ARG;
+      SS_ST(ss_verify_chunk(ctx, d->tail_K, d->tail_V, d->tail_Lc, d->tail_len, r.attn_stream));
+      ++cnt->calls;
+    }
+  }
 
   const size_t esz = 2;
   const int64_t head_elems = (int64_t)L_c * hd;          // one head row of a host block
@@ -152,11 +159,11 @@ ss_status enqueue_layer(ss_ctx* ctx, const ss_stream_desc* d, const ss::PipeRes&
     SS_ST(ss_verify_finalize(ctx, d->O, d->LSE, r.attn_stream));
     if (d->accept_idx) {
       if (!d->accept_cnt || !d->zero_off || !d->commit_k || !d->commit_v) return SS_ERR_ARG;
-      const int64_t row = hd, tl = d->T_q;
+      const int64_t row = hd, tl = d->commit_cap > 0 ? d->commit_cap : d->T_q;
       ss_tensor Kd = {d->commit_k, (int64_t)H_kv * tl * row, tl * row, row};
       ss_tensor Vd = {d->commit_v, (int64_t)H_kv * tl * row, tl * row, row};
       SS_ST(ss_commit_gather(ctx, d->K_loc, d->V_loc, B, d->T_q, d->accept_idx, d->accept_cnt, Kd, Vd,
-                             d->T_q, d->zero_off, r.attn_stream));
+                             (int32_t)tl, d->zero_off, r.attn_stream));
       const size_t bytes = (size_t)B * H_kv * tl * row * esz;
       if (d->host_commit_k) {
         SS_CK(cudaMemcpyAsync(d->host_commit_k, d->commit_k, bytes, cudaMemcpyDeviceToHost, r.attn_stream));
