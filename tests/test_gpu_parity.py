@@ -231,3 +231,27 @@ def test_hinted_chunk_calls_match_unhinted():
     assert st == 0, dev_bits
     util.compare(cfg, O, LSE, ref)
     ctx.close()
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_ragged_shapes(seed):
+    # seeded sweep over batch, GQA group, candidate count, head dim, chunk size, ragged lengths,
+    # mask kind and kernel choice; short and peaked cases give the masks real weight
+    import random
+    rng = random.Random(1000 + seed)
+    d = rng.choice([64, 128, 128])
+    H_kv = rng.choice([1, 2, 3])
+    G = rng.choice([1, 2, 4, 5, 8])
+    T_q = rng.randint(1, 12)
+    B = rng.randint(1, 4)
+    L_c = rng.choice([64, 96, 128, 200, 256, 448])
+    hi = rng.choice([0, 40, 300, 900])
+    mask = rng.choice(["chain", "tree"])
+    cfg = inputs.VerifyConfig("rnd", 0xA000 + seed, B, H_kv * G, H_kv, d, L_c, T_q, 0, hi, mask=mask,
+                              k_mult=rng.choice([1.0, 2.0, 6.0]))
+    lens = [rng.randint(0, hi) for _ in range(B)]
+    flags = rng.choice([0, 0, 1, 4, 8]) | rng.choice([0, 2])
+    n = inputs.num_chunks(cfg, lens)
+    order = list(range(n))
+    rng.shuffle(order)
+    _run(cfg, lens=lens, flags=flags, order=order, local_at=rng.randint(0, n), max_chunks=rng.choice([0, 2]))
