@@ -264,7 +264,7 @@ def run_reference(args, cfg, rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_qwen3_8b", choices=sorted(inputs.CONFIGS))
@@ -341,7 +341,8 @@ def main():
     ms = e0.elapsed_time(e1)
     ms = ssdist.max_over_ranks(ms, dev)
     ms_per_step = ms / args.steps
-    value = world * nbytes / (ms_per_step * 1e-3) / 1e9
+    job_bytes = ssdist.sum_over_ranks(nbytes, dev)   # whole job: every rank's own requests
+    value = job_bytes / (ms_per_step * 1e-3) / 1e9
     st, dev_bits = ctx.ss_poll_status()
     if st != 0:
         raise SystemExit(f"device status word set: {dev_bits}")
@@ -422,7 +423,7 @@ def main():
         desc.copy_only = 0
         full = [ctx.ss_stream_round(desc).ms_device for _ in range(3)]
         h2d_gbps = stats.h2d_bytes / (min(full) * 1e-3) / 1e9
-        e2e = {"value": world * nbytes / dt / 1e9, "unit": UNIT,
+        e2e = {"value": job_bytes / dt / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": int(stats.h2d_bytes + small_in),
                "d2h_bytes_per_step": int(stats.d2h_bytes), "ms_per_step": dt * 1e3,
                "api": "ss_stream_round (pinned host history, 2 staging buffers)",

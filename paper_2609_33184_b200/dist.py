@@ -40,6 +40,16 @@ def max_over_ranks(value: float, device="cpu") -> float:
     return float(t.item())
 
 
+def sum_over_ranks(value: float, device="cpu") -> float:
+    """Sum of a per-rank scalar (bytes processed) over all ranks; identity without a process group."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
 def barrier(cuda: bool = False):
     import torch.distributed as dist
     if dist.is_available() and dist.is_initialized():

@@ -40,6 +40,7 @@ def _worker(rank, world, port, out):
         ssdist.barrier()
         t = ssdist.max_over_ranks(1.0 + rank)
         assert t == float(world)
+        assert ssdist.sum_over_ranks(10.0 * (rank + 1)) == 30.0   # whole-job units = sum over ranks
         out.put((rank, "ok"))
     except Exception as e:  # pragma: no cover
         out.put((rank, repr(e)))
@@ -61,7 +62,7 @@ def test_two_rank_gloo_plumbing():
 
 
 def test_single_process_helpers():
-    assert ssdist.max_over_ranks(3.5) == 3.5
+    assert ssdist.max_over_ranks(3.5) == 3.5 and ssdist.sum_over_ranks(2.0) == 2.0
     assert list(ssdist.shard_requests(5, 0, 1)) == [0, 1, 2, 3, 4]
     sizes = [len(ssdist.shard_requests(10, r, 4)) for r in range(4)]
     assert sizes == [3, 3, 2, 2]
