@@ -62,6 +62,7 @@ typedef enum {
 #define SS_DEV_BAD_ACCEPT 2u    /* accept_cnt/accept_idx out of range: row skipped     */
 #define SS_DEV_DST_OVERFLOW 4u  /* dst_off + k outside [0, cap): row skipped           */
 #define SS_DEV_WAIT_EXPIRED 8u  /* a bounded in-kernel wait gave up: round is invalid  */
+#define SS_DEV_BAD_PAGE 16u     /* page id outside the pool: its tokens read as zeros  */
 
 typedef struct {
   int32_t max_B;      /* requests per call                                          */
@@ -129,6 +130,18 @@ ss_status ss_verify_chunk(ss_ctx* ctx, ss_tensor K, ss_tensor V, int32_t L_c,
 ss_status ss_verify_chunk_hinted(ss_ctx* ctx, ss_tensor K, ss_tensor V, int32_t L_c,
                                  const int32_t* valid_len, const int32_t* valid_len_host,
                                  void* stream);
+
+/* A chunk whose tokens live in pages of a pool (requests keep independent KV indices): K_pool,
+ * V_pool are [n_pages, H_kv, page_size, d] (ss_tensor: stride_b = page stride); the chunk of
+ * request b is the concatenation of pages page_table[b][0 .. pages_per_req) (device int32
+ * [B, pages_per_req]), i.e. L_c = pages_per_req * page_size tokens of which valid_len[b] are
+ * valid (NULL = all).  Same result as ss_verify_chunk on the gathered chunk.  The tensor-core
+ * kernels need page_size to be a multiple of 128 (keys on M) or 64 (rows on M); other page sizes
+ * take the CUDA-core kernel.  valid_len_host (HOST, may be NULL) is the scheduling hint of
+ * ss_verify_chunk_hinted.  A page id outside [0, n_pages) raises SS_DEV_BAD_PAGE. */
+ss_status ss_verify_chunk_paged(ss_ctx* ctx, ss_tensor K_pool, ss_tensor V_pool, int32_t n_pages,
+                                int32_t page_size, const int32_t* page_table, int32_t pages_per_req,
+                                const int32_t* valid_len, const int32_t* valid_len_host, void* stream);
 
 /* a4. The on-GPU candidate segment: K_loc, V_loc [B, H_kv, T_loc, d].  Query i of request
  * b sees local token j iff

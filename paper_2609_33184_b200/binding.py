@@ -21,7 +21,7 @@ STATUS_NAMES = ["SS_OK", "SS_ERR_ARG", "SS_ERR_SHAPE", "SS_ERR_ALIGN", "SS_ERR_S
                 "SS_ERR_TIMEOUT"]
 (SS_ERR_ARG, SS_ERR_SHAPE, SS_ERR_ALIGN, SS_ERR_STATE, SS_ERR_CAPACITY, SS_ERR_UNSUPPORTED,
  SS_ERR_CUDA, SS_ERR_DEVICE_FLAG, SS_ERR_TIMEOUT) = range(1, 10)
-SS_DEV_BAD_VALID_LEN, SS_DEV_BAD_ACCEPT, SS_DEV_DST_OVERFLOW, SS_DEV_WAIT_EXPIRED = 1, 2, 4, 8
+SS_DEV_BAD_VALID_LEN, SS_DEV_BAD_ACCEPT, SS_DEV_DST_OVERFLOW, SS_DEV_WAIT_EXPIRED, SS_DEV_BAD_PAGE = 1, 2, 4, 8, 16
 SS_FLAG_FORCE_SIMT, SS_FLAG_OVERLAP_CHUNKS, SS_FLAG_ROWS_ON_M, SS_FLAG_KEYS_ON_M = 1, 2, 4, 8
 SS_MASK_CHAIN, SS_MASK_TREE_BITS = 0, 1
 
@@ -31,7 +31,7 @@ EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "
            "ss_last_chunk_kernel", "ss_trace_enable", "ss_trace_read", "ss_verify_round_static", "ss_verify_chunk_hinted", "ss_verify_export_state",
            "ss_verify_import_state", "ss_stream_layers", "ss_tier_create", "ss_tier_destroy",
            "ss_tier_reset", "ss_tier_get", "ss_tier_tail", "ss_tier_commit", "ss_tier_migrate", "ss_tier_poll",
-           "ss_tier_d2h_bytes"]
+           "ss_tier_d2h_bytes", "ss_verify_chunk_paged"]
 
 
 class ss_config(C.Structure):
@@ -119,6 +119,8 @@ def load() -> C.CDLL:
     lib.ss_verify_chunk.argtypes = [vp, ss_tensor, ss_tensor, i32, vp, vp]
     lib.ss_verify_chunk_hinted.restype = C.c_int
     lib.ss_verify_chunk_hinted.argtypes = [vp, ss_tensor, ss_tensor, i32, vp, C.POINTER(C.c_int32), vp]
+    lib.ss_verify_chunk_paged.restype = C.c_int
+    lib.ss_verify_chunk_paged.argtypes = [vp, ss_tensor, ss_tensor, i32, i32, vp, i32, vp, C.POINTER(C.c_int32), vp]
     lib.ss_verify_local.restype = C.c_int
     lib.ss_verify_local.argtypes = [vp, ss_tensor, ss_tensor, i32, C.c_int, vp, vp]
     lib.ss_verify_export_state.restype = C.c_int
@@ -256,6 +258,18 @@ class Context:
         self._check(self.lib.ss_verify_chunk_hinted(self.handle, as_ss_tensor(K), as_ss_tensor(V), L_c,
                                                     _ptr(valid_len), valid_len_host, _stream_ptr(stream)),
                     "ss_verify_chunk_hinted")
+
+    def ss_verify_chunk_paged(self, K_pool: torch.Tensor, V_pool: torch.Tensor, page_table: torch.Tensor,
+                              valid_len: Optional[torch.Tensor] = None, valid_len_host=None, stream=None):
+        """K_pool, V_pool [n_pages, H_kv, page_size, d]; page_table int32 [B, pages_per_req] on the device."""
+        n_pages, _, page_size, _ = K_pool.shape
+        assert page_table.dtype == torch.int32 and page_table.is_cuda and page_table.is_contiguous()
+        if valid_len_host is not None and not isinstance(valid_len_host, C.Array):
+            valid_len_host = (C.c_int32 * len(valid_len_host))(*valid_len_host)
+        self._check(self.lib.ss_verify_chunk_paged(self.handle, as_ss_tensor(K_pool), as_ss_tensor(V_pool),
+                                                   n_pages, page_size, page_table.data_ptr(),
+                                                   page_table.shape[1], _ptr(valid_len), valid_len_host,
+                                                   _stream_ptr(stream)), "ss_verify_chunk_paged")
 
     def ss_verify_local(self, K_loc: torch.Tensor, V_loc: torch.Tensor, mask_kind: int = SS_MASK_CHAIN,
                         mask_bits: Optional[torch.Tensor] = None, stream=None):

@@ -321,8 +321,12 @@ ss_status ss_verify_begin(ss_ctx* c, ss_tensor Q, int32_t B, int32_t T_q, float 
   return SS_OK;
 }
 
+struct PagedArgs {
+  int32_t n_pages, page_size, pages_per_req;
+  const int32_t* page_table;
+};
 static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, const int32_t* valid_len,
-                            const int32_t* valid_len_host, void* stream);
+                            const int32_t* valid_len_host, void* stream, const PagedArgs* pg = nullptr);
 
 ss_status ss_verify_chunk(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c,
                           const int32_t* valid_len, void* stream) {
@@ -335,8 +339,18 @@ ss_status ss_verify_chunk_hinted(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_
   return chunk_impl(c, K, V, L_c, valid_len, valid_len_host, stream);
 }
 
+ss_status ss_verify_chunk_paged(ss_ctx* c, ss_tensor K_pool, ss_tensor V_pool, int32_t n_pages,
+                                int32_t page_size, const int32_t* page_table, int32_t pages_per_req,
+                                const int32_t* valid_len, const int32_t* valid_len_host, void* stream) {
+  if (!page_table || n_pages <= 0 || page_size <= 0 || pages_per_req <= 0) return SS_ERR_ARG;
+  if ((uintptr_t)page_table & 3) return SS_ERR_ALIGN;
+  if ((int64_t)page_size * pages_per_req > 0x7fffffff) return SS_ERR_SHAPE;
+  const PagedArgs pg = {n_pages, page_size, pages_per_req, page_table};
+  return chunk_impl(c, K_pool, V_pool, page_size * pages_per_req, valid_len, valid_len_host, stream, &pg);
+}
+
 static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, const int32_t* valid_len,
-                            const int32_t* valid_len_host, void* stream) {
+                            const int32_t* valid_len_host, void* stream, const PagedArgs* pg) {
   if (!c || !K.ptr || !V.ptr) return SS_ERR_ARG;
   if (L_c <= 0) return SS_ERR_ARG;
   if (L_c > c->cfg.max_Lc) return SS_ERR_SHAPE;
@@ -368,12 +382,19 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   }
   CUtensorMap tmK, tmV;
   bool tc = c->tc_ok;
+  // paged chunks: a tile must not straddle pages
+  if (pg && (pg->page_size % kTileKeys)) tc = false;
   // up to 32 rows per kv-head the keys ride the MMA's M axis (tiles of 128 tokens); with more
   // rows the kernel with the rows on M is faster (measured).  SS_FLAG_ROWS_ON_M /
   // SS_FLAG_KEYS_ON_M (or SS_CHUNK_KERNEL=rows|keys) force one of them.
-  const bool keys_on_m = tc && !c->force_rows_kernel && (R <= 32 || c->force_keys_kernel);
+  const bool keys_on_m = tc && !c->force_rows_kernel && (R <= 32 || c->force_keys_kernel) &&
+                         (!pg || pg->page_size % 128 == 0);
   const int box = keys_on_m ? 128 : kTileKeys;
-  if (tc) tc = get_tensor_map(c, K, c->B, L_c, box, &tmK) && get_tensor_map(c, V, c->B, L_c, box, &tmV);
+  // tensor map over [outer, H_kv, tokens, d]: (requests, chunk tokens) or (pages, page tokens)
+  const int tm_outer = pg ? pg->n_pages : c->B, tm_tokens = pg ? pg->page_size : L_c;
+  if (tc)
+    tc = get_tensor_map(c, K, tm_outer, tm_tokens, box, &tmK) &&
+         get_tensor_map(c, V, tm_outer, tm_tokens, box, &tmV);
 
   ss::ChunkParams p;
   memset(&p, 0, sizeof(p));
@@ -454,6 +475,12 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   p.status = c->status;
   p.wait_first = 0;
   p.trace = c->trace_on ? c->trace : nullptr;
+  if (pg) {
+    p.page_table = pg->page_table;
+    p.pages_per_req = pg->pages_per_req;
+    p.page_size = pg->page_size;
+    p.n_pages = pg->n_pages;
+  }
 
   const bool pdl = use_pdl(c);
   cudaError_t e = !tc ? ss::launch_chunk_simt(p, s, pdl)

@@ -85,8 +85,19 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const ChunkParams 
 #pragma unroll
   for (int r = 0; r < kRows; ++r) acc[r][0] = acc[r][1] = 0.f;
 
-  const __nv_bfloat16* Kb = p.K + b * p.k_sb + kvh * p.k_sh;
-  const __nv_bfloat16* Vb = p.V + b * p.v_sb + kvh * p.v_sh;
+  // row of token tok (contiguous chunk or page of a pool)
+  auto k_row = [&](int tok) {
+    int outer, inner;
+    locate_token(p, b, tok, &outer, &inner);
+    return outer == p.n_pages && p.page_table ? (const __nv_bfloat16*)nullptr
+                                              : p.K + outer * p.k_sb + kvh * p.k_sh + inner * p.k_st;
+  };
+  auto v_row = [&](int tok) {
+    int outer, inner;
+    locate_token(p, b, tok, &outer, &inner);
+    return outer == p.n_pages && p.page_table ? (const __nv_bfloat16*)nullptr
+                                              : p.V + outer * p.v_sb + kvh * p.v_sh + inner * p.v_st;
+  };
   const int cp = tid % CP, tg = tid / CP;
 
   for (int t0 = tok0; t0 < tok1; t0 += kKeys) {
@@ -96,7 +107,10 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const ChunkParams 
     for (int i = tid; i < kKeys * (D / 8); i += kThreads) {
       const int k = i / (D / 8), c8 = i % (D / 8);
       uint4 raw = make_uint4(0, 0, 0, 0);
-      if (k < nk) raw = *reinterpret_cast<const uint4*>(Kb + (int64_t)(t0 + k) * p.k_st + c8 * 8);
+      if (k < nk) {
+        const __nv_bfloat16* row = k_row(t0 + k);
+        if (row) raw = *reinterpret_cast<const uint4*>(row + c8 * 8);
+      }
       *reinterpret_cast<uint4*>(&k_s[k * KS + c8 * 8]) = raw;
     }
     __syncthreads();
@@ -168,8 +182,9 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const ChunkParams 
     }
     const int kend = min(nk, (tg + 1) * KPG);
     for (int k = tg * KPG; k < kend; ++k) {
-      const float2 v = __bfloat1622float2(
-          *reinterpret_cast<const __nv_bfloat162*>(Vb + (int64_t)(t0 + k) * p.v_st + 2 * cp));
+      const __nv_bfloat16* vrow = v_row(t0 + k);
+      const float2 v = vrow ? __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(vrow + 2 * cp))
+                            : make_float2(0.f, 0.f);
 #pragma unroll
       for (int r = 0; r < kRows; ++r) {
         const float pr = p_s[r * (kKeys + 1) + k];

@@ -202,15 +202,16 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   // ---- set-up: barriers, first loads, tensor memory ------------------------------------------
   auto issue_tile = [&](int it, uint64_t pol) {
     const int s = it % kStages;
-    const int tok = tok0 + it * kTileKeys;
+    int outer, tok;
+    locate_token(p, b, tok0 + it * kTileKeys, &outer, &tok);
     const uint32_t kdst = smem_u32(st_s + s * kStageBytes);
     const uint32_t vdst = kdst + kTileBytes;
     mbar_expect_tx(&ctl->kfull[s], kTileBytes);
-    tma_load_4d(kdst, &tmK, 0, tok, kvh, b, &ctl->kfull[s], pol);
-    tma_load_4d(kdst + kHalfTile, &tmK, 64, tok, kvh, b, &ctl->kfull[s], pol);
+    tma_load_4d(kdst, &tmK, 0, tok, kvh, outer, &ctl->kfull[s], pol);
+    tma_load_4d(kdst + kHalfTile, &tmK, 64, tok, kvh, outer, &ctl->kfull[s], pol);
     mbar_expect_tx(&ctl->vfull[s], kTileBytes);
-    tma_load_4d(vdst, &tmV, 0, tok, kvh, b, &ctl->vfull[s], pol);
-    tma_load_4d(vdst + kHalfTile, &tmV, 64, tok, kvh, b, &ctl->vfull[s], pol);
+    tma_load_4d(vdst, &tmV, 0, tok, kvh, outer, &ctl->vfull[s], pol);
+    tma_load_4d(vdst + kHalfTile, &tmV, 64, tok, kvh, outer, &ctl->vfull[s], pol);
   };
   const int n_pre = min(n_tiles, kStages);
   uint32_t qreg[64];  // softmax threads: this lane's Q row (bf16 pairs)
@@ -270,15 +271,16 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       for (int it = n_pre; it < n_tiles; ++it) {
         const int s = it % kStages;
         const uint32_t ph = (it / kStages) & 1;
-        const int tok = tok0 + it * kTileKeys;
+        int outer, tok;
+        locate_token(p, b, tok0 + it * kTileKeys, &outer, &tok);
         const uint32_t kdst = smem_u32(st_s + s * kStageBytes);
         const uint32_t vdst = kdst + kTileBytes;
         trace(tr, 0, it, 0);
         if (!mbar_wait(&ctl->kempty[s], ph ^ 1, ctl, p.status)) break;
         trace(tr, 0, it, 1);
         mbar_expect_tx(&ctl->kfull[s], kTileBytes);
-        tma_load_4d(kdst, &tmK, 0, tok, kvh, b, &ctl->kfull[s], pol);
-        tma_load_4d(kdst + kHalfTile, &tmK, 64, tok, kvh, b, &ctl->kfull[s], pol);
+        tma_load_4d(kdst, &tmK, 0, tok, kvh, outer, &ctl->kfull[s], pol);
+        tma_load_4d(kdst + kHalfTile, &tmK, 64, tok, kvh, outer, &ctl->kfull[s], pol);
         // the V slot frees after the K slot; its load is accounted with the K load: on a
         // failed wait the K copy above is still waited for below through `issued`
         if (!mbar_wait(&ctl->vempty[s], ph ^ 1, ctl, p.status)) {
@@ -288,8 +290,8 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         }
         trace(tr, 0, it, 2);
         mbar_expect_tx(&ctl->vfull[s], kTileBytes);
-        tma_load_4d(vdst, &tmV, 0, tok, kvh, b, &ctl->vfull[s], pol);
-        tma_load_4d(vdst + kHalfTile, &tmV, 64, tok, kvh, b, &ctl->vfull[s], pol);
+        tma_load_4d(vdst, &tmV, 0, tok, kvh, outer, &ctl->vfull[s], pol);
+        tma_load_4d(vdst + kHalfTile, &tmV, 64, tok, kvh, outer, &ctl->vfull[s], pol);
         issued = it + 1;
       }
       if (ctl->abort) {

@@ -145,15 +145,16 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
   // use j of the ring: K of tile t is j = 2t, V of tile t is j = 2t + 1; unit j % UNITS
   auto issue_use = [&](int j, uint64_t pol) {
     const int u = j % UNITS;
-    const int tok = tok0 + (j >> 1) * kKeys;
+    int outer, tok;
+    locate_token(p, b, tok0 + (j >> 1) * kKeys, &outer, &tok);
     const uint32_t dst = smem_u32(smem + u * kUnitBytes);
     mbar_expect_tx(&ctl->ufull[u], kUnitBytes);
     if (j & 1) {  // (no runtime-selected pointer: the tensor maps stay in the parameter space)
-      tma_load_4d(dst, &tmV, 0, tok, kvh, b, &ctl->ufull[u], pol);
-      tma_load_4d(dst + kHalf, &tmV, 64, tok, kvh, b, &ctl->ufull[u], pol);
+      tma_load_4d(dst, &tmV, 0, tok, kvh, outer, &ctl->ufull[u], pol);
+      tma_load_4d(dst + kHalf, &tmV, 64, tok, kvh, outer, &ctl->ufull[u], pol);
     } else {
-      tma_load_4d(dst, &tmK, 0, tok, kvh, b, &ctl->ufull[u], pol);
-      tma_load_4d(dst + kHalf, &tmK, 64, tok, kvh, b, &ctl->ufull[u], pol);
+      tma_load_4d(dst, &tmK, 0, tok, kvh, outer, &ctl->ufull[u], pol);
+      tma_load_4d(dst + kHalf, &tmK, 64, tok, kvh, outer, &ctl->ufull[u], pol);
     }
   };
   const int n_uses = 2 * n_tiles;

@@ -45,6 +45,10 @@ struct ChunkParams {
   uint32_t* status;
   int wait_first;       // 1: wait for the preceding kernel before reading inputs
   unsigned long long* trace;  // optional: per-tile clock stamps of CTA (0,0,0), see ss_trace_read
+  // paged chunk (null = contiguous): token tok of request b lives in page
+  // page_table[b][tok / page_size] of the pool, at token offset tok % page_size
+  const int32_t* page_table;
+  int pages_per_req, page_size, n_pages;
 };
 
 struct LocalParams {
@@ -132,6 +136,26 @@ __device__ __forceinline__ void pdl_launch_dependents() {
 }
 __device__ __forceinline__ void pdl_wait_prior() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+// Where token `tok` of request b lives: (index along the tensor's outermost axis, token within
+// it).  Contiguous chunks: (b, tok).  Paged chunks: (page id, offset); a page id outside the pool
+// raises SS_DEV_BAD_PAGE and maps to index n_pages, which loads read as zeros.
+__device__ __forceinline__ void locate_token(const ChunkParams& p, int b, int tok, int* outer,
+                                             int* inner) {
+  if (!p.page_table) {
+    *outer = b;
+    *inner = tok;
+    return;
+  }
+  const int pg = tok / p.page_size;
+  int id = (pg < p.pages_per_req) ? p.page_table[(int64_t)b * p.pages_per_req + pg] : -1;
+  if (id < 0 || id >= p.n_pages) {
+    atomicOr(p.status, SS_DEV_BAD_PAGE);
+    id = p.n_pages;
+  }
+  *outer = id;
+  *inner = tok - pg * p.page_size;
 }
 
 }  // namespace ss

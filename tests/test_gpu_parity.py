@@ -255,3 +255,61 @@ def test_random_ragged_shapes(seed):
     order = list(range(n))
     rng.shuffle(order)
     _run(cfg, lens=lens, flags=flags, order=order, local_at=rng.randint(0, n), max_chunks=rng.choice([0, 2]))
+
+
+@pytest.mark.parametrize("page_size,flags", [(128, 0), (128, 4), (64, 0), (64, 8), (16, 0), (128, 1), (256, 0)])
+def test_paged_chunks_match_contiguous_and_oracle(page_size, flags):
+    # the chunk's tokens live in shuffled pages of a pool; same result as the gathered chunk
+    ssb = _ssb()
+    cfg = inputs.VerifyConfig("pg", 0x5D + page_size, 3, 8, 2, 128, 512, 6, 40, 1500, k_mult=2.0)
+    lens = [1500, 40, 1024]
+    case = util.gen_case(cfg, lens, DEV, fill=float("nan"))
+    Q, chunks, K_loc, V_loc, bits = case
+    ref = util.oracle_case(cfg, lens, *case)
+    ppr = cfg.L_c // page_size
+    g = torch.Generator().manual_seed(page_size)
+    ctx = util.make_ctx(cfg, flags=flags)
+    O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
+    LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
+    ctx.ss_verify_begin(Q, cfg.scale)
+    for K, V, vl in chunks:
+        n_pages = cfg.B * ppr + 3                      # a few unused pages
+        perm = torch.randperm(n_pages, generator=g)[:cfg.B * ppr].to(torch.int32)
+        table = perm.view(cfg.B, ppr).contiguous()
+        K_pool = torch.full((n_pages, cfg.H_kv, page_size, cfg.d), float("nan"), dtype=torch.bfloat16, device=DEV)
+        V_pool = torch.full_like(K_pool, float("nan"))
+        Kp = K.view(cfg.B, cfg.H_kv, ppr, page_size, cfg.d).permute(0, 2, 1, 3, 4).reshape(-1, cfg.H_kv, page_size, cfg.d)
+        Vp = V.view(cfg.B, cfg.H_kv, ppr, page_size, cfg.d).permute(0, 2, 1, 3, 4).reshape(-1, cfg.H_kv, page_size, cfg.d)
+        K_pool[table.view(-1).long()] = Kp
+        V_pool[table.view(-1).long()] = Vp
+        ctx.ss_verify_chunk_paged(K_pool, V_pool, table.to(DEV), vl, vl.tolist())
+    ctx.ss_verify_local(K_loc, V_loc)
+    ctx.ss_verify_finalize(O, LSE)
+    torch.cuda.synchronize()
+    st, dev_bits = ctx.ss_poll_status()
+    assert st == 0, dev_bits
+    expect = "simt" if (flags & 1 or page_size % 64) else ("tcgen05-keys" if (page_size % 128 == 0 and not flags & 4) else "tcgen05")
+    assert ctx.last_chunk_kernel() == expect, (ctx.last_chunk_kernel(), expect)
+    util.compare(cfg, O, LSE, ref)
+    ctx.close()
+
+
+def test_paged_chunk_bad_page_id_is_flagged():
+    ssb = _ssb()
+    cfg = inputs.VerifyConfig("pg", 0x5E, 2, 8, 2, 128, 256, 4, 256, 256)
+    lens = [256, 256]
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    K, V, vl = chunks[0]
+    table = torch.tensor([[0, 7], [1, -2]], dtype=torch.int32, device=DEV)      # pool has 2 pages
+    K_pool = K.view(2, 2, 2, 128, 128)[:, :, 0].contiguous()
+    V_pool = V.view(2, 2, 2, 128, 128)[:, :, 0].contiguous()
+    for flags in (0, 1):
+        ctx = util.make_ctx(cfg, flags=flags)
+        O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
+        ctx.ss_verify_begin(Q, cfg.scale)
+        ctx.ss_verify_chunk_paged(K_pool, V_pool, table, None)
+        ctx.ss_verify_finalize(O, None)
+        st, dev_bits = ctx.ss_poll_status()
+        assert st == ssb.SS_ERR_DEVICE_FLAG and dev_bits & ssb.SS_DEV_BAD_PAGE
+        assert torch.isfinite(O.float()).all()
+        ctx.close()
