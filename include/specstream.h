@@ -287,6 +287,46 @@ ss_status ss_tier_migrate(ss_tier* tier, void* stream, int32_t* n_requests);
 ss_status ss_tier_poll(ss_tier* tier, int32_t wait, void* stream, int32_t* advanced);
 int64_t ss_tier_d2h_bytes(ss_tier* tier);
 
+/* I/O-aware dynamic verification width (Section 4.2): q* = argmin_q T_round(q) / U(q) over the
+ * candidate widths, from running means of the rounds observed at each width.  Host logic only.
+ * T_round = t_draft + max(t_transfer, t_compute) + t_other (overlapped transfer and compute are
+ * counted once); means are exponential moving averages with weight `ema` (the first observation
+ * is taken as is); every width is tried `sample_rounds` times, in list order, before any estimate
+ * is trusted; afterwards the width changes only if the best width's cost per committed token is
+ * below the current one's by more than `switch_threshold` (relative).  Times are floats in any
+ * one unit; `committed` is the number of tokens the round committed. */
+typedef struct ss_width ss_width;
+typedef struct {
+  int32_t n_widths;       /* 1..8                                                         */
+  int32_t widths[8];      /* candidate set, e.g. {2, 4, 6, 8}                             */
+  int32_t sample_rounds;  /* >= 1                                                         */
+  float switch_threshold; /* >= 0, e.g. 0.05                                              */
+  float ema;              /* in (0, 1]                                                    */
+} ss_width_config;
+typedef struct {
+  float t_draft, t_transfer, t_compute, t_other;
+  int32_t committed;
+} ss_width_obs;
+ss_status ss_width_create(ss_width** out, const ss_width_config* cfg);
+ss_status ss_width_destroy(ss_width* w);
+ss_status ss_width_observe(ss_width* w, int32_t q, const ss_width_obs* obs); /* end of a round at width q */
+int32_t ss_width_next(ss_width* w);                                          /* width of the next round  */
+ss_status ss_width_estimate(ss_width* w, int32_t q, double* t_round, double* committed, double* cost,
+                            int32_t* n_obs);
+
+/* Cohort builder (Section 4.2, cohort batching).  Tasks that one batched kernel can process
+ * (same layer, width, dtype, n_kv, d_h, chunk_size) are grouped; inside a cohort requests are
+ * ordered by decreasing history length (stable), cohorts keep the order of their first task and
+ * are cut into pieces of at most max_batch.  order [n] receives the task indices cohort by
+ * cohort, cohort_start [n + 1] the start of each cohort in `order` (and the total at the end).
+ * Returns the number of cohorts, -1 on invalid arguments.  HOST pointers. */
+typedef struct {
+  int32_t layer, width, dtype, n_kv, d_h, chunk_size;
+  int32_t request_id, hist_len;
+} ss_task;
+int32_t ss_cohort_build(const ss_task* tasks, int32_t n, int32_t max_batch, int32_t* order,
+                        int32_t* cohort_start);
+
 typedef enum { SS_LAYERS_PREFETCH = 0, SS_LAYERS_STREAM = 1, SS_LAYERS_RESTORE = 2 } ss_layers_mode;
 typedef struct {
   int32_t n_layers;            /* <= 256                                                   */

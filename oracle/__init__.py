@@ -9,4 +9,5 @@ path.
 from .attention import verify_attention, verify_attention_rows  # noqa: F401
 from .streaming import (chunk_partial, merge, streamed_verify_attention,  # noqa: F401
                         IDENTITY)
-from .commit import commit_gather, migration_endpoint  # noqa: F401
+from .commit import cohort_build, commit_gather, migration_endpoint  # noqa: F401
+from .width import WidthController  # noqa: F401

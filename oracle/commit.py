@@ -40,3 +40,19 @@ def commit_gather(k_loc, v_loc, accept_idx, accept_cnt, k_dst, v_dst, dst_off):
 def migration_endpoint(H, C_r, T, g):
     """Eq. 9: end of the next batched offload interval [H, E)."""
     return max(H, g * (max(0, C_r - T) // g))
+
+
+def cohort_build(tasks, max_batch):
+    """Cohort batching (Section 4.2): group tasks with equal (layer, width, dtype, n_kv, d_h,
+    chunk_size); inside a group order by decreasing history length (stable); groups keep the
+    order of their first task; groups larger than max_batch are cut into consecutive pieces.
+    tasks: list of dicts.  Returns a list of cohorts, each a list of task indices."""
+    key = lambda t: (t["layer"], t["width"], t["dtype"], t["n_kv"], t["d_h"], t["chunk_size"])
+    groups = {}
+    for i, t in enumerate(tasks):
+        groups.setdefault(key(t), []).append(i)
+    out = []
+    for idx in groups.values():                       # dicts keep insertion order
+        idx = sorted(idx, key=lambda i: -tasks[i]["hist_len"])   # sorted() is stable
+        out += [idx[k:k + max_batch] for k in range(0, len(idx), max_batch)]
+    return out

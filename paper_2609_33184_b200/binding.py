@@ -31,7 +31,8 @@ EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "
            "ss_last_chunk_kernel", "ss_trace_enable", "ss_trace_read", "ss_verify_round_static", "ss_verify_chunk_hinted", "ss_verify_export_state",
            "ss_verify_import_state", "ss_stream_layers", "ss_tier_create", "ss_tier_destroy",
            "ss_tier_reset", "ss_tier_get", "ss_tier_tail", "ss_tier_commit", "ss_tier_migrate", "ss_tier_poll",
-           "ss_tier_d2h_bytes", "ss_verify_chunk_paged"]
+           "ss_tier_d2h_bytes", "ss_verify_chunk_paged", "ss_width_create", "ss_width_destroy",
+           "ss_width_observe", "ss_width_next", "ss_width_estimate", "ss_cohort_build"]
 
 
 class ss_config(C.Structure):
@@ -67,6 +68,21 @@ class ss_stream_desc(C.Structure):
 class ss_tier_config(C.Structure):
     _fields_ = [("B", C.c_int32), ("H_kv", C.c_int32), ("d", C.c_int32), ("L_c", C.c_int32),
                 ("tail_target", C.c_int32), ("granularity", C.c_int32), ("tail_capacity", C.c_int32)]
+
+
+class ss_task(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("layer", "width", "dtype", "n_kv", "d_h", "chunk_size",
+                                         "request_id", "hist_len")]
+
+
+class ss_width_config(C.Structure):
+    _fields_ = [("n_widths", C.c_int32), ("widths", C.c_int32 * 8), ("sample_rounds", C.c_int32),
+                ("switch_threshold", C.c_float), ("ema", C.c_float)]
+
+
+class ss_width_obs(C.Structure):
+    _fields_ = [("t_draft", C.c_float), ("t_transfer", C.c_float), ("t_compute", C.c_float),
+                ("t_other", C.c_float), ("committed", C.c_int32)]
 
 
 class ss_layers_desc(C.Structure):
@@ -158,6 +174,19 @@ def load() -> C.CDLL:
     lib.ss_tier_poll.argtypes = [vp, i32, vp, i32p]
     lib.ss_tier_d2h_bytes.restype = C.c_int64
     lib.ss_tier_d2h_bytes.argtypes = [vp]
+    lib.ss_width_create.restype = C.c_int
+    lib.ss_width_create.argtypes = [C.POINTER(vp), C.POINTER(ss_width_config)]
+    lib.ss_width_destroy.restype = C.c_int
+    lib.ss_width_destroy.argtypes = [vp]
+    lib.ss_width_observe.restype = C.c_int
+    lib.ss_width_observe.argtypes = [vp, i32, C.POINTER(ss_width_obs)]
+    lib.ss_width_next.restype = i32
+    lib.ss_width_next.argtypes = [vp]
+    lib.ss_width_estimate.restype = C.c_int
+    lib.ss_width_estimate.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                      C.POINTER(C.c_double), C.POINTER(C.c_int32)]
+    lib.ss_cohort_build.restype = i32
+    lib.ss_cohort_build.argtypes = [C.POINTER(ss_task), i32, i32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     lib.ss_strerror.restype = C.c_char_p
     lib.ss_strerror.argtypes = [C.c_int]
     lib.ss_sizeof_stream_desc.restype = C.c_size_t
