@@ -22,6 +22,8 @@
  *  - Asynchrony: every call validates its arguments on the host, enqueues work on the
  *    given CUDA stream and returns; results are valid once the stream reaches that
  *    point.  All calls of one round must use the same stream.
+ *    Nothing synchronises or allocates, so a whole round can be recorded into a CUDA graph
+ *    by stream capture and replayed (the call-order state machine runs at capture time).
  *  - Call order per round: begin -> {chunk | local}* -> finalize.  Chunks may come in
  *    any order and any number (including zero); local at most once.  Anything else
  *    returns SS_ERR_STATE.

@@ -313,3 +313,34 @@ def test_paged_chunk_bad_page_id_is_flagged():
         assert st == ssb.SS_ERR_DEVICE_FLAG and dev_bits & ssb.SS_DEV_BAD_PAGE
         assert torch.isfinite(O.float()).all()
         ctx.close()
+
+
+def test_round_can_be_captured_in_a_cuda_graph():
+    # the calls only enqueue on the stream: a captured round replays bit-identically
+    ssb = _ssb()
+    cfg = inputs.VerifyConfig("v", 0x5F, 2, 8, 2, 128, 256, 8, 300, 700)
+    lens = inputs.history_lengths(cfg)
+    case = util.gen_case(cfg, lens, DEV)
+    ctx = util.make_ctx(cfg, flags=ssb.SS_FLAG_OVERLAP_CHUNKS)
+    O_ref, L_ref = util.gpu_case(ctx, cfg, *case)
+    O_ref, L_ref = O_ref.clone(), L_ref.clone()
+    Q, chunks, K_loc, V_loc, bits = case
+    O = torch.zeros_like(O_ref)
+    LSE = torch.zeros_like(L_ref)
+
+    def one_round():
+        ctx.ss_verify_begin(Q, cfg.scale)
+        for K, V, vl in chunks:
+            ctx.ss_verify_chunk(K, V, vl)
+        ctx.ss_verify_local(K_loc, V_loc)
+        ctx.ss_verify_finalize(O, LSE)
+
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        one_round()
+    for _ in range(3):
+        O.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(O.view(torch.int16), O_ref.view(torch.int16)) and torch.equal(LSE, L_ref)
+    ctx.close()
