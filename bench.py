@@ -272,6 +272,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="plain launches (no programmatic dependent launch)")
     ap.add_argument("--simt", action="store_true", help="force the CUDA-core chunk kernel")
+    ap.add_argument("--flags", type=int, default=0, help="extra SS_FLAG_* bits for the context (A/B runs)")
     ap.add_argument("--layers", type=int, default=0,
                     help="also time N streamed layers back to back in the three pipeline modes "
                          "(cross-layer prefetch / layer by layer / restore-then-verify)")
@@ -308,6 +309,7 @@ def main():
     flags = 0 if args.no_overlap else ssb.SS_FLAG_OVERLAP_CHUNKS
     if args.simt:
         flags |= ssb.SS_FLAG_FORCE_SIMT
+    flags |= args.flags
     ctx = ssb.Context(cfg.B, cfg.H_q, cfg.H_kv, cfg.d, cfg.T_q, cfg.T_q, cfg.L_c, max_chunks=len(chunks) or 1,
                       device=local_rank, flags=flags)
     O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=dev)

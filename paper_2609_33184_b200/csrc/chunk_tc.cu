@@ -1,23 +1,29 @@
-// Tensor-core chunk attention for sm_100a: TMA-staged K/V tiles, tcgen05 MMAs with the
-// score tile S, the probabilities P and the unnormalised output O held in tensor memory.
+// Tensor-core chunk attention for sm_100a: TMA-staged K/V tiles, tcgen05 MMAs with two score
+// tiles S (double-buffered), the probabilities P and the unnormalised output O held in tensor
+// memory.
 //
 // One CTA owns one (request, kv-head, token split, tile of <= 128 query rows).  All rows of
 // the kv-head (T_q candidate queries x G query heads) ride in the M dimension of the MMAs,
 // so every K/V byte is fetched from HBM once and serves the whole query group.
 //
-//   warp 4 (one lane)  TMA producer: K tile and V tile of 64 tokens per stage, 3 stages,
+//   warp 4 (one lane)  TMA producer: K tiles and V tiles of 64 tokens, two slots each,
 //                      128-byte swizzle, evict-first L2 policy (the history is streamed).
-//                      A K tile is released as soon as its score MMAs retire, a V tile
+//                      A K slot is released as soon as its score MMAs retire, a V slot
 //                      after its output MMAs.
-//   warp 5 (one lane)  MMA issuer:   S = Q K^T   (M=128, N=64,  K=d=128: 8 x k16, tmem x smem)
-//                                    O += P V    (M=128, N=128, K=64:    4 x k16, tmem x smem)
-//   warps 0-3          softmax: each thread owns one TMEM lane (= one MMA row): loads its
-//                      Q row into tensor memory once, then per tile reads its scores, keeps
-//                      (m, l) in registers and writes P as packed bf16 over the score columns.
+//   warp 5 (one lane)  MMA issuer:   S[t%2] = Q K_t^T  (M=128, N=64,  K=d=128: 8 x k16, smem x smem)
+//                                    O += P_t V_t      (M=128, N=128, K=64:    4 x k16, tmem x smem)
+//                      in the order QK(0) QK(1) | PV(0) QK(2) | PV(1) QK(3) | ...: the scores of
+//                      tile t+1 are ready before the softmax of tile t ends, so the softmax
+//                      warps never wait for the tensor pipe in steady state, and PV(t) runs
+//                      under the softmax of tile t+1.
+//   warps 0-3          softmax: each thread owns one TMEM lane (= one MMA row): per tile it
+//                      reads its scores, keeps (m, l) in registers and writes P as packed
+//                      bf16 over the leading columns of the same score buffer.
 //
-// Tensor memory (256 columns): [0,64) S (fp32) with P (bf16 pairs) over [0,32); [64,128) Q
-// (bf16 pairs); [128,256) O (fp32).  Shared memory holds nothing but K/V tiles, so three
-// stages (96 KB) fit twice per SM and about 128 KB per SM are in flight from HBM.
+// Tensor memory (256 columns): [0,64) S0, [64,128) S1 (fp32; P of a tile as bf16 pairs over
+// the first 32 columns of its buffer); [128,256) O (fp32).  Shared memory: the Q tile
+// (32 KB, written once by the softmax threads in the swizzled K-major layout) and two slots
+// of K and V (64 KB); two CTAs fit per SM.
 //
 // When the row tile has <= 32 (<= 64) rows the Q rows are replicated 4x (2x) along M and
 // each replica takes a quarter (half) of the tile's keys: lane L holds row L % R_pad and
@@ -26,8 +32,8 @@
 //
 // Running maximum: a row's reference maximum m only moves when the tile maximum exceeds it
 // by more than 8 (base-2 domain), which keeps exp2(s - m) <= 256 and makes the rescale of O
-// in tensor memory rare.  Two CTAs fit per SM, so one CTA's ramp-up and tail overlap the
-// other's steady state.
+// in tensor memory rare.  Because PV(t-1) may still be accumulating into O while the softmax
+// of tile t runs, a rescale first waits for the commit of PV(t-1).
 //
 // Every wait on an mbarrier is bounded; on expiry the CTA raises SS_DEV_WAIT_EXPIRED, lets
 // its own copies land (bounded), frees its tensor memory and returns.
@@ -38,21 +44,24 @@ namespace ss {
 namespace {
 
 constexpr int kThreads = 192;
-constexpr int kStages = 3;
+constexpr int kStages = 2;
 constexpr int kD = 128;
 constexpr int kHalfTile = kTileKeys * 64 * 2;       // 8 KB: [64 keys][64 d] bf16
 constexpr int kTileBytes = 2 * kHalfTile;           // 16 KB: one K tile or one V tile
 constexpr int kStageBytes = 2 * kTileBytes;         // K then V
-constexpr int kSmemData = kStages * kStageBytes;            // 96 KB
+constexpr int kQHalf = 128 * 64 * 2;                // 16 KB: [128 rows][64 d] bf16
+constexpr int kQBytes = 2 * kQHalf;                 // 32 KB: the Q tile
+constexpr int kSmemData = kQBytes + kStages * kStageBytes;  // 96 KB
 constexpr int kSmemCtl = 2048;
 constexpr int kSmemTotal = kSmemData + kSmemCtl + 1024;     // + alignment slack
 constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColS = 0, kColP = 0, kColQ = 64, kColO = 128;
+constexpr uint32_t kColS = 0, kColO = 128;          // S buffer t%2 at kColS + 64 (t%2)
 constexpr float kRescaleThreshold = 8.f;
 
 struct Ctl {
   uint64_t kfull[kStages], vfull[kStages], kempty[kStages], vempty[kStages];
-  uint64_t sfull, pready, pvdone;
+  uint64_t sfull[2], pready[2];  // per score buffer
+  uint64_t odone;                // one phase per tile: PV(t) has retired
   uint32_t tmem_base;
   volatile uint32_t abort;
   float2 ml[128];
@@ -90,9 +99,12 @@ __device__ __forceinline__ void store_p(uint32_t t_s, const uint32_t (&pk)[NC / 
 // MASK = the tile straddles the valid length (columns >= n_valid are invisible).  The scale is
 // positive (checked at ss_verify_begin), so the maximum is taken on the raw scores and the
 // scaling rides in the FMA that subtracts the reference.
+// Returns false when the wait for PV(it - 1) in the rescale path gave up.
 template <int NC, bool MASK>
-__device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_o, int c0, int n_valid,
-                                             bool have_o, float scale_log2, float& m, float& l) {
+__device__ __forceinline__ bool softmax_tile(uint32_t t_s, uint32_t t_o, int c0, int n_valid,
+                                             int it, float scale_log2, float& m, float& l,
+                                             Ctl* ctl, uint32_t* status) {
+  const bool have_o = it > 0;
   uint32_t raw[NC / 16][16];
 #pragma unroll
   for (int q = 0; q < NC / 16; ++q) tmem_ld16(t_s + c0 + q * 16, raw[q]);
@@ -114,7 +126,10 @@ __device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_o, int c0,
   }
   const bool need = have_o && (f != 1.f);
   if (__any_sync(0xffffffffu, need)) {
-    // rare: move this lane's O row to the new reference maximum
+    // rare: move this lane's O row to the new reference maximum, once PV(it - 1) has retired
+    // (its phase is the latest the barrier can have completed: PV(it) needs this tile's P)
+    if (!mbar_wait(&ctl->odone, (it - 1) & 1, ctl, status)) return false;
+    tc_fence_after();
 #pragma unroll 1
     for (int q = 0; q < kD / 16; ++q) {
       uint32_t o[16];
@@ -152,6 +167,7 @@ __device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_o, int c0,
     }
   }
   tc_wait_st();
+  return true;
 }
 
 __global__ void __launch_bounds__(kThreads, 2)
@@ -159,7 +175,8 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* st_s = smem;
+  uint8_t* q_s = smem;             // Q tile: two halves [128 rows][64 d], 128-byte swizzle
+  uint8_t* st_s = smem + kQBytes;  // K/V slots
   Ctl* ctl = reinterpret_cast<Ctl*>(smem + kSmemData);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -199,22 +216,26 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     return;
   }
 
-  // ---- set-up: barriers, first loads, tensor memory ------------------------------------------
-  auto issue_tile = [&](int it, uint64_t pol) {
+  // ---- set-up: barriers, first loads, tensor memory, the Q tile --------------------------------
+  auto issue_k = [&](int it, uint64_t pol) {
     const int s = it % kStages;
     int outer, tok;
     locate_token(p, b, tok0 + it * kTileKeys, &outer, &tok);
     const uint32_t kdst = smem_u32(st_s + s * kStageBytes);
-    const uint32_t vdst = kdst + kTileBytes;
     mbar_expect_tx(&ctl->kfull[s], kTileBytes);
     tma_load_4d(kdst, &tmK, 0, tok, kvh, outer, &ctl->kfull[s], pol);
     tma_load_4d(kdst + kHalfTile, &tmK, 64, tok, kvh, outer, &ctl->kfull[s], pol);
+  };
+  auto issue_v = [&](int it, uint64_t pol) {
+    const int s = it % kStages;
+    int outer, tok;
+    locate_token(p, b, tok0 + it * kTileKeys, &outer, &tok);
+    const uint32_t vdst = smem_u32(st_s + s * kStageBytes) + kTileBytes;
     mbar_expect_tx(&ctl->vfull[s], kTileBytes);
     tma_load_4d(vdst, &tmV, 0, tok, kvh, outer, &ctl->vfull[s], pol);
     tma_load_4d(vdst + kHalfTile, &tmV, 64, tok, kvh, outer, &ctl->vfull[s], pol);
   };
   const int n_pre = min(n_tiles, kStages);
-  uint32_t qreg[64];  // softmax threads: this lane's Q row (bf16 pairs)
   if (warp == 4) {
     if (lane == 0) {
       for (int s = 0; s < kStages; ++s) {
@@ -223,15 +244,19 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         mbar_init(&ctl->kempty[s], 1);
         mbar_init(&ctl->vempty[s], 1);
       }
-      mbar_init(&ctl->sfull, 1);
-      mbar_init(&ctl->pready, 128);
-      mbar_init(&ctl->pvdone, 1);
+      for (int i = 0; i < 2; ++i) {
+        mbar_init(&ctl->sfull[i], 1);
+        mbar_init(&ctl->pready[i], 128);
+      }
+      mbar_init(&ctl->odone, 1);
       ctl->abort = 0;
       fence_barrier_init();
-      // the first tiles go out before the rest of the CTA is set up
+      // the first tiles go out before the rest of the CTA is set up (K first: the score
+      // MMAs of both tiles come before the first output MMAs)
       // streamed once: evict first; shared by the row groups of a kv-head through L2: keep
       const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
-      for (int it = 0; it < n_pre; ++it) issue_tile(it, pol);
+      for (int it = 0; it < n_pre; ++it) issue_k(it, pol);
+      for (int it = 0; it < n_pre; ++it) issue_v(it, pol);
     }
     __syncwarp();
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
@@ -240,6 +265,8 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   } else if (warp < 4) {
+    // this lane's Q row -> shared memory, K-major with the 128-byte swizzle the MMA descriptor
+    // expects: 16-byte chunk c of row L sits at chunk c ^ (L % 8) of the row's 128 bytes
     const int r = tid % r_pad;
     const uint4* src = nullptr;
     if (r < nrows) {
@@ -250,11 +277,9 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
 #pragma unroll
     for (int v = 0; v < 16; ++v) {
       const uint4 x = src ? src[v] : make_uint4(0, 0, 0, 0);
-      qreg[v * 4 + 0] = x.x;
-      qreg[v * 4 + 1] = x.y;
-      qreg[v * 4 + 2] = x.z;
-      qreg[v * 4 + 3] = x.w;
+      *reinterpret_cast<uint4*>(q_s + (v >> 3) * kQHalf + tid * 128 + (((v & 7) ^ (tid & 7)) << 4)) = x;
     }
+    fence_proxy_async();  // generic-proxy writes -> visible to the tensor core's reads
   }
   tc_fence_before();
   __syncthreads();
@@ -267,42 +292,36 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     if (lane == 0) {
       // streamed once: evict first; shared by the row groups of a kv-head through L2: keep
       const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
-      int issued = n_pre;
-      for (int it = n_pre; it < n_tiles; ++it) {
-        const int s = it % kStages;
-        const uint32_t ph = (it / kStages) & 1;
-        int outer, tok;
-        locate_token(p, b, tok0 + it * kTileKeys, &outer, &tok);
-        const uint32_t kdst = smem_u32(st_s + s * kStageBytes);
-        const uint32_t vdst = kdst + kTileBytes;
-        trace(tr, 0, it, 0);
-        if (!mbar_wait(&ctl->kempty[s], ph ^ 1, ctl, p.status)) break;
-        trace(tr, 0, it, 1);
-        mbar_expect_tx(&ctl->kfull[s], kTileBytes);
-        tma_load_4d(kdst, &tmK, 0, tok, kvh, outer, &ctl->kfull[s], pol);
-        tma_load_4d(kdst + kHalfTile, &tmK, 64, tok, kvh, outer, &ctl->kfull[s], pol);
-        // the V slot frees after the K slot; its load is accounted with the K load: on a
-        // failed wait the K copy above is still waited for below through `issued`
-        if (!mbar_wait(&ctl->vempty[s], ph ^ 1, ctl, p.status)) {
-          mbar_expect_tx(&ctl->vfull[s], 0);  // nothing will arrive for V
-          issued = it + 1;
-          break;
+      // K(j) can go out once QK(j - 2) has retired, V(i) once PV(i - 2) has: in time order
+      // that is K(j) next to V(j - 2)
+      int issued_k = n_pre, issued_v = n_pre;
+      for (int j = n_pre; j < n_tiles + 2; ++j) {
+        if (j < n_tiles) {
+          trace(tr, 0, j, 0);
+          if (!mbar_wait(&ctl->kempty[j % kStages], ((j / kStages) & 1) ^ 1, ctl, p.status)) break;
+          trace(tr, 0, j, 1);
+          issue_k(j, pol);
+          issued_k = j + 1;
         }
-        trace(tr, 0, it, 2);
-        mbar_expect_tx(&ctl->vfull[s], kTileBytes);
-        tma_load_4d(vdst, &tmV, 0, tok, kvh, outer, &ctl->vfull[s], pol);
-        tma_load_4d(vdst + kHalfTile, &tmV, 64, tok, kvh, outer, &ctl->vfull[s], pol);
-        issued = it + 1;
+        const int i = j - 2;
+        if (i >= n_pre && i < n_tiles) {
+          if (!mbar_wait(&ctl->vempty[i % kStages], ((i / kStages) & 1) ^ 1, ctl, p.status)) break;
+          trace(tr, 0, i, 2);
+          issue_v(i, pol);
+          issued_v = i + 1;
+        }
       }
       if (ctl->abort) {
         // let the copies this thread started land before the CTA leaves (bounded)
         const unsigned long long t0 = gtime_ns();
-        for (int it = max(0, issued - kStages); it < issued; ++it) {
-          const int s = it % kStages;
-          const uint32_t ph = (it / kStages) & 1;
-          while (!mbar_try_wait(&ctl->kfull[s], ph) && gtime_ns() - t0 < kWaitNs) {
+        for (int it = max(0, issued_k - kStages); it < issued_k; ++it) {
+          while (!mbar_try_wait(&ctl->kfull[it % kStages], (it / kStages) & 1) &&
+                 gtime_ns() - t0 < kWaitNs) {
           }
-          while (!mbar_try_wait(&ctl->vfull[s], ph) && gtime_ns() - t0 < kWaitNs) {
+        }
+        for (int it = max(0, issued_v - kStages); it < issued_v; ++it) {
+          while (!mbar_try_wait(&ctl->vfull[it % kStages], (it / kStages) & 1) &&
+                 gtime_ns() - t0 < kWaitNs) {
           }
         }
       }
@@ -313,27 +332,37 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     constexpr uint32_t idesc_qk = make_idesc(128, kTileKeys, false);
     constexpr uint32_t idesc_pv = make_idesc(128, kD, true);
     const bool leader = elect_one();
-    const uint32_t st_addr = smem_u32(st_s);
-    // Q is in tensor memory once the softmax warps have arrived on pready (phase 0)
-    bool ok = mbar_wait(&ctl->pready, 0, ctl, p.status) && mbar_wait(&ctl->kfull[0], 0, ctl, p.status);
-    if (ok) {
-      tc_fence_after();
+    const uint32_t st_addr = smem_u32(st_s), q_addr = smem_u32(q_s);
+    // S[it % 2] = Q K_it^T; releases the K slot and signals the softmax warps
+    auto issue_qk = [&](int it) {
+      const int s = it % kStages;
+      const uint32_t k_addr = st_addr + s * kStageBytes;
       if (leader) {
 #pragma unroll
         for (int kk = 0; kk < kD / 16; ++kk) {
+          const uint32_t qoff = (kk >> 2) * kQHalf + (kk & 3) * 32;
           const uint32_t koff = (kk >> 2) * kHalfTile + (kk & 3) * 32;
-          mma_ts(tmem + kColS, tmem + kColQ + kk * 8, desc_kmajor(st_addr + koff), idesc_qk, kk > 0);
+          mma_ss(tmem + kColS + (it & 1) * 64, desc_kmajor(q_addr + qoff), desc_kmajor(k_addr + koff),
+                 idesc_qk, kk > 0);
         }
-        tc_commit(&ctl->kempty[0]);
-        tc_commit(&ctl->sfull);
+        tc_commit(&ctl->kempty[s]);
+        tc_commit(&ctl->sfull[it & 1]);
       }
       __syncwarp();
+    };
+    // the Q tile was written before the CTA-wide barrier above (with a proxy fence)
+    bool ok = true;
+    for (int it = 0; ok && it < n_pre; ++it) {
+      ok = mbar_wait(&ctl->kfull[it], 0, ctl, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      issue_qk(it);
     }
     for (int it = 0; ok && it < n_tiles; ++it) {
       const int s = it % kStages;
       const uint32_t ph = (it / kStages) & 1;
       trace(trl, 1, it, 0);
-      ok = mbar_wait(&ctl->pready, (it + 1) & 1, ctl, p.status);
+      ok = mbar_wait(&ctl->pready[it & 1], (it >> 1) & 1, ctl, p.status);
       trace(trl, 1, it, 1);
       ok = ok && mbar_wait(&ctl->vfull[s], ph, ctl, p.status);
       if (!ok) break;
@@ -343,38 +372,23 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       if (leader) {
 #pragma unroll
         for (int kk = 0; kk < kTileKeys / 16; ++kk) {
-          mma_ts(tmem + kColO, tmem + kColP + kk * 8, desc_mnmajor(v_addr + kk * 2048, kHalfTile),
-                 idesc_pv, (it > 0 || kk > 0));
+          mma_ts(tmem + kColO, tmem + kColS + (it & 1) * 64 + kk * 8,
+                 desc_mnmajor(v_addr + kk * 2048, kHalfTile), idesc_pv, (it > 0 || kk > 0));
         }
         tc_commit(&ctl->vempty[s]);
+        tc_commit(&ctl->odone);
       }
       __syncwarp();
       trace(trl, 1, it, 3);
-      if (it + 1 < n_tiles) {
-        const int s2 = (it + 1) % kStages;
-        const uint32_t ph2 = ((it + 1) / kStages) & 1;
-        ok = mbar_wait(&ctl->kfull[s2], ph2, ctl, p.status);
+      if (it + 2 < n_tiles) {
+        // overwrites the score buffer P(it) was read from: the tensor pipe runs this thread's
+        // MMAs in issue order, so the P V products above have consumed P before these write S
+        ok = mbar_wait(&ctl->kfull[s], ph ^ 1, ctl, p.status);
         if (!ok) break;
         trace(trl, 1, it, 4);
         tc_fence_after();
-        const uint32_t k_addr = st_addr + s2 * kStageBytes;
-        // overwrites the S/P columns: the tensor pipe runs this thread's MMAs in issue
-        // order, so the P V products above have consumed P before these write S
-        if (leader) {
-#pragma unroll
-          for (int kk = 0; kk < kD / 16; ++kk) {
-            const uint32_t koff = (kk >> 2) * kHalfTile + (kk & 3) * 32;
-            mma_ts(tmem + kColS, tmem + kColQ + kk * 8, desc_kmajor(k_addr + koff), idesc_qk,
-                   kk > 0);
-          }
-          tc_commit(&ctl->kempty[s2]);
-          tc_commit(&ctl->sfull);
-        }
-        __syncwarp();
+        issue_qk(it + 2);
         trace(trl, 1, it, 5);
-      } else {
-        if (leader) tc_commit(&ctl->pvdone);
-        __syncwarp();
       }
     }
   } else {
@@ -385,27 +399,15 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     const int nc = kTileKeys / groups;
     const int c0 = grp * nc;
     const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
-    const uint32_t t_s = tmem + lane_off + kColS;
     const uint32_t t_o = tmem + lane_off + kColO;
     float m = -INFINITY, l = 0.f;
-    {  // this lane's Q row -> tensor memory as bf16 pairs (zero for padding rows)
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint32_t w[16];
-#pragma unroll
-        for (int v = 0; v < 16; ++v) w[v] = qreg[q * 16 + v];
-        tmem_st16(tmem + lane_off + kColQ + q * 16, w);
-      }
-      tc_wait_st();
-      tc_fence_before();
-      mbar_arrive(&ctl->pready);  // phase 0: Q is in place
-    }
     bool ok = true;
     for (int it = 0; it < n_tiles; ++it) {
       const int s = it % kStages;
       const uint32_t ph = (it / kStages) & 1;
+      const uint32_t t_s = tmem + lane_off + kColS + (it & 1) * 64;
       if (L == 0) trace(tr, 2, it, 0);
-      ok = mbar_wait(&ctl->sfull, it & 1, ctl, p.status);
+      ok = mbar_wait(&ctl->sfull[it & 1], (it >> 1) & 1, ctl, p.status);
       if (!ok) break;
       tc_fence_after();
       if (L == 0) trace(tr, 2, it, 1);
@@ -424,31 +426,40 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         }
         fence_proxy_async();
       }
+#define SS_SOFTMAX_TILE(NC_, MASK_) \
+  softmax_tile<NC_, MASK_>(t_s, t_o, c0, n_valid, it, p.scale_log2, m, l, ctl, p.status)
       if (n_valid < kTileKeys) {
         if (nc == 16)
-          softmax_tile<16, true>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+          ok = SS_SOFTMAX_TILE(16, true);
         else if (nc == 32)
-          softmax_tile<32, true>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+          ok = SS_SOFTMAX_TILE(32, true);
         else
-          softmax_tile<64, true>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+          ok = SS_SOFTMAX_TILE(64, true);
       } else {
         if (nc == 16)
-          softmax_tile<16, false>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+          ok = SS_SOFTMAX_TILE(16, false);
         else if (nc == 32)
-          softmax_tile<32, false>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+          ok = SS_SOFTMAX_TILE(32, false);
         else
-          softmax_tile<64, false>(t_s, t_o, c0, n_valid, it > 0, p.scale_log2, m, l);
+          ok = SS_SOFTMAX_TILE(64, false);
       }
+#undef SS_SOFTMAX_TILE
+      if (!ok) break;
       tc_fence_before();
-      mbar_arrive(&ctl->pready);
+      mbar_arrive(&ctl->pready[it & 1]);
       if (L == 0) trace(tr, 2, it, 2);
     }
-    ok = ok && mbar_wait(&ctl->pvdone, 0, ctl, p.status);
+    // all output MMAs have retired: odone completes one phase per tile and PV(n - 3) is known
+    // to have retired (the scores of the last tile came after it), so the phases of the last
+    // two tiles are waited for one after the other (a single parity could not tell PV(n - 1)
+    // from PV(n - 3))
+    if (n_tiles >= 2) ok = ok && mbar_wait(&ctl->odone, (n_tiles - 2) & 1, ctl, p.status);
+    ok = ok && mbar_wait(&ctl->odone, (n_tiles - 1) & 1, ctl, p.status);
     named_bar_sync(2, 128);
     if (ctl->abort == 0) {  // uniform over the 128 threads after the barrier
       tc_fence_after();
       // ---- merge the key groups of each row and write the partial state ----
-      float* o_s = reinterpret_cast<float*>(st_s);  // [128][128] fp32 over the free stage buffers
+      float* o_s = reinterpret_cast<float*>(smem);  // [128][128] fp32 over the Q tile and the slots
       ctl->ml[L] = make_float2(m, l);
       named_bar_sync(1, 128);
       float M = -INFINITY;
