@@ -57,11 +57,16 @@ constexpr int kSmemTotal = kSmemData + kSmemCtl + 1024;     // + alignment slack
 constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kColS = 0, kColO = 128;          // S buffer t%2 at kColS + 64 (t%2)
 constexpr float kRescaleThreshold = 8.f;
+#ifndef SS_POLY_EVERY
+#define SS_POLY_EVERY 0
+#endif
+constexpr int kPolyEvery = SS_POLY_EVERY;  // 0: every exponential on the special-function unit
 
 struct Ctl {
   uint64_t kfull[kStages], vfull[kStages], kempty[kStages], vempty[kStages];
   uint64_t sfull[2], pready[2];  // per score buffer
   uint64_t odone;                // one phase per tile: PV(t) has retired
+  uint64_t pvdone;               // the last PV has retired
   uint32_t tmem_base;
   volatile uint32_t abort;
   float2 ml[128];
@@ -110,13 +115,15 @@ __device__ __forceinline__ bool softmax_tile(uint32_t t_s, uint32_t t_o, int c0,
   for (int q = 0; q < NC / 16; ++q) tmem_ld16(t_s + c0 + q * 16, raw[q]);
   tc_wait_ld();
   float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // independent chains
+  if (MASK) {
 #pragma unroll
-  for (int c = 0; c < NC; ++c) {
-    float v = __uint_as_float(raw[c / 16][c % 16]);
-    if (MASK && c0 + c >= n_valid) v = -INFINITY;
-    if (MASK) raw[c / 16][c % 16] = __float_as_uint(v);
-    mx4[c & 3] = fmaxf(mx4[c & 3], v);
+    for (int c = 0; c < NC; ++c)
+      if (c0 + c >= n_valid) raw[c / 16][c % 16] = __float_as_uint(-INFINITY);
   }
+#pragma unroll
+  for (int c = 0; c < NC; c += 2)
+    mx4[(c >> 1) & 3] = max3_f(mx4[(c >> 1) & 3], __uint_as_float(raw[c / 16][c % 16]),
+                               __uint_as_float(raw[(c + 1) / 16][(c + 1) % 16]));
   const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
   float f = 1.f;
   if (mx > m + kRescaleThreshold) {  // also the first finite maximum (m = -inf)
@@ -142,16 +149,24 @@ __device__ __forceinline__ bool softmax_tile(uint32_t t_s, uint32_t t_o, int c0,
   }
   const float neg_m = (m == -INFINITY) ? 0.f : -m;
   uint32_t pk[NC / 16][8];
-  float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+  // two keys per packed fp32 instruction: x = s * scale - m, then the row sum
+  float2 sum2[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+  const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(neg_m, neg_m);
 #pragma unroll
   for (int c = 0; c < NC; c += 2) {
-    const float p0 = ex2_ftz(fmaf(__uint_as_float(raw[c / 16][c % 16]), scale_log2, neg_m));
-    const float p1 = ex2_ftz(fmaf(__uint_as_float(raw[(c + 1) / 16][(c + 1) % 16]), scale_log2, neg_m));
-    sum4[(c >> 1) & 3] += p0 + p1;
-    __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);  // low half = even key
+    const float2 x = fma2_f(make_float2(__uint_as_float(raw[c / 16][c % 16]),
+                                        __uint_as_float(raw[(c + 1) / 16][(c + 1) % 16])),
+                            sc2, nm2);
+    // one pair in kPolyEvery takes the polynomial on the FMA pipe: the special-function unit,
+    // shared by the softmax warps of both resident CTAs, is the busiest unit of this kernel
+    const bool poly = !MASK && kPolyEvery > 0 && ((c >> 1) % (kPolyEvery > 0 ? kPolyEvery : 1)) == 0;
+    const float2 pp = poly ? ex2_poly2(x) : make_float2(ex2_ftz(x.x), ex2_ftz(x.y));
+    sum2[(c >> 1) & 3] = add2_f(sum2[(c >> 1) & 3], pp);
+    __nv_bfloat162 h = __floats2bfloat162_rn(pp.x, pp.y);  // low half = even key
     pk[c / 16][(c / 2) % 8] = *reinterpret_cast<uint32_t*>(&h);
   }
-  l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+  const float2 s01 = add2_f(sum2[0], sum2[1]), s23 = add2_f(sum2[2], sum2[3]);
+  l += (s01.x + s01.y) + (s23.x + s23.y);
   // c0 is uniform across a warp; dispatching on it keeps pk[] in registers
   if (NC == 64) {
     store_p<NC, 0>(t_s, pk);
@@ -249,6 +264,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         mbar_init(&ctl->pready[i], 128);
       }
       mbar_init(&ctl->odone, 1);
+      mbar_init(&ctl->pvdone, 1);
       ctl->abort = 0;
       fence_barrier_init();
       // the first tiles go out before the rest of the CTA is set up (K first: the score
@@ -377,6 +393,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         }
         tc_commit(&ctl->vempty[s]);
         tc_commit(&ctl->odone);
+        if (it + 1 == n_tiles) tc_commit(&ctl->pvdone);
       }
       __syncwarp();
       trace(trl, 1, it, 3);
@@ -449,12 +466,9 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       mbar_arrive(&ctl->pready[it & 1]);
       if (L == 0) trace(tr, 2, it, 2);
     }
-    // all output MMAs have retired: odone completes one phase per tile and PV(n - 3) is known
-    // to have retired (the scores of the last tile came after it), so the phases of the last
-    // two tiles are waited for one after the other (a single parity could not tell PV(n - 1)
-    // from PV(n - 3))
-    if (n_tiles >= 2) ok = ok && mbar_wait(&ctl->odone, (n_tiles - 2) & 1, ctl, p.status);
-    ok = ok && mbar_wait(&ctl->odone, (n_tiles - 1) & 1, ctl, p.status);
+    // all output MMAs have retired (a barrier of its own: by now odone may be one or two
+    // phases past the last one this thread looked at, which a parity cannot tell apart)
+    ok = ok && mbar_wait(&ctl->pvdone, 0, ctl, p.status);
     named_bar_sync(2, 128);
     if (ctl->abort == 0) {  // uniform over the 128 threads after the barrier
       tc_fence_after();
