@@ -35,6 +35,7 @@ from paper_2609_33184_b200 import inputs  # noqa: E402
 METRIC = "verify_attention_kv_GBps"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1400.0
 
 
 def peaks():
@@ -43,6 +44,15 @@ def peaks():
         with open(p) as f:
             return float(json.load(f)["hbm_gbs"]), "measured"
     return FALLBACK_HBM_GBS, "fallback"
+
+
+def tensor_peak():
+    """Dense bf16 TFLOP/s, the sustained figure (the chunk kernel is timed inside a long step)."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "measured (sustained)"
+    return FALLBACK_BF16_TFLOPS, "fallback (sustained)"
 
 
 # DRAM bytes (read + write) per chunk-kernel launch from an ncu capture of the same kernel;
@@ -383,6 +393,17 @@ def main():
                 "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(cfg.name),
                 "algorithmic_bytes_per_launch": alg_bytes_per_launch,
                 "us_per_launch": chunk_ms * 1e3 if chunk_ms else None}
+    # Useful flops of a launch: QK^T and PV, 2 * 2 * d per (query row, key).  When they take
+    # longer at the tensor peak than the bytes take at the HBM peak (many query rows per kv-head:
+    # the tree workload), the kernel's roofline is the tensor pipe and is reported against it.
+    alg_flops_per_launch = 4.0 * cfg.d * cfg.G * cfg.T_q * (alg_bytes_per_launch / (cfg.d * 2 * 2))
+    tpeak, tpeak_kind = tensor_peak()
+    if alg_flops_per_launch / (tpeak * 1e12) > alg_bytes_per_launch / (peak * 1e9):
+        tf = alg_flops_per_launch / (chunk_ms * 1e-3) / 1e12 if chunk_ms else None
+        roofline.update({"bound": "tensor", "achieved": tf, "peak": tpeak, "peak_kind": tpeak_kind,
+                         "unit": "TFLOP/s", "frac": (tf / tpeak) if tf else None,
+                         "algorithmic_flops_per_launch": alg_flops_per_launch,
+                         "kv_GBps": achieved})
 
     # ---- the same round replayed from a CUDA graph (launch-bound workloads gain; the calls
     # only enqueue on the stream, so a captured round can be replayed without the host API) -----

@@ -57,10 +57,6 @@ constexpr int kSmemTotal = kSmemData + kSmemCtl + 1024;     // + alignment slack
 constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kColS = 0, kColO = 128;          // S buffer t%2 at kColS + 64 (t%2)
 constexpr float kRescaleThreshold = 8.f;
-#ifndef SS_POLY_EVERY
-#define SS_POLY_EVERY 0
-#endif
-constexpr int kPolyEvery = SS_POLY_EVERY;  // 0: every exponential on the special-function unit
 
 struct Ctl {
   uint64_t kfull[kStages], vfull[kStages], kempty[kStages], vempty[kStages];
@@ -157,10 +153,7 @@ __device__ __forceinline__ bool softmax_tile(uint32_t t_s, uint32_t t_o, int c0,
     const float2 x = fma2_f(make_float2(__uint_as_float(raw[c / 16][c % 16]),
                                         __uint_as_float(raw[(c + 1) / 16][(c + 1) % 16])),
                             sc2, nm2);
-    // one pair in kPolyEvery takes the polynomial on the FMA pipe: the special-function unit,
-    // shared by the softmax warps of both resident CTAs, is the busiest unit of this kernel
-    const bool poly = !MASK && kPolyEvery > 0 && ((c >> 1) % (kPolyEvery > 0 ? kPolyEvery : 1)) == 0;
-    const float2 pp = poly ? ex2_poly2(x) : make_float2(ex2_ftz(x.x), ex2_ftz(x.y));
+    const float2 pp = make_float2(ex2_ftz(x.x), ex2_ftz(x.y));
     sum2[(c >> 1) & 3] = add2_f(sum2[(c >> 1) & 3], pp);
     __nv_bfloat162 h = __floats2bfloat162_rn(pp.x, pp.y);  // low half = even key
     pk[c / 16][(c / 2) % 8] = *reinterpret_cast<uint32_t*>(&h);

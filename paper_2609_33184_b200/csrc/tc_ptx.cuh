@@ -209,25 +209,6 @@ __device__ __forceinline__ float2 add2_f(float2 a, float2 b) {
       : "l"(reinterpret_cast<uint64_t&>(a)), "l"(reinterpret_cast<uint64_t&>(b)));
   return reinterpret_cast<float2&>(d);
 }
-// exp2 of two finite values on the FMA pipe (no special-function unit): split x into
-// round(x) + r with |r| <= 1/2 by the add-a-large-constant trick, evaluate a degree-3 polynomial
-// for 2^r (relative error 7.6e-5, below half an ulp of the bf16 the result is rounded to) and
-// add round(x) to the exponent field.  x <= 127; values below -125 return about 2^-125.
-__device__ __forceinline__ float2 ex2_poly2(float2 x) {
-  const float kBig = 12582912.f;  // 1.5 * 2^23: x + kBig has round(x) in its low mantissa bits
-  x.x = fmaxf(x.x, -125.f);
-  x.y = fmaxf(x.y, -125.f);
-  const float2 t = add2_f(x, make_float2(kBig, kBig));
-  const float2 n = add2_f(t, make_float2(-kBig, -kBig));
-  const float2 r = fma2_f(n, make_float2(-1.f, -1.f), x);
-  float2 q = fma2_f(r, make_float2(0.05520550534129143f, 0.05520550534129143f),
-                    make_float2(0.24261397123336792f, 0.24261397123336792f));
-  q = fma2_f(q, r, make_float2(0.6932547688484192f, 0.6932547688484192f));
-  q = fma2_f(q, r, make_float2(0.9999276995658875f, 0.9999276995658875f));
-  q.x = __int_as_float(__float_as_int(q.x) + (__float_as_int(t.x) << 23));
-  q.y = __int_as_float(__float_as_int(q.y) + (__float_as_int(t.y) << 23));
-  return q;
-}
 // exp2 on the special-function unit, flush-to-zero (no denormal fix-up code around it)
 __device__ __forceinline__ float ex2_ftz(float x) {
   float y;
