@@ -388,6 +388,16 @@ int32_t ss_last_cuda_error(ss_ctx* ctx);
  * max_words 64-bit words to HOST memory and returns the count. */
 ss_status ss_trace_enable(ss_ctx* ctx, int32_t on);
 int32_t ss_trace_read(ss_ctx* ctx, uint64_t* out, int32_t max_words);
+/* Measurement aid (the paper has no counterpart): read n segments of DEVICE memory once, in
+ * one kernel, with streaming 16-byte loads from every SM, and XOR-fold them into the 64-bit
+ * DEVICE word *sink (the caller zeroes it or ignores it; it exists so that the loads cannot be
+ * dropped).  srcs and bytes are HOST arrays of n <= 64 entries (SS_ERR_CAPACITY above), read
+ * before the call returns; every segment 16-byte aligned with a length that is a multiple of
+ * 16, sink 8-byte aligned (SS_ERR_ALIGN otherwise).  Timed by the caller with events on
+ * `stream`, it gives the read bandwidth a kernel that streams memory once can reach on this
+ * GPU in its current clock state. */
+ss_status ss_probe_read(const void* const* srcs, const size_t* bytes, int32_t n, uint64_t* sink,
+                        void* stream);
 /* Number of kernels this context has launched since creation. */
 int64_t ss_launch_count(ss_ctx* ctx);
 /* "simt" or "tcgen05": the chunk kernel the last ss_verify_chunk used. */

@@ -32,7 +32,7 @@ EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "
            "ss_verify_import_state", "ss_stream_layers", "ss_tier_create", "ss_tier_destroy",
            "ss_tier_reset", "ss_tier_get", "ss_tier_tail", "ss_tier_commit", "ss_tier_migrate", "ss_tier_poll",
            "ss_tier_d2h_bytes", "ss_verify_chunk_paged", "ss_width_create", "ss_width_destroy",
-           "ss_width_observe", "ss_width_next", "ss_width_estimate", "ss_cohort_build"]
+           "ss_width_observe", "ss_width_next", "ss_width_estimate", "ss_cohort_build", "ss_probe_read"]
 
 
 class ss_config(C.Structure):
@@ -203,6 +203,8 @@ def load() -> C.CDLL:
     lib.ss_launch_count.argtypes = [vp]
     lib.ss_last_chunk_kernel.restype = C.c_char_p
     lib.ss_last_chunk_kernel.argtypes = [vp]
+    lib.ss_probe_read.restype = C.c_int
+    lib.ss_probe_read.argtypes = [C.POINTER(vp), C.POINTER(C.c_size_t), i32, vp, vp]
     _lib = lib
     return lib
 
@@ -371,6 +373,16 @@ class Context:
 
     def last_chunk_kernel(self) -> str:
         return self.lib.ss_last_chunk_kernel(self.handle).decode()
+
+
+def ss_probe_read(srcs: Sequence[torch.Tensor], sink: torch.Tensor, stream=None) -> None:
+    """Enqueue one streaming read of up to 64 contiguous device tensors; `sink` is a device int64[1]."""
+    n = len(srcs)
+    ptrs = (C.c_void_p * n)(*[t.data_ptr() for t in srcs])
+    sizes = (C.c_size_t * n)(*[t.numel() * t.element_size() for t in srcs])
+    st = load().ss_probe_read(ptrs, sizes, n, sink.data_ptr(), _stream_ptr(stream))
+    if st != SS_OK:
+        raise SpecStreamError(st, "ss_probe_read")
 
 
 def verify_round(ctx: Context, Q, chunks: Sequence, K_loc, V_loc, scale: float, mask_kind=SS_MASK_CHAIN,

@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libspecstream.so")
-SOURCES = ["api.cu", "chunk_simt.cu", "chunk_tc.cu", "chunk_tc_keys.cu", "local_finalize.cu", "stream_round.cu", "static_round.cu", "tier.cu", "width.cu", "cohort.cu"]
+SOURCES = ["api.cu", "chunk_simt.cu", "chunk_tc.cu", "chunk_tc_keys.cu", "local_finalize.cu", "stream_round.cu", "static_round.cu", "tier.cu", "width.cu", "cohort.cu", "probe.cu"]
 
 
 def _newest_source_mtime() -> float:

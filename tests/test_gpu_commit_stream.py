@@ -305,3 +305,23 @@ def test_stream_layers_modes_match_oracle_and_each_other():
         for (O0, L0), (O1, L1) in zip(outs[ssb.SS_LAYERS_PREFETCH], outs[mode]):
             assert torch.equal(O0.view(torch.int16), O1.view(torch.int16)) and torch.equal(L0, L1)
     ctx.close()
+
+
+def test_probe_read_folds_every_word_once():
+    # the read-bandwidth probe must touch every 16-byte vector of every segment exactly once:
+    # its sink is the XOR of all 32-bit words
+    import numpy as np
+    ssb = _ssb()
+    g = torch.Generator(device="cpu").manual_seed(5)
+    sizes = [16, 4096 + 16, (1 << 20) + 48, 3 * (1 << 17)]   # bytes: below, across and past a 128 KiB slab
+    segs = [torch.randint(-2**31, 2**31 - 1, (n // 4,), dtype=torch.int32, generator=g) for n in sizes]
+    want = 0
+    for t in segs:
+        want ^= int(np.bitwise_xor.reduce(t.numpy().view(np.uint32)))
+    dev_segs = [t.to(DEV) for t in segs]
+    sink = torch.zeros(1, dtype=torch.int64, device=DEV)
+    ssb.ss_probe_read(dev_segs, sink)
+    torch.cuda.synchronize()
+    assert int(sink.item()) == want
+    with pytest.raises(ssb.SpecStreamError):
+        ssb.ss_probe_read([dev_segs[1][1:]], sink)   # 4-byte offset: not 16-byte aligned
