@@ -217,6 +217,7 @@ def make_stream_desc(ssb, cfg, lens, host, dev, Q, K_loc, V_loc, bits, O, LSE, b
     for s in range(2):
         d.stage_k[s] = bufs["stage_k"][s].data_ptr()
         d.stage_v[s] = bufs["stage_v"][s].data_ptr()
+    d.stage_fused = 1 if bufs.get("fused") else 0
     d.scratch_fills = bufs["fills"]
     d.valid_len_host = bufs["vl_host"].data_ptr()
     d.valid_len_dev = bufs["vl_dev"].data_ptr()
@@ -235,12 +236,19 @@ def make_stream_desc(ssb, cfg, lens, host, dev, Q, K_loc, V_loc, bits, O, LSE, b
     return d
 
 
-def stream_buffers(cfg, dev, n_chunks, batch_chunks=1):
+def stream_buffers(cfg, dev, n_chunks, batch_chunks=1, fused=True):
+    """Device staging + scratch of ss_stream_round.  fused: one buffer [B][2 (K,V)][H_kv][Ls][d]
+    per slot (each (request, chunk) block is then one copy); else separate K and V buffers."""
     Ls = cfg.L_c * batch_chunks
     fills = (n_chunks + batch_chunks - 1) // batch_chunks + 1
+    if fused:
+        kv = [torch.zeros(cfg.B, 2, cfg.H_kv, Ls, cfg.d, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+        stage_k, stage_v = [t[:, 0] for t in kv], [t[:, 1] for t in kv]   # views of the fused buffers
+    else:
+        stage_k = [torch.zeros(cfg.B, cfg.H_kv, Ls, cfg.d, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+        stage_v = [torch.zeros(cfg.B, cfg.H_kv, Ls, cfg.d, dtype=torch.bfloat16, device=dev) for _ in range(2)]
     return {
-        "stage_k": [torch.zeros(cfg.B, cfg.H_kv, Ls, cfg.d, dtype=torch.bfloat16, device=dev) for _ in range(2)],
-        "stage_v": [torch.zeros(cfg.B, cfg.H_kv, Ls, cfg.d, dtype=torch.bfloat16, device=dev) for _ in range(2)],
+        "stage_k": stage_k, "stage_v": stage_v, "fused": fused,
         "fills": fills,
         "vl_host": torch.zeros(fills * cfg.B, dtype=torch.int32).pin_memory(),
         "vl_dev": torch.zeros(fills * cfg.B, dtype=torch.int32, device=dev),

@@ -230,6 +230,10 @@ typedef struct {
   int32_t commit_cap;        /* token capacity of commit_k / commit_v rows (0 = T_q); with a
                                 tail, commit_k/v may be the tail buffers and zero_off their
                                 lengths, so accepted rows are appended to the tail in place   */
+  int32_t stage_fused;       /* 1: stage_k[s] is ONE buffer [B][2 (K,V)][H_kv][batch_chunks*L_c][d]
+                                (stage_v ignored), the host block's own order, so every
+                                (request, chunk) block crosses the link in one copy instead of
+                                two: copies twice as large reach a few % more of the link     */
 } ss_stream_desc;
 
 typedef struct {

@@ -62,7 +62,7 @@ class ss_stream_desc(C.Structure):
                 ("O_host", C.c_void_p), ("LSE_host", C.c_void_p),
                 ("copy_only", C.c_int32),
                 ("tail_K", ss_tensor), ("tail_V", ss_tensor), ("tail_Lc", C.c_int32),
-                ("tail_len", C.c_void_p), ("commit_cap", C.c_int32)]
+                ("tail_len", C.c_void_p), ("commit_cap", C.c_int32), ("stage_fused", C.c_int32)]
 
 
 class ss_tier_config(C.Structure):

@@ -45,7 +45,8 @@ struct LayerCounts {
 ss_status validate_desc(ss_ctx* ctx, const ss_stream_desc* d, int* n_fills_out) {
   if (!d || !d->hist || !d->hist_len) return SS_ERR_ARG;
   if (d->B <= 0 || d->T_q <= 0 || d->L_c <= 0 || d->batch_chunks <= 0) return SS_ERR_ARG;
-  if (!d->stage_k[0] || !d->stage_k[1] || !d->stage_v[0] || !d->stage_v[1]) return SS_ERR_ARG;
+  if (!d->stage_k[0] || !d->stage_k[1]) return SS_ERR_ARG;
+  if (!d->stage_fused && (!d->stage_v[0] || !d->stage_v[1])) return SS_ERR_ARG;
   if (!d->valid_len_host || !d->valid_len_dev) return SS_ERR_ARG;
   if (!d->copy_only && (!d->Q.ptr || !d->K_loc.ptr || !d->V_loc.ptr || !d->O)) return SS_ERR_ARG;
   int H_q, H_kv, hd;
@@ -73,6 +74,7 @@ ss_status enqueue_layer(ss_ctx* ctx, const ss_stream_desc* d, const ss::PipeRes&
   ss::ctx_dims(ctx, &H_q, &H_kv, &hd);
   const int B = d->B, L_c = d->L_c, bc = d->batch_chunks;
   const bool restore = restore_k != nullptr;
+  const bool fused = d->stage_fused && !restore;  // K and V of a block in one staging buffer
   const int64_t Ls = restore ? restore_tokens : (int64_t)bc * L_c;  // tokens per device buffer row
   if (restore && (int64_t)n_fills * bc * L_c > restore_tokens) return SS_ERR_CAPACITY;
 
@@ -107,6 +109,21 @@ ss_status enqueue_layer(ss_ctx* ctx, const ss_stream_desc* d, const ss::PipeRes&
         if (v <= 0) continue;
         if (v > L_c) v = L_c;
         const uint16_t* src = (const uint16_t*)d->hist[b] + (int64_t)j * block_elems;
+        if (fused) {
+          // K and V of the block in one copy: the staging buffer keeps the host block's order
+          uint16_t* dst = (uint16_t*)d->stage_k[buf] + ((int64_t)b * 2 * H_kv * Ls + (int64_t)jj * L_c) * hd;
+          if (v == L_c && Ls == L_c) {
+            SS_CK(cudaMemcpyAsync(dst, src, (size_t)block_elems * esz, cudaMemcpyHostToDevice,
+                                  r.copy_stream));
+          } else {
+            SS_CK(cudaMemcpy2DAsync(dst, (size_t)Ls * hd * esz, src, (size_t)head_elems * esz,
+                                    (size_t)v * hd * esz, 2 * H_kv, cudaMemcpyHostToDevice,
+                                    r.copy_stream));
+          }
+          cnt->h2d += 2 * (int64_t)H_kv * v * hd * esz;
+          ++cnt->copies;
+          continue;
+        }
         for (int kv = 0; kv < 2; ++kv) {
           uint16_t* base = restore ? (uint16_t*)(kv ? restore_v : restore_k)
                                    : (uint16_t*)(kv ? d->stage_v[buf] : d->stage_k[buf]);
@@ -132,6 +149,10 @@ ss_status enqueue_layer(ss_ctx* ctx, const ss_stream_desc* d, const ss::PipeRes&
     if (!d->copy_only) {
       ss_tensor K = {d->stage_k[buf], (int64_t)H_kv * Ls * hd, Ls * hd, hd};
       ss_tensor V = {d->stage_v[buf], (int64_t)H_kv * Ls * hd, Ls * hd, hd};
+      if (fused) {
+        K.stride_b = V.stride_b = 2 * (int64_t)H_kv * Ls * hd;
+        V.ptr = (const uint16_t*)d->stage_k[buf] + (int64_t)H_kv * Ls * hd;
+      }
       SS_ST(ss_verify_chunk_hinted(ctx, K, V, (int32_t)Ls, d->valid_len_dev + (int64_t)f * B,
                                    d->valid_len_host + (int64_t)f * B, r.attn_stream));
       ++cnt->calls;

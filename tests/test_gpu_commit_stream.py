@@ -121,7 +121,7 @@ def test_call_order_and_argument_errors():
         ssb.Context(2, 9, 2, 128, 4, 4, 128)       # H_q % H_kv != 0
 
 
-def _stream_case(cfg, lens, batch_chunks=1, copy_only=0, accept=True):
+def _stream_case(cfg, lens, batch_chunks=1, copy_only=0, accept=True, fused=True):
     ssb = _ssb()
     Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV, fill=0.0)
     host = bench.pinned_history(cfg, lens, chunks)
@@ -130,7 +130,7 @@ def _stream_case(cfg, lens, batch_chunks=1, copy_only=0, accept=True):
         j, r = divmod(lens[b], cfg.L_c)
         if r and j < host.shape[1]:
             host[b, j, :, :, r:] = float("nan")
-    bufs = bench.stream_buffers(cfg, DEV, len(chunks), batch_chunks)
+    bufs = bench.stream_buffers(cfg, DEV, len(chunks), batch_chunks, fused=fused)
     for s in range(2):
         bufs["stage_k"][s].fill_(float("nan"))
         bufs["stage_v"][s].fill_(float("nan"))
@@ -154,12 +154,15 @@ def _stream_case(cfg, lens, batch_chunks=1, copy_only=0, accept=True):
     return ctx, (Q, chunks, K_loc, V_loc, bits), O, LSE, bufs, acc, stats, desc
 
 
+@pytest.mark.parametrize("fused", [True, False])   # K|V of a block in one staging buffer / two
 @pytest.mark.parametrize("batch_chunks", [1, 2, 3])
-def test_stream_round_matches_oracle_ragged(batch_chunks):
+def test_stream_round_matches_oracle_ragged(batch_chunks, fused):
     import oracle
     cfg = inputs.VerifyConfig("v", 0x62, 5, 8, 2, 128, 128, 8, 0, 900, accept=True)
     lens = [900, 0, 128, 257, 513]
-    ctx, case, O, LSE, bufs, acc, stats, _ = _stream_case(cfg, lens, batch_chunks)
+    ctx, case, O, LSE, bufs, acc, stats, _ = _stream_case(cfg, lens, batch_chunks, fused=fused)
+    n_blocks = sum(-(-l // cfg.L_c) for l in lens)
+    assert stats.copies == (n_blocks if fused else 2 * n_blocks)
     ref = util.oracle_case(cfg, lens, *case)
     util.compare(cfg, O, LSE, ref)
     assert torch.equal(bufs["O_host"], O.cpu()) and torch.equal(bufs["LSE_host"], LSE.cpu())
