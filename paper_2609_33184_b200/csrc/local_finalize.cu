@@ -18,10 +18,29 @@ __device__ __forceinline__ float warp_sum(float v) {
 }
 
 // ---------------------------------------------------------------------------------------
-// Local segment: one warp per query row (b, h_q, i).  Lanes split the local keys for the
-// scores and the head dim for the weighted sum.  The visible set of row i is given by the
-// chain rule j <= i + (T_loc - T_q) or by bit j of the row's mask words.
+// Local segment: one warp per query row (b, h_q, i).  The lanes split the head dim (each holds
+// D / 32 elements of q); the warp walks the VISIBLE local keys only - bit j of the row's mask
+// words, or the chain rule j <= i + (T_loc - T_q) - four at a time so that their K (then V)
+// loads are in flight together.  A tree row sees depth + 1 keys of the T_loc, so the work
+// follows the mask, not T_loc.  Scores go through a per-warp shared array (two passes: maximum,
+// then weights), which keeps the result independent of the order of the keys.
 // ---------------------------------------------------------------------------------------
+constexpr int kLocalBatch = 4;
+
+// visible keys of row i among local keys [w0, w0 + 64)
+__device__ __forceinline__ unsigned long long visible_word(const uint64_t* bits, int w0, int chain_last,
+                                                           int T_loc) {
+  unsigned long long vis;
+  if (bits) {
+    vis = bits[w0 >> 6];
+  } else {
+    const int n = chain_last - w0 + 1;  // keys w0 .. chain_last
+    vis = n >= 64 ? ~0ull : (n <= 0 ? 0ull : ((1ull << n) - 1));
+  }
+  if (T_loc - w0 < 64) vis &= (1ull << (T_loc - w0)) - 1;
+  return vis;
+}
+
 template <int D>
 __global__ void __launch_bounds__(kWarpsPerCta * 32) local_kernel(const LocalParams p) {
   constexpr int CPL = D / 32;  // columns per lane
@@ -36,63 +55,95 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) local_kernel(const LocalPar
     const int h = (int)((row_id / p.T_q) % p.H_q);
     const int b = (int)(row_id / ((int64_t)p.T_q * p.H_q));
     const int kvh = h / p.G;
-    const __nv_bfloat16* q = p.Q + b * p.q_sb + (int64_t)h * p.q_sh + i * p.q_st;
-    const __nv_bfloat16* Kb = p.K + b * p.k_sb + kvh * p.k_sh;
-    const __nv_bfloat16* Vb = p.V + b * p.v_sb + kvh * p.v_sh;
+    const __nv_bfloat16* Kb = p.K + b * p.k_sb + kvh * p.k_sh + lane * CPL;
+    const __nv_bfloat16* Vb = p.V + b * p.v_sb + kvh * p.v_sh + lane * CPL;
     const uint64_t* bits =
         p.mask_bits ? p.mask_bits + ((int64_t)b * p.T_q + i) * p.mask_words : nullptr;
     const int chain_last = i + (p.T_loc - p.T_q);
 
+    // this lane's CPL elements of a bf16 row as floats
+    auto load_row = [&](const __nv_bfloat16* ptr, float (&v)[CPL]) {
+      if (CPL == 4) {
+        const uint2 raw = *reinterpret_cast<const uint2*>(ptr);
+        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+        const float2 c = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+        v[0] = a.x;
+        v[1] = a.y;
+        v[CPL - 2] = c.x;
+        v[CPL - 1] = c.y;
+      } else {
+        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(ptr));
+        v[0] = a.x;
+        v[1] = a.y;
+      }
+    };
+    float q[CPL];
+    load_row(p.Q + b * p.q_sb + (int64_t)h * p.q_sh + i * p.q_st + lane * CPL, q);
+
+    // pass 1: scores of the visible keys and their maximum
     float mx = -INFINITY;
-    for (int j = lane; j < p.T_loc; j += 32) {
-      const bool vis = bits ? ((bits[j >> 6] >> (j & 63)) & 1ull) : (j <= chain_last);
-      float s = -INFINITY;
-      if (vis) {
-        const uint4* kr = reinterpret_cast<const uint4*>(Kb + (int64_t)j * p.k_st);
-        const uint4* qr = reinterpret_cast<const uint4*>(q);
-        float dot = 0.f;
-#pragma unroll 4
-        for (int c8 = 0; c8 < D / 8; ++c8) {
-          const uint4 kq = kr[c8], qq = qr[c8];
-          const __nv_bfloat162* kh = reinterpret_cast<const __nv_bfloat162*>(&kq);
-          const __nv_bfloat162* qh = reinterpret_cast<const __nv_bfloat162*>(&qq);
+    for (int w0 = 0; w0 < p.T_loc; w0 += 64) {
+      unsigned long long vis = visible_word(bits, w0, chain_last, p.T_loc);
+      while (vis) {
+        int jj[kLocalBatch];
+        float dot[kLocalBatch];
 #pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            const float2 kf = __bfloat1622float2(kh[t]), qf = __bfloat1622float2(qh[t]);
-            dot = fmaf(qf.x, kf.x, dot);
-            dot = fmaf(qf.y, kf.y, dot);
+        for (int u = 0; u < kLocalBatch; ++u) {
+          jj[u] = vis ? w0 + __ffsll((long long)vis) - 1 : -1;
+          vis &= vis - 1;  // 0 stays 0
+          dot[u] = 0.f;
+          if (jj[u] >= 0) {
+            float k[CPL];
+            load_row(Kb + (int64_t)jj[u] * p.k_st, k);
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) dot[u] = fmaf(q[c], k[c], dot[u]);
           }
         }
-        s = dot * p.scale_log2;
+#pragma unroll
+        for (int o = 16; o; o >>= 1) {
+#pragma unroll
+          for (int u = 0; u < kLocalBatch; ++u) dot[u] += __shfl_xor_sync(0xffffffffu, dot[u], o);
+        }
+#pragma unroll
+        for (int u = 0; u < kLocalBatch; ++u) {
+          if (jj[u] >= 0) {
+            const float sv = dot[u] * p.scale_log2;
+            if (lane == 0) sc[jj[u]] = sv;
+            mx = fmaxf(mx, sv);
+          }
+        }
       }
-      sc[j] = s;
-      mx = fmaxf(mx, s);
     }
-    mx = warp_max(mx);
     __syncwarp();
+
+    // pass 2: weights, row sum and weighted V sum over the same keys
     float acc[CPL];
 #pragma unroll
     for (int c = 0; c < CPL; ++c) acc[c] = 0.f;
     float l = 0.f;
     if (mx > -INFINITY) {
-      for (int j = 0; j < p.T_loc; ++j) {
-        const float s = sc[j];
-        if (s == -INFINITY) continue;  // warp-uniform
-        const float w = exp2f(s - mx);
-        l += w;
-        const __nv_bfloat16* vr = Vb + (int64_t)j * p.v_st + lane * CPL;
-        if (CPL == 4) {
-          const uint2 raw = *reinterpret_cast<const uint2*>(vr);
-          const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
-          const float2 c = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-          acc[0] = fmaf(w, a.x, acc[0]);
-          acc[1] = fmaf(w, a.y, acc[1]);
-          acc[CPL - 2] = fmaf(w, c.x, acc[CPL - 2]);
-          acc[CPL - 1] = fmaf(w, c.y, acc[CPL - 1]);
-        } else {
-          const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(vr));
-          acc[0] = fmaf(w, a.x, acc[0]);
-          acc[1] = fmaf(w, a.y, acc[1]);
+      for (int w0 = 0; w0 < p.T_loc; w0 += 64) {
+        unsigned long long vis = visible_word(bits, w0, chain_last, p.T_loc);
+        while (vis) {
+          float wgt[kLocalBatch], v[kLocalBatch][CPL];
+#pragma unroll
+          for (int u = 0; u < kLocalBatch; ++u) {
+            const int j = vis ? w0 + __ffsll((long long)vis) - 1 : -1;
+            vis &= vis - 1;
+            wgt[u] = 0.f;
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) v[u][c] = 0.f;
+            if (j >= 0) {
+              load_row(Vb + (int64_t)j * p.v_st, v[u]);
+              wgt[u] = exp2f(sc[j] - mx);
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < kLocalBatch; ++u) {
+            l += wgt[u];
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) acc[c] = fmaf(wgt[u], v[u][c], acc[c]);
+          }
         }
       }
     }
@@ -114,11 +165,35 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) local_kernel(const LocalPar
 // and LSE (finalize) or the merged state itself (fold).  One warp per row.
 // ---------------------------------------------------------------------------------------
 // MODE 0: finalize (O, LSE); 1: fold into set 0; 2: export the merged state in row order.
+//
+// A row has one partial per (set, token split): 17 for a 16-chunk round, up to a few hundred.
+// They are read with as many loads in flight as the warp can hold: the (m, l) pairs one per
+// lane (32 at a time), the a[] rows eight at a time with the weight and the address of each
+// broadcast from the lane that owns the partial.
+constexpr int kMergeBatch = 8;
+
 template <int D, int MODE>
 __global__ void __launch_bounds__(kWarpsPerCta * 32) merge_kernel(const MergeParams p) {
   constexpr bool FOLD = MODE == 1;
   constexpr int CPL = D / 32;
+  // flat partial index f -> set: first_s[s] = partials before set s (sets in launch order, the
+  // local set last); built before the wait below, it depends on the launch parameters only
+  __shared__ int first_s[kMaxSets + 2];
+  __shared__ uint8_t set_of[(kMaxSets + 1) * kMaxSplits];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int n_total = p.n_sets + (p.has_local ? 1 : 0);
+  if (threadIdx.x == 0) {
+    int acc = 0;
+    for (int s = 0; s < n_total; ++s) {
+      first_s[s] = acc;
+      acc += (s < p.n_sets) ? p.splits[s] : 1;
+    }
+    first_s[n_total] = acc;
+  }
+  __syncthreads();
+  for (int s = threadIdx.x; s < n_total; s += kWarpsPerCta * 32)
+    for (int f = first_s[s]; f < first_s[s + 1]; ++f) set_of[f] = (uint8_t)s;
+  __syncthreads();
   const int64_t row_id = (int64_t)blockIdx.x * kWarpsPerCta + warp;
   const int64_t n_rows = (int64_t)p.B * p.H_q * p.T_q;
   if (MODE == 0) pdl_wait_prior();  // every partial of the round must be complete
@@ -130,16 +205,21 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) merge_kernel(const MergePar
   const int r = (h % p.G) * p.T_q + i;
   const size_t slot0 = (size_t)b * p.H_kv + kvh;
   const size_t split_stride = (size_t)p.B * p.H_kv;
-
-  // pass 1: global maximum over partials
-  const int n_total = p.n_sets + (p.has_local ? 1 : 0);
-  float M = -INFINITY;
-  for (int s = 0; s < n_total; ++s) {
+  const int n_part = first_s[n_total];
+  // (m, l) of partial f and the element offset of its a[] row
+  auto load_ml = [&](int f, int64_t* a_off) {
+    const int s = set_of[f], k = f - first_s[s];
     const int set = (s < p.n_sets) ? s : p.local_set;
-    const int ns = (s < p.n_sets) ? p.splits[s] : 1;
-    const float2* ml = p.part_ml + (int64_t)set * p.set_stride_ml;
-    for (int k = lane; k < ns; k += 32)
-      M = fmaxf(M, ml[(slot0 + k * split_stride) * p.R_stride + r].x);
+    const size_t idx = (slot0 + k * split_stride) * p.R_stride + r;
+    *a_off = (int64_t)set * p.set_stride_a + (int64_t)idx * D;
+    return p.part_ml[(int64_t)set * p.set_stride_ml + idx];
+  };
+
+  // pass 1: global maximum over the partials, one per lane
+  float M = -INFINITY;
+  for (int f = lane; f < n_part; f += 32) {
+    int64_t off;
+    M = fmaxf(M, load_ml(f, &off).x);
   }
   M = warp_max(M);
 
@@ -148,31 +228,54 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) merge_kernel(const MergePar
   for (int c = 0; c < CPL; ++c) acc[c] = 0.f;
   float L = 0.f;
   if (M > -INFINITY) {
-    for (int s = 0; s < n_total; ++s) {
-      const int set = (s < p.n_sets) ? s : p.local_set;
-      const int ns = (s < p.n_sets) ? p.splits[s] : 1;
-      const float2* ml = p.part_ml + (int64_t)set * p.set_stride_ml;
-      const float* pa = p.part_a + (int64_t)set * p.set_stride_a;
-      for (int k = 0; k < ns; ++k) {
-        const size_t idx = (slot0 + k * split_stride) * p.R_stride + r;
-        const float2 st = ml[idx];
-        if (st.y == 0.f || st.x == -INFINITY) continue;  // identity: a[] undefined
-        const float w = exp2f(st.x - M);
-        L = fmaf(w, st.y, L);
-        const float* a = pa + idx * D + lane * CPL;
-        if (CPL == 4) {
-          const float4 v = *reinterpret_cast<const float4*>(a);
-          acc[0] = fmaf(w, v.x, acc[0]);
-          acc[1] = fmaf(w, v.y, acc[1]);
-          acc[CPL - 2] = fmaf(w, v.z, acc[CPL - 2]);
-          acc[CPL - 1] = fmaf(w, v.w, acc[CPL - 1]);
-        } else {
-          const float2 v = *reinterpret_cast<const float2*>(a);
-          acc[0] = fmaf(w, v.x, acc[0]);
-          acc[1] = fmaf(w, v.y, acc[1]);
+    for (int base = 0; base < n_part; base += 32) {
+      // lane j owns partial base + j: its weight (0 for an identity state, whose a[] is
+      // undefined and must not be read) and the offset of its a[] row
+      float w = 0.f;
+      int64_t off = 0;
+      if (base + lane < n_part) {
+        const float2 st = load_ml(base + lane, &off);
+        if (st.y != 0.f && st.x != -INFINITY) {
+          w = exp2f(st.x - M);
+          L = fmaf(w, st.y, L);
+        }
+      }
+      const int cnt = min(32, n_part - base);
+      for (int j0 = 0; j0 < cnt; j0 += kMergeBatch) {
+        float wj[kMergeBatch];
+        float v[kMergeBatch][CPL];
+#pragma unroll
+        for (int u = 0; u < kMergeBatch; ++u) {
+          const int j = (j0 + u) & 31;
+          wj[u] = __shfl_sync(0xffffffffu, w, j);
+          const int64_t oj = __shfl_sync(0xffffffffu, off, j);
+#pragma unroll
+          for (int c = 0; c < CPL; ++c) v[u][c] = 0.f;
+          if (j0 + u < cnt && wj[u] != 0.f) {  // warp-uniform
+            const float* a = p.part_a + oj + lane * CPL;
+            if (CPL == 4) {
+              const float4 x = *reinterpret_cast<const float4*>(a);
+              v[u][0] = x.x;
+              v[u][1] = x.y;
+              v[u][CPL - 2] = x.z;
+              v[u][CPL - 1] = x.w;
+            } else {
+              const float2 x = *reinterpret_cast<const float2*>(a);
+              v[u][0] = x.x;
+              v[u][1] = x.y;
+            }
+          } else {
+            wj[u] = 0.f;
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < kMergeBatch; ++u) {
+#pragma unroll
+          for (int c = 0; c < CPL; ++c) acc[c] = fmaf(wj[u], v[u][c], acc[c]);
         }
       }
     }
+    L = warp_sum(L);
   }
   if (MODE == 2) {
     if (lane == 0) p.fold_ml[row_id] = make_float2(L > 0.f ? M : -INFINITY, L);
