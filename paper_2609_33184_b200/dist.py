@@ -1,7 +1,15 @@
-"""Multi-GPU plumbing: the path shards by request, so there is no data-path collective.
+"""Multi-GPU plumbing.
 
-Every rank runs the same per-GPU workload on its own requests; the only communication is
+The path shards by request (the cohort axis), so the benchmark has no data-path collective:
+every rank runs the same per-GPU workload on its own requests and the only communication is
 the barrier around the timed region and the max-over-ranks reduction of its duration.
+
+One optional exchange is provided for a history that is sharded by CHUNKS over the ranks
+(context-parallel style): each rank reduces its own chunks of every request to a merged state
+(ss_verify_export_state), `allgather_states` exchanges the states with one all-gather, and the
+peers' states are added to the open round with ss_verify_import_state before finalize.  The
+merge is order-free (Eq. 17), so every rank ends with the full result.  The all-gather writes
+into this rank's own memory; the kernels never read a peer's memory.
 """
 from __future__ import annotations
 
@@ -56,3 +64,36 @@ def barrier(cuda: bool = False):
         dist.barrier()
     if cuda:
         torch.cuda.synchronize()
+
+
+def chunk_shard(n_chunks: int, rank: int, world: int):
+    """Chunk indices of a request's history owned by `rank` (round-robin: every rank gets
+    early and late chunks, so ragged lengths stay balanced)."""
+    return range(rank, n_chunks, world)
+
+
+def allgather_states(ml: torch.Tensor, a: torch.Tensor, group=None):
+    """Exchange exported round states between the ranks of `group` with one all-gather each
+    for ml [rows, 2] and a [rows, d] (fp32; device tensors over NCCL, CPU tensors over gloo).
+
+    Returns the list [(ml_r, a_r) for every OTHER rank r], in rank order: the states to hand
+    to ss_verify_import_state.  Without a process group the list is empty.
+    """
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return []
+    world, rank = dist.get_world_size(group), dist.get_rank(group)
+    ml_all = [torch.empty_like(ml) for _ in range(world)]
+    a_all = [torch.empty_like(a) for _ in range(world)]
+    dist.all_gather(ml_all, ml.contiguous(), group=group)
+    dist.all_gather(a_all, a.contiguous(), group=group)
+    return [(ml_all[r], a_all[r]) for r in range(world) if r != rank]
+
+
+def import_peer_states(ctx, ml: torch.Tensor, a: torch.Tensor, group=None, stream=None) -> int:
+    """Export this rank's state of the open round is given as (ml, a); gather the peers'
+    states and add them to the round.  Returns the number of states imported."""
+    peers = allgather_states(ml, a, group)
+    for ml_r, a_r in peers:
+        ctx.ss_verify_import_state(ml_r, a_r, stream)
+    return len(peers)

@@ -216,8 +216,11 @@ def test_export_import_state_shards_the_history_by_chunks():
     lens = inputs.history_lengths(cfg)
     Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
     rows = cfg.B * cfg.H_q * cfg.T_q
+    from paper_2609_33184_b200 import dist as ssdist
     states = []
-    for part in (chunks[0::2], chunks[1::2]):
+    shards = [[chunks[j] for j in ssdist.chunk_shard(len(chunks), r, 2)] for r in range(2)]
+    assert shards[0] == chunks[0::2] and shards[1] == chunks[1::2]
+    for part in shards:
         ctx = util.make_ctx(cfg)
         ml = torch.empty(rows, 2, dtype=torch.float32, device=DEV)
         a = torch.empty(rows, cfg.d, dtype=torch.float32, device=DEV)
@@ -225,6 +228,7 @@ def test_export_import_state_shards_the_history_by_chunks():
         for K, V, vl in part:
             ctx.ss_verify_chunk(K, V, vl)
         ctx.ss_verify_export_state(ml, a)
+        assert ssdist.import_peer_states(ctx, ml, a) == 0   # no process group: no peers
         O_part = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
         ctx.ss_verify_finalize(O_part, None)      # the round stays usable after an export
         torch.cuda.synchronize()
