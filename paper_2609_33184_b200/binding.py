@@ -225,8 +225,18 @@ def as_ss_tensor(t: torch.Tensor) -> ss_tensor:
     return ss_tensor(t.data_ptr(), t.stride(0), t.stride(1), t.stride(2))
 
 
+_raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
-    return (stream or torch.cuda.current_stream()).cuda_stream
+    """cudaStream_t of `stream`, or of torch's current stream on the current device (the raw
+    getter costs 0.1 us per call against 3 us for building a torch.cuda.Stream object, which
+    matters for rounds of a few small launches)."""
+    if stream is not None:
+        return stream.cuda_stream
+    if _raw_stream is not None:
+        return _raw_stream(torch.cuda.current_device())
+    return torch.cuda.current_stream().cuda_stream
 
 
 def _ptr(t: Optional[torch.Tensor]):
@@ -249,6 +259,15 @@ class Context:
         if st != SS_OK:
             raise SpecStreamError(st, "ss_create")
         self.H_q, self.H_kv, self.d = H_q, H_kv, d
+        self._dev = device
+
+    def _sp(self, stream) -> int:
+        """cudaStream_t of `stream`, else torch's current stream on this context's device."""
+        if stream is not None:
+            return stream.cuda_stream
+        if _raw_stream is not None:
+            return _raw_stream(self._dev)
+        return torch.cuda.current_stream(self._dev).cuda_stream
 
     def _check(self, st: int, where: str):
         if st != SS_OK:
@@ -270,7 +289,7 @@ class Context:
         B, H_q, T_q, d = Q.shape
         assert H_q == self.H_q and d == self.d
         self._check(self.lib.ss_verify_begin(self.handle, as_ss_tensor(Q), B, T_q, scale,
-                                             _stream_ptr(stream)), "ss_verify_begin")
+                                             self._sp(stream)), "ss_verify_begin")
 
     def ss_verify_chunk(self, K: torch.Tensor, V: torch.Tensor, valid_len: Optional[torch.Tensor] = None,
                         stream=None):
@@ -278,7 +297,7 @@ class Context:
         if valid_len is not None:
             assert valid_len.dtype == torch.int32 and valid_len.is_cuda
         self._check(self.lib.ss_verify_chunk(self.handle, as_ss_tensor(K), as_ss_tensor(V), L_c,
-                                             _ptr(valid_len), _stream_ptr(stream)), "ss_verify_chunk")
+                                             _ptr(valid_len), self._sp(stream)), "ss_verify_chunk")
 
     def ss_verify_chunk_hinted(self, K: torch.Tensor, V: torch.Tensor, valid_len: torch.Tensor,
                                valid_len_host, stream=None):
@@ -287,7 +306,7 @@ class Context:
         if not isinstance(valid_len_host, C.Array):
             valid_len_host = (C.c_int32 * len(valid_len_host))(*valid_len_host)
         self._check(self.lib.ss_verify_chunk_hinted(self.handle, as_ss_tensor(K), as_ss_tensor(V), L_c,
-                                                    _ptr(valid_len), valid_len_host, _stream_ptr(stream)),
+                                                    _ptr(valid_len), valid_len_host, self._sp(stream)),
                     "ss_verify_chunk_hinted")
 
     def ss_verify_chunk_paged(self, K_pool: torch.Tensor, V_pool: torch.Tensor, page_table: torch.Tensor,
@@ -300,7 +319,7 @@ class Context:
         self._check(self.lib.ss_verify_chunk_paged(self.handle, as_ss_tensor(K_pool), as_ss_tensor(V_pool),
                                                    n_pages, page_size, page_table.data_ptr(),
                                                    page_table.shape[1], _ptr(valid_len), valid_len_host,
-                                                   _stream_ptr(stream)), "ss_verify_chunk_paged")
+                                                   self._sp(stream)), "ss_verify_chunk_paged")
 
     def ss_verify_local(self, K_loc: torch.Tensor, V_loc: torch.Tensor, mask_kind: int = SS_MASK_CHAIN,
                         mask_bits: Optional[torch.Tensor] = None, stream=None):
@@ -308,25 +327,25 @@ class Context:
         if mask_bits is not None:
             assert mask_bits.dtype == torch.int64 and mask_bits.is_contiguous()
         self._check(self.lib.ss_verify_local(self.handle, as_ss_tensor(K_loc), as_ss_tensor(V_loc),
-                                             T_loc, mask_kind, _ptr(mask_bits), _stream_ptr(stream)),
+                                             T_loc, mask_kind, _ptr(mask_bits), self._sp(stream)),
                     "ss_verify_local")
 
     def ss_verify_export_state(self, ml: torch.Tensor, a: torch.Tensor, stream=None):
         assert ml.dtype == torch.float32 and a.dtype == torch.float32 and ml.is_contiguous() and a.is_contiguous()
         self._check(self.lib.ss_verify_export_state(self.handle, ml.data_ptr(), a.data_ptr(),
-                                                    _stream_ptr(stream)), "ss_verify_export_state")
+                                                    self._sp(stream)), "ss_verify_export_state")
 
     def ss_verify_import_state(self, ml: torch.Tensor, a: torch.Tensor, stream=None):
         assert ml.dtype == torch.float32 and a.dtype == torch.float32 and ml.is_contiguous() and a.is_contiguous()
         self._check(self.lib.ss_verify_import_state(self.handle, ml.data_ptr(), a.data_ptr(),
-                                                    _stream_ptr(stream)), "ss_verify_import_state")
+                                                    self._sp(stream)), "ss_verify_import_state")
 
     def ss_verify_finalize(self, O: torch.Tensor, LSE: Optional[torch.Tensor], stream=None):
         assert O.dtype == torch.bfloat16 and O.is_contiguous()
         if LSE is not None:
             assert LSE.dtype == torch.float32 and LSE.is_contiguous()
         self._check(self.lib.ss_verify_finalize(self.handle, O.data_ptr(), _ptr(LSE),
-                                                _stream_ptr(stream)), "ss_verify_finalize")
+                                                self._sp(stream)), "ss_verify_finalize")
 
     def ss_commit_gather(self, K_loc, V_loc, accept_idx, accept_cnt, K_dst, V_dst, dst_off, stream=None):
         B, _, T_loc, _ = K_loc.shape
@@ -336,12 +355,12 @@ class Context:
         self._check(self.lib.ss_commit_gather(self.handle, as_ss_tensor(K_loc), as_ss_tensor(V_loc), B,
                                               T_loc, accept_idx.data_ptr(), accept_cnt.data_ptr(),
                                               as_ss_tensor(K_dst), as_ss_tensor(V_dst), cap,
-                                              dst_off.data_ptr(), _stream_ptr(stream)), "ss_commit_gather")
+                                              dst_off.data_ptr(), self._sp(stream)), "ss_commit_gather")
 
     def ss_poll_status(self, stream=None, timeout_ms: int = 0):
         """Returns (status, device_bits)."""
         bits = C.c_uint32(0)
-        st = self.lib.ss_poll_status(self.handle, _stream_ptr(stream), timeout_ms, C.byref(bits))
+        st = self.lib.ss_poll_status(self.handle, self._sp(stream), timeout_ms, C.byref(bits))
         return st, bits.value
 
     def ss_stream_round(self, desc: ss_stream_desc) -> ss_stream_stats:
