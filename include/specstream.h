@@ -92,6 +92,11 @@ typedef struct {
 #define SS_FLAG_ROWS_ON_M 4u
 /* Use the keys-on-M kernel for any number of rows per kv-head (default: up to 32). */
 #define SS_FLAG_KEYS_ON_M 8u
+/* Tuning overrides read from the environment by ss_create (for experiments; unset = automatic):
+ *   SS_CHUNK_KERNEL=rows|keys  as SS_FLAG_ROWS_ON_M / SS_FLAG_KEYS_ON_M
+ *   SS_SPLITS=n                token splits of every chunk call (default: sized so that a
+ *                              call launches about one CTA per SM)
+ *   SS_TARGET_CTAS=n           the CTA count the automatic split choice aims at */
 
 typedef struct {
   const void* ptr;                      /* device pointer, bf16                      */
