@@ -42,7 +42,9 @@ def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         with open(p) as f:
-            return float(json.load(f)["hbm_gbs"]), "measured"
+            v = json.load(f).get("hbm_gbs")
+        if v:
+            return float(v), "measured"
     return FALLBACK_HBM_GBS, "fallback"
 
 
@@ -51,7 +53,9 @@ def tensor_peak():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         with open(p) as f:
-            return float(json.load(f)["bf16_tflops_sustained"]), "measured (sustained)"
+            v = json.load(f).get("bf16_tflops_sustained")
+        if v:
+            return float(v), "measured (sustained)"
     return FALLBACK_BF16_TFLOPS, "fallback (sustained)"
 
 
