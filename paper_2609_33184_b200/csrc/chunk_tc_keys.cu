@@ -60,7 +60,7 @@ struct alignas(16) Ctl {
   uint32_t tmem_base;
   volatile uint32_t abort;
   volatile uint32_t flag[3];
-  alignas(16) float m_ref[N];     // read as float4
+  alignas(16) float nm_ref[N];    // NEGATED row references -m[r] (+inf = none yet); read as float4
   alignas(16) float smax[4][N];   // per lane quadrant
 };
 
@@ -196,7 +196,7 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
       const int half = c8 >> 3, j = c8 & 7;
       *reinterpret_cast<uint4*>(q_s + half * C::kQHalf + n * 128 + ((j ^ (n & 7)) << 4)) = raw;
     }
-    if (tid < N) ctl->m_ref[tid] = -INFINITY;
+    if (tid < N) ctl->nm_ref[tid] = INFINITY;
     fence_proxy_async();
   }
   tc_fence_before();
@@ -303,13 +303,14 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
     const int cn = max(0, min(cpg, n_mma - c0));               // multiple of 16, <= NC
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     bool dead = false;
+    const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
     auto wait = [&](uint64_t* bar, uint32_t parity) {
       if (!dead && !mwait(bar, parity)) dead = true;
       dead = __any_sync(0xffffffffu, dead);
     };
-    float lsum[NC];
+    float2 lsum[NC / 2];  // row sums of this key lane, two rows per packed add
 #pragma unroll
-    for (int r = 0; r < NC; ++r) lsum[r] = 0.f;
+    for (int r = 0; r < NC / 2; ++r) lsum[r] = make_float2(0.f, 0.f);
     for (int t = 0; t < n_tiles; ++t) {
       if (tid == 0) trace(tr, 2, t, 0);
       wait(&ctl->sfull[t & 1], (t >> 1) & 1);
@@ -351,11 +352,16 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
             if (q * 16 < cn) {
 #pragma unroll
               for (int c4 = 0; c4 < 4; ++c4) {
-                const float4 mr = *reinterpret_cast<const float4*>(&ctl->m_ref[c0 + q * 16 + c4 * 4]);
-                const float mm[4] = {mr.x, mr.y, mr.z, mr.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e)  // +inf while m_ref is -inf
-                  mx4[e] = fmaxf(mx4[e], fmaf(__uint_as_float(raw[h][c4 * 4 + e]), p.scale_log2, -mm[e]));
+                // s * scale - m for four rows as two packed FMAs (+inf while there is no reference)
+                const float4 nm = *reinterpret_cast<const float4*>(&ctl->nm_ref[c0 + q * 16 + c4 * 4]);
+                const float2 x01 = fma2_f(make_float2(__uint_as_float(raw[h][c4 * 4 + 0]),
+                                                      __uint_as_float(raw[h][c4 * 4 + 1])),
+                                          sc2, make_float2(nm.x, nm.y));
+                const float2 x23 = fma2_f(make_float2(__uint_as_float(raw[h][c4 * 4 + 2]),
+                                                      __uint_as_float(raw[h][c4 * 4 + 3])),
+                                          sc2, make_float2(nm.z, nm.w));
+                mx4[c4 & 1] = max3_f(mx4[c4 & 1], x01.x, x01.y);
+                mx4[2 + (c4 & 1)] = max3_f(mx4[2 + (c4 & 1)], x23.x, x23.y);
               }
             }
           }
@@ -399,11 +405,15 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
 #pragma unroll
               for (int c = 0; c < 16; ++c) {
                 const int r = c0 + q * 16 + c;
-                const float m_old = ctl->m_ref[r];
+                const float m_old = -ctl->nm_ref[r];
                 const float m_new = fmaxf(fmaxf(m_old, ctl->smax[0][r]),
                                           fmaxf(fmaxf(ctl->smax[1][r], ctl->smax[2][r]), ctl->smax[3][r]));
                 f[c] = (m_old == -INFINITY) ? 0.f : exp2f(m_old - m_new);
-                lsum[q * 16 + c] *= f[c];
+              }
+#pragma unroll
+              for (int c = 0; c < 16; c += 2) {
+                lsum[q * 8 + c / 2].x *= f[c];
+                lsum[q * 8 + c / 2].y *= f[c + 1];
               }
               if (t > 0) {
                 uint32_t o[16];
@@ -419,9 +429,9 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
         }
         named_bar_sync(1, C::kSoft);  // every thread has read the old references
         if (tid < n_mma && !dead) {
-          const float m_old = ctl->m_ref[tid];
-          ctl->m_ref[tid] = fmaxf(fmaxf(m_old, ctl->smax[0][tid]),
-                                  fmaxf(fmaxf(ctl->smax[1][tid], ctl->smax[2][tid]), ctl->smax[3][tid]));
+          const float m_old = -ctl->nm_ref[tid];
+          ctl->nm_ref[tid] = -fmaxf(fmaxf(m_old, ctl->smax[0][tid]),
+                                    fmaxf(fmaxf(ctl->smax[1][tid], ctl->smax[2][tid]), ctl->smax[3][tid]));
         }
         named_bar_sync(1, C::kSoft);
       }
@@ -441,22 +451,32 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
           const int q = q0 + h;
           const uint32_t (&raw)[16] = raw2[h];
           if (q * 16 < cn) {
-            // staged so that the 16 exponentials of a chunk are independent instructions
+            // staged so that the 16 exponentials of a chunk are independent instructions;
+            // two rows per packed fp32 instruction
             float pv[16];
 #pragma unroll
             for (int c4 = 0; c4 < 4; ++c4) {
-              const float4 mr = *reinterpret_cast<const float4*>(&ctl->m_ref[c0 + q * 16 + c4 * 4]);
-              pv[c4 * 4 + 0] = fmaf(__uint_as_float(raw[c4 * 4 + 0]), p.scale_log2, -mr.x);
-              pv[c4 * 4 + 1] = fmaf(__uint_as_float(raw[c4 * 4 + 1]), p.scale_log2, -mr.y);
-              pv[c4 * 4 + 2] = fmaf(__uint_as_float(raw[c4 * 4 + 2]), p.scale_log2, -mr.z);
-              pv[c4 * 4 + 3] = fmaf(__uint_as_float(raw[c4 * 4 + 3]), p.scale_log2, -mr.w);
+              const float4 nm = *reinterpret_cast<const float4*>(&ctl->nm_ref[c0 + q * 16 + c4 * 4]);
+              const float2 x01 = fma2_f(make_float2(__uint_as_float(raw[c4 * 4 + 0]),
+                                                    __uint_as_float(raw[c4 * 4 + 1])),
+                                        sc2, make_float2(nm.x, nm.y));
+              const float2 x23 = fma2_f(make_float2(__uint_as_float(raw[c4 * 4 + 2]),
+                                                    __uint_as_float(raw[c4 * 4 + 3])),
+                                        sc2, make_float2(nm.z, nm.w));
+              pv[c4 * 4 + 0] = x01.x;
+              pv[c4 * 4 + 1] = x01.y;
+              pv[c4 * 4 + 2] = x23.x;
+              pv[c4 * 4 + 3] = x23.y;
             }
 #pragma unroll
             for (int c = 0; c < 16; ++c) pv[c] = ex2_ftz(pv[c]);
+            if (n_valid < kKeys) {  // only the tile that straddles the valid length (warp-uniform)
 #pragma unroll
-            for (int c = 0; c < 16; ++c) pv[c] = key_ok ? pv[c] : 0.f;
+              for (int c = 0; c < 16; ++c) pv[c] = key_ok ? pv[c] : 0.f;
+            }
 #pragma unroll
-            for (int c = 0; c < 16; ++c) lsum[q * 16 + c] += pv[c];
+            for (int c = 0; c < 16; c += 2)
+              lsum[q * 8 + c / 2] = add2_f(lsum[q * 8 + c / 2], make_float2(pv[c], pv[c + 1]));
             uint32_t pk[8];
 #pragma unroll
             for (int c = 0; c < 16; c += 2) {
@@ -484,12 +504,12 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
       float* red = reinterpret_cast<float*>(smem);  // [128][N + 1] over the free ring
 #pragma unroll
       for (int r = 0; r < NC; ++r)
-        if (r < cn) red[L * (N + 1) + c0 + r] = lsum[r];
+        if (r < cn) red[L * (N + 1) + c0 + r] = (r & 1) ? lsum[r / 2].y : lsum[r / 2].x;
       named_bar_sync(1, C::kSoft);
       if (tid < nrows) {
         float lt = 0.f;
         for (int k = 0; k < kKeys; ++k) lt += red[k * (N + 1) + tid];
-        out_ml[tid] = make_float2(lt > 0.f ? ctl->m_ref[tid] : -INFINITY, lt);
+        out_ml[tid] = make_float2(lt > 0.f ? -ctl->nm_ref[tid] : -INFINITY, lt);
       }
       // thread (L, cg) holds head dim L of its rows
 #pragma unroll
