@@ -6,10 +6,11 @@
 // the kv-head (T_q candidate queries x G query heads) ride in the M dimension of the MMAs,
 // so every K/V byte is fetched from HBM once and serves the whole query group.
 //
-//   warp 4 (one lane)  TMA producer: K tiles and V tiles of 64 tokens, two slots each,
-//                      128-byte swizzle, evict-first L2 policy (the history is streamed).
-//                      A K slot is released as soon as its score MMAs retire, a V slot
-//                      after its output MMAs.
+//   warp 4 (one lane)  TMA producer: K tiles and V tiles of 64 tokens, two K slots and three V
+//                      slots, 128-byte swizzle, evict-first L2 policy (the history is
+//                      streamed).  A K slot is released as soon as its score MMAs retire
+//                      (two tiles ahead of the output MMAs), a V slot after its output MMAs,
+//                      which is why V gets the third slot.
 //   warp 5 (one lane)  MMA issuer:   S[t%2] = Q K_t^T  (M=128, N=64,  K=d=128: 8 x k16, smem x smem)
 //                                    O += P_t V_t      (M=128, N=128, K=64:    4 x k16, tmem x smem)
 //                      in the order QK(0) QK(1) | PV(0) QK(2) | PV(1) QK(3) | ...: the scores of
@@ -22,8 +23,9 @@
 //
 // Tensor memory (256 columns): [0,64) S0, [64,128) S1 (fp32; P of a tile as bf16 pairs over
 // the first 32 columns of its buffer); [128,256) O (fp32).  Shared memory: the Q tile
-// (32 KB, written once by the softmax threads in the swizzled K-major layout) and two slots
-// of K and V (64 KB); two CTAs fit per SM.
+// (32 KB, written once by the softmax threads in the swizzled K-major layout), two K slots
+// and three V slots (80 KB) and 256 bytes of barriers: 112.25 KB, so that two CTAs fit per SM
+// to the last kilobyte (the window must be 1024-byte aligned; checked at run time).
 //
 // When the row tile has <= 32 (<= 64) rows the Q rows are replicated 4x (2x) along M and
 // each replica takes a quarter (half) of the tile's keys: lane L holds row L % R_pad and
@@ -44,28 +46,30 @@ namespace ss {
 namespace {
 
 constexpr int kThreads = 192;
-constexpr int kStages = 2;
+constexpr int kKStages = 2, kVStages = 3;
 constexpr int kD = 128;
 constexpr int kHalfTile = kTileKeys * 64 * 2;       // 8 KB: [64 keys][64 d] bf16
 constexpr int kTileBytes = 2 * kHalfTile;           // 16 KB: one K tile or one V tile
-constexpr int kStageBytes = 2 * kTileBytes;         // K then V
 constexpr int kQHalf = 128 * 64 * 2;                // 16 KB: [128 rows][64 d] bf16
 constexpr int kQBytes = 2 * kQHalf;                 // 32 KB: the Q tile
-constexpr int kSmemData = kQBytes + kStages * kStageBytes;  // 96 KB
-constexpr int kSmemCtl = 2048;
-constexpr int kSmemTotal = kSmemData + kSmemCtl + 1024;     // + alignment slack
+constexpr int kOffK = kQBytes;                              // K slots
+constexpr int kOffV = kOffK + kKStages * kTileBytes;        // V slots
+constexpr int kSmemData = kOffV + kVStages * kTileBytes;    // 112 KB
+constexpr int kSmemCtl = 256;
+constexpr int kSmemTotal = kSmemData + kSmemCtl;
+// two CTAs per SM: 227 KB per SM less 1 KB reserved per CTA
+static_assert(2 * (kSmemTotal + 1024) <= 227 * 1024, "two CTAs per SM");
 constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kColS = 0, kColO = 128;          // S buffer t%2 at kColS + 64 (t%2)
 constexpr float kRescaleThreshold = 8.f;
 
 struct Ctl {
-  uint64_t kfull[kStages], vfull[kStages], kempty[kStages], vempty[kStages];
+  uint64_t kfull[kKStages], kempty[kKStages], vfull[kVStages], vempty[kVStages];
   uint64_t sfull[2], pready[2];  // per score buffer
   uint64_t odone;                // one phase per tile: PV(t) has retired
   uint64_t pvdone;               // the last PV has retired
   uint32_t tmem_base;
   volatile uint32_t abort;
-  float2 ml[128];
 };
 static_assert(sizeof(Ctl) <= kSmemCtl, "control block");
 
@@ -181,10 +185,10 @@ __device__ __forceinline__ bool softmax_tile(uint32_t t_s, uint32_t t_o, int c0,
 __global__ void __launch_bounds__(kThreads, 2)
 chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  extern __shared__ __align__(1024) uint8_t smem[];
   uint8_t* q_s = smem;             // Q tile: two halves [128 rows][64 d], 128-byte swizzle
-  uint8_t* st_s = smem + kQBytes;  // K/V slots
+  uint8_t* k_s = smem + kOffK;     // K slots
+  uint8_t* v_s0 = smem + kOffV;    // V slots
   Ctl* ctl = reinterpret_cast<Ctl*>(smem + kSmemData);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -218,7 +222,10 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   float2* out_ml = p.part_ml + slot * p.R_stride + row0;
   float* out_a = p.part_a + (slot * p.R_stride + row0) * kD;
 
-  if (n_tiles == 0) {  // nothing visible here: identity state, no tensor memory taken
+  if (n_tiles == 0 || (smem_u32(smem) & 1023u)) {
+    // nothing visible here (identity state, no tensor memory taken); a misaligned shared
+    // memory window would break the swizzled layouts and is reported instead of run
+    if (n_tiles && tid == 0) atomicOr(p.status, SS_DEV_WAIT_EXPIRED);
     if (tid < nrows) out_ml[tid] = make_float2(-INFINITY, 0.f);
     if (!p.wait_first && chain_cta) pdl_wait_prior();
     return;
@@ -226,30 +233,32 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
 
   // ---- set-up: barriers, first loads, tensor memory, the Q tile --------------------------------
   auto issue_k = [&](int it, uint64_t pol) {
-    const int s = it % kStages;
+    const int s = it % kKStages;
     int outer, tok;
     locate_token(p, b, tok0 + it * kTileKeys, &outer, &tok);
-    const uint32_t kdst = smem_u32(st_s + s * kStageBytes);
+    const uint32_t kdst = smem_u32(k_s + s * kTileBytes);
     mbar_expect_tx(&ctl->kfull[s], kTileBytes);
     tma_load_4d(kdst, &tmK, 0, tok, kvh, outer, &ctl->kfull[s], pol);
     tma_load_4d(kdst + kHalfTile, &tmK, 64, tok, kvh, outer, &ctl->kfull[s], pol);
   };
   auto issue_v = [&](int it, uint64_t pol) {
-    const int s = it % kStages;
+    const int s = it % kVStages;
     int outer, tok;
     locate_token(p, b, tok0 + it * kTileKeys, &outer, &tok);
-    const uint32_t vdst = smem_u32(st_s + s * kStageBytes) + kTileBytes;
+    const uint32_t vdst = smem_u32(v_s0 + s * kTileBytes);
     mbar_expect_tx(&ctl->vfull[s], kTileBytes);
     tma_load_4d(vdst, &tmV, 0, tok, kvh, outer, &ctl->vfull[s], pol);
     tma_load_4d(vdst + kHalfTile, &tmV, 64, tok, kvh, outer, &ctl->vfull[s], pol);
   };
-  const int n_pre = min(n_tiles, kStages);
+  const int n_pre_k = min(n_tiles, kKStages), n_pre_v = min(n_tiles, kVStages);
   if (warp == 4) {
     if (lane == 0) {
-      for (int s = 0; s < kStages; ++s) {
+      for (int s = 0; s < kKStages; ++s) {
         mbar_init(&ctl->kfull[s], 1);
-        mbar_init(&ctl->vfull[s], 1);
         mbar_init(&ctl->kempty[s], 1);
+      }
+      for (int s = 0; s < kVStages; ++s) {
+        mbar_init(&ctl->vfull[s], 1);
         mbar_init(&ctl->vempty[s], 1);
       }
       for (int i = 0; i < 2; ++i) {
@@ -264,8 +273,8 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       // MMAs of both tiles come before the first output MMAs)
       // streamed once: evict first; shared by the row groups of a kv-head through L2: keep
       const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
-      for (int it = 0; it < n_pre; ++it) issue_k(it, pol);
-      for (int it = 0; it < n_pre; ++it) issue_v(it, pol);
+      for (int it = 0; it < n_pre_k; ++it) issue_k(it, pol);
+      for (int it = 0; it < n_pre_v; ++it) issue_v(it, pol);
     }
     __syncwarp();
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
@@ -301,20 +310,18 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     if (lane == 0) {
       // streamed once: evict first; shared by the row groups of a kv-head through L2: keep
       const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
-      // K(j) can go out once QK(j - 2) has retired, V(i) once PV(i - 2) has: in time order
-      // that is K(j) next to V(j - 2)
-      int issued_k = n_pre, issued_v = n_pre;
-      for (int j = n_pre; j < n_tiles + 2; ++j) {
-        if (j < n_tiles) {
-          trace(tr, 0, j, 0);
-          if (!mbar_wait(&ctl->kempty[j % kStages], ((j / kStages) & 1) ^ 1, ctl, p.status)) break;
-          trace(tr, 0, j, 1);
-          issue_k(j, pol);
-          issued_k = j + 1;
-        }
-        const int i = j - 2;
-        if (i >= n_pre && i < n_tiles) {
-          if (!mbar_wait(&ctl->vempty[i % kStages], ((i / kStages) & 1) ^ 1, ctl, p.status)) break;
+      // K(j) can go out once QK(j - 2) has retired, V(i) once PV(i - 3) has; the score MMAs
+      // run two tiles ahead of the output MMAs, so in time order that is K(j) next to V(j + 1)
+      int issued_k = n_pre_k, issued_v = n_pre_v;
+      for (int j = n_pre_k; j < n_tiles; ++j) {
+        trace(tr, 0, j, 0);
+        if (!mbar_wait(&ctl->kempty[j % kKStages], ((j / kKStages) & 1) ^ 1, ctl, p.status)) break;
+        trace(tr, 0, j, 1);
+        issue_k(j, pol);
+        issued_k = j + 1;
+        const int i = j + 1;
+        if (i >= n_pre_v && i < n_tiles) {
+          if (!mbar_wait(&ctl->vempty[i % kVStages], ((i / kVStages) & 1) ^ 1, ctl, p.status)) break;
           trace(tr, 0, i, 2);
           issue_v(i, pol);
           issued_v = i + 1;
@@ -323,13 +330,13 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       if (ctl->abort) {
         // let the copies this thread started land before the CTA leaves (bounded)
         const unsigned long long t0 = gtime_ns();
-        for (int it = max(0, issued_k - kStages); it < issued_k; ++it) {
-          while (!mbar_try_wait(&ctl->kfull[it % kStages], (it / kStages) & 1) &&
+        for (int it = max(0, issued_k - kKStages); it < issued_k; ++it) {
+          while (!mbar_try_wait(&ctl->kfull[it % kKStages], (it / kKStages) & 1) &&
                  gtime_ns() - t0 < kWaitNs) {
           }
         }
-        for (int it = max(0, issued_v - kStages); it < issued_v; ++it) {
-          while (!mbar_try_wait(&ctl->vfull[it % kStages], (it / kStages) & 1) &&
+        for (int it = max(0, issued_v - kVStages); it < issued_v; ++it) {
+          while (!mbar_try_wait(&ctl->vfull[it % kVStages], (it / kVStages) & 1) &&
                  gtime_ns() - t0 < kWaitNs) {
           }
         }
@@ -341,11 +348,11 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     constexpr uint32_t idesc_qk = make_idesc(128, kTileKeys, false);
     constexpr uint32_t idesc_pv = make_idesc(128, kD, true);
     const bool leader = elect_one();
-    const uint32_t st_addr = smem_u32(st_s), q_addr = smem_u32(q_s);
+    const uint32_t k_base = smem_u32(k_s), v_base = smem_u32(v_s0), q_addr = smem_u32(q_s);
     // S[it % 2] = Q K_it^T; releases the K slot and signals the softmax warps
     auto issue_qk = [&](int it) {
-      const int s = it % kStages;
-      const uint32_t k_addr = st_addr + s * kStageBytes;
+      const int s = it % kKStages;
+      const uint32_t k_addr = k_base + s * kTileBytes;
       if (leader) {
 #pragma unroll
         for (int kk = 0; kk < kD / 16; ++kk) {
@@ -361,15 +368,16 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     };
     // the Q tile was written before the CTA-wide barrier above (with a proxy fence)
     bool ok = true;
-    for (int it = 0; ok && it < n_pre; ++it) {
+    for (int it = 0; ok && it < n_pre_k; ++it) {  // one per score buffer (= per K slot)
       ok = mbar_wait(&ctl->kfull[it], 0, ctl, p.status);
       if (!ok) break;
       tc_fence_after();
       issue_qk(it);
     }
+    static_assert(kKStages == 2, "the score MMAs of tile t + 2 reuse the K slot and the S buffer of tile t");
     for (int it = 0; ok && it < n_tiles; ++it) {
-      const int s = it % kStages;
-      const uint32_t ph = (it / kStages) & 1;
+      const int s = it % kVStages;
+      const uint32_t ph = (it / kVStages) & 1;
       trace(trl, 1, it, 0);
       ok = mbar_wait(&ctl->pready[it & 1], (it >> 1) & 1, ctl, p.status);
       trace(trl, 1, it, 1);
@@ -377,7 +385,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       if (!ok) break;
       trace(trl, 1, it, 2);
       tc_fence_after();
-      const uint32_t v_addr = st_addr + s * kStageBytes + kTileBytes;
+      const uint32_t v_addr = v_base + s * kTileBytes;
       if (leader) {
 #pragma unroll
         for (int kk = 0; kk < kTileKeys / 16; ++kk) {
@@ -393,7 +401,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       if (it + 2 < n_tiles) {
         // overwrites the score buffer P(it) was read from: the tensor pipe runs this thread's
         // MMAs in issue order, so the P V products above have consumed P before these write S
-        ok = mbar_wait(&ctl->kfull[s], ph ^ 1, ctl, p.status);
+        ok = mbar_wait(&ctl->kfull[it & 1], (((it + 2) / kKStages) & 1), ctl, p.status);
         if (!ok) break;
         trace(trl, 1, it, 4);
         tc_fence_after();
@@ -413,8 +421,8 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     float m = -INFINITY, l = 0.f;
     bool ok = true;
     for (int it = 0; it < n_tiles; ++it) {
-      const int s = it % kStages;
-      const uint32_t ph = (it / kStages) & 1;
+      const int s = it % kVStages;
+      const uint32_t ph = (it / kVStages) & 1;
       const uint32_t t_s = tmem + lane_off + kColS + (it & 1) * 64;
       if (L == 0) trace(tr, 2, it, 0);
       ok = mbar_wait(&ctl->sfull[it & 1], (it >> 1) & 1, ctl, p.status);
@@ -427,7 +435,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         // be finite: clear those rows of the staged V tile (whole 128-byte rows, both halves)
         ok = mbar_wait(&ctl->vfull[s], ph, ctl, p.status);
         if (!ok) break;
-        uint8_t* v_s = st_s + s * kStageBytes + kTileBytes;
+        uint8_t* v_s = v_s0 + s * kTileBytes;
         const int n_vec = (kTileKeys - n_valid) * 16;
         for (int i = L; i < n_vec; i += 128) {
           const int row = n_valid + (i >> 4), half = (i >> 3) & 1, ch = i & 7;
@@ -466,11 +474,15 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     if (ctl->abort == 0) {  // uniform over the 128 threads after the barrier
       tc_fence_after();
       // ---- merge the key groups of each row and write the partial state ----
-      float* o_s = reinterpret_cast<float*>(smem);  // [128][128] fp32 over the Q tile and the slots
-      ctl->ml[L] = make_float2(m, l);
+      // everything below lives over the idle Q tile and K/V slots: O as [128][128] fp32 over
+      // the first 64 KB (Q and the K slots), the lanes' (m, l) at the start of the V slots
+      float* o_s = reinterpret_cast<float*>(smem);
+      float2* ml_s = reinterpret_cast<float2*>(v_s0);
+      static_assert(kOffV >= 128 * 128 * 4, "O staging must end before the (m, l) array");
+      ml_s[L] = make_float2(m, l);
       named_bar_sync(1, 128);
       float M = -INFINITY;
-      for (int g = 0; g < groups; ++g) M = fmaxf(M, ctl->ml[g * r_pad + r].x);
+      for (int g = 0; g < groups; ++g) M = fmaxf(M, ml_s[g * r_pad + r].x);
       const float f = (m == -INFINITY) ? 0.f : exp2f(m - M);
 #pragma unroll 1
       for (int q = 0; q < kD / 16; ++q) {
@@ -490,7 +502,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       if (L < nrows) {
         float lt = 0.f;
         for (int g = 0; g < groups; ++g) {
-          const float2 st = ctl->ml[g * r_pad + r];
+          const float2 st = ml_s[g * r_pad + r];
           if (st.x > -INFINITY) lt += exp2f(st.x - M) * st.y;
         }
         out_ml[L] = make_float2(lt > 0.f ? M : -INFINITY, lt);
