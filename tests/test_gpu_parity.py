@@ -91,6 +91,15 @@ def test_peaked_softmax(k_mult, flags):
     _run(cfg, flags=flags)
 
 
+@pytest.mark.parametrize("flags", [0, 1, 4, 8])
+@pytest.mark.parametrize("T_q", [8, 20])
+def test_one_hot_softmax_large_scores(flags, T_q):
+    # K x 32: scaled scores of several hundred, the softmax is one-hot up to ties and the
+    # reference maximum jumps by far more than the lazy-rescale thresholds on most tiles
+    cfg = inputs.VerifyConfig("v", 0x2222 + T_q, 2, 8, 2, 128, 192, T_q, 300, 1000, k_mult=32.0)
+    _run(cfg, flags=flags)
+
+
 def test_needle_keys_and_rescale_path():
     # one key per request with a score ~ +20 above the rest, placed late in the history, so the
     # running maximum jumps by more than the rescale threshold after many tiles
