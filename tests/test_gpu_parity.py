@@ -100,6 +100,74 @@ def test_one_hot_softmax_large_scores(flags, T_q):
     _run(cfg, flags=flags)
 
 
+@pytest.mark.parametrize("flags", [0, 1, 4])
+def test_equal_keys_closed_form_without_the_oracle(flags):
+    # every history key and every local key of a kv-head equals one vector k: the softmax is
+    # uniform over the visible keys, so O_i = mean of the visible V rows and
+    # LSE_i = scale * q_i . k + ln(n_vis(i)) with n_vis(i) = len_b + i + 1 (inclusive chain mask)
+    cfg = inputs.VerifyConfig("v", 0x3131, 3, 8, 2, 128, 192, 6, 0, 700)
+    lens = [0, 385, 700]
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV, fill=0.0)
+    kvec = K_loc[:, :, :1, :].clone()                       # [B, H_kv, 1, d]
+    K_loc.copy_(kvec.expand_as(K_loc))
+    for K, V, vl in chunks:
+        K.copy_(kvec.expand_as(K))
+    ctx = util.make_ctx(cfg, flags=flags)
+    O, LSE = util.gpu_case(ctx, cfg, Q, chunks, K_loc, V_loc, bits)
+    ctx.close()
+    G = cfg.G
+    for b in range(cfg.B):
+        for h in range(cfg.H_q):
+            kvh = h // G
+            vh = np.concatenate([util.f64(V[b, kvh, :int(vl[b])]) for K, V, vl in chunks] + [np.zeros((0, cfg.d))])
+            assert vh.shape[0] == lens[b]
+            for i in range(cfg.T_q):
+                vis = np.concatenate([vh, util.f64(V_loc[b, kvh, :i + 1])])
+                want_o = vis.mean(axis=0)
+                want_lse = cfg.scale * float(util.f64(Q[b, h, i]) @ util.f64(kvec[b, kvh, 0])) + np.log(len(vis))
+                got = util.f64(O[b, h, i])
+                assert np.abs(got - want_o).max() <= 2.0 ** -7 * (np.abs(want_o).max() + 1e-3), (b, h, i)
+                assert abs(float(LSE[b, h, i]) - want_lse) <= 1e-3, (b, h, i)
+
+
+@pytest.mark.parametrize("flags", [0, 1])
+def test_single_visible_key_returns_its_value_bit_exact(flags):
+    # no history, chain mask: row 0 sees local key 0 only, so O = V_0 exactly (the weight is
+    # exp2(0) = 1, the row sum 1) and LSE = scale * q . k_0
+    cfg = inputs.VerifyConfig("v", 0x3232, 2, 8, 2, 128, 64, 5, 0, 0)
+    lens = [0, 0]
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    ctx = util.make_ctx(cfg, flags=flags)
+    O, LSE = util.gpu_case(ctx, cfg, Q, chunks, K_loc, V_loc, bits)
+    ctx.close()
+    for h in range(cfg.H_q):
+        kvh = h // cfg.G
+        assert torch.equal(O[:, h, 0].view(torch.int16), V_loc[:, kvh, 0].view(torch.int16))
+        want = cfg.scale * (util.f64(Q[:, h, 0]) * util.f64(K_loc[:, kvh, 0])).sum(axis=1)
+        assert np.abs(util.f64(LSE[:, h, 0]) - want).max() <= 1e-4
+
+
+@pytest.mark.parametrize("flags", [0, 4])
+def test_later_candidates_do_not_change_earlier_rows(flags):
+    # causality of the chain mask: rewriting local K/V at positions j > i leaves row i
+    # bit-identical (the kernels are deterministic)
+    cfg = inputs.VerifyConfig("v", 0x3333, 2, 8, 2, 128, 128, 8, 200, 500)
+    lens = inputs.history_lengths(cfg)
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    ctx = util.make_ctx(cfg, flags=flags)
+    O1, L1 = util.gpu_case(ctx, cfg, Q, chunks, K_loc, V_loc, bits)
+    O1, L1 = O1.clone(), L1.clone()
+    i = 3
+    K2, V2 = K_loc.clone(), V_loc.clone()
+    K2[:, :, i + 1:] = -K2[:, :, i + 1:] * 3
+    V2[:, :, i + 1:] = V2[:, :, i + 1:] + 5
+    O2, L2 = util.gpu_case(ctx, cfg, Q, chunks, K2, V2, bits)
+    ctx.close()
+    assert torch.equal(O1[:, :, :i + 1].view(torch.int16), O2[:, :, :i + 1].view(torch.int16))
+    assert torch.equal(L1[:, :, :i + 1], L2[:, :, :i + 1])
+    assert not torch.equal(O1[:, :, i + 1:], O2[:, :, i + 1:])
+
+
 def test_needle_keys_and_rescale_path():
     # one key per request with a score ~ +20 above the rest, placed late in the history, so the
     # running maximum jumps by more than the rescale threshold after many tiles
