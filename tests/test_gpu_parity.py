@@ -168,6 +168,54 @@ def test_later_candidates_do_not_change_earlier_rows(flags):
     assert not torch.equal(O1[:, :, i + 1:], O2[:, :, i + 1:])
 
 
+def test_tree_row_equals_chain_over_its_root_path():
+    # a tree node sees the history and its ancestors-or-self: row i of a tree round equals the
+    # LAST row of a chain round whose candidates are the path root -> i (other subtrees are
+    # invisible to it)
+    import dataclasses
+    cfg = inputs.VerifyConfig("v", 0x3434, 1, 8, 2, 128, 128, 24, 300, 300, mask="tree", k_mult=2.0)
+    lens = [300]
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    ctx = util.make_ctx(cfg)
+    O_t, L_t = util.gpu_case(ctx, cfg, Q, chunks, K_loc, V_loc, bits)
+    ctx.close()
+    vis = inputs.mask_bits_to_bool(bits, cfg.T_q)[0]          # [T_q, T_loc]
+    for i in (0, 7, 23):
+        path = [j for j in range(cfg.T_q) if bool(vis[i, j])]
+        assert path[-1] == i and path[0] == 0
+        ccfg = dataclasses.replace(cfg, T_q=len(path), mask="chain")
+        idx = torch.tensor(path, device=DEV)
+        Qc = Q[:, :, idx].contiguous()
+        Kc, Vc = K_loc[:, :, idx].contiguous(), V_loc[:, :, idx].contiguous()
+        cctx = util.make_ctx(ccfg)
+        O_c, L_c = util.gpu_case(cctx, ccfg, Qc, chunks, Kc, Vc, inputs.make_mask_bits(ccfg, DEV))
+        cctx.close()
+        d = (O_t[:, :, i].float() - O_c[:, :, -1].float()).abs().max().item()
+        assert d <= 2.0 ** -7 * max(1.0, O_t[:, :, i].float().abs().max().item()), (i, d)
+        assert (L_t[:, :, i] - L_c[:, :, -1]).abs().max().item() <= 1e-4, i
+
+
+def test_gqa_equals_mha_with_replicated_kv_heads():
+    # consecutive query heads share a kv-head: replicating every kv-head G times and running
+    # with H_kv = H_q gives the same result
+    import dataclasses
+    cfg = inputs.VerifyConfig("v", 0x3535, 2, 8, 2, 128, 128, 6, 200, 450, k_mult=2.0)
+    lens = inputs.history_lengths(cfg)
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    ctx = util.make_ctx(cfg)
+    O_g, L_g = util.gpu_case(ctx, cfg, Q, chunks, K_loc, V_loc, bits)
+    ctx.close()
+    G = cfg.G
+    rep = lambda t: t.repeat_interleave(G, dim=1).contiguous()
+    mcfg = dataclasses.replace(cfg, H_kv=cfg.H_q)
+    mchunks = [(rep(K), rep(V), vl) for K, V, vl in chunks]
+    mctx = util.make_ctx(mcfg)
+    O_m, L_m = util.gpu_case(mctx, mcfg, Q, mchunks, rep(K_loc), rep(V_loc), bits)
+    mctx.close()
+    assert (O_g.float() - O_m.float()).abs().max().item() <= 2.0 ** -7 * max(1.0, O_g.float().abs().max().item())
+    assert (L_g - L_m).abs().max().item() <= 1e-4
+
+
 def test_needle_keys_and_rescale_path():
     # one key per request with a score ~ +20 above the rest, placed late in the history, so the
     # running maximum jumps by more than the rescale threshold after many tiles
