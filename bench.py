@@ -557,8 +557,9 @@ def main():
             # N layers sharing this layer's host history (same lengths); one descriptor each
             descs = [make_stream_desc(ssb, cfg, lens, host, dev, Qd, Kld, Vld, bits, O, LSE, bufs)
                      for _ in range(args.layers)]
-            rk = torch.empty(cfg.B, cfg.H_kv, n_chunk_calls * cfg.L_c, cfg.d, dtype=torch.bfloat16, device=dev)
-            rv = torch.empty_like(rk)
+            # restore buffer in the same fused K|V layout as the staging slots (one copy per block)
+            rk = torch.empty(cfg.B, 2, cfg.H_kv, n_chunk_calls * cfg.L_c, cfg.d, dtype=torch.bfloat16, device=dev)
+            rv = None
             abl = {}
             for name, mode in (("stream_prefetch", ssb.SS_LAYERS_PREFETCH), ("stream_layerwise", ssb.SS_LAYERS_STREAM),
                                ("restore_then_verify", ssb.SS_LAYERS_RESTORE)):
@@ -569,7 +570,7 @@ def main():
             abl["prefetch_vs_layerwise"] = abl["stream_layerwise_ms"] / abl["stream_prefetch_ms"]
             abl["stream_vs_restore"] = abl["restore_then_verify_ms"] / abl["stream_layerwise_ms"]
             e2e["layers_ablation"] = abl
-            del rk, rv
+            del rk
         del host
 
     cpu = None

@@ -261,7 +261,9 @@ ss_status ss_stream_round(ss_ctx* ctx, const ss_stream_desc* desc, ss_stream_sta
  *                       previous layer's work is done;
  *   SS_LAYERS_RESTORE   restore-then-verify baseline: the whole history of a layer is copied into
  *                       restore_k / restore_v (device, [B, H_kv, restore_tokens, d]) and only then
- *                       attended to; layers run strictly one after the other.
+ *                       attended to; layers run strictly one after the other.  With restore_v
+ *                       NULL, restore_k is one buffer [B][2 (K,V)][H_kv][restore_tokens][d]
+ *                       and every (request, chunk) block is restored with one copy.
  * Every layer has its own descriptor (history, Q, local KV, outputs); all layers use the same
  * B, T_q, L_c, batch_chunks and staging buffers.  Layers may share the valid_len scratch arrays
  * only if their history lengths are identical.  Synchronous; `total` covers all layers. */
@@ -344,7 +346,7 @@ typedef struct {
   const ss_stream_desc* layers; /* HOST array [n_layers]                                   */
   int32_t mode;                /* ss_layers_mode                                           */
   void* restore_k;             /* device; SS_LAYERS_RESTORE only                           */
-  void* restore_v;
+  void* restore_v;             /* NULL: restore_k holds K and V (see above)                */
   int64_t restore_tokens;      /* token capacity of a restore buffer row                   */
 } ss_layers_desc;
 ss_status ss_stream_layers(ss_ctx* ctx, const ss_layers_desc* layers, ss_stream_stats* total);

@@ -379,10 +379,11 @@ class Context:
         return [[[buf[(r * 32 + t) * 8 + e] for e in range(8)] for t in range(32)] for r in range(3)][:3] if got else None
 
     def ss_stream_layers(self, descs, mode: int = SS_LAYERS_PREFETCH, restore_k=None, restore_v=None) -> ss_stream_stats:
-        """descs: list of ss_stream_desc, one per layer."""
+        """descs: list of ss_stream_desc, one per layer.  restore_k [B, H_kv, tokens, d] with
+        restore_v of the same shape, or restore_k [B, 2, H_kv, tokens, d] alone (K and V fused)."""
         arr = (ss_stream_desc * len(descs))(*descs)
         ld = ss_layers_desc(len(descs), arr, mode, _ptr(restore_k), _ptr(restore_v),
-                            restore_k.shape[2] if restore_k is not None else 0)
+                            restore_k.shape[-2] if restore_k is not None else 0)
         stats = ss_stream_stats()
         self._check(self.lib.ss_stream_layers(self.handle, C.byref(ld), C.byref(stats)), "ss_stream_layers")
         return stats

@@ -74,7 +74,9 @@ ss_status enqueue_layer(ss_ctx* ctx, const ss_stream_desc* d, const ss::PipeRes&
   ss::ctx_dims(ctx, &H_q, &H_kv, &hd);
   const int B = d->B, L_c = d->L_c, bc = d->batch_chunks;
   const bool restore = restore_k != nullptr;
-  const bool fused = d->stage_fused && !restore;  // K and V of a block in one staging buffer
+  // K and V of a block next to each other in one device buffer ([B][K|V][H_kv][Ls][d]): the
+  // staging slots with stage_fused, the restore buffer when restore_v is null
+  const bool fused = restore ? restore_v == nullptr : d->stage_fused != 0;
   const int64_t Ls = restore ? restore_tokens : (int64_t)bc * L_c;  // tokens per device buffer row
   if (restore && (int64_t)n_fills * bc * L_c > restore_tokens) return SS_ERR_CAPACITY;
 
@@ -111,7 +113,9 @@ ss_status enqueue_layer(ss_ctx* ctx, const ss_stream_desc* d, const ss::PipeRes&
         const uint16_t* src = (const uint16_t*)d->hist[b] + (int64_t)j * block_elems;
         if (fused) {
           // K and V of the block in one copy: the staging buffer keeps the host block's order
-          uint16_t* dst = (uint16_t*)d->stage_k[buf] + ((int64_t)b * 2 * H_kv * Ls + (int64_t)jj * L_c) * hd;
+          uint16_t* dst = (restore ? (uint16_t*)restore_k + (int64_t)j * L_c * hd
+                                   : (uint16_t*)d->stage_k[buf] + (int64_t)jj * L_c * hd) +
+                          (int64_t)b * 2 * H_kv * Ls * hd;
           if (v == L_c && Ls == L_c) {
             SS_CK(cudaMemcpyAsync(dst, src, (size_t)block_elems * esz, cudaMemcpyHostToDevice,
                                   r.copy_stream));
@@ -169,6 +173,10 @@ ss_status enqueue_layer(ss_ctx* ctx, const ss_stream_desc* d, const ss::PipeRes&
       const int64_t tok = (int64_t)f * bc * L_c;
       ss_tensor K = {(uint16_t*)restore_k + tok * hd, (int64_t)H_kv * Ls * hd, Ls * hd, hd};
       ss_tensor V = {(uint16_t*)restore_v + tok * hd, (int64_t)H_kv * Ls * hd, Ls * hd, hd};
+      if (fused) {
+        K.stride_b = V.stride_b = 2 * (int64_t)H_kv * Ls * hd;
+        V.ptr = (const uint16_t*)restore_k + (int64_t)H_kv * Ls * hd + tok * hd;
+      }
       SS_ST(ss_verify_chunk_hinted(ctx, K, V, bc * L_c, d->valid_len_dev + (int64_t)f * B,
                                    d->valid_len_host + (int64_t)f * B, r.attn_stream));
       ++cnt->calls;
@@ -241,7 +249,7 @@ ss_status stream_round_impl(ss_ctx* ctx, const ss_stream_desc* d, ss_stream_stat
 ss_status stream_layers_impl(ss_ctx* ctx, const ss_layers_desc* ld, ss_stream_stats* total) {
   if (!ld || !ld->layers || ld->n_layers <= 0) return SS_ERR_ARG;
   if (ld->mode < SS_LAYERS_PREFETCH || ld->mode > SS_LAYERS_RESTORE) return SS_ERR_ARG;
-  if (ld->mode == SS_LAYERS_RESTORE && (!ld->restore_k || !ld->restore_v || ld->restore_tokens <= 0))
+  if (ld->mode == SS_LAYERS_RESTORE && (!ld->restore_k || ld->restore_tokens <= 0))
     return SS_ERR_ARG;
   if (ld->n_layers > 256) return SS_ERR_SHAPE;
   ss::PipeRes r;

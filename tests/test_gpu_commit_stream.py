@@ -282,7 +282,8 @@ def _layer_descs(ssb, cfg, lens, n_layers, bufs):
     return layers
 
 
-def test_stream_layers_modes_match_oracle_and_each_other():
+@pytest.mark.parametrize("fused_restore", [False, True])
+def test_stream_layers_modes_match_oracle_and_each_other(fused_restore):
     ssb = _ssb()
     cfg = inputs.VerifyConfig("v", 0x66, 3, 8, 2, 128, 256, 8, 200, 1300)
     lens = [1300, 200, 777]
@@ -290,8 +291,13 @@ def test_stream_layers_modes_match_oracle_and_each_other():
     bufs = bench.stream_buffers(cfg, DEV, n_chunks)
     layers = _layer_descs(ssb, cfg, lens, 3, bufs)
     ctx = ssb.Context(cfg.B, cfg.H_q, cfg.H_kv, cfg.d, cfg.T_q, cfg.T_q, cfg.L_c)
-    rk = torch.full((cfg.B, cfg.H_kv, n_chunks * cfg.L_c, cfg.d), float("nan"), dtype=torch.bfloat16, device=DEV)
-    rv = torch.full_like(rk, float("nan"))
+    if fused_restore:   # K and V of a request next to each other in one buffer
+        rk = torch.full((cfg.B, 2, cfg.H_kv, n_chunks * cfg.L_c, cfg.d), float("nan"), dtype=torch.bfloat16,
+                        device=DEV)
+        rv = None
+    else:
+        rk = torch.full((cfg.B, cfg.H_kv, n_chunks * cfg.L_c, cfg.d), float("nan"), dtype=torch.bfloat16, device=DEV)
+        rv = torch.full_like(rk, float("nan"))
     outs = {}
     for mode in (ssb.SS_LAYERS_PREFETCH, ssb.SS_LAYERS_STREAM, ssb.SS_LAYERS_RESTORE):
         for L in layers:
