@@ -26,30 +26,13 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const ChunkParams 
   __shared__ float m_s[kRows], l_s[kRows], corr_s[kRows];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int rt = blockIdx.x % p.row_tiles;
-  const int split = blockIdx.x / p.row_tiles;
-  const int kvh = blockIdx.y, b = blockIdx.z;
-  const int row0 = rt * kRows;
-  const int nrows = min(kRows, p.R - row0);
-
-  const bool chain_cta = (blockIdx.x | blockIdx.y | blockIdx.z) == 0;
   if (p.wait_first) pdl_wait_prior();
   pdl_launch_dependents();
-
-  int valid = p.L_c;
-  if (p.valid_len) {
-    valid = p.valid_len[b];
-    if (valid < 0 || valid > p.L_c) {
-      if (tid == 0) atomicOr(p.status, SS_DEV_BAD_VALID_LEN);
-      valid = max(0, min(valid, p.L_c));
-    }
-  }
-  const int tok0 = split * p.tiles_per_split * kKeys;
-  const int tok1 = min(valid, tok0 + p.tiles_per_split * kKeys);
-
-  const size_t slot = ((size_t)split * p.B + b) * p.H_kv + kvh;
-  float2* out_ml = p.part_ml + slot * p.R_stride + row0;
-  float* out_a = p.part_a + (slot * p.R_stride + row0) * D;
+  const ChunkWork w = chunk_work(p, kRows);
+  const int b = w.b, kvh = w.kvh, row0 = w.row0, nrows = w.nrows, tok0 = w.tok0, tok1 = w.tok1;
+  const bool chain_cta = w.chain_cta;
+  float2* out_ml = w.out_ml;
+  float* out_a = w.out_a;
 
   if (tok0 >= tok1) {  // nothing visible here: identity state
     if (tid < nrows) out_ml[tid] = make_float2(-INFINITY, 0.f);

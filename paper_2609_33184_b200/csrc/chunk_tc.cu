@@ -192,35 +192,18 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   Ctl* ctl = reinterpret_cast<Ctl*>(smem + kSmemData);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int rt = blockIdx.x % p.row_tiles;
-  const int split = blockIdx.x / p.row_tiles;
-  const int kvh = blockIdx.y, b = blockIdx.z;
-  const int row0 = rt * p.rows_per_tile;
-  const int nrows = min(p.rows_per_tile, p.R - row0);
+  if (p.wait_first) pdl_wait_prior();
+  pdl_launch_dependents();
+  const ChunkWork w = chunk_work(p, p.rows_per_tile);
+  const int b = w.b, kvh = w.kvh, row0 = w.row0, nrows = w.nrows, tok0 = w.tok0, tok1 = w.tok1;
+  const bool chain_cta = w.chain_cta;
+  float2* out_ml = w.out_ml;
+  float* out_a = w.out_a;
   // key groups sharing the 128 lanes: the Q rows are replicated when the tile has few rows
   const int groups = nrows <= 32 ? 4 : (nrows <= 64 ? 2 : 1);
   const int r_pad = 128 / groups;
-  unsigned long long* tr = (blockIdx.x | blockIdx.y | blockIdx.z) ? nullptr : p.trace;
-
-  const bool chain_cta = (blockIdx.x | blockIdx.y | blockIdx.z) == 0;
-  if (p.wait_first) pdl_wait_prior();
-  pdl_launch_dependents();
-
-  int valid = p.L_c;
-  if (p.valid_len) {
-    valid = p.valid_len[b];
-    if (valid < 0 || valid > p.L_c) {
-      if (tid == 0) atomicOr(p.status, SS_DEV_BAD_VALID_LEN);
-      valid = max(0, min(valid, p.L_c));
-    }
-  }
-  const int tok0 = split * p.tiles_per_split * kTileKeys;
-  const int tok1 = min(valid, tok0 + p.tiles_per_split * kTileKeys);
+  unsigned long long* tr = chain_cta ? p.trace : nullptr;
   const int n_tiles = (tok1 > tok0) ? (tok1 - tok0 + kTileKeys - 1) / kTileKeys : 0;
-
-  const size_t slot = ((size_t)split * p.B + b) * p.H_kv + kvh;
-  float2* out_ml = p.part_ml + slot * p.R_stride + row0;
-  float* out_a = p.part_a + (slot * p.R_stride + row0) * kD;
 
   if (n_tiles == 0 || (smem_u32(smem) & 1023u)) {
     // nothing visible here (identity state, no tensor memory taken); a misaligned shared

@@ -100,34 +100,17 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
   uint8_t* p_s = smem + C::kOffP;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int rt = blockIdx.x % p.row_tiles;
-  const int split = blockIdx.x / p.row_tiles;
-  const int kvh = blockIdx.y, b = blockIdx.z;
-  const int row0 = rt * p.rows_per_tile;
-  const int nrows = min(p.rows_per_tile, p.R - row0);  // <= N
-  const int n_mma = (nrows + 15) & ~15;                 // MMA N of this CTA
-  unsigned long long* tr = (blockIdx.x | blockIdx.y | blockIdx.z) ? nullptr : p.trace;
-
-  const bool chain_cta = (blockIdx.x | blockIdx.y | blockIdx.z) == 0;
   if (p.wait_first) pdl_wait_prior();
   pdl_launch_dependents();
-
-  int valid = p.L_c;
-  if (p.valid_len) {
-    valid = p.valid_len[b];
-    if (valid < 0 || valid > p.L_c) {
-      if (tid == 0) atomicOr(p.status, SS_DEV_BAD_VALID_LEN);
-      valid = max(0, min(valid, p.L_c));
-    }
-  }
+  const ChunkWork w = chunk_work(p, p.rows_per_tile);
+  const int b = w.b, kvh = w.kvh, row0 = w.row0, nrows = w.nrows, tok0 = w.tok0, tok1 = w.tok1;  // nrows <= N
+  const bool chain_cta = w.chain_cta;
+  float2* out_ml = w.out_ml;
+  float* out_a = w.out_a;
+  const int n_mma = (nrows + 15) & ~15;                 // MMA N of this CTA
+  unsigned long long* tr = chain_cta ? p.trace : nullptr;
   // splits are given in 64-token tiles by the host; this kernel walks 128-token tiles
-  const int tok0 = split * p.tiles_per_split * kTileKeys;
-  const int tok1 = min(valid, tok0 + p.tiles_per_split * kTileKeys);
   const int n_tiles = (tok1 > tok0) ? (tok1 - tok0 + kKeys - 1) / kKeys : 0;
-
-  const size_t slot = ((size_t)split * p.B + b) * p.H_kv + kvh;
-  float2* out_ml = p.part_ml + slot * p.R_stride + row0;
-  float* out_a = p.part_a + (slot * p.R_stride + row0) * kD;
 
   if (n_tiles == 0 || (smem_u32(smem) & 1023u)) {
     // nothing visible here (identity state, no tensor memory taken); a misaligned shared

@@ -138,6 +138,42 @@ __device__ __forceinline__ void pdl_wait_prior() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+// What one CTA of a chunk kernel owns: a tile of query rows of one (request, kv-head) and a
+// range of the chunk's tokens (its token split), plus where its partial state goes.  Shared
+// by the three chunk kernels; `tile_rows` is the kernel's rows per row tile.
+struct ChunkWork {
+  int b, kvh, split;
+  int row0, nrows;      // query rows [row0, row0 + nrows) of the kv-head
+  int tok0, tok1;       // visible tokens [tok0, tok1) of the chunk (tok1 <= tok0: nothing to do)
+  float2* out_ml;       // partial state of the CTA's rows
+  float* out_a;
+  bool chain_cta;       // the one CTA of the grid that keeps the completion order (see below)
+};
+__device__ __forceinline__ ChunkWork chunk_work(const ChunkParams& p, int tile_rows) {
+  ChunkWork w;
+  const int rt = blockIdx.x % p.row_tiles;
+  w.split = blockIdx.x / p.row_tiles;
+  w.kvh = blockIdx.y;
+  w.b = blockIdx.z;
+  w.row0 = rt * tile_rows;
+  w.nrows = min(tile_rows, p.R - w.row0);
+  w.chain_cta = (blockIdx.x | blockIdx.y | blockIdx.z) == 0;
+  int valid = p.L_c;
+  if (p.valid_len) {
+    valid = p.valid_len[w.b];
+    if (valid < 0 || valid > p.L_c) {  // flagged and clamped, never trusted
+      if (threadIdx.x == 0) atomicOr(p.status, SS_DEV_BAD_VALID_LEN);
+      valid = max(0, min(valid, p.L_c));
+    }
+  }
+  w.tok0 = w.split * p.tiles_per_split * kTileKeys;
+  w.tok1 = min(valid, w.tok0 + p.tiles_per_split * kTileKeys);
+  const size_t slot = ((size_t)w.split * p.B + w.b) * p.H_kv + w.kvh;
+  w.out_ml = p.part_ml + slot * p.R_stride + w.row0;
+  w.out_a = p.part_a + (slot * p.R_stride + w.row0) * p.d;
+  return w;
+}
+
 // Where token `tok` of request b lives: (index along the tensor's outermost axis, token within
 // it).  Contiguous chunks: (b, tok).  Paged chunks: (page id, offset); a page id outside the pool
 // raises SS_DEV_BAD_PAGE and maps to index n_pages, which loads read as zeros.
