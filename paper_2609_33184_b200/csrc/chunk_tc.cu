@@ -73,11 +73,6 @@ struct Ctl {
 };
 static_assert(sizeof(Ctl) <= kSmemCtl, "control block");
 
-// Optional trace: CTA (0,0,0) stamps clock64 at fixed points of each role's tile loop.
-// role 0 = TMA producer, 1 = MMA issuer, 2 = softmax thread 0.
-__device__ __forceinline__ void trace(unsigned long long* tr, int role, int it, int ev) {
-  if (tr && it < kTraceTiles) tr[(role * kTraceTiles + it) * 8 + ev] = clock64();
-}
 
 using namespace ss::tc;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Ctl* ctl, uint32_t* status) {

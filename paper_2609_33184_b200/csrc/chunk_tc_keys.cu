@@ -84,9 +84,6 @@ struct Cfg {
   static_assert(NC % 16 == 0 && UNITS <= 8, "shape");
 };
 
-__device__ __forceinline__ void trace(unsigned long long* tr, int role, int it, int ev) {
-  if (tr && it < kTraceTiles) tr[(role * kTraceTiles + it) * 8 + ev] = clock64();
-}
 
 template <int NC, int WG, int UNITS>
 __global__ void __launch_bounds__(Cfg<NC, WG, UNITS>::kThreads, Cfg<NC, WG, UNITS>::kMinBlocks)

@@ -138,6 +138,12 @@ __device__ __forceinline__ void pdl_wait_prior() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+// Optional trace of the tensor-core chunk kernels: CTA (0,0,0) stamps clock64 at fixed points
+// of each role's tile loop.  role 0 = TMA producer, 1 = MMA issuer, 2 = softmax thread 0.
+__device__ __forceinline__ void trace(unsigned long long* tr, int role, int it, int ev) {
+  if (tr && it < kTraceTiles) tr[(role * kTraceTiles + it) * 8 + ev] = clock64();
+}
+
 // What one CTA of a chunk kernel owns: a tile of query rows of one (request, kv-head) and a
 // range of the chunk's tokens (its token split), plus where its partial state goes.  Shared
 // by the three chunk kernels; `tile_rows` is the kernel's rows per row tile.
