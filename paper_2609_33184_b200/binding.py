@@ -486,3 +486,60 @@ class Tier:
         if self.handle:
             self.lib.ss_tier_destroy(self.handle)
             self.handle = C.c_void_p()
+
+
+class WidthController:
+    """Owns an ss_width: the I/O-aware choice of the verification width q (Section 4.2)."""
+
+    def __init__(self, widths: Sequence[int], sample_rounds: int = 2, switch_threshold: float = 0.05,
+                 ema: float = 0.5):
+        self.lib = load()
+        cfg = ss_width_config(len(widths), (C.c_int32 * 8)(*widths), sample_rounds, switch_threshold, ema)
+        self.handle = C.c_void_p()
+        st = self.lib.ss_width_create(C.byref(self.handle), C.byref(cfg))
+        if st != SS_OK:
+            raise SpecStreamError(st, "ss_width_create")
+
+    def observe(self, q: int, t_draft: float, t_transfer: float, t_compute: float, t_other: float,
+                committed: int) -> None:
+        obs = ss_width_obs(t_draft, t_transfer, t_compute, t_other, committed)
+        st = self.lib.ss_width_observe(self.handle, q, C.byref(obs))
+        if st != SS_OK:
+            raise SpecStreamError(st, "ss_width_observe")
+
+    def next(self) -> int:
+        return int(self.lib.ss_width_next(self.handle))
+
+    def estimate(self, q: int):
+        """(T_round, committed, cost = T_round / committed, observations) of width q."""
+        t, u, c, n = C.c_double(), C.c_double(), C.c_double(), C.c_int32()
+        st = self.lib.ss_width_estimate(self.handle, q, C.byref(t), C.byref(u), C.byref(c), C.byref(n))
+        if st != SS_OK:
+            raise SpecStreamError(st, "ss_width_estimate")
+        return t.value, u.value, c.value, n.value
+
+    def close(self):
+        if self.handle:
+            self.lib.ss_width_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def cohort_build(tasks: Sequence[dict], max_batch: int):
+    """Group the tasks of a scheduled batch into cohorts (ss_cohort_build).  Each task is a dict
+    with layer, width, dtype, n_kv, d_h, chunk_size, hist_len; returns a list of lists of task
+    indices, cohort by cohort, longest history first inside a cohort."""
+    n = len(tasks)
+    arr = (ss_task * max(1, n))(*[ss_task(t["layer"], t["width"], t["dtype"], t["n_kv"], t["d_h"],
+                                         t["chunk_size"], i, t["hist_len"]) for i, t in enumerate(tasks)])
+    order = (C.c_int32 * max(1, n))()
+    start = (C.c_int32 * (n + 1))()
+    k = load().ss_cohort_build(arr, n, max_batch, order, start)
+    if k < 0:
+        raise SpecStreamError(SS_ERR_ARG, "ss_cohort_build")
+    return [list(order[start[c]:start[c + 1]]) for c in range(k)]

@@ -153,3 +153,11 @@ def test_cohort_builder_against_oracle_and_a_hand_case():
         assert got == oracle.cohort_build(tasks, mb)
         assert sorted(i for c in got for i in c) == list(range(len(tasks)))     # every task exactly once
     assert lib.ss_cohort_build(None, 1, 1, None, None) == -1
+    # the binding's wrappers marshal the same calls
+    assert ssb.cohort_build(tasks, mb) == got
+    wc = ssb.WidthController([2, 4], sample_rounds=1, switch_threshold=0.0, ema=1.0)
+    for q, t in ((2, 1.0), (4, 1.2)):
+        assert wc.next() == q
+        wc.observe(q, 0.0, t, 0.0, 0.0, q)
+    assert wc.next() == 4 and wc.estimate(4)[2] == pytest.approx(0.3)
+    wc.close()
