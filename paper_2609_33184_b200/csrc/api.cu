@@ -79,6 +79,8 @@ bool cfg_valid(const ss_config* c) {
   if (c->max_Tloc > 1024) return false;
   if (c->max_chunks < 0 || c->max_chunks > kMaxSets) return false;
   if ((int64_t)c->max_Tq * (c->H_q / c->H_kv) > 4096) return false;
+  // query rows per round: the row-per-warp kernels index them with 32-bit arithmetic
+  if ((int64_t)c->max_B * c->H_q * c->max_Tq >= (1ll << 31)) return false;
   return true;
 }
 

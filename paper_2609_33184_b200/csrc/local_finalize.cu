@@ -51,9 +51,12 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) local_kernel(const LocalPar
   pdl_launch_dependents();
   if (row_id < n_rows) {
     float* sc = sc_all + (size_t)warp * p.T_loc;
-    const int i = (int)(row_id % p.T_q);
-    const int h = (int)((row_id / p.T_q) % p.H_q);
-    const int b = (int)(row_id / ((int64_t)p.T_q * p.H_q));
+    // 32-bit index arithmetic (the row count fits: checked by the host): a 64-bit division costs
+    // a hundred instructions, more than the rest of a short row
+    const unsigned rid = (unsigned)row_id;
+    const int i = (int)(rid % (unsigned)p.T_q);
+    const int h = (int)((rid / (unsigned)p.T_q) % (unsigned)p.H_q);
+    const int b = (int)(rid / ((unsigned)p.T_q * (unsigned)p.H_q));
     const int kvh = h / p.G;
     const __nv_bfloat16* Kb = p.K + b * p.k_sb + kvh * p.k_sh + lane * CPL;
     const __nv_bfloat16* Vb = p.V + b * p.v_sb + kvh * p.v_sh + lane * CPL;
@@ -198,9 +201,10 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) merge_kernel(const MergePar
   const int64_t n_rows = (int64_t)p.B * p.H_q * p.T_q;
   if (MODE == 0) pdl_wait_prior();  // every partial of the round must be complete
   if (row_id >= n_rows) return;
-  const int i = (int)(row_id % p.T_q);
-  const int h = (int)((row_id / p.T_q) % p.H_q);
-  const int b = (int)(row_id / ((int64_t)p.T_q * p.H_q));
+  const unsigned rid = (unsigned)row_id;  // 32-bit index arithmetic: the row count fits
+  const int i = (int)(rid % (unsigned)p.T_q);
+  const int h = (int)((rid / (unsigned)p.T_q) % (unsigned)p.H_q);
+  const int b = (int)(rid / ((unsigned)p.T_q * (unsigned)p.H_q));
   const int kvh = h / p.G;
   const int r = (h % p.G) * p.T_q + i;
   const size_t slot0 = (size_t)b * p.H_kv + kvh;
@@ -319,9 +323,10 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) import_kernel(const MergePa
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t row_id = (int64_t)blockIdx.x * kWarpsPerCta + warp;
   if (row_id >= (int64_t)p.B * p.H_q * p.T_q) return;
-  const int i = (int)(row_id % p.T_q);
-  const int h = (int)((row_id / p.T_q) % p.H_q);
-  const int b = (int)(row_id / ((int64_t)p.T_q * p.H_q));
+  const unsigned rid = (unsigned)row_id;  // 32-bit index arithmetic: the row count fits
+  const int i = (int)(rid % (unsigned)p.T_q);
+  const int h = (int)((rid / (unsigned)p.T_q) % (unsigned)p.H_q);
+  const int b = (int)(rid / ((unsigned)p.T_q * (unsigned)p.H_q));
   const size_t idx = ((size_t)b * p.H_kv + h / p.G) * p.R_stride + (h % p.G) * p.T_q + i;
   if (lane == 0) p.fold_ml[idx] = reinterpret_cast<const float2*>(p.part_ml)[row_id];
   const float* src = p.part_a + row_id * D + lane * CPL;
