@@ -36,6 +36,7 @@ METRIC = "verify_attention_kv_GBps"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1400.0
+E2E_FILL_CHUNKS = 4   # adjacent history chunks per staging-buffer fill of the streamed leg
 
 
 def peaks():
@@ -223,7 +224,7 @@ def make_stream_desc(ssb, cfg, lens, host, dev, Q, K_loc, V_loc, bits, O, LSE, b
     for s in range(2):
         d.stage_k[s] = bufs["stage_k"][s].data_ptr()
         d.stage_v[s] = bufs["stage_v"][s].data_ptr()
-    d.stage_fused = 1 if bufs.get("fused") else 0
+    d.stage_fused = 2 if bufs.get("fused") == "blocks" else (1 if bufs.get("fused") else 0)
     d.scratch_fills = bufs["fills"]
     d.valid_len_host = bufs["vl_host"].data_ptr()
     d.valid_len_dev = bufs["vl_dev"].data_ptr()
@@ -244,10 +245,17 @@ def make_stream_desc(ssb, cfg, lens, host, dev, Q, K_loc, V_loc, bits, O, LSE, b
 
 def stream_buffers(cfg, dev, n_chunks, batch_chunks=1, fused=True):
     """Device staging + scratch of ss_stream_round.  fused: one buffer [B][2 (K,V)][H_kv][Ls][d]
-    per slot (each (request, chunk) block is then one copy); else separate K and V buffers."""
+    per slot (each (request, chunk) block is then one copy); fused = "blocks": one buffer
+    [B][batch_chunks][2][H_kv][L_c][d] per slot (the adjacent blocks of a request in one copy);
+    else separate K and V buffers."""
     Ls = cfg.L_c * batch_chunks
     fills = (n_chunks + batch_chunks - 1) // batch_chunks + 1
-    if fused:
+    if fused == "blocks":
+        fills = fills * batch_chunks   # one valid-length row per chunk call
+        kv = [torch.zeros(cfg.B, batch_chunks, 2, cfg.H_kv, cfg.L_c, cfg.d, dtype=torch.bfloat16, device=dev)
+              for _ in range(2)]
+        stage_k, stage_v = kv, kv
+    elif fused:
         kv = [torch.zeros(cfg.B, 2, cfg.H_kv, Ls, cfg.d, dtype=torch.bfloat16, device=dev) for _ in range(2)]
         stage_k, stage_v = [t[:, 0] for t in kv], [t[:, 1] for t in kv]   # views of the fused buffers
     else:
@@ -507,10 +515,13 @@ def main():
     e2e = None
     if not args.no_e2e and n_chunk_calls:
         host = pinned_history(cfg, lens, chunks)
-        bufs = stream_buffers(cfg, dev, n_chunk_calls)
+        # fills of E2E_FILL_CHUNKS adjacent chunks in the host's own block order: one copy per
+        # request and fill (32 MiB at c2) instead of one per block
+        bufs = stream_buffers(cfg, dev, n_chunk_calls, E2E_FILL_CHUNKS, fused="blocks")
         Qh, Klh, Vlh = Q.cpu().pin_memory(), K_loc.cpu().pin_memory(), V_loc.cpu().pin_memory()
         Qd, Kld, Vld = torch.empty_like(Q), torch.empty_like(K_loc), torch.empty_like(V_loc)
-        desc = make_stream_desc(ssb, cfg, lens, host, dev, Qd, Kld, Vld, bits, O, LSE, bufs)
+        desc = make_stream_desc(ssb, cfg, lens, host, dev, Qd, Kld, Vld, bits, O, LSE, bufs,
+                                batch_chunks=E2E_FILL_CHUNKS)
         n_e2e = max(3, min(args.steps, 10))
         times = []
         for i in range(2 + n_e2e):
@@ -547,7 +558,7 @@ def main():
         e2e = {"value": job_bytes / dt / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": int(stats.h2d_bytes + small_in),
                "d2h_bytes_per_step": int(stats.d2h_bytes), "ms_per_step": dt * 1e3,
-               "api": "ss_stream_round (pinned host history, 2 staging buffers)",
+               "api": f"ss_stream_round (pinned host history, 2 staging buffers, fills of {E2E_FILL_CHUNKS} chunks)",
                "pipeline_device_ms": min(full), "copy_only_device_ms": min(co),
                "exposed_attention_ms": min(full) - min(co),
                "h2d_GBps": h2d_gbps, "link_peak_GBps": best, "pct_of_link": 100.0 * h2d_gbps / best,
@@ -555,7 +566,8 @@ def main():
         del probe_h, probe_d
         if args.layers > 1 and rank == 0:
             # N layers sharing this layer's host history (same lengths); one descriptor each
-            descs = [make_stream_desc(ssb, cfg, lens, host, dev, Qd, Kld, Vld, bits, O, LSE, bufs)
+            descs = [make_stream_desc(ssb, cfg, lens, host, dev, Qd, Kld, Vld, bits, O, LSE, bufs,
+                                      batch_chunks=E2E_FILL_CHUNKS)
                      for _ in range(args.layers)]
             # restore buffer in the same fused K|V layout as the staging slots (one copy per block)
             rk = torch.empty(cfg.B, 2, cfg.H_kv, n_chunk_calls * cfg.L_c, cfg.d, dtype=torch.bfloat16, device=dev)

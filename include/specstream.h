@@ -238,7 +238,12 @@ typedef struct {
   int32_t stage_fused;       /* 1: stage_k[s] is ONE buffer [B][2 (K,V)][H_kv][batch_chunks*L_c][d]
                                 (stage_v ignored), the host block's own order, so every
                                 (request, chunk) block crosses the link in one copy instead of
-                                two: copies twice as large reach a few % more of the link     */
+                                two: copies twice as large reach a few % more of the link.
+                                2: stage_k[s] is [B][batch_chunks][2 (K,V)][H_kv][L_c][d], the
+                                host's block sequence itself: a fill moves the batch_chunks
+                                adjacent blocks of a request with ONE copy (plus one for a
+                                partial block) and is consumed by batch_chunks chunk calls of
+                                L_c tokens; scratch_fills then counts chunk calls, not fills  */
 } ss_stream_desc;
 
 typedef struct {

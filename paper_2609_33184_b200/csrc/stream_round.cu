@@ -58,7 +58,10 @@ ss_status validate_desc(ss_ctx* ctx, const ss_stream_desc* d, int* n_fills_out) 
   }
   const int n_chunks = (max_len + d->L_c - 1) / d->L_c;
   const int n_fills = (n_chunks + d->batch_chunks - 1) / d->batch_chunks;
-  if (n_fills > d->scratch_fills) return SS_ERR_CAPACITY;
+  // the valid-length scratch holds one row of B entries per chunk call
+  const int n_calls = d->stage_fused == 2 ? n_fills * d->batch_chunks : n_fills;
+  if (n_calls > d->scratch_fills) return SS_ERR_CAPACITY;
+  if (d->stage_fused < 0 || d->stage_fused > 2) return SS_ERR_ARG;
   *n_fills_out = n_fills;
   return SS_OK;
 }
@@ -77,17 +80,27 @@ ss_status enqueue_layer(ss_ctx* ctx, const ss_stream_desc* d, const ss::PipeRes&
   // K and V of a block next to each other in one device buffer ([B][K|V][H_kv][Ls][d]): the
   // staging slots with stage_fused, the restore buffer when restore_v is null
   const bool fused = restore ? restore_v == nullptr : d->stage_fused != 0;
-  const int64_t Ls = restore ? restore_tokens : (int64_t)bc * L_c;  // tokens per device buffer row
+  // block-major staging: a slot is [B][bc][K|V][H_kv][L_c][d], the host's own block order, so a
+  // fill moves up to bc adjacent blocks of a request with ONE copy and is consumed by bc chunk
+  // calls of L_c tokens
+  const bool blocks = !restore && d->stage_fused == 2;
+  const int64_t Ls = restore ? restore_tokens : (blocks ? L_c : (int64_t)bc * L_c);  // tokens per device row
+  // with stage_fused == 2 every chunk call takes L_c tokens (also on the restored copy)
+  const bool per_chunk = d->stage_fused == 2;
+  const int rows_vl = per_chunk ? n_fills * bc : n_fills;   // rows of the valid-length scratch
+  const int64_t span = per_chunk ? L_c : (int64_t)bc * L_c; // tokens one scratch row covers
   if (restore && (int64_t)n_fills * bc * L_c > restore_tokens) return SS_ERR_CAPACITY;
+  int64_t max_len = 0;
+  for (int b = 0; b < B; ++b) max_len = d->hist_len[b] > max_len ? d->hist_len[b] : max_len;
 
-  for (int f = 0; f < n_fills; ++f)
+  for (int f = 0; f < rows_vl; ++f)
     for (int b = 0; b < B; ++b) {
-      int64_t v = (int64_t)d->hist_len[b] - (int64_t)f * bc * L_c;
-      v = v < 0 ? 0 : (v > (int64_t)bc * L_c ? (int64_t)bc * L_c : v);
+      int64_t v = (int64_t)d->hist_len[b] - (int64_t)f * span;
+      v = v < 0 ? 0 : (v > span ? span : v);
       d->valid_len_host[f * B + b] = (int32_t)v;
     }
-  if (n_fills)
-    SS_CK(cudaMemcpyAsync(d->valid_len_dev, d->valid_len_host, sizeof(int32_t) * n_fills * B,
+  if (rows_vl)
+    SS_CK(cudaMemcpyAsync(d->valid_len_dev, d->valid_len_host, sizeof(int32_t) * rows_vl * B,
                           cudaMemcpyHostToDevice, r.copy_stream));
   if (!d->copy_only) {
     SS_ST(ss_verify_begin(ctx, d->Q, B, d->T_q, d->scale, r.attn_stream));
@@ -104,6 +117,50 @@ ss_status enqueue_layer(ss_ctx* ctx, const ss_stream_desc* d, const ss::PipeRes&
   for (int f = 0; f < n_fills; ++f) {
     const int buf = (fill_base + f) & 1;
     if (!restore && fill_base + f >= 2) SS_CK(cudaStreamWaitEvent(r.copy_stream, r.ev_free[buf], 0));
+    if (blocks) {
+      int last_chunk = -1;  // last chunk index of this fill that holds tokens of any request
+      for (int b = 0; b < B; ++b) {
+        const int64_t j0 = (int64_t)f * bc;
+        const int64_t rem = (int64_t)d->hist_len[b] - j0 * L_c;
+        if (rem <= 0) continue;
+        int64_t nfull = rem / L_c;
+        if (nfull > bc) nfull = bc;
+        const int64_t part = nfull < bc ? rem - nfull * L_c : 0;  // tokens of a partial block
+        const uint16_t* src = (const uint16_t*)d->hist[b] + j0 * block_elems;
+        uint16_t* dst = (uint16_t*)d->stage_k[buf] + (int64_t)b * bc * block_elems;
+        if (nfull > 0) {
+          SS_CK(cudaMemcpyAsync(dst, src, (size_t)(nfull * block_elems) * esz, cudaMemcpyHostToDevice,
+                                r.copy_stream));
+          cnt->h2d += nfull * block_elems * (int64_t)esz;
+          ++cnt->copies;
+        }
+        if (part > 0) {
+          SS_CK(cudaMemcpy2DAsync(dst + nfull * block_elems, (size_t)head_elems * esz,
+                                  src + nfull * block_elems, (size_t)head_elems * esz,
+                                  (size_t)part * hd * esz, 2 * H_kv, cudaMemcpyHostToDevice,
+                                  r.copy_stream));
+          cnt->h2d += 2 * (int64_t)H_kv * part * hd * esz;
+          ++cnt->copies;
+        }
+        const int lastb = (int)(j0 + nfull + (part > 0 ? 1 : 0)) - 1;
+        if (lastb > last_chunk) last_chunk = lastb;
+      }
+      SS_CK(cudaEventRecord(r.ev_ready[buf], r.copy_stream));
+      SS_CK(cudaStreamWaitEvent(r.attn_stream, r.ev_ready[buf], 0));
+      if (!d->copy_only) {
+        for (int jj = 0; jj < bc && f * bc + jj <= last_chunk; ++jj) {
+          const int j = f * bc + jj;
+          const uint16_t* kb = (const uint16_t*)d->stage_k[buf] + (int64_t)jj * block_elems;
+          ss_tensor K = {kb, (int64_t)bc * block_elems, head_elems, hd};
+          ss_tensor V = {kb + (int64_t)H_kv * head_elems, (int64_t)bc * block_elems, head_elems, hd};
+          SS_ST(ss_verify_chunk_hinted(ctx, K, V, L_c, d->valid_len_dev + (int64_t)j * B,
+                                       d->valid_len_host + (int64_t)j * B, r.attn_stream));
+          ++cnt->calls;
+        }
+      }
+      SS_CK(cudaEventRecord(r.ev_free[buf], r.attn_stream));
+      continue;
+    }
     for (int jj = 0; jj < bc; ++jj) {
       const int j = f * bc + jj;
       for (int b = 0; b < B; ++b) {
@@ -169,15 +226,16 @@ ss_status enqueue_layer(ss_ctx* ctx, const ss_stream_desc* d, const ss::PipeRes&
     SS_CK(cudaStreamWaitEvent(r.attn_stream, r.ev_ready[0], 0));
   }
   if (restore && !d->copy_only) {
-    for (int f = 0; f < n_fills; ++f) {  // the streamed path's chunk calls, on the restored copy
-      const int64_t tok = (int64_t)f * bc * L_c;
+    for (int f = 0; f < rows_vl; ++f) {  // the streamed path's chunk calls, on the restored copy
+      const int64_t tok = (int64_t)f * span;
+      if (per_chunk && tok >= max_len) break;
       ss_tensor K = {(uint16_t*)restore_k + tok * hd, (int64_t)H_kv * Ls * hd, Ls * hd, hd};
       ss_tensor V = {(uint16_t*)restore_v + tok * hd, (int64_t)H_kv * Ls * hd, Ls * hd, hd};
       if (fused) {
         K.stride_b = V.stride_b = 2 * (int64_t)H_kv * Ls * hd;
         V.ptr = (const uint16_t*)restore_k + (int64_t)H_kv * Ls * hd + tok * hd;
       }
-      SS_ST(ss_verify_chunk_hinted(ctx, K, V, bc * L_c, d->valid_len_dev + (int64_t)f * B,
+      SS_ST(ss_verify_chunk_hinted(ctx, K, V, (int32_t)span, d->valid_len_dev + (int64_t)f * B,
                                    d->valid_len_host + (int64_t)f * B, r.attn_stream));
       ++cnt->calls;
     }

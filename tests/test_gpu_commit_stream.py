@@ -145,7 +145,8 @@ def _stream_case(cfg, lens, batch_chunks=1, copy_only=0, accept=True, fused=True
                "cv": torch.zeros(shape, dtype=torch.bfloat16, device=DEV),
                "hk": torch.zeros(shape, dtype=torch.bfloat16).pin_memory(),
                "hv": torch.zeros(shape, dtype=torch.bfloat16).pin_memory(), "cnt_host": cnt, "idx_host": idx}
-    ctx = ssb.Context(cfg.B, cfg.H_q, cfg.H_kv, cfg.d, cfg.T_q, cfg.T_q, cfg.L_c * batch_chunks)
+    ctx = ssb.Context(cfg.B, cfg.H_q, cfg.H_kv, cfg.d, cfg.T_q, cfg.T_q,
+                      cfg.L_c * (1 if fused == "blocks" else batch_chunks))
     desc = bench.make_stream_desc(ssb, cfg, lens, host, DEV, Q, K_loc, V_loc, bits, O, LSE, bufs,
                                   batch_chunks=batch_chunks, accept=acc, copy_only=copy_only)
     stats = ctx.ss_stream_round(desc)
@@ -154,7 +155,7 @@ def _stream_case(cfg, lens, batch_chunks=1, copy_only=0, accept=True, fused=True
     return ctx, (Q, chunks, K_loc, V_loc, bits), O, LSE, bufs, acc, stats, desc
 
 
-@pytest.mark.parametrize("fused", [True, False])   # K|V of a block in one staging buffer / two
+@pytest.mark.parametrize("fused", [True, False, "blocks"])   # K|V fused / separate / block-major fills
 @pytest.mark.parametrize("batch_chunks", [1, 2, 3])
 def test_stream_round_matches_oracle_ragged(batch_chunks, fused):
     import oracle
@@ -162,13 +163,23 @@ def test_stream_round_matches_oracle_ragged(batch_chunks, fused):
     lens = [900, 0, 128, 257, 513]
     ctx, case, O, LSE, bufs, acc, stats, _ = _stream_case(cfg, lens, batch_chunks, fused=fused)
     n_blocks = sum(-(-l // cfg.L_c) for l in lens)
-    assert stats.copies == (n_blocks if fused else 2 * n_blocks)
+    n_fills = (max(lens) + cfg.L_c * batch_chunks - 1) // (cfg.L_c * batch_chunks)
+    if fused == "blocks":   # per request and fill: one copy for the full blocks, one for a partial block
+        want = 0
+        for l in lens:
+            for f in range(n_fills):
+                rem = l - f * batch_chunks * cfg.L_c
+                if rem > 0:
+                    nfull = min(batch_chunks, rem // cfg.L_c)
+                    want += (1 if nfull else 0) + (1 if nfull < batch_chunks and rem - nfull * cfg.L_c > 0 else 0)
+        assert stats.copies == want
+    else:
+        assert stats.copies == (n_blocks if fused else 2 * n_blocks)
     ref = util.oracle_case(cfg, lens, *case)
     util.compare(cfg, O, LSE, ref)
     assert torch.equal(bufs["O_host"], O.cpu()) and torch.equal(bufs["LSE_host"], LSE.cpu())
     assert stats.h2d_bytes == sum(lens) * cfg.H_kv * cfg.d * 4
-    n_fills = (max(lens) + cfg.L_c * batch_chunks - 1) // (cfg.L_c * batch_chunks)
-    assert stats.chunk_calls == n_fills
+    assert stats.chunk_calls == (-(-max(lens) // cfg.L_c) if fused == "blocks" else n_fills)
     # committed rows arrived on the host, bit exact
     zero = np.zeros((cfg.B, cfg.H_kv, cfg.T_q, cfg.d), np.uint16)
     ko, vo = oracle.commit_gather(_u16(case[2]), _u16(case[3]), acc["idx_host"].numpy(), acc["cnt_host"].numpy(),
@@ -263,7 +274,7 @@ def test_export_import_state_shards_the_history_by_chunks():
     ctx.close()
 
 
-def _layer_descs(ssb, cfg, lens, n_layers, bufs):
+def _layer_descs(ssb, cfg, lens, n_layers, bufs, batch_chunks=1):
     """One stream descriptor per layer: own history / Q / local KV / outputs, shared staging."""
     import dataclasses
     layers = []
@@ -276,20 +287,24 @@ def _layer_descs(ssb, cfg, lens, n_layers, bufs):
         lb = dict(bufs)
         lb["O_host"] = torch.zeros(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16).pin_memory()
         lb["LSE_host"] = torch.zeros(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32).pin_memory()
-        desc = bench.make_stream_desc(ssb, cfg_l, lens, host, DEV, Q, K_loc, V_loc, bits, O, LSE, lb)
+        desc = bench.make_stream_desc(ssb, cfg_l, lens, host, DEV, Q, K_loc, V_loc, bits, O, LSE, lb,
+                                      batch_chunks=batch_chunks)
         layers.append(dict(cfg=cfg_l, case=(Q, chunks, K_loc, V_loc, bits), host=host, O=O, LSE=LSE, desc=desc,
                            bufs=lb))
     return layers
 
 
-@pytest.mark.parametrize("fused_restore", [False, True])
-def test_stream_layers_modes_match_oracle_and_each_other(fused_restore):
+@pytest.mark.parametrize("fused_restore,fills", [(False, 1), (True, 1), (True, 3)])
+def test_stream_layers_modes_match_oracle_and_each_other(fused_restore, fills):
     ssb = _ssb()
     cfg = inputs.VerifyConfig("v", 0x66, 3, 8, 2, 128, 256, 8, 200, 1300)
     lens = [1300, 200, 777]
     n_chunks = inputs.num_chunks(cfg, lens)
-    bufs = bench.stream_buffers(cfg, DEV, n_chunks)
-    layers = _layer_descs(ssb, cfg, lens, 3, bufs)
+    if fills > 1:   # block-major fills of `fills` chunks, one copy per request and fill
+        bufs = bench.stream_buffers(cfg, DEV, n_chunks, fills, fused="blocks")
+    else:
+        bufs = bench.stream_buffers(cfg, DEV, n_chunks)
+    layers = _layer_descs(ssb, cfg, lens, 3, bufs, batch_chunks=fills)
     ctx = ssb.Context(cfg.B, cfg.H_q, cfg.H_kv, cfg.d, cfg.T_q, cfg.T_q, cfg.L_c)
     if fused_restore:   # K and V of a request next to each other in one buffer
         rk = torch.full((cfg.B, 2, cfg.H_kv, n_chunks * cfg.L_c, cfg.d), float("nan"), dtype=torch.bfloat16,
