@@ -19,9 +19,9 @@
 //    the tile and a block of the score columns (= rows); with WG = 2 two threads share a lane
 //    and split the columns.  Ragged tails are a per-thread select (key >= valid -> weight 0).
 //  * The row reference m[r] is shared by all keys, so it cannot follow each tile's maximum
-//    without a cross-lane reduction.  It is kept lazily: weights are exp2(s - m[r]) with the
-//    current m[r]; only if some s - m[r] exceeds 16 (always on the first tile, m = -inf) do
-//    the softmax threads agree (one named barrier per tile) to take the exact tile maxima
+//    without a cross-lane reduction.  It is kept lazily: it starts as the exact maxima of the
+//    first tile; weights are exp2(s - m[r]) with the current m[r]; only if some s - m[r] exceeds
+//    16 do the softmax threads agree (one named barrier per tile) to take the exact tile maxima
 //    (warp shuffles + shared memory), raise m, and rescale O^T and the row sums.  Any common
 //    reference gives the same a / l (Eq. 17), so this is exact.
 //  * Row sums l[r] accumulate per thread in registers and are reduced across the 128 key
@@ -316,6 +316,32 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
       // The scores are read from tensor memory twice (first for the overflow test, then for the
       // weights) instead of being held in registers across the barrier below.
       const uint32_t t_s = tmem + lane_off + (t & 1) * N + c0;
+      if (t == 0) {
+        // First references: the exact maxima of the first tile, which keeps its largest weight at
+        // exactly 1.  Done here without the bookkeeping of the general path below (nothing to
+        // rescale yet), which would cost three tiles' time while the CTA's ring sits full.
+        if (!dead) {
+#pragma unroll
+          for (int q = 0; q < NC / 16; ++q) {
+            if (q * 16 < cn) {
+              uint32_t raw[16];
+              tmem_ld16(t_s + q * 16, raw);
+              tc_wait_ld();
+#pragma unroll
+              for (int c = 0; c < 16; ++c) {
+                float v = key_ok ? __uint_as_float(raw[c]) * p.scale_log2 : -INFINITY;
+                v = warp_max_f(v);
+                if (lane == 0) ctl->smax[warp & 3][c0 + q * 16 + c] = v;
+              }
+            }
+          }
+        }
+        named_bar_sync(1, C::kSoft);
+        if (tid < n_mma && !dead)  // the tile's first key is valid, so the maximum is finite
+          ctl->nm_ref[tid] = -fmaxf(fmaxf(ctl->smax[0][tid], ctl->smax[1][tid]),
+                                    fmaxf(ctl->smax[2][tid], ctl->smax[3][tid]));
+        named_bar_sync(1, C::kSoft);
+      }
       bool over = false;
       if (!dead) {
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // independent chains
