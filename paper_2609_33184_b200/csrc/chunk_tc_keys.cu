@@ -165,16 +165,29 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   } else if (warp < 4 * WG) {
     // Q rows -> shared memory as the K-major B operand (128-byte swizzle), zero padding rows
-    for (int i = tid; i < n_mma * (kD / 8); i += C::kSoft) {
+    // (N rows x 16 pieces of 16 bytes over 128 * WG threads = 4 pieces per thread: all four
+    // global loads go out before the first store, one memory latency instead of four)
+    constexpr int kQPieces = N * (kD / 8) / C::kSoft;
+    static_assert(kQPieces * C::kSoft == N * (kD / 8), "Q pieces per thread");
+    uint4 qraw[kQPieces];
+#pragma unroll
+    for (int u = 0; u < kQPieces; ++u) {
+      const int i = tid + u * C::kSoft;
       const int n = i / (kD / 8), c8 = i % (kD / 8);
-      uint4 raw = make_uint4(0, 0, 0, 0);
+      qraw[u] = make_uint4(0, 0, 0, 0);
       if (n < nrows) {
         const int rg = row0 + n, g = rg / p.T_q, t = rg % p.T_q;
-        raw = *reinterpret_cast<const uint4*>(p.Q + b * p.q_sb + (int64_t)(kvh * p.G + g) * p.q_sh +
-                                              t * p.q_st + c8 * 8);
+        qraw[u] = *reinterpret_cast<const uint4*>(p.Q + b * p.q_sb + (int64_t)(kvh * p.G + g) * p.q_sh +
+                                                  t * p.q_st + c8 * 8);
       }
+    }
+#pragma unroll
+    for (int u = 0; u < kQPieces; ++u) {
+      const int i = tid + u * C::kSoft;
+      const int n = i / (kD / 8), c8 = i % (kD / 8);
       const int half = c8 >> 3, j = c8 & 7;
-      *reinterpret_cast<uint4*>(q_s + half * C::kQHalf + n * 128 + ((j ^ (n & 7)) << 4)) = raw;
+      if (n < n_mma)
+        *reinterpret_cast<uint4*>(q_s + half * C::kQHalf + n * 128 + ((j ^ (n & 7)) << 4)) = qraw[u];
     }
     if (tid < N) ctl->nm_ref[tid] = INFINITY;
     fence_proxy_async();
