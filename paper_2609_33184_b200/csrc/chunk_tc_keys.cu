@@ -97,6 +97,10 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
   uint8_t* p_s = smem + C::kOffP;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 32 * (4 * WG)) {  // the producer lane: fetch the tensor maps while the work item is read
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmK) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmV) : "memory");
+  }
   if (p.wait_first) pdl_wait_prior();
   pdl_launch_dependents();
   const ChunkWork w = chunk_work(p, p.rows_per_tile);
@@ -142,10 +146,13 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
   constexpr int kProducerWarp = 4 * WG, kMmaWarp = 4 * WG + 1;
   if (warp == kProducerWarp) {
     if (lane == 0) {
-      for (int u = 0; u < UNITS; ++u) {
-        mbar_init(&ctl->ufull[u], 1);
-        mbar_init(&ctl->uempty[u], 1);
-      }
+      // the first loads go out as early as possible: only their own barriers exist yet
+      for (int u = 0; u < UNITS; ++u) mbar_init(&ctl->ufull[u], 1);
+      fence_barrier_init();
+      // streamed once: evict first; shared by the row groups of a kv-head through L2: keep
+      const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
+      for (int j = 0; j < n_pre; ++j) issue_use(j, pol);
+      for (int u = 0; u < UNITS; ++u) mbar_init(&ctl->uempty[u], 1);
       mbar_init(&ctl->sfull[0], 1);
       mbar_init(&ctl->sfull[1], 1);
       mbar_init(&ctl->pready, C::kSoft);
@@ -153,9 +160,6 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
       ctl->abort = 0;
       ctl->flag[0] = ctl->flag[1] = ctl->flag[2] = 0;
       fence_barrier_init();
-      // streamed once: evict first; shared by the row groups of a kv-head through L2: keep
-      const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
-      for (int j = 0; j < n_pre; ++j) issue_use(j, pol);  // first loads before the rest is set up
     }
     __syncwarp();
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
