@@ -404,6 +404,12 @@ int32_t ss_last_cuda_error(ss_ctx* ctx);
  * max_words 64-bit words to HOST memory and returns the count. */
 ss_status ss_trace_enable(ss_ctx* ctx, int32_t on);
 int32_t ss_trace_read(ss_ctx* ctx, uint64_t* out, int32_t max_words);
+/* Self-test of the bounded waits (the paper has no counterpart): one small kernel whose 64
+ * threads wait, with the chunk kernels' own wait routine and a limit of limit_ms (1..1000), on
+ * a barrier that nothing will ever complete.  Every thread must give up: *gave_up (DEVICE
+ * uint32, zeroed by the caller) counts them, SS_DEV_WAIT_EXPIRED is raised in the context's
+ * status word (read and cleared with ss_poll_status) and the context stays usable. */
+ss_status ss_selftest_wait_expiry(ss_ctx* ctx, int32_t limit_ms, uint32_t* gave_up, void* stream);
 /* Measurement aid (the paper has no counterpart): read n segments of DEVICE memory once, in
  * one kernel, with streaming 16-byte loads from every SM, and XOR-fold them into the 64-bit
  * DEVICE word *sink (the caller zeroes it or ignores it; it exists so that the loads cannot be

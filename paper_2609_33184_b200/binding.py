@@ -32,7 +32,8 @@ EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "
            "ss_verify_import_state", "ss_stream_layers", "ss_tier_create", "ss_tier_destroy",
            "ss_tier_reset", "ss_tier_get", "ss_tier_tail", "ss_tier_commit", "ss_tier_migrate", "ss_tier_poll",
            "ss_tier_d2h_bytes", "ss_verify_chunk_paged", "ss_width_create", "ss_width_destroy",
-           "ss_width_observe", "ss_width_next", "ss_width_estimate", "ss_cohort_build", "ss_probe_read"]
+           "ss_width_observe", "ss_width_next", "ss_width_estimate", "ss_cohort_build", "ss_probe_read",
+           "ss_selftest_wait_expiry"]
 
 
 class ss_config(C.Structure):
@@ -203,6 +204,8 @@ def load() -> C.CDLL:
     lib.ss_launch_count.argtypes = [vp]
     lib.ss_last_chunk_kernel.restype = C.c_char_p
     lib.ss_last_chunk_kernel.argtypes = [vp]
+    lib.ss_selftest_wait_expiry.restype = C.c_int
+    lib.ss_selftest_wait_expiry.argtypes = [vp, i32, vp, vp]
     lib.ss_probe_read.restype = C.c_int
     lib.ss_probe_read.argtypes = [C.POINTER(vp), C.POINTER(C.c_size_t), i32, vp, vp]
     _lib = lib
@@ -387,6 +390,12 @@ class Context:
         stats = ss_stream_stats()
         self._check(self.lib.ss_stream_layers(self.handle, C.byref(ld), C.byref(stats)), "ss_stream_layers")
         return stats
+
+    def ss_selftest_wait_expiry(self, limit_ms: int, gave_up: torch.Tensor, stream=None):
+        """gave_up: device int32[1], zeroed by the caller; counts the threads whose wait ran out."""
+        assert gave_up.dtype == torch.int32 and gave_up.is_cuda
+        self._check(self.lib.ss_selftest_wait_expiry(self.handle, limit_ms, gave_up.data_ptr(), self._sp(stream)),
+                    "ss_selftest_wait_expiry")
 
     def launch_count(self) -> int:
         return int(self.lib.ss_launch_count(self.handle))

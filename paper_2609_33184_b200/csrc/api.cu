@@ -745,6 +745,7 @@ int ctx_dims(ss_ctx* c, int* H_q, int* H_kv, int* d) {
   return c->cfg.max_B;
 }
 void ctx_set_cuda_error(ss_ctx* c, cudaError_t e) { c->last_cuda = (int32_t)e; }
+uint32_t* ctx_status_word(ss_ctx* c) { return c->status; }
 void ctx_pipeline_mode(ss_ctx* c, bool on) {
   c->no_overlap = on;
   if (!on) c->state = ss_ctx::IDLE;  // a round the pipeline left open (error path) is dropped

@@ -4,6 +4,7 @@
 // as the verification round, in the same process and clock state, so that the round's KV GB/s
 // can be read against what a plain streaming read reaches on this GPU right now.
 #include "ss_internal.h"
+#include "tc_ptx.cuh"
 
 namespace {
 
@@ -92,5 +93,33 @@ extern "C" ss_status ss_probe_read(const void* const* srcs, const size_t* bytes,
   const unsigned full = (unsigned)sms * 4;  // four CTAs of 512 threads per SM: every warp slot taken
   probe_read_kernel<<<total < full ? total : full, kThreads, 0, (cudaStream_t)stream>>>(
       seg, reinterpret_cast<unsigned long long*>(sink));
+  return cudaGetLastError() == cudaSuccess ? SS_OK : SS_ERR_CUDA;
+}
+
+namespace ss {
+uint32_t* ctx_status_word(ss_ctx* c);  // api.cu
+}
+namespace {
+// A wait nothing will ever satisfy: every thread waits on an mbarrier whose phase never
+// completes, with the kernels' own bounded wait and a short limit.
+__global__ void __launch_bounds__(64) wait_expiry_kernel(uint32_t* status, unsigned long long limit_ns,
+                                                         uint32_t* gave_up) {
+  __shared__ uint64_t bar;
+  __shared__ volatile uint32_t abort_word;
+  if (threadIdx.x == 0) {
+    ss::tc::mbar_init(&bar, 1);
+    abort_word = 0;
+    ss::tc::fence_barrier_init();
+  }
+  __syncthreads();
+  const bool ok = ss::tc::mbar_wait_abortable(&bar, 0, &abort_word, status, limit_ns);
+  if (!ok) atomicAdd(gave_up, 1u);
+}
+}  // namespace
+
+extern "C" ss_status ss_selftest_wait_expiry(ss_ctx* ctx, int32_t limit_ms, uint32_t* gave_up, void* stream) {
+  if (!ctx || !gave_up || limit_ms <= 0 || limit_ms > 1000) return SS_ERR_ARG;
+  wait_expiry_kernel<<<1, 64, 0, (cudaStream_t)stream>>>(ss::ctx_status_word(ctx),
+                                                         (unsigned long long)limit_ms * 1000000ull, gave_up);
   return cudaGetLastError() == cudaSuccess ? SS_OK : SS_ERR_CUDA;
 }

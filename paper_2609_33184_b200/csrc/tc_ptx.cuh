@@ -43,14 +43,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false when the deadline passed or another role aborted.
 __device__ __forceinline__ bool mbar_wait_abortable(uint64_t* bar, uint32_t parity,
-                                                    volatile uint32_t* abort_word, uint32_t* status) {
+                                                    volatile uint32_t* abort_word, uint32_t* status,
+                                                    unsigned long long limit_ns = kWaitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = gtime_ns();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 255u) == 0) {
       if (*abort_word) return false;
-      if (gtime_ns() - t0 > kWaitNs) {
+      if (gtime_ns() - t0 > limit_ns) {
         *abort_word = 1;
         atomicOr(status, SS_DEV_WAIT_EXPIRED);
         return false;

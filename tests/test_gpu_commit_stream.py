@@ -1,6 +1,7 @@
 """GPU tests of commit-gather (bit exact), the streamed round, the call-order state machine
 and the trace facility, all through the C ABI."""
 import ctypes as C
+import time
 
 import numpy as np
 import pytest
@@ -353,3 +354,26 @@ def test_probe_read_folds_every_word_once():
     assert int(sink.item()) == want
     with pytest.raises(ssb.SpecStreamError):
         ssb.ss_probe_read([dev_segs[1][1:]], sink)   # 4-byte offset: not 16-byte aligned
+
+
+def test_a_wait_that_nothing_satisfies_gives_up_and_the_context_stays_usable():
+    # the chunk kernels bound every wait and report SS_DEV_WAIT_EXPIRED instead of hanging; the
+    # self-test kernel makes that routine run out on a barrier nobody completes (50 ms limit)
+    ssb = _ssb()
+    cfg = inputs.VerifyConfig("v", 0x70, 2, 8, 2, 128, 128, 4, 100, 300)
+    lens = inputs.history_lengths(cfg)
+    case = util.gen_case(cfg, lens, DEV)
+    ctx = util.make_ctx(cfg)
+    O1, L1 = util.gpu_case(ctx, cfg, *case)
+    O1 = O1.clone()
+    gave_up = torch.zeros(1, dtype=torch.int32, device=DEV)
+    t0 = time.time()
+    ctx.ss_selftest_wait_expiry(50, gave_up)
+    st, bits = ctx.ss_poll_status(timeout_ms=5000)
+    assert time.time() - t0 < 3.0
+    assert st == ssb.SS_ERR_DEVICE_FLAG and bits & 8          # SS_DEV_WAIT_EXPIRED
+    assert int(gave_up.item()) == 64                          # every waiting thread returned
+    assert ctx.ss_poll_status() == (0, 0)                     # reading cleared the word
+    O2, _ = util.gpu_case(ctx, cfg, *case)                    # and the context still works
+    assert torch.equal(O1.view(torch.int16), O2.view(torch.int16))
+    ctx.close()
