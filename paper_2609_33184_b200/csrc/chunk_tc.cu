@@ -346,17 +346,23 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     constexpr uint32_t idesc_pv = make_idesc(128, kD, true);
     const bool leader = elect_one();
     const uint32_t k_base = smem_u32(k_s), v_base = smem_u32(v_s0), q_addr = smem_u32(q_s);
+    // The operand descriptors of one slot differ only in their address field (bits 0-13, the
+    // shared-memory address / 16): they are built once and advanced by constants, which keeps
+    // the issue loop - the critical path when a tile's softmax is short - to a few
+    // instructions per MMA.  (All operand addresses are below 256 KB, so the field never carries.)
+    const uint64_t q_desc = desc_kmajor(q_addr);
+    const uint64_t k_desc0 = desc_kmajor(k_base);
+    const uint64_t v_desc0 = desc_mnmajor(v_base, kHalfTile);
     // S[it % 2] = Q K_it^T; releases the K slot and signals the softmax warps
     auto issue_qk = [&](int it) {
       const int s = it % kKStages;
-      const uint32_t k_addr = k_base + s * kTileBytes;
+      const uint64_t k_desc = k_desc0 + (uint64_t)(s * (kTileBytes >> 4));
       if (leader) {
 #pragma unroll
         for (int kk = 0; kk < kD / 16; ++kk) {
           const uint32_t qoff = (kk >> 2) * kQHalf + (kk & 3) * 32;
           const uint32_t koff = (kk >> 2) * kHalfTile + (kk & 3) * 32;
-          mma_ss(tmem + kColS + (it & 1) * 64, desc_kmajor(q_addr + qoff), desc_kmajor(k_addr + koff),
-                 idesc_qk, kk > 0);
+          mma_ss(tmem + kColS + (it & 1) * 64, q_desc + (qoff >> 4), k_desc + (koff >> 4), idesc_qk, kk > 0);
         }
         tc_commit(&ctl->kempty[s]);
         tc_commit(&ctl->sfull[it & 1]);
@@ -382,12 +388,12 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       if (!ok) break;
       trace(trl, 1, it, 2);
       tc_fence_after();
-      const uint32_t v_addr = v_base + s * kTileBytes;
+      const uint64_t v_desc = v_desc0 + (uint64_t)(s * (kTileBytes >> 4));
       if (leader) {
 #pragma unroll
         for (int kk = 0; kk < kTileKeys / 16; ++kk) {
-          mma_ts(tmem + kColO, tmem + kColS + (it & 1) * 64 + kk * 8,
-                 desc_mnmajor(v_addr + kk * 2048, kHalfTile), idesc_pv, (it > 0 || kk > 0));
+          mma_ts(tmem + kColO, tmem + kColS + (it & 1) * 64 + kk * 8, v_desc + (kk * 2048 >> 4), idesc_pv,
+                 (it > 0 || kk > 0));
         }
         tc_commit(&ctl->vempty[s]);
         tc_commit(&ctl->odone);
