@@ -246,31 +246,12 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
       }
       __syncwarp();
     };
-    bool ok = mwait(&ctl->ufull[0], 0);
-    if (ok) {
-      tc_fence_after();
-      issue_qk(0);
-    }
-    for (int t = 0; ok && t < n_tiles; ++t) {
-      trace(trl, 1, t, 0);
-      if (t + 1 < n_tiles) {
-        // scores of the next tile go out first: its softmax overlaps this tile's output MMAs.
-        // S^T[(t+1) & 1] was last read for tile t-1, whose pready was awaited in iteration t-1.
-        const int j = 2 * (t + 1);
-        ok = mwait(&ctl->ufull[j % UNITS], (j / UNITS) & 1);
-        if (!ok) break;
-        trace(trl, 1, t, 1);
-        tc_fence_after();
-        issue_qk(t + 1);
-        trace(trl, 1, t, 2);
-      }
+    // The issuer polls for whichever of its two next operations can go: the score MMAs of tile
+    // qi (K landed; its score buffer free, i.e. the output MMAs of tile qi - 2 issued) or the
+    // output MMAs of tile pi (weights ready, V landed).  Walking them in a fixed order would
+    // hold back an output MMA - and the release of its V unit - behind a K tile that is late.
+    auto issue_pv = [&](int t) {
       const int jv = 2 * t + 1;
-      ok = mwait(&ctl->pready, t & 1);
-      trace(trl, 1, t, 3);
-      ok = ok && mwait(&ctl->ufull[jv % UNITS], (jv / UNITS) & 1);
-      if (!ok) break;
-      trace(trl, 1, t, 4);
-      tc_fence_after();
       const uint32_t v_addr = base + (jv % UNITS) * kUnitBytes;
       if (leader) {
 #pragma unroll
@@ -284,7 +265,49 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
         tc_commit(&ctl->pfree);
       }
       __syncwarp();
-      trace(trl, 1, t, 5);
+    };
+    int qi = 0, pi = 0;
+    unsigned long long t0 = gtime_ns();
+    uint32_t spins = 0;
+    while (pi < n_tiles) {
+      bool did = false;
+      if (qi < n_tiles && qi < pi + 2) {
+        const int j = 2 * qi;
+        if (__all_sync(0xffffffffu, mbar_test(&ctl->ufull[j % UNITS], (j / UNITS) & 1))) {
+          trace(trl, 1, qi, 0);  // the tile's first stamp: its K has landed
+          tc_fence_after();
+          trace(trl, 1, qi, 1);
+          issue_qk(qi);
+          trace(trl, 1, qi, 2);
+          ++qi;
+          did = true;
+        }
+      }
+      if (pi < qi) {
+        const int jv = 2 * pi + 1;
+        if (__all_sync(0xffffffffu, mbar_test(&ctl->pready, pi & 1) &&
+                                        mbar_test(&ctl->ufull[jv % UNITS], (jv / UNITS) & 1))) {
+          tc_fence_after();
+          trace(trl, 1, pi, 4);
+          issue_pv(pi);
+          trace(trl, 1, pi, 5);
+          ++pi;
+          did = true;
+        }
+      }
+      if (did) {
+        spins = 0;
+        t0 = gtime_ns();
+      } else if ((++spins & 255u) == 0) {  // bounded like every other wait
+        const bool stop = ctl->abort != 0 || gtime_ns() - t0 > kWaitNs;
+        if (__any_sync(0xffffffffu, stop)) {
+          if (lane == 0 && ctl->abort == 0) {
+            ctl->abort = 1;
+            atomicOr(p.status, SS_DEV_WAIT_EXPIRED);
+          }
+          break;
+        }
+      }
     }
   } else {
     // ===== softmax warps: TMEM lane L = key L of the tile; columns [c0, c0 + cn) = rows =====
