@@ -369,25 +369,9 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       }
       __syncwarp();
     };
-    // the Q tile was written before the CTA-wide barrier above (with a proxy fence)
-    bool ok = true;
-    for (int it = 0; ok && it < n_pre_k; ++it) {  // one per score buffer (= per K slot)
-      ok = mbar_wait(&ctl->kfull[it], 0, ctl, p.status);
-      if (!ok) break;
-      tc_fence_after();
-      issue_qk(it);
-    }
-    static_assert(kKStages == 2, "the score MMAs of tile t + 2 reuse the K slot and the S buffer of tile t");
-    for (int it = 0; ok && it < n_tiles; ++it) {
+    // O += P_it V_it; releases the V slot, counts the tile on odone
+    auto issue_pv = [&](int it) {
       const int s = it % kVStages;
-      const uint32_t ph = (it / kVStages) & 1;
-      trace(trl, 1, it, 0);
-      ok = mbar_wait(&ctl->pready[it & 1], (it >> 1) & 1, ctl, p.status);
-      trace(trl, 1, it, 1);
-      ok = ok && mbar_wait(&ctl->vfull[s], ph, ctl, p.status);
-      if (!ok) break;
-      trace(trl, 1, it, 2);
-      tc_fence_after();
       const uint64_t v_desc = v_desc0 + (uint64_t)(s * (kTileBytes >> 4));
       if (leader) {
 #pragma unroll
@@ -400,16 +384,49 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         if (it + 1 == n_tiles) tc_commit(&ctl->pvdone);
       }
       __syncwarp();
-      trace(trl, 1, it, 3);
-      if (it + 2 < n_tiles) {
-        // overwrites the score buffer P(it) was read from: the tensor pipe runs this thread's
-        // MMAs in issue order, so the P V products above have consumed P before these write S
-        ok = mbar_wait(&ctl->kfull[it & 1], (((it + 2) / kKStages) & 1), ctl, p.status);
-        if (!ok) break;
-        trace(trl, 1, it, 4);
+    };
+    // The issuer polls for whichever of its two next operations can go: the score MMAs of tile
+    // qi (K landed; score buffer qi % 2 free, i.e. the output MMAs of tile qi - 2 issued: the
+    // tensor pipe runs this thread's MMAs in issue order, so they have consumed P before the
+    // new scores overwrite it) or the output MMAs of tile pi (P ready, V landed).  The Q tile
+    // was written before the CTA-wide barrier above (with a proxy fence).
+    static_assert(kKStages == 2, "the score MMAs of tile t + 2 reuse the K slot and the S buffer of tile t");
+    int qi = 0, pi = 0;
+    unsigned long long t0 = gtime_ns();
+    uint32_t spins = 0;
+    while (pi < n_tiles) {
+      bool did = false;
+      if (qi < n_tiles && qi < pi + 2 &&
+          __all_sync(0xffffffffu, mbar_test(&ctl->kfull[qi % kKStages], (qi / kKStages) & 1))) {
+        trace(trl, 1, qi, 0);
         tc_fence_after();
-        issue_qk(it + 2);
-        trace(trl, 1, it, 5);
+        issue_qk(qi);
+        trace(trl, 1, qi, 5);
+        ++qi;
+        did = true;
+      }
+      if (pi < qi &&
+          __all_sync(0xffffffffu, mbar_test(&ctl->pready[pi & 1], (pi >> 1) & 1) &&
+                                      mbar_test(&ctl->vfull[pi % kVStages], (pi / kVStages) & 1))) {
+        trace(trl, 1, pi, 2);
+        tc_fence_after();
+        issue_pv(pi);
+        trace(trl, 1, pi, 3);
+        ++pi;
+        did = true;
+      }
+      if (did) {
+        spins = 0;
+        t0 = gtime_ns();
+      } else if ((++spins & 255u) == 0) {  // bounded like every other wait
+        const bool stop = ctl->abort != 0 || gtime_ns() - t0 > kWaitNs;
+        if (__any_sync(0xffffffffu, stop)) {
+          if (lane == 0 && ctl->abort == 0) {
+            ctl->abort = 1;
+            atomicOr(p.status, SS_DEV_WAIT_EXPIRED);
+          }
+          break;
+        }
       }
     }
   } else {
