@@ -63,8 +63,8 @@ def tensor_peak():
 # DRAM bytes (read + write) per chunk-kernel launch from an ncu capture of the same kernel;
 # filled from the summaries under profiles/ (None until a capture exists for the workload).
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    # profiles/chunk_tc_keys_kernel_c2_qwen3_8b.md: 135.33 MB read + 3.47 MB written per launch
-    "c2_qwen3_8b": 138.8e6,
+    # profiles/chunk_tc_keys_kernel_c2_qwen3_8b.md: 135.34 MB read + 3.54 MB written per launch
+    "c2_qwen3_8b": 138.9e6,
     # profiles/chunk_tc_kernel_c4_tree.md: 69.80 MB read + 1.67 MB written per launch
     "c4_tree": 71.5e6,
 }
