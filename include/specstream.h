@@ -398,8 +398,9 @@ int32_t ss_last_cuda_error(ss_ctx* ctx);
 /* Tracing.  While enabled, CTA (0,0,0) of every tensor-core chunk kernel stamps the SM clock
  * at fixed points of its tile loop into a region of the workspace: words
  * [role][tile < 32][event < 8], role 0 = TMA producer, 1 = MMA issuer, 2 = softmax lane 0;
- * event 0 is the top of the role's loop for that tile, the other events are the kernel's own
- * wait / issue points (see the kernel sources).  Enabling clears the region (synchronous).
+ * event 0 is the role's first stamp for that tile (the softmax thread reaching the tile, the
+ * MMA issuer finding the tile's K landed), the other events are the kernel's own wait / issue
+ * points (see the kernel sources).  Enabling clears the region (synchronous).
  * ss_trace_read synchronises nothing: call it after the stream is idle; it copies up to
  * max_words 64-bit words to HOST memory and returns the count. */
 ss_status ss_trace_enable(ss_ctx* ctx, int32_t on);
