@@ -172,6 +172,12 @@ ss_status ss_verify_import_state(ss_ctx* ctx, const float* ml, const float* a, v
  * scores) into LSE [B, H_q, T_q] fp32 (may be NULL).  Ends the round. */
 ss_status ss_verify_finalize(ss_ctx* ctx, void* O, float* LSE, void* stream);
 
+/* Drops the open round without producing an output (for a caller whose chunk or local call
+ * failed, or that no longer wants the result).  Host-side only: kernels already enqueued run to
+ * completion and their partial states are never merged; the next ss_verify_begin starts from the
+ * identity state again.  With no round open it does nothing.  Returns SS_ERR_ARG for a NULL ctx. */
+ss_status ss_verify_abort(ss_ctx* ctx);
+
 /* a6. Commit-gather (Section 4.1: accepted candidates join the committed prefix).  For each
  * request b and k < accept_cnt[b]: row accept_idx[b][k] of K_loc/V_loc (all kv heads) is
  * copied, bit for bit, to row dst_off[b] + k of K_dst/V_dst [B, H_kv, cap, d].  Nothing else

@@ -33,7 +33,7 @@ EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "
            "ss_tier_reset", "ss_tier_get", "ss_tier_tail", "ss_tier_commit", "ss_tier_migrate", "ss_tier_poll",
            "ss_tier_d2h_bytes", "ss_verify_chunk_paged", "ss_width_create", "ss_width_destroy",
            "ss_width_observe", "ss_width_next", "ss_width_estimate", "ss_cohort_build", "ss_probe_read",
-           "ss_selftest_wait_expiry"]
+           "ss_selftest_wait_expiry", "ss_verify_abort"]
 
 
 class ss_config(C.Structure):
@@ -146,6 +146,8 @@ def load() -> C.CDLL:
     lib.ss_verify_import_state.argtypes = [vp, vp, vp, vp]
     lib.ss_verify_finalize.restype = C.c_int
     lib.ss_verify_finalize.argtypes = [vp, vp, vp, vp]
+    lib.ss_verify_abort.restype = C.c_int
+    lib.ss_verify_abort.argtypes = [vp]
     lib.ss_commit_gather.restype = C.c_int
     lib.ss_commit_gather.argtypes = [vp, ss_tensor, ss_tensor, i32, i32, vp, vp, ss_tensor,
                                      ss_tensor, i32, vp, vp]
@@ -349,6 +351,9 @@ class Context:
             assert LSE.dtype == torch.float32 and LSE.is_contiguous()
         self._check(self.lib.ss_verify_finalize(self.handle, O.data_ptr(), _ptr(LSE),
                                                 self._sp(stream)), "ss_verify_finalize")
+
+    def ss_verify_abort(self):
+        self._check(self.lib.ss_verify_abort(self.handle), "ss_verify_abort")
 
     def ss_commit_gather(self, K_loc, V_loc, accept_idx, accept_cnt, K_dst, V_dst, dst_off, stream=None):
         B, _, T_loc, _ = K_loc.shape

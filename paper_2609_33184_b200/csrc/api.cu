@@ -55,6 +55,10 @@ struct ss_ctx {
   bool trace_on;
 };
 
+namespace ss {
+void ctx_pipeline_release(ss_ctx* c);
+}
+
 namespace {
 
 using ss::kMaxSets;
@@ -287,16 +291,7 @@ ss_status ss_create(ss_ctx** out, const ss_config* cfg, void* workspace, size_t 
 
 ss_status ss_destroy(ss_ctx* c) {
   if (!c) return SS_ERR_ARG;
-  if (c->pipe_ready) {
-    cudaStreamDestroy(c->copy_stream);
-    cudaStreamDestroy(c->attn_stream);
-    for (int i = 0; i < 2; ++i) {
-      cudaEventDestroy(c->ev_ready[i]);
-      cudaEventDestroy(c->ev_free[i]);
-    }
-    cudaEventDestroy(c->ev_t0);
-    cudaEventDestroy(c->ev_t1);
-  }
+  ss::ctx_pipeline_release(c);
   delete c;
   return SS_OK;
 }
@@ -403,17 +398,14 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   if (tc && keys_on_m) {
     p.row_tiles = (R + 127) / 128;
     p.rows_per_tile = R < 128 ? R : 128;
-    p.groups = 1;
   } else if (tc) {
     // row tiles of 128 rows and a remainder tile; a tile with <= 64 (<= 32) rows replicates its
     // rows 2x (4x) along M, so no lane computes padding
     p.row_tiles = (R + 127) / 128;
     p.rows_per_tile = R < 128 ? R : 128;
-    p.groups = 0;  // decided per CTA from its row count
   } else {
     p.rows_per_tile = 32;
     p.row_tiles = (R + 31) / 32;
-    p.groups = 1;
   }
   // tensor-core CTAs amortise their set-up over at least 256 tokens; CUDA-core CTAs take one tile
   const int min_tiles = tc ? 4 : 1;
@@ -597,6 +589,16 @@ ss_status ss_verify_finalize(ss_ctx* c, void* O, float* LSE, void* stream) {
   return SS_OK;
 }
 
+ss_status ss_verify_abort(ss_ctx* c) {
+  if (!c) return SS_ERR_ARG;
+  // Kernels already enqueued finish on their own; their partial states are simply never merged.
+  c->state = ss_ctx::IDLE;
+  c->Q.ptr = nullptr;
+  c->n_sets = 0;
+  c->has_local = false;
+  return SS_OK;
+}
+
 ss_status ss_commit_gather(ss_ctx* c, ss_tensor K_loc, ss_tensor V_loc, int32_t B, int32_t T_loc,
                            const int32_t* accept_idx, const int32_t* accept_cnt, ss_tensor K_dst,
                            ss_tensor V_dst, int32_t cap, const int32_t* dst_off, void* stream) {
@@ -717,17 +719,37 @@ struct PipeRes {
   cudaStream_t copy_stream, attn_stream;
   cudaEvent_t *ev_ready, *ev_free, ev_t0, ev_t1;
 };
+namespace {
+// Releases whatever pipeline resources exist (handles are null until created).
+void pipeline_release(ss_ctx* c) {
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+  if (c->attn_stream) cudaStreamDestroy(c->attn_stream);
+  for (int i = 0; i < 2; ++i) {
+    if (c->ev_ready[i]) cudaEventDestroy(c->ev_ready[i]);
+    if (c->ev_free[i]) cudaEventDestroy(c->ev_free[i]);
+  }
+  if (c->ev_t0) cudaEventDestroy(c->ev_t0);
+  if (c->ev_t1) cudaEventDestroy(c->ev_t1);
+  c->copy_stream = c->attn_stream = nullptr;
+  c->ev_ready[0] = c->ev_ready[1] = c->ev_free[0] = c->ev_free[1] = c->ev_t0 = c->ev_t1 = nullptr;
+  c->pipe_ready = false;
+}
+}  // namespace
+void ctx_pipeline_release(ss_ctx* c) { pipeline_release(c); }
 cudaError_t ctx_pipeline(ss_ctx* c, PipeRes* out) {
   if (!c->pipe_ready) {
-    cudaError_t e;
-    if ((e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking)) != cudaSuccess) return e;
-    if ((e = cudaStreamCreateWithFlags(&c->attn_stream, cudaStreamNonBlocking)) != cudaSuccess) return e;
-    for (int i = 0; i < 2; ++i) {
-      if ((e = cudaEventCreateWithFlags(&c->ev_ready[i], cudaEventDisableTiming)) != cudaSuccess) return e;
-      if ((e = cudaEventCreateWithFlags(&c->ev_free[i], cudaEventDisableTiming)) != cudaSuccess) return e;
+    cudaError_t e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->attn_stream, cudaStreamNonBlocking);
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+      e = cudaEventCreateWithFlags(&c->ev_ready[i], cudaEventDisableTiming);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_free[i], cudaEventDisableTiming);
     }
-    if ((e = cudaEventCreate(&c->ev_t0)) != cudaSuccess) return e;
-    if ((e = cudaEventCreate(&c->ev_t1)) != cudaSuccess) return e;
+    if (e == cudaSuccess) e = cudaEventCreate(&c->ev_t0);
+    if (e == cudaSuccess) e = cudaEventCreate(&c->ev_t1);
+    if (e != cudaSuccess) {
+      pipeline_release(c);  // nothing half-built stays behind
+      return e;
+    }
     c->pipe_ready = true;
   }
   out->copy_stream = c->copy_stream;
@@ -749,5 +771,12 @@ uint32_t* ctx_status_word(ss_ctx* c) { return c->status; }
 void ctx_pipeline_mode(ss_ctx* c, bool on) {
   c->no_overlap = on;
   if (!on) c->state = ss_ctx::IDLE;  // a round the pipeline left open (error path) is dropped
+}
+// Error path of the pipeline: what was enqueued before the failing call still reads the caller's
+// buffers, so wait for it before the error is returned.
+void ctx_pipeline_drain(ss_ctx* c) {
+  if (!c->pipe_ready) return;
+  cudaStreamSynchronize(c->copy_stream);
+  cudaStreamSynchronize(c->attn_stream);
 }
 }  // namespace ss

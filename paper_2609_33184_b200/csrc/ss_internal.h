@@ -37,7 +37,6 @@ struct ChunkParams {
   int tiles_per_split;  // kTileKeys-token tiles per split
   int row_tiles;        // tiles of query rows per (b, kvh)
   int rows_per_tile;    // rows in each row tile but possibly the last
-  int groups;           // unused (the rows-on-M kernel derives its key groups from the row count)
   float scale_log2;     // scale * log2(e)
   float2* part_ml;      // partial set of this call
   float* part_a;

@@ -130,7 +130,6 @@ extern "C" ss_status ss_verify_round_static(const ss_static_round* r, void* stre
     p.tiles_per_split = tiles_per_split;
     p.row_tiles = row_tiles;
     p.rows_per_tile = 32;
-    p.groups = 1;
     p.scale_log2 = scale_log2;
     p.part_ml = part_ml;
     p.part_a = part_a;

@@ -19,6 +19,7 @@ cudaError_t ctx_pipeline(ss_ctx* c, PipeRes* out);
 int ctx_dims(ss_ctx* c, int* H_q, int* H_kv, int* d);
 void ctx_set_cuda_error(ss_ctx* c, cudaError_t e);
 void ctx_pipeline_mode(ss_ctx* c, bool on);
+void ctx_pipeline_drain(ss_ctx* c);
 }  // namespace ss
 
 #define SS_CK(expr)                          \
@@ -347,6 +348,7 @@ extern "C" ss_status ss_stream_round(ss_ctx* ctx, const ss_stream_desc* d, ss_st
   if (!ctx) return SS_ERR_ARG;
   ss::ctx_pipeline_mode(ctx, true);
   const ss_status st = stream_round_impl(ctx, d, stats);
+  if (st != SS_OK) ss::ctx_pipeline_drain(ctx);
   ss::ctx_pipeline_mode(ctx, false);
   return st;
 }
@@ -355,6 +357,7 @@ extern "C" ss_status ss_stream_layers(ss_ctx* ctx, const ss_layers_desc* layers,
   if (!ctx) return SS_ERR_ARG;
   ss::ctx_pipeline_mode(ctx, true);
   const ss_status st = stream_layers_impl(ctx, layers, total);
+  if (st != SS_OK) ss::ctx_pipeline_drain(ctx);
   ss::ctx_pipeline_mode(ctx, false);
   return st;
 }

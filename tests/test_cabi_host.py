@@ -62,4 +62,5 @@ def test_null_arguments_are_rejected_without_a_device(lib):
     assert lib.ss_verify_begin(None, t, 1, 1, 1.0, None) == ssb.SS_ERR_ARG
     assert lib.ss_verify_chunk(None, t, t, 1, None, None) == ssb.SS_ERR_ARG
     assert lib.ss_verify_finalize(None, None, None, None) == ssb.SS_ERR_ARG
+    assert lib.ss_verify_abort(None) == ssb.SS_ERR_ARG
     assert lib.ss_stream_round(None, None, None) == ssb.SS_ERR_ARG

@@ -117,6 +117,20 @@ def test_call_order_and_argument_errors():
     assert (O == 0).all() and torch.isinf(L).all() and (L < 0).all()
     too_many = torch.zeros(3, 8, 4, 128, dtype=torch.bfloat16, device=DEV)
     assert status(ctx.ss_verify_begin, too_many, cfg.scale) == ssb.SS_ERR_SHAPE
+    # an aborted round leaves nothing behind: the next round sees only its own calls
+    ctx.ss_verify_begin(Q, cfg.scale)
+    ctx.ss_verify_chunk(K, V, vl)
+    ctx.ss_verify_local(K_loc, V_loc)
+    ctx.ss_verify_abort()
+    assert status(ctx.ss_verify_finalize, O, None) == ssb.SS_ERR_STATE
+    ctx.ss_verify_abort()                                                      # no round open: no-op
+    ctx.ss_verify_begin(Q, cfg.scale)
+    ctx.ss_verify_finalize(O, L)
+    torch.cuda.synchronize()
+    assert (O == 0).all() and torch.isinf(L).all()
+    O2, L2 = util.gpu_case(ctx, cfg, Q, chunks, K_loc, V_loc, bits)
+    ref = util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits, groups=[(1, 1)])
+    util.compare(cfg, O2, L2, ref)
     ctx.close()
     with pytest.raises(ssb.SpecStreamError):
         ssb.Context(2, 9, 2, 128, 4, 4, 128)       # H_q % H_kv != 0
