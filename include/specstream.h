@@ -26,11 +26,14 @@
  *    by stream capture and replayed (the call-order state machine runs at capture time).
  *  - Call order per round: begin -> {chunk | local}* -> finalize.  Chunks may come in
  *    any order and any number (including zero); local at most once.  Anything else
- *    returns SS_ERR_STATE.
+ *    returns SS_ERR_STATE.  ss_verify_abort drops an open round.
  *  - Errors: host-detectable problems return a code and enqueue nothing.  Problems only
  *    the device can see (valid_len outside [0, L_c], accept index outside [0, T_loc),
  *    destination overflow, a bounded wait that expired) set a status word in the
  *    workspace, skip the offending item, never trap; read it with ss_poll_status.
+ *  - Threads: a context holds the state of one round at a time and is not thread-safe; calls
+ *    on one context from several host threads must be serialised by the caller.  Different
+ *    contexts (each with its own workspace) are independent and may be used concurrently.
  *  - Determinism: same inputs, same call sequence, same config -> bitwise-same output.
  *  - A query row with no visible key yields O = 0 and LSE = -inf.
  */

@@ -149,11 +149,13 @@ ss_status ss_tier_migrate(ss_tier* t, void* stream, int32_t* n_requests) {
   const size_t esz = 2;
   const int64_t cap = c.tail_capacity;
   int moved = 0;
+  // every end point is checked against its host capacity before the first copy is enqueued
+  for (int b = 0; b < c.B; ++b)
+    if (endpoint(t->H[b], t->C[b], c.tail_target, c.granularity) > t->host_cap[b]) return SS_ERR_CAPACITY;
   for (int b = 0; b < c.B; ++b) {
     const int32_t E = endpoint(t->H[b], t->C[b], c.tail_target, c.granularity);
     t->E[b] = E;
     if (E <= t->H[b]) continue;
-    if (E > t->host_cap[b]) return SS_ERR_CAPACITY;
     ++moved;
     // [H, E) -> host chunk blocks [chunk][K|V][H_kv][L_c][d]; one 2-D copy per chunk segment and K|V
     for (int32_t tok = t->H[b]; tok < E;) {

@@ -492,3 +492,44 @@ def test_round_can_be_captured_in_a_cuda_graph():
         torch.cuda.synchronize()
         assert torch.equal(O.view(torch.int16), O_ref.view(torch.int16)) and torch.equal(LSE, L_ref)
     ctx.close()
+
+
+def test_two_contexts_on_two_streams_do_not_interfere():
+    # Two contexts (own workspaces) whose rounds interleave call by call on two streams give,
+    # bit for bit, what each gives alone: no state is shared between contexts.
+    ssb = _ssb()
+    cfgs = [inputs.VerifyConfig("v", 0x71, 4, 16, 4, 128, 512, 8, 900, 2000),
+            inputs.VerifyConfig("v", 0x72, 3, 8, 2, 128, 256, 24, 500, 1500, mask="tree")]
+    cases, alone, ctxs = [], [], []
+    for cfg in cfgs:
+        lens = inputs.history_lengths(cfg)
+        case = util.gen_case(cfg, lens, DEV)
+        ctx = util.make_ctx(cfg, flags=ssb.SS_FLAG_OVERLAP_CHUNKS)
+        O, L = util.gpu_case(ctx, cfg, *case)
+        cases.append(case)
+        alone.append((O.clone(), L.clone()))
+        ctxs.append(ctx)
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = [(torch.zeros_like(o), torch.zeros_like(l)) for o, l in alone]
+    for rep in range(20):
+        for i in (0, 1):
+            ctxs[i].ss_verify_begin(cases[i][0], cfgs[i].scale, streams[i])
+        n = max(len(c[1]) for c in cases)
+        for j in range(n):
+            for i in (0, 1):
+                if j < len(cases[i][1]):
+                    K, V, vl = cases[i][1][j]
+                    ctxs[i].ss_verify_chunk(K, V, vl, streams[i])
+        for i in (0, 1):
+            Q, chunks, K_loc, V_loc, bits = cases[i]
+            tree = cfgs[i].mask == "tree"
+            ctxs[i].ss_verify_local(K_loc, V_loc, ssb.SS_MASK_TREE_BITS if tree else ssb.SS_MASK_CHAIN,
+                                    bits if tree else None, streams[i])
+            ctxs[i].ss_verify_finalize(outs[i][0], outs[i][1], streams[i])
+    torch.cuda.synchronize()
+    for i in (0, 1):
+        assert ctxs[i].ss_poll_status() == (0, 0)
+        assert torch.equal(outs[i][0].view(torch.int16), alone[i][0].view(torch.int16))
+        assert torch.equal(outs[i][1], alone[i][1])
+        ctxs[i].close()
