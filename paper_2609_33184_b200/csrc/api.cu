@@ -46,6 +46,7 @@ struct ss_ctx {
   } tm[64];
   int tm_n;
   uint64_t tm_clock;
+  CUtensorMap tm_a;         // all partial a[]: [sets * slots][R_stride][d] fp32, box [128 rows][32]
   // pipeline resources (created lazily by ss_stream_round)
   cudaStream_t copy_stream, attn_stream;
   cudaEvent_t ev_ready[2], ev_free[2], ev_t0, ev_t1;
@@ -176,6 +177,22 @@ bool get_tensor_map(ss_ctx* c, const ss_tensor& t, int B, int L_c, int box_token
   return true;
 }
 
+// Tensor map over every partial a[] of the workspace, [sets * slots][R_stride][d] fp32, for the
+// rows-on-M kernel's write-out: boxes of 128 rows x 32 floats, 128-byte swizzle.  A box that
+// reaches past row R_stride of its slot is clipped there by the hardware.
+bool encode_partials_map(ss_ctx* c) {
+  if (!g_encode) return false;
+  const uint64_t d = (uint64_t)c->cfg.d, rows = (uint64_t)c->R_stride;
+  const uint64_t slots = (uint64_t)(c->n_set_cap + 1) * c->slots_per_set;
+  cuuint64_t dims[3] = {d, rows, slots};
+  cuuint64_t strides[2] = {d * 4, rows * d * 4};
+  cuuint32_t box[3] = {32, (cuuint32_t)(rows < 128 ? rows : 128), 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return g_encode(&c->tm_a, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, c->part_a, dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool use_pdl(ss_ctx* c) {
   return (c->cfg.flags & SS_FLAG_OVERLAP_CHUNKS) && !c->first_launch && !c->no_overlap;
 }
@@ -272,6 +289,7 @@ ss_status ss_create(ss_ctx** out, const ss_config* cfg, void* workspace, size_t 
       g_encode = (EncodeTiledFn)fn;
   }
   c->tc_ok = (g_encode != nullptr) && (cfg->d == 128) && !(cfg->flags & SS_FLAG_FORCE_SIMT);
+  if (c->tc_ok) c->tc_ok = encode_partials_map(c);
   if (c->tc_ok) {
     e = ss::chunk_tc_prepare();
     if (e == cudaSuccess) e = ss::chunk_tc_keys_prepare();
@@ -466,6 +484,7 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   p.part_ml = c->part_ml + (int64_t)c->n_sets * c->set_stride_ml;
   p.part_a = c->part_a + (int64_t)c->n_sets * c->set_stride_a;
   p.R_stride = c->R_stride;
+  p.a_slot0 = c->n_sets * c->slots_per_set;
   p.status = c->status;
   p.wait_first = 0;
   p.trace = c->trace_on ? c->trace : nullptr;
@@ -479,7 +498,7 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   const bool pdl = use_pdl(c);
   cudaError_t e = !tc ? ss::launch_chunk_simt(p, s, pdl)
                   : keys_on_m ? ss::launch_chunk_tc_keys(p, tmK, tmV, s, pdl)
-                              : ss::launch_chunk_tc(p, tmK, tmV, s, pdl);
+                              : ss::launch_chunk_tc(p, tmK, tmV, c->tm_a, s, pdl);
   if (e != cudaSuccess) return cuda_fail(c, e);
   c->last_kernel = !tc ? "simt" : keys_on_m ? "tcgen05-keys" : "tcgen05";
   ++c->launches;

@@ -179,7 +179,7 @@ __device__ __forceinline__ bool softmax_tile(uint32_t t_s, uint32_t t_o, int c0,
 
 __global__ void __launch_bounds__(kThreads, 2)
 chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
-                const __grid_constant__ CUtensorMap tmV) {
+                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmA) {
   extern __shared__ __align__(1024) uint8_t smem[];
   uint8_t* q_s = smem;             // Q tile: two halves [128 rows][64 d], 128-byte swizzle
   uint8_t* k_s = smem + kOffK;     // K slots
@@ -193,7 +193,6 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   const int b = w.b, kvh = w.kvh, row0 = w.row0, nrows = w.nrows, tok0 = w.tok0, tok1 = w.tok1;
   const bool chain_cta = w.chain_cta;
   float2* out_ml = w.out_ml;
-  float* out_a = w.out_a;
   // key groups sharing the 128 lanes: the Q rows are replicated when the tile has few rows
   const int groups = nrows <= 32 ? 4 : (nrows <= 64 ? 2 : 1);
   const int r_pad = 128 / groups;
@@ -494,29 +493,37 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     if (ctl->abort == 0) {  // uniform over the 128 threads after the barrier
       tc_fence_after();
       // ---- merge the key groups of each row and write the partial state ----
-      // everything below lives over the idle Q tile and K/V slots: O as [128][128] fp32 over
-      // the first 64 KB (Q and the K slots), the lanes' (m, l) at the start of the V slots
+      // Everything below lives over the idle Q tile and K/V slots.  The 128 lanes' O rows are
+      // staged as fp32 in the layout a TMA store with the 128-byte swizzle reads: four blocks
+      // of [128 rows][32 floats], 16-byte chunk c of a row at chunk c ^ (row % 8) (so a warp's
+      // 16-byte accesses, one row per lane, spread over all banks); the lanes' (m, l) sit
+      // behind them in the V slots.
       float* o_s = reinterpret_cast<float*>(smem);
       float2* ml_s = reinterpret_cast<float2*>(v_s0);
       static_assert(kOffV >= 128 * 128 * 4, "O staging must end before the (m, l) array");
+      auto o_at = [&](int row, int c4) {  // float4 number c4 (0..31) of a staged row
+        return reinterpret_cast<float4*>(o_s + (c4 >> 3) * (128 * 32) + row * 32 +
+                                         (((c4 & 7) ^ (row & 7)) << 2));
+      };
       ml_s[L] = make_float2(m, l);
       named_bar_sync(1, 128);
       float M = -INFINITY;
       for (int g = 0; g < groups; ++g) M = fmaxf(M, ml_s[g * r_pad + r].x);
       const float f = (m == -INFINITY) ? 0.f : exp2f(m - M);
 #pragma unroll 1
-      for (int q = 0; q < kD / 16; ++q) {
-        uint32_t o[16];
-        tmem_ld16(t_o + q * 16, o);
+      for (int q = 0; q < kD / 32; ++q) {
+        uint32_t o[2][16];
+        tmem_ld16(t_o + q * 32, o[0]);
+        tmem_ld16(t_o + q * 32 + 16, o[1]);
         tc_wait_ld();
 #pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4) {
+        for (int c4 = 0; c4 < 8; ++c4) {
           float4 v;
-          v.x = __uint_as_float(o[c4 * 4 + 0]) * f;
-          v.y = __uint_as_float(o[c4 * 4 + 1]) * f;
-          v.z = __uint_as_float(o[c4 * 4 + 2]) * f;
-          v.w = __uint_as_float(o[c4 * 4 + 3]) * f;
-          *reinterpret_cast<float4*>(&o_s[L * kD + (((q * 4 + c4) ^ (L & 31)) << 2)]) = v;
+          v.x = __uint_as_float(o[c4 >> 2][(c4 & 3) * 4 + 0]) * f;
+          v.y = __uint_as_float(o[c4 >> 2][(c4 & 3) * 4 + 1]) * f;
+          v.z = __uint_as_float(o[c4 >> 2][(c4 & 3) * 4 + 2]) * f;
+          v.w = __uint_as_float(o[c4 >> 2][(c4 & 3) * 4 + 3]) * f;
+          *o_at(L, q * 8 + c4) = v;
         }
       }
       if (L < nrows) {
@@ -527,18 +534,40 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         }
         out_ml[L] = make_float2(lt > 0.f ? M : -INFINITY, lt);
       }
-      named_bar_sync(1, 128);
-      for (int rr = warp; rr < nrows; rr += 4) {
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int g = 0; g < groups; ++g) {
-          const int LL = g * r_pad + rr;
-          const float4 v = *reinterpret_cast<const float4*>(&o_s[LL * kD + ((lane ^ (LL & 31)) << 2)]);
-          acc.x += v.x;
-          acc.y += v.y;
-          acc.z += v.z;
-          acc.w += v.w;
+      if (groups > 1) {
+        // lane (r, grp) sums columns [grp * 128/groups, (grp + 1) * 128/groups) of row r over
+        // the row's `groups` staged copies and puts them back over the first copy
+        named_bar_sync(1, 128);
+        const int n4 = 32 / groups, c40 = grp * n4;
+        for (int c = 0; c < n4; c += 4) {
+          float4 acc[4];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) acc[k] = *o_at(r, c40 + c + k);
+          for (int g = 1; g < groups; ++g) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const float4 v = *o_at(g * r_pad + r, c40 + c + k);
+              acc[k].x += v.x;
+              acc[k].y += v.y;
+              acc[k].z += v.z;
+              acc[k].w += v.w;
+            }
+          }
+#pragma unroll
+          for (int k = 0; k < 4; ++k) *o_at(r, c40 + c + k) = acc[k];
         }
-        *reinterpret_cast<float4*>(out_a + (size_t)rr * kD + lane * 4) = acc;
+      }
+      // Four TMA stores move rows [row0, row0 + 128) of the slot.  Rows past `nrows` carry
+      // padding lanes (or the other groups' copies): they land in rows >= R of this slot, which
+      // nothing reads, or past the slot's last row, where the hardware clips the box.
+      fence_proxy_async();  // generic-proxy writes -> visible to the TMA store
+      named_bar_sync(1, 128);
+      if (L == 0) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          tma_store_3d(&tmA, smem_u32(o_s + j * (128 * 32)), j * 32, row0, p.a_slot0 + w.slot);
+        bulk_commit();
+        bulk_wait_read();  // shared memory is released when the CTA leaves
       }
     }
   }
@@ -563,9 +592,9 @@ cudaError_t chunk_tc_prepare() {
 }
 
 cudaError_t launch_chunk_tc(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
-                            cudaStream_t s, bool pdl) {
+                            const CUtensorMap& tmA, cudaStream_t s, bool pdl) {
   dim3 grid(p.splits * p.row_tiles, p.H_kv, p.B), block(kThreads);
-  return launch_kernel(chunk_tc_kernel, grid, block, kSmemTotal, s, pdl, p, tmK, tmV);
+  return launch_kernel(chunk_tc_kernel, grid, block, kSmemTotal, s, pdl, p, tmK, tmV, tmA);
 }
 
 }  // namespace ss

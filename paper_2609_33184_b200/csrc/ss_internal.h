@@ -41,6 +41,8 @@ struct ChunkParams {
   float2* part_ml;      // partial set of this call
   float* part_a;
   int R_stride;
+  int a_slot0;          // index of the call's first (split, b, kvh) slot along the outermost axis of
+                        // the tensor map over all partial a[] (tensor-core kernel with rows on M)
   uint32_t* status;
   int wait_first;       // 1: wait for the preceding kernel before reading inputs
   unsigned long long* trace;  // optional: per-tile clock stamps of CTA (0,0,0), see ss_trace_read
@@ -99,7 +101,7 @@ struct GatherParams {
 // launchers (each returns the cudaError_t of the launch)
 cudaError_t launch_chunk_simt(const ChunkParams& p, cudaStream_t s, bool pdl);
 cudaError_t launch_chunk_tc(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
-                            cudaStream_t s, bool pdl);
+                            const CUtensorMap& tmA, cudaStream_t s, bool pdl);
 cudaError_t chunk_tc_prepare();  // one-time function attributes
 cudaError_t launch_chunk_tc_keys(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
                                  cudaStream_t s, bool pdl);
@@ -148,6 +150,7 @@ __device__ __forceinline__ void trace(unsigned long long* tr, int role, int it, 
 // by the three chunk kernels; `tile_rows` is the kernel's rows per row tile.
 struct ChunkWork {
   int b, kvh, split;
+  int slot;             // (split, b, kvh) slot of the call's partial set
   int row0, nrows;      // query rows [row0, row0 + nrows) of the kv-head
   int tok0, tok1;       // visible tokens [tok0, tok1) of the chunk (tok1 <= tok0: nothing to do)
   float2* out_ml;       // partial state of the CTA's rows
@@ -174,6 +177,7 @@ __device__ __forceinline__ ChunkWork chunk_work(const ChunkParams& p, int tile_r
   w.tok0 = w.split * p.tiles_per_split * kTileKeys;
   w.tok1 = min(valid, w.tok0 + p.tiles_per_split * kTileKeys);
   const size_t slot = ((size_t)w.split * p.B + w.b) * p.H_kv + w.kvh;
+  w.slot = (int)slot;
   w.out_ml = p.part_ml + slot * p.R_stride + w.row0;
   w.out_a = p.part_a + (slot * p.R_stride + w.row0) * p.d;
   return w;
