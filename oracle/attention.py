@@ -25,7 +25,7 @@ def verify_attention_rows(q, k_vis, v_vis, scale):
 
     q [R, d], k_vis [n, d], v_vis [n, d] (fp64).  Returns O [R, d], LSE [R].
     """
-    R, d = q.shape
+    R = q.shape[0]
     n = k_vis.shape[0]
     if n == 0:
         return np.zeros((R, v_vis.shape[1])), np.full(R, -np.inf)
@@ -47,7 +47,7 @@ def verify_attention(Q, K_hist, V_hist, K_loc, V_loc, mask, scale):
     Returns O [B, H_q, T_q, d] fp64, LSE [B, H_q, T_q] fp64.
     """
     Q = np.asarray(Q, dtype=np.float64)
-    B, H_q, T_q, d = Q.shape
+    B, H_q, T_q, _ = Q.shape
     H_kv = K_loc.shape[1]
     G = H_q // H_kv
     assert G * H_kv == H_q

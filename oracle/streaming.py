@@ -81,7 +81,6 @@ def streamed_verify_attention(q, k_hist, v_hist, k_loc, v_loc, vis_loc, scale, L
     order = list(range(J)) if order is None else list(order)
     local_at = J if local_at is None else local_at
     state = IDENTITY(q.shape[0], v_loc.shape[1])
-    done = 0
     for pos in range(J + 1):
         if pos == local_at:
             state = merge(state, chunk_partial(q, k_loc, v_loc, scale, vis_loc))
@@ -89,5 +88,4 @@ def streamed_verify_attention(q, k_hist, v_hist, k_loc, v_loc, vis_loc, scale, L
             j = order[pos]
             sl = slice(j * L_c, min(n, (j + 1) * L_c))
             state = merge(state, chunk_partial(q, k_hist[sl], v_hist[sl], scale))
-            done += 1
     return finalize(state)

@@ -1,6 +1,5 @@
 """GPU tests of commit-gather (bit exact), the streamed round, the call-order state machine
 and the trace facility, all through the C ABI."""
-import ctypes as C
 import time
 
 import numpy as np

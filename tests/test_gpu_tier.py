@@ -2,7 +2,6 @@
 into the on-GPU Active Tail, batched offload of [H, E) by Eq. 9 and streamed attention over
 host history + tail + candidates, checked every round against the oracle (attention over the
 true committed sequence, Eq. 9 boundaries, bit-exact placement of every committed token)."""
-import ctypes as C
 
 import numpy as np
 import pytest
