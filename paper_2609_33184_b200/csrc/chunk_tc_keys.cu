@@ -33,7 +33,7 @@
 //
 // Rows <= 32: 3 ring units, 113 KB shared memory, 128 TMEM columns -> two CTAs per SM, so one
 // CTA's ramp-up and tail overlap the other's steady state (also across consecutive kernels).
-// Rows up to 64 / 128: 5 ring units, one CTA per SM, 8 / 16 softmax warps (the latency of
+// Rows up to 64 / 128: 6 / 5 ring units, one CTA per SM, 8 / 16 softmax warps (the latency of
 // tensor-memory loads is hidden by warps, not by holding more columns per thread).
 // Every mbarrier wait is bounded; on expiry the CTA raises SS_DEV_WAIT_EXPIRED, lets its own
 // copies land (bounded), frees its tensor memory and returns.
@@ -604,7 +604,7 @@ cudaError_t prepare_cfg() {
 
 cudaError_t chunk_tc_keys_prepare() {
   cudaError_t e = prepare_cfg<32, 1, 3>();
-  if (e == cudaSuccess) e = prepare_cfg<32, 2, 5>();
+  if (e == cudaSuccess) e = prepare_cfg<32, 2, 6>();
   if (e == cudaSuccess) e = prepare_cfg<32, 4, 5>();
   return e;
 }
@@ -614,7 +614,7 @@ cudaError_t chunk_tc_keys_prepare() {
 cudaError_t launch_chunk_tc_keys(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
                                  cudaStream_t s, bool pdl) {
   if (p.rows_per_tile <= 32) return launch_cfg<32, 1, 3>(p, tmK, tmV, s, pdl);
-  if (p.rows_per_tile <= 64) return launch_cfg<32, 2, 5>(p, tmK, tmV, s, pdl);
+  if (p.rows_per_tile <= 64) return launch_cfg<32, 2, 6>(p, tmK, tmV, s, pdl);
   return launch_cfg<32, 4, 5>(p, tmK, tmV, s, pdl);
 }
 
