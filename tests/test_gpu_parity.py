@@ -533,3 +533,22 @@ def test_two_contexts_on_two_streams_do_not_interfere():
         assert torch.equal(outs[i][0].view(torch.int16), alone[i][0].view(torch.int16))
         assert torch.equal(outs[i][1], alone[i][1])
         ctxs[i].close()
+
+
+@pytest.mark.parametrize("flags", [0, 4])
+def test_rounds_narrower_than_the_context_limit(flags):
+    # A context sized for max_Tq candidates runs rounds with fewer: the partial-state rows of a
+    # slot then have room past the round's last row (the rows-on-M kernel's write-out may put
+    # padding there), and a later, wider round must not see anything of it.
+    ssb = _ssb()
+    wide = inputs.VerifyConfig("v", 0x81, 2, 16, 4, 128, 512, 40, 700, 1500, k_mult=2.0)
+    ctx = ssb.Context(wide.B, wide.H_q, wide.H_kv, wide.d, wide.T_q, wide.T_q, wide.L_c, flags=flags)
+    for T_q in (40, 20, 9, 33, 40):
+        cfg = inputs.VerifyConfig("v", 0x81 + T_q, 2, 16, 4, 128, 512, T_q, 700, 1500, k_mult=2.0)
+        lens = inputs.history_lengths(cfg)
+        case = util.gen_case(cfg, lens, DEV)
+        O, LSE = util.gpu_case(ctx, cfg, *case)
+        assert ctx.ss_poll_status() == (0, 0)
+        ref = util.oracle_case(cfg, lens, *case, groups=[(0, 0), (1, 3)])
+        util.compare(cfg, O, LSE, ref)
+    ctx.close()
