@@ -146,9 +146,12 @@ ss_status ss_verify_chunk_hinted(ss_ctx* ctx, ss_tensor K, ss_tensor V, int32_t 
  * request b is the concatenation of pages page_table[b][0 .. pages_per_req) (device int32
  * [B, pages_per_req]), i.e. L_c = pages_per_req * page_size tokens of which valid_len[b] are
  * valid (NULL = all).  Same result as ss_verify_chunk on the gathered chunk.  The tensor-core
- * kernels need page_size to be a multiple of 128 (keys on M) or 64 (rows on M); other page sizes
- * take the CUDA-core kernel.  valid_len_host (HOST, may be NULL) is the scheduling hint of
- * ss_verify_chunk_hinted.  A page id outside [0, n_pages) raises SS_DEV_BAD_PAGE. */
+ * kernels take pages of 16, 32, 64 tokens (gathered page by page into their tiles) and any
+ * multiple of 64 (rows on M) or 128 (keys on M); other page sizes take the CUDA-core kernel,
+ * which is an order of magnitude slower.  Only the pages that hold valid tokens are looked up:
+ * table entries past ceil(valid_len[b] / page_size) may hold anything.  valid_len_host (HOST,
+ * may be NULL) is the scheduling hint of ss_verify_chunk_hinted.  A looked-up page id outside
+ * [0, n_pages) raises SS_DEV_BAD_PAGE and its tokens read as zeros. */
 ss_status ss_verify_chunk_paged(ss_ctx* ctx, ss_tensor K_pool, ss_tensor V_pool, int32_t n_pages,
                                 int32_t page_size, const int32_t* page_table, int32_t pages_per_req,
                                 const int32_t* valid_len, const int32_t* valid_len_host, void* stream);

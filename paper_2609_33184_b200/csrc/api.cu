@@ -397,14 +397,20 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   }
   CUtensorMap tmK, tmV;
   bool tc = c->tc_ok;
-  // paged chunks: a tile must not straddle pages
-  if (pg && (pg->page_size % kTileKeys)) tc = false;
+  // paged chunks: a tile is one page, a whole number of pages (16, 32 or 64 tokens each,
+  // gathered page by page) or part of a page; anything else takes the CUDA-core kernel
+  const auto pages_fit = [&](int tile) {
+    const int ps = pg->page_size;
+    return ps % tile == 0 || (ps >= 16 && tile % ps == 0);
+  };
   // up to 32 rows per kv-head the keys ride the MMA's M axis (tiles of 128 tokens); with more
   // rows the kernel with the rows on M is faster (measured).  SS_FLAG_ROWS_ON_M /
   // SS_FLAG_KEYS_ON_M (or SS_CHUNK_KERNEL=rows|keys) force one of them.
   const bool keys_on_m = tc && !c->force_rows_kernel && (R <= 32 || c->force_keys_kernel) &&
-                         (!pg || pg->page_size % 128 == 0);
-  const int box = keys_on_m ? 128 : kTileKeys;
+                         (!pg || pages_fit(128));
+  if (pg && !keys_on_m && !pages_fit(kTileKeys)) tc = false;
+  int box = keys_on_m ? 128 : kTileKeys;
+  if (pg && pg->page_size < box) box = pg->page_size;
   // tensor map over [outer, H_kv, tokens, d]: (requests, chunk tokens) or (pages, page tokens)
   const int tm_outer = pg ? pg->n_pages : c->B, tm_tokens = pg ? pg->page_size : L_c;
   if (tc)

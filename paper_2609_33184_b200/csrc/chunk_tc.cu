@@ -209,25 +209,35 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   }
 
   // ---- set-up: barriers, first loads, tensor memory, the Q tile --------------------------------
-  auto issue_k = [&](int it, uint64_t pol) {
-    const int s = it % kKStages;
+  // both 64-column halves of a box of tokens starting at (outer, tok) -> dst (K when !is_v)
+  auto load_rows = [&](bool is_v, uint32_t dst, int tok, int outer, uint64_t* bar, uint64_t pol) {
+    if (is_v) {  // (no runtime-selected pointer: the tensor maps stay in the parameter space)
+      tma_load_4d(dst, &tmV, 0, tok, kvh, outer, bar, pol);
+      tma_load_4d(dst + kHalfTile, &tmV, 64, tok, kvh, outer, bar, pol);
+    } else {
+      tma_load_4d(dst, &tmK, 0, tok, kvh, outer, bar, pol);
+      tma_load_4d(dst + kHalfTile, &tmK, 64, tok, kvh, outer, bar, pol);
+    }
+  };
+  // Pages smaller than a tile (16 or 32 tokens): the tile is gathered page by page by the whole
+  // producer warp, see below; this path is for contiguous chunks and pages of a tile or more.
+  const bool small_pages = p.page_table && p.page_size < kTileKeys;
+  auto issue_tile = [&](bool is_v, int it, uint32_t dst, uint64_t* bar, uint64_t pol) {
     int outer, tok;
     locate_token(p, b, tok0 + it * kTileKeys, &outer, &tok);
-    const uint32_t kdst = smem_u32(k_s + s * kTileBytes);
-    mbar_expect_tx(&ctl->kfull[s], kTileBytes);
-    tma_load_4d(kdst, &tmK, 0, tok, kvh, outer, &ctl->kfull[s], pol);
-    tma_load_4d(kdst + kHalfTile, &tmK, 64, tok, kvh, outer, &ctl->kfull[s], pol);
+    mbar_expect_tx(bar, kTileBytes);
+    load_rows(is_v, dst, tok, outer, bar, pol);
+  };
+  auto issue_k = [&](int it, uint64_t pol) {
+    const int s = it % kKStages;
+    issue_tile(false, it, smem_u32(k_s + s * kTileBytes), &ctl->kfull[s], pol);
   };
   auto issue_v = [&](int it, uint64_t pol) {
     const int s = it % kVStages;
-    int outer, tok;
-    locate_token(p, b, tok0 + it * kTileKeys, &outer, &tok);
-    const uint32_t vdst = smem_u32(v_s0 + s * kTileBytes);
-    mbar_expect_tx(&ctl->vfull[s], kTileBytes);
-    tma_load_4d(vdst, &tmV, 0, tok, kvh, outer, &ctl->vfull[s], pol);
-    tma_load_4d(vdst + kHalfTile, &tmV, 64, tok, kvh, outer, &ctl->vfull[s], pol);
+    issue_tile(true, it, smem_u32(v_s0 + s * kTileBytes), &ctl->vfull[s], pol);
   };
-  const int n_pre_k = min(n_tiles, kKStages), n_pre_v = min(n_tiles, kVStages);
+  // (small pages: all copies go out from the producer warp's loop)
+  const int n_pre_k = small_pages ? 0 : min(n_tiles, kKStages), n_pre_v = small_pages ? 0 : min(n_tiles, kVStages);
   if (warp == 4) {
     if (lane == 0) {
       for (int s = 0; s < kKStages; ++s) {
@@ -282,7 +292,93 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   const uint32_t tmem = ctl->tmem_base;
   unsigned long long* trl = lane == 0 ? tr : nullptr;
 
-  if (warp == 4) {
+  if (warp == 4 && small_pages) {
+    // ===== TMA producer, pages smaller than a tile =====
+    // The tensor map's box is one page; page i of a tile lands at row i * page_size of the slot,
+    // which keeps the swizzled layout of a single 64-token box.  Lane l copies 64-column half
+    // l % 2 of page l / 2 of the tile, so a tile's 4 or 8 copies and their page look-ups go out
+    // side by side; each lane fetches the page id of a ring's next tile right after its copy,
+    // off the path of the next one.  Pages that start at or past the valid length are not
+    // looked up (index n_pages is outside the pool and reads as zeros).  Lane 0 polls the two
+    // rings as in the loop below, arms the barriers and shares what to issue through a shuffle.
+    const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
+    const int ps = p.page_size, n_sub = kTileKeys / ps;  // 2 or 4 pages per tile
+    const int sub = lane >> 1, half = lane & 1;
+    const bool mine = lane < 2 * n_sub;
+    auto lane_page = [&](int tile) {  // page id of this lane's page of `tile`; -2: not looked up
+      const int tk = tok0 + tile * kTileKeys + sub * ps;
+      if (!mine || tk >= tok1) return -2;
+      const int pg = tk / ps;
+      return pg < p.pages_per_req ? p.page_table[(int64_t)b * p.pages_per_req + pg] : -1;
+    };
+    auto checked = [&](int id) {
+      if (id == -2) return p.n_pages;
+      if (id < 0 || id >= p.n_pages) {
+        atomicOr(p.status, SS_DEV_BAD_PAGE);
+        return p.n_pages;
+      }
+      return id;
+    };
+    int issued_k = 0, issued_v = 0;
+    int page_k = lane_page(0), page_v = page_k;
+    unsigned long long t0 = gtime_ns();
+    uint32_t spins = 0;
+    while (issued_k < n_tiles || issued_v < n_tiles) {
+      int act = 0;  // bit 0: K tile, bit 1: V tile, bit 2: give up
+      if (lane == 0) {
+        if (issued_k < n_tiles &&
+            mbar_test(&ctl->kempty[issued_k % kKStages], ((issued_k / kKStages) & 1) ^ 1)) {
+          mbar_expect_tx(&ctl->kfull[issued_k % kKStages], kTileBytes);
+          act |= 1;
+        }
+        if (issued_v < n_tiles &&
+            mbar_test(&ctl->vempty[issued_v % kVStages], ((issued_v / kVStages) & 1) ^ 1)) {
+          mbar_expect_tx(&ctl->vfull[issued_v % kVStages], kTileBytes);
+          act |= 2;
+        }
+        if (act) {
+          spins = 0;
+          t0 = gtime_ns();
+        } else if ((++spins & 255u) == 0) {  // bounded like every other wait
+          if (ctl->abort) {
+            act = 4;
+          } else if (gtime_ns() - t0 > kWaitNs) {
+            ctl->abort = 1;
+            atomicOr(p.status, SS_DEV_WAIT_EXPIRED);
+            act = 4;
+          }
+        }
+      }
+      act = __shfl_sync(0xffffffffu, act, 0);  // also orders the arming before the copies
+      if (act & 4) break;
+      if (act & 1) {
+        const int s = issued_k % kKStages;
+        if (mine)
+          tma_load_4d(smem_u32(k_s + s * kTileBytes) + half * kHalfTile + sub * ps * 128, &tmK, half * 64, 0,
+                      kvh, checked(page_k), &ctl->kfull[s], pol);
+        ++issued_k;
+        page_k = lane_page(issued_k);
+      }
+      if (act & 2) {
+        const int s = issued_v % kVStages;
+        if (mine)
+          tma_load_4d(smem_u32(v_s0 + s * kTileBytes) + half * kHalfTile + sub * ps * 128, &tmV, half * 64, 0,
+                      kvh, checked(page_v), &ctl->vfull[s], pol);
+        ++issued_v;
+        page_v = lane_page(issued_v);
+      }
+    }
+    if (lane == 0 && ctl->abort) {
+      // let the copies the warp started land before the CTA leaves (bounded)
+      const unsigned long long t1 = gtime_ns();
+      for (int it = max(0, issued_k - kKStages); it < issued_k; ++it)
+        while (!mbar_try_wait(&ctl->kfull[it % kKStages], (it / kKStages) & 1) && gtime_ns() - t1 < kWaitNs) {
+        }
+      for (int it = max(0, issued_v - kVStages); it < issued_v; ++it)
+        while (!mbar_try_wait(&ctl->vfull[it % kVStages], (it / kVStages) & 1) && gtime_ns() - t1 < kWaitNs) {
+        }
+    }
+  } else if (warp == 4) {
     // ===== TMA producer =====
     if (lane == 0) {
       // streamed once: evict first; shared by the row groups of a kv-head through L2: keep

@@ -127,22 +127,28 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
 
   // ---- set-up ------------------------------------------------------------------------------
   // use j of the ring: K of tile t is j = 2t, V of tile t is j = 2t + 1; unit j % UNITS
+  // both 64-column halves of `rows` tokens starting at (outer, tok) -> dst (K when !is_v)
+  auto load_rows = [&](bool is_v, uint32_t dst, int tok, int outer, uint64_t* bar, uint64_t pol) {
+    if (is_v) {  // (no runtime-selected pointer: the tensor maps stay in the parameter space)
+      tma_load_4d(dst, &tmV, 0, tok, kvh, outer, bar, pol);
+      tma_load_4d(dst + kHalf, &tmV, 64, tok, kvh, outer, bar, pol);
+    } else {
+      tma_load_4d(dst, &tmK, 0, tok, kvh, outer, bar, pol);
+      tma_load_4d(dst + kHalf, &tmK, 64, tok, kvh, outer, bar, pol);
+    }
+  };
+  // Pages smaller than a tile (16, 32 or 64 tokens): the tile is gathered page by page by the
+  // whole producer warp, see below; this path is for contiguous chunks and pages of a tile or more.
+  const bool small_pages = p.page_table && p.page_size < kKeys;
   auto issue_use = [&](int j, uint64_t pol) {
     const int u = j % UNITS;
     int outer, tok;
     locate_token(p, b, tok0 + (j >> 1) * kKeys, &outer, &tok);
-    const uint32_t dst = smem_u32(smem + u * kUnitBytes);
     mbar_expect_tx(&ctl->ufull[u], kUnitBytes);
-    if (j & 1) {  // (no runtime-selected pointer: the tensor maps stay in the parameter space)
-      tma_load_4d(dst, &tmV, 0, tok, kvh, outer, &ctl->ufull[u], pol);
-      tma_load_4d(dst + kHalf, &tmV, 64, tok, kvh, outer, &ctl->ufull[u], pol);
-    } else {
-      tma_load_4d(dst, &tmK, 0, tok, kvh, outer, &ctl->ufull[u], pol);
-      tma_load_4d(dst + kHalf, &tmK, 64, tok, kvh, outer, &ctl->ufull[u], pol);
-    }
+    load_rows(j & 1, smem_u32(smem + u * kUnitBytes), tok, outer, &ctl->ufull[u], pol);
   };
   const int n_uses = 2 * n_tiles;
-  const int n_pre = min(n_uses, UNITS);
+  const int n_pre = small_pages ? 0 : min(n_uses, UNITS);  // small pages: all copies go out below
   constexpr int kProducerWarp = 4 * WG, kMmaWarp = 4 * WG + 1;
   if (warp == kProducerWarp) {
     if (lane == 0) {
@@ -202,7 +208,59 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
   const uint32_t tmem = ctl->tmem_base;
   unsigned long long* trl = lane == 0 ? tr : nullptr;
 
-  if (warp == kProducerWarp) {
+  if (warp == kProducerWarp && small_pages) {
+    // ===== TMA producer, pages smaller than a tile =====
+    // The tensor map's box is one page; page i of a tile lands at row i * page_size of the ring
+    // unit, which keeps the swizzled layout of a single 128-token box.  Lane l copies 64-column
+    // half l % 2 of page l / 2 of the tile, so a unit's 4 to 16 copies and their page look-ups
+    // go out side by side; each lane fetches the page id of the next tile right after a tile's
+    // V copy, off the path of the next copy.  Pages that start at or past the valid length are
+    // not looked up (index n_pages is outside the pool and reads as zeros).  Lane 0 waits for
+    // the unit (bounded) and arms its barrier; the outcome is shared through a shuffle.
+    const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
+    const int ps = p.page_size, n_sub = kKeys / ps;  // 2, 4 or 8 pages per tile
+    const int sub = lane >> 1, half = lane & 1;
+    const bool mine = lane < 2 * n_sub;
+    auto lane_page = [&](int tile) {  // page id of this lane's page of `tile`; -2: not looked up
+      const int tk = tok0 + tile * kKeys + sub * ps;
+      if (!mine || tk >= tok1) return -2;
+      const int pg = tk / ps;
+      return pg < p.pages_per_req ? p.page_table[(int64_t)b * p.pages_per_req + pg] : -1;
+    };
+    int page = lane_page(0), issued = 0;
+    for (int j = 0; j < n_uses; ++j) {
+      const int u = j % UNITS;
+      const uint32_t ph = (j / UNITS) & 1;
+      int ok = 1;
+      if (lane == 0) {
+        ok = mwait(&ctl->uempty[u], ph ^ 1);
+        if (ok) mbar_expect_tx(&ctl->ufull[u], kUnitBytes);
+      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);  // also orders the arming before the copies
+      if (!ok) break;
+      if (mine) {
+        int id = page;
+        if (id == -2) {
+          id = p.n_pages;
+        } else if (id < 0 || id >= p.n_pages) {
+          atomicOr(p.status, SS_DEV_BAD_PAGE);
+          id = p.n_pages;
+        }
+        const uint32_t dst = smem_u32(smem + u * kUnitBytes) + half * kHalf + sub * ps * 128;
+        if (j & 1) tma_load_4d(dst, &tmV, half * 64, 0, kvh, id, &ctl->ufull[u], pol);
+        else tma_load_4d(dst, &tmK, half * 64, 0, kvh, id, &ctl->ufull[u], pol);
+      }
+      if (j & 1) page = lane_page((j >> 1) + 1);
+      issued = j + 1;
+    }
+    if (lane == 0 && ctl->abort) {
+      // let the copies the warp started land before the CTA leaves (bounded)
+      const unsigned long long t0 = gtime_ns();
+      for (int j = max(0, issued - UNITS); j < issued; ++j)
+        while (!mbar_try_wait(&ctl->ufull[j % UNITS], (j / UNITS) & 1) && gtime_ns() - t0 < kWaitNs) {
+        }
+    }
+  } else if (warp == kProducerWarp) {
     // ===== TMA producer =====
     if (lane == 0) {
       // streamed once: evict first; shared by the row groups of a kv-head through L2: keep

@@ -405,7 +405,8 @@ def test_random_ragged_shapes(seed):
     _run(cfg, lens=lens, flags=flags, order=order, local_at=rng.randint(0, n), max_chunks=rng.choice([0, 2]))
 
 
-@pytest.mark.parametrize("page_size,flags", [(128, 0), (128, 4), (64, 0), (64, 8), (16, 0), (128, 1), (256, 0)])
+@pytest.mark.parametrize("page_size,flags", [(128, 0), (128, 4), (64, 0), (64, 8), (64, 4), (32, 0), (32, 4), (16, 0),
+                                             (16, 4), (16, 8), (8, 0), (128, 1), (16, 1), (256, 0), (256, 4)])
 def test_paged_chunks_match_contiguous_and_oracle(page_size, flags):
     # the chunk's tokens live in shuffled pages of a pool; same result as the gathered chunk
     ssb = _ssb()
@@ -436,7 +437,8 @@ def test_paged_chunks_match_contiguous_and_oracle(page_size, flags):
     torch.cuda.synchronize()
     st, dev_bits = ctx.ss_poll_status()
     assert st == 0, dev_bits
-    expect = "simt" if (flags & 1 or page_size % 64) else ("tcgen05-keys" if (page_size % 128 == 0 and not flags & 4) else "tcgen05")
+    # pages of 16 tokens and more are gathered into the tensor-core kernels' tiles
+    expect = "simt" if (flags & 1 or page_size < 16) else ("tcgen05" if flags & 4 else "tcgen05-keys")
     assert ctx.last_chunk_kernel() == expect, (ctx.last_chunk_kernel(), expect)
     util.compare(cfg, O, LSE, ref)
     ctx.close()
@@ -461,6 +463,44 @@ def test_paged_chunk_bad_page_id_is_flagged():
         assert st == ssb.SS_ERR_DEVICE_FLAG and dev_bits & ssb.SS_DEV_BAD_PAGE
         assert torch.isfinite(O.float()).all()
         ctx.close()
+
+
+@pytest.mark.parametrize("flags", [0, 4, 1])
+def test_small_pages_bad_ids_and_unused_table_entries(flags):
+    # pages of 16 tokens: a bad id among the pages that hold valid tokens is flagged and reads as
+    # zeros; entries past the valid length hold garbage ids and must never be looked up
+    ssb = _ssb()
+    cfg = inputs.VerifyConfig("pg", 0x60, 2, 8, 2, 128, 256, 4, 100, 100)
+    lens = [100, 37]
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    K, V, vl = chunks[0]
+    ps, ppr = 16, 16
+    Kp = K.view(2, 2, ppr, ps, 128).permute(0, 2, 1, 3, 4).reshape(-1, 2, ps, 128).contiguous()
+    Vp = V.view(2, 2, ppr, ps, 128).permute(0, 2, 1, 3, 4).reshape(-1, 2, ps, 128).contiguous()
+    table = torch.arange(2 * ppr, dtype=torch.int32).view(2, ppr).clone()
+    table[0, 7:] = 1 << 30          # request 0 has 100 tokens = 7 pages (6 full + 4 tokens): rest unused
+    table[1, 3:] = -5               # request 1 has 37 tokens = 3 pages
+    table = table.to(DEV)
+    ref = util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits)
+    ctx = util.make_ctx(cfg, flags=flags)
+    O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
+    LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
+    ctx.ss_verify_begin(Q, cfg.scale)
+    ctx.ss_verify_chunk_paged(Kp, Vp, table, vl, vl.tolist())
+    ctx.ss_verify_local(K_loc, V_loc)
+    ctx.ss_verify_finalize(O, LSE)
+    assert ctx.ss_poll_status() == (0, 0)
+    util.compare(cfg, O, LSE, ref)
+    # now break a page that is in use
+    table[0, 2] = 2 * ppr + 9
+    ctx.ss_verify_begin(Q, cfg.scale)
+    ctx.ss_verify_chunk_paged(Kp, Vp, table, vl, vl.tolist())
+    ctx.ss_verify_local(K_loc, V_loc)
+    ctx.ss_verify_finalize(O, LSE)
+    st, dev_bits = ctx.ss_poll_status()
+    assert st == ssb.SS_ERR_DEVICE_FLAG and dev_bits & ssb.SS_DEV_BAD_PAGE
+    assert torch.isfinite(O.float()).all()
+    ctx.close()
 
 
 def test_round_can_be_captured_in_a_cuda_graph():
