@@ -72,7 +72,7 @@ typedef enum {
 typedef struct {
   int32_t max_B;      /* requests per call                                          */
   int32_t H_q, H_kv;  /* query heads, kv heads (H_q % H_kv == 0)                     */
-  int32_t d;          /* head dim, 64 or 128                                         */
+  int32_t d;          /* head dim, 64 or 128 (both on the tensor-core kernels)       */
   int32_t max_Tq;     /* candidate queries per request                               */
   int32_t max_Tloc;   /* local candidate KV tokens per request (<= 1024)             */
   int32_t max_Lc;     /* tokens per history chunk call                               */

@@ -288,7 +288,7 @@ ss_status ss_create(ss_ctx** out, const ss_config* cfg, void* workspace, size_t 
         qr == cudaDriverEntryPointSuccess)
       g_encode = (EncodeTiledFn)fn;
   }
-  c->tc_ok = (g_encode != nullptr) && (cfg->d == 128) && !(cfg->flags & SS_FLAG_FORCE_SIMT);
+  c->tc_ok = (g_encode != nullptr) && !(cfg->flags & SS_FLAG_FORCE_SIMT);
   if (c->tc_ok) c->tc_ok = encode_partials_map(c);
   if (c->tc_ok) {
     e = ss::chunk_tc_prepare();
@@ -406,9 +406,15 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   // up to 32 rows per kv-head the keys ride the MMA's M axis (tiles of 128 tokens); with more
   // rows the kernel with the rows on M is faster (measured).  SS_FLAG_ROWS_ON_M /
   // SS_FLAG_KEYS_ON_M (or SS_CHUNK_KERNEL=rows|keys) force one of them.
-  const bool keys_on_m = tc && !c->force_rows_kernel && (R <= 32 || c->force_keys_kernel) &&
+  // The rows-on-M kernel exists for head dim 128 only: head dim 64 always takes keys on M -
+  // unless the call is tiny (a few tiles in all): the CUDA-core kernel's small CTAs then finish
+  // sooner than one tensor-core CTA gets going (measured on the 1,024-token chain workload:
+  // 43 vs 46 us per round).  SS_FLAG_KEYS_ON_M overrides.
+  const bool d64 = c->cfg.d == 64;
+  if (d64 && !c->force_keys_kernel && (int64_t)pairs * n_tiles <= 8) tc = false;
+  const bool keys_on_m = tc && (d64 || (!c->force_rows_kernel && (R <= 32 || c->force_keys_kernel))) &&
                          (!pg || pages_fit(128));
-  if (pg && !keys_on_m && !pages_fit(kTileKeys)) tc = false;
+  if (!keys_on_m && (d64 || (pg && !pages_fit(kTileKeys)))) tc = false;
   int box = keys_on_m ? 128 : kTileKeys;
   if (pg && pg->page_size < box) box = pg->page_size;
   // tensor map over [outer, H_kv, tokens, d]: (requests, chunk tokens) or (pages, page tokens)

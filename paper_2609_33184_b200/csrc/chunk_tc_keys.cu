@@ -47,10 +47,8 @@ namespace {
 
 using namespace ss::tc;
 
-constexpr int kD = 128;
 constexpr int kKeys = 128;                  // keys per tile = MMA M
-constexpr int kHalf = kKeys * 64 * 2;       // 16 KB: [128 keys][64 d] bf16
-constexpr int kUnitBytes = 2 * kHalf;       // 32 KB: one K tile or one V tile
+constexpr int kHalf = kKeys * 64 * 2;       // 16 KB: [128 keys][64 d] bf16, one TMA box
 constexpr float kLazyThreshold = 16.f;
 
 template <int N>
@@ -65,32 +63,40 @@ struct alignas(16) Ctl {
 };
 
 // NC = score columns per softmax thread, WG = softmax warpgroups (threads sharing a TMEM lane),
-// UNITS = ring units.  N = NC * WG is the widest row group the instantiation takes.
-template <int NC, int WG, int UNITS>
+// UNITS = ring units, D = head dim (64 or 128).  N = NC * WG is the widest row group the
+// instantiation takes.  A K or V tile is D / 64 boxes of [128 keys][64 d].
+// Head dim 64: the output MMA still runs with M = 128; the upper 64 rows of its A operand
+// (V^T) are whatever lies one box further in shared memory, their results land in TMEM lanes
+// 64..127 and are never read.  kSmem keeps that box inside the CTA's window.
+template <int NC, int WG, int UNITS, int D>
 struct Cfg {
   static constexpr int N = NC * WG;
+  static constexpr int kHalves = D / 64;
+  static constexpr int kUnitBytes = kHalves * kHalf;  // one K tile or one V tile
   static constexpr int kSoft = 128 * WG;              // softmax threads
   static constexpr int kThreads = kSoft + 64;
   static constexpr int kQHalf = N * 64 * 2;           // [N rows][64 d]
   static constexpr int kOffQ = UNITS * kUnitBytes;
-  static constexpr int kOffP = kOffQ + 2 * kQHalf;
+  static constexpr int kOffP = kOffQ + kHalves * kQHalf;
   static constexpr int kOffCtl = kOffP + kKeys * N * 2;
   static constexpr int kCtlBytes = (sizeof(Ctl<N>) + 1023) / 1024 * 1024;
-  static constexpr int kSmem = kOffCtl + kCtlBytes;
+  static constexpr int kSmemUsed = kOffCtl + kCtlBytes;
+  static constexpr int kSmem = (D == 64 && kSmemUsed < kOffQ + kHalf) ? kOffQ + kHalf : kSmemUsed;
   static constexpr uint32_t kTmemCols = (3 * N <= 128) ? 128 : (3 * N <= 256 ? 256 : 512);
   static constexpr uint32_t kColO = 2 * N;            // S^T buffers at 0 and N, O^T at 2N
-  static constexpr int kMinBlocks = (kSmem <= 113 * 1024 && kTmemCols <= 256) ? 2 : 1;
+  static constexpr int kMinBlocks = (kSmem <= 113 * 1024 && kTmemCols <= 256 && WG == 1) ? 2 : 1;
   static_assert(kSmem <= 227 * 1024, "shared memory");
-  static_assert(NC % 16 == 0 && UNITS <= 8, "shape");
+  static_assert(NC % 16 == 0 && UNITS <= 8 && (D == 64 || D == 128), "shape");
 };
 
 
-template <int NC, int WG, int UNITS>
-__global__ void __launch_bounds__(Cfg<NC, WG, UNITS>::kThreads, Cfg<NC, WG, UNITS>::kMinBlocks)
+template <int NC, int WG, int UNITS, int D>
+__global__ void __launch_bounds__(Cfg<NC, WG, UNITS, D>::kThreads, Cfg<NC, WG, UNITS, D>::kMinBlocks)
 chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
                      const __grid_constant__ CUtensorMap tmV) {
-  using C = Cfg<NC, WG, UNITS>;
+  using C = Cfg<NC, WG, UNITS, D>;
   constexpr int N = C::N;
+  constexpr int kD = D, kUnitBytes = C::kUnitBytes;
   extern __shared__ __align__(1024) uint8_t smem[];
   Ctl<N>* ctl = reinterpret_cast<Ctl<N>*>(smem + C::kOffCtl);
   uint8_t* q_s = smem + C::kOffQ;
@@ -131,10 +137,10 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
   auto load_rows = [&](bool is_v, uint32_t dst, int tok, int outer, uint64_t* bar, uint64_t pol) {
     if (is_v) {  // (no runtime-selected pointer: the tensor maps stay in the parameter space)
       tma_load_4d(dst, &tmV, 0, tok, kvh, outer, bar, pol);
-      tma_load_4d(dst + kHalf, &tmV, 64, tok, kvh, outer, bar, pol);
+      if (D == 128) tma_load_4d(dst + kHalf, &tmV, 64, tok, kvh, outer, bar, pol);
     } else {
       tma_load_4d(dst, &tmK, 0, tok, kvh, outer, bar, pol);
-      tma_load_4d(dst + kHalf, &tmK, 64, tok, kvh, outer, bar, pol);
+      if (D == 128) tma_load_4d(dst + kHalf, &tmK, 64, tok, kvh, outer, bar, pol);
     }
   };
   // Pages smaller than a tile (16, 32 or 64 tokens): the tile is gathered page by page by the
@@ -219,8 +225,8 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
     // the unit (bounded) and arms its barrier; the outcome is shared through a shuffle.
     const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
     const int ps = p.page_size, n_sub = kKeys / ps;  // 2, 4 or 8 pages per tile
-    const int sub = lane >> 1, half = lane & 1;
-    const bool mine = lane < 2 * n_sub;
+    const int sub = lane / C::kHalves, half = lane % C::kHalves;
+    const bool mine = lane < C::kHalves * n_sub;
     auto lane_page = [&](int tile) {  // page id of this lane's page of `tile`; -2: not looked up
       const int tk = tok0 + tile * kKeys + sub * ps;
       if (!mine || tk >= tok1) return -2;
@@ -403,9 +409,10 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
         wait(&ctl->ufull[jv % UNITS], (jv / UNITS) & 1);
         if (!dead) {
           uint8_t* v_s = smem + (jv % UNITS) * kUnitBytes;
-          const int n_vec = (kKeys - n_valid) * 16;
+          constexpr int kVecRow = 8 * C::kHalves;  // 16-byte pieces per token row
+          const int n_vec = (kKeys - n_valid) * kVecRow;
           for (int i = tid; i < n_vec; i += C::kSoft) {
-            const int row = n_valid + (i >> 4), half = (i >> 3) & 1, ch = i & 7;
+            const int row = n_valid + i / kVecRow, half = (i % kVecRow) >> 3, ch = i & 7;
             *reinterpret_cast<uint4*>(v_s + half * kHalf + row * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
           }
         }
@@ -625,7 +632,7 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
 #pragma unroll
           for (int c = 0; c < 16; ++c) {
             const int r = c0 + q * 16 + c;
-            if (r < nrows) out_a[(size_t)r * kD + L] = __uint_as_float(o[c]);
+            if (r < nrows && L < kD) out_a[(size_t)r * kD + L] = __uint_as_float(o[c]);
           }
         }
       }
@@ -644,36 +651,45 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
   if (!p.wait_first && chain_cta) pdl_wait_prior();
 }
 
-template <int NC, int WG, int UNITS>
+template <int NC, int WG, int UNITS, int D>
 cudaError_t launch_cfg(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
                        cudaStream_t s, bool pdl) {
-  using C = Cfg<NC, WG, UNITS>;
+  using C = Cfg<NC, WG, UNITS, D>;
   dim3 grid(p.splits * p.row_tiles, p.H_kv, p.B), block(C::kThreads);
-  return launch_kernel(chunk_tc_keys_kernel<NC, WG, UNITS>, grid, block, C::kSmem, s, pdl, p, tmK, tmV);
+  return launch_kernel(chunk_tc_keys_kernel<NC, WG, UNITS, D>, grid, block, C::kSmem, s, pdl, p, tmK, tmV);
 }
 
-template <int NC, int WG, int UNITS>
+template <int NC, int WG, int UNITS, int D>
 cudaError_t prepare_cfg() {
-  return cudaFuncSetAttribute(chunk_tc_keys_kernel<NC, WG, UNITS>,
-                              cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<NC, WG, UNITS>::kSmem);
+  return cudaFuncSetAttribute(chunk_tc_keys_kernel<NC, WG, UNITS, D>,
+                              cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<NC, WG, UNITS, D>::kSmem);
 }
 
 }  // namespace
 
 cudaError_t chunk_tc_keys_prepare() {
-  cudaError_t e = prepare_cfg<32, 1, 3>();
-  if (e == cudaSuccess) e = prepare_cfg<32, 2, 6>();
-  if (e == cudaSuccess) e = prepare_cfg<32, 4, 5>();
+  cudaError_t e = prepare_cfg<32, 1, 3, 128>();
+  if (e == cudaSuccess) e = prepare_cfg<32, 2, 6, 128>();
+  if (e == cudaSuccess) e = prepare_cfg<32, 4, 5, 128>();
+  if (e == cudaSuccess) e = prepare_cfg<32, 1, 6, 64>();
+  if (e == cudaSuccess) e = prepare_cfg<32, 2, 8, 64>();
+  if (e == cudaSuccess) e = prepare_cfg<32, 4, 8, 64>();
   return e;
 }
 
 // Rows per CTA (p.rows_per_tile): <= 32 -> two CTAs per SM with 4 softmax warps; <= 64 and
 // <= 128 -> one CTA per SM with 8 and 16 softmax warps (32 score columns per thread each).
+// Head dim 64 halves a tile's bytes, so its rings have twice the units.
 cudaError_t launch_chunk_tc_keys(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
                                  cudaStream_t s, bool pdl) {
-  if (p.rows_per_tile <= 32) return launch_cfg<32, 1, 3>(p, tmK, tmV, s, pdl);
-  if (p.rows_per_tile <= 64) return launch_cfg<32, 2, 6>(p, tmK, tmV, s, pdl);
-  return launch_cfg<32, 4, 5>(p, tmK, tmV, s, pdl);
+  if (p.d == 64) {
+    if (p.rows_per_tile <= 32) return launch_cfg<32, 1, 6, 64>(p, tmK, tmV, s, pdl);
+    if (p.rows_per_tile <= 64) return launch_cfg<32, 2, 8, 64>(p, tmK, tmV, s, pdl);
+    return launch_cfg<32, 4, 8, 64>(p, tmK, tmV, s, pdl);
+  }
+  if (p.rows_per_tile <= 32) return launch_cfg<32, 1, 3, 128>(p, tmK, tmV, s, pdl);
+  if (p.rows_per_tile <= 64) return launch_cfg<32, 2, 6, 128>(p, tmK, tmV, s, pdl);
+  return launch_cfg<32, 4, 5, 128>(p, tmK, tmV, s, pdl);
 }
 
 }  // namespace ss

@@ -33,9 +33,10 @@ def _run(cfg, lens=None, flags=0, fill=None, order=None, local_at=None, strict=T
     return O, LSE, worst
 
 
-def test_c1_tiny_chain_exact_config():
+@pytest.mark.parametrize("flags,kernel", [(0, "simt"), (8, "tcgen05-keys")])
+def test_c1_tiny_chain_exact_config(flags, kernel):
     cfg = inputs.CONFIGS["c1_tiny_chain"]
-    _run(cfg, kernel="simt")
+    _run(cfg, flags=flags, kernel=kernel)
 
 
 def _small(name, **kw):
@@ -591,4 +592,54 @@ def test_rounds_narrower_than_the_context_limit(flags):
         assert ctx.ss_poll_status() == (0, 0)
         ref = util.oracle_case(cfg, lens, *case, groups=[(0, 0), (1, 3)])
         util.compare(cfg, O, LSE, ref)
+    ctx.close()
+
+
+@pytest.mark.parametrize("T_q,G,n", [(2, 4, 300), (5, 4, 129), (8, 4, 1000), (9, 4, 127), (7, 8, 640), (33, 2, 500),
+                                      (17, 8, 257), (40, 4, 384), (3, 1, 1), (6, 4, 0)])
+def test_head_dim_64_runs_on_the_tensor_cores(T_q, G, n):
+    # head dim 64: the keys-on-M kernel with one 64-column box per tile (its output MMA pads M
+    # with rows that are never read), every row-group width, ragged tails, several chunks
+    cfg = inputs.VerifyConfig("v", 0x90 + T_q + G + n, 3, 2 * G, 2, 64, 256, T_q, n, n, k_mult=2.0,
+                              mask="tree" if T_q % 2 else "chain")
+    lens = [n, max(0, n - 77), n // 2]
+    O, LSE, _ = _run(cfg, lens=lens, fill=float("nan"), kernel="tcgen05-keys")
+    # and the CUDA-core kernel agrees
+    case = util.gen_case(cfg, lens, DEV, float("nan"))
+    ctx = util.make_ctx(cfg, flags=1)
+    O2, L2 = util.gpu_case(ctx, cfg, *case)
+    ctx.close()
+    assert (O.float() - O2.float()).abs().max() < 2e-2
+    fin = torch.isfinite(L2)
+    assert torch.equal(torch.isfinite(LSE), fin) and (LSE[fin] - L2[fin]).abs().max() < 1e-4
+
+
+@pytest.mark.parametrize("page_size", [16, 64, 128])
+def test_head_dim_64_paged(page_size):
+    ssb = _ssb()
+    cfg = inputs.VerifyConfig("pg", 0xA0 + page_size, 3, 8, 2, 64, 512, 6, 40, 1500, k_mult=2.0)
+    lens = [1500, 40, 1024]
+    case = util.gen_case(cfg, lens, DEV, fill=float("nan"))
+    Q, chunks, K_loc, V_loc, bits = case
+    ref = util.oracle_case(cfg, lens, *case)
+    ppr = cfg.L_c // page_size
+    g = torch.Generator().manual_seed(page_size)
+    ctx = util.make_ctx(cfg)
+    O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
+    LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
+    ctx.ss_verify_begin(Q, cfg.scale)
+    for K, V, vl in chunks:
+        n_pages = cfg.B * ppr + 3
+        table = torch.randperm(n_pages, generator=g)[:cfg.B * ppr].to(torch.int32).view(cfg.B, ppr).contiguous()
+        K_pool = torch.full((n_pages, cfg.H_kv, page_size, cfg.d), float("nan"), dtype=torch.bfloat16, device=DEV)
+        V_pool = torch.full_like(K_pool, float("nan"))
+        K_pool[table.view(-1).long()] = K.view(cfg.B, cfg.H_kv, ppr, page_size, cfg.d).permute(0, 2, 1, 3, 4).reshape(-1, cfg.H_kv, page_size, cfg.d)
+        V_pool[table.view(-1).long()] = V.view(cfg.B, cfg.H_kv, ppr, page_size, cfg.d).permute(0, 2, 1, 3, 4).reshape(-1, cfg.H_kv, page_size, cfg.d)
+        ctx.ss_verify_chunk_paged(K_pool, V_pool, table.to(DEV), vl, vl.tolist())
+    ctx.ss_verify_local(K_loc, V_loc)
+    ctx.ss_verify_finalize(O, LSE)
+    torch.cuda.synchronize()
+    assert ctx.ss_poll_status() == (0, 0)
+    assert ctx.last_chunk_kernel() == "tcgen05-keys"
+    util.compare(cfg, O, LSE, ref)
     ctx.close()
