@@ -79,3 +79,12 @@ def test_c5_streamed_full():
     assert np.array_equal(_u16(acc["hk"]), ko) and np.array_equal(_u16(acc["hv"]), vo)
     print("c5", worst, "GB/s", stats.h2d_bytes / stats.ms_device / 1e6)
     ctx.close()
+
+
+def test_sweep_tool_runs_a_small_shape():
+    # the sizing aid goes through the same C ABI; keep it working
+    from paper_2609_33184_b200 import sweep
+    for d, page in ((128, 0), (64, 0), (128, 16)):
+        gbps, ms, kernel = sweep.measure(rows=8, d=d, page_size=page, B=2, H_kv=2, L_c=512, tokens=2048,
+                                         flags=0, rounds=2, dev="cuda:0")
+        assert gbps > 0 and ms > 0 and kernel.startswith("tcgen05")
