@@ -91,8 +91,7 @@ typedef struct {
  * same stream between two ss_ calls. */
 #define SS_FLAG_OVERLAP_CHUNKS 2u
 /* Use the tensor-core chunk kernel that puts the query rows on the MMA's M axis instead of
- * the default one that puts the keys there.  For cross-checks.  Head dim 128 only: at head
- * dim 64 the flag is ignored (there the keys-on-M kernel serves every row count). */
+ * the default one that puts the keys there.  For cross-checks. */
 #define SS_FLAG_ROWS_ON_M 4u
 /* Use the keys-on-M kernel for any number of rows per kv-head (default: up to 32). */
 #define SS_FLAG_KEYS_ON_M 8u

@@ -406,15 +406,17 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   // up to 32 rows per kv-head the keys ride the MMA's M axis (tiles of 128 tokens); with more
   // rows the kernel with the rows on M is faster (measured).  SS_FLAG_ROWS_ON_M /
   // SS_FLAG_KEYS_ON_M (or SS_CHUNK_KERNEL=rows|keys) force one of them.
-  // The rows-on-M kernel exists for head dim 128 only: head dim 64 always takes keys on M -
-  // unless the call is tiny (a few tiles in all): the CUDA-core kernel's small CTAs then finish
-  // sooner than one tensor-core CTA gets going (measured on the 1,024-token chain workload:
-  // 43 vs 46 us per round).  SS_FLAG_KEYS_ON_M overrides.
-  const bool d64 = c->cfg.d == 64;
-  if (d64 && !c->force_keys_kernel && (int64_t)pairs * n_tiles <= 8) tc = false;
-  const bool keys_on_m = tc && (d64 || (!c->force_rows_kernel && (R <= 32 || c->force_keys_kernel))) &&
+  // Head dim 64, tiny call (a few tiles in all): the CUDA-core kernel's small CTAs finish sooner
+  // than one tensor-core CTA gets going (measured on the 1,024-token chain workload: 43 vs 46 us
+  // per round).  SS_FLAG_KEYS_ON_M / SS_FLAG_ROWS_ON_M override.
+  if (c->cfg.d == 64 && !c->force_keys_kernel && !c->force_rows_kernel && (int64_t)pairs * n_tiles <= 8)
+    tc = false;
+  // (At head dim 64 a tile has half the bytes for the same softmax work and the rows-on-M kernel
+  // already wins above 16 rows: 4.8 vs 4.5 TB/s at 32 rows, 4.9 vs 5.1 at 16.)
+  const int keys_max_rows = c->cfg.d == 64 ? 16 : 32;
+  const bool keys_on_m = tc && !c->force_rows_kernel && (R <= keys_max_rows || c->force_keys_kernel) &&
                          (!pg || pages_fit(128));
-  if (!keys_on_m && (d64 || (pg && !pages_fit(kTileKeys)))) tc = false;
+  if (pg && !keys_on_m && !pages_fit(kTileKeys)) tc = false;
   int box = keys_on_m ? 128 : kTileKeys;
   if (pg && pg->page_size < box) box = pg->page_size;
   // tensor map over [outer, H_kv, tokens, d]: (requests, chunk tokens) or (pages, page tokens)

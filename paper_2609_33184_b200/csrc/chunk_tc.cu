@@ -6,6 +6,10 @@
 // the kv-head (T_q candidate queries x G query heads) ride in the M dimension of the MMAs,
 // so every K/V byte is fetched from HBM once and serves the whole query group.
 //
+// The kernel is a template over the head dim (64 or 128); the figures below are for 128.  At 64
+// a tile is one [64][64] box per operand, the rings hold four K and six V slots (the same
+// bytes), the score MMA takes four k-steps and the output MMA has N = 64.
+//
 //   warp 4 (one lane)  TMA producer: K tiles and V tiles of 64 tokens, two K slots and three V
 //                      slots, 128-byte swizzle, evict-first L2 policy (the history is
 //                      streamed).  A K slot is released as soon as its score MMAs retire
@@ -46,36 +50,46 @@ namespace ss {
 namespace {
 
 constexpr int kThreads = 192;
-constexpr int kKStages = 2, kVStages = 3;
-constexpr int kD = 128;
-constexpr int kHalfTile = kTileKeys * 64 * 2;       // 8 KB: [64 keys][64 d] bf16
-constexpr int kTileBytes = 2 * kHalfTile;           // 16 KB: one K tile or one V tile
+constexpr int kHalfTile = kTileKeys * 64 * 2;       // 8 KB: [64 keys][64 d] bf16, one TMA box
 constexpr int kQHalf = 128 * 64 * 2;                // 16 KB: [128 rows][64 d] bf16
-constexpr int kQBytes = 2 * kQHalf;                 // 32 KB: the Q tile
-constexpr int kOffK = kQBytes;                              // K slots
-constexpr int kOffV = kOffK + kKStages * kTileBytes;        // V slots
-constexpr int kSmemData = kOffV + kVStages * kTileBytes;    // 112 KB
 constexpr int kSmemCtl = 256;
-constexpr int kSmemTotal = kSmemData + kSmemCtl;
-// two CTAs per SM: 227 KB per SM less 1 KB reserved per CTA
-static_assert(2 * (kSmemTotal + 1024) <= 227 * 1024, "two CTAs per SM");
 constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kColS = 0, kColO = 128;          // S buffer t%2 at kColS + 64 (t%2)
 constexpr float kRescaleThreshold = 8.f;
 
-struct Ctl {
-  uint64_t kfull[kKStages], kempty[kKStages], vfull[kVStages], vempty[kVStages];
+// Shared-memory layout for head dim D (64 or 128): the Q tile, then the K slots, then the V
+// slots, D / 64 boxes of 64 columns each.  Head dim 64 halves a tile's bytes, so it takes twice
+// the slots (the same bytes in flight).
+template <int D>
+struct Lay {
+  static constexpr int kHalves = D / 64;
+  static constexpr int kKStages = D == 128 ? 2 : 4, kVStages = D == 128 ? 3 : 6;
+  static constexpr int kTileBytes = kHalves * kHalfTile;      // one K tile or one V tile
+  static constexpr int kQBytes = kHalves * kQHalf;            // the Q tile
+  static constexpr int kOffK = kQBytes;                       // K slots
+  static constexpr int kOffV = kOffK + kKStages * kTileBytes; // V slots
+  static constexpr int kSmemData = kOffV + kVStages * kTileBytes;  // 112 KB (d = 128), 96 KB (64)
+  static constexpr int kSmemTotal = kSmemData + kSmemCtl;
+  // two CTAs per SM: 227 KB per SM less 1 KB reserved per CTA
+  static_assert(2 * (kSmemTotal + 1024) <= 227 * 1024, "two CTAs per SM");
+  static_assert(D == 64 || D == 128, "head dim");
+};
+
+template <int KS, int VS>
+struct CtlT {
+  uint64_t kfull[KS], kempty[KS], vfull[VS], vempty[VS];
   uint64_t sfull[2], pready[2];  // per score buffer
   uint64_t odone;                // one phase per tile: PV(t) has retired
   uint64_t pvdone;               // the last PV has retired
   uint32_t tmem_base;
   volatile uint32_t abort;
 };
-static_assert(sizeof(Ctl) <= kSmemCtl, "control block");
+static_assert(sizeof(CtlT<2, 3>) <= kSmemCtl && sizeof(CtlT<4, 6>) <= kSmemCtl, "control block");
 
 
 using namespace ss::tc;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Ctl* ctl, uint32_t* status) {
+template <typename C>
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, C* ctl, uint32_t* status) {
   return mbar_wait_abortable(bar, parity, &ctl->abort, status);
 }
 
@@ -100,10 +114,10 @@ __device__ __forceinline__ void store_p(uint32_t t_s, const uint32_t (&pk)[NC / 
 // positive (checked at ss_verify_begin), so the maximum is taken on the raw scores and the
 // scaling rides in the FMA that subtracts the reference.
 // Returns false when the wait for PV(it - 1) in the rescale path gave up.
-template <int NC, bool MASK>
+template <int NC, bool MASK, int D, typename C>
 __device__ __forceinline__ bool softmax_tile(uint32_t t_s, uint32_t t_o, int c0, int n_valid,
                                              int it, float scale_log2, float& m, float& l,
-                                             Ctl* ctl, uint32_t* status) {
+                                             C* ctl, uint32_t* status) {
   const bool have_o = it > 0;
   uint32_t raw[NC / 16][16];
 #pragma unroll
@@ -133,7 +147,7 @@ __device__ __forceinline__ bool softmax_tile(uint32_t t_s, uint32_t t_o, int c0,
     if (!mbar_wait(&ctl->odone, (it - 1) & 1, ctl, status)) return false;
     tc_fence_after();
 #pragma unroll 1
-    for (int q = 0; q < kD / 16; ++q) {
+    for (int q = 0; q < D / 16; ++q) {
       uint32_t o[16];
       tmem_ld16(t_o + q * 16, o);
       tc_wait_ld();
@@ -177,11 +191,16 @@ __device__ __forceinline__ bool softmax_tile(uint32_t t_s, uint32_t t_o, int c0,
   return true;
 }
 
+template <int D>
 __global__ void __launch_bounds__(kThreads, 2)
 chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmA) {
+  using L_ = Lay<D>;
+  constexpr int kD = D, kHalves = L_::kHalves, kKStages = L_::kKStages, kVStages = L_::kVStages;
+  constexpr int kTileBytes = L_::kTileBytes, kOffK = L_::kOffK, kOffV = L_::kOffV, kSmemData = L_::kSmemData;
+  using Ctl = CtlT<kKStages, kVStages>;
   extern __shared__ __align__(1024) uint8_t smem[];
-  uint8_t* q_s = smem;             // Q tile: two halves [128 rows][64 d], 128-byte swizzle
+  uint8_t* q_s = smem;             // Q tile: D / 64 halves [128 rows][64 d], 128-byte swizzle
   uint8_t* k_s = smem + kOffK;     // K slots
   uint8_t* v_s0 = smem + kOffV;    // V slots
   Ctl* ctl = reinterpret_cast<Ctl*>(smem + kSmemData);
@@ -213,10 +232,10 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   auto load_rows = [&](bool is_v, uint32_t dst, int tok, int outer, uint64_t* bar, uint64_t pol) {
     if (is_v) {  // (no runtime-selected pointer: the tensor maps stay in the parameter space)
       tma_load_4d(dst, &tmV, 0, tok, kvh, outer, bar, pol);
-      tma_load_4d(dst + kHalfTile, &tmV, 64, tok, kvh, outer, bar, pol);
+      if (D == 128) tma_load_4d(dst + kHalfTile, &tmV, 64, tok, kvh, outer, bar, pol);
     } else {
       tma_load_4d(dst, &tmK, 0, tok, kvh, outer, bar, pol);
-      tma_load_4d(dst + kHalfTile, &tmK, 64, tok, kvh, outer, bar, pol);
+      if (D == 128) tma_load_4d(dst + kHalfTile, &tmK, 64, tok, kvh, outer, bar, pol);
     }
   };
   // Pages smaller than a tile (16 or 32 tokens): the tile is gathered page by page by the whole
@@ -280,7 +299,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
                                            t * p.q_st);
     }
 #pragma unroll
-    for (int v = 0; v < 16; ++v) {
+    for (int v = 0; v < kD / 8; ++v) {
       const uint4 x = src ? src[v] : make_uint4(0, 0, 0, 0);
       *reinterpret_cast<uint4*>(q_s + (v >> 3) * kQHalf + tid * 128 + (((v & 7) ^ (tid & 7)) << 4)) = x;
     }
@@ -303,8 +322,8 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     // rings as in the loop below, arms the barriers and shares what to issue through a shuffle.
     const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
     const int ps = p.page_size, n_sub = kTileKeys / ps;  // 2 or 4 pages per tile
-    const int sub = lane >> 1, half = lane & 1;
-    const bool mine = lane < 2 * n_sub;
+    const int sub = lane / kHalves, half = lane % kHalves;
+    const bool mine = lane < kHalves * n_sub;
     auto lane_page = [&](int tile) {  // page id of this lane's page of `tile`; -2: not looked up
       const int tk = tok0 + tile * kTileKeys + sub * ps;
       if (!mine || tk >= tok1) return -2;
@@ -485,7 +504,8 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     // tensor pipe runs this thread's MMAs in issue order, so they have consumed P before the
     // new scores overwrite it) or the output MMAs of tile pi (P ready, V landed).  The Q tile
     // was written before the CTA-wide barrier above (with a proxy fence).
-    static_assert(kKStages == 2, "the score MMAs of tile t + 2 reuse the K slot and the S buffer of tile t");
+    // (The two score buffers bound qi to pi + 1; the K ring may be deeper than that.)
+    static_assert(kKStages >= 2, "the score MMAs run up to two tiles ahead of the output MMAs");
     int qi = 0, pi = 0;
     unsigned long long t0 = gtime_ns();
     uint32_t spins = 0;
@@ -551,16 +571,17 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         ok = mbar_wait(&ctl->vfull[s], ph, ctl, p.status);
         if (!ok) break;
         uint8_t* v_s = v_s0 + s * kTileBytes;
-        const int n_vec = (kTileKeys - n_valid) * 16;
+        constexpr int kVecRow = kD / 8;  // 16-byte pieces per token row
+        const int n_vec = (kTileKeys - n_valid) * kVecRow;
         for (int i = L; i < n_vec; i += 128) {
-          const int row = n_valid + (i >> 4), half = (i >> 3) & 1, ch = i & 7;
+          const int row = n_valid + i / kVecRow, half = (i % kVecRow) >> 3, ch = i & 7;
           *reinterpret_cast<uint4*>(v_s + half * kHalfTile + row * 128 + ch * 16) =
               make_uint4(0, 0, 0, 0);
         }
         fence_proxy_async();
       }
 #define SS_SOFTMAX_TILE(NC_, MASK_) \
-  softmax_tile<NC_, MASK_>(t_s, t_o, c0, n_valid, it, p.scale_log2, m, l, ctl, p.status)
+  softmax_tile<NC_, MASK_, D>(t_s, t_o, c0, n_valid, it, p.scale_log2, m, l, ctl, p.status)
       if (n_valid < kTileKeys) {
         if (nc == 16)
           ok = SS_SOFTMAX_TILE(16, true);
@@ -596,7 +617,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       // behind them in the V slots.
       float* o_s = reinterpret_cast<float*>(smem);
       float2* ml_s = reinterpret_cast<float2*>(v_s0);
-      static_assert(kOffV >= 128 * 128 * 4, "O staging must end before the (m, l) array");
+      static_assert(kOffV >= 128 * kD * 4, "O staging must end before the (m, l) array");
       auto o_at = [&](int row, int c4) {  // float4 number c4 (0..31) of a staged row
         return reinterpret_cast<float4*>(o_s + (c4 >> 3) * (128 * 32) + row * 32 +
                                          (((c4 & 7) ^ (row & 7)) << 2));
@@ -634,7 +655,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         // lane (r, grp) sums columns [grp * 128/groups, (grp + 1) * 128/groups) of row r over
         // the row's `groups` staged copies and puts them back over the first copy
         named_bar_sync(1, 128);
-        const int n4 = 32 / groups, c40 = grp * n4;
+        const int n4 = (kD / 4) / groups, c40 = grp * n4;
         for (int c = 0; c < n4; c += 4) {
           float4 acc[4];
 #pragma unroll
@@ -660,7 +681,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       named_bar_sync(1, 128);
       if (L == 0) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
+        for (int j = 0; j < kD / 32; ++j)
           tma_store_3d(&tmA, smem_u32(o_s + j * (128 * 32)), j * 32, row0, p.a_slot0 + w.slot);
         bulk_commit();
         bulk_wait_read();  // shared memory is released when the CTA leaves
@@ -683,14 +704,20 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
 }  // namespace
 
 cudaError_t chunk_tc_prepare() {
-  return cudaFuncSetAttribute(chunk_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              kSmemTotal);
+  cudaError_t e = cudaFuncSetAttribute(chunk_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       Lay<128>::kSmemTotal);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(chunk_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Lay<64>::kSmemTotal);
+  return e;
 }
 
 cudaError_t launch_chunk_tc(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
                             const CUtensorMap& tmA, cudaStream_t s, bool pdl) {
   dim3 grid(p.splits * p.row_tiles, p.H_kv, p.B), block(kThreads);
-  return launch_kernel(chunk_tc_kernel, grid, block, kSmemTotal, s, pdl, p, tmK, tmV, tmA);
+  if (p.d == 64)
+    return launch_kernel(chunk_tc_kernel<64>, grid, block, Lay<64>::kSmemTotal, s, pdl, p, tmK, tmV, tmA);
+  return launch_kernel(chunk_tc_kernel<128>, grid, block, Lay<128>::kSmemTotal, s, pdl, p, tmK, tmV, tmA);
 }
 
 }  // namespace ss

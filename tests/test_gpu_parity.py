@@ -597,13 +597,16 @@ def test_rounds_narrower_than_the_context_limit(flags):
 
 @pytest.mark.parametrize("T_q,G,n", [(2, 4, 300), (5, 4, 129), (8, 4, 1000), (9, 4, 127), (7, 8, 640), (33, 2, 500),
                                       (17, 8, 257), (40, 4, 384), (3, 1, 1), (6, 4, 0)])
-def test_head_dim_64_runs_on_the_tensor_cores(T_q, G, n):
-    # head dim 64: the keys-on-M kernel with one 64-column box per tile (its output MMA pads M
-    # with rows that are never read), every row-group width, ragged tails, several chunks
+@pytest.mark.parametrize("flags", [0, 8])
+def test_head_dim_64_runs_on_the_tensor_cores(T_q, G, n, flags):
+    # head dim 64: one 64-column box per tile in both tensor-core kernels (the keys-on-M kernel's
+    # output MMA pads M with rows that are never read), every row-group width, ragged tails,
+    # several chunks; flags = 8 takes the keys-on-M kernel for every row count
     cfg = inputs.VerifyConfig("v", 0x90 + T_q + G + n, 3, 2 * G, 2, 64, 256, T_q, n, n, k_mult=2.0,
                               mask="tree" if T_q % 2 else "chain")
     lens = [n, max(0, n - 77), n // 2]
-    O, LSE, _ = _run(cfg, lens=lens, fill=float("nan"), kernel="tcgen05-keys")
+    want = "tcgen05-keys" if (flags or T_q * G <= 16) else "tcgen05"
+    O, LSE, _ = _run(cfg, lens=lens, flags=flags, fill=float("nan"), kernel=want)
     # and the CUDA-core kernel agrees
     case = util.gen_case(cfg, lens, DEV, float("nan"))
     ctx = util.make_ctx(cfg, flags=1)
@@ -640,6 +643,6 @@ def test_head_dim_64_paged(page_size):
     ctx.ss_verify_finalize(O, LSE)
     torch.cuda.synchronize()
     assert ctx.ss_poll_status() == (0, 0)
-    assert ctx.last_chunk_kernel() == "tcgen05-keys"
+    assert ctx.last_chunk_kernel() == "tcgen05"      # 24 rows per kv-head: rows on M at head dim 64
     util.compare(cfg, O, LSE, ref)
     ctx.close()
