@@ -202,6 +202,18 @@ def test_stream_round_matches_oracle_ragged(batch_chunks, fused):
     ctx.close()
 
 
+def test_stream_round_head_dim_64():
+    # the streamed round with 64-wide heads (host block layout, staging strides and kernels follow d)
+    cfg = inputs.VerifyConfig("v", 0x63, 4, 8, 2, 64, 256, 8, 0, 1500, accept=True)
+    lens = [1500, 0, 256, 700]
+    ctx, case, O, LSE, bufs, acc, stats, _ = _stream_case(cfg, lens, 2, fused="blocks")
+    ref = util.oracle_case(cfg, lens, *case)
+    util.compare(cfg, O, LSE, ref)
+    assert ctx.last_chunk_kernel().startswith("tcgen05")
+    assert stats.h2d_bytes == sum(lens) * cfg.H_kv * cfg.d * 4
+    ctx.close()
+
+
 def test_stream_round_copy_only_and_reuse():
     cfg = inputs.VerifyConfig("v", 0x63, 3, 8, 2, 128, 256, 6, 300, 1500)
     lens = inputs.history_lengths(cfg)
