@@ -646,3 +646,28 @@ def test_head_dim_64_paged(page_size):
     assert ctx.last_chunk_kernel() == "tcgen05"      # 24 rows per kv-head: rows on M at head dim 64
     util.compare(cfg, O, LSE, ref)
     ctx.close()
+
+
+def test_graph_round_helper_replays_with_refreshed_inputs():
+    # the binding's GraphRound: capture once, refresh the inputs in place, replay
+    ssb = _ssb()
+    cfg = inputs.CONFIGS["c1_tiny_chain"]
+    lens = inputs.history_lengths(cfg)
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    ctx = util.make_ctx(cfg, flags=ssb.SS_FLAG_OVERLAP_CHUNKS)
+    g = ssb.GraphRound(ctx, Q, chunks, K_loc, V_loc, cfg.scale)
+    O, LSE = g.replay()
+    torch.cuda.synchronize()
+    util.compare(cfg, O, LSE, util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits))
+    # new contents in the same buffers
+    cfg2 = inputs.VerifyConfig(cfg.name, cfg.seed + 1, cfg.B, cfg.H_q, cfg.H_kv, cfg.d, cfg.L_c, cfg.T_q,
+                               cfg.len_lo, cfg.len_hi)
+    Q2, chunks2, K_loc2, V_loc2, bits2 = util.gen_case(cfg2, lens, DEV)
+    Q.copy_(Q2); K_loc.copy_(K_loc2); V_loc.copy_(V_loc2)
+    for (K, V, vl), (K2, V2, vl2) in zip(chunks, chunks2):
+        K.copy_(K2); V.copy_(V2); vl.copy_(vl2)
+    O, LSE = g.replay()
+    torch.cuda.synchronize()
+    assert ctx.ss_poll_status() == (0, 0)
+    util.compare(cfg2, O, LSE, util.oracle_case(cfg2, lens, Q2, chunks2, K_loc2, V_loc2, bits2))
+    ctx.close()
