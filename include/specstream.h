@@ -146,7 +146,7 @@ ss_status ss_verify_chunk_hinted(ss_ctx* ctx, ss_tensor K, ss_tensor V, int32_t 
  * request b is the concatenation of pages page_table[b][0 .. pages_per_req) (device int32
  * [B, pages_per_req]), i.e. L_c = pages_per_req * page_size tokens of which valid_len[b] are
  * valid (NULL = all).  Same result as ss_verify_chunk on the gathered chunk.  The tensor-core
- * kernels take pages of 16, 32, 64 tokens (gathered page by page into their tiles) and any
+ * kernels take pages of 8, 16, 32, 64 tokens (gathered page by page into their tiles) and any
  * multiple of 64 (rows on M) or 128 (keys on M); other page sizes take the CUDA-core kernel,
  * which is an order of magnitude slower.  Only the pages that hold valid tokens are looked up:
  * table entries past ceil(valid_len[b] / page_size) may hold anything.  valid_len_host (HOST,

@@ -397,11 +397,12 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   }
   CUtensorMap tmK, tmV;
   bool tc = c->tc_ok;
-  // paged chunks: a tile is one page, a whole number of pages (16, 32 or 64 tokens each,
-  // gathered page by page) or part of a page; anything else takes the CUDA-core kernel
+  // paged chunks: a tile is one page, a whole number of pages (8, 16, 32 or 64 tokens each,
+  // gathered page by page: a page of 8 tokens is one 1024-byte swizzle atom, the smallest box
+  // that keeps the tile's layout) or part of a page; anything else takes the CUDA-core kernel
   const auto pages_fit = [&](int tile) {
     const int ps = pg->page_size;
-    return ps % tile == 0 || (ps >= 16 && tile % ps == 0);
+    return ps % tile == 0 || (ps >= 8 && tile % ps == 0);
   };
   // up to 32 rows per kv-head the keys ride the MMA's M axis (tiles of 128 tokens); with more
   // rows the kernel with the rows on M is faster (measured).  SS_FLAG_ROWS_ON_M /

@@ -238,7 +238,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       if (D == 128) tma_load_4d(dst + kHalfTile, &tmK, 64, tok, kvh, outer, bar, pol);
     }
   };
-  // Pages smaller than a tile (16 or 32 tokens): the tile is gathered page by page by the whole
+  // Pages smaller than a tile (8, 16 or 32 tokens): the tile is gathered page by page by the whole
   // producer warp, see below; this path is for contiguous chunks and pages of a tile or more.
   const bool small_pages = p.page_table && p.page_size < kTileKeys;
   auto issue_tile = [&](bool is_v, int it, uint32_t dst, uint64_t* bar, uint64_t pol) {
@@ -315,13 +315,13 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     // ===== TMA producer, pages smaller than a tile =====
     // The tensor map's box is one page; page i of a tile lands at row i * page_size of the slot,
     // which keeps the swizzled layout of a single 64-token box.  Lane l copies 64-column half
-    // l % 2 of page l / 2 of the tile, so a tile's 4 or 8 copies and their page look-ups go out
+    // l % 2 of page l / 2 of the tile, so a tile's 4 to 16 copies and their page look-ups go out
     // side by side; each lane fetches the page id of a ring's next tile right after its copy,
     // off the path of the next one.  Pages that start at or past the valid length are not
     // looked up (index n_pages is outside the pool and reads as zeros).  Lane 0 polls the two
     // rings as in the loop below, arms the barriers and shares what to issue through a shuffle.
     const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
-    const int ps = p.page_size, n_sub = kTileKeys / ps;  // 2 or 4 pages per tile
+    const int ps = p.page_size, n_sub = kTileKeys / ps;  // 2 to 8 pages per tile (pages of 32 to 8 tokens)
     const int sub = lane / kHalves, half = lane % kHalves;
     const bool mine = lane < kHalves * n_sub;
     auto lane_page = [&](int tile) {  // page id of this lane's page of `tile`; -2: not looked up

@@ -143,7 +143,7 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
       if (D == 128) tma_load_4d(dst + kHalf, &tmK, 64, tok, kvh, outer, bar, pol);
     }
   };
-  // Pages smaller than a tile (16, 32 or 64 tokens): the tile is gathered page by page by the
+  // Pages smaller than a tile (8 to 64 tokens): the tile is gathered page by page by the
   // whole producer warp, see below; this path is for contiguous chunks and pages of a tile or more.
   const bool small_pages = p.page_table && p.page_size < kKeys;
   auto issue_use = [&](int j, uint64_t pol) {
@@ -218,13 +218,13 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
     // ===== TMA producer, pages smaller than a tile =====
     // The tensor map's box is one page; page i of a tile lands at row i * page_size of the ring
     // unit, which keeps the swizzled layout of a single 128-token box.  Lane l copies 64-column
-    // half l % 2 of page l / 2 of the tile, so a unit's 4 to 16 copies and their page look-ups
+    // half l % 2 of page l / 2 of the tile, so a unit's 4 to 32 copies and their page look-ups
     // go out side by side; each lane fetches the page id of the next tile right after a tile's
     // V copy, off the path of the next copy.  Pages that start at or past the valid length are
     // not looked up (index n_pages is outside the pool and reads as zeros).  Lane 0 waits for
     // the unit (bounded) and arms its barrier; the outcome is shared through a shuffle.
     const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
-    const int ps = p.page_size, n_sub = kKeys / ps;  // 2, 4 or 8 pages per tile
+    const int ps = p.page_size, n_sub = kKeys / ps;  // 2 to 16 pages per tile (pages of 64 to 8 tokens)
     const int sub = lane / C::kHalves, half = lane % C::kHalves;
     const bool mine = lane < C::kHalves * n_sub;
     auto lane_page = [&](int tile) {  // page id of this lane's page of `tile`; -2: not looked up

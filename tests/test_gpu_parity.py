@@ -407,7 +407,7 @@ def test_random_ragged_shapes(seed):
 
 
 @pytest.mark.parametrize("page_size,flags", [(128, 0), (128, 4), (64, 0), (64, 8), (64, 4), (32, 0), (32, 4), (16, 0),
-                                             (16, 4), (16, 8), (8, 0), (128, 1), (16, 1), (256, 0), (256, 4)])
+                                             (16, 4), (16, 8), (8, 0), (8, 4), (4, 0), (128, 1), (16, 1), (256, 0), (256, 4)])
 def test_paged_chunks_match_contiguous_and_oracle(page_size, flags):
     # the chunk's tokens live in shuffled pages of a pool; same result as the gathered chunk
     ssb = _ssb()
@@ -438,8 +438,8 @@ def test_paged_chunks_match_contiguous_and_oracle(page_size, flags):
     torch.cuda.synchronize()
     st, dev_bits = ctx.ss_poll_status()
     assert st == 0, dev_bits
-    # pages of 16 tokens and more are gathered into the tensor-core kernels' tiles
-    expect = "simt" if (flags & 1 or page_size < 16) else ("tcgen05" if flags & 4 else "tcgen05-keys")
+    # pages of 8 tokens and more are gathered into the tensor-core kernels' tiles
+    expect = "simt" if (flags & 1 or page_size < 8) else ("tcgen05" if flags & 4 else "tcgen05-keys")
     assert ctx.last_chunk_kernel() == expect, (ctx.last_chunk_kernel(), expect)
     util.compare(cfg, O, LSE, ref)
     ctx.close()
@@ -617,7 +617,7 @@ def test_head_dim_64_runs_on_the_tensor_cores(T_q, G, n, flags):
     assert torch.equal(torch.isfinite(LSE), fin) and (LSE[fin] - L2[fin]).abs().max() < 1e-4
 
 
-@pytest.mark.parametrize("page_size", [16, 64, 128])
+@pytest.mark.parametrize("page_size", [8, 16, 64, 128])
 def test_head_dim_64_paged(page_size):
     ssb = _ssb()
     cfg = inputs.VerifyConfig("pg", 0xA0 + page_size, 3, 8, 2, 64, 512, 6, 40, 1500, k_mult=2.0)
