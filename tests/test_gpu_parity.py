@@ -345,6 +345,28 @@ def test_strided_inputs():
         ctx.close()
 
 
+@pytest.mark.parametrize("d", [64, 128])
+def test_token_major_layouts(d):
+    # K/V (and Q, local KV) stored token-major, [B, tokens, heads, d], passed as permuted views:
+    # the head stride is then smaller than the token stride
+    cfg = inputs.VerifyConfig("v", 0x5B + d, 2, 8, 2, d, 256, 12, 300, 700, k_mult=2.0)
+    lens = [700, 300]
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+
+    def token_major(t):     # same values, [B, T, H, d] memory, [B, H, T, d] view
+        return t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+
+    chunks_tm = [(token_major(K), token_major(V), vl) for K, V, vl in chunks]
+    assert chunks_tm[0][0].stride(1) < chunks_tm[0][0].stride(2)
+    ref = util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits)
+    for flags in (0, 1, 4, 8):
+        ctx = util.make_ctx(cfg, flags=flags)
+        O, L = util.gpu_case(ctx, cfg, token_major(Q), chunks_tm, token_major(K_loc), token_major(V_loc), bits)
+        assert ctx.ss_poll_status() == (0, 0)
+        util.compare(cfg, O, L, ref)
+        ctx.close()
+
+
 def test_bad_valid_len_sets_status_and_is_clamped():
     ssb = _ssb()
     cfg = inputs.VerifyConfig("v", 0x5B, 2, 8, 2, 128, 128, 4, 128, 128)
