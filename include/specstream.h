@@ -142,7 +142,9 @@ ss_status ss_verify_chunk_hinted(ss_ctx* ctx, ss_tensor K, ss_tensor V, int32_t 
                                  void* stream);
 
 /* A chunk whose tokens live in pages of a pool (requests keep independent KV indices): K_pool,
- * V_pool are [n_pages, H_kv, page_size, d] (ss_tensor: stride_b = page stride); the chunk of
+ * V_pool are [n_pages, H_kv, page_size, d] (ss_tensor: stride_b = page stride; any strides
+ * that are multiples of 8 elements, so a pool stored [n_pages, page_size, H_kv, d] is passed
+ * with stride_t = H_kv * d and stride_h = d); the chunk of
  * request b is the concatenation of pages page_table[b][0 .. pages_per_req) (device int32
  * [B, pages_per_req]), i.e. L_c = pages_per_req * page_size tokens of which valid_len[b] are
  * valid (NULL = all).  Same result as ss_verify_chunk on the gathered chunk.  The tensor-core

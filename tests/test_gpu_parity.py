@@ -526,6 +526,37 @@ def test_small_pages_bad_ids_and_unused_table_entries(flags):
     ctx.close()
 
 
+@pytest.mark.parametrize("flags", [0, 4, 1])
+def test_paged_pool_stored_token_major(flags):
+    # the pool as paged KV caches commonly store it, [n_pages, page_size, H_kv, d], passed as a
+    # permuted view [n_pages, H_kv, page_size, d]
+    cfg = inputs.VerifyConfig("pg", 0x61, 3, 8, 2, 128, 256, 6, 30, 700, k_mult=2.0)
+    lens = [700, 30, 512]
+    case = util.gen_case(cfg, lens, DEV, fill=float("nan"))
+    Q, chunks, K_loc, V_loc, bits = case
+    ref = util.oracle_case(cfg, lens, *case)
+    ps, ppr = 16, cfg.L_c // 16
+    g = torch.Generator().manual_seed(5)
+    ctx = util.make_ctx(cfg, flags=flags)
+    O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
+    LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
+    ctx.ss_verify_begin(Q, cfg.scale)
+    for K, V, vl in chunks:
+        n_pages = cfg.B * ppr + 2
+        table = torch.randperm(n_pages, generator=g)[:cfg.B * ppr].to(torch.int32).view(cfg.B, ppr).contiguous()
+        pools = []
+        for X in (K, V):
+            pool = torch.full((n_pages, ps, cfg.H_kv, cfg.d), float("nan"), dtype=torch.bfloat16, device=DEV)
+            pool[table.view(-1).long()] = X.view(cfg.B, cfg.H_kv, ppr, ps, cfg.d).permute(0, 2, 3, 1, 4).reshape(-1, ps, cfg.H_kv, cfg.d)
+            pools.append(pool.permute(0, 2, 1, 3))
+        ctx.ss_verify_chunk_paged(pools[0], pools[1], table.to(DEV), vl, vl.tolist())
+    ctx.ss_verify_local(K_loc, V_loc)
+    ctx.ss_verify_finalize(O, LSE)
+    assert ctx.ss_poll_status() == (0, 0)
+    util.compare(cfg, O, LSE, ref)
+    ctx.close()
+
+
 def test_round_can_be_captured_in_a_cuda_graph():
     # the calls only enqueue on the stream: a captured round replays bit-identically
     ssb = _ssb()
