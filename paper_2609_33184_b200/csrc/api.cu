@@ -26,6 +26,7 @@ struct ss_ctx {
   float scale;
   int n_sets;
   uint8_t splits[ss::kMaxSets];
+  uint64_t absent[ss::kMaxSets];  // per chunk set: requests (bits, b < 64) the call skipped
   bool has_local;
   bool first_launch;       // next kernel is the first of the round (or follows a fold)
   cudaStream_t stream;
@@ -215,6 +216,7 @@ void fill_merge(ss_ctx* c, ss::MergeParams* m) {
   m->d = c->cfg.d;
   m->R_stride = c->R_stride;
   memcpy(m->splits, c->splits, sizeof(m->splits));
+  memcpy(m->absent, c->absent, sizeof(m->absent));
 }
 
 // All partial sets in use: fold them into set 0 (Eq. 14 is associative).
@@ -229,6 +231,7 @@ cudaError_t fold_sets(ss_ctx* c, cudaStream_t s) {
   ++c->launches;
   c->n_sets = 1;
   c->splits[0] = 1;
+  c->absent[0] = 0;        // the folded set holds every request
   c->first_launch = true;  // the next kernel must not overlap the fold
   return cudaSuccess;
 }
@@ -386,14 +389,30 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   const int n_tiles = (L_c + kTileKeys - 1) / kTileKeys;
   // host copy of the valid lengths (a hint): size the splits for the requests that are active
   int active_pairs = pairs, used_tiles = n_tiles;
+  // requests without tokens in this chunk (by the host copy) get no CTAs at all when the batch
+  // has at most 64 requests: the launch covers the listed requests only and the merge skips
+  // this set for the others
+  int n_listed = 0;
+  uint8_t listed[64];
+  uint64_t absent = 0;
   if (valid_len && valid_len_host) {
     int active = 0, longest = 0;
     for (int b = 0; b < c->B; ++b) {
       int v = valid_len_host[b];
       v = v < 0 ? 0 : (v > L_c ? L_c : v);
-      if (v > 0) ++active;
+      if (v > 0) {
+        ++active;
+        if (c->B <= 64) listed[n_listed++] = (uint8_t)b;
+      } else if (c->B <= 64) {
+        absent |= 1ull << b;
+      }
       if (v > longest) longest = v;
     }
+    if (c->B <= 64 && n_listed == 0) {  // nobody has tokens: one request keeps the launch well-formed
+      listed[n_listed++] = 0;
+      absent &= ~1ull;
+    }
+    if (n_listed == c->B) n_listed = 0;  // everybody is in: plain launch
     active_pairs = (active > 0 ? active : 1) * c->cfg.H_kv;
     used_tiles = longest > 0 ? (longest + kTileKeys - 1) / kTileKeys : 1;
   }
@@ -509,6 +528,8 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   p.part_ml = c->part_ml + (int64_t)c->n_sets * c->set_stride_ml;
   p.part_a = c->part_a + (int64_t)c->n_sets * c->set_stride_a;
   p.R_stride = c->R_stride;
+  p.n_active = n_listed;
+  if (n_listed) memcpy(p.active_b, listed, (size_t)n_listed);
   p.a_slot0 = c->n_sets * c->slots_per_set;
   p.status = c->status;
   p.wait_first = 0;
@@ -528,6 +549,7 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   c->last_kernel = !tc ? "simt" : keys_on_m ? "tcgen05-keys" : "tcgen05";
   ++c->launches;
   c->splits[c->n_sets] = (uint8_t)splits;
+  c->absent[c->n_sets] = n_listed ? absent : 0;
   ++c->n_sets;
   c->first_launch = false;
   return SS_OK;
@@ -612,6 +634,7 @@ ss_status ss_verify_import_state(ss_ctx* c, const float* ml, const float* a, voi
   if (e != cudaSuccess) return cuda_fail(c, e);
   ++c->launches;
   c->splits[c->n_sets] = 1;
+  c->absent[c->n_sets] = 0;
   ++c->n_sets;
   c->first_launch = true;
   return SS_OK;

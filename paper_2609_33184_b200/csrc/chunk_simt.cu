@@ -210,7 +210,7 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const ChunkParams 
 }  // namespace
 
 cudaError_t launch_chunk_simt(const ChunkParams& p, cudaStream_t s, bool pdl) {
-  dim3 grid(p.splits * p.row_tiles, p.H_kv, p.B), block(kThreads);
+  dim3 grid(p.splits * p.row_tiles, p.H_kv, p.n_active ? p.n_active : p.B), block(kThreads);
   if (p.d == 128) return launch_kernel(chunk_simt_kernel<128>, grid, block, 0, s, pdl, p);
   return launch_kernel(chunk_simt_kernel<64>, grid, block, 0, s, pdl, p);
 }

@@ -714,7 +714,7 @@ cudaError_t chunk_tc_prepare() {
 
 cudaError_t launch_chunk_tc(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
                             const CUtensorMap& tmA, cudaStream_t s, bool pdl) {
-  dim3 grid(p.splits * p.row_tiles, p.H_kv, p.B), block(kThreads);
+  dim3 grid(p.splits * p.row_tiles, p.H_kv, p.n_active ? p.n_active : p.B), block(kThreads);
   if (p.d == 64)
     return launch_kernel(chunk_tc_kernel<64>, grid, block, Lay<64>::kSmemTotal, s, pdl, p, tmK, tmV, tmA);
   return launch_kernel(chunk_tc_kernel<128>, grid, block, Lay<128>::kSmemTotal, s, pdl, p, tmK, tmV, tmA);

@@ -655,7 +655,7 @@ template <int NC, int WG, int UNITS, int D>
 cudaError_t launch_cfg(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
                        cudaStream_t s, bool pdl) {
   using C = Cfg<NC, WG, UNITS, D>;
-  dim3 grid(p.splits * p.row_tiles, p.H_kv, p.B), block(C::kThreads);
+  dim3 grid(p.splits * p.row_tiles, p.H_kv, p.n_active ? p.n_active : p.B), block(C::kThreads);
   return launch_kernel(chunk_tc_keys_kernel<NC, WG, UNITS, D>, grid, block, C::kSmem, s, pdl, p, tmK, tmV);
 }
 

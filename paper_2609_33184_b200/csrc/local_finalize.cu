@@ -213,6 +213,10 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) merge_kernel(const MergePar
   // (m, l) of partial f and the element offset of its a[] row
   auto load_ml = [&](int f, int64_t* a_off) {
     const int s = set_of[f], k = f - first_s[s];
+    if (s < p.n_sets && b < 64 && ((p.absent[s] >> b) & 1)) {  // the call skipped this request
+      *a_off = 0;
+      return make_float2(-INFINITY, 0.f);
+    }
     const int set = (s < p.n_sets) ? s : p.local_set;
     const size_t idx = (slot0 + k * split_stride) * p.R_stride + r;
     *a_off = (int64_t)set * p.set_stride_a + (int64_t)idx * D;

@@ -46,6 +46,10 @@ struct ChunkParams {
   uint32_t* status;
   int wait_first;       // 1: wait for the preceding kernel before reading inputs
   unsigned long long* trace;  // optional: per-tile clock stamps of CTA (0,0,0), see ss_trace_read
+  // requests this launch covers: 0 = all B (grid.z = B, b = blockIdx.z); otherwise grid.z =
+  // n_active and b = active_b[blockIdx.z] (the host knew which requests have tokens in this chunk)
+  int n_active;
+  uint8_t active_b[64];
   // paged chunk (null = contiguous): token tok of request b lives in page
   // page_table[b][tok / page_size] of the pool, at token offset tok % page_size
   const int32_t* page_table;
@@ -76,6 +80,7 @@ struct MergeParams {
   int local_set;          // index of the local set
   int B, H_q, H_kv, G, T_q, d, R_stride;
   uint8_t splits[kMaxSets];
+  uint64_t absent[kMaxSets];  // bit b set: chunk set s holds no partial of request b (b < 64)
   // finalize outputs
   __nv_bfloat16* O;
   float* LSE;
@@ -162,7 +167,7 @@ __device__ __forceinline__ ChunkWork chunk_work(const ChunkParams& p, int tile_r
   const int rt = blockIdx.x % p.row_tiles;
   w.split = blockIdx.x / p.row_tiles;
   w.kvh = blockIdx.y;
-  w.b = blockIdx.z;
+  w.b = p.n_active ? p.active_b[blockIdx.z] : blockIdx.z;
   w.row0 = rt * tile_rows;
   w.nrows = min(tile_rows, p.R - w.row0);
   w.chain_cta = (blockIdx.x | blockIdx.y | blockIdx.z) == 0;

@@ -404,6 +404,48 @@ def test_hinted_chunk_calls_match_unhinted():
     ctx.close()
 
 
+@pytest.mark.parametrize("flags", [0, 1, 4])
+@pytest.mark.parametrize("max_chunks", [0, 2])
+def test_hinted_calls_skip_requests_without_tokens(flags, max_chunks):
+    # With a host copy of the lengths, requests that have no tokens in a chunk get no thread
+    # blocks in that call and the merge skips that call's partial set for them - also after the
+    # sets were folded (max_chunks = 2 forces folds), with a NaN-poisoned workspace (a skipped
+    # slot holds whatever an earlier round left there), with a chunk nobody has tokens in, and
+    # through an exported state.
+    import bench
+    ssb = _ssb()
+    cfg = inputs.VerifyConfig("v", 0x5E, 6, 8, 2, 128, 256, 12, 0, 1300, k_mult=2.0)
+    lens = [900, 0, 300, 1300, 0, 257]
+    case = util.gen_case(cfg, lens, DEV, fill=float("nan"))
+    Q, chunks, K_loc, V_loc, bits = case
+    ref = util.oracle_case(cfg, lens, *case)
+    hints = bench.host_valid(cfg, lens, len(chunks))
+    empty = (torch.zeros_like(chunks[0][0]), torch.zeros_like(chunks[0][1]), torch.zeros_like(chunks[0][2]))
+    ctx = util.make_ctx(cfg, flags=flags, max_chunks=max_chunks)
+    ctx.workspace[4096:].view(torch.float32)[:] = float("nan")   # past the status word and trace region
+    O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
+    LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
+    ml = torch.empty(cfg.B * cfg.H_q * cfg.T_q, 2, dtype=torch.float32, device=DEV)
+    a = torch.empty(cfg.B * cfg.H_q * cfg.T_q, cfg.d, dtype=torch.float32, device=DEV)
+    for use_export in (False, True):
+        ctx.ss_verify_begin(Q, cfg.scale)
+        for j, (K, V, vl) in enumerate(chunks):
+            ctx.ss_verify_chunk_hinted(K, V, vl, hints[j])
+            if j == 1:
+                ctx.ss_verify_chunk_hinted(*empty, [0] * cfg.B)       # nobody has tokens here
+        if use_export:                                                  # state out, round dropped, state back in
+            ctx.ss_verify_export_state(ml, a)
+            ctx.ss_verify_abort()
+            ctx.ss_verify_begin(Q, cfg.scale)
+            ctx.ss_verify_import_state(ml, a)
+        ctx.ss_verify_local(K_loc, V_loc)
+        ctx.ss_verify_finalize(O, LSE)
+        torch.cuda.synchronize()
+        assert ctx.ss_poll_status() == (0, 0)
+        util.compare(cfg, O, LSE, ref)
+    ctx.close()
+
+
 @pytest.mark.parametrize("seed", range(24))
 def test_random_ragged_shapes(seed):
     # seeded sweep over batch, GQA group, candidate count, head dim, chunk size, ragged lengths,
