@@ -617,9 +617,19 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
       for (int r = 0; r < NC; ++r)
         if (r < cn) red[L * (N + 1) + c0 + r] = (r & 1) ? lsum[r / 2].y : lsum[r / 2].x;
       named_bar_sync(1, C::kSoft);
+      // four threads per row, each over a quarter of the key lanes (kSoft / N = 4), then one
+      // thread per row over the four partial sums
+      float* red4 = red + kKeys * (N + 1);  // [4][N]
+      {
+        const int row = tid % N, part = tid / N;
+        float ps = 0.f;
+#pragma unroll 8
+        for (int k = part * (kKeys / 4); k < (part + 1) * (kKeys / 4); ++k) ps += red[k * (N + 1) + row];
+        red4[part * N + row] = ps;
+      }
+      named_bar_sync(1, C::kSoft);
       if (tid < nrows) {
-        float lt = 0.f;
-        for (int k = 0; k < kKeys; ++k) lt += red[k * (N + 1) + tid];
+        const float lt = (red4[tid] + red4[N + tid]) + (red4[2 * N + tid] + red4[3 * N + tid]);
         out_ml[tid] = make_float2(lt > 0.f ? -ctl->nm_ref[tid] : -INFINITY, lt);
       }
       // thread (L, cg) holds head dim L of its rows
