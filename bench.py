@@ -63,10 +63,10 @@ def tensor_peak():
 # DRAM bytes (read + write) per chunk-kernel launch from an ncu capture of the same kernel;
 # filled from the summaries under profiles/ (None until a capture exists for the workload).
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    # profiles/chunk_tc_keys_kernel_c2_qwen3_8b.md: 135.34 MB read + 3.54 MB written per launch
-    "c2_qwen3_8b": 138.9e6,
-    # profiles/chunk_tc_kernel_c4_tree.md: 69.80 MB read + 1.67 MB written per launch
-    "c4_tree": 71.5e6,
+    # profiles/chunk_tc_keys_kernel_c2_qwen3_8b.md: 135.34 MB read + 3.87 MB written per launch
+    "c2_qwen3_8b": 139.2e6,
+    # profiles/chunk_tc_kernel_c4_tree.md: 69.80 MB read + 2.28 MB written per launch
+    "c4_tree": 72.1e6,
 }
 
 
