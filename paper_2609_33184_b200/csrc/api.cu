@@ -236,6 +236,92 @@ cudaError_t fold_sets(ss_ctx* c, cudaStream_t s) {
   return cudaSuccess;
 }
 
+
+// What the host copy of the valid lengths says about a chunk call.
+struct HintScan {
+  int active;         // requests with tokens in this chunk (>= 1; all B without a host copy)
+  int longest;        // tokens of the longest of them (>= 1; L_c without a host copy)
+  int n_listed;       // > 0: the launch covers only the requests in listed[] (batches of <= 64)
+  uint8_t listed[64];
+  uint64_t absent;    // bit b: request b is not in listed[]
+};
+
+// Requests without tokens in this chunk (by the host copy) get no CTAs at all when the batch
+// has at most 64 requests: the launch covers the listed requests only and the merge skips this
+// call's set for the others.
+HintScan scan_hint(const ss_ctx* c, const int32_t* valid_len_host, int L_c) {
+  HintScan h;
+  h.active = c->B;
+  h.longest = L_c;
+  h.n_listed = 0;
+  h.absent = 0;
+  if (!valid_len_host) return h;
+  const bool can_list = c->B <= 64;
+  int active = 0, longest = 0;
+  for (int b = 0; b < c->B; ++b) {
+    int v = valid_len_host[b];
+    v = v < 0 ? 0 : (v > L_c ? L_c : v);
+    if (v > 0) {
+      ++active;
+      if (can_list) h.listed[h.n_listed++] = (uint8_t)b;
+    } else if (can_list) {
+      h.absent |= 1ull << b;
+    }
+    if (v > longest) longest = v;
+  }
+  if (can_list && h.n_listed == 0) {  // nobody has tokens: one request keeps the launch well-formed
+    h.listed[h.n_listed++] = 0;
+    h.absent &= ~1ull;
+  }
+  if (h.n_listed == c->B) h.n_listed = 0;  // everybody is in: plain launch
+  h.active = active > 0 ? active : 1;
+  h.longest = longest > 0 ? longest : 1;
+  return h;
+}
+
+// Token splits of a chunk call: `ctas1` CTAs have work with one split, `used_tiles` 64-token
+// tiles reach the longest request's last token.
+int pick_splits(ss_ctx* c, bool tensor_core, bool whole_waves, int pairs, int ctas1, int used_tiles) {
+  // tensor-core CTAs amortise their set-up over at least 256 tokens; CUDA-core CTAs take one tile
+  const int min_tiles = tensor_core ? 4 : 1;
+  int max_splits = c->slots_per_set / pairs;
+  if (max_splits > kMaxSplits) max_splits = kMaxSplits;
+  if (max_splits > (used_tiles + min_tiles - 1) / min_tiles) max_splits = (used_tiles + min_tiles - 1) / min_tiles;
+  if (max_splits < 1) max_splits = 1;
+  int splits;
+  if (c->force_splits > 0) {
+    splits = c->force_splits;
+  } else if (whole_waves) {
+    // one CTA per SM and no co-residency with the next launch: pick the split count whose CTA
+    // count fills whole waves of SMs best (smallest such count: fewer partial states)
+    double best = 0.0;
+    splits = 1;
+    for (int sp = 1; sp <= max_splits; ++sp) {
+      const int ctas = ctas1 * sp;
+      const int waves = (ctas + ss::kNumSM - 1) / ss::kNumSM;
+      const double eff = (double)ctas / ((double)waves * ss::kNumSM);
+      if (eff > best + 0.05) {
+        best = eff;
+        splits = sp;
+      }
+    }
+  } else {
+    // About one CTA per SM for the first chunk call of a round.  A later call whose kernel
+    // overlaps the one before it (programmatic dependent launch) finds the SMs partly taken and
+    // more launches on their way: half as many CTAs, each with twice the tiles, leave less
+    // set-up and fewer partial states per byte (measured on the ragged 7B-shaped workload,
+    // 64 kv-head groups per call: 6.39 -> 6.68 TB/s; unchanged where a call has 128 groups or
+    // more).  The choice depends on the position in the round only, so results stay
+    // reproducible bit for bit.
+    int target = c->target_ctas;
+    if (!c->target_forced && use_pdl(c)) target = target / 2 > 0 ? target / 2 : 1;
+    splits = target / ctas1;
+  }
+  if (splits > max_splits) splits = max_splits;
+  if (splits < 1) splits = 1;
+  return splits;
+}
+
 }  // namespace
 
 extern "C" {
@@ -387,35 +473,10 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   const int R = c->T_q * c->G;
   const int pairs = c->B * c->cfg.H_kv;
   const int n_tiles = (L_c + kTileKeys - 1) / kTileKeys;
-  // host copy of the valid lengths (a hint): size the splits for the requests that are active
-  int active_pairs = pairs, used_tiles = n_tiles;
-  // requests without tokens in this chunk (by the host copy) get no CTAs at all when the batch
-  // has at most 64 requests: the launch covers the listed requests only and the merge skips
-  // this set for the others
-  int n_listed = 0;
-  uint8_t listed[64];
-  uint64_t absent = 0;
-  if (valid_len && valid_len_host) {
-    int active = 0, longest = 0;
-    for (int b = 0; b < c->B; ++b) {
-      int v = valid_len_host[b];
-      v = v < 0 ? 0 : (v > L_c ? L_c : v);
-      if (v > 0) {
-        ++active;
-        if (c->B <= 64) listed[n_listed++] = (uint8_t)b;
-      } else if (c->B <= 64) {
-        absent |= 1ull << b;
-      }
-      if (v > longest) longest = v;
-    }
-    if (c->B <= 64 && n_listed == 0) {  // nobody has tokens: one request keeps the launch well-formed
-      listed[n_listed++] = 0;
-      absent &= ~1ull;
-    }
-    if (n_listed == c->B) n_listed = 0;  // everybody is in: plain launch
-    active_pairs = (active > 0 ? active : 1) * c->cfg.H_kv;
-    used_tiles = longest > 0 ? (longest + kTileKeys - 1) / kTileKeys : 1;
-  }
+  // host copy of the valid lengths (a hint): which requests have tokens here, how far they reach
+  const HintScan hint = scan_hint(c, valid_len ? valid_len_host : nullptr, L_c);
+  const int active_pairs = hint.active * c->cfg.H_kv;
+  const int used_tiles = (hint.longest + kTileKeys - 1) / kTileKeys;
   CUtensorMap tmK, tmV;
   bool tc = c->tc_ok;
   // paged chunks: a tile is one page, a whole number of pages (8, 16, 32 or 64 tokens each,
@@ -461,44 +522,8 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
     p.rows_per_tile = 32;
     p.row_tiles = (R + 31) / 32;
   }
-  // tensor-core CTAs amortise their set-up over at least 256 tokens; CUDA-core CTAs take one tile
-  const int min_tiles = tc ? 4 : 1;
-  int max_splits = c->slots_per_set / pairs;
-  if (max_splits > kMaxSplits) max_splits = kMaxSplits;
-  if (max_splits > (used_tiles + min_tiles - 1) / min_tiles) max_splits = (used_tiles + min_tiles - 1) / min_tiles;
-  if (max_splits < 1) max_splits = 1;
   const int ctas1 = active_pairs * p.row_tiles;  // CTAs with work when splits = 1
-  int splits;
-  if (c->force_splits > 0) {
-    splits = c->force_splits;
-  } else if (tc && keys_on_m && R > 32) {
-    // one CTA per SM and no co-residency with the next launch: pick the split count whose CTA
-    // count fills whole waves of SMs best (smallest such count: fewer partial states)
-    double best = 0.0;
-    splits = 1;
-    for (int sp = 1; sp <= max_splits; ++sp) {
-      const int ctas = ctas1 * sp;
-      const int waves = (ctas + ss::kNumSM - 1) / ss::kNumSM;
-      const double eff = (double)ctas / ((double)waves * ss::kNumSM);
-      if (eff > best + 0.05) {
-        best = eff;
-        splits = sp;
-      }
-    }
-  } else {
-    // About one CTA per SM for the first chunk call of a round.  A later call whose kernel
-    // overlaps the one before it (programmatic dependent launch) finds the SMs partly taken and
-    // more launches on their way: half as many CTAs, each with twice the tiles, leave less
-    // set-up and fewer partial states per byte (measured on the ragged 7B-shaped workload,
-    // 64 kv-head groups per call: 6.39 -> 6.68 TB/s; unchanged where a call has 128 groups or
-    // more).  The choice depends on the position in the round only, so results stay
-    // reproducible bit for bit.
-    int target = c->target_ctas;
-    if (!c->target_forced && use_pdl(c)) target = target / 2 > 0 ? target / 2 : 1;
-    splits = target / ctas1;
-  }
-  if (splits > max_splits) splits = max_splits;
-  if (splits < 1) splits = 1;
+  int splits = pick_splits(c, tc, tc && keys_on_m && R > 32, pairs, ctas1, used_tiles);
   p.tiles_per_split = (used_tiles + splits - 1) / splits;
   if (tc && keys_on_m) p.tiles_per_split += p.tiles_per_split & 1;  // whole 128-token tiles
   splits = (used_tiles + p.tiles_per_split - 1) / p.tiles_per_split;
@@ -528,8 +553,8 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   p.part_ml = c->part_ml + (int64_t)c->n_sets * c->set_stride_ml;
   p.part_a = c->part_a + (int64_t)c->n_sets * c->set_stride_a;
   p.R_stride = c->R_stride;
-  p.n_active = n_listed;
-  if (n_listed) memcpy(p.active_b, listed, (size_t)n_listed);
+  p.n_active = hint.n_listed;
+  if (hint.n_listed) memcpy(p.active_b, hint.listed, (size_t)hint.n_listed);
   p.a_slot0 = c->n_sets * c->slots_per_set;
   p.status = c->status;
   p.wait_first = 0;
@@ -549,7 +574,7 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   c->last_kernel = !tc ? "simt" : keys_on_m ? "tcgen05-keys" : "tcgen05";
   ++c->launches;
   c->splits[c->n_sets] = (uint8_t)splits;
-  c->absent[c->n_sets] = n_listed ? absent : 0;
+  c->absent[c->n_sets] = hint.n_listed ? hint.absent : 0;
   ++c->n_sets;
   c->first_launch = false;
   return SS_OK;
