@@ -134,7 +134,7 @@ ss_status ss_verify_chunk(ss_ctx* ctx, ss_tensor K, ss_tensor V, int32_t L_c,
 
 /* Same as ss_verify_chunk, with a HOST copy of valid_len ([B], may be NULL) as a scheduling
  * hint: the token splits are sized for the requests that are still active, which keeps the GPU
- * full when most of a ragged batch has run out of history, and (batches of up to 64 requests)
+ * full when most of a ragged batch has run out of history, and (batches of up to 256 requests)
  * requests whose hinted length is 0 get no thread blocks at all in this call.  The device
  * array stays authoritative for the lengths that are used; a wrong hint can cost speed or, if
  * it understates a length, drop tokens (those past the hinted maximum of the batch; all of a

@@ -26,7 +26,7 @@ struct ss_ctx {
   float scale;
   int n_sets;
   uint8_t splits[ss::kMaxSets];
-  uint64_t absent[ss::kMaxSets];  // per chunk set: requests (bits, b < 64) the call skipped
+  uint64_t absent[ss::kMaxSets][ss::kMaxListed / 64];  // per chunk set: requests (bits) the call skipped
   bool has_local;
   bool first_launch;       // next kernel is the first of the round (or follows a fold)
   cudaStream_t stream;
@@ -231,7 +231,7 @@ cudaError_t fold_sets(ss_ctx* c, cudaStream_t s) {
   ++c->launches;
   c->n_sets = 1;
   c->splits[0] = 1;
-  c->absent[0] = 0;        // the folded set holds every request
+  memset(c->absent[0], 0, sizeof(c->absent[0]));  // the folded set holds every request
   c->first_launch = true;  // the next kernel must not overlap the fold
   return cudaSuccess;
 }
@@ -241,22 +241,22 @@ cudaError_t fold_sets(ss_ctx* c, cudaStream_t s) {
 struct HintScan {
   int active;         // requests with tokens in this chunk (>= 1; all B without a host copy)
   int longest;        // tokens of the longest of them (>= 1; L_c without a host copy)
-  int n_listed;       // > 0: the launch covers only the requests in listed[] (batches of <= 64)
-  uint8_t listed[64];
-  uint64_t absent;    // bit b: request b is not in listed[]
+  int n_listed;       // > 0: the launch covers only the requests in listed[] (batches of <= 256)
+  uint8_t listed[ss::kMaxListed];
+  uint64_t absent[ss::kMaxListed / 64];  // bit b: request b is not in listed[]
 };
 
 // Requests without tokens in this chunk (by the host copy) get no CTAs at all when the batch
-// has at most 64 requests: the launch covers the listed requests only and the merge skips this
+// has at most 256 requests: the launch covers the listed requests only and the merge skips this
 // call's set for the others.
 HintScan scan_hint(const ss_ctx* c, const int32_t* valid_len_host, int L_c) {
   HintScan h;
   h.active = c->B;
   h.longest = L_c;
   h.n_listed = 0;
-  h.absent = 0;
+  memset(h.absent, 0, sizeof(h.absent));
   if (!valid_len_host) return h;
-  const bool can_list = c->B <= 64;
+  const bool can_list = c->B <= ss::kMaxListed;
   int active = 0, longest = 0;
   for (int b = 0; b < c->B; ++b) {
     int v = valid_len_host[b];
@@ -265,13 +265,13 @@ HintScan scan_hint(const ss_ctx* c, const int32_t* valid_len_host, int L_c) {
       ++active;
       if (can_list) h.listed[h.n_listed++] = (uint8_t)b;
     } else if (can_list) {
-      h.absent |= 1ull << b;
+      h.absent[b >> 6] |= 1ull << (b & 63);
     }
     if (v > longest) longest = v;
   }
   if (can_list && h.n_listed == 0) {  // nobody has tokens: one request keeps the launch well-formed
     h.listed[h.n_listed++] = 0;
-    h.absent &= ~1ull;
+    h.absent[0] &= ~1ull;
   }
   if (h.n_listed == c->B) h.n_listed = 0;  // everybody is in: plain launch
   h.active = active > 0 ? active : 1;
@@ -574,7 +574,8 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   c->last_kernel = !tc ? "simt" : keys_on_m ? "tcgen05-keys" : "tcgen05";
   ++c->launches;
   c->splits[c->n_sets] = (uint8_t)splits;
-  c->absent[c->n_sets] = hint.n_listed ? hint.absent : 0;
+  if (hint.n_listed) memcpy(c->absent[c->n_sets], hint.absent, sizeof(hint.absent));
+  else memset(c->absent[c->n_sets], 0, sizeof(hint.absent));
   ++c->n_sets;
   c->first_launch = false;
   return SS_OK;
@@ -659,7 +660,7 @@ ss_status ss_verify_import_state(ss_ctx* c, const float* ml, const float* a, voi
   if (e != cudaSuccess) return cuda_fail(c, e);
   ++c->launches;
   c->splits[c->n_sets] = 1;
-  c->absent[c->n_sets] = 0;
+  memset(c->absent[c->n_sets], 0, sizeof(c->absent[0]));
   ++c->n_sets;
   c->first_launch = true;
   return SS_OK;

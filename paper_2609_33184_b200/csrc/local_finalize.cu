@@ -213,7 +213,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) merge_kernel(const MergePar
   // (m, l) of partial f and the element offset of its a[] row
   auto load_ml = [&](int f, int64_t* a_off) {
     const int s = set_of[f], k = f - first_s[s];
-    if (s < p.n_sets && b < 64 && ((p.absent[s] >> b) & 1)) {  // the call skipped this request
+    if (s < p.n_sets && b < kMaxListed && ((p.absent[s][b >> 6] >> (b & 63)) & 1)) {  // the call skipped this request
       *a_off = 0;
       return make_float2(-INFINITY, 0.f);
     }

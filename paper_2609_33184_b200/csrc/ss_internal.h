@@ -12,6 +12,7 @@ namespace ss {
 constexpr int kMaxSets = 128;      // chunk-call partial sets a finalize launch can take
 constexpr int kMaxSplits = 16;     // token splits of one chunk call
 constexpr int kTileKeys = 64;      // keys per shared-memory tile of the tensor-core kernel
+constexpr int kMaxListed = 256;    // largest batch whose requests a chunk call can list one by one
 constexpr int kNumSM = 148;
 constexpr int kTraceTiles = 32;    // tiles of CTA (0,0,0) a trace records
 constexpr int kTraceWords = 3 * kTraceTiles * 8;  // [role][tile][event] clock64 stamps
@@ -49,7 +50,7 @@ struct ChunkParams {
   // requests this launch covers: 0 = all B (grid.z = B, b = blockIdx.z); otherwise grid.z =
   // n_active and b = active_b[blockIdx.z] (the host knew which requests have tokens in this chunk)
   int n_active;
-  uint8_t active_b[64];
+  uint8_t active_b[kMaxListed];
   // paged chunk (null = contiguous): token tok of request b lives in page
   // page_table[b][tok / page_size] of the pool, at token offset tok % page_size
   const int32_t* page_table;
@@ -80,7 +81,10 @@ struct MergeParams {
   int local_set;          // index of the local set
   int B, H_q, H_kv, G, T_q, d, R_stride;
   uint8_t splits[kMaxSets];
-  uint64_t absent[kMaxSets];  // bit b set: chunk set s holds no partial of request b (b < 64)
+  // bit b of absent[s] (kMaxListed bits): chunk set s holds no partial of request b.  (With
+  // this table the structure is larger than 4 KB: it relies on the large kernel parameter
+  // space of CUDA 12.1+ on sm_70 and later.)
+  uint64_t absent[kMaxSets][kMaxListed / 64];
   // finalize outputs
   __nv_bfloat16* O;
   float* LSE;

@@ -446,6 +446,30 @@ def test_hinted_calls_skip_requests_without_tokens(flags, max_chunks):
     ctx.close()
 
 
+def test_hinted_calls_with_a_batch_of_more_than_64_requests():
+    # request lists and the merge's "absent" bits cover batches of up to 256 requests
+    import bench
+    ssb = _ssb()
+    B = 130
+    cfg = inputs.VerifyConfig("v", 0x5F, B, 4, 2, 128, 128, 4, 0, 400, k_mult=2.0)
+    lens = [(37 * b) % 401 if b % 3 else 0 for b in range(B)]
+    lens[129] = 400
+    case = util.gen_case(cfg, lens, DEV, fill=float("nan"))
+    Q, chunks, K_loc, V_loc, bits = case
+    hints = bench.host_valid(cfg, lens, len(chunks))
+    ctx = util.make_ctx(cfg)
+    ctx.workspace[8192:].view(torch.float32)[:] = float("nan")
+    O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
+    LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
+    bench.run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, hints=hints)
+    torch.cuda.synchronize()
+    assert ctx.ss_poll_status() == (0, 0)
+    groups = [(0, 0), (1, 1), (64, 0), (65, 1), (127, 0), (128, 1), (129, 0), (129, 1)]
+    util.compare(cfg, O, LSE, util.oracle_case(cfg, lens, *case, groups=groups))
+    assert torch.isfinite(O.float()).all()
+    ctx.close()
+
+
 @pytest.mark.parametrize("seed", range(24))
 def test_random_ragged_shapes(seed):
     # seeded sweep over batch, GQA group, candidate count, head dim, chunk size, ragged lengths,
