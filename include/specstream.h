@@ -421,6 +421,13 @@ int32_t ss_last_cuda_error(ss_ctx* ctx);
  * max_words 64-bit words to HOST memory and returns the count. */
 ss_status ss_trace_enable(ss_ctx* ctx, int32_t on);
 int32_t ss_trace_read(ss_ctx* ctx, uint64_t* out, int32_t max_words);
+/* Per-CTA log of the tensor-core chunk kernels (a measurement aid; the paper has no
+ * counterpart).  `log` is a DEVICE buffer of 4 * (capacity + 1) 64-bit words that the caller
+ * owns and zeroes: word 0 counts the entries, entry i occupies words 4 (i + 1) .. 4 (i + 1) + 3:
+ * the CTA's start and end on the GPU's nanosecond timer, (SM id << 32 | the context's launch
+ * number), (linear block id << 32 | tiles processed).  Entries past `capacity` are counted but
+ * not stored.  log = NULL switches it off.  Takes effect from the next chunk call. */
+ss_status ss_cta_log_set(ss_ctx* ctx, uint64_t* log, int32_t capacity);
 /* Self-test of the bounded waits (the paper has no counterpart): one small kernel whose 64
  * threads wait, with the chunk kernels' own wait routine and a limit of limit_ms (1..1000), on
  * a barrier that nothing will ever complete.  Every thread must give up: *gave_up (DEVICE

@@ -33,7 +33,7 @@ EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "
            "ss_tier_reset", "ss_tier_get", "ss_tier_tail", "ss_tier_commit", "ss_tier_migrate", "ss_tier_poll",
            "ss_tier_d2h_bytes", "ss_verify_chunk_paged", "ss_width_create", "ss_width_destroy",
            "ss_width_observe", "ss_width_next", "ss_width_estimate", "ss_cohort_build", "ss_probe_read",
-           "ss_selftest_wait_expiry", "ss_verify_abort"]
+           "ss_selftest_wait_expiry", "ss_verify_abort", "ss_cta_log_set"]
 
 
 class ss_config(C.Structure):
@@ -198,6 +198,8 @@ def load() -> C.CDLL:
     lib.ss_last_cuda_error.argtypes = [vp]
     lib.ss_trace_enable.restype = C.c_int
     lib.ss_trace_enable.argtypes = [vp, i32]
+    lib.ss_cta_log_set.restype = C.c_int
+    lib.ss_cta_log_set.argtypes = [vp, vp, i32]
     lib.ss_trace_read.restype = i32
     lib.ss_trace_read.argtypes = [vp, C.POINTER(C.c_uint64), i32]
     lib.ss_verify_round_static.restype = C.c_int
@@ -378,6 +380,11 @@ class Context:
 
     def ss_trace_enable(self, on: bool):
         self._check(self.lib.ss_trace_enable(self.handle, 1 if on else 0), "ss_trace_enable")
+
+    def ss_cta_log_set(self, log, capacity: int = 0):
+        """log: zeroed device int64 tensor of 4 * (capacity + 1) words, or None to switch the log off."""
+        self._check(self.lib.ss_cta_log_set(self.handle, _ptr(log), capacity if log is not None else 0),
+                    "ss_cta_log_set")
 
     def ss_trace_read(self):
         """[3 roles][32 tiles][8 events] clock stamps of CTA (0,0,0) of the last traced chunk kernel."""

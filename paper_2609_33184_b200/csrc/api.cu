@@ -56,6 +56,8 @@ struct ss_ctx {
   bool no_overlap;          // set while ss_stream_round drives the context
   unsigned long long* trace;  // device trace region (in the workspace)
   bool trace_on;
+  unsigned long long* cta_log;  // caller's per-CTA log buffer (ss_cta_log_set) or null
+  int cta_log_cap;
 };
 
 namespace ss {
@@ -559,6 +561,9 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   p.status = c->status;
   p.wait_first = 0;
   p.trace = c->trace_on ? c->trace : nullptr;
+  p.cta_log = c->cta_log;
+  p.cta_log_cap = c->cta_log_cap;
+  p.launch_seq = (unsigned int)c->launches;
   if (pg) {
     p.page_table = pg->page_table;
     p.pages_per_req = pg->pages_per_req;
@@ -799,6 +804,14 @@ int32_t ss_trace_read(ss_ctx* c, uint64_t* out, int32_t max_words) {
   if (cudaMemcpy(out, c->trace, (size_t)n * sizeof(uint64_t), cudaMemcpyDeviceToHost) != cudaSuccess)
     return 0;
   return n;
+}
+
+ss_status ss_cta_log_set(ss_ctx* c, uint64_t* log, int32_t capacity) {
+  if (!c || capacity < 0 || (log && capacity == 0)) return SS_ERR_ARG;
+  if ((uintptr_t)log & 7) return SS_ERR_ALIGN;
+  c->cta_log = (unsigned long long*)log;
+  c->cta_log_cap = log ? capacity : 0;
+  return SS_OK;
 }
 
 int64_t ss_launch_count(ss_ctx* c) { return c ? c->launches : 0; }

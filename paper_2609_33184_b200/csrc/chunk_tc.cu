@@ -1,35 +1,42 @@
-// Tensor-core chunk attention for sm_100a: TMA-staged K/V tiles, tcgen05 MMAs with two score
-// tiles S (double-buffered), the probabilities P and the unnormalised output O held in tensor
-// memory.
+// Tensor-core chunk attention for sm_100a: TMA-staged K/V tiles, tcgen05 MMAs with the query
+// tile Q, the score tile S, the probabilities P and the unnormalised output O all held in
+// tensor memory.
 //
 // One CTA owns one (request, kv-head, token split, tile of <= 128 query rows).  All rows of
 // the kv-head (T_q candidate queries x G query heads) ride in the M dimension of the MMAs,
 // so every K/V byte is fetched from HBM once and serves the whole query group.
 //
 // The kernel is a template over the head dim (64 or 128); the figures below are for 128.  At 64
-// a tile is one [64][64] box per operand, the rings hold four K and six V slots (the same
-// bytes), the score MMA takes four k-steps and the output MMA has N = 64.
+// a tile is one [64][64] box per operand, the rings hold six K and six V slots, the score
+// MMA takes four k-steps and the output MMA has N = 64.
 //
-//   warp 4 (one lane)  TMA producer: K tiles and V tiles of 64 tokens, two K slots and three V
+//   warp 4 (one lane)  TMA producer: K tiles and V tiles of 64 tokens, three K slots and four V
 //                      slots, 128-byte swizzle, evict-first L2 policy (the history is
-//                      streamed).  A K slot is released as soon as its score MMAs retire
-//                      (two tiles ahead of the output MMAs), a V slot after its output MMAs,
-//                      which is why V gets the third slot.
-//   warp 5 (one lane)  MMA issuer:   S[t%2] = Q K_t^T  (M=128, N=64,  K=d=128: 8 x k16, smem x smem)
-//                                    O += P_t V_t      (M=128, N=128, K=64:    4 x k16, tmem x smem)
-//                      in the order QK(0) QK(1) | PV(0) QK(2) | PV(1) QK(3) | ...: the scores of
-//                      tile t+1 are ready before the softmax of tile t ends, so the softmax
-//                      warps never wait for the tensor pipe in steady state, and PV(t) runs
-//                      under the softmax of tile t+1.
+//                      streamed).  A K slot is released as soon as its score MMAs retire, a V
+//                      slot after its output MMAs.
+//   warp 5 (one lane)  MMA issuer:   S = Q K_t^T     (M=128, N=64,  K=d=128: 8 x k16, tmem x smem)
+//                                    O += P_t V_t    (M=128, N=128, K=64:    4 x k16, tmem x smem)
+//                      Both A operands come from tensor memory, so an MMA reads only its B
+//                      operand from shared memory (2 KB and 4 KB per k-step).  With Q in shared
+//                      memory a score MMA read 6 KB per k-step and ran at the shared-memory
+//                      bandwidth (48 instead of 32 cycles, measured), which made the tensor
+//                      pipe's queue the bound of the many-rows workloads.
 //   warps 0-3          softmax: each thread owns one TMEM lane (= one MMA row): per tile it
-//                      reads its scores, keeps (m, l) in registers and writes P as packed
-//                      bf16 over the leading columns of the same score buffer.
+//                      computes P from the scores it holds in registers, reads the NEXT tile's
+//                      scores from the score buffer into registers, and only then writes P as
+//                      packed bf16 over the leading columns of the same buffer.
 //
-// Tensor memory (256 columns): [0,64) S0, [64,128) S1 (fp32; P of a tile as bf16 pairs over
-// the first 32 columns of its buffer); [128,256) O (fp32).  Shared memory: the Q tile
-// (32 KB, written once by the softmax threads in the swizzled K-major layout), two K slots
-// and three V slots (80 KB) and 256 bytes of barriers: 112.25 KB, so that two CTAs fit per SM
-// to the last kilobyte (the window must be 1024-byte aligned; checked at run time).
+// One score buffer is enough because the double buffering happens in registers.  Arrival k of
+// the softmax threads means "S(k) is in registers and P(k-1) is in the buffer"; on it the
+// issuer runs PV(k-1) and then QK(k+1), which overwrites the buffer.  While the threads work on
+// tile k (about a thousand cycles) the tensor pipe finishes PV(k-1) and QK(k+1), so neither
+// side waits for the other in steady state.
+//
+// Tensor memory (256 columns): [0,64) S (fp32; P of a tile as bf16 pairs over its first 32
+// columns); [64,128) Q as bf16 pairs (column j of lane r = head dims 2j, 2j+1 of row r);
+// [128,256) O (fp32).  Shared memory: three K slots and four V slots (112 KB) and 256 bytes of
+// barriers, so that two CTAs fit per SM (the window must be 1024-byte aligned; checked at run
+// time).
 //
 // When the row tile has <= 32 (<= 64) rows the Q rows are replicated 4x (2x) along M and
 // each replica takes a quarter (half) of the tile's keys: lane L holds row L % R_pad and
@@ -51,40 +58,44 @@ namespace {
 
 constexpr int kThreads = 192;
 constexpr int kHalfTile = kTileKeys * 64 * 2;       // 8 KB: [64 keys][64 d] bf16, one TMA box
-constexpr int kQHalf = 128 * 64 * 2;                // 16 KB: [128 rows][64 d] bf16
 constexpr int kSmemCtl = 256;
 constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColS = 0, kColO = 128;          // S buffer t%2 at kColS + 64 (t%2)
+constexpr uint32_t kColS = 0, kColQ = 64, kColO = 128;
 constexpr float kRescaleThreshold = 8.f;
 
-// Shared-memory layout for head dim D (64 or 128): the Q tile, then the K slots, then the V
-// slots, D / 64 boxes of 64 columns each.  Head dim 64 halves a tile's bytes, so it takes twice
-// the slots (the same bytes in flight).
+// Shared-memory layout for head dim D (64 or 128): the K slots, then the V slots, D / 64 boxes
+// of 64 columns each.  Head dim 64 halves a tile's bytes, so it takes about twice the slots.
 template <int D>
 struct Lay {
   static constexpr int kHalves = D / 64;
-  static constexpr int kKStages = D == 128 ? 2 : 4, kVStages = D == 128 ? 3 : 6;
+  static constexpr int kKStages = D == 128 ? 3 : 6, kVStages = D == 128 ? 4 : 6;
   static constexpr int kTileBytes = kHalves * kHalfTile;      // one K tile or one V tile
-  static constexpr int kQBytes = kHalves * kQHalf;            // the Q tile
-  static constexpr int kOffK = kQBytes;                       // K slots
+  static constexpr int kOffK = 0;                             // K slots
   static constexpr int kOffV = kOffK + kKStages * kTileBytes; // V slots
   static constexpr int kSmemData = kOffV + kVStages * kTileBytes;  // 112 KB (d = 128), 96 KB (64)
   static constexpr int kSmemTotal = kSmemData + kSmemCtl;
   // two CTAs per SM: 227 KB per SM less 1 KB reserved per CTA
   static_assert(2 * (kSmemTotal + 1024) <= 227 * 1024, "two CTAs per SM");
+  // the write-out stages 128 rows x D floats and 128 (m, l) pairs over the idle slots
+  static_assert(kSmemData >= 128 * D * 4 + 128 * 8, "write-out staging");
   static_assert(D == 64 || D == 128, "head dim");
 };
 
 template <int KS, int VS>
 struct CtlT {
   uint64_t kfull[KS], kempty[KS], vfull[VS], vempty[VS];
-  uint64_t sfull[2], pready[2];  // per score buffer
+  uint64_t qready;               // the Q rows are in tensor memory
+  uint64_t sfull;                // one phase per tile: S(t) = Q K_t^T has retired
+  uint64_t pready[2];            // arrival k of the softmax threads (S(k) in registers, P(k-1) stored)
+                                 // goes to pready[k % 2]: a thread may make its last arrival before the
+                                 // issuer has looked at the one before it, and one barrier's parity
+                                 // could not tell the two phases apart
   uint64_t odone;                // one phase per tile: PV(t) has retired
   uint64_t pvdone;               // the last PV has retired
   uint32_t tmem_base;
   volatile uint32_t abort;
 };
-static_assert(sizeof(CtlT<2, 3>) <= kSmemCtl && sizeof(CtlT<4, 6>) <= kSmemCtl, "control block");
+static_assert(sizeof(CtlT<3, 4>) <= kSmemCtl && sizeof(CtlT<6, 6>) <= kSmemCtl, "control block");
 
 
 using namespace ss::tc;
@@ -108,21 +119,25 @@ __device__ __forceinline__ void store_p(uint32_t t_s, const uint32_t (&pk)[NC / 
 }
 
 // ---- softmax of one tile for one TMEM lane --------------------------------------------------
-// NC = number of key columns this lane owns in a 64-key tile.  P (bf16 pairs) is written
-// over the first 32 score columns: this lane's keys at [c0/2, c0/2 + NC/2), zeros elsewhere.
+// NC = number of key columns this lane owns in a 64-key tile (columns [c0, c0 + NC)).
+template <int NC>
+__device__ __forceinline__ void load_scores(uint32_t t_s, int c0, uint32_t (&raw)[NC / 16][16]) {
+#pragma unroll
+  for (int q = 0; q < NC / 16; ++q) tmem_ld16(t_s + c0 + q * 16, raw[q]);
+  tc_wait_ld();
+}
+
+// From the scores in `raw` to P as packed bf16 pairs in `pk`, updating the row state (m, l).
 // MASK = the tile straddles the valid length (columns >= n_valid are invisible).  The scale is
 // positive (checked at ss_verify_begin), so the maximum is taken on the raw scores and the
 // scaling rides in the FMA that subtracts the reference.
 // Returns false when the wait for PV(it - 1) in the rescale path gave up.
 template <int NC, bool MASK, int D, typename C>
-__device__ __forceinline__ bool softmax_tile(uint32_t t_s, uint32_t t_o, int c0, int n_valid,
-                                             int it, float scale_log2, float& m, float& l,
-                                             C* ctl, uint32_t* status) {
+__device__ __forceinline__ bool softmax_compute(uint32_t (&raw)[NC / 16][16], uint32_t t_o, int c0,
+                                                int n_valid, int it, float scale_log2, float& m,
+                                                float& l, C* ctl, uint32_t* status,
+                                                uint32_t (&pk)[NC / 16][8]) {
   const bool have_o = it > 0;
-  uint32_t raw[NC / 16][16];
-#pragma unroll
-  for (int q = 0; q < NC / 16; ++q) tmem_ld16(t_s + c0 + q * 16, raw[q]);
-  tc_wait_ld();
   float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // independent chains
   if (MASK) {
 #pragma unroll
@@ -157,7 +172,6 @@ __device__ __forceinline__ bool softmax_tile(uint32_t t_s, uint32_t t_o, int c0,
     }
   }
   const float neg_m = (m == -INFINITY) ? 0.f : -m;
-  uint32_t pk[NC / 16][8];
   // two keys per packed fp32 instruction: x = s * scale - m, then the row sum
   float2 sum2[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
   const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(neg_m, neg_m);
@@ -173,6 +187,13 @@ __device__ __forceinline__ bool softmax_tile(uint32_t t_s, uint32_t t_o, int c0,
   }
   const float2 s01 = add2_f(sum2[0], sum2[1]), s23 = add2_f(sum2[2], sum2[3]);
   l += (s01.x + s01.y) + (s23.x + s23.y);
+  return true;
+}
+
+// P of this lane's keys -> the leading 32 columns of the score buffer (zeros for the other
+// lanes' key groups), then wait for every tensor-memory store of this thread.
+template <int NC>
+__device__ __forceinline__ void store_p_at(uint32_t t_s, int c0, const uint32_t (&pk)[NC / 16][8]) {
   // c0 is uniform across a warp; dispatching on it keeps pk[] in registers
   if (NC == 64) {
     store_p<NC, 0>(t_s, pk);
@@ -188,6 +209,63 @@ __device__ __forceinline__ bool softmax_tile(uint32_t t_s, uint32_t t_o, int c0,
     }
   }
   tc_wait_st();
+}
+
+// The tile loop of one softmax thread (TMEM lane L, key columns [c0, c0 + NC) of every tile).
+// Arrival k on `pready` says: S(k) is in this thread's registers and P(k-1) is in the buffer.
+// Returns false when a bounded wait gave up.
+template <int NC, int D, typename C>
+__device__ __forceinline__ bool softmax_loop(const ChunkParams& p, C* ctl, uint32_t tmem_lane, int c0,
+                                             int n_tiles, int tok0, int tok1, uint8_t* v_s0, int L,
+                                             float& m, float& l, unsigned long long* tr) {
+  constexpr int kVStages = Lay<D>::kVStages, kTileBytes = Lay<D>::kTileBytes;
+  const uint32_t t_s = tmem_lane + kColS, t_o = tmem_lane + kColO;
+  uint32_t raw[NC / 16][16];
+  if (!mbar_wait(&ctl->sfull, 0, ctl, p.status)) return false;
+  tc_fence_after();
+  load_scores<NC>(t_s, c0, raw);
+  tc_fence_before();
+  mbar_arrive(&ctl->pready[0]);  // arrival 0: the issuer may overwrite the buffer with S(1)
+  for (int it = 0; it < n_tiles; ++it) {
+    if (L == 0) trace(tr, 2, it, 0);
+    const int n_valid = min(kTileKeys, tok1 - (tok0 + it * kTileKeys));
+    if (n_valid < kTileKeys) {
+      // ragged tail: rows past the valid length may hold anything; P is 0 there, so V must
+      // be finite: clear those rows of the staged V tile (whole 128-byte rows, both halves)
+      const int s = it % kVStages;
+      if (!mbar_wait(&ctl->vfull[s], (it / kVStages) & 1, ctl, p.status)) return false;
+      uint8_t* v_s = v_s0 + s * kTileBytes;
+      constexpr int kVecRow = D / 8;  // 16-byte pieces per token row
+      const int n_vec = (kTileKeys - n_valid) * kVecRow;
+      for (int i = L; i < n_vec; i += 128) {
+        const int row = n_valid + i / kVecRow, half = (i % kVecRow) >> 3, ch = i & 7;
+        *reinterpret_cast<uint4*>(v_s + half * kHalfTile + row * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
+      }
+      fence_proxy_async();
+    }
+    uint32_t pk[NC / 16][8];
+    const bool ok = (n_valid < kTileKeys)
+                        ? softmax_compute<NC, true, D>(raw, t_o, c0, n_valid, it, p.scale_log2, m, l, ctl, p.status, pk)
+                        : softmax_compute<NC, false, D>(raw, t_o, c0, n_valid, it, p.scale_log2, m, l, ctl, p.status, pk);
+    if (!ok) return false;
+    if (L == 0) trace(tr, 2, it, 1);
+    if (it + 1 < n_tiles) {
+      // the next tile's scores move into registers before P takes their place
+      if (!mbar_wait(&ctl->sfull, (it + 1) & 1, ctl, p.status)) return false;
+      tc_fence_after();
+      load_scores<NC>(t_s, c0, raw);
+      if (L == 0) trace(tr, 2, it, 3);
+    } else if (it > 0) {
+      // Last tile: no new scores to wait for.  PV(it - 1) still reads P(it - 1) from the columns
+      // P(it) is about to take (S(it + 1) having retired implies it in the other iterations).
+      if (!mbar_wait(&ctl->odone, (it - 1) & 1, ctl, p.status)) return false;
+      tc_fence_after();
+    }
+    store_p_at<NC>(t_s, c0, pk);
+    tc_fence_before();
+    mbar_arrive(&ctl->pready[(it + 1) & 1]);  // arrival it + 1
+    if (L == 0) trace(tr, 2, it, 2);
+  }
   return true;
 }
 
@@ -200,12 +278,12 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   constexpr int kTileBytes = L_::kTileBytes, kOffK = L_::kOffK, kOffV = L_::kOffV, kSmemData = L_::kSmemData;
   using Ctl = CtlT<kKStages, kVStages>;
   extern __shared__ __align__(1024) uint8_t smem[];
-  uint8_t* q_s = smem;             // Q tile: D / 64 halves [128 rows][64 d], 128-byte swizzle
   uint8_t* k_s = smem + kOffK;     // K slots
   uint8_t* v_s0 = smem + kOffV;    // V slots
   Ctl* ctl = reinterpret_cast<Ctl*>(smem + kSmemData);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const unsigned long long t_cta0 = p.cta_log ? cta_log_now() : 0ull;
   if (p.wait_first) pdl_wait_prior();
   pdl_launch_dependents();
   const ChunkWork w = chunk_work(p, p.rows_per_tile);
@@ -257,6 +335,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   };
   // (small pages: all copies go out from the producer warp's loop)
   const int n_pre_k = small_pages ? 0 : min(n_tiles, kKStages), n_pre_v = small_pages ? 0 : min(n_tiles, kVStages);
+  uint4 qreg[kD / 8];  // softmax threads: this lane's Q row on its way to tensor memory
   if (warp == 4) {
     if (lane == 0) {
       for (int s = 0; s < kKStages; ++s) {
@@ -267,10 +346,10 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         mbar_init(&ctl->vfull[s], 1);
         mbar_init(&ctl->vempty[s], 1);
       }
-      for (int i = 0; i < 2; ++i) {
-        mbar_init(&ctl->sfull[i], 1);
-        mbar_init(&ctl->pready[i], 128);
-      }
+      mbar_init(&ctl->qready, 128);
+      mbar_init(&ctl->sfull, 1);
+      mbar_init(&ctl->pready[0], 128);
+      mbar_init(&ctl->pready[1], 128);
       mbar_init(&ctl->odone, 1);
       mbar_init(&ctl->pvdone, 1);
       ctl->abort = 0;
@@ -289,8 +368,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   } else if (warp < 4) {
-    // this lane's Q row -> shared memory, K-major with the 128-byte swizzle the MMA descriptor
-    // expects: 16-byte chunk c of row L sits at chunk c ^ (L % 8) of the row's 128 bytes
+    // this lane's Q row, fetched while the barriers and the tensor memory are being set up
     const int r = tid % r_pad;
     const uint4* src = nullptr;
     if (r < nrows) {
@@ -299,11 +377,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
                                            t * p.q_st);
     }
 #pragma unroll
-    for (int v = 0; v < kD / 8; ++v) {
-      const uint4 x = src ? src[v] : make_uint4(0, 0, 0, 0);
-      *reinterpret_cast<uint4*>(q_s + (v >> 3) * kQHalf + tid * 128 + (((v & 7) ^ (tid & 7)) << 4)) = x;
-    }
-    fence_proxy_async();  // generic-proxy writes -> visible to the tensor core's reads
+    for (int v = 0; v < kD / 8; ++v) qreg[v] = src ? src[v] : make_uint4(0, 0, 0, 0);
   }
   tc_fence_before();
   __syncthreads();
@@ -459,38 +533,36 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     constexpr uint32_t idesc_qk = make_idesc(128, kTileKeys, false);
     constexpr uint32_t idesc_pv = make_idesc(128, kD, true);
     const bool leader = elect_one();
-    const uint32_t k_base = smem_u32(k_s), v_base = smem_u32(v_s0), q_addr = smem_u32(q_s);
+    const uint32_t k_base = smem_u32(k_s), v_base = smem_u32(v_s0);
     // The operand descriptors of one slot differ only in their address field (bits 0-13, the
     // shared-memory address / 16): they are built once and advanced by constants, which keeps
-    // the issue loop - the critical path when a tile's softmax is short - to a few
-    // instructions per MMA.  (All operand addresses are below 256 KB, so the field never carries.)
-    const uint64_t q_desc = desc_kmajor(q_addr);
+    // the issue loop to a few instructions per MMA.  (All operand addresses are below 256 KB,
+    // so the field never carries.)
     const uint64_t k_desc0 = desc_kmajor(k_base);
     const uint64_t v_desc0 = desc_mnmajor(v_base, kHalfTile);
-    // S[it % 2] = Q K_it^T; releases the K slot and signals the softmax warps
+    // S = Q K_it^T (A = Q from tensor memory); releases the K slot and signals the softmax warps
     auto issue_qk = [&](int it) {
       const int s = it % kKStages;
       const uint64_t k_desc = k_desc0 + (uint64_t)(s * (kTileBytes >> 4));
       if (leader) {
 #pragma unroll
         for (int kk = 0; kk < kD / 16; ++kk) {
-          const uint32_t qoff = (kk >> 2) * kQHalf + (kk & 3) * 32;
           const uint32_t koff = (kk >> 2) * kHalfTile + (kk & 3) * 32;
-          mma_ss(tmem + kColS + (it & 1) * 64, q_desc + (qoff >> 4), k_desc + (koff >> 4), idesc_qk, kk > 0);
+          mma_ts(tmem + kColS, tmem + kColQ + kk * 8, k_desc + (koff >> 4), idesc_qk, kk > 0);
         }
         tc_commit(&ctl->kempty[s]);
-        tc_commit(&ctl->sfull[it & 1]);
+        tc_commit(&ctl->sfull);
       }
       __syncwarp();
     };
-    // O += P_it V_it; releases the V slot, counts the tile on odone
+    // O += P_it V_it (A = P from the score buffer); releases the V slot, counts the tile on odone
     auto issue_pv = [&](int it) {
       const int s = it % kVStages;
       const uint64_t v_desc = v_desc0 + (uint64_t)(s * (kTileBytes >> 4));
       if (leader) {
 #pragma unroll
         for (int kk = 0; kk < kTileKeys / 16; ++kk) {
-          mma_ts(tmem + kColO, tmem + kColS + (it & 1) * 64 + kk * 8, v_desc + (kk * 2048 >> 4), idesc_pv,
+          mma_ts(tmem + kColO, tmem + kColS + kk * 8, v_desc + (kk * 2048 >> 4), idesc_pv,
                  (it > 0 || kk > 0));
         }
         tc_commit(&ctl->vempty[s]);
@@ -499,49 +571,41 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       }
       __syncwarp();
     };
-    // The issuer polls for whichever of its two next operations can go: the score MMAs of tile
-    // qi (K landed; score buffer qi % 2 free, i.e. the output MMAs of tile qi - 2 issued: the
-    // tensor pipe runs this thread's MMAs in issue order, so they have consumed P before the
-    // new scores overwrite it) or the output MMAs of tile pi (P ready, V landed).  The Q tile
-    // was written before the CTA-wide barrier above (with a proxy fence).
-    // (The two score buffers bound qi to pi + 1; the K ring may be deeper than that.)
-    static_assert(kKStages >= 2, "the score MMAs run up to two tiles ahead of the output MMAs");
-    int qi = 0, pi = 0;
-    unsigned long long t0 = gtime_ns();
-    uint32_t spins = 0;
-    while (pi < n_tiles) {
-      bool did = false;
-      if (qi < n_tiles && qi < pi + 2 &&
-          __all_sync(0xffffffffu, mbar_test(&ctl->kfull[qi % kKStages], (qi / kKStages) & 1))) {
-        trace(trl, 1, qi, 0);
+    // every lane waits (bounded); the outcome is made uniform
+    auto wwait = [&](uint64_t* bar, uint32_t parity) {
+      const bool ok = mbar_wait(bar, parity, ctl, p.status);
+      return __all_sync(0xffffffffu, ok);
+    };
+    // Arrival k of the softmax threads (S(k) in their registers, P(k-1) in the buffer) lets
+    // PV(k-1) and then QK(k+1) go: the tensor pipe runs one thread's MMAs in issue order, so
+    // PV(k-1) has consumed P before the new scores overwrite it.
+    bool ok = wwait(&ctl->qready, 0) && wwait(&ctl->kfull[0], 0);
+    if (ok) {
+      trace(trl, 1, 0, 0);
+      tc_fence_after();
+      issue_qk(0);
+      trace(trl, 1, 0, 5);
+    }
+    for (int k = 0; ok && k <= n_tiles; ++k) {
+      ok = wwait(&ctl->pready[k & 1], (k >> 1) & 1);
+      if (!ok) break;
+      if (k >= 1) {
+        const int it = k - 1;
+        ok = wwait(&ctl->vfull[it % kVStages], (it / kVStages) & 1);
+        if (!ok) break;
+        trace(trl, 1, it, 2);
         tc_fence_after();
-        issue_qk(qi);
-        trace(trl, 1, qi, 5);
-        ++qi;
-        did = true;
+        issue_pv(it);
+        trace(trl, 1, it, 3);
       }
-      if (pi < qi &&
-          __all_sync(0xffffffffu, mbar_test(&ctl->pready[pi & 1], (pi >> 1) & 1) &&
-                                      mbar_test(&ctl->vfull[pi % kVStages], (pi / kVStages) & 1))) {
-        trace(trl, 1, pi, 2);
+      if (k + 1 < n_tiles) {
+        const int it = k + 1;
+        ok = wwait(&ctl->kfull[it % kKStages], (it / kKStages) & 1);
+        if (!ok) break;
+        trace(trl, 1, it, 0);
         tc_fence_after();
-        issue_pv(pi);
-        trace(trl, 1, pi, 3);
-        ++pi;
-        did = true;
-      }
-      if (did) {
-        spins = 0;
-        t0 = gtime_ns();
-      } else if ((++spins & 255u) == 0) {  // bounded like every other wait
-        const bool stop = ctl->abort != 0 || gtime_ns() - t0 > kWaitNs;
-        if (__any_sync(0xffffffffu, stop)) {
-          if (lane == 0 && ctl->abort == 0) {
-            ctl->abort = 1;
-            atomicOr(p.status, SS_DEV_WAIT_EXPIRED);
-          }
-          break;
-        }
+        issue_qk(it);
+        trace(trl, 1, it, 5);
       }
     }
   } else {
@@ -553,56 +617,31 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     const int c0 = grp * nc;
     const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
     const uint32_t t_o = tmem + lane_off + kColO;
-    float m = -INFINITY, l = 0.f;
-    bool ok = true;
-    for (int it = 0; it < n_tiles; ++it) {
-      const int s = it % kVStages;
-      const uint32_t ph = (it / kVStages) & 1;
-      const uint32_t t_s = tmem + lane_off + kColS + (it & 1) * 64;
-      if (L == 0) trace(tr, 2, it, 0);
-      ok = mbar_wait(&ctl->sfull[it & 1], (it >> 1) & 1, ctl, p.status);
-      if (!ok) break;
-      tc_fence_after();
-      if (L == 0) trace(tr, 2, it, 1);
-      const int n_valid = min(kTileKeys, tok1 - (tok0 + it * kTileKeys));
-      if (n_valid < kTileKeys) {
-        // ragged tail: rows past the valid length may hold anything; P is 0 there, so V must
-        // be finite: clear those rows of the staged V tile (whole 128-byte rows, both halves)
-        ok = mbar_wait(&ctl->vfull[s], ph, ctl, p.status);
-        if (!ok) break;
-        uint8_t* v_s = v_s0 + s * kTileBytes;
-        constexpr int kVecRow = kD / 8;  // 16-byte pieces per token row
-        const int n_vec = (kTileKeys - n_valid) * kVecRow;
-        for (int i = L; i < n_vec; i += 128) {
-          const int row = n_valid + i / kVecRow, half = (i % kVecRow) >> 3, ch = i & 7;
-          *reinterpret_cast<uint4*>(v_s + half * kHalfTile + row * 128 + ch * 16) =
-              make_uint4(0, 0, 0, 0);
-        }
-        fence_proxy_async();
+    // the Q row -> tensor memory as the A operand of the score MMAs: column j of this lane
+    // holds head dims 2j and 2j + 1 (the pair's memory order)
+#pragma unroll
+    for (int q = 0; q < kD / 32; ++q) {
+      uint32_t wq[16];
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        wq[v * 4 + 0] = qreg[q * 4 + v].x;
+        wq[v * 4 + 1] = qreg[q * 4 + v].y;
+        wq[v * 4 + 2] = qreg[q * 4 + v].z;
+        wq[v * 4 + 3] = qreg[q * 4 + v].w;
       }
-#define SS_SOFTMAX_TILE(NC_, MASK_) \
-  softmax_tile<NC_, MASK_, D>(t_s, t_o, c0, n_valid, it, p.scale_log2, m, l, ctl, p.status)
-      if (n_valid < kTileKeys) {
-        if (nc == 16)
-          ok = SS_SOFTMAX_TILE(16, true);
-        else if (nc == 32)
-          ok = SS_SOFTMAX_TILE(32, true);
-        else
-          ok = SS_SOFTMAX_TILE(64, true);
-      } else {
-        if (nc == 16)
-          ok = SS_SOFTMAX_TILE(16, false);
-        else if (nc == 32)
-          ok = SS_SOFTMAX_TILE(32, false);
-        else
-          ok = SS_SOFTMAX_TILE(64, false);
-      }
-#undef SS_SOFTMAX_TILE
-      if (!ok) break;
-      tc_fence_before();
-      mbar_arrive(&ctl->pready[it & 1]);
-      if (L == 0) trace(tr, 2, it, 2);
+      tmem_st16(tmem + lane_off + kColQ + q * 16, wq);
     }
+    tc_wait_st();
+    tc_fence_before();
+    mbar_arrive(&ctl->qready);
+    float m = -INFINITY, l = 0.f;
+    bool ok;
+    if (nc == 16)
+      ok = softmax_loop<16, D>(p, ctl, tmem + lane_off, c0, n_tiles, tok0, tok1, v_s0, L, m, l, tr);
+    else if (nc == 32)
+      ok = softmax_loop<32, D>(p, ctl, tmem + lane_off, c0, n_tiles, tok0, tok1, v_s0, L, m, l, tr);
+    else
+      ok = softmax_loop<64, D>(p, ctl, tmem + lane_off, c0, n_tiles, tok0, tok1, v_s0, L, m, l, tr);
     // all output MMAs have retired (a barrier of its own: by now odone may be one or two
     // phases past the last one this thread looked at, which a parity cannot tell apart)
     ok = ok && mbar_wait(&ctl->pvdone, 0, ctl, p.status);
@@ -610,14 +649,13 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     if (ctl->abort == 0) {  // uniform over the 128 threads after the barrier
       tc_fence_after();
       // ---- merge the key groups of each row and write the partial state ----
-      // Everything below lives over the idle Q tile and K/V slots.  The 128 lanes' O rows are
+      // Everything below lives over the idle K/V slots.  The 128 lanes' O rows are
       // staged as fp32 in the layout a TMA store with the 128-byte swizzle reads: four blocks
       // of [128 rows][32 floats], 16-byte chunk c of a row at chunk c ^ (row % 8) (so a warp's
       // 16-byte accesses, one row per lane, spread over all banks); the lanes' (m, l) sit
-      // behind them in the V slots.
+      // behind them.
       float* o_s = reinterpret_cast<float*>(smem);
-      float2* ml_s = reinterpret_cast<float2*>(v_s0);
-      static_assert(kOffV >= 128 * kD * 4, "O staging must end before the (m, l) array");
+      float2* ml_s = reinterpret_cast<float2*>(smem + 128 * kD * 4);
       auto o_at = [&](int row, int c4) {  // float4 number c4 (0..31) of a staged row
         return reinterpret_cast<float4*>(o_s + (c4 >> 3) * (128 * 32) + row * 32 +
                                          (((c4 & 7) ^ (row & 7)) << 2));
@@ -696,6 +734,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols)
                  : "memory");
   }
+  if (tid == 0) cta_log_write(p, t_cta0, n_tiles);
   // Completion order along the stream: one CTA of this grid waits for the previous grid, so
   // this grid cannot complete before it (the other CTAs leave at once and free their SM slot).
   if (!p.wait_first && chain_cta) pdl_wait_prior();

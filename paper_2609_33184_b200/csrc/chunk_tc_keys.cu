@@ -107,6 +107,7 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmK) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmV) : "memory");
   }
+  const unsigned long long t_cta0 = p.cta_log ? cta_log_now() : 0ull;
   if (p.wait_first) pdl_wait_prior();
   pdl_launch_dependents();
   const ChunkWork w = chunk_work(p, p.rows_per_tile);
@@ -656,6 +657,7 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::kTmemCols)
                  : "memory");
   }
+  if (tid == 0) cta_log_write(p, t_cta0, n_tiles);
   // Completion order along the stream: one CTA of this grid waits for the previous grid, so
   // this grid cannot complete before it (the other CTAs leave at once and free their SM slot).
   if (!p.wait_first && chain_cta) pdl_wait_prior();

@@ -55,6 +55,11 @@ struct ChunkParams {
   // page_table[b][tok / page_size] of the pool, at token offset tok % page_size
   const int32_t* page_table;
   int pages_per_req, page_size, n_pages;
+  // optional per-CTA log (ss_cta_log_set): word 0 counts entries, entry i = 4 words from word
+  // 4 * (i + 1): start ns, end ns, (SM id << 32 | launch number), (linear block id << 32 | tiles)
+  unsigned long long* cta_log;
+  int cta_log_cap;
+  unsigned int launch_seq;
 };
 
 struct LocalParams {
@@ -152,6 +157,26 @@ __device__ __forceinline__ void pdl_wait_prior() {
 // of each role's tile loop.  role 0 = TMA producer, 1 = MMA issuer, 2 = softmax thread 0.
 __device__ __forceinline__ void trace(unsigned long long* tr, int role, int it, int ev) {
   if (tr && it < kTraceTiles) tr[(role * kTraceTiles + it) * 8 + ev] = clock64();
+}
+
+// Per-CTA log entry, written by one thread when the CTA leaves (no-op without a log buffer).
+__device__ __forceinline__ unsigned long long cta_log_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void cta_log_write(const ChunkParams& p, unsigned long long t_start, int n_tiles) {
+  if (!p.cta_log) return;
+  const unsigned long long i = atomicAdd(p.cta_log, 1ull);
+  if (i >= (unsigned long long)p.cta_log_cap) return;
+  unsigned int smid;
+  asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+  const unsigned long long lin = blockIdx.x + (unsigned long long)gridDim.x * (blockIdx.y + (unsigned long long)gridDim.y * blockIdx.z);
+  unsigned long long* e = p.cta_log + 4 * (i + 1);
+  e[0] = t_start;
+  e[1] = cta_log_now();
+  e[2] = ((unsigned long long)smid << 32) | p.launch_seq;
+  e[3] = (lin << 32) | (unsigned int)n_tiles;
 }
 
 // What one CTA of a chunk kernel owns: a tile of query rows of one (request, kv-head) and a

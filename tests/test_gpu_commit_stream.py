@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 import torch
 
-import bench
+from paper_2609_33184_b200 import harness
 from paper_2609_33184_b200 import inputs
 from tests import util
 
@@ -138,13 +138,13 @@ def test_call_order_and_argument_errors():
 def _stream_case(cfg, lens, batch_chunks=1, copy_only=0, accept=True, fused=True):
     ssb = _ssb()
     Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV, fill=0.0)
-    host = bench.pinned_history(cfg, lens, chunks)
+    host = harness.pinned_history(cfg, lens, chunks)
     # poison the padding of partial host blocks: those tokens must never be read into results
     for b in range(cfg.B):
         j, r = divmod(lens[b], cfg.L_c)
         if r and j < host.shape[1]:
             host[b, j, :, :, r:] = float("nan")
-    bufs = bench.stream_buffers(cfg, DEV, len(chunks), batch_chunks, fused=fused)
+    bufs = harness.stream_buffers(cfg, DEV, len(chunks), batch_chunks, fused=fused)
     for s in range(2):
         bufs["stage_k"][s].fill_(float("nan"))
         bufs["stage_v"][s].fill_(float("nan"))
@@ -161,7 +161,7 @@ def _stream_case(cfg, lens, batch_chunks=1, copy_only=0, accept=True, fused=True
                "hv": torch.zeros(shape, dtype=torch.bfloat16).pin_memory(), "cnt_host": cnt, "idx_host": idx}
     ctx = ssb.Context(cfg.B, cfg.H_q, cfg.H_kv, cfg.d, cfg.T_q, cfg.T_q,
                       cfg.L_c * (1 if fused == "blocks" else batch_chunks))
-    desc = bench.make_stream_desc(ssb, cfg, lens, host, DEV, Q, K_loc, V_loc, bits, O, LSE, bufs,
+    desc = harness.make_stream_desc(ssb, cfg, lens, host, DEV, Q, K_loc, V_loc, bits, O, LSE, bufs,
                                   batch_chunks=batch_chunks, accept=acc, copy_only=copy_only)
     stats = ctx.ss_stream_round(desc)
     st, dev_bits = ctx.ss_poll_status()
@@ -307,13 +307,13 @@ def _layer_descs(ssb, cfg, lens, n_layers, bufs, batch_chunks=1):
     for l in range(n_layers):
         cfg_l = dataclasses.replace(cfg, seed=cfg.seed + 17 * l)
         Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg_l, lens, DEV, fill=0.0)
-        host = bench.pinned_history(cfg_l, lens, chunks)
+        host = harness.pinned_history(cfg_l, lens, chunks)
         O = torch.zeros(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
         LSE = torch.zeros(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
         lb = dict(bufs)
         lb["O_host"] = torch.zeros(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16).pin_memory()
         lb["LSE_host"] = torch.zeros(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32).pin_memory()
-        desc = bench.make_stream_desc(ssb, cfg_l, lens, host, DEV, Q, K_loc, V_loc, bits, O, LSE, lb,
+        desc = harness.make_stream_desc(ssb, cfg_l, lens, host, DEV, Q, K_loc, V_loc, bits, O, LSE, lb,
                                       batch_chunks=batch_chunks)
         layers.append(dict(cfg=cfg_l, case=(Q, chunks, K_loc, V_loc, bits), host=host, O=O, LSE=LSE, desc=desc,
                            bufs=lb))
@@ -327,9 +327,9 @@ def test_stream_layers_modes_match_oracle_and_each_other(fused_restore, fills):
     lens = [1300, 200, 777]
     n_chunks = inputs.num_chunks(cfg, lens)
     if fills > 1:   # block-major fills of `fills` chunks, one copy per request and fill
-        bufs = bench.stream_buffers(cfg, DEV, n_chunks, fills, fused="blocks")
+        bufs = harness.stream_buffers(cfg, DEV, n_chunks, fills, fused="blocks")
     else:
-        bufs = bench.stream_buffers(cfg, DEV, n_chunks)
+        bufs = harness.stream_buffers(cfg, DEV, n_chunks)
     layers = _layer_descs(ssb, cfg, lens, 3, bufs, batch_chunks=fills)
     ctx = ssb.Context(cfg.B, cfg.H_q, cfg.H_kv, cfg.d, cfg.T_q, cfg.T_q, cfg.L_c)
     if fused_restore:   # K and V of a request next to each other in one buffer

@@ -390,13 +390,13 @@ def test_hinted_chunk_calls_match_unhinted():
     case = util.gen_case(cfg, lens, DEV)
     Q, chunks, K_loc, V_loc, bits = case
     ref = util.oracle_case(cfg, lens, *case)
-    import bench
-    hints = bench.host_valid(cfg, lens, len(chunks))
+    from paper_2609_33184_b200 import harness
+    hints = harness.host_valid(cfg, lens, len(chunks))
     ssb = _ssb()
     ctx = util.make_ctx(cfg)
     O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
     LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
-    bench.run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, hints=hints)
+    harness.run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, hints=hints)
     torch.cuda.synchronize()
     st, dev_bits = ctx.ss_poll_status()
     assert st == 0, dev_bits
@@ -412,14 +412,14 @@ def test_hinted_calls_skip_requests_without_tokens(flags, max_chunks):
     # sets were folded (max_chunks = 2 forces folds), with a NaN-poisoned workspace (a skipped
     # slot holds whatever an earlier round left there), with a chunk nobody has tokens in, and
     # through an exported state.
-    import bench
+    from paper_2609_33184_b200 import harness
     ssb = _ssb()
     cfg = inputs.VerifyConfig("v", 0x5E, 6, 8, 2, 128, 256, 12, 0, 1300, k_mult=2.0)
     lens = [900, 0, 300, 1300, 0, 257]
     case = util.gen_case(cfg, lens, DEV, fill=float("nan"))
     Q, chunks, K_loc, V_loc, bits = case
     ref = util.oracle_case(cfg, lens, *case)
-    hints = bench.host_valid(cfg, lens, len(chunks))
+    hints = harness.host_valid(cfg, lens, len(chunks))
     empty = (torch.zeros_like(chunks[0][0]), torch.zeros_like(chunks[0][1]), torch.zeros_like(chunks[0][2]))
     ctx = util.make_ctx(cfg, flags=flags, max_chunks=max_chunks)
     ctx.workspace[4096:].view(torch.float32)[:] = float("nan")   # past the status word and trace region
@@ -448,7 +448,7 @@ def test_hinted_calls_skip_requests_without_tokens(flags, max_chunks):
 
 def test_hinted_calls_with_a_batch_of_more_than_64_requests():
     # request lists and the merge's "absent" bits cover batches of up to 256 requests
-    import bench
+    from paper_2609_33184_b200 import harness
     ssb = _ssb()
     B = 130
     cfg = inputs.VerifyConfig("v", 0x5F, B, 4, 2, 128, 128, 4, 0, 400, k_mult=2.0)
@@ -456,12 +456,12 @@ def test_hinted_calls_with_a_batch_of_more_than_64_requests():
     lens[129] = 400
     case = util.gen_case(cfg, lens, DEV, fill=float("nan"))
     Q, chunks, K_loc, V_loc, bits = case
-    hints = bench.host_valid(cfg, lens, len(chunks))
+    hints = harness.host_valid(cfg, lens, len(chunks))
     ctx = util.make_ctx(cfg)
     ctx.workspace[8192:].view(torch.float32)[:] = float("nan")
     O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
     LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
-    bench.run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, hints=hints)
+    harness.run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, hints=hints)
     torch.cuda.synchronize()
     assert ctx.ss_poll_status() == (0, 0)
     groups = [(0, 0), (1, 1), (64, 0), (65, 1), (127, 0), (128, 1), (129, 0), (129, 1)]

@@ -7,7 +7,7 @@ import numpy as np
 import pytest
 import torch
 
-import bench
+from paper_2609_33184_b200 import harness
 import oracle
 from paper_2609_33184_b200 import inputs
 from tests import util
@@ -27,7 +27,7 @@ def test_tiering_rounds_match_oracle_and_eq9():
     tier = ssb.Tier(B, H_kv, d, L_c, T, g, cap, host, DEV)
     tier.reset([0] * B, [0] * B)
     ctx = ssb.Context(B, H_q, H_kv, d, T_q, T_q, max(L_c, cap))
-    bufs = bench.stream_buffers(cfg, DEV, max_tokens // L_c)
+    bufs = harness.stream_buffers(cfg, DEV, max_tokens // L_c)
     O = torch.empty(B, H_q, T_q, d, dtype=torch.bfloat16, device=DEV)
     LSE = torch.empty(B, H_q, T_q, dtype=torch.float32, device=DEV)
     bits = inputs.make_mask_bits(cfg, DEV)
@@ -45,7 +45,7 @@ def test_tiering_rounds_match_oracle_and_eq9():
         cnt_dev = torch.tensor(cnt, dtype=torch.int32, device=DEV)
         Hs, Cs, _, _ = tier.get()
         tk, tv, tK, tV = tier.tail()
-        desc = bench.make_stream_desc(ssb, cfg, Hs, host, DEV, Q, K_loc, V_loc,
+        desc = harness.make_stream_desc(ssb, cfg, Hs, host, DEV, Q, K_loc, V_loc,
                                       bits, O, LSE, bufs)
         desc.tail_K, desc.tail_V, desc.tail_Lc, desc.tail_len = tK, tV, cap, tier.len_dev.data_ptr()
         desc.accept_idx, desc.accept_cnt = idx.data_ptr(), cnt_dev.data_ptr()

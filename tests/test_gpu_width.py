@@ -7,7 +7,7 @@ import statistics
 import pytest
 import torch
 
-import bench
+from paper_2609_33184_b200 import harness
 from paper_2609_33184_b200 import inputs
 from tests import util
 from tests.test_width_controller import LibController
@@ -27,11 +27,11 @@ def _measured_round_ms():
     for q in WIDTHS:
         cfg = dataclasses.replace(base, T_q=q + 1)
         Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV, fill=0.0)
-        host = bench.pinned_history(cfg, lens, chunks)
-        bufs = bench.stream_buffers(cfg, DEV, len(chunks))
+        host = harness.pinned_history(cfg, lens, chunks)
+        bufs = harness.stream_buffers(cfg, DEV, len(chunks))
         O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
         LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
-        desc = bench.make_stream_desc(ssb, cfg, lens, host, DEV, Q, K_loc, V_loc, bits, O, LSE, bufs)
+        desc = harness.make_stream_desc(ssb, cfg, lens, host, DEV, Q, K_loc, V_loc, bits, O, LSE, bufs)
         ms = [ctx.ss_stream_round(desc).ms_device for _ in range(7)]
         assert ctx.ss_poll_status() == (0, 0)
         out[q] = statistics.median(ms[2:])
