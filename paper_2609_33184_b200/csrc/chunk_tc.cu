@@ -476,40 +476,24 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     if (lane == 0) {
       // streamed once: evict first; shared by the row groups of a kv-head through L2: keep
       const uint64_t pol = p.row_tiles > 1 ? l2_evict_normal_policy() : l2_evict_first_policy();
-      // K(j) can go out once QK(j - 2) has retired, V(i) once PV(i - 3) has.  The two rings free
-      // up at different times (the score MMAs run two tiles ahead of the output MMAs), so the
-      // producer polls both and issues whichever is free: a K load never queues behind a V slot
-      // that is still in use (it did in a first version, which left the K load one tile period
-      // instead of two and made the MMA issuer wait for K on every other tile).
+      // A K slot frees when its score MMAs retire, a V slot when its output MMAs do, and the
+      // issuer runs them in a fixed order: QK(0), then QK(j), PV(j - 1) for j = 1, 2, ...  The
+      // producer follows that order with blocking (bounded) waits - K(j + 3) after QK(j), V(j + 3)
+      // after PV(j - 1) - so that it sleeps in the barrier instead of taking issue slots from
+      // the softmax warp on its scheduler.
       int issued_k = n_pre_k, issued_v = n_pre_v;
-      unsigned long long t0 = gtime_ns();
-      uint32_t spins = 0;
-      while (issued_k < n_tiles || issued_v < n_tiles) {
-        bool progressed = false;
-        if (issued_k < n_tiles &&
-            mbar_test(&ctl->kempty[issued_k % kKStages], ((issued_k / kKStages) & 1) ^ 1)) {
+      for (int j = 0; issued_k < n_tiles || issued_v < n_tiles; ++j) {
+        if (issued_k < n_tiles) {
+          if (!mbar_wait(&ctl->kempty[issued_k % kKStages], ((issued_k / kKStages) & 1) ^ 1, ctl, p.status)) break;
           trace(tr, 0, issued_k, 1);
           issue_k(issued_k, pol);
           ++issued_k;
-          progressed = true;
         }
-        if (issued_v < n_tiles &&
-            mbar_test(&ctl->vempty[issued_v % kVStages], ((issued_v / kVStages) & 1) ^ 1)) {
+        if (j >= 1 && issued_v < n_tiles) {
+          if (!mbar_wait(&ctl->vempty[issued_v % kVStages], ((issued_v / kVStages) & 1) ^ 1, ctl, p.status)) break;
           trace(tr, 0, issued_v, 2);
           issue_v(issued_v, pol);
           ++issued_v;
-          progressed = true;
-        }
-        if (progressed) {
-          spins = 0;
-          t0 = gtime_ns();
-        } else if ((++spins & 255u) == 0) {  // bounded like every other wait
-          if (ctl->abort) break;
-          if (gtime_ns() - t0 > kWaitNs) {
-            ctl->abort = 1;
-            atomicOr(p.status, SS_DEV_WAIT_EXPIRED);
-            break;
-          }
         }
       }
       if (ctl->abort) {
