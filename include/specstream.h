@@ -95,6 +95,9 @@ typedef struct {
 #define SS_FLAG_ROWS_ON_M 4u
 /* Use the keys-on-M kernel for any number of rows per kv-head (default: up to 32). */
 #define SS_FLAG_KEYS_ON_M 8u
+/* ss_stream_round also times its phases with device events (read with ss_get_stats):
+ * an event pair around every chunk call and one around the local / finalize / commit tail. */
+#define SS_FLAG_STREAM_TIMING 16u
 /* Tuning overrides read from the environment by ss_create (for experiments; unset = automatic):
  *   SS_CHUNK_KERNEL=rows|keys  as SS_FLAG_ROWS_ON_M / SS_FLAG_KEYS_ON_M
  *   SS_SPLITS=n                token splits of every chunk call (default: sized so that a
@@ -160,9 +163,12 @@ ss_status ss_verify_chunk_paged(ss_ctx* ctx, ss_tensor K_pool, ss_tensor V_pool,
                                 int32_t page_size, const int32_t* page_table, int32_t pages_per_req,
                                 const int32_t* valid_len, const int32_t* valid_len_host, void* stream);
 
-/* a4. The on-GPU candidate segment: K_loc, V_loc [B, H_kv, T_loc, d].  Query i of request
- * b sees local token j iff
- *   SS_MASK_CHAIN:     j <= i + (T_loc - T_q)   (causal, inclusive; mask_bits ignored)
+/* a4. The on-GPU candidate segment (Section 4.2: the pass over the GPU-resident Active Tail and
+ * Speculative Frontier; the mask M of Eq. 12): K_loc, V_loc [B, H_kv, T_loc, d].  Query i of
+ * request b sees local token j iff
+ *   SS_MASK_CHAIN:     j <= i + (T_loc - T_q)   (causal, inclusive; mask_bits ignored;
+ *                      T_loc >= T_q, SS_ERR_ARG otherwise: the T_loc - T_q leading local
+ *                      tokens - an Active Tail passed with the candidates - are seen by all)
  *   SS_MASK_TREE_BITS: bit j of mask_bits[b][i][j/64] is set (device uint64
  *                      [B, T_q, ceil(T_loc/64)]; row i = ancestors of node i and i itself). */
 ss_status ss_verify_local(ss_ctx* ctx, ss_tensor K_loc, ss_tensor V_loc, int32_t T_loc,
@@ -271,6 +277,7 @@ typedef struct {
   int32_t copies;
 } ss_stream_stats;
 
+/* SS_ERR_STATE, touching nothing, while the caller has a round open on this context. */
 ss_status ss_stream_round(ss_ctx* ctx, const ss_stream_desc* desc, ss_stream_stats* stats);
 
 /* Several layers back to back through the same two staging buffers (Section 4.2, pipelined KV
@@ -288,6 +295,16 @@ ss_status ss_stream_round(ss_ctx* ctx, const ss_stream_desc* desc, ss_stream_sta
  * Every layer has its own descriptor (history, Q, local KV, outputs); all layers use the same
  * B, T_q, L_c, batch_chunks and staging buffers.  Layers may share the valid_len scratch arrays
  * only if their history lengths are identical.  Synchronous; `total` covers all layers. */
+typedef enum { SS_LAYERS_PREFETCH = 0, SS_LAYERS_STREAM = 1, SS_LAYERS_RESTORE = 2 } ss_layers_mode;
+typedef struct {
+  int32_t n_layers;            /* <= 256                                                   */
+  const ss_stream_desc* layers; /* HOST array [n_layers]                                   */
+  int32_t mode;                /* ss_layers_mode                                           */
+  void* restore_k;             /* device; SS_LAYERS_RESTORE only                           */
+  void* restore_v;             /* NULL: restore_k holds K and V (see above)                */
+  int64_t restore_tokens;      /* token capacity of a restore buffer row                   */
+} ss_layers_desc;
+ss_status ss_stream_layers(ss_ctx* ctx, const ss_layers_desc* layers, ss_stream_stats* total);
 /* Commit-aware KV tiering (Section 4.1).  Per request: Sealed History [0, H) in pinned host
  * memory (chunk-block layout of ss_stream_round), Active Tail [H, C) in a device buffer
  * [B, H_kv, tail_capacity, d] (token t at index t - H).  ss_tier_commit advances C by the rows a
@@ -361,16 +378,6 @@ typedef struct {
 int32_t ss_cohort_build(const ss_task* tasks, int32_t n, int32_t max_batch, int32_t* order,
                         int32_t* cohort_start);
 
-typedef enum { SS_LAYERS_PREFETCH = 0, SS_LAYERS_STREAM = 1, SS_LAYERS_RESTORE = 2 } ss_layers_mode;
-typedef struct {
-  int32_t n_layers;            /* <= 256                                                   */
-  const ss_stream_desc* layers; /* HOST array [n_layers]                                   */
-  int32_t mode;                /* ss_layers_mode                                           */
-  void* restore_k;             /* device; SS_LAYERS_RESTORE only                           */
-  void* restore_v;             /* NULL: restore_k holds K and V (see above)                */
-  int64_t restore_tokens;      /* token capacity of a restore buffer row                   */
-} ss_layers_desc;
-ss_status ss_stream_layers(ss_ctx* ctx, const ss_layers_desc* layers, ss_stream_stats* total);
 
 /* A whole round (one history chunk + local segment -> O, LSE) that allocates nothing and
  * needs no context or workspace.  The paper has no counterpart: this exists for callers that
@@ -385,7 +392,12 @@ ss_status ss_stream_layers(ss_ctx* ctx, const ss_layers_desc* layers, ss_stream_
  *  - Returns SS_ERR_CAPACITY, enqueuing nothing, when the round's partial states
  *    (2 * splits * B * H_kv * T_q * G rows of (d + 2) floats, splits <= 16) do not fit.
  *  - The first call on a device looks up the array's device address (with that device
- *    current); make that first call before any stream capture.  No call allocates or frees.
+ *    current; host threads may race to it); make that first call before any stream capture.
+ *    Any call does, even one that is rejected for its arguments: ss_verify_round_static(NULL,
+ *    NULL) is a valid warm-up (it returns SS_ERR_ARG).  No call allocates or frees.
+ *  - Shapes are limited like the regular entry points' (T_q * H_q / H_kv <= 4096,
+ *    B * H_q * T_q < 2^31: SS_ERR_SHAPE); mask_kind must be one of the two kinds and a chain
+ *    mask needs T_loc >= T_q (SS_ERR_ARG).
  *  - All calls share the array: it keeps the last call's contents (the call clears what must
  *    start at zero), and calls whose kernels may overlap on the GPU race - serialise them.
  *  - `status` (optional DEVICE word, OR-ed with SS_DEV_* bits) receives device-detected
@@ -444,9 +456,30 @@ ss_status ss_selftest_wait_expiry(ss_ctx* ctx, int32_t limit_ms, uint32_t* gave_
  * GPU in its current clock state. */
 ss_status ss_probe_read(const void* const* srcs, const size_t* bytes, int32_t n, uint64_t* sink,
                         void* stream);
+/* Counters of a context (the paper has no counterpart; its width controller, Section 4.2,
+ * consumes the transfer and compute times of a round, which the last_* fields provide).
+ * The last_* fields describe the most recent ss_stream_round of a context created with
+ * SS_FLAG_STREAM_TIMING and are 0 otherwise; they are device-event times in nanoseconds. */
+typedef struct {
+  int64_t launches;      /* kernels launched since creation                                      */
+  int64_t rounds;        /* rounds finalized                                                     */
+  int64_t rows;          /* query rows finalized (B * H_q * T_q summed over the rounds)          */
+  int64_t chunk_calls;   /* chunk calls of any kind                                              */
+  int64_t kv_bytes;      /* K/V bytes those calls covered: the valid tokens where the call had a
+                            host copy of the lengths (or no lengths at all), else every token
+                            of the chunk (an upper bound)                                        */
+  int64_t last_round_ns;     /* first copy enqueued -> last device-to-host copy done             */
+  int64_t last_transfer_ns;  /* copy stream: first history copy -> last history copy done        */
+  int64_t last_chunk_ns;     /* attention stream: sum over the chunk calls of their kernel time  */
+  int64_t last_tail_ns;      /* local segment + finalize + commit-gather + copies to the host    */
+  int64_t last_wait_ns;      /* last_round_ns - last_chunk_ns - last_tail_ns: the attention
+                                stream waiting for transfers (the paper's exposed transfer time)  */
+} ss_stats;
+ss_status ss_get_stats(ss_ctx* ctx, ss_stats* out);
 /* Number of kernels this context has launched since creation. */
 int64_t ss_launch_count(ss_ctx* ctx);
-/* "simt" or "tcgen05": the chunk kernel the last ss_verify_chunk used. */
+/* "simt", "tcgen05" (rows on M) or "tcgen05-keys" (keys on M): the chunk kernel the last chunk
+ * call used; "none" before the first. */
 const char* ss_last_chunk_kernel(ss_ctx* ctx);
 
 #ifdef __cplusplus

@@ -22,7 +22,7 @@ STATUS_NAMES = ["SS_OK", "SS_ERR_ARG", "SS_ERR_SHAPE", "SS_ERR_ALIGN", "SS_ERR_S
 (SS_ERR_ARG, SS_ERR_SHAPE, SS_ERR_ALIGN, SS_ERR_STATE, SS_ERR_CAPACITY, SS_ERR_UNSUPPORTED,
  SS_ERR_CUDA, SS_ERR_DEVICE_FLAG, SS_ERR_TIMEOUT) = range(1, 10)
 SS_DEV_BAD_VALID_LEN, SS_DEV_BAD_ACCEPT, SS_DEV_DST_OVERFLOW, SS_DEV_WAIT_EXPIRED, SS_DEV_BAD_PAGE = 1, 2, 4, 8, 16
-SS_FLAG_FORCE_SIMT, SS_FLAG_OVERLAP_CHUNKS, SS_FLAG_ROWS_ON_M, SS_FLAG_KEYS_ON_M = 1, 2, 4, 8
+SS_FLAG_FORCE_SIMT, SS_FLAG_OVERLAP_CHUNKS, SS_FLAG_ROWS_ON_M, SS_FLAG_KEYS_ON_M, SS_FLAG_STREAM_TIMING = 1, 2, 4, 8, 16
 SS_MASK_CHAIN, SS_MASK_TREE_BITS = 0, 1
 
 EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "ss_verify_chunk",
@@ -33,7 +33,13 @@ EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "
            "ss_tier_reset", "ss_tier_get", "ss_tier_tail", "ss_tier_commit", "ss_tier_migrate", "ss_tier_poll",
            "ss_tier_d2h_bytes", "ss_verify_chunk_paged", "ss_width_create", "ss_width_destroy",
            "ss_width_observe", "ss_width_next", "ss_width_estimate", "ss_cohort_build", "ss_probe_read",
-           "ss_selftest_wait_expiry", "ss_verify_abort", "ss_cta_log_set"]
+           "ss_selftest_wait_expiry", "ss_verify_abort", "ss_cta_log_set", "ss_get_stats"]
+
+
+class ss_stats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("launches", "rounds", "rows", "chunk_calls", "kv_bytes",
+                                         "last_round_ns", "last_transfer_ns", "last_chunk_ns",
+                                         "last_tail_ns", "last_wait_ns")]
 
 
 class ss_config(C.Structure):
@@ -198,6 +204,8 @@ def load() -> C.CDLL:
     lib.ss_last_cuda_error.argtypes = [vp]
     lib.ss_trace_enable.restype = C.c_int
     lib.ss_trace_enable.argtypes = [vp, i32]
+    lib.ss_get_stats.restype = C.c_int
+    lib.ss_get_stats.argtypes = [vp, C.POINTER(ss_stats)]
     lib.ss_cta_log_set.restype = C.c_int
     lib.ss_cta_log_set.argtypes = [vp, vp, i32]
     lib.ss_trace_read.restype = i32
@@ -380,6 +388,11 @@ class Context:
 
     def ss_trace_enable(self, on: bool):
         self._check(self.lib.ss_trace_enable(self.handle, 1 if on else 0), "ss_trace_enable")
+
+    def ss_get_stats(self) -> ss_stats:
+        st = ss_stats()
+        self._check(self.lib.ss_get_stats(self.handle, C.byref(st)), "ss_get_stats")
+        return st
 
     def ss_cta_log_set(self, log, capacity: int = 0):
         """log: zeroed device int64 tensor of 4 * (capacity + 1) words, or None to switch the log off."""

@@ -58,6 +58,9 @@ struct ss_ctx {
   bool trace_on;
   unsigned long long* cta_log;  // caller's per-CTA log buffer (ss_cta_log_set) or null
   int cta_log_cap;
+  ss_stats stats;           // counters (launches is filled in when they are read)
+  cudaEvent_t* ev_pool;     // timing events of the streamed round (SS_FLAG_STREAM_TIMING)
+  int ev_pool_n;
 };
 
 namespace ss {
@@ -578,6 +581,18 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   if (e != cudaSuccess) return cuda_fail(c, e);
   c->last_kernel = !tc ? "simt" : keys_on_m ? "tcgen05-keys" : "tcgen05";
   ++c->launches;
+  ++c->stats.chunk_calls;
+  {
+    int64_t tokens = (int64_t)c->B * L_c;  // no lengths, or lengths only the device knows
+    if (valid_len && valid_len_host) {
+      tokens = 0;
+      for (int b = 0; b < c->B; ++b) {
+        const int v = valid_len_host[b];
+        tokens += v < 0 ? 0 : (v > L_c ? L_c : v);
+      }
+    }
+    c->stats.kv_bytes += tokens * c->cfg.H_kv * c->cfg.d * 4;  // K and V, 2 bytes each
+  }
   c->splits[c->n_sets] = (uint8_t)splits;
   if (hint.n_listed) memcpy(c->absent[c->n_sets], hint.absent, sizeof(hint.absent));
   else memset(c->absent[c->n_sets], 0, sizeof(hint.absent));
@@ -597,6 +612,9 @@ ss_status ss_verify_local(ss_ctx* c, ss_tensor K_loc, ss_tensor V_loc, int32_t T
   if (mask_bits && ((uintptr_t)mask_bits & 7)) return SS_ERR_ALIGN;
   if (c->state != ss_ctx::OPEN || (cudaStream_t)stream != c->stream || c->has_local)
     return SS_ERR_STATE;
+  // chain rule j <= i + (T_loc - T_q): with fewer local tokens than queries the leading rows
+  // would see nothing of the local segment, which no caller means
+  if (kind == SS_MASK_CHAIN && T_loc < c->T_q) return SS_ERR_ARG;
   ss::LocalParams p;
   memset(&p, 0, sizeof(p));
   p.Q = (const __nv_bfloat16*)c->Q.ptr;
@@ -682,6 +700,8 @@ ss_status ss_verify_finalize(ss_ctx* c, void* O, float* LSE, void* stream) {
   cudaError_t e = ss::launch_finalize(m, c->stream, use_pdl(c));
   if (e != cudaSuccess) return cuda_fail(c, e);
   ++c->launches;
+  ++c->stats.rounds;
+  c->stats.rows += (int64_t)c->B * c->cfg.H_q * c->T_q;
   c->state = ss_ctx::IDLE;
   c->Q.ptr = nullptr;
   return SS_OK;
@@ -814,6 +834,13 @@ ss_status ss_cta_log_set(ss_ctx* c, uint64_t* log, int32_t capacity) {
   return SS_OK;
 }
 
+ss_status ss_get_stats(ss_ctx* c, ss_stats* out) {
+  if (!c || !out) return SS_ERR_ARG;
+  *out = c->stats;
+  out->launches = c->launches;
+  return SS_OK;
+}
+
 int64_t ss_launch_count(ss_ctx* c) { return c ? c->launches : 0; }
 const char* ss_last_chunk_kernel(ss_ctx* c) { return c ? c->last_kernel : "none"; }
 
@@ -836,6 +863,10 @@ void pipeline_release(ss_ctx* c) {
   }
   if (c->ev_t0) cudaEventDestroy(c->ev_t0);
   if (c->ev_t1) cudaEventDestroy(c->ev_t1);
+  for (int i = 0; i < c->ev_pool_n; ++i) cudaEventDestroy(c->ev_pool[i]);
+  delete[] c->ev_pool;
+  c->ev_pool = nullptr;
+  c->ev_pool_n = 0;
   c->copy_stream = c->attn_stream = nullptr;
   c->ev_ready[0] = c->ev_ready[1] = c->ev_free[0] = c->ev_free[1] = c->ev_t0 = c->ev_t1 = nullptr;
   c->pipe_ready = false;
@@ -866,6 +897,30 @@ cudaError_t ctx_pipeline(ss_ctx* c, PipeRes* out) {
   out->ev_t1 = c->ev_t1;
   return cudaSuccess;
 }
+// Timing events for the streamed round: at least n of them, or null when the context was
+// created without SS_FLAG_STREAM_TIMING (or they cannot be had).  Grown on demand, kept.
+cudaEvent_t* ctx_timing_events(ss_ctx* c, int n) {
+  if (!(c->cfg.flags & SS_FLAG_STREAM_TIMING)) return nullptr;
+  if (n <= c->ev_pool_n) return c->ev_pool;
+  cudaEvent_t* grown = new (std::nothrow) cudaEvent_t[n];
+  if (!grown) return nullptr;
+  for (int i = 0; i < c->ev_pool_n; ++i) grown[i] = c->ev_pool[i];
+  int have = c->ev_pool_n;
+  for (; have < n; ++have)
+    if (cudaEventCreate(&grown[have]) != cudaSuccess) break;
+  delete[] c->ev_pool;
+  c->ev_pool = grown;
+  c->ev_pool_n = have;
+  return have >= n ? c->ev_pool : nullptr;
+}
+void ctx_set_stream_times(ss_ctx* c, int64_t round_ns, int64_t transfer_ns, int64_t chunk_ns, int64_t tail_ns) {
+  c->stats.last_round_ns = round_ns;
+  c->stats.last_transfer_ns = transfer_ns;
+  c->stats.last_chunk_ns = chunk_ns;
+  c->stats.last_tail_ns = tail_ns;
+  const int64_t w = round_ns - chunk_ns - tail_ns;
+  c->stats.last_wait_ns = w > 0 ? w : 0;
+}
 int ctx_dims(ss_ctx* c, int* H_q, int* H_kv, int* d) {
   *H_q = c->cfg.H_q;
   *H_kv = c->cfg.H_kv;
@@ -874,9 +929,12 @@ int ctx_dims(ss_ctx* c, int* H_q, int* H_kv, int* d) {
 }
 void ctx_set_cuda_error(ss_ctx* c, cudaError_t e) { c->last_cuda = (int32_t)e; }
 uint32_t* ctx_status_word(ss_ctx* c) { return c->status; }
+bool ctx_round_open(ss_ctx* c) { return c->state != ss_ctx::IDLE; }
+// The streamed entry points refuse to start while the caller has a round open, so a round
+// that is open when they finish is one of their own (error path) and is dropped.
 void ctx_pipeline_mode(ss_ctx* c, bool on) {
   c->no_overlap = on;
-  if (!on) c->state = ss_ctx::IDLE;  // a round the pipeline left open (error path) is dropped
+  if (!on) c->state = ss_ctx::IDLE;
 }
 // Error path of the pipeline: what was enqueued before the failing call still reads the caller's
 // buffers, so wait for it before the error is returned.

@@ -15,6 +15,7 @@
 // reads is rewritten by the call itself.  Two calls whose kernels can overlap on the GPU
 // (different streams) race on the array: callers serialise them.
 #include <cstring>
+#include <mutex>
 
 #include "ss_internal.h"
 
@@ -30,11 +31,13 @@ struct DeviceSlot {
   unsigned char* base;  // device address of g_static_scratch on this device
 };
 DeviceSlot g_slots[kMaxDevices];
+std::mutex g_slots_mutex;  // host threads may make their first calls on a device at the same time
 
 // First call on a device: resolve the array's device address (no allocation involved).
 ss_status scratch_for_current_device(unsigned char** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SS_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_slots_mutex);
   DeviceSlot& s = g_slots[dev];
   if (!s.ready) {
     int major = 0;
@@ -59,25 +62,37 @@ bool tensor_ok(const ss_tensor& t) {
 }  // namespace
 
 extern "C" ss_status ss_verify_round_static(const ss_static_round* r, void* stream) {
+  // The set-up (address of the scratch array on the current device) comes first, so that any
+  // call - even one rejected for its arguments, e.g. with r == NULL - serves as the warm-up
+  // call that has to precede a stream capture.  Its own error is reported after the argument
+  // checks, which need no device.
+  unsigned char* base = nullptr;
+  const ss_status setup = scratch_for_current_device(&base);
   if (!r || !r->O) return SS_ERR_ARG;
   if (r->B <= 0 || r->H_q <= 0 || r->H_kv <= 0 || r->T_q <= 0 || r->L_c < 0 || r->T_loc < 0)
     return SS_ERR_ARG;
   if (r->H_q % r->H_kv || (r->d != 64 && r->d != 128) || r->T_loc > 1024) return SS_ERR_SHAPE;
+  // the limits of the regular entry points: the row-per-warp kernels index query rows with
+  // 32-bit arithmetic and a kv-head carries at most 4096 rows
+  if ((int64_t)r->T_q * (r->H_q / r->H_kv) > 4096) return SS_ERR_SHAPE;
+  if ((int64_t)r->B * r->H_q * r->T_q >= (1ll << 31)) return SS_ERR_SHAPE;
   if (r->L_c == 0 && r->T_loc == 0) return SS_ERR_ARG;
   if (!(r->scale > 0.f) || !(r->scale < 3.0e38f)) return SS_ERR_ARG;
+  if (r->T_loc > 0 && r->mask_kind != SS_MASK_CHAIN && r->mask_kind != SS_MASK_TREE_BITS) return SS_ERR_ARG;
+  if (r->T_loc > 0 && r->mask_kind == SS_MASK_CHAIN && r->T_loc < r->T_q) return SS_ERR_ARG;
   if (!tensor_ok(r->Q) || !aligned16(r->O)) return SS_ERR_ALIGN;
   if (r->L_c > 0 && (!tensor_ok(r->K) || !tensor_ok(r->V))) return SS_ERR_ALIGN;
   if (r->T_loc > 0 && (!tensor_ok(r->K_loc) || !tensor_ok(r->V_loc))) return SS_ERR_ALIGN;
   if (r->T_loc > 0 && r->mask_kind == SS_MASK_TREE_BITS && !r->mask_bits) return SS_ERR_ARG;
 
   const int G = r->H_q / r->H_kv;
-  const int R = r->T_q * G;
-  const int pairs = r->B * r->H_kv;
+  const int R = r->T_q * G;                                  // <= 4096
+  const int64_t pairs = (int64_t)r->B * r->H_kv;
+  const int64_t row_tiles = (R + 31) / 32;
   const int n_tiles = (r->L_c + ss::kTileKeys - 1) / ss::kTileKeys;
-  const int row_tiles = (R + 31) / 32;
   int splits = 1;
   if (n_tiles > 0) {
-    splits = ss::kNumSM / (pairs * row_tiles);
+    splits = (int)(ss::kNumSM / (pairs * row_tiles));   // pairs * row_tiles >= 1
     if (splits > ss::kMaxSplits) splits = ss::kMaxSplits;
     if (splits > (n_tiles + 1) / 2) splits = (n_tiles + 1) / 2;
     if (splits < 1) splits = 1;
@@ -86,15 +101,15 @@ extern "C" ss_status ss_verify_round_static(const ss_static_round* r, void* stre
   if (n_tiles) splits = (n_tiles + tiles_per_split - 1) / tiles_per_split;
 
   // layout inside the scratch: [256 B header: status word] [ml: sets x slots x R] [a: ... x d]
-  const size_t rows_per_set = (size_t)splits * pairs * R;   // set 0 = history chunk, set 1 = local
+  // (rows of one set: at most 16 * 2^31 / T_q, far inside 64 bits; a set that large fails the
+  // capacity check below)
+  const size_t rows_per_set = (size_t)splits * (size_t)pairs * (size_t)R;   // set 0 = history chunk, set 1 = local
+  if (rows_per_set > SS_STATIC_SCRATCH_BYTES) return SS_ERR_CAPACITY;
   const size_t ml_bytes = 2 * rows_per_set * sizeof(float2);
   const size_t off_a = 256 + ((ml_bytes + 255) / 256) * 256;
   const size_t need = off_a + 2 * rows_per_set * r->d * sizeof(float);
   if (need > SS_STATIC_SCRATCH_BYTES) return SS_ERR_CAPACITY;
-
-  unsigned char* base = nullptr;
-  ss_status st = scratch_for_current_device(&base);
-  if (st != SS_OK) return st;
+  if (setup != SS_OK) return setup;
   cudaStream_t s = (cudaStream_t)stream;
   uint32_t* status = r->status ? r->status : reinterpret_cast<uint32_t*>(base);
   // the shared array keeps the last call's contents: clear the word that must start at zero
@@ -128,7 +143,7 @@ extern "C" ss_status ss_verify_round_static(const ss_static_round* r, void* stre
     p.L_c = r->L_c;
     p.splits = splits;
     p.tiles_per_split = tiles_per_split;
-    p.row_tiles = row_tiles;
+    p.row_tiles = (int)row_tiles;
     p.rows_per_tile = 32;
     p.scale_log2 = scale_log2;
     p.part_ml = part_ml;

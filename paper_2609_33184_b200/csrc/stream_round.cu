@@ -19,6 +19,9 @@ cudaError_t ctx_pipeline(ss_ctx* c, PipeRes* out);
 int ctx_dims(ss_ctx* c, int* H_q, int* H_kv, int* d);
 void ctx_set_cuda_error(ss_ctx* c, cudaError_t e);
 void ctx_pipeline_mode(ss_ctx* c, bool on);
+bool ctx_round_open(ss_ctx* c);
+cudaEvent_t* ctx_timing_events(ss_ctx* c, int n);
+void ctx_set_stream_times(ss_ctx* c, int64_t round_ns, int64_t transfer_ns, int64_t chunk_ns, int64_t tail_ns);
 void ctx_pipeline_drain(ss_ctx* c);
 }  // namespace ss
 
@@ -41,7 +44,26 @@ namespace {
 struct LayerCounts {
   int64_t h2d = 0, d2h = 0;
   int copies = 0, calls = 0, fills = 0;
+  // phase timing (ss_stream_round with SS_FLAG_STREAM_TIMING): ev[0] = last history copy done,
+  // ev[1] = start of the local / finalize / commit tail, ev[2 + 2i], ev[3 + 2i] around chunk call i
+  cudaEvent_t* ev = nullptr;
+  int ev_cap = 0, timed_calls = 0;
 };
+
+// A chunk call of the streamed round, with an event pair around it when the round is timed.
+ss_status timed_chunk(ss_ctx* ctx, LayerCounts* cnt, cudaStream_t s, ss_tensor K, ss_tensor V, int32_t L_c,
+                      const int32_t* vl_dev, const int32_t* vl_host) {
+  const bool timed = cnt->ev && 3 + 2 * cnt->timed_calls < cnt->ev_cap;
+  if (timed) SS_CK(cudaEventRecord(cnt->ev[2 + 2 * cnt->timed_calls], s));
+  SS_ST(vl_host ? ss_verify_chunk_hinted(ctx, K, V, L_c, vl_dev, vl_host, s)
+                : ss_verify_chunk(ctx, K, V, L_c, vl_dev, s));
+  if (timed) {
+    SS_CK(cudaEventRecord(cnt->ev[3 + 2 * cnt->timed_calls], s));
+    ++cnt->timed_calls;
+  }
+  ++cnt->calls;
+  return SS_OK;
+}
 
 ss_status validate_desc(ss_ctx* ctx, const ss_stream_desc* d, int* n_fills_out) {
   if (!d || !d->hist || !d->hist_len) return SS_ERR_ARG;
@@ -107,8 +129,7 @@ ss_status enqueue_layer(ss_ctx* ctx, const ss_stream_desc* d, const ss::PipeRes&
     SS_ST(ss_verify_begin(ctx, d->Q, B, d->T_q, d->scale, r.attn_stream));
     if (d->tail_K.ptr) {  // on-GPU Active Tail: no copy, runs while the first fills arrive
       if (!d->tail_V.ptr || d->tail_Lc <= 0) return SS_ERR_ARG;
-      SS_ST(ss_verify_chunk(ctx, d->tail_K, d->tail_V, d->tail_Lc, d->tail_len, r.attn_stream));
-      ++cnt->calls;
+      SS_ST(timed_chunk(ctx, cnt, r.attn_stream, d->tail_K, d->tail_V, d->tail_Lc, d->tail_len, nullptr));
     }
   }
 
@@ -154,9 +175,8 @@ ss_status enqueue_layer(ss_ctx* ctx, const ss_stream_desc* d, const ss::PipeRes&
           const uint16_t* kb = (const uint16_t*)d->stage_k[buf] + (int64_t)jj * block_elems;
           ss_tensor K = {kb, (int64_t)bc * block_elems, head_elems, hd};
           ss_tensor V = {kb + (int64_t)H_kv * head_elems, (int64_t)bc * block_elems, head_elems, hd};
-          SS_ST(ss_verify_chunk_hinted(ctx, K, V, L_c, d->valid_len_dev + (int64_t)j * B,
-                                       d->valid_len_host + (int64_t)j * B, r.attn_stream));
-          ++cnt->calls;
+          SS_ST(timed_chunk(ctx, cnt, r.attn_stream, K, V, L_c, d->valid_len_dev + (int64_t)j * B,
+                            d->valid_len_host + (int64_t)j * B));
         }
       }
       SS_CK(cudaEventRecord(r.ev_free[buf], r.attn_stream));
@@ -215,9 +235,8 @@ ss_status enqueue_layer(ss_ctx* ctx, const ss_stream_desc* d, const ss::PipeRes&
         K.stride_b = V.stride_b = 2 * (int64_t)H_kv * Ls * hd;
         V.ptr = (const uint16_t*)d->stage_k[buf] + (int64_t)H_kv * Ls * hd;
       }
-      SS_ST(ss_verify_chunk_hinted(ctx, K, V, (int32_t)Ls, d->valid_len_dev + (int64_t)f * B,
-                                   d->valid_len_host + (int64_t)f * B, r.attn_stream));
-      ++cnt->calls;
+      SS_ST(timed_chunk(ctx, cnt, r.attn_stream, K, V, (int32_t)Ls, d->valid_len_dev + (int64_t)f * B,
+                        d->valid_len_host + (int64_t)f * B));
     }
     SS_CK(cudaEventRecord(r.ev_free[buf], r.attn_stream));
   }
@@ -236,12 +255,15 @@ ss_status enqueue_layer(ss_ctx* ctx, const ss_stream_desc* d, const ss::PipeRes&
         K.stride_b = V.stride_b = 2 * (int64_t)H_kv * Ls * hd;
         V.ptr = (const uint16_t*)restore_k + (int64_t)H_kv * Ls * hd + tok * hd;
       }
-      SS_ST(ss_verify_chunk_hinted(ctx, K, V, (int32_t)span, d->valid_len_dev + (int64_t)f * B,
-                                   d->valid_len_host + (int64_t)f * B, r.attn_stream));
-      ++cnt->calls;
+      SS_ST(timed_chunk(ctx, cnt, r.attn_stream, K, V, (int32_t)span, d->valid_len_dev + (int64_t)f * B,
+                        d->valid_len_host + (int64_t)f * B));
     }
   }
   cnt->fills += n_fills;
+  if (cnt->ev) {
+    SS_CK(cudaEventRecord(cnt->ev[0], r.copy_stream));   // the last history copy is behind this
+    SS_CK(cudaEventRecord(cnt->ev[1], r.attn_stream));   // the tail starts here
+  }
   if (!d->copy_only) {
     SS_ST(ss_verify_local(ctx, d->K_loc, d->V_loc, d->T_q, d->mask_kind, d->mask_bits, r.attn_stream));
     SS_ST(ss_verify_finalize(ctx, d->O, d->LSE, r.attn_stream));
@@ -294,12 +316,28 @@ ss_status stream_round_impl(ss_ctx* ctx, const ss_stream_desc* d, ss_stream_stat
   const auto wall0 = std::chrono::steady_clock::now();
   SS_CK(cudaEventRecord(r.ev_t0, r.copy_stream));
   LayerCounts cnt;
+  // one event pair per chunk call (a fill of the block-major layout is batch_chunks calls, the
+  // Active Tail one more) plus the two phase marks
+  cnt.ev_cap = 2 + 2 * (n_fills * d->batch_chunks + 1);
+  cnt.ev = ss::ctx_timing_events(ctx, cnt.ev_cap);
   SS_ST(enqueue_layer(ctx, d, r, n_fills, 0, nullptr, nullptr, 0, &cnt));
   SS_CK(cudaEventRecord(r.ev_t1, r.attn_stream));
   SS_CK(cudaEventSynchronize(r.ev_t1));
   SS_CK(cudaStreamSynchronize(r.copy_stream));
   float ms = 0.f;
   SS_CK(cudaEventElapsedTime(&ms, r.ev_t0, r.ev_t1));
+  if (cnt.ev) {
+    float t = 0.f, transfer = 0.f, tail = 0.f;
+    double chunk = 0.0;
+    SS_CK(cudaEventElapsedTime(&transfer, r.ev_t0, cnt.ev[0]));
+    SS_CK(cudaEventElapsedTime(&tail, cnt.ev[1], r.ev_t1));
+    for (int i = 0; i < cnt.timed_calls; ++i) {
+      SS_CK(cudaEventElapsedTime(&t, cnt.ev[2 + 2 * i], cnt.ev[3 + 2 * i]));
+      chunk += t;
+    }
+    ss::ctx_set_stream_times(ctx, (int64_t)(ms * 1e6), (int64_t)(transfer * 1e6), (int64_t)(chunk * 1e6),
+                             (int64_t)(tail * 1e6));
+  }
   fill_stats(stats, cnt, ms,
              std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - wall0).count());
   return SS_OK;
@@ -346,6 +384,8 @@ ss_status stream_layers_impl(ss_ctx* ctx, const ss_layers_desc* ld, ss_stream_st
 
 extern "C" ss_status ss_stream_round(ss_ctx* ctx, const ss_stream_desc* d, ss_stream_stats* stats) {
   if (!ctx) return SS_ERR_ARG;
+  // a round the caller has open stays as it is: the pipeline only ever drops rounds it opened
+  if (ss::ctx_round_open(ctx)) return SS_ERR_STATE;
   ss::ctx_pipeline_mode(ctx, true);
   const ss_status st = stream_round_impl(ctx, d, stats);
   if (st != SS_OK) ss::ctx_pipeline_drain(ctx);
@@ -355,6 +395,7 @@ extern "C" ss_status ss_stream_round(ss_ctx* ctx, const ss_stream_desc* d, ss_st
 
 extern "C" ss_status ss_stream_layers(ss_ctx* ctx, const ss_layers_desc* layers, ss_stream_stats* total) {
   if (!ctx) return SS_ERR_ARG;
+  if (ss::ctx_round_open(ctx)) return SS_ERR_STATE;
   ss::ctx_pipeline_mode(ctx, true);
   const ss_status st = stream_layers_impl(ctx, layers, total);
   if (st != SS_OK) ss::ctx_pipeline_drain(ctx);

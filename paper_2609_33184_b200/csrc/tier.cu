@@ -21,8 +21,11 @@ struct ss_tier {
   void* tail_k[2];
   void* tail_v[2];
   int32_t* len_dev;     // device [B]: tail length C - H (valid_len of the tail chunk, gather offset)
-  int32_t* len_host;    // pinned [4][B]: a ring, so an update never rewrites a slot a copy still reads
+  int32_t* len_host;    // pinned [4][B]: a ring; a slot is rewritten only after the copy that read it
+                        // has finished (one event per slot, waited for before reuse)
   int len_slot;
+  cudaEvent_t ev_len[4];
+  bool len_used[4];
   int32_t H[1024], C[1024], E[1024];
   int cur;              // buffer holding the tail
   bool pending;         // a migration is in flight
@@ -70,7 +73,13 @@ ss_status ss_tier_create(ss_tier** out, const ss_tier_config* cfg, void* const* 
   t->tail_v[1] = tail_v1;
   t->len_dev = len_dev;
   t->len_host = len_host;
-  if (cudaEventCreateWithFlags(&t->ev_copied, cudaEventDisableTiming) != cudaSuccess) {
+  bool ok = cudaEventCreateWithFlags(&t->ev_copied, cudaEventDisableTiming) == cudaSuccess;
+  for (int i = 0; i < 4 && ok; ++i)
+    ok = cudaEventCreateWithFlags(&t->ev_len[i], cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) {
+    if (t->ev_copied) cudaEventDestroy(t->ev_copied);
+    for (int i = 0; i < 4; ++i)
+      if (t->ev_len[i]) cudaEventDestroy(t->ev_len[i]);
     delete t;
     return SS_ERR_CUDA;
   }
@@ -81,6 +90,7 @@ ss_status ss_tier_create(ss_tier** out, const ss_tier_config* cfg, void* const* 
 ss_status ss_tier_destroy(ss_tier* t) {
   if (!t) return SS_ERR_ARG;
   cudaEventDestroy(t->ev_copied);
+  for (int i = 0; i < 4; ++i) cudaEventDestroy(t->ev_len[i]);
   delete t;
   return SS_OK;
 }
@@ -88,11 +98,16 @@ ss_status ss_tier_destroy(ss_tier* t) {
 // Publish the tail lengths C - H to the device through the next slot of the pinned ring.
 static ss_status publish_lengths(ss_tier* t, cudaStream_t s) {
   t->len_slot = (t->len_slot + 1) & 3;
-  int32_t* slot = t->len_host + (size_t)t->len_slot * t->cfg.B;
+  const int i = t->len_slot;
+  // the copy that last read this slot (four publishes ago) must have finished
+  if (t->len_used[i] && cudaEventSynchronize(t->ev_len[i]) != cudaSuccess) return SS_ERR_CUDA;
+  int32_t* slot = t->len_host + (size_t)i * t->cfg.B;
   for (int b = 0; b < t->cfg.B; ++b) slot[b] = t->C[b] - t->H[b];
   if (cudaMemcpyAsync(t->len_dev, slot, sizeof(int32_t) * t->cfg.B, cudaMemcpyHostToDevice, s) !=
       cudaSuccess)
     return SS_ERR_CUDA;
+  if (cudaEventRecord(t->ev_len[i], s) != cudaSuccess) return SS_ERR_CUDA;
+  t->len_used[i] = true;
   return SS_OK;
 }
 
@@ -167,8 +182,14 @@ ss_status ss_tier_migrate(ss_tier* t, void* stream, int32_t* n_requests) {
         uint16_t* dst = (uint16_t*)t->host_hist[b] +
                         ((int64_t)j * 2 * c.H_kv + (int64_t)kv * c.H_kv) * c.L_c * c.d + (int64_t)r * c.d;
         if (cudaMemcpy2DAsync(dst, (size_t)c.L_c * c.d * esz, src, (size_t)cap * c.d * esz,
-                              (size_t)n * c.d * esz, c.H_kv, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+                              (size_t)n * c.d * esz, c.H_kv, cudaMemcpyDeviceToHost, s) != cudaSuccess) {
+          // Copies of this call may already be in flight.  Let them finish and leave every
+          // boundary where it was: the host blocks they wrote lie past H and are written
+          // again by the next migration.
+          cudaStreamSynchronize(s);
+          for (int q = 0; q < c.B; ++q) t->E[q] = t->H[q];
           return SS_ERR_CUDA;
+        }
         t->d2h_bytes += (int64_t)n * c.d * esz * c.H_kv;
       }
       tok += n;

@@ -1,5 +1,6 @@
 """GPU tests of commit-gather (bit exact), the streamed round, the call-order state machine
 and the trace facility, all through the C ABI."""
+import ctypes as C
 import time
 
 import numpy as np
@@ -401,4 +402,33 @@ def test_a_wait_that_nothing_satisfies_gives_up_and_the_context_stays_usable():
     assert ctx.ss_poll_status() == (0, 0)                     # reading cleared the word
     O2, _ = util.gpu_case(ctx, cfg, *case)                    # and the context still works
     assert torch.equal(O1.view(torch.int16), O2.view(torch.int16))
+    ctx.close()
+
+
+def test_stream_round_leaves_an_open_round_alone():
+    """The streamed entry points refuse to run while the caller has a round open, and the open
+    round survives the refusal."""
+    ssb = _ssb()
+    cfg = inputs.VerifyConfig("v", 0x6a, 2, 8, 2, 128, 128, 4, 0, 300)
+    lens = [300, 129]
+    ctx, case, O, LSE, bufs, acc, stats, desc = _stream_case(cfg, lens)
+    Q, chunks, K_loc, V_loc, bits = case
+    O_stream, L_stream = O.clone(), LSE.clone()
+    ctx.ss_verify_begin(Q, cfg.scale)
+    K, V, vl = chunks[0]
+    ctx.ss_verify_chunk(K, V, vl)
+    st = ssb.ss_stream_stats()
+    assert ctx.lib.ss_stream_round(ctx.handle, C.byref(desc), C.byref(st)) == ssb.SS_ERR_STATE
+    arr = (ssb.ss_stream_desc * 1)(desc)
+    ld = ssb.ss_layers_desc(1, arr, ssb.SS_LAYERS_STREAM, None, None, 0)
+    assert ctx.lib.ss_stream_layers(ctx.handle, C.byref(ld), C.byref(st)) == ssb.SS_ERR_STATE
+    # the caller's round is still open and complete-able
+    for K, V, vl in chunks[1:]:
+        ctx.ss_verify_chunk(K, V, vl)
+    ctx.ss_verify_local(K_loc, V_loc)
+    O2, L2 = torch.empty_like(O), torch.empty_like(LSE)
+    ctx.ss_verify_finalize(O2, L2)
+    torch.cuda.synchronize()
+    util.compare(cfg, O2, L2, util.oracle_case(cfg, lens, *case))
+    assert float((O2.float() - O_stream.float()).abs().max()) <= util.TOL_MAX_O
     ctx.close()

@@ -790,3 +790,43 @@ def test_graph_round_helper_replays_with_refreshed_inputs():
     assert ctx.ss_poll_status() == (0, 0)
     util.compare(cfg2, O, LSE, util.oracle_case(cfg2, lens, Q2, chunks2, K_loc2, V_loc2, bits2))
     ctx.close()
+
+
+@pytest.mark.parametrize("T_q,T_loc,G", [(4, 9, 4), (8, 40, 2), (1, 17, 8)])
+def test_chain_with_more_local_tokens_than_queries(T_q, T_loc, G):
+    """The GPU-resident pass over Active Tail + Speculative Frontier (Section 4.2): T_loc - T_q
+    leading local tokens every query sees, then the causal part.  The chain rule is computed in
+    the kernel; the oracle gets the explicit boolean mask j <= i + (T_loc - T_q)."""
+    import oracle
+    from paper_2609_33184_b200 import binding as ssb
+    cfg = inputs.VerifyConfig("tail", 0x90 + T_q, 2, 2 * G, 2, 128, 128, T_q, 0, 200, k_mult=2.0)
+    lens = [200, 37]
+    Q, chunks, _, _, _ = util.gen_case(cfg, lens, DEV)
+    shape = (cfg.B, cfg.H_kv, T_loc, cfg.d)
+    K_loc = inputs.normal_bf16(cfg.seed, inputs.TID_KLOC, shape, mult=2.0, device=DEV)
+    V_loc = inputs.normal_bf16(cfg.seed, inputs.TID_VLOC, shape, device=DEV)
+    ctx = ssb.Context(cfg.B, cfg.H_q, cfg.H_kv, cfg.d, T_q, T_loc, cfg.L_c)
+    O = torch.empty(cfg.B, cfg.H_q, T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
+    LSE = torch.empty(cfg.B, cfg.H_q, T_q, dtype=torch.float32, device=DEV)
+    ctx.ss_verify_begin(Q, cfg.scale)
+    for K, V, vl in chunks:
+        ctx.ss_verify_chunk(K, V, vl)
+    ctx.ss_verify_local(K_loc, V_loc)
+    ctx.ss_verify_finalize(O, LSE)
+    torch.cuda.synchronize()
+    i, j = np.arange(T_q)[:, None], np.arange(T_loc)[None, :]
+    mask = np.broadcast_to(j <= i + (T_loc - T_q), (cfg.B, T_q, T_loc))
+    f64 = util.f64
+    kh = [np.concatenate([f64(K[b, :, :int(vl[b])]) for K, V, vl in chunks], axis=1) for b in range(cfg.B)]
+    vh = [np.concatenate([f64(V[b, :, :int(vl[b])]) for K, V, vl in chunks], axis=1) for b in range(cfg.B)]
+    Or, Lr = oracle.verify_attention(f64(Q), kh, vh, f64(K_loc), f64(V_loc), mask, cfg.scale)
+    ref = {(b, h): (Or[b, h * G:(h + 1) * G], Lr[b, h * G:(h + 1) * G]) for b in range(cfg.B)
+           for h in range(cfg.H_kv)}
+    util.compare(cfg, O, LSE, ref)
+    # fewer local tokens than queries under the chain rule is rejected, not silently run
+    ctx.ss_verify_begin(Q, cfg.scale)
+    if T_q > 1:
+        with pytest.raises(ssb.SpecStreamError):
+            ctx.ss_verify_local(K_loc[:, :, :T_q - 1], V_loc[:, :, :T_q - 1])
+    ctx.ss_verify_abort()
+    ctx.close()
