@@ -244,6 +244,38 @@ class Workload:
         run_round(self.ctx, self.ssb, self.cfg, self.Q, self.chunk_sets[i % self.n_sets], self.K_loc,
                   self.V_loc, self.bits, self.O, self.LSE, ev_pair=ev_pair, hints=self.hints)
 
+    def single_call(self, n_rounds):
+        """The same round through ss_verify_round (one host call per round), and both ways from
+        a C caller (ss_time_rounds: no binding overhead).  Microseconds per round, device time
+        of n_rounds rounds enqueued back to back over the rotating history buffers."""
+        ssb, cfg = self.ssb, self.cfg
+        kind = ssb.SS_MASK_TREE_BITS if cfg.mask == "tree" else ssb.SS_MASK_CHAIN
+        bits = self.bits if cfg.mask == "tree" else None
+        per_set = [self.ctx.chunk_descs([cs], self.hints) for cs in self.chunk_sets]
+        all_sets = self.ctx.chunk_descs(self.chunk_sets, self.hints)
+        n = len(self.chunks)
+
+        def one(i):
+            self.ctx.ss_verify_round(self.Q, cfg.scale, self.chunk_sets[i % self.n_sets], self.K_loc, self.V_loc,
+                                     kind, bits, self.O, self.LSE, descs=per_set[i % self.n_sets])
+        for i in range(10):
+            one(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n_rounds):
+            one(i)
+        e1.record()
+        torch.cuda.synchronize()
+        out = {"python_us_per_round": e0.elapsed_time(e1) / n_rounds * 1e3, "kernel": self.ctx.last_chunk_kernel(),
+               "rounds": n_rounds}
+        for key, single in (("c_caller_us_per_round", 1), ("c_caller_separate_calls_us_per_round", 0)):
+            args = (self.Q, cfg.scale, all_sets, n, self.n_sets, self.K_loc, self.V_loc, kind, bits, self.O, self.LSE)
+            self.ctx.ss_time_rounds(*args, min(n_rounds, 50), single)
+            out[key] = self.ctx.ss_time_rounds(*args, n_rounds, single) / n_rounds * 1e3
+        out["kv_GBps"] = self.nbytes / (out["c_caller_us_per_round"] * 1e-6) / 1e9
+        return out
+
     def l2_note(self):
         if self.n_sets == 1:
             return ("inputs larger than L2 (each round streams all history chunks, "
@@ -555,7 +587,8 @@ def secondary(ssb, name, dev, local_rank, flags, sampler, barrier, overlap):
     out = {"config": w.config(overlap), "steps": steps, "kv_GBps": value, "ms_per_round": ms_per_step,
            "rounds_per_s": 1e3 / ms_per_step, "pct_hbm_nominal_8TBps": 100.0 * value / 8000.0,
            "gpu_launches": int(launches), "clocks": clocks_for(sampler, w, window),
-           "roofline": chunk_roofline(w, min(steps, 50))}
+           "roofline": chunk_roofline(w, min(steps, 50)),
+           "single_call": w.single_call(min(steps, 2000))}
     if cfg.accept:
         out["streamed"] = streamed_leg(w, 3, barrier, local_rank, w.nbytes)
     w.close()
@@ -632,6 +665,7 @@ def main():
     round_stats = round_distribution(w, max(1, min(args.steps, 200)))
     probe = read_probe(w) if len(w.chunks) else None
     graph_info = graph_replay(w, max(10, min(args.steps, 200)))
+    single = w.single_call(max(10, min(args.steps, 500))) if len(w.chunks) else None
 
     # ---- end to end: history in pinned host memory, streamed through ss_stream_round ---------
     e2e = None
@@ -669,7 +703,7 @@ def main():
             "rounds_per_s": world * 1e3 / ms_per_step,
             "pct_hbm_nominal_8TBps": 100.0 * value / world / 8000.0,
             "round_ms": round_stats, "hbm_read_probe": probe,
-            "cuda_graph_replay": graph_info,
+            "cuda_graph_replay": graph_info, "single_call": single,
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
             "roofline": roofline, "cpu_baseline": cpu,
             "sustained": sustained, "workloads": others,

@@ -174,6 +174,38 @@ ss_status ss_verify_chunk_paged(ss_ctx* ctx, ss_tensor K_pool, ss_tensor V_pool,
 ss_status ss_verify_local(ss_ctx* ctx, ss_tensor K_loc, ss_tensor V_loc, int32_t T_loc,
                           ss_mask_kind kind, const uint64_t* mask_bits, void* stream);
 
+/* A whole round with ONE host call (the paper has no counterpart for the call itself; it
+ * computes Eq. 12 like begin + chunk* + local + finalize).  chunks is a HOST array of n_chunks
+ * (>= 0) descriptors, read before the call returns; T_loc = 0 skips the local segment.  Same
+ * tensors, checks and results as the separate calls, which it replaces one for one when the
+ * round is large.  A small round (at most 16 chunks and 32 tiles of 64 tokens in all, T_loc <=
+ * 64) takes a single launch of the CUDA-core kernel that walks the chunks and the local
+ * segment and finalizes in place, so that no partial state goes through HBM and a tiny round
+ * costs one launch instead of n_chunks + 2.  SS_ERR_STATE while a round is open; on any
+ * error nothing of the round is merged and the context is idle again. */
+typedef struct {
+  ss_tensor K, V;                 /* [B, H_kv, L_c, d] bf16, device                          */
+  int32_t L_c;
+  const int32_t* valid_len;       /* device [B], 0..L_c; NULL = all L_c                      */
+  const int32_t* valid_len_host;  /* HOST copy of valid_len or NULL (scheduling hint)        */
+} ss_chunk_desc;
+ss_status ss_verify_round(ss_ctx* ctx, ss_tensor Q, int32_t B, int32_t T_q, float scale,
+                          const ss_chunk_desc* chunks, int32_t n_chunks, ss_tensor K_loc,
+                          ss_tensor V_loc, int32_t T_loc, ss_mask_kind kind, const uint64_t* mask_bits,
+                          void* O, float* LSE, void* stream);
+
+/* Measurement aid (the paper has no counterpart): n_rounds rounds enqueued back to back by a
+ * C caller - this function - and timed with two events on `stream`; *ms_total (HOST) receives
+ * the device time of all of them.  single_call != 0: one ss_verify_round per round; 0: the
+ * separate calls.  chunks holds n_sets consecutive groups of n_chunks descriptors and round i
+ * uses group i % n_sets (rotating history buffers keep a small round from living in L2).
+ * Synchronous.  It shows what a round costs without a binding's per-call overhead. */
+ss_status ss_time_rounds(ss_ctx* ctx, ss_tensor Q, int32_t B, int32_t T_q, float scale,
+                         const ss_chunk_desc* chunks, int32_t n_chunks, int32_t n_sets, ss_tensor K_loc,
+                         ss_tensor V_loc, int32_t T_loc, ss_mask_kind kind, const uint64_t* mask_bits,
+                         void* O, float* LSE, void* stream, int32_t n_rounds, int32_t single_call,
+                         float* ms_total);
+
 /* Checkpoint of a round (between begin and finalize).  export writes, for every query row in
  * [B, H_q, T_q] order, the merged state of everything seen so far: ml[row] = (m, l) with m in
  * the base-2 domain (maximum reference of score*scale*log2(e); -inf and l = 0 for an empty
@@ -478,8 +510,8 @@ typedef struct {
 ss_status ss_get_stats(ss_ctx* ctx, ss_stats* out);
 /* Number of kernels this context has launched since creation. */
 int64_t ss_launch_count(ss_ctx* ctx);
-/* "simt", "tcgen05" (rows on M) or "tcgen05-keys" (keys on M): the chunk kernel the last chunk
- * call used; "none" before the first. */
+/* "simt", "tcgen05" (rows on M), "tcgen05-keys" (keys on M) or "simt-round" (a small round in
+ * one launch): the chunk kernel the last chunk call or ss_verify_round used; "none" before. */
 const char* ss_last_chunk_kernel(ss_ctx* ctx);
 
 #ifdef __cplusplus

@@ -33,7 +33,8 @@ EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "
            "ss_tier_reset", "ss_tier_get", "ss_tier_tail", "ss_tier_commit", "ss_tier_migrate", "ss_tier_poll",
            "ss_tier_d2h_bytes", "ss_verify_chunk_paged", "ss_width_create", "ss_width_destroy",
            "ss_width_observe", "ss_width_next", "ss_width_estimate", "ss_cohort_build", "ss_probe_read",
-           "ss_selftest_wait_expiry", "ss_verify_abort", "ss_cta_log_set", "ss_get_stats"]
+           "ss_selftest_wait_expiry", "ss_verify_abort", "ss_cta_log_set", "ss_get_stats", "ss_verify_round",
+           "ss_time_rounds"]
 
 
 class ss_stats(C.Structure):
@@ -98,6 +99,11 @@ class ss_layers_desc(C.Structure):
 
 
 SS_LAYERS_PREFETCH, SS_LAYERS_STREAM, SS_LAYERS_RESTORE = 0, 1, 2
+
+
+class ss_chunk_desc(C.Structure):
+    _fields_ = [("K", ss_tensor), ("V", ss_tensor), ("L_c", C.c_int32), ("valid_len", C.c_void_p),
+                ("valid_len_host", C.POINTER(C.c_int32))]
 
 
 class ss_static_round(C.Structure):
@@ -204,6 +210,13 @@ def load() -> C.CDLL:
     lib.ss_last_cuda_error.argtypes = [vp]
     lib.ss_trace_enable.restype = C.c_int
     lib.ss_trace_enable.argtypes = [vp, i32]
+    lib.ss_verify_round.restype = C.c_int
+    lib.ss_verify_round.argtypes = [vp, ss_tensor, i32, i32, C.c_float, C.POINTER(ss_chunk_desc), i32, ss_tensor,
+                                    ss_tensor, i32, C.c_int, vp, vp, vp, vp]
+    lib.ss_time_rounds.restype = C.c_int
+    lib.ss_time_rounds.argtypes = [vp, ss_tensor, i32, i32, C.c_float, C.POINTER(ss_chunk_desc), i32, i32,
+                                   ss_tensor, ss_tensor, i32, C.c_int, vp, vp, vp, vp, i32, i32,
+                                   C.POINTER(C.c_float)]
     lib.ss_get_stats.restype = C.c_int
     lib.ss_get_stats.argtypes = [vp, C.POINTER(ss_stats)]
     lib.ss_cta_log_set.restype = C.c_int
@@ -388,6 +401,49 @@ class Context:
 
     def ss_trace_enable(self, on: bool):
         self._check(self.lib.ss_trace_enable(self.handle, 1 if on else 0), "ss_trace_enable")
+
+    @staticmethod
+    def chunk_descs(chunk_sets, hints=None):
+        """ctypes array of ss_chunk_desc for a list of chunk lists [(K, V, valid_len), ...] (all of
+        the same length); hints: per chunk a ctypes int32 array with the host copy of valid_len."""
+        n = len(chunk_sets[0])
+        arr = (ss_chunk_desc * (n * len(chunk_sets)))()
+        for s_, chunks in enumerate(chunk_sets):
+            assert len(chunks) == n
+            for j, (K, V, vl) in enumerate(chunks):
+                d = arr[s_ * n + j]
+                d.K, d.V, d.L_c = as_ss_tensor(K), as_ss_tensor(V), K.shape[2]
+                d.valid_len = _ptr(vl)
+                if hints is not None and vl is not None:
+                    d.valid_len_host = C.cast(hints[j], C.POINTER(C.c_int32))
+        arr._keep = (chunk_sets, hints)
+        return arr
+
+    def ss_verify_round(self, Q, scale, chunks, K_loc, V_loc, mask_kind=SS_MASK_CHAIN, mask_bits=None,
+                        O=None, LSE=None, hints=None, descs=None, stream=None):
+        """One call for a whole round.  chunks: [(K, V, valid_len), ...]; descs: a prebuilt
+        chunk_descs array for the same chunks (saves rebuilding it every round)."""
+        if descs is None:
+            descs = self.chunk_descs([chunks], hints) if chunks else None
+        n = len(chunks)
+        B, _, T_q, _ = Q.shape
+        T_loc = K_loc.shape[2] if K_loc is not None else 0
+        zero = ss_tensor(None, 0, 0, 0)
+        self._check(self.lib.ss_verify_round(
+            self.handle, as_ss_tensor(Q), B, T_q, scale, descs, n,
+            as_ss_tensor(K_loc) if T_loc else zero, as_ss_tensor(V_loc) if T_loc else zero, T_loc, mask_kind,
+            _ptr(mask_bits), O.data_ptr(), _ptr(LSE), self._sp(stream)), "ss_verify_round")
+
+    def ss_time_rounds(self, Q, scale, descs, n_chunks, n_sets, K_loc, V_loc, mask_kind, mask_bits, O, LSE,
+                       n_rounds, single_call, stream=None) -> float:
+        """Device milliseconds of n_rounds rounds enqueued back to back from C."""
+        B, _, T_q, _ = Q.shape
+        ms = C.c_float(0.0)
+        self._check(self.lib.ss_time_rounds(
+            self.handle, as_ss_tensor(Q), B, T_q, scale, descs, n_chunks, n_sets, as_ss_tensor(K_loc),
+            as_ss_tensor(V_loc), K_loc.shape[2], mask_kind, _ptr(mask_bits), O.data_ptr(), _ptr(LSE),
+            self._sp(stream), n_rounds, 1 if single_call else 0, C.byref(ms)), "ss_time_rounds")
+        return ms.value
 
     def ss_get_stats(self) -> ss_stats:
         st = ss_stats()

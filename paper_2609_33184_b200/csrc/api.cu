@@ -55,6 +55,7 @@ struct ss_ctx {
   bool pipe_ready;
   bool no_overlap;          // set while ss_stream_round drives the context
   unsigned long long* trace;  // device trace region (in the workspace)
+  unsigned int* round_counters;  // ticket counters of split small rounds (zero between rounds)
   bool trace_on;
   unsigned long long* cta_log;  // caller's per-CTA log buffer (ss_cta_log_set) or null
   int cta_log_cap;
@@ -128,7 +129,8 @@ Layout layout_for(const ss_config* c) {
   L.set_stride_ml = rows;                 // float2 elements
   L.set_stride_a = rows * c->d;           // float elements
   const int sets = set_cap(c) + 1;
-  L.off_ml = 256 + align_up(ss::kTraceWords * sizeof(unsigned long long), 256);
+  L.off_ml = 256 + align_up(ss::kTraceWords * sizeof(unsigned long long), 256) +
+             ss::kRoundCounters * sizeof(unsigned int);   // status, trace region, round counters
   L.off_a = align_up(L.off_ml + (size_t)sets * rows * sizeof(float2), 256);
   L.total = align_up(L.off_a + (size_t)sets * rows * c->d * sizeof(float), 256);
   return L;
@@ -362,6 +364,7 @@ ss_status ss_create(ss_ctx** out, const ss_config* cfg, void* workspace, size_t 
   c->ws_bytes = workspace_bytes;
   c->status = (uint32_t*)c->ws;
   c->trace = (unsigned long long*)(c->ws + 256);
+  c->round_counters = (unsigned int*)(c->ws + 256 + align_up(ss::kTraceWords * sizeof(unsigned long long), 256));
   c->part_ml = (float2*)(c->ws + L.off_ml);
   c->part_a = (float*)(c->ws + L.off_a);
   c->set_stride_ml = L.set_stride_ml;
@@ -384,6 +387,10 @@ ss_status ss_create(ss_ctx** out, const ss_config* cfg, void* workspace, size_t 
         qr == cudaDriverEntryPointSuccess)
       g_encode = (EncodeTiledFn)fn;
   }
+  if (ss::chunk_simt_prepare() != cudaSuccess) {
+    delete c;
+    return SS_ERR_CUDA;
+  }
   c->tc_ok = (g_encode != nullptr) && !(cfg->flags & SS_FLAG_FORCE_SIMT);
   if (c->tc_ok) c->tc_ok = encode_partials_map(c);
   if (c->tc_ok) {
@@ -395,6 +402,7 @@ ss_status ss_create(ss_ctx** out, const ss_config* cfg, void* workspace, size_t 
     }
   }
   e = cudaMemset(c->status, 0, 256);
+  if (e == cudaSuccess) e = cudaMemset(c->round_counters, 0, ss::kRoundCounters * sizeof(unsigned int));
   if (e != cudaSuccess) {
     delete c;
     return SS_ERR_CUDA;
@@ -524,8 +532,8 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
     p.row_tiles = (R + 127) / 128;
     p.rows_per_tile = R < 128 ? R : 128;
   } else {
-    p.rows_per_tile = 32;
-    p.row_tiles = (R + 31) / 32;
+    p.rows_per_tile = ss::simt_rows_per_tile(R);
+    p.row_tiles = (R + p.rows_per_tile - 1) / p.rows_per_tile;
   }
   const int ctas1 = active_pairs * p.row_tiles;  // CTAs with work when splits = 1
   int splits = pick_splits(c, tc, tc && keys_on_m && R > 32, pairs, ctas1, used_tiles);
@@ -705,6 +713,150 @@ ss_status ss_verify_finalize(ss_ctx* c, void* O, float* LSE, void* stream) {
   c->state = ss_ctx::IDLE;
   c->Q.ptr = nullptr;
   return SS_OK;
+}
+
+ss_status ss_verify_round(ss_ctx* c, ss_tensor Q, int32_t B, int32_t T_q, float scale,
+                          const ss_chunk_desc* chunks, int32_t n_chunks, ss_tensor K_loc, ss_tensor V_loc,
+                          int32_t T_loc, ss_mask_kind kind, const uint64_t* mask_bits, void* O, float* LSE,
+                          void* stream) {
+  if (!c || !O || n_chunks < 0 || (n_chunks > 0 && !chunks) || T_loc < 0) return SS_ERR_ARG;
+  if (c->state != ss_ctx::IDLE) return SS_ERR_STATE;
+  // A round of a few tiles in all takes one launch: chunks, local segment and finalize in one
+  // CUDA-core kernel, no partial state in HBM.  Everything is checked as the separate calls do.
+  int64_t tiles = 0;
+  bool small = n_chunks <= ss::kMaxRoundChunks && T_loc <= 64 && !(c->cfg.flags & (SS_FLAG_ROWS_ON_M | SS_FLAG_KEYS_ON_M));
+  for (int j = 0; small && j < n_chunks; ++j) {
+    if (chunks[j].L_c <= 0) return SS_ERR_ARG;
+    tiles += (chunks[j].L_c + kTileKeys - 1) / kTileKeys;
+  }
+  if (small && tiles <= 32 && B > 0 && T_q > 0) {
+    if (!Q.ptr) return SS_ERR_ARG;
+    if (!(scale > 0.f) || !(scale < 3.0e38f)) return SS_ERR_ARG;
+    if (B > c->cfg.max_B || T_q > c->cfg.max_Tq || T_loc > c->cfg.max_Tloc) return SS_ERR_SHAPE;
+    if (!tensor_ok(Q) || !aligned16(O) || (LSE && ((uintptr_t)LSE & 3))) return SS_ERR_ALIGN;
+    ss::RoundParams p;
+    memset(&p, 0, sizeof(p));
+    for (int j = 0; j < n_chunks; ++j) {
+      const ss_chunk_desc& d = chunks[j];
+      if (!d.K.ptr || !d.V.ptr) return SS_ERR_ARG;
+      if (d.L_c > c->cfg.max_Lc) return SS_ERR_SHAPE;
+      if (!tensor_ok(d.K) || !tensor_ok(d.V) || (d.valid_len && ((uintptr_t)d.valid_len & 3))) return SS_ERR_ALIGN;
+      p.chunk[j] = {(const __nv_bfloat16*)d.K.ptr, (const __nv_bfloat16*)d.V.ptr, d.K.stride_b, d.K.stride_h,
+                    d.K.stride_t, d.V.stride_b, d.V.stride_h, d.V.stride_t, d.valid_len, d.L_c};
+    }
+    if (T_loc > 0) {
+      if (!K_loc.ptr || !V_loc.ptr) return SS_ERR_ARG;
+      if (kind != SS_MASK_CHAIN && kind != SS_MASK_TREE_BITS) return SS_ERR_ARG;
+      if (kind == SS_MASK_TREE_BITS && !mask_bits) return SS_ERR_ARG;
+      if (kind == SS_MASK_CHAIN && T_loc < T_q) return SS_ERR_ARG;
+      if (!tensor_ok(K_loc) || !tensor_ok(V_loc) || (mask_bits && ((uintptr_t)mask_bits & 7))) return SS_ERR_ALIGN;
+    }
+    p.Q = (const __nv_bfloat16*)Q.ptr;
+    p.q_sb = Q.stride_b;
+    p.q_sh = Q.stride_h;
+    p.q_st = Q.stride_t;
+    p.B = B;
+    p.H_q = c->cfg.H_q;
+    p.H_kv = c->cfg.H_kv;
+    p.G = c->G;
+    p.T_q = T_q;
+    p.d = c->cfg.d;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.n_chunks = n_chunks;
+    p.K_loc = (const __nv_bfloat16*)K_loc.ptr;
+    p.V_loc = (const __nv_bfloat16*)V_loc.ptr;
+    p.kl_sb = K_loc.stride_b;
+    p.kl_sh = K_loc.stride_h;
+    p.kl_st = K_loc.stride_t;
+    p.vl_sb = V_loc.stride_b;
+    p.vl_sh = V_loc.stride_h;
+    p.vl_st = V_loc.stride_t;
+    p.T_loc = T_loc;
+    p.mask_bits = (T_loc > 0 && kind == SS_MASK_TREE_BITS) ? mask_bits : nullptr;
+    p.mask_words = (T_loc + 63) / 64;
+    // few CTAs in all: tiles of 8 rows spread a kv-head's rows over more SMs (K/V are re-read
+    // through L2, which a round this small fits into)
+    const int R = T_q * c->G;
+    p.rows_per_tile = ((int64_t)B * c->cfg.H_kv * ((R + 7) / 8) <= 2 * ss::kNumSM) ? 8 : ss::simt_rows_per_tile(R);
+    // token splits: about two CTAs per SM in all, at most 16 and at most one per tile; the
+    // partial states go to the (otherwise idle) partial-set area of the workspace
+    const int64_t units = (int64_t)B * c->cfg.H_kv * ((R + p.rows_per_tile - 1) / p.rows_per_tile);
+    int splits = (int)((2 * ss::kNumSM) / units);
+    if (splits > (T_loc > 0 ? 15 : 16)) splits = T_loc > 0 ? 15 : 16;  // the local segment's CTA makes 16
+    if (splits > tiles) splits = (int)tiles;
+    const int64_t slot_floats = (int64_t)p.rows_per_tile * (c->cfg.d + 2);
+    if (units > ss::kRoundCounters ||
+        units * (splits + 1) * slot_floats * (int64_t)sizeof(float) >
+            (int64_t)(c->ws_bytes - ((uint8_t*)c->part_a - c->ws)))
+      splits = 1;
+    if (splits < 1) splits = 1;
+    p.tiles_per_split = tiles ? (int)((tiles + splits - 1) / splits) : 0;
+    p.splits = tiles ? (int)((tiles + p.tiles_per_split - 1) / p.tiles_per_split) : 1;
+    p.loc_split = p.splits - 1;
+    if (splits > 1 && p.splits > 1 && T_loc > 0 && p.splits < 16) p.loc_split = p.splits++;  // a CTA of its own
+    p.scratch = c->part_a;
+    p.counters = c->round_counters;
+    p.O = (__nv_bfloat16*)O;
+    p.LSE = LSE;
+    p.status = c->status;
+    cudaError_t e = ss::launch_round_simt(p, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->last_kernel = "simt-round";
+    ++c->launches;
+    ++c->stats.rounds;
+    c->stats.rows += (int64_t)B * c->cfg.H_q * T_q;
+    c->stats.chunk_calls += n_chunks;
+    for (int j = 0; j < n_chunks; ++j)
+      c->stats.kv_bytes += (int64_t)B * chunks[j].L_c * c->cfg.H_kv * c->cfg.d * 4;
+    return SS_OK;
+  }
+  // the general case: the separate calls, enqueued from here
+  ss_status st = ss_verify_begin(c, Q, B, T_q, scale, stream);
+  if (st != SS_OK) return st;
+  for (int j = 0; j < n_chunks && st == SS_OK; ++j)
+    st = chunk_impl(c, chunks[j].K, chunks[j].V, chunks[j].L_c, chunks[j].valid_len,
+                    chunks[j].valid_len_host, stream);
+  if (st == SS_OK && T_loc > 0) st = ss_verify_local(c, K_loc, V_loc, T_loc, kind, mask_bits, stream);
+  if (st == SS_OK) st = ss_verify_finalize(c, O, LSE, stream);
+  if (st != SS_OK) ss_verify_abort(c);  // kernels already enqueued finish; nothing is merged
+  return st;
+}
+
+ss_status ss_time_rounds(ss_ctx* c, ss_tensor Q, int32_t B, int32_t T_q, float scale,
+                         const ss_chunk_desc* chunks, int32_t n_chunks, int32_t n_sets, ss_tensor K_loc,
+                         ss_tensor V_loc, int32_t T_loc, ss_mask_kind kind, const uint64_t* mask_bits, void* O,
+                         float* LSE, void* stream, int32_t n_rounds, int32_t single_call, float* ms_total) {
+  if (!c || !ms_total || n_rounds <= 0 || n_sets <= 0 || n_chunks < 0 || (n_chunks > 0 && !chunks))
+    return SS_ERR_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaEvent_t e0, e1;
+  if (cudaEventCreate(&e0) != cudaSuccess) return SS_ERR_CUDA;
+  if (cudaEventCreate(&e1) != cudaSuccess) {
+    cudaEventDestroy(e0);
+    return SS_ERR_CUDA;
+  }
+  ss_status st = SS_OK;
+  cudaError_t e = cudaEventRecord(e0, s);
+  for (int i = 0; i < n_rounds && st == SS_OK && e == cudaSuccess; ++i) {
+    const ss_chunk_desc* set = chunks + (size_t)(i % n_sets) * n_chunks;   // round i's history buffers
+    if (single_call) {
+      st = ss_verify_round(c, Q, B, T_q, scale, set, n_chunks, K_loc, V_loc, T_loc, kind, mask_bits, O, LSE, stream);
+    } else {
+      st = ss_verify_begin(c, Q, B, T_q, scale, stream);
+      for (int j = 0; j < n_chunks && st == SS_OK; ++j)
+        st = chunk_impl(c, set[j].K, set[j].V, set[j].L_c, set[j].valid_len, set[j].valid_len_host, stream);
+      if (st == SS_OK && T_loc > 0) st = ss_verify_local(c, K_loc, V_loc, T_loc, kind, mask_bits, stream);
+      if (st == SS_OK) st = ss_verify_finalize(c, O, LSE, stream);
+      if (st != SS_OK) ss_verify_abort(c);
+    }
+  }
+  if (e == cudaSuccess) e = cudaEventRecord(e1, s);
+  if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+  if (e == cudaSuccess) e = cudaEventElapsedTime(ms_total, e0, e1);
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  if (st != SS_OK) return st;
+  return e == cudaSuccess ? SS_OK : cuda_fail(c, e);
 }
 
 ss_status ss_verify_abort(ss_ctx* c) {

@@ -62,6 +62,40 @@ struct ChunkParams {
   unsigned int launch_seq;
 };
 
+// A whole small round for round_simt_kernel: every history chunk, the local segment, outputs.
+constexpr int kMaxRoundChunks = 16;
+constexpr int kRoundCounters = 1024;  // ticket counters in the workspace (units of a split round)
+struct RoundChunk {
+  const __nv_bfloat16* K;
+  const __nv_bfloat16* V;
+  int64_t k_sb, k_sh, k_st, v_sb, v_sh, v_st;
+  const int32_t* valid_len;  // device [B] or null
+  int L_c;
+};
+struct RoundParams {
+  const __nv_bfloat16* Q;
+  int64_t q_sb, q_sh, q_st;
+  int B, H_q, H_kv, G, T_q, d;
+  float scale_log2;
+  int n_chunks;
+  RoundChunk chunk[kMaxRoundChunks];
+  const __nv_bfloat16* K_loc;  // T_loc == 0: no local segment
+  const __nv_bfloat16* V_loc;
+  int64_t kl_sb, kl_sh, kl_st, vl_sb, vl_sh, vl_st;
+  int T_loc;
+  const uint64_t* mask_bits;   // null for chain
+  int mask_words;
+  int rows_per_tile;           // 8, 16 or 32
+  int splits, tiles_per_split; // CTAs per (b, kvh, row tile): token splits over the history's 64-token
+                               // tiles (all chunks), plus one for the local segment when it has its own
+  int loc_split;               // the split that takes the local segment
+  float* scratch;              // splits > 1: [unit][split][(m, l)[RT], a[RT][d]], unit = (b, kvh, row tile)
+  unsigned int* counters;      // splits > 1: one ticket counter per unit, zero between rounds
+  __nv_bfloat16* O;
+  float* LSE;                  // may be null
+  uint32_t* status;            // may be null
+};
+
 struct LocalParams {
   const __nv_bfloat16* Q;
   int64_t q_sb, q_sh, q_st;
@@ -114,6 +148,9 @@ struct GatherParams {
 
 // launchers (each returns the cudaError_t of the launch)
 cudaError_t launch_chunk_simt(const ChunkParams& p, cudaStream_t s, bool pdl);
+cudaError_t launch_round_simt(const RoundParams& p, cudaStream_t s);
+cudaError_t chunk_simt_prepare();    // one-time function attributes
+int simt_rows_per_tile(int R);       // rows per CTA tile of the CUDA-core chunk kernel
 cudaError_t launch_chunk_tc(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
                             const CUtensorMap& tmA, cudaStream_t s, bool pdl);
 cudaError_t chunk_tc_prepare();  // one-time function attributes

@@ -47,6 +47,7 @@ ss_status scratch_for_current_device(unsigned char** out) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr)
       return SS_ERR_CUDA;
+    if (ss::chunk_simt_prepare() != cudaSuccess) return SS_ERR_CUDA;  // function attributes only
     s.base = static_cast<unsigned char*>(p);
     s.ready = true;
   }
@@ -88,7 +89,8 @@ extern "C" ss_status ss_verify_round_static(const ss_static_round* r, void* stre
   const int G = r->H_q / r->H_kv;
   const int R = r->T_q * G;                                  // <= 4096
   const int64_t pairs = (int64_t)r->B * r->H_kv;
-  const int64_t row_tiles = (R + 31) / 32;
+  const int rows_per_tile = ss::simt_rows_per_tile(R);
+  const int64_t row_tiles = (R + rows_per_tile - 1) / rows_per_tile;
   const int n_tiles = (r->L_c + ss::kTileKeys - 1) / ss::kTileKeys;
   int splits = 1;
   if (n_tiles > 0) {
@@ -144,7 +146,7 @@ extern "C" ss_status ss_verify_round_static(const ss_static_round* r, void* stre
     p.splits = splits;
     p.tiles_per_split = tiles_per_split;
     p.row_tiles = (int)row_tiles;
-    p.rows_per_tile = 32;
+    p.rows_per_tile = rows_per_tile;
     p.scale_log2 = scale_log2;
     p.part_ml = part_ml;
     p.part_a = part_a;

@@ -830,3 +830,70 @@ def test_chain_with_more_local_tokens_than_queries(T_q, T_loc, G):
             ctx.ss_verify_local(K_loc[:, :, :T_q - 1], V_loc[:, :, :T_q - 1])
     ctx.ss_verify_abort()
     ctx.close()
+
+
+@pytest.mark.parametrize("name,cfg,lens", [
+    ("tiny chain", inputs.CONFIGS["c1_tiny_chain"], None),
+    ("ragged, G=4, d=128", inputs.VerifyConfig("r1", 0xa1, 3, 8, 2, 128, 256, 7, 0, 700, k_mult=2.0), [700, 0, 257]),
+    ("tree, one row tile of 8", inputs.VerifyConfig("r2", 0xa2, 2, 2, 2, 64, 128, 8, 0, 300, mask="tree"), [300, 64]),
+    ("tree, G=5", inputs.VerifyConfig("r3", 0xa3, 2, 10, 2, 128, 192, 12, 0, 500, mask="tree"), [1, 500]),
+    ("plain decode", inputs.VerifyConfig("r4", 0xa4, 4, 16, 2, 64, 512, 1, 0, 1500), [1500, 511, 512, 513]),
+])
+def test_whole_round_in_one_call_small(name, cfg, lens):
+    """ss_verify_round on rounds small enough for its single-launch kernel: equal to the oracle
+    and (within rounding) to the separate calls."""
+    from paper_2609_33184_b200 import binding as ssb
+    lens = lens or inputs.history_lengths(cfg)
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    ctx = util.make_ctx(cfg)
+    kind = ssb.SS_MASK_TREE_BITS if cfg.mask == "tree" else ssb.SS_MASK_CHAIN
+    O = torch.full((cfg.B, cfg.H_q, cfg.T_q, cfg.d), float("nan"), dtype=torch.bfloat16, device=DEV)
+    LSE = torch.full((cfg.B, cfg.H_q, cfg.T_q), float("nan"), dtype=torch.float32, device=DEV)
+    ctx.ss_verify_round(Q, cfg.scale, chunks, K_loc, V_loc, kind, bits if cfg.mask == "tree" else None, O, LSE)
+    torch.cuda.synchronize()
+    assert ctx.last_chunk_kernel() == "simt-round"
+    assert ctx.ss_poll_status() == (0, 0)
+    ref = util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits)
+    util.compare(cfg, O, LSE, ref)
+    O2, L2 = util.gpu_case(ctx, cfg, Q, chunks, K_loc, V_loc, bits)
+    mag = max(1.0, float(O2.float().abs().max()))
+    assert float((O.float() - O2.float()).abs().max()) <= util.TOL_MAX_O * mag
+    assert float((LSE - L2).abs().max()) <= util.TOL_LSE
+    # no local segment, no LSE, chunks in reverse order: still Eq. 12 over the history alone
+    O3 = torch.empty_like(O)
+    ctx.ss_verify_round(Q, cfg.scale, chunks[::-1], None, None, kind, None, O3, None)
+    torch.cuda.synchronize()
+    ctx.ss_verify_begin(Q, cfg.scale)
+    for K, V, vl in chunks:
+        ctx.ss_verify_chunk(K, V, vl)
+    O4, L4 = torch.empty_like(O), torch.empty_like(LSE)
+    ctx.ss_verify_finalize(O4, L4)
+    torch.cuda.synchronize()
+    assert float((O3.float() - O4.float()).abs().max()) <= util.TOL_MAX_O * max(1.0, float(O4.float().abs().max()))
+    ctx.close()
+
+
+def test_whole_round_in_one_call_large_and_errors():
+    """A round too large for the single launch goes through the separate kernels (bit-identical
+    to calling them one by one); errors leave the context idle."""
+    from paper_2609_33184_b200 import binding as ssb
+    cfg = inputs.VerifyConfig("big", 0xa5, 2, 8, 2, 128, 1024, 8, 0, 5000)
+    lens = [5000, 1025]
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    ctx = util.make_ctx(cfg, flags=ssb.SS_FLAG_OVERLAP_CHUNKS)
+    O, LSE = util.gpu_case(ctx, cfg, Q, chunks, K_loc, V_loc, bits)
+    O2, L2 = torch.empty_like(O), torch.empty_like(LSE)
+    ctx.ss_verify_round(Q, cfg.scale, chunks, K_loc, V_loc, ssb.SS_MASK_CHAIN, None, O2, L2)
+    torch.cuda.synchronize()
+    assert ctx.last_chunk_kernel().startswith("tcgen05")
+    assert torch.equal(O, O2) and torch.equal(LSE, L2)
+    util.compare(cfg, O2, L2, util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits))
+    # a failing call (chunk longer than the context allows) leaves no round open
+    big = torch.zeros(2, 2, 2048, 128, dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(ssb.SpecStreamError):
+        ctx.ss_verify_round(Q, cfg.scale, chunks + [(big, big, None)], K_loc, V_loc, ssb.SS_MASK_CHAIN, None, O2, L2)
+    ctx.ss_verify_begin(Q, cfg.scale)          # idle again: a new round can start
+    with pytest.raises(ssb.SpecStreamError):   # and ss_verify_round refuses to run over it
+        ctx.ss_verify_round(Q, cfg.scale, chunks, K_loc, V_loc, ssb.SS_MASK_CHAIN, None, O2, L2)
+    ctx.ss_verify_abort()
+    ctx.close()
