@@ -597,7 +597,7 @@ def secondary(ssb, name, dev, local_rank, flags, sampler, barrier, overlap):
     return out
 
 
-def main():
+def arg_parser():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
@@ -614,9 +614,85 @@ def main():
     ap.add_argument("--layers", type=int, default=0,
                     help="also time N streamed layers back to back in the three pipeline modes "
                          "(cross-layer prefetch / layer by layer / restore-then-verify)")
+    ap.add_argument("--shard", default="requests", choices=["requests", "chunks"],
+                    help="how N ranks split the work: by request (every rank its own batch, no data-path "
+                         "collective; weak scaling) or by history chunks of ONE batch (each rank reduces its "
+                         "chunks, one all-gather of the (m, l, a) states, strong scaling)")
     ap.add_argument("--history-tokens", type=int, default=0,
                     help="shrink every request's history to this many tokens (small cases for profiler captures)")
-    args = ap.parse_args()
+    return ap
+
+
+def run_chunk_sharded(args, cfg, ssb, rank, local_rank, world, dev, flags):
+    """--shard chunks: ONE batch whose history chunks are dealt round-robin to the ranks.  Each
+    round: every rank reduces its chunks (rank 0 also the local segment), the merged states are
+    exchanged with one all-gather, imported and finalized; time = max over ranks, value = the
+    batch's KV bytes per second (strong scaling).  Rank 0 checks sampled groups with the oracle."""
+    lens = inputs.history_lengths(cfg)
+    n_chunks = inputs.num_chunks(cfg, lens)
+    plan = ssdist.chunk_shard_plan(cfg, n_chunks, rank, world)
+    Q = inputs.make_q(cfg, dev)
+    K_loc, V_loc = inputs.make_local(cfg, dev)
+    bits = inputs.make_mask_bits(cfg, dev)
+    mine = [inputs.make_history_chunk(cfg, j, lens, dev, fill=0.0) for j in plan.chunks]
+    ctx = ssb.Context(cfg.B, cfg.H_q, cfg.H_kv, cfg.d, cfg.T_q, cfg.T_q, cfg.L_c,
+                      max_chunks=len(mine) + world, device=local_rank, flags=flags)
+    O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=dev)
+    LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=dev)
+    ml, a = ssdist.state_buffers(plan, dev)
+
+    def one_round():
+        ssdist.chunk_sharded_round(ctx, ssb, cfg, Q, mine, K_loc, V_loc, bits, O, LSE, plan, ml, a)
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    for _ in range(args.warmup):
+        one_round()
+    ssdist.barrier(cuda=True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0, t0 = ctx.launch_count(), time.time()
+    e0.record()
+    for _ in range(args.steps):
+        one_round()
+    e1.record()
+    ssdist.barrier(cuda=True)
+    t1 = time.time()
+    ms = ssdist.max_over_ranks(e0.elapsed_time(e1), dev) / args.steps
+    st, dev_bits = ctx.ss_poll_status()
+    if st != 0:
+        raise SystemExit(f"device status word set: {dev_bits}")
+    nbytes = kv_bytes(cfg, lens)
+    check = None
+    if rank == 0 and not args.no_cpu_baseline:
+        # the oracle needs the whole history of the sampled groups: regenerate those chunks here
+        from tests import util
+        full = [inputs.make_history_chunk(cfg, j, lens, dev, fill=0.0) for j in range(n_chunks)]
+        groups = [(0, 0), (cfg.B - 1, cfg.H_kv - 1)]
+        worst = util.compare(cfg, O, LSE, util.oracle_case(cfg, lens, Q, full, K_loc, V_loc, bits, groups=groups))
+        check = {"groups": groups, "max_abs_O": float(worst["max_o"]), "max_abs_LSE": float(worst["lse"])}
+        del full
+    if rank == 0:
+        sampler.stop()
+        value = nbytes / (ms * 1e-3) / 1e9
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg.name, "shard": "chunks", "chunks_per_rank": len(plan.chunks),
+                       "chunk_calls_per_round": n_chunks, "kv_bytes_per_round": nbytes,
+                       "l2": "inputs larger than L2 (distinct chunk buffers)" if nbytes > 2 * L2_BYTES
+                             else "history smaller than twice L2: not an HBM figure"},
+            "collective": {"kind": "all_gather of the merged (m, l) and a[] states, fp32", "per_round": 2,
+                           "bytes_per_rank_per_round": plan.state_bytes},
+            "rounds_per_s": 1e3 / ms, "gpu_launches": int(ctx.launch_count() - launches0),
+            "clocks": sampler.summary(t0, t1), "oracle_check": check,
+        }))
+    ctx.close()
+
+
+def main():
+    args = arg_parser().parse_args()
     args.warmup = max(args.warmup, 3)
     cfg = inputs.CONFIGS[args.workload]
     if args.history_tokens:
@@ -640,12 +716,17 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
-    # per-rank requests: same shapes, rank-specific seed (weak scaling, sharded by request)
-    cfg = ssdist.rank_config(cfg, rank)
     flags = 0 if args.no_overlap else ssb.SS_FLAG_OVERLAP_CHUNKS
     if args.simt:
         flags |= ssb.SS_FLAG_FORCE_SIMT
     flags |= args.flags
+    if args.shard == "chunks":
+        run_chunk_sharded(args, cfg, ssb, rank, local_rank, world, dev, flags)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    # per-rank requests: same shapes, rank-specific seed (weak scaling, sharded by request)
+    cfg = ssdist.rank_config(cfg, rank)
     w = Workload(ssb, cfg, dev, local_rank, flags)
 
     def barrier():

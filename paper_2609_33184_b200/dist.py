@@ -97,3 +97,42 @@ def import_peer_states(ctx, ml: torch.Tensor, a: torch.Tensor, group=None, strea
     for ml_r, a_r in peers:
         ctx.ss_verify_import_state(ml_r, a_r, stream)
     return len(peers)
+
+
+@dataclasses.dataclass
+class ChunkShardPlan:
+    """What one rank does in a round whose history is sharded by chunks."""
+    chunks: list            # chunk indices this rank reduces
+    owns_local: bool        # the local candidate segment is attended to once, by rank 0
+    rows: int               # query rows of the round: B * H_q * T_q
+    d: int
+    state_bytes: int        # bytes of one exported state (ml [rows, 2] + a [rows, d], fp32)
+
+
+def chunk_shard_plan(cfg, n_chunks: int, rank: int, world: int) -> ChunkShardPlan:
+    rows = cfg.B * cfg.H_q * cfg.T_q
+    return ChunkShardPlan(list(chunk_shard(n_chunks, rank, world)), rank == 0, rows, cfg.d,
+                          rows * (cfg.d + 2) * 4)
+
+
+def state_buffers(plan: ChunkShardPlan, device):
+    """Export buffers of a round state in the library's format."""
+    return (torch.empty(plan.rows, 2, dtype=torch.float32, device=device),
+            torch.empty(plan.rows, plan.d, dtype=torch.float32, device=device))
+
+
+def chunk_sharded_round(ctx, ssb, cfg, Q, my_chunks, K_loc, V_loc, bits, O, LSE, plan, ml, a, group=None):
+    """One round with the history sharded by chunks over the ranks (the merge of Eq. 14 is
+    order-free, Eq. 17): this rank's chunks (and, on rank 0, the local segment) -> exported
+    state -> one all-gather of the states (they land in this rank's own memory) -> the peers'
+    states imported as further partials -> finalize.  Every rank ends with the full result.
+    my_chunks: [(K, V, valid_len), ...] for plan.chunks, in that order."""
+    kind = ssb.SS_MASK_TREE_BITS if cfg.mask == "tree" else ssb.SS_MASK_CHAIN
+    ctx.ss_verify_begin(Q, cfg.scale)
+    for K, V, vl in my_chunks:
+        ctx.ss_verify_chunk(K, V, vl)
+    if plan.owns_local:
+        ctx.ss_verify_local(K_loc, V_loc, kind, bits if cfg.mask == "tree" else None)
+    ctx.ss_verify_export_state(ml, a)
+    import_peer_states(ctx, ml, a, group)
+    ctx.ss_verify_finalize(O, LSE)

@@ -119,3 +119,72 @@ def test_two_rank_gloo_chunk_sharded_states():
     for p in procs:
         p.join(timeout=60)
     assert res == {0: "ok", 1: "ok"}, res
+
+
+def _plan_worker(rank, world, port, out):
+    """bench.py --shard chunks as far as a CPU goes: argument plumbing, the per-rank plan, shard
+    coverage, the shapes of the exchanged states, and the round's sequence of calls (recorded by a
+    stand-in context) with the all-gather running over gloo."""
+    import bench
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank),
+                      LOCAL_RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        args = bench.arg_parser().parse_args(["--gpus", str(world), "--shard", "chunks", "--workload", "c4_tree"])
+        assert args.shard == "chunks" and bench.arg_parser().parse_args([]).shard == "requests"
+        cfg = inputs.scaled(inputs.CONFIGS[args.workload], len_lo=5 * 4096, len_hi=5 * 4096)
+        lens = inputs.history_lengths(cfg)
+        n_chunks = inputs.num_chunks(cfg, lens)
+        plan = ssdist.chunk_shard_plan(cfg, n_chunks, rank, world)
+        assert plan.chunks == list(range(rank, n_chunks, world)) and plan.owns_local == (rank == 0)
+        assert plan.rows == cfg.B * cfg.H_q * cfg.T_q and plan.state_bytes == plan.rows * (cfg.d + 2) * 4
+        covered = torch.zeros(n_chunks, dtype=torch.int32)
+        covered[plan.chunks] = 1
+        dist.all_reduce(covered)
+        assert covered.tolist() == [1] * n_chunks
+        ml, a = ssdist.state_buffers(plan, "cpu")
+        assert ml.shape == (plan.rows, 2) and a.shape == (plan.rows, cfg.d)
+
+        class Recorder:   # stands in for the library's context: records the calls of a round
+            def __init__(self):
+                self.calls = []
+
+            def __getattr__(self, name):
+                def call(*args, **kw):
+                    self.calls.append(name)
+                    if name == "ss_verify_export_state":
+                        args[0].fill_(float(rank + 1))
+                        args[1].fill_(float(10 * (rank + 1)))
+                    if name == "ss_verify_import_state":   # a peer's state arrived intact
+                        peer = 1 - rank
+                        assert bool((args[0] == float(peer + 1)).all()) and bool((args[1] == float(10 * (peer + 1))).all())
+                return call
+
+        class Consts:
+            SS_MASK_TREE_BITS, SS_MASK_CHAIN = 1, 0
+
+        rec = Recorder()
+        mine = [(None, None, None)] * len(plan.chunks)
+        ssdist.chunk_sharded_round(rec, Consts, cfg, None, mine, None, None, None, None, None, plan, ml, a)
+        want = (["ss_verify_begin"] + ["ss_verify_chunk"] * len(plan.chunks) +
+                (["ss_verify_local"] if rank == 0 else []) + ["ss_verify_export_state"] +
+                ["ss_verify_import_state"] * (world - 1) + ["ss_verify_finalize"])
+        assert rec.calls == want, rec.calls
+        out.put((rank, "ok"))
+    except Exception as e:  # pragma: no cover
+        out.put((rank, repr(e)))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_rank_gloo_chunk_sharded_bench_path():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_plan_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = dict(out.get(timeout=180) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+    assert res == {0: "ok", 1: "ok"}, res
