@@ -39,7 +39,7 @@ import torch  # noqa: E402
 from paper_2609_33184_b200 import dist as ssdist  # noqa: E402
 from paper_2609_33184_b200 import inputs  # noqa: E402
 from paper_2609_33184_b200.harness import (build_resident, host_valid, kv_bytes, make_stream_desc,  # noqa: E402
-                                            pinned_history, run_round, stream_buffers)
+                                            paged_views, pinned_history, run_round, stream_buffers)
 
 METRIC = "verify_attention_kv_GBps"
 UNIT = "GB/s"
@@ -70,7 +70,7 @@ def tensor_peak():
     return FALLBACK_BF16_TFLOPS, "fallback (sustained)"
 
 
-def ncu_traffic(workload: str, kernel: str):
+def ncu_traffic(workload: str, kernel: str, alg_bytes: float = 0.0):
     """DRAM bytes (read + write) per chunk-kernel launch from the tracked table of ncu captures
     (profiles/ncu_traffic.json: one entry per workload with the kernel it was captured on).
     Returns (bytes or None, note): None with the reason when there is no capture for the
@@ -86,6 +86,8 @@ def ncu_traffic(workload: str, kernel: str):
         return None, "no ncu capture of this workload"
     if e.get("kernel") != kernel:
         return None, f"captured on kernel {e.get('kernel')!r}, this run routed {kernel!r}"
+    if "ratio_to_algorithmic" in e:
+        return float(e["ratio_to_algorithmic"]) * alg_bytes, e.get("note", "")
     return float(e["dram_bytes_per_launch"]), e.get("note", "")
 
 
@@ -221,8 +223,9 @@ def run_reference(args, cfg, rank):
 class Workload:
     """One workload resident on the device: tensors, context, outputs, and the round driver."""
 
-    def __init__(self, ssb, cfg, dev, local_rank, flags):
+    def __init__(self, ssb, cfg, dev, local_rank, flags, page_size=0):
         self.ssb, self.cfg, self.dev = ssb, cfg, dev
+        self.page_size = page_size
         self.lens = inputs.history_lengths(cfg)
         self.Q, self.chunks, self.K_loc, self.V_loc, self.bits = build_resident(cfg, self.lens, dev)
         self.ctx = ssb.Context(cfg.B, cfg.H_q, cfg.H_kv, cfg.d, cfg.T_q, cfg.T_q, cfg.L_c,
@@ -239,10 +242,13 @@ class Workload:
             self.n_sets = min(4096, -(-2 * L2_BYTES // self.nbytes))
         self.chunk_sets = [self.chunks] + [[(K.clone(), V.clone(), vl) for (K, V, vl) in self.chunks]
                                            for _ in range(self.n_sets - 1)]
+        # --page-size: the same buffers read through shuffled page tables (ss_verify_chunk_paged)
+        self.paged_sets = [paged_views(cfg, cs, page_size, dev) for cs in self.chunk_sets] if page_size else None
 
     def round(self, i=0, ev_pair=None):
         run_round(self.ctx, self.ssb, self.cfg, self.Q, self.chunk_sets[i % self.n_sets], self.K_loc,
-                  self.V_loc, self.bits, self.O, self.LSE, ev_pair=ev_pair, hints=self.hints)
+                  self.V_loc, self.bits, self.O, self.LSE, ev_pair=ev_pair, hints=self.hints,
+                  paged=self.paged_sets[i % self.n_sets] if self.paged_sets else None)
 
     def single_call(self, n_rounds):
         """The same round through ss_verify_round (one host call per round), and both ways from
@@ -290,7 +296,8 @@ class Workload:
                 "history_tokens": self.lens if len(set(self.lens)) > 1 else self.lens[0],
                 "chunk_calls_per_round": len(self.chunks), "mask": cfg.mask,
                 "kv_bytes_per_round": self.nbytes, "l2": self.l2_note(),
-                "overlap_chunks": overlap, "host_length_hints": self.hints is not None}
+                "overlap_chunks": overlap, "host_length_hints": self.hints is not None,
+                "page_size": self.page_size or None}
 
     def close(self):
         self.ctx.close()
@@ -356,7 +363,7 @@ def chunk_roofline(w, n_rounds):
     kernel = w.ctx.last_chunk_kernel()
     alg_bytes = w.nbytes / n_calls
     achieved = alg_bytes / (chunk_ms * 1e-3) / 1e9
-    traffic, traffic_note = ncu_traffic(cfg.name, kernel)
+    traffic, traffic_note = ncu_traffic(cfg.name, kernel, alg_bytes)
     roofline = {"bound": "hbm", "kernel": f"chunk attention ({kernel})",
                 "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": traffic, "traffic_note": traffic_note,
@@ -618,8 +625,12 @@ def arg_parser():
                     help="how N ranks split the work: by request (every rank its own batch, no data-path "
                          "collective; weak scaling) or by history chunks of ONE batch (each rank reduces its "
                          "chunks, one all-gather of the (m, l, a) states, strong scaling)")
-    ap.add_argument("--history-tokens", type=int, default=0,
-                    help="shrink every request's history to this many tokens (small cases for profiler captures)")
+    ap.add_argument("--history-tokens", default="",
+                    help="shrink every request's history to this many tokens, or to a seeded ragged range "
+                         "LO:HI (small cases for profiler captures)")
+    ap.add_argument("--page-size", type=int, default=0,
+                    help="read the history through shuffled page tables of this many tokens per page "
+                         "(ss_verify_chunk_paged; throughput only: the outputs are those of permuted tokens)")
     return ap
 
 
@@ -696,7 +707,8 @@ def main():
     args.warmup = max(args.warmup, 3)
     cfg = inputs.CONFIGS[args.workload]
     if args.history_tokens:
-        cfg = inputs.scaled(cfg, len_lo=args.history_tokens, len_hi=args.history_tokens)
+        lo, _, hi = args.history_tokens.partition(":")
+        cfg = inputs.scaled(cfg, len_lo=int(lo), len_hi=int(hi or lo))
 
     rank, local_rank, world = ssdist.env_rank()
     if args.impl == "reference":
@@ -727,7 +739,7 @@ def main():
         return
     # per-rank requests: same shapes, rank-specific seed (weak scaling, sharded by request)
     cfg = ssdist.rank_config(cfg, rank)
-    w = Workload(ssb, cfg, dev, local_rank, flags)
+    w = Workload(ssb, cfg, dev, local_rank, flags, page_size=args.page_size)
 
     def barrier():
         ssdist.barrier(cuda=True)
@@ -746,16 +758,16 @@ def main():
     round_stats = round_distribution(w, max(1, min(args.steps, 200)))
     probe = read_probe(w) if len(w.chunks) else None
     graph_info = graph_replay(w, max(10, min(args.steps, 200)))
-    single = w.single_call(max(10, min(args.steps, 500))) if len(w.chunks) else None
+    single = w.single_call(max(10, min(args.steps, 500))) if len(w.chunks) and not args.page_size else None
 
     # ---- end to end: history in pinned host memory, streamed through ss_stream_round ---------
     e2e = None
-    if not args.no_e2e and len(w.chunks):
+    if not args.no_e2e and len(w.chunks) and not args.page_size:
         e2e = streamed_leg(w, max(3, min(args.steps, 10)), barrier, local_rank, job_bytes,
                            layers=args.layers, rank=rank)
 
     sustained = None
-    if rank == 0 and world == 1 and not args.no_sustained and not args.history_tokens:
+    if rank == 0 and world == 1 and not args.no_sustained and not args.history_tokens and not args.page_size:
         sustained = sustained_leg(w, sampler)
 
     cpu = None
@@ -768,7 +780,7 @@ def main():
 
     # ---- the other workloads (one GPU only: they are reported beside the headline, not scaled)
     others = None
-    if rank == 0 and world == 1 and not args.no_workloads and not args.history_tokens:
+    if rank == 0 and world == 1 and not args.no_workloads and not args.history_tokens and not args.page_size:
         others = {}
         for name in sorted(inputs.CONFIGS):
             if name != cfg.name:

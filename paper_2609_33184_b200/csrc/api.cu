@@ -532,7 +532,9 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
     p.row_tiles = (R + 127) / 128;
     p.rows_per_tile = R < 128 ? R : 128;
   } else {
-    p.rows_per_tile = ss::simt_rows_per_tile(R);
+    // a call of a few CTAs in all is latency bound: tiles of 8 rows spread a kv-head's rows over
+    // more SMs (K/V are re-read through L2, which such a call fits into)
+    p.rows_per_tile = ((int64_t)pairs * ((R + 7) / 8) * n_tiles <= 2 * ss::kNumSM) ? 8 : ss::simt_rows_per_tile(R);
     p.row_tiles = (R + p.rows_per_tile - 1) / p.rows_per_tile;
   }
   const int ctas1 = active_pairs * p.row_tiles;  // CTAs with work when splits = 1

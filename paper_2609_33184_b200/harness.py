@@ -30,13 +30,32 @@ def host_valid(cfg, lens, n_chunks):
             for j in range(n_chunks)]
 
 
-def run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, ev_pair=None, hints=None):
+def paged_views(cfg, chunks, page_size, dev):
+    """Every chunk's own memory re-read as a pool of pages [n_pages, H_kv, page_size, d] with a
+    shuffled page table (for throughput runs of the paged chunk call: the tokens a request sees
+    are a permutation of the batch's, so the outputs are not those of the contiguous chunks)."""
+    assert cfg.L_c % page_size == 0
+    ppr = cfg.L_c // page_size
+    g = torch.Generator().manual_seed(page_size)
+    n_pages = cfg.B * ppr
+    out = []
+    for K, V, vl in chunks:
+        table = torch.randperm(n_pages, generator=g).to(torch.int32).view(cfg.B, ppr).contiguous().to(dev)
+        shape = (n_pages, cfg.H_kv, page_size, cfg.d)
+        out.append((K.reshape(-1).view(shape), V.reshape(-1).view(shape), table))
+    return out
+
+
+def run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, ev_pair=None, hints=None, paged=None):
     kind = ssb.SS_MASK_TREE_BITS if cfg.mask == "tree" else ssb.SS_MASK_CHAIN
     ctx.ss_verify_begin(Q, cfg.scale)
     if ev_pair:
         ev_pair[0].record()
     for j, (K, V, vl) in enumerate(chunks):
-        if hints is not None:
+        if paged is not None:
+            Kp, Vp, table = paged[j]
+            ctx.ss_verify_chunk_paged(Kp, Vp, table, vl, hints[j] if hints is not None else None)
+        elif hints is not None:
             ctx.ss_verify_chunk_hinted(K, V, vl, hints[j])
         else:
             ctx.ss_verify_chunk(K, V, vl)
