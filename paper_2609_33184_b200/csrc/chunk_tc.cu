@@ -8,7 +8,9 @@
 //
 // The kernel is a template over the head dim (64 or 128); the figures below are for 128.  At 64
 // a tile is one [64][64] box per operand, the rings hold six K and six V slots, the score
-// MMA takes four k-steps and the output MMA has N = 64.
+// MMA takes four k-steps, the output MMA has N = 64, and tensor memory has room for a second
+// score buffer (see Tm below), so the score MMAs run two tiles ahead instead of the register
+// double-buffering described next.
 //
 //   warp 4 (one lane)  TMA producer: K tiles and V tiles of 64 tokens, three K slots and four V
 //                      slots, 128-byte swizzle, evict-first L2 policy (the history is
@@ -60,7 +62,16 @@ constexpr int kThreads = 192;
 constexpr int kHalfTile = kTileKeys * 64 * 2;       // 8 KB: [64 keys][64 d] bf16, one TMA box
 constexpr int kSmemCtl = 256;
 constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColS = 0, kColQ = 64, kColO = 128;
+// Tensor-memory columns for head dim D: NS score buffers of 64 columns, Q as bf16 pairs (D / 2
+// columns), O (D columns).  Head dim 128: one score buffer (64 + 64 + 128 = 256 columns, what a
+// CTA can take with two CTAs per SM).  Head dim 64: room for two (128 + 32 + 64 = 224), so the
+// scores of tile t+1 can be computed while tile t is still in its buffer.
+template <int D>
+struct Tm {
+  static constexpr int NS = D == 64 ? 2 : 1;
+  static constexpr uint32_t kColS = 0, kColQ = NS * 64, kColO = NS * 64 + D / 2;
+  static_assert(kColO + D <= 256, "tensor-memory columns");
+};
 constexpr float kRescaleThreshold = 8.f;
 
 // Shared-memory layout for head dim D (64 or 128): the K slots, then the V slots, D / 64 boxes
@@ -85,7 +96,8 @@ template <int KS, int VS>
 struct CtlT {
   uint64_t kfull[KS], kempty[KS], vfull[VS], vempty[VS];
   uint64_t qready;               // the Q rows are in tensor memory
-  uint64_t sfull;                // one phase per tile: S(t) = Q K_t^T has retired
+  uint64_t sfull[2];             // S(t) = Q K_t^T has retired: one score buffer -> sfull[0], one phase per
+                                 // tile; two score buffers -> sfull[t % 2]
   uint64_t pready[2];            // arrival k of the softmax threads (S(k) in registers, P(k-1) stored)
                                  // goes to pready[k % 2]: a thread may make its last arrival before the
                                  // issuer has looked at the one before it, and one barrier's parity
@@ -219,9 +231,9 @@ __device__ __forceinline__ bool softmax_loop(const ChunkParams& p, C* ctl, uint3
                                              int n_tiles, int tok0, int tok1, uint8_t* v_s0, int L,
                                              float& m, float& l, unsigned long long* tr) {
   constexpr int kVStages = Lay<D>::kVStages, kTileBytes = Lay<D>::kTileBytes;
-  const uint32_t t_s = tmem_lane + kColS, t_o = tmem_lane + kColO;
+  const uint32_t t_s = tmem_lane + Tm<D>::kColS, t_o = tmem_lane + Tm<D>::kColO;
   uint32_t raw[NC / 16][16];
-  if (!mbar_wait(&ctl->sfull, 0, ctl, p.status)) return false;
+  if (!mbar_wait(&ctl->sfull[0], 0, ctl, p.status)) return false;
   tc_fence_after();
   load_scores<NC>(t_s, c0, raw);
   tc_fence_before();
@@ -251,7 +263,7 @@ __device__ __forceinline__ bool softmax_loop(const ChunkParams& p, C* ctl, uint3
     if (L == 0) trace(tr, 2, it, 1);
     if (it + 1 < n_tiles) {
       // the next tile's scores move into registers before P takes their place
-      if (!mbar_wait(&ctl->sfull, (it + 1) & 1, ctl, p.status)) return false;
+      if (!mbar_wait(&ctl->sfull[0], (it + 1) & 1, ctl, p.status)) return false;
       tc_fence_after();
       load_scores<NC>(t_s, c0, raw);
       if (L == 0) trace(tr, 2, it, 3);
@@ -264,6 +276,51 @@ __device__ __forceinline__ bool softmax_loop(const ChunkParams& p, C* ctl, uint3
     store_p_at<NC>(t_s, c0, pk);
     tc_fence_before();
     mbar_arrive(&ctl->pready[(it + 1) & 1]);  // arrival it + 1
+    if (L == 0) trace(tr, 2, it, 2);
+  }
+  return true;
+}
+
+// The same loop with two score buffers (head dim 64): tile t lives in buffer t % 2, its P goes
+// over the leading columns of the same buffer, and the issuer runs the score MMAs two tiles
+// ahead, so a thread finds S(t) ready when it gets there and needs no second set of registers.
+template <int NC, int D, typename C>
+__device__ __forceinline__ bool softmax_loop2(const ChunkParams& p, C* ctl, uint32_t tmem_lane, int c0,
+                                              int n_tiles, int tok0, int tok1, uint8_t* v_s0, int L,
+                                              float& m, float& l, unsigned long long* tr) {
+  constexpr int kVStages = Lay<D>::kVStages, kTileBytes = Lay<D>::kTileBytes;
+  const uint32_t t_o = tmem_lane + Tm<D>::kColO;
+  for (int it = 0; it < n_tiles; ++it) {
+    const uint32_t t_s = tmem_lane + Tm<D>::kColS + (it & 1) * 64;
+    if (L == 0) trace(tr, 2, it, 0);
+    if (!mbar_wait(&ctl->sfull[it & 1], (it >> 1) & 1, ctl, p.status)) return false;
+    tc_fence_after();
+    uint32_t raw[NC / 16][16];
+    load_scores<NC>(t_s, c0, raw);
+    if (L == 0) trace(tr, 2, it, 3);
+    const int n_valid = min(kTileKeys, tok1 - (tok0 + it * kTileKeys));
+    if (n_valid < kTileKeys) {
+      // ragged tail: clear the rows of the staged V tile past the valid length (see softmax_loop)
+      const int s = it % kVStages;
+      if (!mbar_wait(&ctl->vfull[s], (it / kVStages) & 1, ctl, p.status)) return false;
+      uint8_t* v_s = v_s0 + s * kTileBytes;
+      constexpr int kVecRow = D / 8;
+      const int n_vec = (kTileKeys - n_valid) * kVecRow;
+      for (int i = L; i < n_vec; i += 128) {
+        const int row = n_valid + i / kVecRow, half = (i % kVecRow) >> 3, ch = i & 7;
+        *reinterpret_cast<uint4*>(v_s + half * kHalfTile + row * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
+      }
+      fence_proxy_async();
+    }
+    uint32_t pk[NC / 16][8];
+    const bool ok = (n_valid < kTileKeys)
+                        ? softmax_compute<NC, true, D>(raw, t_o, c0, n_valid, it, p.scale_log2, m, l, ctl, p.status, pk)
+                        : softmax_compute<NC, false, D>(raw, t_o, c0, n_valid, it, p.scale_log2, m, l, ctl, p.status, pk);
+    if (!ok) return false;
+    if (L == 0) trace(tr, 2, it, 1);
+    store_p_at<NC>(t_s, c0, pk);
+    tc_fence_before();
+    mbar_arrive(&ctl->pready[it & 1]);
     if (L == 0) trace(tr, 2, it, 2);
   }
   return true;
@@ -347,7 +404,8 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         mbar_init(&ctl->vempty[s], 1);
       }
       mbar_init(&ctl->qready, 128);
-      mbar_init(&ctl->sfull, 1);
+      mbar_init(&ctl->sfull[0], 1);
+      mbar_init(&ctl->sfull[1], 1);
       mbar_init(&ctl->pready[0], 128);
       mbar_init(&ctl->pready[1], 128);
       mbar_init(&ctl->odone, 1);
@@ -516,6 +574,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     // lane issues =====
     constexpr uint32_t idesc_qk = make_idesc(128, kTileKeys, false);
     constexpr uint32_t idesc_pv = make_idesc(128, kD, true);
+    constexpr int kNS = Tm<D>::NS;
     const bool leader = elect_one();
     const uint32_t k_base = smem_u32(k_s), v_base = smem_u32(v_s0);
     // The operand descriptors of one slot differ only in their address field (bits 0-13, the
@@ -532,10 +591,11 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
 #pragma unroll
         for (int kk = 0; kk < kD / 16; ++kk) {
           const uint32_t koff = (kk >> 2) * kHalfTile + (kk & 3) * 32;
-          mma_ts(tmem + kColS, tmem + kColQ + kk * 8, k_desc + (koff >> 4), idesc_qk, kk > 0);
+          mma_ts(tmem + Tm<D>::kColS + (kNS == 2 ? (it & 1) * 64 : 0), tmem + Tm<D>::kColQ + kk * 8,
+                 k_desc + (koff >> 4), idesc_qk, kk > 0);
         }
         tc_commit(&ctl->kempty[s]);
-        tc_commit(&ctl->sfull);
+        tc_commit(&ctl->sfull[kNS == 2 ? (it & 1) : 0]);
       }
       __syncwarp();
     };
@@ -546,7 +606,8 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       if (leader) {
 #pragma unroll
         for (int kk = 0; kk < kTileKeys / 16; ++kk) {
-          mma_ts(tmem + kColO, tmem + kColS + kk * 8, v_desc + (kk * 2048 >> 4), idesc_pv,
+          mma_ts(tmem + Tm<D>::kColO, tmem + Tm<D>::kColS + (kNS == 2 ? (it & 1) * 64 : 0) + kk * 8,
+                 v_desc + (kk * 2048 >> 4), idesc_pv,
                  (it > 0 || kk > 0));
         }
         tc_commit(&ctl->vempty[s]);
@@ -560,36 +621,68 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
       const bool ok = mbar_wait(bar, parity, ctl, p.status);
       return __all_sync(0xffffffffu, ok);
     };
-    // Arrival k of the softmax threads (S(k) in their registers, P(k-1) in the buffer) lets
-    // PV(k-1) and then QK(k+1) go: the tensor pipe runs one thread's MMAs in issue order, so
-    // PV(k-1) has consumed P before the new scores overwrite it.
-    bool ok = wwait(&ctl->qready, 0) && wwait(&ctl->kfull[0], 0);
-    if (ok) {
-      trace(trl, 1, 0, 0);
-      tc_fence_after();
-      issue_qk(0);
-      trace(trl, 1, 0, 5);
-    }
-    for (int k = 0; ok && k <= n_tiles; ++k) {
-      ok = wwait(&ctl->pready[k & 1], (k >> 1) & 1);
-      if (!ok) break;
-      if (k >= 1) {
-        const int it = k - 1;
-        ok = wwait(&ctl->vfull[it % kVStages], (it / kVStages) & 1);
-        if (!ok) break;
-        trace(trl, 1, it, 2);
-        tc_fence_after();
-        issue_pv(it);
-        trace(trl, 1, it, 3);
-      }
-      if (k + 1 < n_tiles) {
-        const int it = k + 1;
+    if (kNS == 2) {
+      // Two score buffers: QK(0), QK(1) go out as their K tiles land; arrival t of the softmax
+      // threads (P(t) stored in buffer t % 2) lets PV(t) and then QK(t+2), which overwrites that
+      // buffer, go: the pipe runs one thread's MMAs in issue order.
+      bool ok = wwait(&ctl->qready, 0);
+      for (int it = 0; ok && it < min(2, n_tiles); ++it) {
         ok = wwait(&ctl->kfull[it % kKStages], (it / kKStages) & 1);
         if (!ok) break;
         trace(trl, 1, it, 0);
         tc_fence_after();
         issue_qk(it);
         trace(trl, 1, it, 5);
+      }
+      for (int t = 0; ok && t < n_tiles; ++t) {
+        ok = wwait(&ctl->pready[t & 1], (t >> 1) & 1) && wwait(&ctl->vfull[t % kVStages], (t / kVStages) & 1);
+        if (!ok) break;
+        trace(trl, 1, t, 2);
+        tc_fence_after();
+        issue_pv(t);
+        trace(trl, 1, t, 3);
+        if (t + 2 < n_tiles) {
+          const int it = t + 2;
+          ok = wwait(&ctl->kfull[it % kKStages], (it / kKStages) & 1);
+          if (!ok) break;
+          trace(trl, 1, it, 0);
+          tc_fence_after();
+          issue_qk(it);
+          trace(trl, 1, it, 5);
+        }
+      }
+    } else {
+      // Arrival k of the softmax threads (S(k) in their registers, P(k-1) in the buffer) lets
+      // PV(k-1) and then QK(k+1) go: the tensor pipe runs one thread's MMAs in issue order, so
+      // PV(k-1) has consumed P before the new scores overwrite it.
+      bool ok = wwait(&ctl->qready, 0) && wwait(&ctl->kfull[0], 0);
+      if (ok) {
+        trace(trl, 1, 0, 0);
+        tc_fence_after();
+        issue_qk(0);
+        trace(trl, 1, 0, 5);
+      }
+      for (int k = 0; ok && k <= n_tiles; ++k) {
+        ok = wwait(&ctl->pready[k & 1], (k >> 1) & 1);
+        if (!ok) break;
+        if (k >= 1) {
+          const int it = k - 1;
+          ok = wwait(&ctl->vfull[it % kVStages], (it / kVStages) & 1);
+          if (!ok) break;
+          trace(trl, 1, it, 2);
+          tc_fence_after();
+          issue_pv(it);
+          trace(trl, 1, it, 3);
+        }
+        if (k + 1 < n_tiles) {
+          const int it = k + 1;
+          ok = wwait(&ctl->kfull[it % kKStages], (it / kKStages) & 1);
+          if (!ok) break;
+          trace(trl, 1, it, 0);
+          tc_fence_after();
+          issue_qk(it);
+          trace(trl, 1, it, 5);
+        }
       }
     }
   } else {
@@ -600,7 +693,7 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     const int nc = kTileKeys / groups;
     const int c0 = grp * nc;
     const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
-    const uint32_t t_o = tmem + lane_off + kColO;
+    const uint32_t t_o = tmem + lane_off + Tm<D>::kColO;
     // the Q row -> tensor memory as the A operand of the score MMAs: column j of this lane
     // holds head dims 2j and 2j + 1 (the pair's memory order)
 #pragma unroll
@@ -613,19 +706,23 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         wq[v * 4 + 2] = qreg[q * 4 + v].z;
         wq[v * 4 + 3] = qreg[q * 4 + v].w;
       }
-      tmem_st16(tmem + lane_off + kColQ + q * 16, wq);
+      tmem_st16(tmem + lane_off + Tm<D>::kColQ + q * 16, wq);
     }
     tc_wait_st();
     tc_fence_before();
     mbar_arrive(&ctl->qready);
     float m = -INFINITY, l = 0.f;
     bool ok;
+#define SS_LOOP(NC_)                                                                                        \
+  (Tm<D>::NS == 2 ? softmax_loop2<NC_, D>(p, ctl, tmem + lane_off, c0, n_tiles, tok0, tok1, v_s0, L, m, l, tr) \
+                  : softmax_loop<NC_, D>(p, ctl, tmem + lane_off, c0, n_tiles, tok0, tok1, v_s0, L, m, l, tr))
     if (nc == 16)
-      ok = softmax_loop<16, D>(p, ctl, tmem + lane_off, c0, n_tiles, tok0, tok1, v_s0, L, m, l, tr);
+      ok = SS_LOOP(16);
     else if (nc == 32)
-      ok = softmax_loop<32, D>(p, ctl, tmem + lane_off, c0, n_tiles, tok0, tok1, v_s0, L, m, l, tr);
+      ok = SS_LOOP(32);
     else
-      ok = softmax_loop<64, D>(p, ctl, tmem + lane_off, c0, n_tiles, tok0, tok1, v_s0, L, m, l, tr);
+      ok = SS_LOOP(64);
+#undef SS_LOOP
     // all output MMAs have retired (a barrier of its own: by now odone may be one or two
     // phases past the last one this thread looked at, which a parity cannot tell apart)
     ok = ok && mbar_wait(&ctl->pvdone, 0, ctl, p.status);
