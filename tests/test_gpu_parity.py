@@ -266,14 +266,16 @@ def test_deterministic_bitwise(flags):
     ctx.close()
 
 
-@pytest.mark.parametrize("flags,T_q", [(0, 8), (0, 24), (0, 40), (8, 24)])
-def test_many_rounds_stay_bitwise_identical_and_never_stall(flags, T_q):
+@pytest.mark.parametrize("flags,T_q,B,H_q,k_mult", [
+    (0, 8, 16, 32, 2.0), (0, 24, 16, 32, 2.0), (0, 40, 16, 32, 2.0), (8, 24, 16, 32, 2.0),
+    (0, 64, 4, 40, 1.0)])  # the last: 320 rows per kv-head (row tiles of 128 + 128 + 64), the tree workload's score spread
+def test_many_rounds_stay_bitwise_identical_and_never_stall(flags, T_q, B, H_q, k_mult):
     # Hand-off races between the TMA, MMA and softmax roles show up as a rare wrong tile or as
     # a bounded wait that runs out (status word), typically once in 10^5 CTAs and only when the
     # SMs are full (two CTAs per SM, overlapping launches): repeat rounds of a launch shape
     # that fills the GPU and compare every round with the first, bit for bit.
     ssb = _ssb()
-    cfg = inputs.VerifyConfig("v", 0x5A + T_q, 16, 32, 8, 128, 1024, T_q, 3000, 4096, k_mult=2.0)
+    cfg = inputs.VerifyConfig("v", 0x5A + T_q, B, H_q, 8, 128, 1024, T_q, 3000, 4096, k_mult=k_mult)
     lens = inputs.history_lengths(cfg)
     case = util.gen_case(cfg, lens, DEV)
     ctx = util.make_ctx(cfg, flags=flags | ssb.SS_FLAG_OVERLAP_CHUNKS)
@@ -284,7 +286,7 @@ def test_many_rounds_stay_bitwise_identical_and_never_stall(flags, T_q):
         if i % 50 == 49:
             assert ctx.ss_poll_status() == (0, 0)
             assert torch.equal(O1.view(torch.int16), O2.view(torch.int16)) and torch.equal(L1, L2)
-    ref = util.oracle_case(cfg, lens, *case, groups=[(0, 0), (15, 7)])
+    ref = util.oracle_case(cfg, lens, *case, groups=[(0, 0), (B - 1, 7)])
     util.compare(cfg, O1, L1, ref)
     ctx.close()
 
