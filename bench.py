@@ -223,9 +223,10 @@ def run_reference(args, cfg, rank):
 class Workload:
     """One workload resident on the device: tensors, context, outputs, and the round driver."""
 
-    def __init__(self, ssb, cfg, dev, local_rank, flags, page_size=0):
+    def __init__(self, ssb, cfg, dev, local_rank, flags, page_size=0, chunk_calls="one"):
         self.ssb, self.cfg, self.dev = ssb, cfg, dev
         self.page_size = page_size
+        self.chunk_calls = chunk_calls
         self.lens = inputs.history_lengths(cfg)
         self.Q, self.chunks, self.K_loc, self.V_loc, self.bits = build_resident(cfg, self.lens, dev)
         self.ctx = ssb.Context(cfg.B, cfg.H_q, cfg.H_kv, cfg.d, cfg.T_q, cfg.T_q, cfg.L_c,
@@ -244,11 +245,15 @@ class Workload:
                                            for _ in range(self.n_sets - 1)]
         # --page-size: the same buffers read through shuffled page tables (ss_verify_chunk_paged)
         self.paged_sets = [paged_views(cfg, cs, page_size, dev) for cs in self.chunk_sets] if page_size else None
+        # a round's chunks go in with ONE ss_verify_chunks call (--chunk-calls separate: one call each)
+        self.descs = ([self.ctx.chunk_descs([cs], self.hints) for cs in self.chunk_sets]
+                      if chunk_calls == "one" and not page_size and self.chunks else None)
 
     def round(self, i=0, ev_pair=None):
         run_round(self.ctx, self.ssb, self.cfg, self.Q, self.chunk_sets[i % self.n_sets], self.K_loc,
                   self.V_loc, self.bits, self.O, self.LSE, ev_pair=ev_pair, hints=self.hints,
-                  paged=self.paged_sets[i % self.n_sets] if self.paged_sets else None)
+                  paged=self.paged_sets[i % self.n_sets] if self.paged_sets else None,
+                  descs=self.descs[i % self.n_sets] if self.descs else None)
 
     def single_call(self, n_rounds):
         """The same round through ss_verify_round (one host call per round), and both ways from
@@ -294,7 +299,9 @@ class Workload:
         return {"workload": cfg.name, "B": cfg.B, "H_q": cfg.H_q, "H_kv": cfg.H_kv, "d": cfg.d,
                 "T_q": cfg.T_q, "L_c": cfg.L_c,
                 "history_tokens": self.lens if len(set(self.lens)) > 1 else self.lens[0],
-                "chunk_calls_per_round": len(self.chunks), "mask": cfg.mask,
+                "chunks_per_round": len(self.chunks),
+                "chunk_calls": ("one ss_verify_chunks call per round" if self.descs else "one call per chunk"),
+                "mask": cfg.mask,
                 "kv_bytes_per_round": self.nbytes, "l2": self.l2_note(),
                 "overlap_chunks": overlap, "host_length_hints": self.hints is not None,
                 "page_size": self.page_size or None}
@@ -358,9 +365,11 @@ def chunk_roofline(w, n_rounds):
     for i, p in enumerate(pairs):
         w.round(i, ev_pair=p)
     torch.cuda.synchronize()
+    kernel = w.ctx.last_chunk_kernel()
+    if kernel == "tcgen05-round":   # the whole list of chunks went out as one launch
+        n_calls = 1
     chunk_ms = statistics.mean(a.elapsed_time(b) for a, b in pairs) / n_calls
     peak, peak_kind = peaks()
-    kernel = w.ctx.last_chunk_kernel()
     alg_bytes = w.nbytes / n_calls
     achieved = alg_bytes / (chunk_ms * 1e-3) / 1e9
     traffic, traffic_note = ncu_traffic(cfg.name, kernel, alg_bytes)
@@ -628,6 +637,8 @@ def arg_parser():
     ap.add_argument("--history-tokens", default="",
                     help="shrink every request's history to this many tokens, or to a seeded ragged range "
                          "LO:HI (small cases for profiler captures)")
+    ap.add_argument("--chunk-calls", default="one", choices=["one", "separate"],
+                    help="a round's history chunks in one ss_verify_chunks call (default) or one call per chunk")
     ap.add_argument("--page-size", type=int, default=0,
                     help="read the history through shuffled page tables of this many tokens per page "
                          "(ss_verify_chunk_paged; throughput only: the outputs are those of permuted tokens)")
@@ -739,7 +750,7 @@ def main():
         return
     # per-rank requests: same shapes, rank-specific seed (weak scaling, sharded by request)
     cfg = ssdist.rank_config(cfg, rank)
-    w = Workload(ssb, cfg, dev, local_rank, flags, page_size=args.page_size)
+    w = Workload(ssb, cfg, dev, local_rank, flags, page_size=args.page_size, chunk_calls=args.chunk_calls)
 
     def barrier():
         ssdist.barrier(cuda=True)

@@ -163,6 +163,24 @@ ss_status ss_verify_chunk_paged(ss_ctx* ctx, ss_tensor K_pool, ss_tensor V_pool,
                                 int32_t page_size, const int32_t* page_table, int32_t pages_per_req,
                                 const int32_t* valid_len, const int32_t* valid_len_host, void* stream);
 
+/* a2, several chunks with one call (Section 4.2: the chunks of a request are reduced into one
+ * running state; Eq. 13-14).  chunks is a HOST array of n_chunks (>= 0) descriptors, read before
+ * the call returns; the result is that of one ss_verify_chunk_hinted per descriptor, in order.
+ * Where the rows-on-M tensor-core kernel would take every chunk (more than
+ * 128 query rows per kv-head, 2 to 32 contiguous chunks, one CTA per (request, kv-head, row tile)
+ * fitting the GPU at once) the whole list takes ONE launch: a CTA walks an equal share of its
+ * request's 64-token tiles across the chunk boundaries with one accumulator, so the list leaves
+ * a few partial states per row instead of one per chunk and its CTAs are equally long
+ * ("tcgen05-round" in ss_last_chunk_kernel).  Otherwise the chunks are enqueued one by one.
+ * SS_ERR_STATE outside an open round; an error leaves the round open (ss_verify_abort ends it). */
+typedef struct {
+  ss_tensor K, V;                 /* [B, H_kv, L_c, d] bf16, device                          */
+  int32_t L_c;
+  const int32_t* valid_len;       /* device [B], 0..L_c; NULL = all L_c                      */
+  const int32_t* valid_len_host;  /* HOST copy of valid_len or NULL (scheduling hint)        */
+} ss_chunk_desc;
+ss_status ss_verify_chunks(ss_ctx* ctx, const ss_chunk_desc* chunks, int32_t n_chunks, void* stream);
+
 /* a4. The on-GPU candidate segment (Section 4.2: the pass over the GPU-resident Active Tail and
  * Speculative Frontier; the mask M of Eq. 12): K_loc, V_loc [B, H_kv, T_loc, d].  Query i of
  * request b sees local token j iff
@@ -177,18 +195,12 @@ ss_status ss_verify_local(ss_ctx* ctx, ss_tensor K_loc, ss_tensor V_loc, int32_t
 /* A whole round with ONE host call (the paper has no counterpart for the call itself; it
  * computes Eq. 12 like begin + chunk* + local + finalize).  chunks is a HOST array of n_chunks
  * (>= 0) descriptors, read before the call returns; T_loc = 0 skips the local segment.  Same
- * tensors, checks and results as the separate calls, which it replaces one for one when the
- * round is large.  A small round (at most 16 chunks and 32 tiles of 64 tokens in all, T_loc <=
+ * tensors, checks and results as the separate calls: a large round is begin + ss_verify_chunks
+ * + local + finalize.  A small round (at most 16 chunks and 32 tiles of 64 tokens in all, T_loc <=
  * 64) takes a single launch of the CUDA-core kernel that walks the chunks and the local
  * segment and finalizes in place, so that no partial state goes through HBM and a tiny round
  * costs one launch instead of n_chunks + 2.  SS_ERR_STATE while a round is open; on any
  * error nothing of the round is merged and the context is idle again. */
-typedef struct {
-  ss_tensor K, V;                 /* [B, H_kv, L_c, d] bf16, device                          */
-  int32_t L_c;
-  const int32_t* valid_len;       /* device [B], 0..L_c; NULL = all L_c                      */
-  const int32_t* valid_len_host;  /* HOST copy of valid_len or NULL (scheduling hint)        */
-} ss_chunk_desc;
 ss_status ss_verify_round(ss_ctx* ctx, ss_tensor Q, int32_t B, int32_t T_q, float scale,
                           const ss_chunk_desc* chunks, int32_t n_chunks, ss_tensor K_loc,
                           ss_tensor V_loc, int32_t T_loc, ss_mask_kind kind, const uint64_t* mask_bits,
@@ -510,8 +522,9 @@ typedef struct {
 ss_status ss_get_stats(ss_ctx* ctx, ss_stats* out);
 /* Number of kernels this context has launched since creation. */
 int64_t ss_launch_count(ss_ctx* ctx);
-/* "simt", "tcgen05" (rows on M), "tcgen05-keys" (keys on M) or "simt-round" (a small round in
- * one launch): the chunk kernel the last chunk call or ss_verify_round used; "none" before. */
+/* "simt", "tcgen05" (rows on M), "tcgen05-keys" (keys on M), "tcgen05-round" (rows on M, a list
+ * of chunks in one launch) or "simt-round" (a small round in one launch): the chunk kernel the
+ * last chunk call, ss_verify_chunks or ss_verify_round used; "none" before. */
 const char* ss_last_chunk_kernel(ss_ctx* ctx);
 
 #ifdef __cplusplus

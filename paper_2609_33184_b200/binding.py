@@ -33,7 +33,7 @@ EXPORTS = ["ss_workspace_bytes", "ss_create", "ss_destroy", "ss_verify_begin", "
            "ss_tier_reset", "ss_tier_get", "ss_tier_tail", "ss_tier_commit", "ss_tier_migrate", "ss_tier_poll",
            "ss_tier_d2h_bytes", "ss_verify_chunk_paged", "ss_width_create", "ss_width_destroy",
            "ss_width_observe", "ss_width_next", "ss_width_estimate", "ss_cohort_build", "ss_probe_read",
-           "ss_selftest_wait_expiry", "ss_verify_abort", "ss_cta_log_set", "ss_get_stats", "ss_verify_round",
+           "ss_selftest_wait_expiry", "ss_verify_abort", "ss_cta_log_set", "ss_get_stats", "ss_verify_round", "ss_verify_chunks",
            "ss_time_rounds"]
 
 
@@ -210,6 +210,8 @@ def load() -> C.CDLL:
     lib.ss_last_cuda_error.argtypes = [vp]
     lib.ss_trace_enable.restype = C.c_int
     lib.ss_trace_enable.argtypes = [vp, i32]
+    lib.ss_verify_chunks.restype = C.c_int
+    lib.ss_verify_chunks.argtypes = [vp, C.POINTER(ss_chunk_desc), i32, vp]
     lib.ss_verify_round.restype = C.c_int
     lib.ss_verify_round.argtypes = [vp, ss_tensor, i32, i32, C.c_float, C.POINTER(ss_chunk_desc), i32, ss_tensor,
                                     ss_tensor, i32, C.c_int, vp, vp, vp, vp]
@@ -418,6 +420,10 @@ class Context:
                     d.valid_len_host = C.cast(hints[j], C.POINTER(C.c_int32))
         arr._keep = (chunk_sets, hints)
         return arr
+
+    def ss_verify_chunks(self, descs, n_chunks: int, stream=None):
+        """Several chunks of the open round with one call; descs: a chunk_descs array."""
+        self._check(self.lib.ss_verify_chunks(self.handle, descs, n_chunks, self._sp(stream)), "ss_verify_chunks")
 
     def ss_verify_round(self, Q, scale, chunks, K_loc, V_loc, mask_kind=SS_MASK_CHAIN, mask_bits=None,
                         O=None, LSE=None, hints=None, descs=None, stream=None):

@@ -60,6 +60,11 @@ struct ss_ctx {
   unsigned long long* cta_log;  // caller's per-CTA log buffer (ss_cta_log_set) or null
   int cta_log_cap;
   ss_stats stats;           // counters (launches is filled in when they are read)
+  // tensor maps of a whole-history launch: kHistSlots lists in the workspace, their host mirrors
+  CUtensorMap* hist_maps;   // device [kHistSlots][2 * kMaxHistChunks]
+  CUtensorMap hist_host[4][2 * ss::kMaxHistChunks];
+  int hist_n[4];            // maps in use per slot (0 = empty)
+  uint64_t hist_age[4];
   cudaEvent_t* ev_pool;     // timing events of the streamed round (SS_FLAG_STREAM_TIMING)
   int ev_pool_n;
 };
@@ -115,8 +120,9 @@ int slots_for(const ss_config* c) {
   return pairs * s;
 }
 
+constexpr int kHistSlots = 4;
 struct Layout {
-  size_t off_ml, off_a, total;
+  size_t off_hist, off_ml, off_a, total;
   int64_t set_stride_ml, set_stride_a;
   int R_stride;
 };
@@ -129,8 +135,9 @@ Layout layout_for(const ss_config* c) {
   L.set_stride_ml = rows;                 // float2 elements
   L.set_stride_a = rows * c->d;           // float elements
   const int sets = set_cap(c) + 1;
-  L.off_ml = 256 + align_up(ss::kTraceWords * sizeof(unsigned long long), 256) +
-             ss::kRoundCounters * sizeof(unsigned int);   // status, trace region, round counters
+  L.off_hist = 256 + align_up(ss::kTraceWords * sizeof(unsigned long long), 256) +
+               ss::kRoundCounters * sizeof(unsigned int);   // status, trace region, round counters
+  L.off_ml = L.off_hist + kHistSlots * 2 * ss::kMaxHistChunks * sizeof(CUtensorMap);  // lists of tensor maps
   L.off_a = align_up(L.off_ml + (size_t)sets * rows * sizeof(float2), 256);
   L.total = align_up(L.off_a + (size_t)sets * rows * c->d * sizeof(float), 256);
   return L;
@@ -365,6 +372,7 @@ ss_status ss_create(ss_ctx** out, const ss_config* cfg, void* workspace, size_t 
   c->status = (uint32_t*)c->ws;
   c->trace = (unsigned long long*)(c->ws + 256);
   c->round_counters = (unsigned int*)(c->ws + 256 + align_up(ss::kTraceWords * sizeof(unsigned long long), 256));
+  c->hist_maps = (CUtensorMap*)(c->ws + L.off_hist);
   c->part_ml = (float2*)(c->ws + L.off_ml);
   c->part_a = (float*)(c->ws + L.off_a);
   c->set_stride_ml = L.set_stride_ml;
@@ -717,6 +725,137 @@ ss_status ss_verify_finalize(ss_ctx* c, void* O, float* LSE, void* stream) {
   return SS_OK;
 }
 
+// The whole history of a round in ONE launch of the rows-on-M kernel (Section 4.2: the chunks of a
+// request are reduced into one running state; Eq. 13-14).  Taken when that kernel would run every
+// chunk anyway and one CTA per (request, kv-head, row tile, split) fills the GPU at most once:
+// the CTAs are equally long, keep their accumulator across chunk boundaries and leave `splits`
+// partial states per row instead of one per chunk.  Returns SS_OK with *taken = false when the
+// round does not qualify (nothing has been enqueued then).
+static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunks, bool* taken) {
+  *taken = false;
+  if (!c->tc_ok || n_chunks < 2 || n_chunks > ss::kMaxHistChunks || c->force_keys_kernel) return SS_OK;
+  if (getenv("SS_NO_HISTORY_LAUNCH")) return SS_OK;
+  const int R = c->T_q * c->G, pairs = c->B * c->cfg.H_kv;
+  const int keys_max_rows = c->cfg.d == 64 ? 16 : 32;
+  if (R <= keys_max_rows && !c->force_rows_kernel) return SS_OK;   // the keys-on-M kernel's rounds
+  // With up to 128 rows per kv-head the chunk kernels run at the HBM ceiling while the GPU is full
+  // and successive launches keep it full; the one launch pays off where the tile's arithmetic
+  // bounds the kernel (measured: +5 % at 192 rows, +11-13 % on the 320-row tree workload, -4 % at 48).
+  const int row_tiles = (R + 127) / 128;
+  if (row_tiles < 2 && !getenv("SS_HISTORY_LAUNCH_ALWAYS")) return SS_OK;
+  const int64_t units = (int64_t)pairs * row_tiles;
+  const int wave = 2 * ss::kNumSM;                                  // two CTAs per SM
+  if (units > wave) return SS_OK;
+  int64_t tiles = 0;
+  for (int j = 0; j < n_chunks; ++j) {
+    const ss_chunk_desc& d = chunks[j];
+    if (!d.K.ptr || !d.V.ptr || d.L_c <= 0) return SS_ERR_ARG;
+    if (d.L_c > c->cfg.max_Lc) return SS_ERR_SHAPE;
+    if (!tensor_ok(d.K) || !tensor_ok(d.V) || (d.valid_len && ((uintptr_t)d.valid_len & 3))) return SS_ERR_ALIGN;
+    tiles += (d.L_c + kTileKeys - 1) / kTileKeys;
+  }
+  if (tiles > 0x3fffffff) return SS_OK;
+  int splits = (int)(wave / units);
+  if (splits > kMaxSplits) splits = kMaxSplits;
+  if (splits > c->slots_per_set / pairs) splits = c->slots_per_set / pairs;
+  if (splits > tiles / 8) splits = (int)(tiles / 8);               // at least eight tiles per CTA
+  if (c->force_splits > 0 && c->force_splits < splits) splits = c->force_splits;
+  if (splits < 1) splits = 1;
+
+  // the chunks' tensor maps, K and V alternating, in one of the workspace's lists
+  CUtensorMap maps[2 * ss::kMaxHistChunks];
+  for (int j = 0; j < n_chunks; ++j)
+    if (!get_tensor_map(c, chunks[j].K, c->B, chunks[j].L_c, kTileKeys, &maps[2 * j]) ||
+        !get_tensor_map(c, chunks[j].V, c->B, chunks[j].L_c, kTileKeys, &maps[2 * j + 1]))
+      return SS_OK;
+  int slot = -1;
+  for (int i = 0; i < kHistSlots && slot < 0; ++i)
+    if (c->hist_n[i] == 2 * n_chunks && memcmp(c->hist_host[i], maps, (size_t)2 * n_chunks * sizeof(CUtensorMap)) == 0)
+      slot = i;
+  cudaStream_t s = c->stream;
+  if (slot < 0) {
+    slot = 0;
+    for (int i = 1; i < kHistSlots; ++i)
+      if (c->hist_age[i] < c->hist_age[slot]) slot = i;
+    memcpy(c->hist_host[slot], maps, (size_t)2 * n_chunks * sizeof(CUtensorMap));
+    c->hist_n[slot] = 0;  // (not valid until the copy has been enqueued)
+    // stream order: the copy runs after every kernel already enqueued, which may still read the list
+    cudaError_t e = cudaMemcpyAsync(c->hist_maps + (size_t)slot * 2 * ss::kMaxHistChunks, c->hist_host[slot],
+                                    (size_t)2 * n_chunks * sizeof(CUtensorMap), cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->hist_n[slot] = 2 * n_chunks;
+  }
+  c->hist_age[slot] = ++c->tm_clock;
+
+  ss::ChunkParams p;
+  memset(&p, 0, sizeof(p));
+  ss::HistParams h;
+  memset(&h, 0, sizeof(h));
+  h.n_chunks = n_chunks;
+  h.maps = c->hist_maps + (size_t)slot * 2 * ss::kMaxHistChunks;
+  int64_t tokens = 0;
+  for (int j = 0; j < n_chunks; ++j) {
+    h.valid_len[j] = chunks[j].valid_len;
+    h.L_c[j] = chunks[j].L_c;
+    if (chunks[j].valid_len && chunks[j].valid_len_host) {
+      for (int b = 0; b < c->B; ++b) {
+        const int v = chunks[j].valid_len_host[b];
+        tokens += v < 0 ? 0 : (v > chunks[j].L_c ? chunks[j].L_c : v);
+      }
+    } else {
+      tokens += (int64_t)c->B * chunks[j].L_c;
+    }
+  }
+  p.row_tiles = row_tiles;
+  p.rows_per_tile = R < 128 ? R : 128;
+  p.splits = splits;
+  p.tiles_per_split = 0;
+  p.Q = (const __nv_bfloat16*)c->Q.ptr;
+  p.q_sb = c->Q.stride_b;
+  p.q_sh = c->Q.stride_h;
+  p.q_st = c->Q.stride_t;
+  p.B = c->B;
+  p.H_kv = c->cfg.H_kv;
+  p.G = c->G;
+  p.T_q = c->T_q;
+  p.R = R;
+  p.d = c->cfg.d;
+  p.L_c = 0;
+  p.scale_log2 = c->scale * 1.4426950408889634f;
+  p.part_ml = c->part_ml + (int64_t)c->n_sets * c->set_stride_ml;
+  p.part_a = c->part_a + (int64_t)c->n_sets * c->set_stride_a;
+  p.R_stride = c->R_stride;
+  p.a_slot0 = c->n_sets * c->slots_per_set;
+  p.status = c->status;
+  p.trace = c->trace_on ? c->trace : nullptr;
+  p.cta_log = c->cta_log;
+  p.cta_log_cap = c->cta_log_cap;
+  p.launch_seq = (unsigned int)c->launches;
+  cudaError_t e = ss::launch_chunk_tc_hist(p, h, c->tm_a, s, use_pdl(c));
+  if (e != cudaSuccess) return cuda_fail(c, e);
+  c->last_kernel = "tcgen05-round";
+  ++c->launches;
+  c->stats.chunk_calls += n_chunks;
+  c->stats.kv_bytes += tokens * c->cfg.H_kv * c->cfg.d * 4;
+  c->splits[c->n_sets] = (uint8_t)splits;
+  memset(c->absent[c->n_sets], 0, sizeof(c->absent[0]));
+  ++c->n_sets;
+  c->first_launch = false;
+  *taken = true;
+  return SS_OK;
+}
+
+ss_status ss_verify_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int32_t n_chunks, void* stream) {
+  if (!c || n_chunks < 0 || (n_chunks > 0 && !chunks)) return SS_ERR_ARG;
+  if (c->state != ss_ctx::OPEN || (cudaStream_t)stream != c->stream) return SS_ERR_STATE;
+  bool one_launch = false;
+  ss_status st = hist_chunks(c, chunks, n_chunks, &one_launch);
+  for (int j = 0; !one_launch && j < n_chunks && st == SS_OK; ++j)
+    st = chunk_impl(c, chunks[j].K, chunks[j].V, chunks[j].L_c, chunks[j].valid_len,
+                    chunks[j].valid_len_host, stream);
+  return st;
+}
+
 ss_status ss_verify_round(ss_ctx* c, ss_tensor Q, int32_t B, int32_t T_q, float scale,
                           const ss_chunk_desc* chunks, int32_t n_chunks, ss_tensor K_loc, ss_tensor V_loc,
                           int32_t T_loc, ss_mask_kind kind, const uint64_t* mask_bits, void* O, float* LSE,
@@ -815,9 +954,7 @@ ss_status ss_verify_round(ss_ctx* c, ss_tensor Q, int32_t B, int32_t T_q, float 
   // the general case: the separate calls, enqueued from here
   ss_status st = ss_verify_begin(c, Q, B, T_q, scale, stream);
   if (st != SS_OK) return st;
-  for (int j = 0; j < n_chunks && st == SS_OK; ++j)
-    st = chunk_impl(c, chunks[j].K, chunks[j].V, chunks[j].L_c, chunks[j].valid_len,
-                    chunks[j].valid_len_host, stream);
+  st = ss_verify_chunks(c, chunks, n_chunks, stream);
   if (st == SS_OK && T_loc > 0) st = ss_verify_local(c, K_loc, V_loc, T_loc, kind, mask_bits, stream);
   if (st == SS_OK) st = ss_verify_finalize(c, O, LSE, stream);
   if (st != SS_OK) ss_verify_abort(c);  // kernels already enqueued finish; nothing is merged

@@ -60,7 +60,7 @@ namespace {
 
 constexpr int kThreads = 192;
 constexpr int kHalfTile = kTileKeys * 64 * 2;       // 8 KB: [64 keys][64 d] bf16, one TMA box
-constexpr int kSmemCtl = 256;
+constexpr int kSmemCtl = 512;   // barriers (<= 256 bytes), then the chunk table of a launch over a list of chunks
 constexpr uint32_t kTmemCols = 256;
 // Tensor-memory columns for head dim D: NS score buffers of 64 columns, Q as bf16 pairs (D / 2
 // columns), O (D columns).  Head dim 128: one score buffer (64 + 64 + 128 = 256 columns, what a
@@ -223,12 +223,40 @@ __device__ __forceinline__ void store_p_at(uint32_t t_s, int c0, const uint32_t 
   tc_wait_st();
 }
 
+// Which tokens the CTA's tile `it` holds.  One chunk: tokens [tok0, tok1) in tiles of 64.  A list
+// of chunks: the CTA's tiles are numbers [g0, g0 + n_tiles) of the request's tiles counted chunk
+// by chunk; prefix[j] = tiles before chunk j, valid[j] = the request's tokens in chunk j (a table
+// in shared memory); a role walks the tiles in order and keeps the chunk it is in.
+template <bool HIST>
+struct TileMap {
+  int tok0, tok1;
+  __device__ __forceinline__ int n_valid(int it) { return min(kTileKeys, tok1 - (tok0 + it * kTileKeys)); }
+};
+template <>
+struct TileMap<true> {
+  const int* prefix;
+  const int* valid;
+  int g0, j;
+  // chunk of tile `it` (tiles are asked for in ascending order) and the tile's first token in it
+  __device__ __forceinline__ int locate(int it, int* tok) {
+    const int g = g0 + it;
+    while (g >= prefix[j + 1]) ++j;
+    *tok = (g - prefix[j]) * kTileKeys;
+    return j;
+  }
+  __device__ __forceinline__ int n_valid(int it) {
+    int tok;
+    const int c = locate(it, &tok);
+    return min(kTileKeys, valid[c] - tok);
+  }
+};
+
 // The tile loop of one softmax thread (TMEM lane L, key columns [c0, c0 + NC) of every tile).
 // Arrival k on `pready` says: S(k) is in this thread's registers and P(k-1) is in the buffer.
 // Returns false when a bounded wait gave up.
-template <int NC, int D, typename C>
+template <int NC, int D, typename C, typename TM>
 __device__ __forceinline__ bool softmax_loop(const ChunkParams& p, C* ctl, uint32_t tmem_lane, int c0,
-                                             int n_tiles, int tok0, int tok1, uint8_t* v_s0, int L,
+                                             int n_tiles, TM tm, uint8_t* v_s0, int L,
                                              float& m, float& l, unsigned long long* tr) {
   constexpr int kVStages = Lay<D>::kVStages, kTileBytes = Lay<D>::kTileBytes;
   const uint32_t t_s = tmem_lane + Tm<D>::kColS, t_o = tmem_lane + Tm<D>::kColO;
@@ -240,7 +268,7 @@ __device__ __forceinline__ bool softmax_loop(const ChunkParams& p, C* ctl, uint3
   mbar_arrive(&ctl->pready[0]);  // arrival 0: the issuer may overwrite the buffer with S(1)
   for (int it = 0; it < n_tiles; ++it) {
     if (L == 0) trace(tr, 2, it, 0);
-    const int n_valid = min(kTileKeys, tok1 - (tok0 + it * kTileKeys));
+    const int n_valid = tm.n_valid(it);
     if (n_valid < kTileKeys) {
       // ragged tail: rows past the valid length may hold anything; P is 0 there, so V must
       // be finite: clear those rows of the staged V tile (whole 128-byte rows, both halves)
@@ -284,9 +312,9 @@ __device__ __forceinline__ bool softmax_loop(const ChunkParams& p, C* ctl, uint3
 // The same loop with two score buffers (head dim 64): tile t lives in buffer t % 2, its P goes
 // over the leading columns of the same buffer, and the issuer runs the score MMAs two tiles
 // ahead, so a thread finds S(t) ready when it gets there and needs no second set of registers.
-template <int NC, int D, typename C>
+template <int NC, int D, typename C, typename TM>
 __device__ __forceinline__ bool softmax_loop2(const ChunkParams& p, C* ctl, uint32_t tmem_lane, int c0,
-                                              int n_tiles, int tok0, int tok1, uint8_t* v_s0, int L,
+                                              int n_tiles, TM tm, uint8_t* v_s0, int L,
                                               float& m, float& l, unsigned long long* tr) {
   constexpr int kVStages = Lay<D>::kVStages, kTileBytes = Lay<D>::kTileBytes;
   const uint32_t t_o = tmem_lane + Tm<D>::kColO;
@@ -298,7 +326,7 @@ __device__ __forceinline__ bool softmax_loop2(const ChunkParams& p, C* ctl, uint
     uint32_t raw[NC / 16][16];
     load_scores<NC>(t_s, c0, raw);
     if (L == 0) trace(tr, 2, it, 3);
-    const int n_valid = min(kTileKeys, tok1 - (tok0 + it * kTileKeys));
+    const int n_valid = tm.n_valid(it);
     if (n_valid < kTileKeys) {
       // ragged tail: clear the rows of the staged V tile past the valid length (see softmax_loop)
       const int s = it % kVStages;
@@ -326,10 +354,11 @@ __device__ __forceinline__ bool softmax_loop2(const ChunkParams& p, C* ctl, uint
   return true;
 }
 
-template <int D>
+template <int D, bool HIST>
 __global__ void __launch_bounds__(kThreads, 2)
 chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
-                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmA) {
+                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmA,
+                const __grid_constant__ HistParams h) {
   using L_ = Lay<D>;
   constexpr int kD = D, kHalves = L_::kHalves, kKStages = L_::kKStages, kVStages = L_::kVStages;
   constexpr int kTileBytes = L_::kTileBytes, kOffK = L_::kOffK, kOffV = L_::kOffV, kSmemData = L_::kSmemData;
@@ -344,14 +373,50 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   if (p.wait_first) pdl_wait_prior();
   pdl_launch_dependents();
   const ChunkWork w = chunk_work(p, p.rows_per_tile);
-  const int b = w.b, kvh = w.kvh, row0 = w.row0, nrows = w.nrows, tok0 = w.tok0, tok1 = w.tok1;
+  const int b = w.b, kvh = w.kvh, row0 = w.row0, nrows = w.nrows;
+  int tok0 = w.tok0, tok1 = w.tok1;
   const bool chain_cta = w.chain_cta;
   float2* out_ml = w.out_ml;
   // key groups sharing the 128 lanes: the Q rows are replicated when the tile has few rows
   const int groups = nrows <= 32 ? 4 : (nrows <= 64 ? 2 : 1);
   const int r_pad = 128 / groups;
   unsigned long long* tr = chain_cta ? p.trace : nullptr;
-  const int n_tiles = (tok1 > tok0) ? (tok1 - tok0 + kTileKeys - 1) / kTileKeys : 0;
+  int n_tiles = (tok1 > tok0) ? (tok1 - tok0 + kTileKeys - 1) / kTileKeys : 0;
+  // a list of chunks: the table of the request's tiles per chunk, then this CTA's share of them
+  int* const hist_prefix = reinterpret_cast<int*>(smem + kSmemData + 256);   // [kMaxHistChunks + 1]
+  int* const hist_valid = hist_prefix + kMaxHistChunks + 1;                  // [kMaxHistChunks]
+  int g0 = 0;
+  if (HIST) {
+    if (warp == 0) {
+      int v = 0;
+      if (lane < h.n_chunks) {
+        const int L = h.L_c[lane];
+        v = h.valid_len[lane] ? h.valid_len[lane][b] : L;
+        if (v < 0 || v > L) {  // flagged and clamped, never trusted
+          atomicOr(p.status, SS_DEV_BAD_VALID_LEN);
+          v = max(0, min(v, L));
+        }
+      }
+      int incl = (v + kTileKeys - 1) / kTileKeys;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+      }
+      if (lane < h.n_chunks) {
+        hist_prefix[lane + 1] = incl;
+        hist_valid[lane] = v;
+      }
+      if (lane == 0) hist_prefix[0] = 0;
+      // (entries past the last chunk repeat the total, so a walk never runs off the table)
+      const int total = __shfl_sync(0xffffffffu, incl, 31);
+      if (lane >= h.n_chunks) hist_prefix[lane + 1] = total;
+    }
+    __syncthreads();
+    const int total = hist_prefix[h.n_chunks];
+    g0 = (int)((int64_t)total * w.split / p.splits);
+    n_tiles = (int)((int64_t)total * (w.split + 1) / p.splits) - g0;
+  }
 
   if (n_tiles == 0 || (smem_u32(smem) & 1023u)) {
     // nothing visible here (identity state, no tensor memory taken); a misaligned shared
@@ -376,10 +441,19 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   // Pages smaller than a tile (8, 16 or 32 tokens): the tile is gathered page by page by the whole
   // producer warp, see below; this path is for contiguous chunks and pages of a tile or more.
   const bool small_pages = p.page_table && p.page_size < kTileKeys;
+  TileMap<true> map_k = {hist_prefix, hist_valid, g0, 0}, map_v = map_k;  // (list of chunks) the producer's two walks
   auto issue_tile = [&](bool is_v, int it, uint32_t dst, uint64_t* bar, uint64_t pol) {
+    mbar_expect_tx(bar, kTileBytes);
+    if (HIST) {
+      int tok;
+      const int c = is_v ? map_v.locate(it, &tok) : map_k.locate(it, &tok);
+      const CUtensorMap* m = h.maps + 2 * c + (is_v ? 1 : 0);  // in device memory
+      tma_load_4d(dst, m, 0, tok, kvh, b, bar, pol);
+      if (D == 128) tma_load_4d(dst + kHalfTile, m, 64, tok, kvh, b, bar, pol);
+      return;
+    }
     int outer, tok;
     locate_token(p, b, tok0 + it * kTileKeys, &outer, &tok);
-    mbar_expect_tx(bar, kTileBytes);
     load_rows(is_v, dst, tok, outer, bar, pol);
   };
   auto issue_k = [&](int it, uint64_t pol) {
@@ -713,9 +787,12 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
     mbar_arrive(&ctl->qready);
     float m = -INFINITY, l = 0.f;
     bool ok;
+    TileMap<HIST> tmap;
+    if constexpr (HIST) tmap = {hist_prefix, hist_valid, g0, 0};
+    else tmap = {tok0, tok1};
 #define SS_LOOP(NC_)                                                                                        \
-  (Tm<D>::NS == 2 ? softmax_loop2<NC_, D>(p, ctl, tmem + lane_off, c0, n_tiles, tok0, tok1, v_s0, L, m, l, tr) \
-                  : softmax_loop<NC_, D>(p, ctl, tmem + lane_off, c0, n_tiles, tok0, tok1, v_s0, L, m, l, tr))
+  (Tm<D>::NS == 2 ? softmax_loop2<NC_, D>(p, ctl, tmem + lane_off, c0, n_tiles, tmap, v_s0, L, m, l, tr) \
+                  : softmax_loop<NC_, D>(p, ctl, tmem + lane_off, c0, n_tiles, tmap, v_s0, L, m, l, tr))
     if (nc == 16)
       ok = SS_LOOP(16);
     else if (nc == 32)
@@ -823,21 +900,40 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
 
 }  // namespace
 
+namespace {
+template <int D, bool HIST>
+cudaError_t prepare_one() {
+  return cudaFuncSetAttribute(chunk_tc_kernel<D, HIST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              Lay<D>::kSmemTotal);
+}
+}  // namespace
+
 cudaError_t chunk_tc_prepare() {
-  cudaError_t e = cudaFuncSetAttribute(chunk_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       Lay<128>::kSmemTotal);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(chunk_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             Lay<64>::kSmemTotal);
+  cudaError_t e = prepare_one<128, false>();
+  if (e == cudaSuccess) e = prepare_one<64, false>();
+  if (e == cudaSuccess) e = prepare_one<128, true>();
+  if (e == cudaSuccess) e = prepare_one<64, true>();
   return e;
 }
 
 cudaError_t launch_chunk_tc(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
                             const CUtensorMap& tmA, cudaStream_t s, bool pdl) {
   dim3 grid(p.splits * p.row_tiles, p.H_kv, p.n_active ? p.n_active : p.B), block(kThreads);
+  static const HistParams none = {};
   if (p.d == 64)
-    return launch_kernel(chunk_tc_kernel<64>, grid, block, Lay<64>::kSmemTotal, s, pdl, p, tmK, tmV, tmA);
-  return launch_kernel(chunk_tc_kernel<128>, grid, block, Lay<128>::kSmemTotal, s, pdl, p, tmK, tmV, tmA);
+    return launch_kernel(chunk_tc_kernel<64, false>, grid, block, Lay<64>::kSmemTotal, s, pdl, p, tmK, tmV, tmA, none);
+  return launch_kernel(chunk_tc_kernel<128, false>, grid, block, Lay<128>::kSmemTotal, s, pdl, p, tmK, tmV, tmA, none);
+}
+
+cudaError_t launch_chunk_tc_hist(const ChunkParams& p, const HistParams& h, const CUtensorMap& tmA,
+                                 cudaStream_t s, bool pdl) {
+  if (h.n_chunks < 1 || h.n_chunks > kMaxHistChunks || !h.maps || p.n_active || p.page_table)
+    return cudaErrorInvalidValue;
+  dim3 grid(p.splits * p.row_tiles, p.H_kv, p.B), block(kThreads);
+  // (the K/V map parameters are not used by this instantiation: any valid map will do)
+  if (p.d == 64)
+    return launch_kernel(chunk_tc_kernel<64, true>, grid, block, Lay<64>::kSmemTotal, s, pdl, p, tmA, tmA, tmA, h);
+  return launch_kernel(chunk_tc_kernel<128, true>, grid, block, Lay<128>::kSmemTotal, s, pdl, p, tmA, tmA, tmA, h);
 }
 
 }  // namespace ss

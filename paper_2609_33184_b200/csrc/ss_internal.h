@@ -62,6 +62,19 @@ struct ChunkParams {
   unsigned int launch_seq;
 };
 
+// A round's history as a list of contiguous chunks, for ONE launch of the rows-on-M kernel over all
+// of them: a CTA takes an equal share of its request's 64-token tiles (counted chunk by chunk from
+// the valid lengths), keeps one accumulator across the chunk boundaries and writes one partial state,
+// so a round has `splits` partial states per row instead of one per chunk call, and its CTAs are as
+// many as the GPU holds at once and equally long.
+constexpr int kMaxHistChunks = 32;
+struct HistParams {
+  int n_chunks;                               // 0: an ordinary one-chunk launch (ChunkParams alone)
+  const CUtensorMap* maps;                    // device memory: chunk j's K map at [2j], its V map at [2j + 1]
+  const int32_t* valid_len[kMaxHistChunks];   // per chunk: device [B], or null (= L_c[j])
+  int L_c[kMaxHistChunks];
+};
+
 // A whole small round for round_simt_kernel: every history chunk, the local segment, outputs.
 constexpr int kMaxRoundChunks = 16;
 constexpr int kRoundCounters = 1024;  // ticket counters in the workspace (units of a split round)
@@ -153,6 +166,9 @@ cudaError_t chunk_simt_prepare();    // one-time function attributes
 int simt_rows_per_tile(int R);       // rows per CTA tile of the CUDA-core chunk kernel
 cudaError_t launch_chunk_tc(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
                             const CUtensorMap& tmA, cudaStream_t s, bool pdl);
+// The same kernel over a list of chunks (HistParams); p.splits = CTAs per (request, kv-head, row tile).
+cudaError_t launch_chunk_tc_hist(const ChunkParams& p, const HistParams& h, const CUtensorMap& tmA,
+                                 cudaStream_t s, bool pdl);
 cudaError_t chunk_tc_prepare();  // one-time function attributes
 cudaError_t launch_chunk_tc_keys(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
                                  cudaStream_t s, bool pdl);

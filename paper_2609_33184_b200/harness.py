@@ -46,12 +46,17 @@ def paged_views(cfg, chunks, page_size, dev):
     return out
 
 
-def run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, ev_pair=None, hints=None, paged=None):
+def run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, ev_pair=None, hints=None, paged=None,
+              descs=None):
+    """One round through the separate calls.  descs (a Context.chunk_descs array for `chunks`):
+    the chunks go in with one ss_verify_chunks call instead of one call each."""
     kind = ssb.SS_MASK_TREE_BITS if cfg.mask == "tree" else ssb.SS_MASK_CHAIN
     ctx.ss_verify_begin(Q, cfg.scale)
     if ev_pair:
         ev_pair[0].record()
-    for j, (K, V, vl) in enumerate(chunks):
+    if descs is not None and paged is None:
+        ctx.ss_verify_chunks(descs, len(chunks))
+    for j, (K, V, vl) in enumerate(chunks if (descs is None or paged is not None) else ()):
         if paged is not None:
             Kp, Vp, table = paged[j]
             ctx.ss_verify_chunk_paged(Kp, Vp, table, vl, hints[j] if hints is not None else None)

@@ -899,3 +899,64 @@ def test_whole_round_in_one_call_large_and_errors():
         ctx.ss_verify_round(Q, cfg.scale, chunks, K_loc, V_loc, ssb.SS_MASK_CHAIN, None, O2, L2)
     ctx.ss_verify_abort()
     ctx.close()
+
+
+@pytest.mark.parametrize("d,T_q,H_q,H_kv", [(128, 40, 8, 2), (128, 24, 16, 2), (64, 40, 8, 2), (128, 64, 10, 2)])
+def test_chunk_list_in_one_launch(d, T_q, H_q, H_kv):
+    """ss_verify_chunks with more than 128 rows per kv-head: the whole list of chunks goes out as
+    one launch whose CTAs walk tiles across chunk boundaries.  Checked against the oracle with the
+    list in history order and reversed (the ragged chunk and the empty ones then come first and a
+    partly filled chunk sits in the middle of a CTA's walk), against the separate calls, and for
+    bit-identical repeats."""
+    from paper_2609_33184_b200 import binding as ssb
+    cfg = inputs.VerifyConfig("hist", 0xb7 + d + T_q, 4, H_q, H_kv, d, 512, T_q, 0, 3000)
+    lens = [3000, 1, 1537, 0]     # ragged, a single token, one token past a chunk boundary, nothing
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    assert len(chunks) == 6
+    ctx = util.make_ctx(cfg, flags=ssb.SS_FLAG_OVERLAP_CHUNKS)
+    O5, L5 = util.gpu_case(ctx, cfg, Q, chunks, K_loc, V_loc, bits)
+    assert ctx.last_chunk_kernel() == "tcgen05"
+    ref = util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits)
+    util.compare(cfg, O5, L5, ref)
+    outs = []
+    for order in (list(range(6)), list(range(5, -1, -1)), [2, 5, 0, 3, 1, 4]):
+        lst = [chunks[j] for j in order]
+        descs = ctx.chunk_descs([lst])
+        O, LSE = torch.empty_like(O5), torch.empty_like(L5)
+        for rep in range(3):
+            ctx.ss_verify_begin(Q, cfg.scale)
+            ctx.ss_verify_chunks(descs, len(lst))
+            ctx.ss_verify_local(K_loc, V_loc, ssb.SS_MASK_CHAIN, None)
+            ctx.ss_verify_finalize(O, LSE)
+            torch.cuda.synchronize()
+            assert ctx.last_chunk_kernel() == "tcgen05-round"
+            assert ctx.ss_poll_status() == (0, 0)
+            if rep == 0:
+                O0, L0 = O.clone(), LSE.clone()
+            else:
+                assert torch.equal(O0.view(torch.int16), O.view(torch.int16)) and torch.equal(L0, LSE)
+        util.compare(cfg, O, LSE, util.oracle_case(cfg, lens, Q, lst, K_loc, V_loc, bits))
+        outs.append(O0)
+    # the same through ss_verify_round
+    O, LSE = torch.empty_like(O5), torch.empty_like(L5)
+    ctx.ss_verify_round(Q, cfg.scale, chunks, K_loc, V_loc, ssb.SS_MASK_CHAIN, None, O, LSE)
+    torch.cuda.synchronize()
+    assert ctx.last_chunk_kernel() == "tcgen05-round"
+    assert torch.equal(O.view(torch.int16), outs[0].view(torch.int16))
+    # a bad valid length is flagged and clamped; a chunk beyond the context's size is refused and
+    # leaves the round open
+    bad = [(K, V, vl.clone()) for (K, V, vl) in chunks]
+    bad[1][2][0] = 9999
+    ctx.ss_verify_begin(Q, cfg.scale)
+    ctx.ss_verify_chunks(ctx.chunk_descs([bad]), 6)
+    ctx.ss_verify_local(K_loc, V_loc, ssb.SS_MASK_CHAIN, None)
+    ctx.ss_verify_finalize(O, LSE)
+    torch.cuda.synchronize()
+    st, bits_ = ctx.ss_poll_status()
+    assert bits_ & ssb.SS_DEV_BAD_VALID_LEN
+    big = torch.zeros(4, H_kv, 1024, d, dtype=torch.bfloat16, device=DEV)
+    ctx.ss_verify_begin(Q, cfg.scale)
+    with pytest.raises(ssb.SpecStreamError):
+        ctx.ss_verify_chunks(ctx.chunk_descs([chunks[:2] + [(big, big, None)]]), 3)
+    ctx.ss_verify_abort()
+    ctx.close()
