@@ -84,6 +84,8 @@ def ncu_traffic(workload: str, kernel: str, alg_bytes: float = 0.0):
     e = table.get(workload)
     if not e:
         return None, "no ncu capture of this workload"
+    if isinstance(e, list):   # captures of several kernels: the one this run routed, if any
+        e = next((x for x in e if x.get("kernel") == kernel), e[0])
     if e.get("kernel") != kernel:
         return None, f"captured on kernel {e.get('kernel')!r}, this run routed {kernel!r}"
     if "ratio_to_algorithmic" in e:
