@@ -166,9 +166,9 @@ ss_status ss_verify_chunk_paged(ss_ctx* ctx, ss_tensor K_pool, ss_tensor V_pool,
 /* a2, several chunks with one call (Section 4.2: the chunks of a request are reduced into one
  * running state; Eq. 13-14).  chunks is a HOST array of n_chunks (>= 0) descriptors, read before
  * the call returns; the result is that of one ss_verify_chunk_hinted per descriptor, in order.
- * Where the rows-on-M tensor-core kernel would take every chunk (more than
+ * Where the rows-on-M tensor-core kernel would take every chunk (head dim 128, more than
  * 128 query rows per kv-head, 2 to 32 contiguous chunks, one CTA per (request, kv-head, row tile)
- * fitting the GPU at once) the whole list takes ONE launch: a CTA walks an equal share of its
+ * fitting the GPU at once; SS_HISTORY_LAUNCH=never|always in the environment overrides the routing) the whole list takes ONE launch: a CTA walks an equal share of its
  * request's 64-token tiles across the chunk boundaries with one accumulator, so the list leaves
  * a few partial states per row instead of one per chunk and its CTAs are equally long
  * ("tcgen05-round" in ss_last_chunk_kernel).  Otherwise the chunks are enqueued one by one.

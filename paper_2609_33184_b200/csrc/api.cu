@@ -734,15 +734,19 @@ ss_status ss_verify_finalize(ss_ctx* c, void* O, float* LSE, void* stream) {
 static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunks, bool* taken) {
   *taken = false;
   if (!c->tc_ok || n_chunks < 2 || n_chunks > ss::kMaxHistChunks || c->force_keys_kernel) return SS_OK;
-  if (getenv("SS_NO_HISTORY_LAUNCH")) return SS_OK;
+  // SS_HISTORY_LAUNCH=never / always overrides the routing below (not the limits of the launch)
+  const char* hl = getenv("SS_HISTORY_LAUNCH");
+  if (hl && strcmp(hl, "never") == 0) return SS_OK;
+  const bool always = hl && strcmp(hl, "always") == 0;
   const int R = c->T_q * c->G, pairs = c->B * c->cfg.H_kv;
   const int keys_max_rows = c->cfg.d == 64 ? 16 : 32;
   if (R <= keys_max_rows && !c->force_rows_kernel) return SS_OK;   // the keys-on-M kernel's rounds
   // With up to 128 rows per kv-head the chunk kernels run at the HBM ceiling while the GPU is full
   // and successive launches keep it full; the one launch pays off where the tile's arithmetic
-  // bounds the kernel (measured: +5 % at 192 rows, +11-13 % on the 320-row tree workload, -4 % at 48).
+  // bounds the kernel (measured at head dim 128: +5 % at 192 rows, +22 % at 256, +8-13 % on the
+  // 320-row tree workload, -4 % at 48; at head dim 64: -3 % at 192 rows, 0 at 320).
   const int row_tiles = (R + 127) / 128;
-  if (row_tiles < 2 && !getenv("SS_HISTORY_LAUNCH_ALWAYS")) return SS_OK;
+  if (!always && (row_tiles < 2 || c->cfg.d != 128)) return SS_OK;
   const int64_t units = (int64_t)pairs * row_tiles;
   const int wave = 2 * ss::kNumSM;                                  // two CTAs per SM
   if (units > wave) return SS_OK;

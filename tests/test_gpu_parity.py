@@ -902,13 +902,15 @@ def test_whole_round_in_one_call_large_and_errors():
 
 
 @pytest.mark.parametrize("d,T_q,H_q,H_kv", [(128, 40, 8, 2), (128, 24, 16, 2), (64, 40, 8, 2), (128, 64, 10, 2)])
-def test_chunk_list_in_one_launch(d, T_q, H_q, H_kv):
+def test_chunk_list_in_one_launch(d, T_q, H_q, H_kv, monkeypatch):
     """ss_verify_chunks with more than 128 rows per kv-head: the whole list of chunks goes out as
     one launch whose CTAs walk tiles across chunk boundaries.  Checked against the oracle with the
     list in history order and reversed (the ragged chunk and the empty ones then come first and a
     partly filled chunk sits in the middle of a CTA's walk), against the separate calls, and for
     bit-identical repeats."""
     from paper_2609_33184_b200 import binding as ssb
+    if d == 64:   # routed at head dim 128 only (where it is faster); the launch itself takes both
+        monkeypatch.setenv("SS_HISTORY_LAUNCH", "always")
     cfg = inputs.VerifyConfig("hist", 0xb7 + d + T_q, 4, H_q, H_kv, d, 512, T_q, 0, 3000)
     lens = [3000, 1, 1537, 0]     # ragged, a single token, one token past a chunk boundary, nothing
     Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
