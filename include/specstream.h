@@ -77,7 +77,8 @@ typedef struct {
   int32_t max_Tloc;   /* local candidate KV tokens per request (<= 1024)             */
   int32_t max_Lc;     /* tokens per history chunk call                               */
   int32_t max_chunks; /* chunk calls held as separate partial sets before the library
-                         folds them (any number of calls stays legal); 0 = default 64 */
+                         folds them (any number of calls stays legal); 0 = default 64;
+                         1 is taken as 2 (a fold needs a free set to go on with)      */
   int32_t device;     /* CUDA device ordinal                                         */
   uint32_t flags;     /* SS_FLAG_*                                                   */
 } ss_config;

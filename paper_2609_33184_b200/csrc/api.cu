@@ -102,7 +102,8 @@ bool cfg_valid(const ss_config* c) {
   return true;
 }
 
-int set_cap(const ss_config* c) { return c->max_chunks ? c->max_chunks : 64; }
+// partial sets for chunk calls: at least two, so that a fold (all sets -> set 0) leaves one free
+int set_cap(const ss_config* c) { return c->max_chunks ? (c->max_chunks < 2 ? 2 : c->max_chunks) : 64; }
 
 int target_ctas_default() {
   const char* e = getenv("SS_TARGET_CTAS");
@@ -766,6 +767,10 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
   if (c->force_splits > 0 && c->force_splits < splits) splits = c->force_splits;
   if (splits < 1) splits = 1;
 
+  if (c->n_sets == c->n_set_cap) {  // every partial set is in use: fold them into one first
+    cudaError_t e = fold_sets(c, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+  }
   // the chunks' tensor maps, K and V alternating, in one of the workspace's lists
   CUtensorMap maps[2 * ss::kMaxHistChunks];
   for (int j = 0; j < n_chunks; ++j)

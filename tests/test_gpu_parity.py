@@ -962,3 +962,34 @@ def test_chunk_list_in_one_launch(d, T_q, H_q, H_kv, monkeypatch):
         ctx.ss_verify_chunks(ctx.chunk_descs([chunks[:2] + [(big, big, None)]]), 3)
     ctx.ss_verify_abort()
     ctx.close()
+
+
+def test_chunk_list_after_separate_chunks_with_one_partial_set():
+    """A context with a single partial set: a chunk call, then a list of chunks in one launch (the
+    set in use is folded first), then another chunk call; against the oracle."""
+    from paper_2609_33184_b200 import binding as ssb
+    cfg = inputs.VerifyConfig("hist1", 0xc3, 2, 8, 2, 128, 512, 40, 0, 2500)
+    lens = [2500, 900]
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    assert len(chunks) == 5
+    ctx = util.make_ctx(cfg, flags=ssb.SS_FLAG_OVERLAP_CHUNKS, max_chunks=1)
+    O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
+    LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
+    ctx.ss_verify_begin(Q, cfg.scale)
+    ctx.ss_verify_chunk(*chunks[0])
+    ctx.ss_verify_chunks(ctx.chunk_descs([chunks[1:4]]), 3)
+    assert ctx.last_chunk_kernel() == "tcgen05-round"
+    ctx.ss_verify_chunk(*chunks[4])
+    ctx.ss_verify_local(K_loc, V_loc, ssb.SS_MASK_CHAIN, None)
+    ctx.ss_verify_finalize(O, LSE)
+    torch.cuda.synchronize()
+    assert ctx.ss_poll_status() == (0, 0)
+    util.compare(cfg, O, LSE, util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits))
+    ctx.close()
+
+
+def test_two_chunk_calls_with_max_chunks_one():
+    """max_chunks = 1 still leaves room to fold: a second chunk call must not land on the local
+    segment's partial set."""
+    cfg = inputs.VerifyConfig("v", 0x59, 2, 8, 2, 128, 256, 8, 600, 700)
+    _run(cfg, max_chunks=1)
