@@ -89,7 +89,11 @@ typedef struct {
  * launch).  The caller promises that Q and the K/V of a chunk call are complete in
  * memory before the PREVIOUS ss_ call of the round was enqueued on the stream, or were
  * produced by a copy / an event the stream waited on - not by a kernel enqueued on the
- * same stream between two ss_ calls. */
+ * same stream between two ss_ calls.  With the flag a round's FIRST chunk kernel (and the
+ * single launch of a small ss_verify_round) is also launched that way, but waits for the
+ * completion of whatever precedes it on the stream before it reads or writes anything:
+ * only its launch and set-up overlap the previous round's finalize, and the promise above
+ * is not needed for it. */
 #define SS_FLAG_OVERLAP_CHUNKS 2u
 /* Use the tensor-core chunk kernel that puts the query rows on the MMA's M axis instead of
  * the default one that puts the keys there.  For cross-checks. */

@@ -213,6 +213,11 @@ bool encode_partials_map(ss_ctx* c) {
 bool use_pdl(ss_ctx* c) {
   return (c->cfg.flags & SS_FLAG_OVERLAP_CHUNKS) && !c->first_launch && !c->no_overlap;
 }
+// Chunk kernels (and the one-launch small round) can also be the FIRST kernel of a round under
+// programmatic stream serialization: with wait_first they do nothing before the kernel in front of
+// them (the previous round's finalize, a fold, anything else) has completed, so only their launch
+// and set-up overlap it.
+bool use_pdl_first(ss_ctx* c) { return (c->cfg.flags & SS_FLAG_OVERLAP_CHUNKS) && !c->no_overlap; }
 
 void fill_merge(ss_ctx* c, ss::MergeParams* m) {
   memset(m, 0, sizeof(*m));
@@ -581,7 +586,7 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
   if (hint.n_listed) memcpy(p.active_b, hint.listed, (size_t)hint.n_listed);
   p.a_slot0 = c->n_sets * c->slots_per_set;
   p.status = c->status;
-  p.wait_first = 0;
+  p.wait_first = c->first_launch ? 1 : 0;
   p.trace = c->trace_on ? c->trace : nullptr;
   p.cta_log = c->cta_log;
   p.cta_log_cap = c->cta_log_cap;
@@ -593,7 +598,7 @@ static ss_status chunk_impl(ss_ctx* c, ss_tensor K, ss_tensor V, int32_t L_c, co
     p.n_pages = pg->n_pages;
   }
 
-  const bool pdl = use_pdl(c);
+  const bool pdl = use_pdl_first(c);
   cudaError_t e = !tc ? ss::launch_chunk_simt(p, s, pdl)
                   : keys_on_m ? ss::launch_chunk_tc_keys(p, tmK, tmV, s, pdl)
                               : ss::launch_chunk_tc(p, tmK, tmV, c->tm_a, s, pdl);
@@ -840,7 +845,8 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
   p.cta_log = c->cta_log;
   p.cta_log_cap = c->cta_log_cap;
   p.launch_seq = (unsigned int)c->launches;
-  cudaError_t e = ss::launch_chunk_tc_hist(p, h, c->tm_a, s, use_pdl(c));
+  p.wait_first = c->first_launch ? 1 : 0;
+  cudaError_t e = ss::launch_chunk_tc_hist(p, h, c->tm_a, s, use_pdl_first(c));
   if (e != cudaSuccess) return cuda_fail(c, e);
   c->last_kernel = "tcgen05-round";
   ++c->launches;
@@ -949,7 +955,7 @@ ss_status ss_verify_round(ss_ctx* c, ss_tensor Q, int32_t B, int32_t T_q, float 
     p.O = (__nv_bfloat16*)O;
     p.LSE = LSE;
     p.status = c->status;
-    cudaError_t e = ss::launch_round_simt(p, (cudaStream_t)stream);
+    cudaError_t e = ss::launch_round_simt(p, (cudaStream_t)stream, (c->cfg.flags & SS_FLAG_OVERLAP_CHUNKS) && !c->no_overlap);
     if (e != cudaSuccess) return cuda_fail(c, e);
     c->last_kernel = "simt-round";
     ++c->launches;

@@ -363,6 +363,11 @@ __global__ void __launch_bounds__(kThreads) round_simt_kernel(const __grid_const
   const int rt = blockIdx.x % row_tiles, sp = blockIdx.x / row_tiles;
   const int b = blockIdx.z, kvh = blockIdx.y, row0 = rt * RT;
   const int R = p.T_q * p.G, nrows = min(RT, R - row0);
+  // Launched with programmatic stream serialization, the grid is set up while the kernel before
+  // it (typically the previous round's) is still running; nothing is read or written before
+  // that kernel has completed.  The next launch is let in at once on the same terms.
+  pdl_launch_dependents();
+  pdl_wait_prior();
   st.q_fetch(p.Q, p.q_sb, p.q_sh, p.q_st, b, kvh, p.G, p.T_q, row0, nrows);
   bool q_pending = true;
   Source src;
@@ -540,11 +545,11 @@ cudaError_t launch_chunk_simt(const ChunkParams& p, cudaStream_t s, bool pdl) {
   return SS_SIMT_DISPATCH(chunk_simt_kernel, p.d, p.rows_per_tile, grid, block, smem, s, pdl, p);
 }
 
-cudaError_t launch_round_simt(const RoundParams& p, cudaStream_t s) {
+cudaError_t launch_round_simt(const RoundParams& p, cudaStream_t s, bool pdl) {
   const int R = p.T_q * p.G, rt = p.rows_per_tile;
   dim3 grid(((R + rt - 1) / rt) * p.splits, p.H_kv, p.B), block(kThreads);
   const size_t smem = simt_smem(p.d, rt);
-  return SS_SIMT_DISPATCH(round_simt_kernel, p.d, rt, grid, block, smem, s, false, p);
+  return SS_SIMT_DISPATCH(round_simt_kernel, p.d, rt, grid, block, smem, s, pdl, p);
 }
 
 }  // namespace ss

@@ -199,6 +199,9 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) merge_kernel(const MergePar
   __syncthreads();
   const int64_t row_id = (int64_t)blockIdx.x * kWarpsPerCta + warp;
   const int64_t n_rows = (int64_t)p.B * p.H_q * p.T_q;
+  // (finalize) the next kernel may be set up meanwhile: the first chunk kernel of the next round
+  // waits for this grid's completion before it reads or writes anything
+  if (MODE == 0) pdl_launch_dependents();
   if (MODE == 0) pdl_wait_prior();  // every partial of the round must be complete
   if (row_id >= n_rows) return;
   const unsigned rid = (unsigned)row_id;  // 32-bit index arithmetic: the row count fits

@@ -161,7 +161,7 @@ struct GatherParams {
 
 // launchers (each returns the cudaError_t of the launch)
 cudaError_t launch_chunk_simt(const ChunkParams& p, cudaStream_t s, bool pdl);
-cudaError_t launch_round_simt(const RoundParams& p, cudaStream_t s);
+cudaError_t launch_round_simt(const RoundParams& p, cudaStream_t s, bool pdl);
 cudaError_t chunk_simt_prepare();    // one-time function attributes
 int simt_rows_per_tile(int R);       // rows per CTA tile of the CUDA-core chunk kernel
 cudaError_t launch_chunk_tc(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
