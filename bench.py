@@ -236,7 +236,8 @@ class Workload:
         self.O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=dev)
         self.LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=dev)
         self.nbytes = kv_bytes(cfg, self.lens)
-        self.hints = host_valid(cfg, self.lens, len(self.chunks)) if len(set(self.lens)) > 1 else None
+        # the host's copy of the valid lengths goes with every chunk (scheduling hint)
+        self.hints = host_valid(cfg, self.lens, len(self.chunks)) if self.chunks else None
         # A workload whose history fits in L2 (the tiny chain: 256 KiB) is timed over rotating
         # copies of its history buffers, more than two L2 capacities in total, so that every round
         # reads HBM; the large workloads stream more than L2 per round by themselves.

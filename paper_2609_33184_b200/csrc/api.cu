@@ -11,6 +11,7 @@ struct ss_ctx {
   ss_config cfg;
   int G, R_max, R_stride;
   int slots_per_set;       // (split, b, kvh) slots of one partial set
+  int slots_chunk_call;    // of which a single chunk call may use (its split policy's limit)
   int n_set_cap;           // chunk sets (the local set is one more)
   uint8_t* ws;
   size_t ws_bytes;
@@ -120,6 +121,16 @@ int slots_for(const ss_config* c) {
   if (s > kMaxSplits) s = kMaxSplits;
   return pairs * s;
 }
+// Slots a partial set holds: room for two CTAs per SM (a launch over a list of chunks has all of
+// its CTAs resident at once), at least what a chunk call may use.
+int slot_capacity_for(const ss_config* c) {
+  const int pairs = c->max_B * c->H_kv;
+  int s = 2 * ss::kNumSM / pairs;
+  if (s < 1) s = 1;
+  if (s > kMaxSplits) s = kMaxSplits;
+  const int cap = pairs * s, use = slots_for(c);
+  return cap > use ? cap : use;
+}
 
 constexpr int kHistSlots = 4;
 struct Layout {
@@ -132,7 +143,7 @@ Layout layout_for(const ss_config* c) {
   Layout L;
   const int G = c->H_q / c->H_kv;
   L.R_stride = c->max_Tq * G;
-  const int64_t rows = (int64_t)slots_for(c) * L.R_stride;
+  const int64_t rows = (int64_t)slot_capacity_for(c) * L.R_stride;
   L.set_stride_ml = rows;                 // float2 elements
   L.set_stride_a = rows * c->d;           // float elements
   const int sets = set_cap(c) + 1;
@@ -304,7 +315,7 @@ HintScan scan_hint(const ss_ctx* c, const int32_t* valid_len_host, int L_c) {
 int pick_splits(ss_ctx* c, bool tensor_core, bool whole_waves, int pairs, int ctas1, int used_tiles) {
   // tensor-core CTAs amortise their set-up over at least 256 tokens; CUDA-core CTAs take one tile
   const int min_tiles = tensor_core ? 4 : 1;
-  int max_splits = c->slots_per_set / pairs;
+  int max_splits = c->slots_chunk_call / pairs;
   if (max_splits > kMaxSplits) max_splits = kMaxSplits;
   if (max_splits > (used_tiles + min_tiles - 1) / min_tiles) max_splits = (used_tiles + min_tiles - 1) / min_tiles;
   if (max_splits < 1) max_splits = 1;
@@ -371,7 +382,8 @@ ss_status ss_create(ss_ctx** out, const ss_config* cfg, void* workspace, size_t 
   c->G = cfg->H_q / cfg->H_kv;
   c->R_max = cfg->max_Tq * c->G;
   c->R_stride = L.R_stride;
-  c->slots_per_set = slots_for(cfg);
+  c->slots_per_set = slot_capacity_for(cfg);
+  c->slots_chunk_call = slots_for(cfg);
   c->n_set_cap = set_cap(cfg);
   c->ws = (uint8_t*)workspace;
   c->ws_bytes = workspace_bytes;
@@ -739,20 +751,44 @@ ss_status ss_verify_finalize(ss_ctx* c, void* O, float* LSE, void* stream) {
 // round does not qualify (nothing has been enqueued then).
 static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunks, bool* taken) {
   *taken = false;
-  if (!c->tc_ok || n_chunks < 2 || n_chunks > ss::kMaxHistChunks || c->force_keys_kernel) return SS_OK;
+  if (!c->tc_ok || n_chunks < 2 || n_chunks > ss::kMaxHistChunks) return SS_OK;
   // SS_HISTORY_LAUNCH=never / always overrides the routing below (not the limits of the launch)
   const char* hl = getenv("SS_HISTORY_LAUNCH");
   if (hl && strcmp(hl, "never") == 0) return SS_OK;
   const bool always = hl && strcmp(hl, "always") == 0;
   const int R = c->T_q * c->G, pairs = c->B * c->cfg.H_kv;
   const int keys_max_rows = c->cfg.d == 64 ? 16 : 32;
-  if (R <= keys_max_rows && !c->force_rows_kernel) return SS_OK;   // the keys-on-M kernel's rounds
+  const bool keys_on_m = !c->force_rows_kernel && (R <= keys_max_rows || c->force_keys_kernel);
   // With up to 128 rows per kv-head the chunk kernels run at the HBM ceiling while the GPU is full
   // and successive launches keep it full; the one launch pays off where the tile's arithmetic
   // bounds the kernel (measured at head dim 128: +5 % at 192 rows, +22 % at 256, +8-13 % on the
   // 320-row tree workload, -4 % at 48; at head dim 64: -3 % at 192 rows, 0 at 320).
+  // The keys-on-M kernel (up to 32 rows per kv-head) runs at the HBM ceiling, and a CTA that walks
+  // 32,768 tokens instead of one chunk call's 2,048 pays set-up, ring fill and drain once instead
+  // of sixteen times (measured on the Qwen3-8B-shaped workload: +5 %); taken when the requests'
+  // histories are known to be about equally long (the CTAs of one launch should end together):
+  // no lengths at all, or a host copy of the lengths whose totals differ by at most 10 %.
   const int row_tiles = (R + 127) / 128;
-  if (!always && (row_tiles < 2 || c->cfg.d != 128)) return SS_OK;
+  if (keys_on_m) {
+    if (c->cfg.d != 128 || R > 32 || n_chunks > 16) return SS_OK;
+    bool ragged = false;
+    int64_t lo = INT64_MAX, hi = 0;
+    for (int b = 0; b < c->B && !ragged; ++b) {
+      int64_t len = 0;
+      for (int j = 0; j < n_chunks; ++j) {
+        const ss_chunk_desc& d = chunks[j];
+        if (!d.valid_len) len += d.L_c;
+        else if (d.valid_len_host) len += d.valid_len_host[b] < 0 ? 0 : (d.valid_len_host[b] > d.L_c ? d.L_c : d.valid_len_host[b]);
+        else ragged = true;  // unknown to the host
+      }
+      lo = len < lo ? len : lo;
+      hi = len > hi ? len : hi;
+    }
+    ragged = ragged || hi > lo + lo / 10;
+    if (ragged && !always) return SS_OK;
+  } else if (!always && (row_tiles < 2 || c->cfg.d != 128)) {
+    return SS_OK;
+  }
   const int64_t units = (int64_t)pairs * row_tiles;
   const int wave = 2 * ss::kNumSM;                                  // two CTAs per SM
   if (units > wave) return SS_OK;
@@ -763,6 +799,7 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
     if (d.L_c > c->cfg.max_Lc) return SS_ERR_SHAPE;
     if (!tensor_ok(d.K) || !tensor_ok(d.V) || (d.valid_len && ((uintptr_t)d.valid_len & 3))) return SS_ERR_ALIGN;
     tiles += (d.L_c + kTileKeys - 1) / kTileKeys;
+    if (keys_on_m && d.L_c < 128) return SS_OK;   // (a box of 128 tokens)
   }
   if (tiles > 0x3fffffff) return SS_OK;
   int splits = (int)(wave / units);
@@ -779,8 +816,8 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
   // the chunks' tensor maps, K and V alternating, in one of the workspace's lists
   CUtensorMap maps[2 * ss::kMaxHistChunks];
   for (int j = 0; j < n_chunks; ++j)
-    if (!get_tensor_map(c, chunks[j].K, c->B, chunks[j].L_c, kTileKeys, &maps[2 * j]) ||
-        !get_tensor_map(c, chunks[j].V, c->B, chunks[j].L_c, kTileKeys, &maps[2 * j + 1]))
+    if (!get_tensor_map(c, chunks[j].K, c->B, chunks[j].L_c, keys_on_m ? 128 : kTileKeys, &maps[2 * j]) ||
+        !get_tensor_map(c, chunks[j].V, c->B, chunks[j].L_c, keys_on_m ? 128 : kTileKeys, &maps[2 * j + 1]))
       return SS_OK;
   int slot = -1;
   for (int i = 0; i < kHistSlots && slot < 0; ++i)
@@ -846,9 +883,10 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
   p.cta_log_cap = c->cta_log_cap;
   p.launch_seq = (unsigned int)c->launches;
   p.wait_first = c->first_launch ? 1 : 0;
-  cudaError_t e = ss::launch_chunk_tc_hist(p, h, c->tm_a, s, use_pdl_first(c));
+  cudaError_t e = keys_on_m ? ss::launch_chunk_tc_keys_hist(p, h, c->tm_a, s, use_pdl_first(c))
+                            : ss::launch_chunk_tc_hist(p, h, c->tm_a, s, use_pdl_first(c));
   if (e != cudaSuccess) return cuda_fail(c, e);
-  c->last_kernel = "tcgen05-round";
+  c->last_kernel = keys_on_m ? "tcgen05-keys-round" : "tcgen05-round";
   ++c->launches;
   c->stats.chunk_calls += n_chunks;
   c->stats.kv_bytes += tokens * c->cfg.H_kv * c->cfg.d * 4;

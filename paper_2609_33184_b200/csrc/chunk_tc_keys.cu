@@ -50,6 +50,7 @@ using namespace ss::tc;
 constexpr int kKeys = 128;                  // keys per tile = MMA M
 constexpr int kHalf = kKeys * 64 * 2;       // 16 KB: [128 keys][64 d] bf16, one TMA box
 constexpr float kLazyThreshold = 16.f;
+constexpr int kMaxHistChunksKeys = 16;      // chunks one launch over a list of chunks takes (table in the control block)
 
 template <int N>
 struct alignas(16) Ctl {
@@ -60,6 +61,9 @@ struct alignas(16) Ctl {
   volatile uint32_t flag[3];
   alignas(16) float nm_ref[N];    // NEGATED row references -m[r] (+inf = none yet); read as float4
   alignas(16) float smax[4][N];   // per lane quadrant
+  // launch over a list of chunks: 128-token tiles of the request before chunk j, its tokens in chunk j
+  int hist_prefix[kMaxHistChunksKeys + 1];
+  int hist_valid[kMaxHistChunksKeys];
 };
 
 // NC = score columns per softmax thread, WG = softmax warpgroups (threads sharing a TMEM lane),
@@ -90,10 +94,12 @@ struct Cfg {
 };
 
 
-template <int NC, int WG, int UNITS, int D>
+// HIST: the launch covers a list of chunks (HistParams; see ss_internal.h): the CTA walks an equal
+// share of its request's 128-token tiles, counted chunk by chunk, with one accumulator.
+template <int NC, int WG, int UNITS, int D, bool HIST>
 __global__ void __launch_bounds__(Cfg<NC, WG, UNITS, D>::kThreads, Cfg<NC, WG, UNITS, D>::kMinBlocks)
 chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
-                     const __grid_constant__ CUtensorMap tmV) {
+                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ HistParams h) {
   using C = Cfg<NC, WG, UNITS, D>;
   constexpr int N = C::N;
   constexpr int kD = D, kUnitBytes = C::kUnitBytes;
@@ -118,7 +124,46 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
   const int n_mma = (nrows + 15) & ~15;                 // MMA N of this CTA
   unsigned long long* tr = chain_cta ? p.trace : nullptr;
   // splits are given in 64-token tiles by the host; this kernel walks 128-token tiles
-  const int n_tiles = (tok1 > tok0) ? (tok1 - tok0 + kKeys - 1) / kKeys : 0;
+  int n_tiles = (tok1 > tok0) ? (tok1 - tok0 + kKeys - 1) / kKeys : 0;
+  int g0 = 0;  // (list of chunks) the CTA's first tile in the request's numbering
+  if (HIST) {
+    if (warp == 0) {
+      int v = 0;
+      if (lane < h.n_chunks) {
+        const int Lc = h.L_c[lane];
+        v = h.valid_len[lane] ? h.valid_len[lane][b] : Lc;
+        if (v < 0 || v > Lc) {  // flagged and clamped, never trusted
+          atomicOr(p.status, SS_DEV_BAD_VALID_LEN);
+          v = max(0, min(v, Lc));
+        }
+      }
+      int incl = (v + kKeys - 1) / kKeys;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+      }
+      if (lane < h.n_chunks) {
+        ctl->hist_prefix[lane + 1] = incl;
+        ctl->hist_valid[lane] = v;
+      }
+      if (lane == 0) ctl->hist_prefix[0] = 0;
+      const int total = __shfl_sync(0xffffffffu, incl, 31);
+      if (lane >= h.n_chunks && lane < kMaxHistChunksKeys) ctl->hist_prefix[lane + 1] = total;
+    }
+    __syncthreads();
+    const int total = ctl->hist_prefix[h.n_chunks];
+    g0 = (int)((int64_t)total * w.split / p.splits);
+    n_tiles = (int)((int64_t)total * (w.split + 1) / p.splits) - g0;
+  }
+  // (list of chunks) chunk of the CTA's tile t and the tile's first token in it; tiles are asked
+  // for in ascending order, `cur` is the caller's own cursor
+  auto hist_locate = [&](int t, int& cur, int* tok) {
+    const int g = g0 + t;
+    while (g >= ctl->hist_prefix[cur + 1]) ++cur;
+    *tok = (g - ctl->hist_prefix[cur]) * kKeys;
+    return cur;
+  };
 
   if (n_tiles == 0 || (smem_u32(smem) & 1023u)) {
     // nothing visible here (identity state, no tensor memory taken); a misaligned shared
@@ -147,11 +192,21 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
   // Pages smaller than a tile (8 to 64 tokens): the tile is gathered page by page by the
   // whole producer warp, see below; this path is for contiguous chunks and pages of a tile or more.
   const bool small_pages = p.page_table && p.page_size < kKeys;
+  int prod_chunk = 0;  // (list of chunks) the producer's cursor
   auto issue_use = [&](int j, uint64_t pol) {
     const int u = j % UNITS;
+    mbar_expect_tx(&ctl->ufull[u], kUnitBytes);
+    if (HIST) {
+      int tok;
+      const int c = hist_locate(j >> 1, prod_chunk, &tok);
+      const CUtensorMap* m = h.maps + 2 * c + (j & 1);  // in device memory
+      const uint32_t dst = smem_u32(smem + u * kUnitBytes);
+      tma_load_4d(dst, m, 0, tok, kvh, b, &ctl->ufull[u], pol);
+      if (D == 128) tma_load_4d(dst + kHalf, m, 64, tok, kvh, b, &ctl->ufull[u], pol);
+      return;
+    }
     int outer, tok;
     locate_token(p, b, tok0 + (j >> 1) * kKeys, &outer, &tok);
-    mbar_expect_tx(&ctl->ufull[u], kUnitBytes);
     load_rows(j & 1, smem_u32(smem + u * kUnitBytes), tok, outer, &ctl->ufull[u], pol);
   };
   const int n_uses = 2 * n_tiles;
@@ -396,12 +451,20 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
     float2 lsum[NC / 2];  // row sums of this key lane, two rows per packed add
 #pragma unroll
     for (int r = 0; r < NC / 2; ++r) lsum[r] = make_float2(0.f, 0.f);
+    int soft_chunk = 0;  // (list of chunks) this thread's cursor
     for (int t = 0; t < n_tiles; ++t) {
       if (tid == 0) trace(tr, 2, t, 0);
       wait(&ctl->sfull[t & 1], (t >> 1) & 1);
       tc_fence_after();
       if (tid == 0) trace(tr, 2, t, 1);
-      const int n_valid = min(kKeys, tok1 - (tok0 + t * kKeys));
+      int n_valid;
+      if (HIST) {
+        int tok;
+        const int c = hist_locate(t, soft_chunk, &tok);
+        n_valid = min(kKeys, ctl->hist_valid[c] - tok);
+      } else {
+        n_valid = min(kKeys, tok1 - (tok0 + t * kKeys));
+      }
       const bool key_ok = L < n_valid;
       if (n_valid < kKeys) {
         // ragged tail: tokens past the valid length may hold anything; their weights are 0, so
@@ -668,12 +731,13 @@ cudaError_t launch_cfg(const ChunkParams& p, const CUtensorMap& tmK, const CUten
                        cudaStream_t s, bool pdl) {
   using C = Cfg<NC, WG, UNITS, D>;
   dim3 grid(p.splits * p.row_tiles, p.H_kv, p.n_active ? p.n_active : p.B), block(C::kThreads);
-  return launch_kernel(chunk_tc_keys_kernel<NC, WG, UNITS, D>, grid, block, C::kSmem, s, pdl, p, tmK, tmV);
+  static const HistParams none = {};
+  return launch_kernel(chunk_tc_keys_kernel<NC, WG, UNITS, D, false>, grid, block, C::kSmem, s, pdl, p, tmK, tmV, none);
 }
 
 template <int NC, int WG, int UNITS, int D>
 cudaError_t prepare_cfg() {
-  return cudaFuncSetAttribute(chunk_tc_keys_kernel<NC, WG, UNITS, D>,
+  return cudaFuncSetAttribute(chunk_tc_keys_kernel<NC, WG, UNITS, D, false>,
                               cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<NC, WG, UNITS, D>::kSmem);
 }
 
@@ -686,7 +750,22 @@ cudaError_t chunk_tc_keys_prepare() {
   if (e == cudaSuccess) e = prepare_cfg<32, 1, 6, 64>();
   if (e == cudaSuccess) e = prepare_cfg<32, 2, 8, 64>();
   if (e == cudaSuccess) e = prepare_cfg<32, 4, 8, 64>();
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(chunk_tc_keys_kernel<32, 1, 3, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Cfg<32, 1, 3, 128>::kSmem);
   return e;
+}
+
+// A list of chunks in one launch: up to 32 rows per kv-head at head dim 128 (two CTAs per SM).
+cudaError_t launch_chunk_tc_keys_hist(const ChunkParams& p, const HistParams& h, const CUtensorMap& any_map,
+                                      cudaStream_t s, bool pdl) {
+  if (h.n_chunks < 1 || h.n_chunks > kMaxHistChunksKeys || !h.maps || p.n_active || p.page_table || p.d != 128 ||
+      p.rows_per_tile > 32)
+    return cudaErrorInvalidValue;
+  using C = Cfg<32, 1, 3, 128>;
+  dim3 grid(p.splits * p.row_tiles, p.H_kv, p.B), block(C::kThreads);
+  // (the K/V map parameters are not used by this instantiation: any valid map will do)
+  return launch_kernel(chunk_tc_keys_kernel<32, 1, 3, 128, true>, grid, block, C::kSmem, s, pdl, p, any_map, any_map, h);
 }
 
 // Rows per CTA (p.rows_per_tile): <= 32 -> two CTAs per SM with 4 softmax warps; <= 64 and

@@ -901,15 +901,18 @@ def test_whole_round_in_one_call_large_and_errors():
     ctx.close()
 
 
-@pytest.mark.parametrize("d,T_q,H_q,H_kv", [(128, 40, 8, 2), (128, 24, 16, 2), (64, 40, 8, 2), (128, 64, 10, 2)])
+@pytest.mark.parametrize("d,T_q,H_q,H_kv", [(128, 40, 8, 2), (128, 24, 16, 2), (64, 40, 8, 2), (128, 64, 10, 2),
+                                             (128, 8, 8, 2), (128, 3, 4, 4)])
 def test_chunk_list_in_one_launch(d, T_q, H_q, H_kv, monkeypatch):
-    """ss_verify_chunks with more than 128 rows per kv-head: the whole list of chunks goes out as
-    one launch whose CTAs walk tiles across chunk boundaries.  Checked against the oracle with the
-    list in history order and reversed (the ragged chunk and the empty ones then come first and a
-    partly filled chunk sits in the middle of a CTA's walk), against the separate calls, and for
-    bit-identical repeats."""
+    """ss_verify_chunks where the whole list of chunks goes out as one launch whose CTAs walk tiles
+    across chunk boundaries: more than 128 rows per kv-head (rows-on-M kernel) and up to 32 rows
+    (keys-on-M kernel).  Checked against the oracle with the list in history order and reversed
+    (the ragged chunk and the empty ones then come first and a partly filled chunk sits in the
+    middle of a CTA's walk), against the separate calls, and for bit-identical repeats."""
     from paper_2609_33184_b200 import binding as ssb
-    if d == 64:   # routed at head dim 128 only (where it is faster); the launch itself takes both
+    keys = T_q * (H_q // H_kv) <= 32
+    one, each = ("tcgen05-keys-round", "tcgen05-keys") if keys else ("tcgen05-round", "tcgen05")
+    if d == 64 or keys:   # routed at head dim 128 / for equally long histories only; the launch takes these too
         monkeypatch.setenv("SS_HISTORY_LAUNCH", "always")
     cfg = inputs.VerifyConfig("hist", 0xb7 + d + T_q, 4, H_q, H_kv, d, 512, T_q, 0, 3000)
     lens = [3000, 1, 1537, 0]     # ragged, a single token, one token past a chunk boundary, nothing
@@ -917,7 +920,7 @@ def test_chunk_list_in_one_launch(d, T_q, H_q, H_kv, monkeypatch):
     assert len(chunks) == 6
     ctx = util.make_ctx(cfg, flags=ssb.SS_FLAG_OVERLAP_CHUNKS)
     O5, L5 = util.gpu_case(ctx, cfg, Q, chunks, K_loc, V_loc, bits)
-    assert ctx.last_chunk_kernel() == "tcgen05"
+    assert ctx.last_chunk_kernel() == each
     ref = util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits)
     util.compare(cfg, O5, L5, ref)
     outs = []
@@ -931,7 +934,7 @@ def test_chunk_list_in_one_launch(d, T_q, H_q, H_kv, monkeypatch):
             ctx.ss_verify_local(K_loc, V_loc, ssb.SS_MASK_CHAIN, None)
             ctx.ss_verify_finalize(O, LSE)
             torch.cuda.synchronize()
-            assert ctx.last_chunk_kernel() == "tcgen05-round"
+            assert ctx.last_chunk_kernel() == one
             assert ctx.ss_poll_status() == (0, 0)
             if rep == 0:
                 O0, L0 = O.clone(), LSE.clone()
@@ -943,7 +946,7 @@ def test_chunk_list_in_one_launch(d, T_q, H_q, H_kv, monkeypatch):
     O, LSE = torch.empty_like(O5), torch.empty_like(L5)
     ctx.ss_verify_round(Q, cfg.scale, chunks, K_loc, V_loc, ssb.SS_MASK_CHAIN, None, O, LSE)
     torch.cuda.synchronize()
-    assert ctx.last_chunk_kernel() == "tcgen05-round"
+    assert ctx.last_chunk_kernel() == one
     assert torch.equal(O.view(torch.int16), outs[0].view(torch.int16))
     # a bad valid length is flagged and clamped; a chunk beyond the context's size is refused and
     # leaves the round open
