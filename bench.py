@@ -369,7 +369,7 @@ def chunk_roofline(w, n_rounds):
         w.round(i, ev_pair=p)
     torch.cuda.synchronize()
     kernel = w.ctx.last_chunk_kernel()
-    if kernel == "tcgen05-round":   # the whole list of chunks went out as one launch
+    if kernel in ("tcgen05-round", "tcgen05-keys-round"):   # the whole list of chunks went out as one launch
         n_calls = 1
     chunk_ms = statistics.mean(a.elapsed_time(b) for a, b in pairs) / n_calls
     peak, peak_kind = peaks()
