@@ -171,12 +171,18 @@ ss_status ss_verify_chunk_paged(ss_ctx* ctx, ss_tensor K_pool, ss_tensor V_pool,
 /* a2, several chunks with one call (Section 4.2: the chunks of a request are reduced into one
  * running state; Eq. 13-14).  chunks is a HOST array of n_chunks (>= 0) descriptors, read before
  * the call returns; the result is that of one ss_verify_chunk_hinted per descriptor, in order.
- * Where the rows-on-M tensor-core kernel would take every chunk (head dim 128, more than
- * 128 query rows per kv-head, 2 to 32 contiguous chunks, one CTA per (request, kv-head, row tile)
- * fitting the GPU at once; SS_HISTORY_LAUNCH=never|always in the environment overrides the routing) the whole list takes ONE launch: a CTA walks an equal share of its
- * request's 64-token tiles across the chunk boundaries with one accumulator, so the list leaves
- * a few partial states per row instead of one per chunk and its CTAs are equally long
- * ("tcgen05-round" in ss_last_chunk_kernel).  Otherwise the chunks are enqueued one by one.
+ * Where one tensor-core kernel would take every chunk and one CTA per (request, kv-head, row
+ * tile) fits the GPU at once, the whole list takes ONE launch: a CTA walks an equal share of its
+ * request's tiles across the chunk boundaries with one accumulator, so the list leaves a few
+ * partial states per row instead of one per chunk, and set-up and write-out are paid once per
+ * request instead of once per chunk.  This is done at head dim 128 for more than 128 query rows
+ * per kv-head (rows-on-M kernel, 2 to 32 contiguous chunks: "tcgen05-round" in
+ * ss_last_chunk_kernel) and for up to 32 rows per kv-head (keys-on-M kernel, 2 to 16 contiguous
+ * chunks of at least 128 tokens, when the requests' histories are known to be equally long - no
+ * valid_len at all, or valid_len_host for every chunk with totals within 10 % of each other:
+ * "tcgen05-keys-round").  SS_HISTORY_LAUNCH=never|always in the environment overrides the
+ * routing.  Otherwise the chunks are enqueued one by one.  The results agree with separate calls
+ * up to the order of the fp32 sums (one launch merges per split, separate calls per chunk).
  * SS_ERR_STATE outside an open round; an error leaves the round open (ss_verify_abort ends it). */
 typedef struct {
   ss_tensor K, V;                 /* [B, H_kv, L_c, d] bf16, device                          */
@@ -527,9 +533,10 @@ typedef struct {
 ss_status ss_get_stats(ss_ctx* ctx, ss_stats* out);
 /* Number of kernels this context has launched since creation. */
 int64_t ss_launch_count(ss_ctx* ctx);
-/* "simt", "tcgen05" (rows on M), "tcgen05-keys" (keys on M), "tcgen05-round" (rows on M, a list
- * of chunks in one launch) or "simt-round" (a small round in one launch): the chunk kernel the
- * last chunk call, ss_verify_chunks or ss_verify_round used; "none" before. */
+/* "simt", "tcgen05" (rows on M), "tcgen05-keys" (keys on M), "tcgen05-round" / "tcgen05-keys-round"
+ * (the same two over a list of chunks in one launch) or "simt-round" (a small round in one
+ * launch): the chunk kernel the last chunk call, ss_verify_chunks or ss_verify_round used;
+ * "none" before. */
 const char* ss_last_chunk_kernel(ss_ctx* ctx);
 
 #ifdef __cplusplus
