@@ -763,29 +763,33 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
   // and successive launches keep it full; the one launch pays off where the tile's arithmetic
   // bounds the kernel (measured at head dim 128: +5 % at 192 rows, +22 % at 256, +8-13 % on the
   // 320-row tree workload, -4 % at 48; at head dim 64: -3 % at 192 rows, 0 at 320).
-  // The keys-on-M kernel (up to 32 rows per kv-head) runs at the HBM ceiling, and a CTA that walks
-  // 32,768 tokens instead of one chunk call's 2,048 pays set-up, ring fill and drain once instead
-  // of sixteen times (measured on the Qwen3-8B-shaped workload: +5 %); taken when the requests'
-  // histories are known to be about equally long (the CTAs of one launch should end together):
-  // no lengths at all, or a host copy of the lengths whose totals differ by at most 10 %.
+  // What the host knows about the requests' history lengths: every chunk without lengths or with a
+  // host copy of them -> the totals; otherwise unknown.
   const int row_tiles = (R + 127) / 128;
-  if (keys_on_m) {
-    if (c->cfg.d != 128 || R > 32 || n_chunks > 16) return SS_OK;
-    bool ragged = false;
-    int64_t lo = INT64_MAX, hi = 0;
-    for (int b = 0; b < c->B && !ragged; ++b) {
-      int64_t len = 0;
-      for (int j = 0; j < n_chunks; ++j) {
-        const ss_chunk_desc& d = chunks[j];
-        if (!d.valid_len) len += d.L_c;
-        else if (d.valid_len_host) len += d.valid_len_host[b] < 0 ? 0 : (d.valid_len_host[b] > d.L_c ? d.L_c : d.valid_len_host[b]);
-        else ragged = true;  // unknown to the host
-      }
-      lo = len < lo ? len : lo;
-      hi = len > hi ? len : hi;
+  bool known = c->B <= ss::kMaxListed;
+  int64_t len[ss::kMaxListed], lo = INT64_MAX, hi = 0;
+  for (int b = 0; b < c->B && known; ++b) {
+    len[b] = 0;
+    for (int j = 0; j < n_chunks && known; ++j) {
+      const ss_chunk_desc& d = chunks[j];
+      if (!d.valid_len) len[b] += d.L_c;
+      else if (d.valid_len_host) len[b] += d.valid_len_host[b] < 0 ? 0 : (d.valid_len_host[b] > d.L_c ? d.L_c : d.valid_len_host[b]);
+      else known = false;
     }
-    ragged = ragged || hi > lo + lo / 10;
-    if (ragged && !always) return SS_OK;
+    lo = len[b] < lo ? len[b] : lo;
+    hi = len[b] > hi ? len[b] : hi;
+  }
+  const bool uniform = known && hi <= lo + lo / 10;
+  // The keys-on-M kernel (up to 32 rows per kv-head) runs at the HBM ceiling, and a CTA that walks
+  // a request's whole history instead of one chunk call's 2,048 tokens pays set-up, ring fill and
+  // drain once instead of sixteen times (measured on the Qwen3-8B-shaped workload: +9 %).  The CTAs
+  // of the launch should end together, so the host has to know that the histories are about equally
+  // long.  (Ragged batches cut into pieces of equal length, a request-dependent number of them in
+  // two or three waves of CTAs, were measured too: 6.0-6.4 TB/s against 6.2-6.6 with one launch per
+  // chunk, whose hinted grids re-balance at every chunk; not kept.)
+  if (keys_on_m) {
+    if (c->cfg.d != 128 || R > 32) return SS_OK;
+    if (!uniform && !always) return SS_OK;
   } else if (!always && (row_tiles < 2 || c->cfg.d != 128)) {
     return SS_OK;
   }
@@ -801,18 +805,21 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
     tiles += (d.L_c + kTileKeys - 1) / kTileKeys;
     if (keys_on_m && d.L_c < 128) return SS_OK;   // (a box of 128 tokens)
   }
-  if (tiles > 0x3fffffff) return SS_OK;
-  int splits = (int)(wave / units);
-  if (splits > kMaxSplits) splits = kMaxSplits;
-  if (splits > c->slots_per_set / pairs) splits = c->slots_per_set / pairs;
-  if (splits > tiles / 8) splits = (int)(tiles / 8);               // at least eight tiles per CTA
-  if (c->force_splits > 0 && c->force_splits < splits) splits = c->force_splits;
-  if (splits < 1) splits = 1;
-
+  if (tiles > 0x3fffffff || (keys_on_m && tiles / 2 > 65000)) return SS_OK;   // (the keys kernel's 16-bit tile table)
   if (c->n_sets == c->n_set_cap) {  // every partial set is in use: fold them into one first
     cudaError_t e = fold_sets(c, c->stream);
     if (e != cudaSuccess) return cuda_fail(c, e);
   }
+  // the launch's partial states may take the room of several sets (they are contiguous): the
+  // highest split number it may use
+  int64_t split_cap = (int64_t)(c->n_set_cap - c->n_sets) * c->slots_per_set / pairs;
+  if (split_cap > kMaxSplits) split_cap = kMaxSplits;
+  int splits = (int)(wave / units);
+  if (splits > split_cap) splits = (int)split_cap;
+  if (splits > tiles / 8) splits = (int)(tiles / 8);               // at least eight tiles per CTA
+  if (c->force_splits > 0 && c->force_splits < splits) splits = c->force_splits;
+  if (splits < 1) splits = 1;
+  const int sets_taken = (int)(((int64_t)splits * pairs + c->slots_per_set - 1) / c->slots_per_set);
   // the chunks' tensor maps, K and V alternating, in one of the workspace's lists
   CUtensorMap maps[2 * ss::kMaxHistChunks];
   for (int j = 0; j < n_chunks; ++j)
@@ -890,9 +897,11 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
   ++c->launches;
   c->stats.chunk_calls += n_chunks;
   c->stats.kv_bytes += tokens * c->cfg.H_kv * c->cfg.d * 4;
-  c->splits[c->n_sets] = (uint8_t)splits;
-  memset(c->absent[c->n_sets], 0, sizeof(c->absent[0]));
-  ++c->n_sets;
+  for (int k = 0; k < sets_taken; ++k) {  // (the sets whose room the launch's states run into hold none of their own)
+    c->splits[c->n_sets] = k == 0 ? (uint8_t)splits : 0;
+    memset(c->absent[c->n_sets], 0, sizeof(c->absent[0]));
+    ++c->n_sets;
+  }
   c->first_launch = false;
   *taken = true;
   return SS_OK;

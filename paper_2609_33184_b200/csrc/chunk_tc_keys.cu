@@ -50,7 +50,7 @@ using namespace ss::tc;
 constexpr int kKeys = 128;                  // keys per tile = MMA M
 constexpr int kHalf = kKeys * 64 * 2;       // 16 KB: [128 keys][64 d] bf16, one TMA box
 constexpr float kLazyThreshold = 16.f;
-constexpr int kMaxHistChunksKeys = 16;      // chunks one launch over a list of chunks takes (table in the control block)
+constexpr int kMaxHistChunksKeys = kMaxHistChunks;   // chunks one launch over a list of chunks takes (table in the control block)
 
 template <int N>
 struct alignas(16) Ctl {
@@ -61,9 +61,10 @@ struct alignas(16) Ctl {
   volatile uint32_t flag[3];
   alignas(16) float nm_ref[N];    // NEGATED row references -m[r] (+inf = none yet); read as float4
   alignas(16) float smax[4][N];   // per lane quadrant
-  // launch over a list of chunks: 128-token tiles of the request before chunk j, its tokens in chunk j
-  int hist_prefix[kMaxHistChunksKeys + 1];
-  int hist_valid[kMaxHistChunksKeys];
+  // launch over a list of chunks: 128-token tiles of the request before chunk j (a request has
+  // fewer than 65,536 of them: checked by the host), valid tokens of chunk j's last tile (1..128)
+  uint16_t hist_prefix[kMaxHistChunksKeys + 1];
+  uint8_t hist_last[kMaxHistChunksKeys];
 };
 
 // NC = score columns per softmax thread, WG = softmax warpgroups (threads sharing a TMEM lane),
@@ -144,12 +145,12 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
         if (lane >= o) incl += up;
       }
       if (lane < h.n_chunks) {
-        ctl->hist_prefix[lane + 1] = incl;
-        ctl->hist_valid[lane] = v;
+        ctl->hist_prefix[lane + 1] = (uint16_t)incl;
+        ctl->hist_last[lane] = (uint8_t)(v ? v - (v - 1) / kKeys * kKeys : 0);
       }
       if (lane == 0) ctl->hist_prefix[0] = 0;
       const int total = __shfl_sync(0xffffffffu, incl, 31);
-      if (lane >= h.n_chunks && lane < kMaxHistChunksKeys) ctl->hist_prefix[lane + 1] = total;
+      if (lane >= h.n_chunks && lane < kMaxHistChunksKeys) ctl->hist_prefix[lane + 1] = (uint16_t)total;
     }
     __syncthreads();
     const int total = ctl->hist_prefix[h.n_chunks];
@@ -461,7 +462,7 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
       if (HIST) {
         int tok;
         const int c = hist_locate(t, soft_chunk, &tok);
-        n_valid = min(kKeys, ctl->hist_valid[c] - tok);
+        n_valid = (g0 + t + 1 == ctl->hist_prefix[c + 1]) ? ctl->hist_last[c] : kKeys;   // the chunk's last tile?
       } else {
         n_valid = min(kKeys, tok1 - (tok0 + t * kKeys));
       }

@@ -166,7 +166,8 @@ cudaError_t chunk_simt_prepare();    // one-time function attributes
 int simt_rows_per_tile(int R);       // rows per CTA tile of the CUDA-core chunk kernel
 cudaError_t launch_chunk_tc(const ChunkParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
                             const CUtensorMap& tmA, cudaStream_t s, bool pdl);
-// The keys-on-M kernel over a list of at most 16 chunks (head dim 128, up to 32 rows per kv-head).
+// The keys-on-M kernel over a list of chunks (head dim 128, up to 32 rows per kv-head, fewer than
+// 65,536 tiles of 128 tokens per request).
 cudaError_t launch_chunk_tc_keys_hist(const ChunkParams& p, const HistParams& h, const CUtensorMap& any_map,
                                       cudaStream_t s, bool pdl);
 // The same kernel over a list of chunks (HistParams); p.splits = CTAs per (request, kv-head, row tile).

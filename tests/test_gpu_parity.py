@@ -924,9 +924,13 @@ def test_chunk_list_in_one_launch(d, T_q, H_q, H_kv, monkeypatch):
     ref = util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits)
     util.compare(cfg, O5, L5, ref)
     outs = []
-    for order in (list(range(6)), list(range(5, -1, -1)), [2, 5, 0, 3, 1, 4]):
+    import ctypes as C
+    for order, with_host_lengths in ((list(range(6)), False), (list(range(5, -1, -1)), True), ([2, 5, 0, 3, 1, 4], True)):
         lst = [chunks[j] for j in order]
-        descs = ctx.chunk_descs([lst])
+        # with the host's copy of the lengths a ragged batch is cut into pieces of about equal length
+        # (a request-dependent number of them); without, every request into equally many pieces
+        hints = [(C.c_int32 * cfg.B)(*vl.tolist()) for (_, _, vl) in lst] if with_host_lengths else None
+        descs = ctx.chunk_descs([lst], hints)
         O, LSE = torch.empty_like(O5), torch.empty_like(L5)
         for rep in range(3):
             ctx.ss_verify_begin(Q, cfg.scale)
