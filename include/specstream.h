@@ -177,7 +177,7 @@ ss_status ss_verify_chunk_paged(ss_ctx* ctx, ss_tensor K_pool, ss_tensor V_pool,
  * partial states per row instead of one per chunk, and set-up and write-out are paid once per
  * request instead of once per chunk.  This is done at head dim 128 for more than 128 query rows
  * per kv-head (rows-on-M kernel, 2 to 32 contiguous chunks: "tcgen05-round" in
- * ss_last_chunk_kernel) and for up to 32 rows per kv-head (keys-on-M kernel, 2 to 32 contiguous
+ * ss_last_chunk_kernel) and for up to 32 rows per kv-head (16 at head dim 64; keys-on-M kernel, 2 to 32 contiguous
  * chunks of at least 128 tokens, when the requests' histories are known to be equally long - no
  * valid_len at all, or valid_len_host for every chunk with totals within 10 % of each other:
  * "tcgen05-keys-round").  SS_HISTORY_LAUNCH=never|always in the environment overrides the

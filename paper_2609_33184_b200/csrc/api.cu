@@ -788,7 +788,7 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
   // two or three waves of CTAs, were measured too: 6.0-6.4 TB/s against 6.2-6.6 with one launch per
   // chunk, whose hinted grids re-balance at every chunk; not kept.)
   if (keys_on_m) {
-    if (c->cfg.d != 128 || R > 32) return SS_OK;
+    if (R > 32) return SS_OK;
     if (!uniform && !always) return SS_OK;
   } else if (!always && (row_tiles < 2 || c->cfg.d != 128)) {
     return SS_OK;

@@ -754,18 +754,26 @@ cudaError_t chunk_tc_keys_prepare() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(chunk_tc_keys_kernel<32, 1, 3, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              Cfg<32, 1, 3, 128>::kSmem);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(chunk_tc_keys_kernel<32, 1, 6, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Cfg<32, 1, 6, 64>::kSmem);
   return e;
 }
 
-// A list of chunks in one launch: up to 32 rows per kv-head at head dim 128 (two CTAs per SM).
+// A list of chunks in one launch: up to 32 rows per kv-head (two CTAs per SM).
 cudaError_t launch_chunk_tc_keys_hist(const ChunkParams& p, const HistParams& h, const CUtensorMap& any_map,
                                       cudaStream_t s, bool pdl) {
-  if (h.n_chunks < 1 || h.n_chunks > kMaxHistChunksKeys || !h.maps || p.n_active || p.page_table || p.d != 128 ||
+  if (h.n_chunks < 1 || h.n_chunks > kMaxHistChunksKeys || !h.maps || p.n_active || p.page_table ||
       p.rows_per_tile > 32)
     return cudaErrorInvalidValue;
+  // (the K/V map parameters are not used by these instantiations: any valid map will do)
+  if (p.d == 64) {
+    using C = Cfg<32, 1, 6, 64>;
+    dim3 grid(p.splits * p.row_tiles, p.H_kv, p.B), block(C::kThreads);
+    return launch_kernel(chunk_tc_keys_kernel<32, 1, 6, 64, true>, grid, block, C::kSmem, s, pdl, p, any_map, any_map, h);
+  }
   using C = Cfg<32, 1, 3, 128>;
   dim3 grid(p.splits * p.row_tiles, p.H_kv, p.B), block(C::kThreads);
-  // (the K/V map parameters are not used by this instantiation: any valid map will do)
   return launch_kernel(chunk_tc_keys_kernel<32, 1, 3, 128, true>, grid, block, C::kSmem, s, pdl, p, any_map, any_map, h);
 }
 

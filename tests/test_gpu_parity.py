@@ -902,7 +902,7 @@ def test_whole_round_in_one_call_large_and_errors():
 
 
 @pytest.mark.parametrize("d,T_q,H_q,H_kv", [(128, 40, 8, 2), (128, 24, 16, 2), (64, 40, 8, 2), (128, 64, 10, 2),
-                                             (128, 8, 8, 2), (128, 3, 4, 4)])
+                                             (128, 8, 8, 2), (128, 3, 4, 4), (64, 4, 8, 2)])
 def test_chunk_list_in_one_launch(d, T_q, H_q, H_kv, monkeypatch):
     """ss_verify_chunks where the whole list of chunks goes out as one launch whose CTAs walk tiles
     across chunk boundaries: more than 128 rows per kv-head (rows-on-M kernel) and up to 32 rows
@@ -910,7 +910,7 @@ def test_chunk_list_in_one_launch(d, T_q, H_q, H_kv, monkeypatch):
     (the ragged chunk and the empty ones then come first and a partly filled chunk sits in the
     middle of a CTA's walk), against the separate calls, and for bit-identical repeats."""
     from paper_2609_33184_b200 import binding as ssb
-    keys = T_q * (H_q // H_kv) <= 32
+    keys = T_q * (H_q // H_kv) <= (32 if d == 128 else 16)
     one, each = ("tcgen05-keys-round", "tcgen05-keys") if keys else ("tcgen05-round", "tcgen05")
     if d == 64 or keys:   # routed at head dim 128 / for equally long histories only; the launch takes these too
         monkeypatch.setenv("SS_HISTORY_LAUNCH", "always")
