@@ -107,7 +107,9 @@ typedef struct {
  *   SS_CHUNK_KERNEL=rows|keys  as SS_FLAG_ROWS_ON_M / SS_FLAG_KEYS_ON_M
  *   SS_SPLITS=n                token splits of every chunk call (default: sized so that a
  *                              call launches about one CTA per SM)
- *   SS_TARGET_CTAS=n           the CTA count the automatic split choice aims at */
+ *   SS_TARGET_CTAS=n           the CTA count the automatic split choice aims at
+ * and, read at every ss_verify_chunks call:
+ *   SS_HISTORY_LAUNCH=never|always  never / wherever possible take a list of chunks in one launch */
 
 typedef struct {
   const void* ptr;                      /* device pointer, bf16                      */
