@@ -1,5 +1,5 @@
-"""The five workloads at their full sizes, in the launch configuration bench.py times
-(overlapped chunk kernels, host length hints), checked on whole (request, kv-head) groups: every
+"""The five workloads at their full sizes, in the launch configurations bench.py times
+(overlapped chunk kernels, host length hints, a round's chunks with one call or one by one), checked on whole (request, kv-head) groups: every
 query row of the group, all head dims and the LSE, against the oracle.  A whole group covers
 every row tile, replica and token split the full-size launch uses for that kv-head."""
 import random
@@ -46,7 +46,10 @@ def _assert_contract(cfg, O, LSE, ref):
         assert np.abs(Lg[b, kvh * G:(kvh + 1) * G] - Lr).max() <= 1e-3, (b, kvh)
 
 
-def _resident(name, n_random):
+def _resident(name, n_random, one_call=True, kernel=None):
+    """one_call: the round's chunks go in with one ss_verify_chunks call and the host's copy of the
+    lengths, as bench.py does by default (one launch for the whole list where the library takes
+    it); False: one call per chunk (bench.py --chunk-calls separate)."""
     from paper_2609_33184_b200 import binding as ssb
     cfg = inputs.CONFIGS[name]
     lens = inputs.history_lengths(cfg)
@@ -55,10 +58,13 @@ def _resident(name, n_random):
                       flags=ssb.SS_FLAG_OVERLAP_CHUNKS)
     O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
     LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
-    hints = harness.host_valid(cfg, lens, len(chunks)) if len(set(lens)) > 1 else None   # as bench.py does
+    hints = harness.host_valid(cfg, lens, len(chunks))   # as bench.py does
+    descs = ctx.chunk_descs([chunks], hints) if one_call else None
     for _ in range(2):
-        harness.run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, hints=hints)
+        harness.run_round(ctx, ssb, cfg, Q, chunks, K_loc, V_loc, bits, O, LSE, hints=hints, descs=descs)
     torch.cuda.synchronize()
+    if kernel:
+        assert ctx.last_chunk_kernel() == kernel, ctx.last_chunk_kernel()
     st, dev_bits = ctx.ss_poll_status()
     assert st == 0, dev_bits
     assert torch.isfinite(O.float()).all() and torch.isfinite(LSE).all()
@@ -71,16 +77,25 @@ def _resident(name, n_random):
 
 
 def test_c2_qwen3_8b_full():
-    _resident("c2_qwen3_8b", 2)
+    _resident("c2_qwen3_8b", 2, kernel="tcgen05-keys-round")
+
+
+def test_c2_qwen3_8b_full_one_call_per_chunk():
+    _resident("c2_qwen3_8b", 2, one_call=False, kernel="tcgen05-keys")
 
 
 def test_c3_internlm25_7b_ragged_full():
-    _resident("c3_internlm25_7b_ragged", 1)
+    _resident("c3_internlm25_7b_ragged", 1, kernel="tcgen05-keys")   # ragged: one launch per chunk
 
 
 def test_c4_tree_full():
-    # 320 rows per group: all three row tiles of a kv-head, the 64-row remainder tile included
-    _resident("c4_tree", 0)
+    # 320 rows per group: all three row tiles of a kv-head, the 64-row remainder tile included;
+    # the whole list of chunks in one launch (three token splits per row tile)
+    _resident("c4_tree", 0, kernel="tcgen05-round")
+
+
+def test_c4_tree_full_one_call_per_chunk():
+    _resident("c4_tree", 0, one_call=False, kernel="tcgen05")
 
 
 def test_c5_streamed_full():
