@@ -177,12 +177,13 @@ ss_status ss_verify_chunk_paged(ss_ctx* ctx, ss_tensor K_pool, ss_tensor V_pool,
  * tile) fits the GPU at once, the whole list takes ONE launch: a CTA walks an equal share of its
  * request's tiles across the chunk boundaries with one accumulator, so the list leaves a few
  * partial states per row instead of one per chunk, and set-up and write-out are paid once per
- * request instead of once per chunk.  This is done at head dim 128 for more than 128 query rows
- * per kv-head (rows-on-M kernel, 2 to 32 contiguous chunks: "tcgen05-round" in
- * ss_last_chunk_kernel) and for up to 32 rows per kv-head (16 at head dim 64; keys-on-M kernel, 2 to 32 contiguous
- * chunks of at least 128 tokens, when the requests' histories are known to be equally long - no
- * valid_len at all, or valid_len_host for every chunk with totals within 10 % of each other:
- * "tcgen05-keys-round").  SS_HISTORY_LAUNCH=never|always in the environment overrides the
+ * request instead of once per chunk.  This is done (2 to 32 contiguous chunks) when the host
+ * knows the requests' histories to be equally long - no valid_len at all, or valid_len_host for
+ * every chunk with totals within 10 % of each other - for up to 32 rows per kv-head (16 at head
+ * dim 64; keys-on-M kernel, chunks of at least 128 tokens: "tcgen05-keys-round" in
+ * ss_last_chunk_kernel) and for more rows up to 128 (rows-on-M kernel: "tcgen05-round"); and at
+ * head dim 128 for more than 128 rows per kv-head unless the host knows the batch to be ragged
+ * ("tcgen05-round").  SS_HISTORY_LAUNCH=never|always in the environment overrides the
  * routing.  Otherwise the chunks are enqueued one by one.  The results agree with separate calls
  * up to the order of the fp32 sums (one launch merges per split, separate calls per chunk).
  * SS_ERR_STATE outside an open round; an error leaves the round open (ss_verify_abort ends it). */

@@ -759,10 +759,6 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
   const int R = c->T_q * c->G, pairs = c->B * c->cfg.H_kv;
   const int keys_max_rows = c->cfg.d == 64 ? 16 : 32;
   const bool keys_on_m = !c->force_rows_kernel && (R <= keys_max_rows || c->force_keys_kernel);
-  // With up to 128 rows per kv-head the chunk kernels run at the HBM ceiling while the GPU is full
-  // and successive launches keep it full; the one launch pays off where the tile's arithmetic
-  // bounds the kernel (measured at head dim 128: +5 % at 192 rows, +22 % at 256, +8-13 % on the
-  // 320-row tree workload, -4 % at 48; at head dim 64: -3 % at 192 rows, 0 at 320).
   // What the host knows about the requests' history lengths: every chunk without lengths or with a
   // host copy of them -> the totals; otherwise unknown.
   const int row_tiles = (R + 127) / 128;
@@ -787,11 +783,18 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
   // long.  (Ragged batches cut into pieces of equal length, a request-dependent number of them in
   // two or three waves of CTAs, were measured too: 6.0-6.4 TB/s against 6.2-6.6 with one launch per
   // chunk, whose hinted grids re-balance at every chunk; not kept.)
+  // The rows-on-M kernel: with more than 128 rows per kv-head at head dim 128 the tile's arithmetic
+  // bounds it and the one launch pays off whatever the host knows (+5 % at 192 rows, +22 % at 256,
+  // +8-13 % on the 320-row tree workload), unless it knows the batch to be ragged; with up to 128
+  // rows it is taken for histories known to be equally long (B = 16, 16,384 tokens each, head dim
+  // 128: +3 / +4 / +7 / +12 % at 48 / 64 / 96 / 128 rows; head dim 64: +12-15 % at 24-64 rows, +7-10 %
+  // at 96-128; -2 % / +1 % at 192 / 320 rows, where it is not taken).
   if (keys_on_m) {
     if (R > 32) return SS_OK;
     if (!uniform && !always) return SS_OK;
-  } else if (!always && (row_tiles < 2 || c->cfg.d != 128)) {
-    return SS_OK;
+  } else if (!always) {
+    if (known && !uniform) return SS_OK;
+    if (row_tiles >= 2 ? c->cfg.d != 128 : !uniform) return SS_OK;
   }
   const int64_t units = (int64_t)pairs * row_tiles;
   const int wave = 2 * ss::kNumSM;                                  // two CTAs per SM

@@ -912,8 +912,7 @@ def test_chunk_list_in_one_launch(d, T_q, H_q, H_kv, monkeypatch):
     from paper_2609_33184_b200 import binding as ssb
     keys = T_q * (H_q // H_kv) <= (32 if d == 128 else 16)
     one, each = ("tcgen05-keys-round", "tcgen05-keys") if keys else ("tcgen05-round", "tcgen05")
-    if d == 64 or keys:   # routed at head dim 128 / for equally long histories only; the launch takes these too
-        monkeypatch.setenv("SS_HISTORY_LAUNCH", "always")
+    monkeypatch.setenv("SS_HISTORY_LAUNCH", "always")   # (the routing has a test of its own; these lengths are ragged)
     cfg = inputs.VerifyConfig("hist", 0xb7 + d + T_q, 4, H_q, H_kv, d, 512, T_q, 0, 3000)
     lens = [3000, 1, 1537, 0]     # ragged, a single token, one token past a chunk boundary, nothing
     Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
@@ -1000,3 +999,36 @@ def test_two_chunk_calls_with_max_chunks_one():
     segment's partial set."""
     cfg = inputs.VerifyConfig("v", 0x59, 2, 8, 2, 128, 256, 8, 600, 700)
     _run(cfg, max_chunks=1)
+
+
+def test_chunk_list_routing():
+    """Which lists go out as one launch: histories the host knows to be equally long at any row
+    count; more than 128 rows per kv-head at head dim 128 also when it knows nothing; never a batch
+    it knows to be ragged, nor a history of a few tiles."""
+    import ctypes as C
+    from paper_2609_33184_b200 import binding as ssb
+
+    def kernel_for(d, T_q, H_q, H_kv, lens, host_lengths, L_c=512):
+        cfg = inputs.VerifyConfig("route", 0xd1 + T_q, len(lens), H_q, H_kv, d, L_c, T_q, 0, max(lens))
+        Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV, fill=0.0)
+        ctx = util.make_ctx(cfg, flags=ssb.SS_FLAG_OVERLAP_CHUNKS)
+        hints = [(C.c_int32 * cfg.B)(*vl.tolist()) for (_, _, vl) in chunks] if host_lengths else None
+        ctx.ss_verify_begin(Q, cfg.scale)
+        ctx.ss_verify_chunks(ctx.chunk_descs([chunks], hints), len(chunks))
+        ctx.ss_verify_abort()
+        torch.cuda.synchronize()
+        k = ctx.last_chunk_kernel()
+        ctx.close()
+        return k
+
+    even, ragged = [4096, 4096, 4000], [4096, 1000, 2500]
+    assert kernel_for(128, 8, 8, 2, even, True) == "tcgen05-keys-round"      # 32 rows, known equal
+    assert kernel_for(128, 8, 8, 2, even, False) == "tcgen05-keys"           # lengths only on the device
+    assert kernel_for(128, 8, 8, 2, ragged, True) == "tcgen05-keys"
+    assert kernel_for(128, 8, 16, 2, even, True) == "tcgen05-round"          # 64 rows, known equal
+    assert kernel_for(128, 8, 16, 2, even, False) == "tcgen05"
+    assert kernel_for(64, 8, 16, 2, even, True) == "tcgen05-round"           # head dim 64, 64 rows
+    assert kernel_for(128, 40, 8, 2, even, False) == "tcgen05-round"         # 160 rows: whatever the host knows
+    assert kernel_for(128, 40, 8, 2, ragged, True) == "tcgen05"              # ... unless it knows the batch is ragged
+    assert kernel_for(64, 40, 8, 2, even, True) == "tcgen05"                 # head dim 64, 160 rows: not taken
+    assert kernel_for(128, 8, 8, 2, [300, 300], True, L_c=256) == "tcgen05-keys"   # a few tiles in all
