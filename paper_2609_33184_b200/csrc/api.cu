@@ -812,7 +812,7 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
   // a history of a few tiles per request is latency bound: the separate calls (CUDA-core kernel for
   // tiny ones) or the one-launch small round of ss_verify_round do better (measured on the
   // 1,024-token chain workload)
-  if (keys_on_m && tiles < 64 && !always) return SS_OK;
+  if (tiles < 64 && !always) return SS_OK;
   if (c->n_sets == c->n_set_cap) {  // every partial set is in use: fold them into one first
     cudaError_t e = fold_sets(c, c->stream);
     if (e != cudaSuccess) return cuda_fail(c, e);

@@ -970,10 +970,11 @@ def test_chunk_list_in_one_launch(d, T_q, H_q, H_kv, monkeypatch):
     ctx.close()
 
 
-def test_chunk_list_after_separate_chunks_with_one_partial_set():
+def test_chunk_list_after_separate_chunks_with_one_partial_set(monkeypatch):
     """A context with a single partial set: a chunk call, then a list of chunks in one launch (the
     set in use is folded first), then another chunk call; against the oracle."""
     from paper_2609_33184_b200 import binding as ssb
+    monkeypatch.setenv("SS_HISTORY_LAUNCH", "always")   # (a short list: not routed by itself)
     cfg = inputs.VerifyConfig("hist1", 0xc3, 2, 8, 2, 128, 512, 40, 0, 2500)
     lens = [2500, 900]
     Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
