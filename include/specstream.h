@@ -109,7 +109,8 @@ typedef struct {
  *                              call launches about one CTA per SM)
  *   SS_TARGET_CTAS=n           the CTA count the automatic split choice aims at
  * and, read at every ss_verify_chunks call:
- *   SS_HISTORY_LAUNCH=never|always  never / wherever possible take a list of chunks in one launch */
+ *   SS_HISTORY_LAUNCH=never|always  never / wherever possible take a list of chunks in one launch
+ *   SS_HISTORY_WALK=never           ragged batches do not take the one launch with shares across requests */
 
 typedef struct {
   const void* ptr;                      /* device pointer, bf16                      */
@@ -183,8 +184,15 @@ ss_status ss_verify_chunk_paged(ss_ctx* ctx, ss_tensor K_pool, ss_tensor V_pool,
  * dim 64; keys-on-M kernel, chunks of at least 128 tokens: "tcgen05-keys-round" in
  * ss_last_chunk_kernel) and for more rows up to 128 (rows-on-M kernel: "tcgen05-round"); and at
  * head dim 128 for more than 128 rows per kv-head unless the host knows the batch to be ragged
- * ("tcgen05-round").  SS_HISTORY_LAUNCH=never|always in the environment overrides the
- * routing.  Otherwise the chunks are enqueued one by one.  The results agree with separate calls
+ * ("tcgen05-round").  A batch the host knows to be ragged (valid_len_host for every chunk with
+ * lengths, no request empty) also takes one launch with up to 32 rows per kv-head (16 at head dim
+ * 64): the tiles of a kv-head's requests are laid end to end and every CTA takes an equal share,
+ * ending one request and beginning the next where its share says so; the shares are cut on the
+ * host's lengths and scaled to those on the device, so in this launch lengths that are out of
+ * date cost balance, not tokens (pass the device's values all the same: the separate calls drop
+ * tokens that the hint leaves out) ("tcgen05-keys-round"; SS_HISTORY_WALK=never turns this off).
+ * SS_HISTORY_LAUNCH=never|always in the environment overrides the routing.  Otherwise the
+ * chunks are enqueued one by one.  The results agree with separate calls
  * up to the order of the fp32 sums (one launch merges per split, separate calls per chunk).
  * SS_ERR_STATE outside an open round; an error leaves the round open (ss_verify_abort ends it). */
 typedef struct {

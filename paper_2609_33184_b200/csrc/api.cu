@@ -780,18 +780,24 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
   // a request's whole history instead of one chunk call's 2,048 tokens pays set-up, ring fill and
   // drain once instead of sixteen times (measured on the Qwen3-8B-shaped workload: +9 %).  The CTAs
   // of the launch should end together, so the host has to know that the histories are about equally
-  // long.  (Ragged batches cut into pieces of equal length, a request-dependent number of them in
-  // two or three waves of CTAs, were measured too: 6.0-6.4 TB/s against 6.2-6.6 with one launch per
-  // chunk, whose hinted grids re-balance at every chunk; not kept.)
+  // long.  A batch it knows to be ragged gets equally long CTAs another way (below): the tiles of a
+  // kv-head's requests are laid end to end and cut into one share per CTA, whatever request a share
+  // starts or ends in (streamed workload's batch, 8,192 to 65,536 tokens, resident: 6.39 -> 6.93 TB/s;
+  // per-request pieces of equal length in two or three waves of CTAs had measured 6.0-6.4).
   // The rows-on-M kernel: with more than 128 rows per kv-head at head dim 128 the tile's arithmetic
   // bounds it and the one launch pays off whatever the host knows (+5 % at 192 rows, +22 % at 256,
   // +8-13 % on the 320-row tree workload), unless it knows the batch to be ragged; with up to 128
   // rows it is taken for histories known to be equally long (B = 16, 16,384 tokens each, head dim
   // 128: +3 / +4 / +7 / +12 % at 48 / 64 / 96 / 128 rows; head dim 64: +12-15 % at 24-64 rows, +7-10 %
   // at 96-128; -2 % / +1 % at 192 / 320 rows, where it is not taken).
+  // Ragged batches on the keys-on-M kernel whose lengths the host knows (no request empty): the CTAs
+  // of a kv-head walk equal shares of all its requests' tiles laid end to end (HistParams::n_req).
+  // SS_HISTORY_WALK=never leaves such batches to the separate calls.
+  const char* wk = getenv("SS_HISTORY_WALK");
+  const bool walk = keys_on_m && R <= 32 && known && !uniform && lo > 0 && !(wk && strcmp(wk, "never") == 0);
   if (keys_on_m) {
     if (R > 32) return SS_OK;
-    if (!uniform && !always) return SS_OK;
+    if (!uniform && !always && !walk) return SS_OK;
   } else if (!always) {
     if (known && !uniform) return SS_OK;
     if (row_tiles >= 2 ? c->cfg.d != 128 : !uniform) return SS_OK;
@@ -826,6 +832,38 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
   if (splits > tiles / 8) splits = (int)(tiles / 8);               // at least eight tiles per CTA
   if (c->force_splits > 0 && c->force_splits < splits) splits = c->force_splits;
   if (splits < 1) splits = 1;
+  ss::HistParams h;
+  memset(&h, 0, sizeof(h));
+  if (walk) {
+    // 128-token tiles of each request by the host's lengths; the shares and the largest number of
+    // pieces a request is cut into (= partial states per row), with the kernel's own arithmetic
+    h.n_req = c->B;
+    for (int b = 0; b < c->B; ++b) {
+      int64_t t128 = 0;
+      for (int j = 0; j < n_chunks; ++j) {
+        const ss_chunk_desc& d = chunks[j];
+        int64_t v = d.valid_len ? d.valid_len_host[b] : d.L_c;
+        v = v < 0 ? 0 : (v > d.L_c ? d.L_c : v);
+        t128 += (v + 127) / 128;
+      }
+      h.req_prefix[b + 1] = h.req_prefix[b] + (int)t128;
+    }
+    const int64_t all = h.req_prefix[c->B];
+    int ctas = wave / c->cfg.H_kv;
+    if (ctas > all / 8) ctas = (int)(all / 8);                     // at least eight tiles per CTA
+    if (ctas < 1) ctas = 1;
+    h.walk_ctas = ctas;
+    int most = 1;
+    for (int b = 0; b < c->B; ++b) {
+      const int64_t p0 = h.req_prefix[b], p1 = h.req_prefix[b + 1];
+      int first = 0, last = ctas - 1;
+      while (all * (first + 1) / ctas <= p0) ++first;               // the first share that reaches past p0
+      while (last > first && all * last / ctas >= p1) --last;       // the last share that starts before p1
+      if (last - first + 1 > most) most = last - first + 1;
+    }
+    if (most > split_cap) return SS_OK;
+    splits = most;
+  }
   const int sets_taken = (int)(((int64_t)splits * pairs + c->slots_per_set - 1) / c->slots_per_set);
   // the chunks' tensor maps, K and V alternating, in one of the workspace's lists
   CUtensorMap maps[2 * ss::kMaxHistChunks];
@@ -854,8 +892,6 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
 
   ss::ChunkParams p;
   memset(&p, 0, sizeof(p));
-  ss::HistParams h;
-  memset(&h, 0, sizeof(h));
   h.n_chunks = n_chunks;
   h.maps = c->hist_maps + (size_t)slot * 2 * ss::kMaxHistChunks;
   int64_t tokens = 0;

@@ -95,9 +95,12 @@ struct Cfg {
 };
 
 
-// HIST: the launch covers a list of chunks (HistParams; see ss_internal.h): the CTA walks an equal
-// share of its request's 128-token tiles, counted chunk by chunk, with one accumulator.
-template <int NC, int WG, int UNITS, int D, bool HIST>
+// HIST = 1: the launch covers a list of chunks (HistParams; see ss_internal.h): the CTA walks an
+// equal share of its request's 128-token tiles, counted chunk by chunk, with one accumulator.
+// HIST = 2: the same for ragged batches: the CTAs of a kv-head walk equal shares of ALL its requests'
+// tiles laid end to end; a CTA runs the kernel's body once per request its share touches (a new Q
+// tile, a new accumulator, a partial state of its own), the barriers set up anew each time.
+template <int NC, int WG, int UNITS, int D, int HIST>
 __global__ void __launch_bounds__(Cfg<NC, WG, UNITS, D>::kThreads, Cfg<NC, WG, UNITS, D>::kMinBlocks)
 chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
                      const __grid_constant__ CUtensorMap tmV, const __grid_constant__ HistParams h) {
@@ -117,13 +120,52 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
   const unsigned long long t_cta0 = p.cta_log ? cta_log_now() : 0ull;
   if (p.wait_first) pdl_wait_prior();
   pdl_launch_dependents();
+  constexpr bool WALK = HIST == 2;
   const ChunkWork w = chunk_work(p, p.rows_per_tile);
-  const int b = w.b, kvh = w.kvh, row0 = w.row0, nrows = w.nrows, tok0 = w.tok0, tok1 = w.tok1;  // nrows <= N
+  const int kvh = w.kvh, row0 = w.row0, nrows = w.nrows, tok0 = w.tok0, tok1 = w.tok1;  // nrows <= N
   const bool chain_cta = w.chain_cta;
-  float2* out_ml = w.out_ml;
-  float* out_a = w.out_a;
   const int n_mma = (nrows + 15) & ~15;                 // MMA N of this CTA
   unsigned long long* tr = chain_cta ? p.trace : nullptr;
+  // (ragged batches) this CTA's share [share_lo, share_hi) of the kv-head's tiles by the host's lengths
+  long long share_lo = 0, share_hi = 0;
+  int req = w.b, req_end = w.b + 1;  // requests to run the body for: [req, req_end) as long as they overlap the share
+  if (WALK) {
+    const long long all = h.req_prefix[h.n_req];
+    share_lo = all * blockIdx.x / gridDim.x;
+    share_hi = all * (blockIdx.x + 1) / gridDim.x;
+    req = 0;
+    while (req < h.n_req && h.req_prefix[req + 1] <= share_lo) ++req;
+    req_end = h.n_req;
+  }
+  bool tmem_held = false;
+  int tiles_walked = 0;
+  uint32_t tmem = 0;
+  for (; req < req_end && (!WALK || h.req_prefix[req] < share_hi); ++req) {
+  const int b = req;
+  int piece = w.split;        // which of the request's partial states this pass writes
+  bool last_piece = false;    // (ragged batches) no CTA after this one has tiles of the request
+  long long hint_a = 0, hint_e = 0, hint_n = 1;
+  if (WALK) {
+    const long long p0 = h.req_prefix[b], p1 = h.req_prefix[b + 1];
+    hint_n = p1 - p0;
+    hint_a = (share_lo > p0 ? share_lo : p0) - p0;
+    hint_e = (share_hi < p1 ? share_hi : p1) - p0;
+    last_piece = share_hi >= p1;
+    int first = blockIdx.x;   // the first CTA of the kv-head whose share reaches into this request
+    const long long all = h.req_prefix[h.n_req];
+    while (first > 0 && all * first / gridDim.x > p0) --first;
+    piece = blockIdx.x - first;
+  }
+  auto state_ml = [&](int k) {  // (m, l) rows of the request's partial state number k
+    return p.part_ml + (((size_t)k * p.B + b) * p.H_kv + kvh) * p.R_stride + row0;
+  };
+  float2* out_ml = WALK ? state_ml(piece) : w.out_ml;
+  float* out_a = WALK ? p.part_a + ((((size_t)piece * p.B + b) * p.H_kv + kvh) * p.R_stride + row0) * p.d : w.out_a;
+  // the states nobody computes (the request has fewer pieces than the launch has splits) are the identity
+  auto fill_unused = [&]() {
+    if (WALK && last_piece && tid < nrows)
+      for (int k = piece + 1; k < p.splits; ++k) state_ml(k)[tid] = make_float2(-INFINITY, 0.f);
+  };
   // splits are given in 64-token tiles by the host; this kernel walks 128-token tiles
   int n_tiles = (tok1 > tok0) ? (tok1 - tok0 + kKeys - 1) / kKeys : 0;
   int g0 = 0;  // (list of chunks) the CTA's first tile in the request's numbering
@@ -154,8 +196,13 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
     }
     __syncthreads();
     const int total = ctl->hist_prefix[h.n_chunks];
-    g0 = (int)((int64_t)total * w.split / p.splits);
-    n_tiles = (int)((int64_t)total * (w.split + 1) / p.splits) - g0;
+    if (WALK) {  // the share of the request by the host's lengths, scaled to the tiles it really has
+      g0 = (int)((long long)total * hint_a / hint_n);
+      n_tiles = (int)((long long)total * hint_e / hint_n) - g0;
+    } else {
+      g0 = (int)((int64_t)total * w.split / p.splits);
+      n_tiles = (int)((int64_t)total * (w.split + 1) / p.splits) - g0;
+    }
   }
   // (list of chunks) chunk of the CTA's tile t and the tile's first token in it; tiles are asked
   // for in ascending order, `cur` is the caller's own cursor
@@ -171,6 +218,11 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
     // memory window would break the swizzled layouts and is reported instead of run
     if (n_tiles && tid == 0) atomicOr(p.status, SS_DEV_WAIT_EXPIRED);
     if (tid < nrows) out_ml[tid] = make_float2(-INFINITY, 0.f);
+    fill_unused();
+    if (WALK) {
+      __syncthreads();  // (the table in the control block is rebuilt for the next request)
+      continue;
+    }
     if (!p.wait_first && chain_cta) pdl_wait_prior();
     return;
   }
@@ -215,6 +267,16 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
   constexpr int kProducerWarp = 4 * WG, kMmaWarp = 4 * WG + 1;
   if (warp == kProducerWarp) {
     if (lane == 0) {
+      if (tmem_held) {  // a later request of the share: the barriers start over
+        for (int u = 0; u < UNITS; ++u) {
+          mbar_inval(&ctl->ufull[u]);
+          mbar_inval(&ctl->uempty[u]);
+        }
+        mbar_inval(&ctl->sfull[0]);
+        mbar_inval(&ctl->sfull[1]);
+        mbar_inval(&ctl->pready);
+        mbar_inval(&ctl->pfree);
+      }
       // the first loads go out as early as possible: only their own barriers exist yet
       for (int u = 0; u < UNITS; ++u) mbar_init(&ctl->ufull[u], 1);
       fence_barrier_init();
@@ -231,11 +293,13 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
       fence_barrier_init();
     }
     __syncwarp();
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                     smem_u32(&ctl->tmem_base)),
-                 "r"(C::kTmemCols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (!tmem_held) {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                       smem_u32(&ctl->tmem_base)),
+                   "r"(C::kTmemCols)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   } else if (warp < 4 * WG) {
     // Q rows -> shared memory as the K-major B operand (128-byte swizzle), zero padding rows
     // (N rows x 16 pieces of 16 bytes over 128 * WG threads = 4 pieces per thread: all four
@@ -268,7 +332,8 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = ctl->tmem_base;
+  tmem = ctl->tmem_base;
+  tmem_held = true;
   unsigned long long* trl = lane == 0 ? tr : nullptr;
 
   if (warp == kProducerWarp && small_pages) {
@@ -429,6 +494,12 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
           break;
         }
       }
+    }
+    if (WALK && lane == 0 && n_uses >= 2) {
+      // the barriers are set up anew for the share's next request: the last two releases of ring
+      // units (asynchronous arrivals of the tensor core) must have landed
+      mwait(&ctl->uempty[(n_uses - 2) % UNITS], ((n_uses - 2) / UNITS) & 1);
+      mwait(&ctl->uempty[(n_uses - 1) % UNITS], ((n_uses - 1) / UNITS) & 1);
     }
   } else {
     // ===== softmax warps: TMEM lane L = key L of the tile; columns [c0, c0 + cn) = rows =====
@@ -714,17 +785,40 @@ chunk_tc_keys_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tm
     }
   }
 
-  // ---- teardown ----
+  if (warp < 4 * WG) {
+    fill_unused();
+    if (WALK) fence_proxy_async();  // the ring served as scratch; bulk copies write it next
+  }
+  tiles_walked += n_tiles;
+  // every role is done with this request: the ring, the barriers and the tensor memory are free
   tc_fence_before();
   __syncthreads();
-  if (warp == kProducerWarp) {
+  if (ctl->abort) break;
+  }  // for each request of the CTA's share
+
+  // ---- teardown ----
+  if (tmem_held && warp == 4 * WG) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::kTmemCols)
                  : "memory");
   }
-  if (tid == 0) cta_log_write(p, t_cta0, n_tiles);
+  if (tid == 0) cta_log_write(p, t_cta0, tiles_walked);
   // Completion order along the stream: one CTA of this grid waits for the previous grid, so
   // this grid cannot complete before it (the other CTAs leave at once and free their SM slot).
   if (!p.wait_first && chain_cta) pdl_wait_prior();
+}
+
+template <int NC, int WG, int UNITS, int D, int HIST>
+cudaError_t launch_hist_cfg(const ChunkParams& p, const HistParams& h, const CUtensorMap& any_map, dim3 grid,
+                            cudaStream_t s, bool pdl) {
+  using C = Cfg<NC, WG, UNITS, D>;
+  return launch_kernel(chunk_tc_keys_kernel<NC, WG, UNITS, D, HIST>, grid, dim3(C::kThreads), C::kSmem, s, pdl, p,
+                       any_map, any_map, h);
+}
+
+template <int NC, int WG, int UNITS, int D, int HIST>
+cudaError_t prepare_hist() {
+  return cudaFuncSetAttribute(chunk_tc_keys_kernel<NC, WG, UNITS, D, HIST>,
+                              cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<NC, WG, UNITS, D>::kSmem);
 }
 
 template <int NC, int WG, int UNITS, int D>
@@ -733,12 +827,12 @@ cudaError_t launch_cfg(const ChunkParams& p, const CUtensorMap& tmK, const CUten
   using C = Cfg<NC, WG, UNITS, D>;
   dim3 grid(p.splits * p.row_tiles, p.H_kv, p.n_active ? p.n_active : p.B), block(C::kThreads);
   static const HistParams none = {};
-  return launch_kernel(chunk_tc_keys_kernel<NC, WG, UNITS, D, false>, grid, block, C::kSmem, s, pdl, p, tmK, tmV, none);
+  return launch_kernel(chunk_tc_keys_kernel<NC, WG, UNITS, D, 0>, grid, block, C::kSmem, s, pdl, p, tmK, tmV, none);
 }
 
 template <int NC, int WG, int UNITS, int D>
 cudaError_t prepare_cfg() {
-  return cudaFuncSetAttribute(chunk_tc_keys_kernel<NC, WG, UNITS, D, false>,
+  return cudaFuncSetAttribute(chunk_tc_keys_kernel<NC, WG, UNITS, D, 0>,
                               cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<NC, WG, UNITS, D>::kSmem);
 }
 
@@ -751,12 +845,10 @@ cudaError_t chunk_tc_keys_prepare() {
   if (e == cudaSuccess) e = prepare_cfg<32, 1, 6, 64>();
   if (e == cudaSuccess) e = prepare_cfg<32, 2, 8, 64>();
   if (e == cudaSuccess) e = prepare_cfg<32, 4, 8, 64>();
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(chunk_tc_keys_kernel<32, 1, 3, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             Cfg<32, 1, 3, 128>::kSmem);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(chunk_tc_keys_kernel<32, 1, 6, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             Cfg<32, 1, 6, 64>::kSmem);
+  if (e == cudaSuccess) e = prepare_hist<32, 1, 3, 128, 1>();
+  if (e == cudaSuccess) e = prepare_hist<32, 1, 3, 128, 2>();
+  if (e == cudaSuccess) e = prepare_hist<32, 1, 6, 64, 1>();
+  if (e == cudaSuccess) e = prepare_hist<32, 1, 6, 64, 2>();
   return e;
 }
 
@@ -767,14 +859,16 @@ cudaError_t launch_chunk_tc_keys_hist(const ChunkParams& p, const HistParams& h,
       p.rows_per_tile > 32)
     return cudaErrorInvalidValue;
   // (the K/V map parameters are not used by these instantiations: any valid map will do)
-  if (p.d == 64) {
-    using C = Cfg<32, 1, 6, 64>;
-    dim3 grid(p.splits * p.row_tiles, p.H_kv, p.B), block(C::kThreads);
-    return launch_kernel(chunk_tc_keys_kernel<32, 1, 6, 64, true>, grid, block, C::kSmem, s, pdl, p, any_map, any_map, h);
+  if (h.n_req) {
+    // ragged batch: h.walk_ctas CTAs per kv-head share all requests' tiles (one row tile)
+    if (p.row_tiles != 1 || h.n_req != p.B || h.walk_ctas < 1) return cudaErrorInvalidValue;
+    dim3 grid(h.walk_ctas, p.H_kv, 1);
+    return p.d == 64 ? launch_hist_cfg<32, 1, 6, 64, 2>(p, h, any_map, grid, s, pdl)
+                     : launch_hist_cfg<32, 1, 3, 128, 2>(p, h, any_map, grid, s, pdl);
   }
-  using C = Cfg<32, 1, 3, 128>;
-  dim3 grid(p.splits * p.row_tiles, p.H_kv, p.B), block(C::kThreads);
-  return launch_kernel(chunk_tc_keys_kernel<32, 1, 3, 128, true>, grid, block, C::kSmem, s, pdl, p, any_map, any_map, h);
+  dim3 grid(p.splits * p.row_tiles, p.H_kv, p.B);
+  return p.d == 64 ? launch_hist_cfg<32, 1, 6, 64, 1>(p, h, any_map, grid, s, pdl)
+                   : launch_hist_cfg<32, 1, 3, 128, 1>(p, h, any_map, grid, s, pdl);
 }
 
 // Rows per CTA (p.rows_per_tile): <= 32 -> two CTAs per SM with 4 softmax warps; <= 64 and

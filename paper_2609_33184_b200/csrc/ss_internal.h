@@ -72,6 +72,14 @@ struct HistParams {
   int n_chunks;                               // 0: an ordinary one-chunk launch (ChunkParams alone)
   const CUtensorMap* maps;                    // device memory: chunk j's K map at [2j], its V map at [2j + 1]
   const int32_t* valid_len[kMaxHistChunks];   // per chunk: device [B], or null (= L_c[j])
+  // Ragged batches (keys-on-M kernel): the CTAs of a kv-head walk equal shares of ALL its requests'
+  // tiles laid end to end, so a CTA may finish one request and start the next (one partial state
+  // per request it touches).  The shares are cut on the host's copy of the lengths: req_prefix[b] =
+  // 128-token tiles (by that copy, at least one per request) before request b; a CTA's share of a
+  // request is scaled to the tiles the device's lengths give.  n_req = 0: not used.
+  int n_req;
+  int walk_ctas;                              // CTAs per kv-head (grid.x) of that mode
+  int req_prefix[kMaxListed + 1];
   int L_c[kMaxHistChunks];
 };
 

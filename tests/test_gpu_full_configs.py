@@ -85,7 +85,17 @@ def test_c2_qwen3_8b_full_one_call_per_chunk():
 
 
 def test_c3_internlm25_7b_ragged_full():
-    _resident("c3_internlm25_7b_ragged", 1, kernel="tcgen05-keys")   # ragged: one launch per chunk
+    # ragged, lengths known to the host: one launch whose CTAs share all requests' tiles
+    _resident("c3_internlm25_7b_ragged", 1, kernel="tcgen05-keys-round")
+
+
+def test_c3_internlm25_7b_ragged_full_one_call_per_chunk():
+    _resident("c3_internlm25_7b_ragged", 1, one_call=False, kernel="tcgen05-keys")
+
+
+def test_c5_resident_full():
+    # the streamed workload's batch (32 requests, 8,192 to 65,536 tokens) with its history in HBM
+    _resident("c5_streamed", 1, kernel="tcgen05-keys-round")
 
 
 def test_c4_tree_full():

@@ -970,6 +970,64 @@ def test_chunk_list_in_one_launch(d, T_q, H_q, H_kv, monkeypatch):
     ctx.close()
 
 
+@pytest.mark.parametrize("d,T_q,H_q,H_kv,lens", [
+    (128, 8, 8, 2, [6000, 300, 3100, 1500, 5000]),      # 32 rows; five requests over 15 CTAs per kv-head
+    (128, 3, 4, 4, [129, 6000, 128, 127, 1, 4000]),     # requests of a tile or two between long ones
+    (64, 4, 8, 2, [2000, 2100, 5900, 2200, 6000]),
+    (128, 5, 12, 4, [6000, 5000]),                      # 15 rows; fewer requests than CTAs
+])
+def test_chunk_list_ragged_batch_shares_across_requests(d, T_q, H_q, H_kv, lens, monkeypatch):
+    """A batch the host knows to be ragged, up to 32 rows per kv-head: one launch whose CTAs take
+    equal shares of all requests' tiles laid end to end, so a CTA may end one request and begin the
+    next and a request has as many partial states as CTAs touched it.  Against the oracle and the
+    separate calls, with the chunk list in two orders, with host lengths that are out of date (the
+    shares are then scaled to the lengths on the device), and for bit-identical repeats."""
+    import ctypes as C
+    from paper_2609_33184_b200 import binding as ssb
+    monkeypatch.setenv("SS_HISTORY_LAUNCH", "always")   # (a history of a few dozen tiles: not routed by itself)
+    cfg = inputs.VerifyConfig("walk", 0xe9 + d + T_q, len(lens), H_q, H_kv, d, 512, T_q, 0, max(lens))
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    ctx = util.make_ctx(cfg, flags=ssb.SS_FLAG_OVERLAP_CHUNKS)
+    O5, L5 = util.gpu_case(ctx, cfg, Q, chunks, K_loc, V_loc, bits)
+    assert ctx.last_chunk_kernel() == "tcgen05-keys"
+    ref = util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits)
+    util.compare(cfg, O5, L5, ref)
+    n = len(chunks)
+    stale = [max(1, (l * 3) // 5 if i % 2 else min(max(lens), l + 700)) for i, l in enumerate(lens)]
+    for order, host_lens in ((list(range(n)), lens), (list(range(n - 1, -1, -1)), lens), (list(range(n)), stale)):
+        lst = [chunks[j] for j in order]
+        hints = []
+        for j in order:   # the host's idea of chunk j's valid lengths
+            hints.append((C.c_int32 * cfg.B)(*[max(0, min(cfg.L_c, hl - j * cfg.L_c)) for hl in host_lens]))
+        descs = ctx.chunk_descs([lst], hints)
+        O, LSE = torch.empty_like(O5), torch.empty_like(L5)
+        for rep in range(3):
+            ctx.ss_verify_begin(Q, cfg.scale)
+            ctx.ss_verify_chunks(descs, n)
+            ctx.ss_verify_local(K_loc, V_loc, ssb.SS_MASK_CHAIN, None)
+            ctx.ss_verify_finalize(O, LSE)
+            torch.cuda.synchronize()
+            assert ctx.last_chunk_kernel() == "tcgen05-keys-round"
+            assert ctx.ss_poll_status() == (0, 0)
+            if rep == 0:
+                O0, L0 = O.clone(), LSE.clone()
+            else:
+                assert torch.equal(O0.view(torch.int16), O.view(torch.int16)) and torch.equal(L0, LSE)
+        util.compare(cfg, O, LSE, util.oracle_case(cfg, lens, Q, lst, K_loc, V_loc, bits))
+    # a bad valid length on the device is flagged and clamped
+    bad = [(K, V, vl.clone()) for (K, V, vl) in chunks]
+    bad[1][2][0] = 9999
+    hints = [(C.c_int32 * cfg.B)(*vl.tolist()) for (_, _, vl) in chunks]
+    ctx.ss_verify_begin(Q, cfg.scale)
+    ctx.ss_verify_chunks(ctx.chunk_descs([bad], hints), n)
+    ctx.ss_verify_local(K_loc, V_loc, ssb.SS_MASK_CHAIN, None)
+    ctx.ss_verify_finalize(O, LSE)
+    torch.cuda.synchronize()
+    assert ctx.last_chunk_kernel() == "tcgen05-keys-round"
+    assert ctx.ss_poll_status()[1] & ssb.SS_DEV_BAD_VALID_LEN
+    ctx.close()
+
+
 def test_chunk_list_after_separate_chunks_with_one_partial_set(monkeypatch):
     """A context with a single partial set: a chunk call, then a list of chunks in one launch (the
     set in use is folded first), then another chunk call; against the oracle."""
@@ -1004,8 +1062,9 @@ def test_two_chunk_calls_with_max_chunks_one():
 
 def test_chunk_list_routing():
     """Which lists go out as one launch: histories the host knows to be equally long at any row
-    count; more than 128 rows per kv-head at head dim 128 also when it knows nothing; never a batch
-    it knows to be ragged, nor a history of a few tiles."""
+    count; up to 32 rows per kv-head also a batch it knows to be ragged (no request empty); more than
+    128 rows per kv-head at head dim 128 also when it knows nothing, but not a batch it knows to be
+    ragged; never a history of a few tiles."""
     import ctypes as C
     from paper_2609_33184_b200 import binding as ssb
 
@@ -1025,7 +1084,8 @@ def test_chunk_list_routing():
     even, ragged = [4096, 4096, 4000], [4096, 1000, 2500]
     assert kernel_for(128, 8, 8, 2, even, True) == "tcgen05-keys-round"      # 32 rows, known equal
     assert kernel_for(128, 8, 8, 2, even, False) == "tcgen05-keys"           # lengths only on the device
-    assert kernel_for(128, 8, 8, 2, ragged, True) == "tcgen05-keys"
+    assert kernel_for(128, 8, 8, 2, ragged, True) == "tcgen05-keys-round"    # known ragged: shares across requests
+    assert kernel_for(128, 8, 8, 2, [4096, 0, 2500], True) == "tcgen05-keys"  # ... not with an empty request
     assert kernel_for(128, 8, 16, 2, even, True) == "tcgen05-round"          # 64 rows, known equal
     assert kernel_for(128, 8, 16, 2, even, False) == "tcgen05"
     assert kernel_for(64, 8, 16, 2, even, True) == "tcgen05-round"           # head dim 64, 64 rows
