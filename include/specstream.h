@@ -110,7 +110,8 @@ typedef struct {
  *   SS_TARGET_CTAS=n           the CTA count the automatic split choice aims at
  * and, read at every ss_verify_chunks call:
  *   SS_HISTORY_LAUNCH=never|always  never / wherever possible take a list of chunks in one launch
- *   SS_HISTORY_WALK=never           ragged batches do not take the one launch with shares across requests */
+ *   SS_HISTORY_WALK=never|always    ragged batches never take / batches of any known lengths take
+ *                                   the one launch with shares across requests */
 
 typedef struct {
   const void* ptr;                      /* device pointer, bf16                      */

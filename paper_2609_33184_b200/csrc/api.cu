@@ -794,7 +794,8 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
   // of a kv-head walk equal shares of all its requests' tiles laid end to end (HistParams::n_req).
   // SS_HISTORY_WALK=never leaves such batches to the separate calls.
   const char* wk = getenv("SS_HISTORY_WALK");
-  const bool walk = keys_on_m && R <= 32 && known && !uniform && lo > 0 && !(wk && strcmp(wk, "never") == 0);
+  const bool walk = keys_on_m && R <= 32 && known && lo > 0 && (!uniform || (wk && strcmp(wk, "always") == 0)) &&
+                    !(wk && strcmp(wk, "never") == 0);
   if (keys_on_m) {
     if (R > 32) return SS_OK;
     if (!uniform && !always && !walk) return SS_OK;
