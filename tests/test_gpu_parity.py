@@ -1028,6 +1028,43 @@ def test_chunk_list_ragged_batch_shares_across_requests(d, T_q, H_q, H_kv, lens,
     ctx.close()
 
 
+@pytest.mark.parametrize("B,seed", [(3, 1), (7, 2), (16, 3), (32, 4), (32, 5)])
+def test_chunk_list_ragged_batch_random_lengths(B, seed):
+    """Shares across requests on random batches with 8 kv-heads (37 CTAs per kv-head, or one per
+    eight tiles): lengths from one token to the full history, so requests of a tile or two sit
+    between long ones and a request is cut into one to a dozen pieces.  Every request against
+    the separate calls, a sample of (request, kv-head) groups against the oracle."""
+    import ctypes as C
+    from paper_2609_33184_b200 import binding as ssb
+    rng = np.random.default_rng(1000 + seed)
+    hi = 9000
+    lens = [int(x) for x in rng.integers(1, hi + 1, size=B)]
+    lens[int(rng.integers(0, B))] = hi                     # one request has the full history
+    if B > 3:
+        lens[int(rng.integers(0, B))] = int(rng.integers(1, 129))   # and one a single tile
+    cfg = inputs.VerifyConfig("walkr", 0xf300 + seed, B, 8, 8, 128, 1024, 4, 0, hi)
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    n = len(chunks)
+    ctx = util.make_ctx(cfg, flags=ssb.SS_FLAG_OVERLAP_CHUNKS)
+    O5, L5 = util.gpu_case(ctx, cfg, Q, chunks, K_loc, V_loc, bits)
+    hints = [(C.c_int32 * B)(*vl.tolist()) for (_, _, vl) in chunks]
+    O, LSE = torch.empty_like(O5), torch.empty_like(L5)
+    ctx.ss_verify_begin(Q, cfg.scale)
+    ctx.ss_verify_chunks(ctx.chunk_descs([chunks], hints), n)
+    ctx.ss_verify_local(K_loc, V_loc, ssb.SS_MASK_CHAIN, None)
+    ctx.ss_verify_finalize(O, LSE)
+    torch.cuda.synchronize()
+    assert ctx.last_chunk_kernel() == "tcgen05-keys-round"
+    assert ctx.ss_poll_status() == (0, 0)
+    # the two paths sum the same weights in another order: far inside the oracle tolerances
+    assert float((O.float() - O5.float()).abs().max()) <= 2.0 ** -7 * max(1.0, float(O5.float().abs().max()))
+    assert float((LSE - L5).abs().max()) <= 1e-4
+    groups = [(int(rng.integers(0, B)), int(rng.integers(0, 8))) for _ in range(4)]
+    groups += [(int(np.argmax(lens)), 0), (int(np.argmin(lens)), 7)]
+    util.compare(cfg, O, LSE, util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits, groups=groups))
+    ctx.close()
+
+
 def test_chunk_list_after_separate_chunks_with_one_partial_set(monkeypatch):
     """A context with a single partial set: a chunk call, then a list of chunks in one launch (the
     set in use is folded first), then another chunk call; against the oracle."""
