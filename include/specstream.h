@@ -108,6 +108,8 @@ typedef struct {
  *   SS_SPLITS=n                token splits of every chunk call (default: sized so that a
  *                              call launches about one CTA per SM)
  *   SS_TARGET_CTAS=n           the CTA count the automatic split choice aims at
+ *   SS_ROUND_CLUSTER=never     the single-launch small round merges its token splits through
+ *                              scratch memory and a ticket instead of a thread-block cluster
  * and, read at every ss_verify_chunks call:
  *   SS_HISTORY_LAUNCH=never|always  never / wherever possible take a list of chunks in one launch
  *   SS_HISTORY_WALK=never|always    ragged batches never take / batches of any known lengths take

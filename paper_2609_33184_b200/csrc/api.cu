@@ -57,6 +57,7 @@ struct ss_ctx {
   bool no_overlap;          // set while ss_stream_round drives the context
   unsigned long long* trace;  // device trace region (in the workspace)
   unsigned int* round_counters;  // ticket counters of split small rounds (zero between rounds)
+  bool round_clusters;           // split small rounds merge inside a thread-block cluster (until a launch refuses)
   bool trace_on;
   unsigned long long* cta_log;  // caller's per-CTA log buffer (ss_cta_log_set) or null
   int cta_log_cap;
@@ -401,6 +402,8 @@ ss_status ss_create(ss_ctx** out, const ss_config* cfg, void* workspace, size_t 
   c->target_forced = getenv("SS_TARGET_CTAS") != nullptr && atoi(getenv("SS_TARGET_CTAS")) > 0;
   const char* fs = getenv("SS_SPLITS");
   c->force_splits = fs ? atoi(fs) : 0;
+  const char* rc = getenv("SS_ROUND_CLUSTER");
+  c->round_clusters = !(rc && strcmp(rc, "never") == 0);
   const char* ck = getenv("SS_CHUNK_KERNEL");
   c->force_rows_kernel = (ck && strcmp(ck, "rows") == 0) || (cfg->flags & SS_FLAG_ROWS_ON_M);
   c->force_keys_kernel = (ck && strcmp(ck, "keys") == 0) || (cfg->flags & SS_FLAG_KEYS_ON_M);
@@ -1046,7 +1049,17 @@ ss_status ss_verify_round(ss_ctx* c, ss_tensor Q, int32_t B, int32_t T_q, float 
     p.O = (__nv_bfloat16*)O;
     p.LSE = LSE;
     p.status = c->status;
-    cudaError_t e = ss::launch_round_simt(p, (cudaStream_t)stream, (c->cfg.flags & SS_FLAG_OVERLAP_CHUNKS) && !c->no_overlap);
+    const bool pdl = (c->cfg.flags & SS_FLAG_OVERLAP_CHUNKS) && !c->no_overlap;
+    // the splits of a unit as one thread-block cluster: the states are merged through distributed
+    // shared memory instead of scratch, a ticket and two trips to L2
+    p.cluster = (p.splits > 1 && c->round_clusters) ? 1 : 0;
+    cudaError_t e = ss::launch_round_simt(p, (cudaStream_t)stream, pdl);
+    if (e != cudaSuccess && p.cluster) {  // (a device or driver that does not take the cluster: the ticket path)
+      (void)cudaGetLastError();
+      c->round_clusters = false;
+      p.cluster = 0;
+      e = ss::launch_round_simt(p, (cudaStream_t)stream, pdl);
+    }
     if (e != cudaSuccess) return cuda_fail(c, e);
     c->last_kernel = "simt-round";
     ++c->launches;

@@ -348,10 +348,38 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const __grid_const
 // A whole round in one launch: grid = (row tiles x token splits, H_kv, B).  The history's
 // 64-token tiles (all chunks, in order) are dealt to the splits in equal runs, the last split
 // also takes the local segment.  With one split a CTA finalizes its rows itself.  With more,
-// every CTA parks its partial state (m, l, a) in scratch and takes a ticket from the counter
-// of its (request, kv-head, row tile); the CTA that draws the last ticket merges the states
-// (Eq. 14), finalizes, and leaves the counter at zero for the next round.  A round this small
-// is bound by memory latency, not bandwidth: the splits are what puts enough loads in flight.
+// the splits of a (request, kv-head, row tile) form a thread-block cluster (p.cluster): every
+// CTA leaves its partial state (m, l, a) in its own shared memory, and after a cluster barrier
+// the first CTA reads all of them through distributed shared memory, merges (Eq. 14) and
+// finalizes - no state goes through global memory.  Without clusters every CTA parks its state
+// in scratch and takes a ticket from the unit's counter; the CTA that draws the last ticket
+// merges, finalizes and leaves the counter at zero for the next round.  A round this small is
+// bound by memory latency, not bandwidth: the splits are what puts enough loads in flight.
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of this CTA's shared-memory location `p` in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t cluster_map(const void* p, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;"
+               : "=r"(r)
+               : "r"((uint32_t)__cvta_generic_to_shared(p)), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t a) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t a) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "r"(a)
+               : "memory");
+  return v;
+}
+
 template <int D, int RT>
 __global__ void __launch_bounds__(kThreads) round_simt_kernel(const __grid_constant__ RoundParams p) {
   extern __shared__ __align__(16) uint8_t smem_simt[];
@@ -360,7 +388,9 @@ __global__ void __launch_bounds__(kThreads) round_simt_kernel(const __grid_const
   st.init(smem_simt);
   const int tid = threadIdx.x;
   const int row_tiles = gridDim.x / p.splits;   // p.splits counts the local segment's own CTA
-  const int rt = blockIdx.x % row_tiles, sp = blockIdx.x / row_tiles;
+  // (clusters run along x: the splits of a row tile are neighbours there, sp = rank in the cluster)
+  const int rt = p.cluster ? blockIdx.x / p.splits : blockIdx.x % row_tiles;
+  const int sp = p.cluster ? blockIdx.x % p.splits : blockIdx.x / row_tiles;
   const int b = blockIdx.z, kvh = blockIdx.y, row0 = rt * RT;
   const int R = p.T_q * p.G, nrows = min(RT, R - row0);
   // Launched with programmatic stream serialization, the grid is set up while the kernel before
@@ -416,7 +446,54 @@ __global__ void __launch_bounds__(kThreads) round_simt_kernel(const __grid_const
   }
   if (q_pending) st.q_store();  // nothing to attend to here: the identity state
   st.reduce_groups();  // q_s[r][c] = a[r][c]
-  if (p.splits > 1) {
+  if (p.splits > 1 && p.cluster) {
+    // every CTA of the cluster holds its state in q_s / m_s / l_s; CTA 0 merges them (Eq. 14 over
+    // all splits at once, every load of a phase independent of the others) through distributed
+    // shared memory.  The second barrier keeps the other CTAs' shared memory alive until then.
+    cluster_sync_all();
+    if (sp == 0) {
+      float* ml_all = st.p_s;  // [split][2 * RT]: the scores array is free by now
+      for (int i = tid; i < p.splits * 2 * RT; i += kThreads)
+        ml_all[i] = ld_cluster_f32(cluster_map(st.m_s + i % (2 * RT), i / (2 * RT)));  // (l_s follows m_s)
+      __syncthreads();
+      if (tid < RT) {
+        float M = -INFINITY;
+        for (int s2 = 0; s2 < p.splits; ++s2) M = fmaxf(M, ml_all[s2 * 2 * RT + tid]);
+        float l = 0.f;
+        for (int s2 = 0; s2 < p.splits; ++s2) {
+          const float m2 = ml_all[s2 * 2 * RT + tid];
+          const float f = m2 > -INFINITY ? exp2f(m2 - M) : 0.f;
+          l += f * ml_all[s2 * 2 * RT + RT + tid];
+          ml_all[s2 * 2 * RT + tid] = f;  // the split's factor for this row replaces its maximum
+        }
+        st.m_s[tid] = M;
+        st.l_s[tid] = l;
+      }
+      __syncthreads();
+      for (int i = tid; i < RT * D / 4; i += kThreads) {
+        const int r = i / (D / 4);
+        float4 v[16];
+#pragma unroll
+        for (int s2 = 0; s2 < 16; ++s2)
+          v[s2] = s2 < p.splits ? ld_cluster_f32x4(cluster_map(st.q_s + 4 * i, s2)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int s2 = 0; s2 < 16; ++s2) {
+          const float f = s2 < p.splits ? ml_all[s2 * 2 * RT + r] : 0.f;
+          if (f > 0.f) {  // a split that saw nothing holds no a[]
+            a.x += f * v[s2].x;
+            a.y += f * v[s2].y;
+            a.z += f * v[s2].z;
+            a.w += f * v[s2].w;
+          }
+        }
+        reinterpret_cast<float4*>(st.q_s)[i] = a;   // (the thread's own piece of CTA 0's state)
+      }
+      __syncthreads();
+    }
+    cluster_sync_all();
+    if (sp != 0) return;
+  } else if (p.splits > 1) {
     // park the partial state, take a ticket; only the CTA with the last ticket goes on
     const int64_t unit = ((int64_t)b * p.H_kv + kvh) * row_tiles + rt;
     float* slot = p.scratch + (unit * p.splits + sp) * (int64_t)(RT * (D + 2));
@@ -506,6 +583,8 @@ cudaError_t prepare_one() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(round_simt_kernel<D, RT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              Lay<D, RT>::kBytes);
+  if (e == cudaSuccess)  // clusters of up to 16 CTAs (more than the portable 8)
+    e = cudaFuncSetAttribute(round_simt_kernel<D, RT>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
   return e;
 }
 
@@ -545,10 +624,23 @@ cudaError_t launch_chunk_simt(const ChunkParams& p, cudaStream_t s, bool pdl) {
   return SS_SIMT_DISPATCH(chunk_simt_kernel, p.d, p.rows_per_tile, grid, block, smem, s, pdl, p);
 }
 
+#define SS_SIMT_DISPATCH_CLUSTER(KERNEL, D_, RT_, ...)                                           \
+  ((D_) == 128 ? ((RT_) == 8    ? launch_kernel_cluster(KERNEL<128, 8>, __VA_ARGS__)              \
+                  : (RT_) == 16 ? launch_kernel_cluster(KERNEL<128, 16>, __VA_ARGS__)             \
+                                : launch_kernel_cluster(KERNEL<128, 32>, __VA_ARGS__))            \
+               : ((RT_) == 8    ? launch_kernel_cluster(KERNEL<64, 8>, __VA_ARGS__)               \
+                  : (RT_) == 16 ? launch_kernel_cluster(KERNEL<64, 16>, __VA_ARGS__)              \
+                                : launch_kernel_cluster(KERNEL<64, 32>, __VA_ARGS__)))
+
+// p.cluster: the p.splits (2 to 16) CTAs of a unit are launched as one cluster along x.
 cudaError_t launch_round_simt(const RoundParams& p, cudaStream_t s, bool pdl) {
   const int R = p.T_q * p.G, rt = p.rows_per_tile;
   dim3 grid(((R + rt - 1) / rt) * p.splits, p.H_kv, p.B), block(kThreads);
   const size_t smem = simt_smem(p.d, rt);
+  if (p.cluster) {
+    if (p.splits < 2 || p.splits > 16) return cudaErrorInvalidValue;
+    return SS_SIMT_DISPATCH_CLUSTER(round_simt_kernel, p.d, rt, grid, block, smem, s, pdl, (unsigned)p.splits, p);
+  }
   return SS_SIMT_DISPATCH(round_simt_kernel, p.d, rt, grid, block, smem, s, pdl, p);
 }
 

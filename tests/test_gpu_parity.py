@@ -841,11 +841,18 @@ def test_chain_with_more_local_tokens_than_queries(T_q, T_loc, G):
     ("tree, G=5", inputs.VerifyConfig("r3", 0xa3, 2, 10, 2, 128, 192, 12, 0, 500, mask="tree"), [1, 500]),
     ("plain decode", inputs.VerifyConfig("r4", 0xa4, 4, 16, 2, 64, 512, 1, 0, 1500), [1500, 511, 512, 513]),
 ])
-def test_whole_round_in_one_call_small(name, cfg, lens):
+@pytest.mark.parametrize("merge", ["cluster", "ticket"])
+def test_whole_round_in_one_call_small(name, cfg, lens, merge, monkeypatch):
     """ss_verify_round on rounds small enough for its single-launch kernel: equal to the oracle
-    and (within rounding) to the separate calls."""
+    and (within rounding) to the separate calls.  The token splits of a (request, kv-head, row
+    tile) merge inside a thread-block cluster through distributed shared memory, or (clusters
+    turned off) through scratch memory and a ticket counter; both give the same bits."""
     from paper_2609_33184_b200 import binding as ssb
     lens = lens or inputs.history_lengths(cfg)
+    if merge == "ticket":
+        monkeypatch.setenv("SS_ROUND_CLUSTER", "never")   # (read when the context is created)
+    else:
+        monkeypatch.delenv("SS_ROUND_CLUSTER", raising=False)
     Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
     ctx = util.make_ctx(cfg)
     kind = ssb.SS_MASK_TREE_BITS if cfg.mask == "tree" else ssb.SS_MASK_CHAIN
@@ -857,6 +864,16 @@ def test_whole_round_in_one_call_small(name, cfg, lens):
     assert ctx.ss_poll_status() == (0, 0)
     ref = util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits)
     util.compare(cfg, O, LSE, ref)
+    if merge == "cluster":   # the other merge path sums the same states in the same order
+        monkeypatch.setenv("SS_ROUND_CLUSTER", "never")
+        ctx_t = util.make_ctx(cfg)
+        Ot, Lt = torch.empty_like(O), torch.empty_like(LSE)
+        for _ in range(3):
+            ctx_t.ss_verify_round(Q, cfg.scale, chunks, K_loc, V_loc, kind, bits if cfg.mask == "tree" else None, Ot, Lt)
+            ctx.ss_verify_round(Q, cfg.scale, chunks, K_loc, V_loc, kind, bits if cfg.mask == "tree" else None, O, LSE)
+        torch.cuda.synchronize()
+        assert torch.equal(O.view(torch.int16), Ot.view(torch.int16)) and torch.equal(LSE.view(torch.int32), Lt.view(torch.int32))
+        ctx_t.close()
     O2, L2 = util.gpu_case(ctx, cfg, Q, chunks, K_loc, V_loc, bits)
     mag = max(1.0, float(O2.float().abs().max()))
     assert float((O.float() - O2.float()).abs().max()) <= util.TOL_MAX_O * mag
