@@ -797,6 +797,8 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
   // of a kv-head walk equal shares of all its requests' tiles laid end to end (HistParams::n_req).
   // SS_HISTORY_WALK=never leaves such batches to the separate calls.
   const char* wk = getenv("SS_HISTORY_WALK");
+  // (The rows-on-M kernel was given the same mode per (kv-head, row tile) and lost to the separate
+  // calls on ragged batches at every row count but one: not kept.)
   const bool walk = keys_on_m && R <= 32 && known && lo > 0 && (!uniform || (wk && strcmp(wk, "always") == 0)) &&
                     !(wk && strcmp(wk, "never") == 0);
   if (keys_on_m) {
@@ -818,7 +820,7 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
     tiles += (d.L_c + kTileKeys - 1) / kTileKeys;
     if (keys_on_m && d.L_c < 128) return SS_OK;   // (a box of 128 tokens)
   }
-  if (tiles > 0x3fffffff || (keys_on_m && tiles / 2 > 65000)) return SS_OK;   // (the keys kernel's 16-bit tile table)
+  if ((keys_on_m ? tiles / 2 : tiles) > 65000) return SS_OK;   // (the kernels' 16-bit tile tables)
   // a history of a few tiles per request is latency bound: the separate calls (CUDA-core kernel for
   // tiny ones) or the one-launch small round of ss_verify_round do better (measured on the
   // 1,024-token chain workload)
@@ -841,6 +843,7 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
   if (walk) {
     // 128-token tiles of each request by the host's lengths; the shares and the largest number of
     // pieces a request is cut into (= partial states per row), with the kernel's own arithmetic
+    const int tile_tokens = 128;
     h.n_req = c->B;
     for (int b = 0; b < c->B; ++b) {
       int64_t t128 = 0;
@@ -848,7 +851,7 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
         const ss_chunk_desc& d = chunks[j];
         int64_t v = d.valid_len ? d.valid_len_host[b] : d.L_c;
         v = v < 0 ? 0 : (v > d.L_c ? d.L_c : v);
-        t128 += (v + 127) / 128;
+        t128 += (v + tile_tokens - 1) / tile_tokens;
       }
       h.req_prefix[b + 1] = h.req_prefix[b] + (int)t128;
     }

@@ -234,7 +234,7 @@ struct TileMap {
 };
 template <>
 struct TileMap<true> {
-  const int* prefix;
+  const uint16_t* prefix;
   const int* valid;
   int g0, j;
   // chunk of tile `it` (tiles are asked for in ascending order) and the tile's first token in it
@@ -383,8 +383,11 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
   unsigned long long* tr = chain_cta ? p.trace : nullptr;
   int n_tiles = (tok1 > tok0) ? (tok1 - tok0 + kTileKeys - 1) / kTileKeys : 0;
   // a list of chunks: the table of the request's tiles per chunk, then this CTA's share of them
-  int* const hist_prefix = reinterpret_cast<int*>(smem + kSmemData + 256);   // [kMaxHistChunks + 1]
-  int* const hist_valid = hist_prefix + kMaxHistChunks + 1;                  // [kMaxHistChunks]
+  // (16-bit tile counts: the host keeps a request's tiles below 65,536; 256 + 128 + 66 bytes end
+  // inside the control block's 512)
+  int* const hist_valid = reinterpret_cast<int*>(smem + kSmemData + 256);                      // [kMaxHistChunks]
+  uint16_t* const hist_prefix = reinterpret_cast<uint16_t*>(hist_valid + kMaxHistChunks);      // [kMaxHistChunks + 1]
+  static_assert(256 + kMaxHistChunks * 4 + (kMaxHistChunks + 1) * 2 <= kSmemCtl, "chunk table");
   int g0 = 0;
   if (HIST) {
     if (warp == 0) {
@@ -404,13 +407,13 @@ chunk_tc_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap tmK,
         if (lane >= o) incl += up;
       }
       if (lane < h.n_chunks) {
-        hist_prefix[lane + 1] = incl;
+        hist_prefix[lane + 1] = (uint16_t)incl;
         hist_valid[lane] = v;
       }
       if (lane == 0) hist_prefix[0] = 0;
       // (entries past the last chunk repeat the total, so a walk never runs off the table)
       const int total = __shfl_sync(0xffffffffu, incl, 31);
-      if (lane >= h.n_chunks) hist_prefix[lane + 1] = total;
+      if (lane >= h.n_chunks) hist_prefix[lane + 1] = (uint16_t)total;
     }
     __syncthreads();
     const int total = hist_prefix[h.n_chunks];

@@ -1005,8 +1005,10 @@ def test_chunk_list_ragged_batch_shares_across_requests(d, T_q, H_q, H_kv, lens,
     cfg = inputs.VerifyConfig("walk", 0xe9 + d + T_q, len(lens), H_q, H_kv, d, 512, T_q, 0, max(lens))
     Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
     ctx = util.make_ctx(cfg, flags=ssb.SS_FLAG_OVERLAP_CHUNKS)
+    keys = T_q * (H_q // H_kv) <= (32 if d == 128 else 16)
+    one, each = ("tcgen05-keys-round", "tcgen05-keys") if keys else ("tcgen05-round", "tcgen05")
     O5, L5 = util.gpu_case(ctx, cfg, Q, chunks, K_loc, V_loc, bits)
-    assert ctx.last_chunk_kernel() == "tcgen05-keys"
+    assert ctx.last_chunk_kernel() == each
     ref = util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits)
     util.compare(cfg, O5, L5, ref)
     n = len(chunks)
@@ -1024,13 +1026,15 @@ def test_chunk_list_ragged_batch_shares_across_requests(d, T_q, H_q, H_kv, lens,
             ctx.ss_verify_local(K_loc, V_loc, ssb.SS_MASK_CHAIN, None)
             ctx.ss_verify_finalize(O, LSE)
             torch.cuda.synchronize()
-            assert ctx.last_chunk_kernel() == "tcgen05-keys-round"
+            assert ctx.last_chunk_kernel() == one
             assert ctx.ss_poll_status() == (0, 0)
             if rep == 0:
                 O0, L0 = O.clone(), LSE.clone()
             else:
                 assert torch.equal(O0.view(torch.int16), O.view(torch.int16)) and torch.equal(L0, LSE)
         util.compare(cfg, O, LSE, util.oracle_case(cfg, lens, Q, lst, K_loc, V_loc, bits))
+        assert float((O.float() - O5.float()).abs().max()) <= 2.0 ** -7 * max(1.0, float(O5.float().abs().max()))
+        assert float((LSE - L5).abs().max()) <= 1e-4
     # a bad valid length on the device is flagged and clamped
     bad = [(K, V, vl.clone()) for (K, V, vl) in chunks]
     bad[1][2][0] = 9999
@@ -1040,7 +1044,7 @@ def test_chunk_list_ragged_batch_shares_across_requests(d, T_q, H_q, H_kv, lens,
     ctx.ss_verify_local(K_loc, V_loc, ssb.SS_MASK_CHAIN, None)
     ctx.ss_verify_finalize(O, LSE)
     torch.cuda.synchronize()
-    assert ctx.last_chunk_kernel() == "tcgen05-keys-round"
+    assert ctx.last_chunk_kernel() == one
     assert ctx.ss_poll_status()[1] & ssb.SS_DEV_BAD_VALID_LEN
     ctx.close()
 
@@ -1079,6 +1083,32 @@ def test_chunk_list_ragged_batch_random_lengths(B, seed):
     groups = [(int(rng.integers(0, B)), int(rng.integers(0, 8))) for _ in range(4)]
     groups += [(int(np.argmax(lens)), 0), (int(np.argmin(lens)), 7)]
     util.compare(cfg, O, LSE, util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits, groups=groups))
+    ctx.close()
+
+
+@pytest.mark.parametrize("T_q,H_q", [(8, 8), (40, 8)])
+def test_chunk_list_of_32_chunks(T_q, H_q, monkeypatch):
+    """The longest list a launch takes (32 chunks: every entry of the kernels' chunk tables in
+    use), keys-on-M and rows-on-M kernel, the last chunks ragged and one request's empty."""
+    import ctypes as C
+    from paper_2609_33184_b200 import binding as ssb
+    monkeypatch.setenv("SS_HISTORY_LAUNCH", "always")
+    cfg = inputs.VerifyConfig("l32", 0x7a + T_q, 2, H_q, 2, 128, 128, T_q, 0, 4096)
+    lens = [4096, 3900]
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    assert len(chunks) == 32
+    ctx = util.make_ctx(cfg, flags=ssb.SS_FLAG_OVERLAP_CHUNKS)
+    hints = [(C.c_int32 * cfg.B)(*vl.tolist()) for (_, _, vl) in chunks]
+    O = torch.empty(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV)
+    LSE = torch.empty(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV)
+    ctx.ss_verify_begin(Q, cfg.scale)
+    ctx.ss_verify_chunks(ctx.chunk_descs([chunks], hints), 32)
+    ctx.ss_verify_local(K_loc, V_loc, ssb.SS_MASK_CHAIN, None)
+    ctx.ss_verify_finalize(O, LSE)
+    torch.cuda.synchronize()
+    assert ctx.last_chunk_kernel() == ("tcgen05-keys-round" if T_q == 8 else "tcgen05-round")
+    assert ctx.ss_poll_status() == (0, 0)
+    util.compare(cfg, O, LSE, util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits))
     ctx.close()
 
 
