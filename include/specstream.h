@@ -223,8 +223,9 @@ ss_status ss_verify_local(ss_ctx* ctx, ss_tensor K_loc, ss_tensor V_loc, int32_t
  * tensors, checks and results as the separate calls: a large round is begin + ss_verify_chunks
  * + local + finalize.  A small round (at most 16 chunks and 32 tiles of 64 tokens in all, T_loc <=
  * 64) takes a single launch of the CUDA-core kernel that walks the chunks and the local
- * segment and finalizes in place, so that no partial state goes through HBM and a tiny round
- * costs one launch instead of n_chunks + 2.  SS_ERR_STATE while a round is open; on any
+ * segment and finalizes in place (the token splits of a row tile run as one thread-block
+ * cluster and merge their states through distributed shared memory), so that no partial state
+ * goes through HBM and a tiny round costs one launch instead of n_chunks + 2.  SS_ERR_STATE while a round is open; on any
  * error nothing of the round is merged and the context is idle again. */
 ss_status ss_verify_round(ss_ctx* ctx, ss_tensor Q, int32_t B, int32_t T_q, float scale,
                           const ss_chunk_desc* chunks, int32_t n_chunks, ss_tensor K_loc,
