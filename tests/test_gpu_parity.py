@@ -656,6 +656,48 @@ def test_round_can_be_captured_in_a_cuda_graph():
     ctx.close()
 
 
+@pytest.mark.parametrize("lens", [[5000, 4900, 5000], [5000, 700, 2300]])
+def test_chunk_list_round_can_be_captured_in_a_cuda_graph(lens):
+    """A round whose list of chunks is one launch (equally long histories: equal splits per
+    request; a ragged batch: shares across requests) replays from a CUDA graph bit-identically,
+    also after the inputs were refreshed in place."""
+    import ctypes as C
+    ssb = _ssb()
+    cfg = inputs.VerifyConfig("gl", 0x61, len(lens), 8, 2, 128, 1024, 8, 0, max(lens))
+    Q, chunks, K_loc, V_loc, bits = util.gen_case(cfg, lens, DEV)
+    ctx = util.make_ctx(cfg, flags=ssb.SS_FLAG_OVERLAP_CHUNKS)
+    hints = [(C.c_int32 * cfg.B)(*vl.tolist()) for (_, _, vl) in chunks]
+    descs = ctx.chunk_descs([chunks], hints)
+    O, LSE = (torch.zeros(cfg.B, cfg.H_q, cfg.T_q, cfg.d, dtype=torch.bfloat16, device=DEV),
+              torch.zeros(cfg.B, cfg.H_q, cfg.T_q, dtype=torch.float32, device=DEV))
+
+    def one_round():
+        ctx.ss_verify_round(Q, cfg.scale, chunks, K_loc, V_loc, ssb.SS_MASK_CHAIN, None, O, LSE, descs=descs)
+
+    one_round()   # (the list of tensor maps is sent on first use: outside the capture)
+    torch.cuda.synchronize()
+    assert ctx.last_chunk_kernel() == "tcgen05-keys-round"
+    O_ref, L_ref = O.clone(), LSE.clone()
+    util.compare(cfg, O, LSE, util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits))
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        one_round()
+    for _ in range(3):
+        O.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(O.view(torch.int16), O_ref.view(torch.int16)) and torch.equal(LSE, L_ref)
+    # new queries in place: the replay equals a fresh call
+    Q.copy_(inputs.normal_bf16(cfg.seed + 1, inputs.TID_Q, tuple(Q.shape), device=DEV))
+    g.replay()
+    torch.cuda.synchronize()
+    O_g, L_g = O.clone(), LSE.clone()
+    one_round()
+    torch.cuda.synchronize()
+    assert torch.equal(O.view(torch.int16), O_g.view(torch.int16)) and torch.equal(LSE, L_g)
+    ctx.close()
+
+
 def test_two_contexts_on_two_streams_do_not_interfere():
     # Two contexts (own workspaces) whose rounds interleave call by call on two streams give,
     # bit for bit, what each gives alone: no state is shared between contexts.
