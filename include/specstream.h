@@ -197,6 +197,10 @@ ss_status ss_verify_chunk_paged(ss_ctx* ctx, ss_tensor K_pool, ss_tensor V_pool,
  * SS_HISTORY_LAUNCH=never|always in the environment overrides the routing.  Otherwise the
  * chunks are enqueued one by one.  The results agree with separate calls
  * up to the order of the fp32 sums (one launch merges per split, separate calls per chunk).
+ * Stream capture: the one launch reads the chunks' tensor maps from one of four lists in the
+ * workspace, sent when a list of buffers is first used.  Under a capture a list that is already
+ * there is kept for the life of the context (a graph may replay the launch), and a list that is
+ * not is not sent: those chunks are enqueued one by one.  So run a round once before capturing it.
  * SS_ERR_STATE outside an open round; an error leaves the round open (ss_verify_abort ends it). */
 typedef struct {
   ss_tensor K, V;                 /* [B, H_kv, L_c, d] bf16, device                          */

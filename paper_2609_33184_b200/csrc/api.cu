@@ -67,6 +67,7 @@ struct ss_ctx {
   CUtensorMap hist_host[4][2 * ss::kMaxHistChunks];
   int hist_n[4];            // maps in use per slot (0 = empty)
   uint64_t hist_age[4];
+  bool hist_pinned[4];      // the list was used under a stream capture: a graph may replay the launch, never evicted
   cudaEvent_t* ev_pool;     // timing events of the streamed round (SS_FLAG_STREAM_TIMING)
   int ev_pool_n;
 };
@@ -883,10 +884,21 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
     if (c->hist_n[i] == 2 * n_chunks && memcmp(c->hist_host[i], maps, (size_t)2 * n_chunks * sizeof(CUtensorMap)) == 0)
       slot = i;
   cudaStream_t s = c->stream;
+  // Under a stream capture the launch may be replayed from a graph for as long as the context
+  // lives, reading its list of tensor maps every time: a list that is already on the device is kept
+  // for good; a list that would have to be sent now (a copy from pageable memory, and whose slot
+  // could be reused later) is not taken: the chunks go out one by one, their maps as parameters.
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(s, &cap) != cudaSuccess) {
+    (void)cudaGetLastError();
+    cap = cudaStreamCaptureStatusNone;
+  }
+  const bool capturing = cap != cudaStreamCaptureStatusNone;
   if (slot < 0) {
-    slot = 0;
-    for (int i = 1; i < kHistSlots; ++i)
-      if (c->hist_age[i] < c->hist_age[slot]) slot = i;
+    if (capturing) return SS_OK;
+    for (int i = 0; i < kHistSlots; ++i)
+      if (!c->hist_pinned[i] && (slot < 0 || c->hist_age[i] < c->hist_age[slot])) slot = i;
+    if (slot < 0) return SS_OK;  // every list belongs to a captured launch
     memcpy(c->hist_host[slot], maps, (size_t)2 * n_chunks * sizeof(CUtensorMap));
     c->hist_n[slot] = 0;  // (not valid until the copy has been enqueued)
     // stream order: the copy runs after every kernel already enqueued, which may still read the list
@@ -895,6 +907,7 @@ static ss_status hist_chunks(ss_ctx* c, const ss_chunk_desc* chunks, int n_chunk
     if (e != cudaSuccess) return cuda_fail(c, e);
     c->hist_n[slot] = 2 * n_chunks;
   }
+  if (capturing) c->hist_pinned[slot] = true;
   c->hist_age[slot] = ++c->tm_clock;
 
   ss::ChunkParams p;

@@ -695,6 +695,32 @@ def test_chunk_list_round_can_be_captured_in_a_cuda_graph(lens):
     one_round()
     torch.cuda.synchronize()
     assert torch.equal(O.view(torch.int16), O_g.view(torch.int16)) and torch.equal(LSE, L_g)
+    O_ref, L_ref = O.clone(), LSE.clone()
+    # The launch reads its chunks' tensor maps from a list in the workspace, of which there are four:
+    # a list a capture used stays, however many other lists the context sees afterwards
+    O2, L2 = torch.empty_like(O), torch.empty_like(LSE)
+    keep = []   # (alive, so that no later buffer takes an address a list already holds)
+    for k in range(6):
+        other = [(K.clone(), V.clone(), vl) for (K, V, vl) in chunks]
+        keep.append(other)
+        ctx.ss_verify_round(Q, cfg.scale, other, K_loc, V_loc, ssb.SS_MASK_CHAIN, None, O2, L2, hints=hints)
+        torch.cuda.synchronize()
+        assert ctx.last_chunk_kernel() == "tcgen05-keys-round"
+        assert torch.equal(O2.view(torch.int16), O_ref.view(torch.int16))
+    O.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(O.view(torch.int16), O_ref.view(torch.int16)) and torch.equal(LSE, L_ref)
+    # a list first seen inside a capture is not sent from there: the chunks go out one by one
+    fresh = [(K.clone(), V.clone(), vl) for (K, V, vl) in chunks]
+    fresh_descs = ctx.chunk_descs([fresh], hints)
+    g2 = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g2):
+        ctx.ss_verify_round(Q, cfg.scale, fresh, K_loc, V_loc, ssb.SS_MASK_CHAIN, None, O2, L2, descs=fresh_descs)
+    assert ctx.last_chunk_kernel() == "tcgen05-keys"
+    g2.replay()
+    torch.cuda.synchronize()
+    util.compare(cfg, O2, L2, util.oracle_case(cfg, lens, Q, chunks, K_loc, V_loc, bits))
     ctx.close()
 
 
